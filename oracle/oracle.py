@@ -1,0 +1,225 @@
+"""ctypes front end of the C oracle (``rubick_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  Builds ``liboracle.so`` beside the source with gcc on first use
+and marshals numpy arrays into the oracle's own plain layouts (jobs as rows of doubles,
+plans as rows of six int32, environment as a row of doubles).  Nothing here touches the
+CUDA library.
+"""
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "rubick_oracle.c")
+_SO = os.path.join(_HERE, "liboracle.so")
+
+JOB_FIELDS = ["P", "l", "h", "s", "b", "mu_cap", "alpha_act", "tau", "k_bwd", "k_sync", "k_opt",
+              "k_opt_off", "k_off", "k_swap", "k_const", "w", "gmin_idx", "cmin_idx", "host_base_bytes"]
+ENV_FIELDS = ["B_intra", "B_inter", "B_pcie", "gpu_mem_bytes", "gpus_per_node", "cpus_per_node",
+              "mem_per_node_bytes", "bytes_per_elem", "strict_zero_dp_only"]
+TERM_FIELDS = ["valid", "mu", "m", "a", "T_fwd", "T_bwd", "V_dp", "V_tp", "V_pp", "T_dp", "T_tp",
+               "T_pp", "T_cc", "T_opt", "T_off", "T_oo", "T_iter", "thr"]
+MEM_FIELDS = ["params", "grads", "opt", "act", "gpu_total", "gpu_ok", "host_need", "nodes"]
+
+_lib = None
+
+
+def build(force=False):
+    """Compile the oracle with gcc (-O2, no fast-math, no FMA contraction, OpenMP over jobs)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c99", "-fopenmp", "-ffp-contract=off", "-fno-fast-math",
+               "-shared", "-fPIC", "-o", _SO, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+def _p(a, t):
+    return a.ctypes.data_as(C.POINTER(t))
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        build()
+        L = C.CDLL(_SO)
+        L.oracle_overlap.restype = C.c_double
+        L.oracle_overlap.argtypes = [C.c_double, C.c_double, C.c_double]
+        L.oracle_bruteforce.restype = C.c_double
+        L.oracle_feas_word.restype = C.c_uint32
+        L.oracle_enumerate_plans.restype = C.c_int
+        L.oracle_round.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def job_rows(jobs):
+    """dict of per-job arrays (keys = JOB_FIELDS) -> [J, len(JOB_FIELDS)] float64 rows."""
+    J = len(np.atleast_1d(jobs["P"]))
+    rows = np.zeros((J, len(JOB_FIELDS)), dtype=np.float64)
+    for i, k in enumerate(JOB_FIELDS):
+        rows[:, i] = np.asarray(jobs[k], dtype=np.float64)
+    return rows
+
+
+def env_row(env):
+    return _f64([float(env.get(k, 0.0)) for k in ENV_FIELDS])
+
+
+def overlap(k, x, y):
+    return lib().oracle_overlap(float(k), float(x), float(y))
+
+
+def terms(jobs, j, env, plan, c):
+    """All model terms (TERM_FIELDS) of job j under plan = (d, t, p, z, gc, off) with c cores."""
+    rows = job_rows(jobs)
+    out = np.zeros(len(TERM_FIELDS))
+    pl = _i32(plan)
+    lib().oracle_terms(_p(rows[j], C.c_double), _p(env_row(env), C.c_double), _p(pl, C.c_int32),
+                       C.c_double(float(c)), _p(out, C.c_double))
+    return dict(zip(TERM_FIELDS, out.tolist()))
+
+
+def memory(jobs, j, env, plan):
+    rows = job_rows(jobs)
+    out = np.zeros(len(MEM_FIELDS), dtype=np.int64)
+    pl = _i32(plan)
+    lib().oracle_memory(_p(rows[j], C.c_double), _p(env_row(env), C.c_double), _p(pl, C.c_int32),
+                        _p(out, C.c_int64))
+    return dict(zip(MEM_FIELDS, out.tolist()))
+
+
+def feas_word(jobs, j, env, plan, m_levels):
+    rows = job_rows(jobs)
+    ml = _i64(m_levels)
+    return int(lib().oracle_feas_word(_p(rows[j], C.c_double), _p(env_row(env), C.c_double),
+                                      _p(_i32(plan), C.c_int32), _p(ml, C.c_int64), C.c_int(len(ml))))
+
+
+def enumerate_plans(g_levels):
+    """-> (plans [P, 6] int32 = d, t, p, z, gc, off; group_off [nG + 1] int32)."""
+    gl = _i64(g_levels)
+    off = np.zeros(len(gl) + 1, dtype=np.int32)
+    dummy = np.zeros((1, 6), dtype=np.int32)
+    n = lib().oracle_enumerate_plans(_p(gl, C.c_int64), C.c_int(len(gl)), _p(dummy, C.c_int32), C.c_int(0),
+                                     _p(off, C.c_int32))
+    plans = np.zeros((max(n, 1), 6), dtype=np.int32)
+    lib().oracle_enumerate_plans(_p(gl, C.c_int64), C.c_int(len(gl)), _p(plans, C.c_int32), C.c_int(n),
+                                 _p(off, C.c_int32))
+    return plans[:n], off
+
+
+def eval_candidates(jobs, plans, env, c_levels, m_levels, nthreads=1):
+    """-> (thr [J, C, P] float64, feas [J, P] uint32)."""
+    rows = job_rows(jobs)
+    J = rows.shape[0]
+    plans = _i32(plans)
+    Pn = plans.shape[0]
+    cl, ml = _i64(c_levels), _i64(m_levels)
+    thr = np.zeros((J, len(cl), Pn), dtype=np.float64)
+    feas = np.zeros((J, Pn), dtype=np.uint32)
+    lib().oracle_eval(_p(rows, C.c_double), C.c_int(J), _p(plans, C.c_int32), C.c_int(Pn),
+                      _p(env_row(env), C.c_double), _p(cl, C.c_int64), C.c_int(len(cl)),
+                      _p(ml, C.c_int64), C.c_int(len(ml)), _p(thr, C.c_double), _p(feas, C.c_uint32),
+                      C.c_int(nthreads))
+    return thr, feas
+
+
+def best_plan(thr, feas, plans, g_levels, nM, prefix=True, nthreads=1):
+    """thr [J, C, P] (any float dtype; compared in float64), feas [J, P] ->
+    (best_val [J, G, C, M] float64, best_plan int32, best_g int32)."""
+    thr = _f64(thr)
+    feas = np.ascontiguousarray(feas, dtype=np.uint32)
+    J, nC, Pn = thr.shape
+    plans = _i32(plans)
+    gl = _i64(g_levels)
+    nG = len(gl)
+    bv = np.zeros((J, nG, nC, nM), dtype=np.float64)
+    bp = np.zeros((J, nG, nC, nM), dtype=np.int32)
+    bg = np.zeros((J, nG, nC, nM), dtype=np.int32)
+    lib().oracle_best_plan(_p(thr, C.c_double), _p(feas, C.c_uint32), C.c_int(J), _p(plans, C.c_int32),
+                           C.c_int(Pn), _p(gl, C.c_int64), C.c_int(nG), C.c_int(nC), C.c_int(nM),
+                           C.c_int(1 if prefix else 0), _p(bv, C.c_double), _p(bp, C.c_int32),
+                           _p(bg, C.c_int32), C.c_int(nthreads))
+    return bv, bp, bg
+
+
+def gain(jobs, curve_val, g_levels, c_levels, state_g, state_c, state_val):
+    """Marginal gains for a given per-job state -> (gain_gpu, gain_cpu, next_g, next_c)."""
+    rows = job_rows(jobs)
+    J = rows.shape[0]
+    cv = np.ascontiguousarray(curve_val, dtype=np.float32)
+    gl, cl = _i64(g_levels), _i64(c_levels)
+    nM = cv.shape[3]
+    sg, sc = _i64(state_g), _i64(state_c)
+    sv = np.ascontiguousarray(state_val, dtype=np.float32)
+    gg = np.zeros(J, dtype=np.float32)
+    gc = np.zeros(J, dtype=np.float32)
+    ng = np.zeros(J, dtype=np.int32)
+    nc = np.zeros(J, dtype=np.int32)
+    lib().oracle_gain(_p(rows, C.c_double), C.c_int(J), _p(cv, C.c_float), _p(gl, C.c_int64), C.c_int(len(gl)),
+                      _p(cl, C.c_int64), C.c_int(len(cl)), C.c_int(nM), _p(sg, C.c_int64), _p(sc, C.c_int64),
+                      _p(sv, C.c_float), _p(gg, C.c_float), _p(gc, C.c_float), _p(ng, C.c_int32),
+                      _p(nc, C.c_int32))
+    return gg, gc, ng, nc
+
+
+def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,
+                   n_nodes, max_steps=1 << 30, want_log=False):
+    """One greedy round on single-precision curve tables.
+
+    -> dict(g, c, m_bytes, plan, first_node, n_nodes, status, m_level, thr, node (N x 4:
+    free g, free c, free m, owner), steps, capped, log)."""
+    rows = job_rows(jobs)
+    J = rows.shape[0]
+    cv = np.ascontiguousarray(curve_val, dtype=np.float32)
+    cp, cg = _i32(curve_plan), _i32(curve_g)
+    feas = np.ascontiguousarray(feas, dtype=np.uint32)
+    Pn = feas.shape[1] if feas.ndim == 2 else 0
+    gl, cl, ml = _i64(g_levels), _i64(c_levels), _i64(m_levels)
+    out_i = np.zeros((max(J, 1), 8), dtype=np.int64)
+    out_v = np.zeros(max(J, 1), dtype=np.float32)
+    node = np.zeros((n_nodes, 4), dtype=np.int64)
+    cap = int(min(max_steps, J * (len(gl) + len(cl) + 2) + 1))
+    log = np.zeros(max(cap, 1), dtype=np.int32)
+    r = lib().oracle_round(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double), _p(cv, C.c_float),
+                           _p(cp, C.c_int32), _p(cg, C.c_int32), _p(feas, C.c_uint32), C.c_int(Pn),
+                           _p(gl, C.c_int64), C.c_int(len(gl)), _p(cl, C.c_int64), C.c_int(len(cl)),
+                           _p(ml, C.c_int64), C.c_int(len(ml)), C.c_int(n_nodes), C.c_int(cap),
+                           _p(out_i, C.c_int64), _p(out_v, C.c_float), _p(node, C.c_int64),
+                           _p(log, C.c_int32) if want_log else None)
+    capped = r < 0
+    steps = -r - 1 if capped else r
+    out_i = out_i[:J]
+    return dict(g=out_i[:, 0].copy(), c=out_i[:, 1].copy(), m_bytes=out_i[:, 2].copy(),
+                plan=out_i[:, 3].copy(), first_node=out_i[:, 4].copy(), n_nodes=out_i[:, 5].copy(),
+                status=out_i[:, 6].copy(), m_level=out_i[:, 7].copy(), thr=out_v[:J].copy(), node=node,
+                steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
+
+
+def bruteforce(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels):
+    """Best total weighted throughput over all single-node assignments (tiny instances)."""
+    rows = job_rows(jobs)
+    J = rows.shape[0]
+    cv = np.ascontiguousarray(curve_val, dtype=np.float32)
+    cp, cg = _i32(curve_plan), _i32(curve_g)
+    feas = np.ascontiguousarray(feas, dtype=np.uint32)
+    gl, cl, ml = _i64(g_levels), _i64(c_levels), _i64(m_levels)
+    return float(lib().oracle_bruteforce(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double),
+                                         _p(cv, C.c_float), _p(cp, C.c_int32), _p(cg, C.c_int32),
+                                         _p(feas, C.c_uint32), C.c_int(feas.shape[1]), _p(gl, C.c_int64),
+                                         C.c_int(len(gl)), _p(cl, C.c_int64), C.c_int(len(cl)),
+                                         _p(ml, C.c_int64), C.c_int(len(ml))))

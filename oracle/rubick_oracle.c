@@ -1,0 +1,704 @@
+/*
+ * Rubick oracle -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, double-precision CPU statement of what the scheduler's data-parallel
+ * path computes: the training-performance model (paper Section 4), the plan space and
+ * the best-plan / resource-sensitivity-curve step (Section 5.2), the marginal-gain
+ * ("slope") score and one greedy scheduling round (Section 5.2, Algorithm 1, in the
+ * grow-only marginal-gain form), plus an exhaustive search used on tiny instances.
+ *
+ * Only the test-suite, the smoke check and the CPU-baseline leg of the benchmark may
+ * build or call this file.  It shares nothing with the CUDA library: no header, no
+ * table, no helper.  Inputs arrive as plain arrays of doubles / 64-bit integers, in a
+ * layout of its own.
+ *
+ * Every function is written as the definition it follows, one loop nest per definition,
+ * with no blocking, hoisting or caching.
+ *
+ * Pinning status (see tests/test_oracle_*.py):
+ *   - overlap function, communication volumes, pipeline bubble, T_cc, T_opt, T_oo, Eq. 1:
+ *     pinned (limits k=1 / k->inf, ring and pipeline simulations, paper-literal special
+ *     cases coded separately, homogeneity, monotonicity).
+ *   - plan enumeration, best plan, sensitivity curve: pinned (counts, brute force).
+ *   - memory-feasibility rule: the paper prints no formula (it defers to the training
+ *     frameworks' estimators), so the rule here is this project's reading; it is pinned
+ *     only by the three qualitative facts the paper states (Section 2.2, Section 7.2) and
+ *     by an independent big-integer recomputation:  "parity unpinned by the paper".
+ *   - greedy round: Algorithm 1 is a heuristic with unspecified step sizes; the step list
+ *     implemented here is this project's reading; pinned by the exhaustive search
+ *     (upper bound, equality on concave single-resource instances) and capacity
+ *     invariants, otherwise "parity unpinned by the paper".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ---- input layouts (the oracle's own) ------------------------------------------------ */
+
+/* one job = JF_COUNT doubles (integers are stored exactly; all are < 2^53) */
+enum {
+    JF_P = 0,      /* parameter count (Table 1: P)                       */
+    JF_L,          /* layers l                                           */
+    JF_H,          /* hidden size h                                      */
+    JF_S,          /* sequence length s                                  */
+    JF_B,          /* global batch b                                     */
+    JF_MUCAP,      /* largest micro-batch one replica may run at once    */
+    JF_ALPHA,      /* activation bytes per (token x hidden) per layer    */
+    JF_TAU,        /* forward seconds per sample, whole model on one GPU */
+    JF_KBWD, JF_KSYNC, JF_KOPT, JF_KOPTOFF, JF_KOFF, JF_KSWAP, JF_KCONST, /* Table 1 fittables */
+    JF_W,          /* throughput weight of the job                       */
+    JF_GMIN,       /* guaranteed minimum GPU level index, -1 = best effort */
+    JF_CMIN,       /* guaranteed minimum CPU level index, -1 = none        */
+    JF_HOSTBASE,   /* host bytes per training process (one per GPU)      */
+    JF_COUNT
+};
+
+/* environment = EF_COUNT doubles */
+enum {
+    EF_BINTRA = 0, EF_BINTER, EF_BPCIE, /* bytes / second (Table 1 environment row) */
+    EF_GPUMEM,                          /* bytes of memory on one GPU               */
+    EF_GN, EF_CN, EF_MN,                /* GPUs, CPU cores, host bytes per node     */
+    EF_E,                               /* bytes per element (2 = fp16)             */
+    EF_STRICT,                          /* 1: ZeRO / offload only with t = p = 1    */
+    EF_COUNT
+};
+
+/* one plan = 6 int32: d, t, p (degrees themselves), ZeRO stage z, gc, off */
+enum { PF_D = 0, PF_T, PF_P, PF_Z, PF_GC, PF_OFF, PF_COUNT };
+
+/* terms returned by oracle_terms (for unit tests of the individual formulas) */
+enum {
+    TF_VALID = 0, TF_MU, TF_M, TF_A,
+    TF_TFWD, TF_TBWD,
+    TF_VDP, TF_VTP, TF_VPP,
+    TF_TDP, TF_TTP, TF_TPP,
+    TF_TCC, TF_TOPT, TF_TOFF, TF_TOO, TF_TITER, TF_THR,
+    TF_COUNT
+};
+
+/* memory terms returned by oracle_memory */
+enum {
+    MF_PARAMS = 0, MF_GRADS, MF_OPT, MF_ACT, MF_GPU_TOTAL, MF_GPU_OK, MF_HOST_NEED, MF_NODES,
+    MF_COUNT
+};
+
+/* per-job result of a scheduling round = AF_COUNT int64 + value */
+enum { ST_UNALLOCATED = 0, ST_RUNNING = 1, ST_PENDING = 2 };
+
+static int64_t cdiv(int64_t a, int64_t b) { return (a + b - 1) / b; }
+static int64_t imin(int64_t a, int64_t b) { return a < b ? a : b; }
+
+/* ---- Section 4.3, "Modeling overlapping": f^k(x, y) = (x^k + y^k)^(1/k) ------------ */
+double oracle_overlap(double k, double x, double y)
+{
+    if (x == 0.0) return y;      /* a zero stage adds nothing (V = 0 rule, Section 4.1) */
+    if (y == 0.0) return x;
+    return pow(pow(x, k) + pow(y, k), 1.0 / k);
+}
+
+/* ---- structural validity of a plan for a job ---------------------------------------- */
+static int plan_valid(const double *job, const double *env, const int32_t *pl)
+{
+    int64_t d = pl[PF_D], t = pl[PF_T], p = pl[PF_P];
+    int64_t z = pl[PF_Z], off = pl[PF_OFF];
+    int64_t b = (int64_t)job[JF_B], l = (int64_t)job[JF_L], h = (int64_t)job[JF_H];
+    int64_t Gn = (int64_t)env[EF_GN];
+    if (t > Gn) return 0;                 /* TP stays inside a node (Section 4.1)      */
+    if (p > l) return 0;                  /* every stage holds at least one layer      */
+    if (d > b || b % d != 0) return 0;    /* at least one whole sample per replica     */
+    if (off && z < 2) return 0;           /* offload moves partitioned gradients       */
+    if (h % t != 0) return 0;             /* the hidden dimension splits evenly        */
+    if (env[EF_STRICT] != 0.0 && (z > 0 || off) && (t > 1 || p > 1)) return 0;
+    return 1;
+}
+
+/* micro-batching: per-replica batch r = b/d, micro-batch mu = min(r, mu_cap),
+ * n = ceil(r / mu) passes.  With pipelining they are the m micro-batches in flight,
+ * without it they are the a gradient-accumulation steps (Table 1: m, a). */
+static void micro_batching(const double *job, const int32_t *pl, int64_t *mu, int64_t *m, int64_t *a)
+{
+    int64_t b = (int64_t)job[JF_B], d = pl[PF_D], p = pl[PF_P];
+    int64_t r = b / d;
+    *mu = imin(r, (int64_t)job[JF_MUCAP]);
+    int64_t n = cdiv(r, *mu);
+    if (p > 1) { *m = n; *a = 1; } else { *m = 1; *a = n; }
+}
+
+/* ---- Section 4: all terms of the performance model for (job, plan, c CPU cores) ----- */
+void oracle_terms(const double *job, const double *env, const int32_t *pl, double c, double *out)
+{
+    for (int i = 0; i < TF_COUNT; ++i) out[i] = 0.0;
+    if (!plan_valid(job, env, pl)) return;
+    out[TF_VALID] = 1.0;
+
+    double d = pl[PF_D], t = pl[PF_T], p = pl[PF_P];
+    int z = pl[PF_Z], gc = pl[PF_GC], off = pl[PF_OFF];
+    double g = d * t * p;
+    double P = job[JF_P], l = job[JF_L], h = job[JF_H], s = job[JF_S], b = job[JF_B];
+    double e = env[EF_E], Gn = env[EF_GN];
+
+    int64_t mu_i, m_i, a_i;
+    micro_batching(job, pl, &mu_i, &m_i, &a_i);
+    double mu = (double)mu_i, m = (double)m_i, a = (double)a_i;
+    out[TF_MU] = mu; out[TF_M] = m; out[TF_A] = a;
+
+    /* T_fwd (Section 4.1): forward time of one pass, scaled linearly to the micro-batch
+     * and the tensor shard; with pipelining, p stages each holding 1/p of the layers run
+     * m + p - 1 slots. */
+    double T_fwd = job[JF_TAU] * mu / (t * p);
+    if (p > 1) T_fwd *= (m + p - 1.0);
+    /* T_bwd = k_bwd * T_fwd, plus one recomputing forward under gradient checkpointing */
+    double T_bwd = job[JF_KBWD] * T_fwd + (gc ? T_fwd : 0.0);
+
+    /* volumes in bytes; a degree of 1 sends nothing */
+    double V_dp = 0.0, V_tp = 0.0, V_pp = 0.0;
+    if (d > 1) V_dp = e * P * 2.0 * (d - 1.0) / (d * t * p) * (z == 3 ? 1.5 : 1.0);
+    if (t > 1) V_tp = e * 4.0 * 2.0 * (t - 1.0) * b * s * h * l / (d * t);
+    if (p > 1) V_pp = e * 2.0 * p * b * s * h / (d * t);
+
+    /* bottleneck bandwidth of each group under the packed placement: ranks are laid out
+     * TP fastest, then DP, then PP; g <= Gn sits on one node, larger jobs on whole nodes */
+    double B_tp = env[EF_BINTRA];
+    double B_dp = (d * t <= Gn) ? env[EF_BINTRA] : env[EF_BINTER];
+    double B_pp = (g <= Gn) ? env[EF_BINTRA] : env[EF_BINTER];
+    double T_dp = V_dp / B_dp, T_tp = V_tp / B_tp, T_pp = V_pp / B_pp;
+
+    /* T_cc: a forwards, a-1 plain backwards, the last backward overlapped with the
+     * gradient synchronisation, TP / PP traffic on the critical path */
+    double T_cc = a * T_fwd + (a - 1.0) * T_bwd
+                + oracle_overlap(job[JF_KSYNC], T_bwd, T_dp) + T_tp + T_pp;
+
+    /* optimizer and offloading (Section 4.2) */
+    double Psi = P / (t * p);                  /* parameters of one model-parallel shard */
+    double T_opt, T_off = 0.0, T_oo;
+    if (off) {
+        T_opt = job[JF_KOPTOFF] * Psi / (d * c);
+        T_off = e * Psi / (d * env[EF_BPCIE]);
+        T_oo = oracle_overlap(job[JF_KOFF], T_dp, T_off)
+             + oracle_overlap(job[JF_KSWAP], T_opt, T_off);
+    } else {
+        T_opt = job[JF_KOPT] * Psi / (z >= 1 ? d : 1.0);
+        T_oo = T_opt;
+    }
+    double T_iter = T_cc + T_oo + job[JF_KCONST];      /* Eq. 1 */
+
+    out[TF_TFWD] = T_fwd; out[TF_TBWD] = T_bwd;
+    out[TF_VDP] = V_dp; out[TF_VTP] = V_tp; out[TF_VPP] = V_pp;
+    out[TF_TDP] = T_dp; out[TF_TTP] = T_tp; out[TF_TPP] = T_pp;
+    out[TF_TCC] = T_cc; out[TF_TOPT] = T_opt; out[TF_TOFF] = T_off; out[TF_TOO] = T_oo;
+    out[TF_TITER] = T_iter;
+    out[TF_THR] = b / T_iter;                           /* THROUGHPUT = b / T_iter */
+}
+
+/* ---- memory-feasibility rule (integer bytes) ----------------------------------------- */
+void oracle_memory(const double *job, const double *env, const int32_t *pl, int64_t *out)
+{
+    for (int i = 0; i < MF_COUNT; ++i) out[i] = 0;
+    int64_t d = pl[PF_D], t = pl[PF_T], p = pl[PF_P];
+    int64_t z = pl[PF_Z], gc = pl[PF_GC], off = pl[PF_OFF];
+    int64_t g = d * t * p;
+    int64_t Pi = (int64_t)job[JF_P];
+    int64_t l = (int64_t)job[JF_L], h = (int64_t)job[JF_H], s = (int64_t)job[JF_S];
+    int64_t alpha = (int64_t)job[JF_ALPHA];
+    int64_t Gn = (int64_t)env[EF_GN];
+    int64_t mu, m, a;
+    if (!plan_valid(job, env, pl)) return;
+    micro_batching(job, pl, &mu, &m, &a);
+
+    /* model states, mixed-precision Adam: 2 + 2 + 12 bytes per parameter of the shard,
+     * ZeRO stage 1 / 2 / 3 spreading optimizer / + gradients / + parameters over d */
+    int64_t Psi = cdiv(Pi, t * p);
+    int64_t dz1 = z >= 1 ? d : 1, dz2 = z >= 2 ? d : 1, dz3 = z == 3 ? d : 1;
+    int64_t params = 2 * cdiv(Psi, dz3);
+    int64_t grads = off ? 0 : 2 * cdiv(Psi, dz2);
+    int64_t opt = off ? 0 : 12 * cdiv(Psi, dz1);
+
+    /* activations of the layers on one GPU for the micro-batches in flight */
+    int64_t A = cdiv(alpha * s * mu * h, t);
+    int64_t q = p > 1 ? imin(m, p) : 1;
+    int64_t L = cdiv(l, p);
+    int64_t act = gc ? L * q * 2 * s * mu * h + A : L * q * A;
+
+    int64_t total = params + grads + opt + act;
+    out[MF_PARAMS] = params; out[MF_GRADS] = grads; out[MF_OPT] = opt; out[MF_ACT] = act;
+    out[MF_GPU_TOTAL] = total;
+    out[MF_GPU_OK] = total <= (int64_t)env[EF_GPUMEM];
+    /* host memory: one process per GPU, plus fp32 master weights, momentum, variance and
+     * fp16 gradients (4 + 4 + 4 + 2 bytes per parameter) when the optimizer runs on CPUs */
+    out[MF_HOST_NEED] = g * (int64_t)job[JF_HOSTBASE] + (off ? 14 * Pi : 0);
+    out[MF_NODES] = g <= Gn ? 1 : g / Gn;
+}
+
+/* feasibility word: bit i set <=> the plan may run with host-memory level i */
+uint32_t oracle_feas_word(const double *job, const double *env, const int32_t *pl,
+                          const int64_t *m_levels, int nM)
+{
+    int64_t mem[MF_COUNT];
+    if (!plan_valid(job, env, pl)) return 0u;
+    oracle_memory(job, env, pl, mem);
+    if (!mem[MF_GPU_OK]) return 0u;
+    uint32_t word = 0u;
+    for (int i = 0; i < nM; ++i) {
+        int ok = mem[MF_HOST_NEED] <= m_levels[i]
+              && cdiv(mem[MF_HOST_NEED], mem[MF_NODES]) <= (int64_t)env[EF_MN];
+        if (ok) word |= (1u << i);
+    }
+    return word;
+}
+
+/* ---- plan enumeration (Section 3 plan families; canonical order) --------------------- */
+static int is_pow2(int64_t x) { return x > 0 && (x & (x - 1)) == 0; }
+
+/* For every GPU level g that is a power of two: all (d, t, p) with d*t*p = g, TP degree
+ * ascending, then PP degree ascending, then ZeRO stage, gradient checkpointing, offload.
+ * group_off[i] .. group_off[i+1] is the index range of level i.  Returns the plan count
+ * (also when it exceeds cap; nothing beyond cap is written). */
+int oracle_enumerate_plans(const int64_t *g_levels, int nG, int32_t *plans, int cap, int32_t *group_off)
+{
+    int n = 0;
+    for (int gi = 0; gi < nG; ++gi) {
+        group_off[gi] = n;
+        int64_t g = g_levels[gi];
+        if (!is_pow2(g)) continue;
+        for (int64_t t = 1; t <= g; t *= 2)
+            for (int64_t p = 1; t * p <= g; p *= 2) {
+                int64_t d = g / (t * p);
+                for (int z = 0; z < 4; ++z)
+                    for (int gc = 0; gc < 2; ++gc)
+                        for (int off = 0; off < 2; ++off) {
+                            if (n < cap) {
+                                int32_t *pl = plans + (size_t)n * PF_COUNT;
+                                pl[PF_D] = (int32_t)d; pl[PF_T] = (int32_t)t; pl[PF_P] = (int32_t)p;
+                                pl[PF_Z] = z; pl[PF_GC] = gc; pl[PF_OFF] = off;
+                            }
+                            ++n;
+                        }
+            }
+    }
+    group_off[nG] = n;
+    return n;
+}
+
+/* ---- candidate table: thr[J][C][P] and feas[J][P] ------------------------------------ */
+void oracle_eval(const double *jobs, int J, const int32_t *plans, int P, const double *env,
+                 const int64_t *c_levels, int nC, const int64_t *m_levels, int nM,
+                 double *thr, uint32_t *feas, int nthreads)
+{
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+#pragma omp parallel for schedule(static)
+#endif
+    for (int j = 0; j < J; ++j) {
+        const double *job = jobs + (size_t)j * JF_COUNT;
+        double terms[TF_COUNT];
+        for (int pi = 0; pi < P; ++pi) {
+            const int32_t *pl = plans + (size_t)pi * PF_COUNT;
+            for (int ci = 0; ci < nC; ++ci) {
+                oracle_terms(job, env, pl, (double)c_levels[ci], terms);
+                thr[((size_t)j * nC + ci) * P + pi] = terms[TF_VALID] != 0.0 ? terms[TF_THR] : 0.0;
+            }
+            feas[(size_t)j * P + pi] = oracle_feas_word(job, env, pl, m_levels, nM);
+        }
+    }
+    (void)nthreads;
+}
+
+/* ---- best plan per (job, g level, c level, m level), then the sensitivity curve ------
+ * best = the largest predicted throughput among plans using exactly g GPUs that are
+ * feasible at host-memory level mi; the lowest plan index wins a tie; (0, -1, 0) if there
+ * is none (invalid GPU counts have zero throughput, Fig. 6).  With prefix != 0 the result
+ * is the running maximum along g (the curve stays flat over GPU counts that do not
+ * improve, Section 5.2), carrying the plan and the GPU count of the earliest maximum. */
+void oracle_best_plan(const double *thr, const uint32_t *feas, int J, const int32_t *plans, int P,
+                      const int64_t *g_levels, int nG, int nC, int nM, int prefix,
+                      double *best_val, int32_t *best_plan, int32_t *best_g, int nthreads)
+{
+#ifdef _OPENMP
+    if (nthreads > 0) omp_set_num_threads(nthreads);
+#pragma omp parallel for schedule(static)
+#endif
+    for (int j = 0; j < J; ++j)
+        for (int ci = 0; ci < nC; ++ci)
+            for (int mi = 0; mi < nM; ++mi) {
+                double run_val = 0.0; int32_t run_plan = -1, run_g = 0;
+                for (int gi = 0; gi < nG; ++gi) {
+                    double bv = 0.0; int32_t bp = -1;
+                    for (int pi = 0; pi < P; ++pi) {
+                        const int32_t *pl = plans + (size_t)pi * PF_COUNT;
+                        int64_t g = (int64_t)pl[PF_D] * pl[PF_T] * pl[PF_P];
+                        if (g != g_levels[gi]) continue;
+                        if (!((feas[(size_t)j * P + pi] >> mi) & 1u)) continue;
+                        double v = thr[((size_t)j * nC + ci) * P + pi];
+                        if (v > bv) { bv = v; bp = pi; }
+                    }
+                    int32_t bg = bp >= 0 ? (int32_t)g_levels[gi] : 0;
+                    if (prefix) {
+                        if (bv > run_val) { run_val = bv; run_plan = bp; run_g = bg; }
+                        bv = run_val; bp = run_plan; bg = run_g;
+                    }
+                    size_t o = (((size_t)j * nG + gi) * nC + ci) * nM + mi;
+                    best_val[o] = bv; best_plan[o] = bp; best_g[o] = bg;
+                }
+            }
+    (void)nthreads;
+}
+
+/* ======================================================================================
+ * Scheduling: marginal gains and one greedy round.
+ *
+ * All decisions are taken in single precision on the single-precision curve table, with
+ * one rounding per operation in the order written (compile with -ffp-contract=off), so
+ * that a second implementation can reproduce every comparison bit for bit.
+ * ==================================================================================== */
+
+typedef struct {
+    int J, nG, nC, nM, P, N;
+    const float *cv;          /* curve value   [J][G][C][M] */
+    const int32_t *cp;        /* curve plan    [J][G][C][M] */
+    const int32_t *cg;        /* curve g used  [J][G][C][M] */
+    const uint32_t *feas;     /* [J][P] */
+    const double *jobs;
+    const int64_t *g_levels, *c_levels, *m_levels;
+    int64_t Gn, Cn, Mn;
+    /* cluster state */
+    int64_t *free_g, *free_c, *free_m;
+    int32_t *owner;           /* job holding the whole node as part of a multi-node set, or -1 */
+} Sched;
+
+typedef struct {
+    int gi, ci;               /* level indices, gi = -1 when unallocated */
+    int64_t g, c, m;          /* amounts held (m in bytes)               */
+    int plan, node, k;        /* plan index, first node, node count      */
+    float val;                /* predicted throughput of the allocation  */
+    int status;
+    int frozen[2];            /* a rejected GPU / CPU increment is not retried this round */
+} JobState;
+
+typedef struct { int ok; int k; int stay; int node; int need_new; } Place;
+
+static size_t cidx(const Sched *S, int j, int gi, int ci, int mi)
+{
+    return (((size_t)j * S->nG + gi) * S->nC + ci) * S->nM + mi;
+}
+
+static int count_empty(const Sched *S)
+{
+    int n = 0;
+    for (int i = 0; i < S->N; ++i) n += (S->free_g[i] == S->Gn);
+    return n;
+}
+
+/* Where would job js run with g2 GPUs and c2 cores?  One node if g2 <= Gn: its present
+ * node when the increment fits there, else the first node (index order) with room for the
+ * whole job.  Otherwise g2 / Gn whole nodes: those it already holds entirely plus the
+ * lowest-numbered empty ones, with ceil(c2 / k) cores on each. */
+static Place find_place(const Sched *S, const JobState *js, int64_t g2, int64_t c2)
+{
+    Place pl; pl.ok = 0; pl.k = 1; pl.stay = 0; pl.node = -1; pl.need_new = 0;
+    int allocated = js->gi >= 0;
+    if (g2 <= S->Gn) {
+        if (allocated && js->k == 1
+            && S->free_g[js->node] >= g2 - js->g && S->free_c[js->node] >= c2 - js->c) {
+            pl.ok = 1; pl.stay = 1; pl.node = js->node; return pl;
+        }
+        for (int n = 0; n < S->N; ++n)
+            if (S->free_g[n] >= g2 && S->free_c[n] >= c2) { pl.ok = 1; pl.node = n; return pl; }
+        return pl;
+    }
+    if (g2 % S->Gn != 0) return pl;
+    int k2 = (int)(g2 / S->Gn);
+    pl.k = k2;
+    if (cdiv(c2, k2) > S->Cn) return pl;
+    int empty = count_empty(S);
+    if (allocated && js->g >= S->Gn) {            /* holds whole nodes already */
+        if (k2 == js->k) { pl.ok = 1; pl.stay = 1; pl.node = js->node; return pl; }
+        pl.need_new = k2 - js->k;
+        pl.stay = 1;
+    } else {
+        pl.need_new = k2;
+        if (allocated && S->free_g[js->node] + js->g == S->Gn) empty += 1; /* its node empties */
+    }
+    pl.ok = empty >= pl.need_new;
+    return pl;
+}
+
+static void release_job(Sched *S, int j, JobState *js)
+{
+    if (js->gi < 0) return;
+    if (js->k == 1) {
+        S->free_g[js->node] += js->g; S->free_c[js->node] += js->c; S->free_m[js->node] += js->m;
+    } else {
+        for (int n = 0; n < S->N; ++n)
+            if (S->owner[n] == j) {
+                S->free_g[n] += S->Gn; S->free_c[n] += cdiv(js->c, js->k); S->free_m[n] += cdiv(js->m, js->k);
+                S->owner[n] = -1;
+            }
+    }
+}
+
+/* Commit job j to (gi2, ci2) at placement pl: pick the host-memory level that fits the
+ * target node(s), read the curve there (GetBestPlan), allocate that plan's memory
+ * (AllocMem).  Returns 1 on success; 0 leaves everything unchanged.  need_gain != 0
+ * additionally demands a strictly higher value than the job has now. */
+static int commit(Sched *S, int j, JobState *js, int gi2, int ci2, Place pl, int need_gain)
+{
+    int64_t g2 = S->g_levels[gi2], c2 = S->c_levels[ci2];
+    int k2 = pl.k;
+    int64_t avail;
+    if (k2 > 1) avail = S->Mn;
+    else avail = S->free_m[pl.node] + ((pl.stay && js->gi >= 0) ? js->m : 0);
+    int mi = -1;
+    for (int i = 0; i < S->nM; ++i)
+        if (cdiv(S->m_levels[i], k2) <= avail) mi = i;
+    if (mi < 0) return 0;
+    size_t o = cidx(S, j, gi2, ci2, mi);
+    float v = S->cv[o]; int plan = S->cp[o]; int gu = S->cg[o];
+    if (plan < 0 || !(v > 0.0f)) return 0;
+    if ((int64_t)gu != g2) return 0;              /* the level's own plans do not fit */
+    if (need_gain && js->gi >= 0 && !(v > js->val)) return 0;
+    uint32_t word = S->feas[(size_t)j * S->P + plan];
+    int f = 0; while (f < S->nM && !((word >> f) & 1u)) ++f;
+    if (f > mi) return 0;
+    int64_t m2 = S->m_levels[f];
+
+    /* remember whole nodes held, then give everything back and take the new placement */
+    int *keep = NULL; int nkeep = 0;
+    if (k2 > 1 && pl.stay && js->gi >= 0) {
+        keep = (int *)malloc(sizeof(int) * (size_t)S->N);
+        if (js->k == 1) keep[nkeep++] = js->node;
+        else for (int n = 0; n < S->N; ++n) if (S->owner[n] == j) keep[nkeep++] = n;
+    }
+    release_job(S, j, js);
+    if (k2 == 1) {
+        S->free_g[pl.node] -= g2; S->free_c[pl.node] -= c2; S->free_m[pl.node] -= m2;
+        js->node = pl.node;
+    } else {
+        int taken = 0, first = -1;
+        int64_t cs = cdiv(c2, k2), ms = cdiv(m2, k2);
+        for (int i = 0; i < nkeep; ++i) {
+            int n = keep[i];
+            S->free_g[n] -= S->Gn; S->free_c[n] -= cs; S->free_m[n] -= ms; S->owner[n] = j; ++taken;
+        }
+        for (int n = 0; n < S->N && taken < k2; ++n)
+            if (S->owner[n] != j && S->free_g[n] == S->Gn) {
+                S->free_g[n] -= S->Gn; S->free_c[n] -= cs; S->free_m[n] -= ms; S->owner[n] = j; ++taken;
+            }
+        for (int n = 0; n < S->N; ++n) if (S->owner[n] == j) { first = n; break; }
+        js->node = first;
+    }
+    free(keep);
+    js->gi = gi2; js->ci = ci2; js->g = g2; js->c = c2; js->m = m2;
+    js->plan = plan; js->k = k2; js->val = v; js->status = ST_RUNNING;
+    return 1;
+}
+
+/* CPU level an unallocated job starts its search at: its guaranteed minimum, else the lowest */
+static int start_ci(const double *job) { return (int)job[JF_CMIN] > 0 ? (int)job[JF_CMIN] : 0; }
+
+/* GPU / CPU increment the job would ask for next and its gain per unit of resource
+ * (the slope of Section 5.2).  Target GPU level: the smallest level above the present one
+ * whose curve value, at the job's CPU level and the top host-memory level, strictly
+ * exceeds the job's present value.  Target CPU level: the next one.  Returns through
+ * next[0..1] the level indices (-1 = none) and through gain[0..1] the gains. */
+static void job_gains(const Sched *S, int j, const JobState *js, int32_t *next, float *gain)
+{
+    const double *job = S->jobs + (size_t)j * JF_COUNT;
+    float w = (float)job[JF_W];
+    int mt = S->nM - 1;
+    int allocated = js->gi >= 0;
+    int ci = allocated ? js->ci : start_ci(job);
+    float cur = allocated ? js->val : 0.0f;
+    float vcur = allocated ? w * cur : 0.0f;
+    next[0] = next[1] = -1; gain[0] = gain[1] = 0.0f;
+    for (int gi = js->gi + 1; gi < S->nG; ++gi) {
+        float v = S->cv[cidx(S, j, gi, ci, mt)];
+        if (v > cur) {
+            float dg = (float)(S->g_levels[gi] - (allocated ? js->g : 0));
+            next[0] = gi;
+            gain[0] = (w * v - vcur) / dg;
+            break;
+        }
+    }
+    if (allocated && js->ci + 1 < S->nC) {
+        float v = S->cv[cidx(S, j, js->gi, js->ci + 1, mt)];
+        float dc = (float)(S->c_levels[js->ci + 1] - js->c);
+        float gn = (w * v - vcur) / dc;
+        if (gn > 0.0f) { next[1] = js->ci + 1; gain[1] = gn; }
+    }
+}
+
+/* Marginal gains of every job for a given state (no placement test, no commit).
+ * state_g / state_c / state_val: what each job holds (g = 0: nothing). */
+void oracle_gain(const double *jobs, int J, const float *curve_val,
+                 const int64_t *g_levels, int nG, const int64_t *c_levels, int nC, int nM,
+                 const int64_t *state_g, const int64_t *state_c, const float *state_val,
+                 float *gain_gpu, float *gain_cpu, int32_t *next_g, int32_t *next_c)
+{
+    Sched S; memset(&S, 0, sizeof S);
+    S.J = J; S.nG = nG; S.nC = nC; S.nM = nM; S.cv = curve_val; S.jobs = jobs;
+    S.g_levels = g_levels; S.c_levels = c_levels;
+    for (int j = 0; j < J; ++j) {
+        JobState js; memset(&js, 0, sizeof js);
+        js.gi = -1; js.ci = 0;
+        if (state_g[j] > 0) {
+            for (int i = 0; i < nG; ++i) if (g_levels[i] == state_g[j]) js.gi = i;
+            for (int i = 0; i < nC; ++i) if (c_levels[i] == state_c[j]) js.ci = i;
+            js.g = state_g[j]; js.c = state_c[j]; js.val = state_val[j];
+        }
+        int32_t next[2]; float gain[2];
+        job_gains(&S, j, &js, next, gain);
+        gain_gpu[j] = gain[0]; gain_cpu[j] = gain[1]; next_g[j] = next[0]; next_c[j] = next[1];
+    }
+}
+
+/* One scheduling round from an empty cluster of N identical nodes.
+ * Phase A: jobs with a guaranteed minimum, in index order, are placed at it.
+ * Phase B: repeatedly take, among increments that can be placed, the largest positive
+ * GPU gain (lowest job index on ties); when there is none, the largest positive CPU gain;
+ * stop when there is neither or after max_steps increments were tried.
+ * out_i: [J][8] = g, c, m_bytes, plan, first node, node count, status, m level of plan
+ * out_val: [J] predicted throughput; node_out: [N][4] = free g, free c, free m, owner
+ * step_log (optional, length max_steps): (job << 2) | (type << 1) | accepted.
+ * Returns the number of Phase-B steps, negated - 1 if the cap was hit first. */
+int oracle_round(const double *jobs, int J, const double *env,
+                 const float *curve_val, const int32_t *curve_plan, const int32_t *curve_g,
+                 const uint32_t *feas, int P,
+                 const int64_t *g_levels, int nG, const int64_t *c_levels, int nC,
+                 const int64_t *m_levels, int nM, int N, int max_steps,
+                 int64_t *out_i, float *out_val, int64_t *node_out, int32_t *step_log)
+{
+    Sched S; memset(&S, 0, sizeof S);
+    S.J = J; S.nG = nG; S.nC = nC; S.nM = nM; S.P = P; S.N = N;
+    S.cv = curve_val; S.cp = curve_plan; S.cg = curve_g; S.feas = feas; S.jobs = jobs;
+    S.g_levels = g_levels; S.c_levels = c_levels; S.m_levels = m_levels;
+    S.Gn = (int64_t)env[EF_GN]; S.Cn = (int64_t)env[EF_CN]; S.Mn = (int64_t)env[EF_MN];
+    S.free_g = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    S.free_c = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    S.free_m = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    S.owner = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    for (int n = 0; n < N; ++n) { S.free_g[n] = S.Gn; S.free_c[n] = S.Cn; S.free_m[n] = S.Mn; S.owner[n] = -1; }
+    JobState *st = (JobState *)calloc((size_t)(J > 0 ? J : 1), sizeof(JobState));
+    for (int j = 0; j < J; ++j) { st[j].gi = -1; st[j].plan = -1; st[j].node = -1; st[j].status = ST_UNALLOCATED; }
+
+    /* Phase A: guaranteed minima */
+    int mt = nM - 1;
+    for (int j = 0; j < J; ++j) {
+        const double *job = jobs + (size_t)j * JF_COUNT;
+        int gmin = (int)job[JF_GMIN];
+        if (gmin < 0) continue;
+        int cmin = start_ci(job);
+        st[j].status = ST_PENDING;
+        if (gmin >= nG || cmin >= nC) continue;
+        size_t o = cidx(&S, j, gmin, cmin, mt);
+        if (curve_plan[o] < 0) continue;
+        /* the curve may reach this value with fewer GPUs than the level offers */
+        int gi = -1;
+        for (int i = 0; i < nG; ++i) if (g_levels[i] == (int64_t)curve_g[o]) gi = i;
+        if (gi < 0) continue;
+        Place pl = find_place(&S, &st[j], g_levels[gi], c_levels[cmin]);
+        if (!pl.ok) continue;
+        commit(&S, j, &st[j], gi, cmin, pl, 0);
+        if (st[j].gi < 0) st[j].status = ST_PENDING;
+    }
+
+    /* Phase B: greedy increments */
+    int steps = 0, capped = 0;
+    for (;;) {
+        int best_j = -1, best_type = -1, best_next = -1; float best_gain = 0.0f;
+        for (int type = 0; type < 2 && best_j < 0; ++type) {
+            for (int j = 0; j < J; ++j) {
+                if (st[j].status == ST_PENDING || st[j].frozen[type]) continue;
+                int32_t next[2]; float gain[2];
+                job_gains(&S, j, &st[j], next, gain);
+                if (next[type] < 0 || !(gain[type] > 0.0f)) continue;
+                int gi2 = type == 0 ? next[0] : st[j].gi;
+                int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
+                Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+                if (!pl.ok) continue;
+                if (gain[type] > best_gain) { best_gain = gain[type]; best_j = j; best_type = type; best_next = next[type]; }
+            }
+        }
+        if (best_j < 0) break;
+        if (steps >= max_steps) { capped = 1; break; }
+        int j = best_j;
+        int gi2 = best_type == 0 ? best_next : st[j].gi;
+        int ci2 = best_type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : best_next;
+        Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+        int ok = commit(&S, j, &st[j], gi2, ci2, pl, 1);
+        if (!ok) st[j].frozen[best_type] = 1;
+        if (step_log) step_log[steps] = (int32_t)((j << 2) | (best_type << 1) | ok);
+        ++steps;
+    }
+
+    for (int j = 0; j < J; ++j) {
+        int64_t *o = out_i + (size_t)j * 8;
+        int alloc = st[j].gi >= 0;
+        o[0] = alloc ? st[j].g : 0; o[1] = alloc ? st[j].c : 0; o[2] = alloc ? st[j].m : 0;
+        o[3] = alloc ? st[j].plan : -1; o[4] = alloc ? st[j].node : -1; o[5] = alloc ? st[j].k : 0;
+        o[6] = st[j].status;
+        int f = -1;
+        if (alloc) { uint32_t wd = feas[(size_t)j * P + st[j].plan]; f = 0; while (f < nM && !((wd >> f) & 1u)) ++f; }
+        o[7] = f;
+        out_val[j] = alloc ? st[j].val : 0.0f;
+    }
+    if (node_out)
+        for (int n = 0; n < N; ++n) {
+            node_out[(size_t)n * 4 + 0] = S.free_g[n]; node_out[(size_t)n * 4 + 1] = S.free_c[n];
+            node_out[(size_t)n * 4 + 2] = S.free_m[n]; node_out[(size_t)n * 4 + 3] = S.owner[n];
+        }
+    free(S.free_g); free(S.free_c); free(S.free_m); free(S.owner); free(st);
+    return capped ? -steps - 1 : steps;
+}
+
+/* Exhaustive search on one node (tiny instances only): every job is either left out or
+ * given one (g level, c level, m level); the allocation uses the GPUs of the curve entry,
+ * the cores of the level and the memory of the entry's plan; sums must fit the node.
+ * Returns the largest total weighted throughput (double accumulation of w * value, the
+ * products taken in single precision as in the greedy round). */
+typedef struct { float v; int64_t g, c, m; } Opt;
+
+static void bf_rec(int j, int J, const Opt *opts, const int *nopt, int maxopt,
+                   int64_t rg, int64_t rc, int64_t rm, double acc, double *best)
+{
+    if (j == J) { if (acc > *best) *best = acc; return; }
+    bf_rec(j + 1, J, opts, nopt, maxopt, rg, rc, rm, acc, best);
+    for (int i = 0; i < nopt[j]; ++i) {
+        const Opt *o = &opts[(size_t)j * maxopt + i];
+        if (o->g <= rg && o->c <= rc && o->m <= rm)
+            bf_rec(j + 1, J, opts, nopt, maxopt, rg - o->g, rc - o->c, rm - o->m, acc + (double)o->v, best);
+    }
+}
+
+double oracle_bruteforce(const double *jobs, int J, const double *env,
+                         const float *curve_val, const int32_t *curve_plan, const int32_t *curve_g,
+                         const uint32_t *feas, int P,
+                         const int64_t *g_levels, int nG, const int64_t *c_levels, int nC,
+                         const int64_t *m_levels, int nM)
+{
+    int maxopt = nG * nC * nM;
+    Opt *opts = (Opt *)malloc(sizeof(Opt) * (size_t)maxopt * (size_t)(J > 0 ? J : 1));
+    int *nopt = (int *)calloc((size_t)(J > 0 ? J : 1), sizeof(int));
+    (void)g_levels;
+    for (int j = 0; j < J; ++j) {
+        float w = (float)jobs[(size_t)j * JF_COUNT + JF_W];
+        for (int gi = 0; gi < nG; ++gi)
+            for (int ci = 0; ci < nC; ++ci)
+                for (int mi = 0; mi < nM; ++mi) {
+                    size_t o = (((size_t)j * nG + gi) * nC + ci) * nM + mi;
+                    if (curve_plan[o] < 0) continue;
+                    uint32_t wd = feas[(size_t)j * P + curve_plan[o]];
+                    int f = 0; while (f < nM && !((wd >> f) & 1u)) ++f;
+                    if (f > mi) continue;
+                    Opt *op = &opts[(size_t)j * maxopt + nopt[j]++];
+                    op->v = w * curve_val[o]; op->g = curve_g[o]; op->c = c_levels[ci]; op->m = m_levels[f];
+                }
+    }
+    double best = 0.0;
+    bf_rec(0, J, opts, nopt, maxopt, (int64_t)env[EF_GN], (int64_t)env[EF_CN], (int64_t)env[EF_MN], 0.0, &best);
+    free(opts); free(nopt);
+    return best;
+}

@@ -1,0 +1,97 @@
+"""Seeded synthetic workloads shaped like the paper's evaluation (Section 7).
+
+This module only draws numbers.  It holds none of the scheduler's arithmetic and is the one
+piece of code that both the CUDA library's tests and the CPU checker read their inputs from.
+
+Shapes follow the paper's setting: transformer jobs between 125 M and 13 B / 70 B parameters
+(Table 2 spans 86 M - 30 B), nodes of 8 GPUs (80 GB each) with 96 cores, 400 GB/s inside and
+100 GB/s between nodes (Section 7).  The paper prints no fitted coefficients and its job
+trace is not public in numeric form, so coefficients are a nominal constant times a
+uniform factor in [0.5, 2] and arrivals are Poisson with log-normal lengths.
+
+Every floating-point job coefficient is rounded to single precision here, so that a
+double-precision consumer and a single-precision consumer start from identical values.
+"""
+import numpy as np
+
+GIB = 1 << 30
+
+# nominal coefficient values (constants of this generator; the paper gives none)
+NOMINAL = dict(k_bwd=2.0, k_sync=2.0, k_opt=1e-11, k_opt_off=2e-8, k_off=2.0, k_swap=2.0, k_const=0.05)
+PEAK_FLOPS_PER_SAMPLE_DIVISOR = 1.25e14      # tau nominal = 2 * P * s / 1.25e14 seconds per sample
+ALPHA_ACT = 34                               # activation bytes per token x hidden per layer
+HOST_BASE = 4 * GIB                          # host bytes per training process
+
+ENV = dict(B_intra=400e9, B_inter=100e9, B_pcie=25e9, gpu_mem_bytes=80_000_000_000,
+           gpus_per_node=8, cpus_per_node=96, mem_per_node_bytes=1024 * GIB, bytes_per_elem=2,
+           strict_zero_dp_only=0)
+
+CONFIGS = {
+    # name: (seed, jobs, nodes, g levels, c levels, m levels [GiB], largest parameter count)
+    "tiny": dict(seed=0, J=4, N=1, g=list(range(1, 9)), c=[4, 8, 16, 32], m=[64, 128, 256], pmax=13e9),
+    "paper-scale": dict(seed=1, J=64, N=8, g=[1, 2, 4, 8, 16, 32, 64], c=list(range(4, 97, 4)),
+                        m=list(range(32, 1025, 32)), pmax=13e9),
+    "cluster-512": dict(seed=2, J=1024, N=64, g=[1 << i for i in range(9)], c=list(range(4, 97, 4)),
+                        m=list(range(32, 1025, 32)), pmax=70e9),
+    "throughput-stress": dict(seed=3, J=16384, N=512, g=[1 << i for i in range(9)], c=list(range(4, 97, 4)),
+                              m=list(range(32, 1025, 32)), pmax=70e9),
+    "events": dict(seed=4, J=4096, N=512, g=[1 << i for i in range(9)], c=list(range(4, 97, 4)),
+                   m=list(range(32, 1025, 32)), pmax=70e9),
+}
+
+
+def _f32(x):
+    return np.asarray(x, dtype=np.float32).astype(np.float64)
+
+
+def draw_jobs(rng, J, g_levels, n_c_levels, pmax=13e9, pmin=125e6, guaranteed_share=0.25):
+    """Per-job model inputs as a dict of length-J arrays, drawn field by field in a fixed order."""
+    P = np.floor(np.exp(rng.uniform(np.log(pmin), np.log(pmax), J)))
+    l = rng.integers(12, 49, J)
+    h = 128 * rng.integers(768 // 128, 5120 // 128 + 1, J)
+    b = rng.choice([16, 32, 64, 128], J)
+    s = rng.choice([512, 1024, 2048], J)
+    mu_cap = rng.choice([1, 2, 4, 8], J)
+    tau = _f32(2.0 * P * s / PEAK_FLOPS_PER_SAMPLE_DIVISOR * rng.uniform(0.5, 2.0, J))
+    jobs = dict(P=P, l=l, h=h, s=s, b=b, mu_cap=mu_cap, alpha_act=np.full(J, ALPHA_ACT), tau=tau)
+    for k in ("k_bwd", "k_sync", "k_opt", "k_opt_off", "k_off", "k_swap", "k_const"):
+        jobs[k] = _f32(NOMINAL[k] * rng.uniform(0.5, 2.0, J))
+    # weight: seconds of one-GPU compute per sample, so that weighted throughput reads as a
+    # speed-up over a one-GPU run and jobs of different sizes compare (Section 7.2 normalises
+    # each job's throughput before adding them up)
+    jobs["w"] = _f32(3.0 * tau)
+    # a share of the jobs is "guaranteed" with a small minimum demand, the rest best effort
+    pow2_idx = [i for i, g in enumerate(g_levels) if g & (g - 1) == 0][:4]
+    guaranteed = rng.uniform(0.0, 1.0, J) < guaranteed_share
+    gpick = rng.choice(pow2_idx, J)
+    cpick = rng.integers(0, min(3, n_c_levels), J)
+    jobs["gmin_idx"] = np.where(guaranteed, gpick, -1)
+    jobs["cmin_idx"] = np.where(guaranteed, cpick, -1)
+    jobs["host_base_bytes"] = np.full(J, HOST_BASE)
+    return jobs
+
+
+def make(name, J=None, n_nodes=None):
+    """Build a named configuration; J / n_nodes override the size (same seed, same recipe)."""
+    cfg = CONFIGS[name]
+    rng = np.random.Generator(np.random.PCG64(cfg["seed"]))
+    J = cfg["J"] if J is None else J
+    jobs = draw_jobs(rng, J, cfg["g"], len(cfg["c"]), pmax=cfg["pmax"])
+    return dict(name=name, seed=cfg["seed"], jobs=jobs, env=dict(ENV),
+                g_levels=np.asarray(cfg["g"], dtype=np.int64),
+                c_levels=np.asarray(cfg["c"], dtype=np.int64),
+                m_levels=np.asarray(cfg["m"], dtype=np.int64) * GIB,
+                n_nodes=cfg["N"] if n_nodes is None else n_nodes)
+
+
+def take(jobs, idx):
+    """Sub-select jobs (dict of arrays) by index array / slice."""
+    return {k: np.asarray(v)[idx] for k, v in jobs.items()}
+
+
+def draw_events(seed, n_jobs, mean_interarrival_s=30.0, median_len_s=7200.0, sigma=1.5):
+    """Arrival times (Poisson process) and nominal lengths (log-normal) for an event-driven run."""
+    rng = np.random.Generator(np.random.PCG64(seed + 1000))
+    arrivals = np.cumsum(rng.exponential(mean_interarrival_s, n_jobs))
+    lengths = np.exp(rng.normal(np.log(median_len_s), sigma, n_jobs))
+    return arrivals, lengths
