@@ -1,0 +1,216 @@
+/*
+ * rubick.h -- C ABI of the B200 (sm_100a) library for the data-parallel hot path of the
+ * Rubick scheduler (arXiv 2408.08586): batched evaluation of the paper's training-performance
+ * model over every (job x execution plan x resource allocation) candidate, the memory-feasibility
+ * mask, the per-(job, allocation) best plan and resource-sensitivity curve, per-job marginal
+ * gains, and a greedy allocation round that runs entirely on the device.
+ *
+ * Conventions
+ *  - Every call returns an int: RUBICK_OK (0) or a negative error code.  Nothing throws, aborts
+ *    or prints.  rubick_last_error(ctx) returns a context-owned, NUL-terminated description of
+ *    the last failure on that context.
+ *  - Pointer names say where the memory lives: d_ = device memory owned by the CALLER,
+ *    h_ = host memory owned by the caller.  The library frees only what it allocated itself
+ *    (the context, its tables and scratch).
+ *  - All arguments are validated on the host before anything is launched; a rejected call
+ *    launches nothing and writes nothing.
+ *  - Device work is enqueued on the stream given to rubick_create and is complete after
+ *    rubick_sync(ctx) (or the caller's own synchronisation of that stream).  Calls on one
+ *    context must not overlap in time from several host threads.
+ *  - There is no CPU fallback: without a CUDA device every compute call fails with RUBICK_ECUDA.
+ *
+ * Index order of the tables (C order, last index fastest):
+ *    thr        [J][C][P]      float     predicted samples / second, 0 for an invalid plan
+ *    feas       [J][P]         uint32    bit i set <=> plan may run with host-memory level i
+ *    best_*     [J][G][C][M]   float / int32
+ * with J jobs, P plans, and G / C / M levels of GPUs / CPU cores / host memory.
+ */
+#ifndef RUBICK_H
+#define RUBICK_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define RUBICK_OK       0
+#define RUBICK_EINVAL  (-1)   /* bad argument (sizes, ordering, null pointer, unsupported shape)  */
+#define RUBICK_ENOMEM  (-2)   /* a device or host allocation of the library failed                */
+#define RUBICK_ECUDA   (-3)   /* the CUDA runtime reported an error (no device, launch failure)   */
+#define RUBICK_ESTEPS  (-4)   /* the greedy round stopped at max_steps; the partial result is valid */
+#define RUBICK_ESTATE  (-5)   /* call order (no plan space set) or inconsistent table contents    */
+
+#define RUBICK_MAX_G_LEVELS  32
+#define RUBICK_MAX_C_LEVELS  64
+#define RUBICK_MAX_M_LEVELS  32      /* one feasibility word per (job, plan) */
+#define RUBICK_MAX_NODES     4096    /* node state of a round lives in shared memory */
+
+/* per-job status in rubick_assignment */
+#define RUBICK_UNALLOCATED 0
+#define RUBICK_RUNNING     1
+#define RUBICK_PENDING     2         /* guaranteed minimum could not be placed */
+
+/* flags of rubick_best_plan */
+#define RUBICK_BEST_RAW    1u        /* per-level best only; default also takes the running maximum over g */
+
+typedef struct rubick_ctx rubick_ctx;
+
+/* Environment (paper Table 1, "Environment" row, plus the node shape of Section 7). */
+typedef struct {
+    double  B_intra, B_inter, B_pcie;   /* bytes / second inside a node, between nodes, GPU <-> host */
+    int64_t gpu_mem_bytes;              /* memory of one GPU                                         */
+    int64_t mem_per_node_bytes;         /* host memory of one node                                   */
+    int32_t gpus_per_node;              /* must be a power of two                                    */
+    int32_t cpus_per_node;
+    int32_t bytes_per_elem;             /* 2 = fp16 mixed precision                                  */
+    int32_t strict_zero_dp_only;        /* 1: ZeRO stages / offload only for pure data parallelism   */
+} rubick_env;
+
+/* One job: the model, batch and fitted coefficients of paper Table 1.  Exactly 128 bytes. */
+typedef struct {
+    double   P;                  /* parameter count (integer-valued)                                */
+    int64_t  host_base_bytes;    /* host memory of one training process (one per GPU)               */
+    int32_t  l, h, s, b;         /* layers, hidden size, sequence length, global batch              */
+    int32_t  mu_cap;             /* largest micro-batch a replica runs at once                      */
+    int32_t  alpha_act;          /* activation bytes per (token x hidden unit) per layer            */
+    float    tau;                /* forward seconds per sample, whole model on one GPU              */
+    float    k_bwd, k_sync, k_opt, k_opt_off, k_off, k_swap, k_const;  /* fittable coefficients     */
+    float    w;                  /* weight of this job's throughput in the scheduling objective     */
+    int32_t  gmin_idx, cmin_idx; /* guaranteed minimum as level indices; -1 = best effort / none    */
+    uint32_t flags;              /* reserved, 0                                                     */
+    uint8_t  pad[40];
+} rubick_job;
+
+/* One execution plan (paper Section 3): DP / TP / PP degrees as log2, ZeRO stage 0..3, gradient
+ * checkpointing, ZeRO-Offload; g_level = index of its GPU count 2^(log2d+log2t+log2p) in the grid. */
+typedef struct {
+    uint8_t log2d, log2t, log2p, zero, gc, off;
+    uint8_t g_level;
+    uint8_t disabled;            /* non-zero: treat as invalid for every job */
+} rubick_plan;
+
+/* Resource grid: strictly increasing level values on each axis. */
+typedef struct {
+    int32_t nG, nC, nM;
+    int32_t reserved;
+    const int32_t *g_levels;         /* GPUs                 [nG] */
+    const int32_t *c_levels;         /* CPU cores            [nC] */
+    const int64_t *m_levels_bytes;   /* host memory in bytes [nM] */
+} rubick_grid;
+
+/* Homogeneous cluster: n_nodes nodes of the environment's shape, all free at the start of a round. */
+typedef struct { int32_t n_nodes; } rubick_cluster;
+
+/* Result (and input state) per job. 40 bytes. */
+typedef struct {
+    int32_t g, c;                /* GPUs and cores held; g == 0: nothing                            */
+    int64_t m_bytes;             /* host memory held                                                */
+    int32_t plan;                /* plan index, -1 if none                                          */
+    int32_t first_node, n_nodes; /* lowest node index used and number of nodes                      */
+    float   thr;                 /* predicted throughput of (plan, allocation)                      */
+    int32_t status;              /* RUBICK_UNALLOCATED / RUNNING / PENDING                          */
+    int32_t m_level;             /* host-memory level index of m_bytes, -1 if none                  */
+} rubick_assignment;
+
+/* Per-node state after a round. 24 bytes. */
+typedef struct {
+    int32_t free_g, free_c;
+    int64_t free_m;
+    int32_t owner;               /* job that holds this whole node as part of a multi-node set, else -1 */
+    int32_t reserved;
+} rubick_node;
+
+/* ---- context ---------------------------------------------------------------------------------- */
+
+/* Creates a context bound to CUDA device `device` and to `cuda_stream` (a cudaStream_t passed as
+ * void*; NULL = the default stream).  Copies *h_env.  Errors: EINVAL (null pointers, non-positive
+ * sizes or bandwidths, gpus_per_node not a power of two), ECUDA (no such device), ENOMEM. */
+int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *cuda_stream);
+
+/* Frees the context and everything it allocated.  NULL is allowed. */
+void rubick_destroy(rubick_ctx *ctx);
+
+/* Blocks until all work enqueued by this context has finished.  Returns ESTATE if a kernel
+ * found inconsistent table contents (a feasibility word that is not a threshold in the level
+ * index), ECUDA on a runtime error. */
+int rubick_sync(rubick_ctx *ctx);
+
+const char *rubick_last_error(const rubick_ctx *ctx);
+
+/* ---- plan space (host, set-up) ---------------------------------------------------------------- */
+
+/* Enumerates the plan space of Section 3 in canonical order: for every level of h_g_levels that is
+ * a power of two, every (d, t, p) of powers of two with d*t*p = g (TP degree ascending, then PP
+ * degree ascending), then ZeRO stage 0..3, gradient checkpointing off/on, offload off/on.
+ * Writes at most cap plans to h_out, the total count to *n_out (also when it exceeds cap) and, if
+ * h_group_off is not NULL, nG + 1 offsets: level i owns plans [off[i], off[i+1]).
+ * Pure host code; needs no context and no device. */
+int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out, int cap, int *n_out,
+                           int32_t *h_group_off);
+
+/* Installs the plan list and the resource grid (copied; tables are uploaded to the device).
+ * Requirements (EINVAL otherwise): 1 <= nG <= RUBICK_MAX_G_LEVELS, 1 <= nC <= RUBICK_MAX_C_LEVELS,
+ * 1 <= nM <= RUBICK_MAX_M_LEVELS, strictly increasing positive levels, GPU levels above
+ * gpus_per_node multiples of it; P a positive multiple of 4; plans ordered by g_level and laid out
+ * in runs of four that share (log2d, log2t, log2p, zero) with (gc, off) = (0,0), (0,1), (1,0), (1,1),
+ * as rubick_enumerate_plans writes them; each plan's GPU count equals g_levels[g_level]. */
+int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const rubick_grid *h_grid);
+
+/* ---- the hot path ----------------------------------------------------------------------------- */
+
+/* Candidate table (paper Section 4, Eq. 1 with all its terms; THROUGHPUT = b / T_iter) and the
+ * memory-feasibility mask, for jobs d_jobs[0..J).  d_thr: J*C*P floats, d_feas: J*P words, both
+ * 16-byte aligned.  To stream a large job set in tiles, call once per tile with offset pointers.
+ * J == 0 is allowed and does nothing.  Single-precision arithmetic; masks in exact 64-bit integers. */
+int rubick_eval_candidates(rubick_ctx *ctx, const rubick_job *d_jobs, int J, float *d_thr, uint32_t *d_feas);
+
+/* Best plan per (job, GPU level, core level, memory level): the largest d_thr among the level's
+ * plans whose feasibility bit is set, lowest plan index on ties, (0, -1, 0) when there is none
+ * (Section 5.2: invalid GPU counts have zero throughput).  Unless RUBICK_BEST_RAW is given the
+ * result is turned into the resource-sensitivity curve: the running maximum along the GPU axis,
+ * carrying the plan and the GPU count actually used (Section 5.2, Fig. 6).
+ * d_best_val / d_best_plan / d_best_g: J*G*C*M entries each.  Feasibility words must be
+ * thresholds (bit i set implies every higher level bit set); a violation is reported by
+ * rubick_sync as ESTATE. */
+int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
+                     float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g);
+
+/* Marginal gain ("slope", Section 5.2) of the next GPU and the next CPU increment of every job in
+ * state d_state (fields g, c, thr are read; g == 0 means nothing held): the weighted curve gain
+ * per added GPU up to the smallest level that strictly improves on the present value, and per
+ * added core up to the next core level, both at the top host-memory level.  d_next_g / d_next_c
+ * receive the target level indices (-1 = none), d_gain_* the gains (0 = none). */
+int rubick_marginal_gain(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_curve_val,
+                         const rubick_assignment *d_state,
+                         float *d_gain_gpu, float *d_gain_cpu, int32_t *d_next_g, int32_t *d_next_c);
+
+/* One greedy scheduling round (Section 5.2, Algorithm 1 in marginal-gain form) on given curve
+ * tables, from an empty cluster, entirely on the device: guaranteed minima first, in job order;
+ * then repeatedly the placeable increment with the largest positive GPU gain (CPU gain when no
+ * GPU increment is left), lowest job index on ties, committed with the best plan and its host
+ * memory for the chosen node(s).  d_out: J assignments.  Optional (NULL to skip): d_node_out,
+ * n_nodes entries; d_step_log, max_steps int32 entries (job << 2 | type << 1 | accepted);
+ * h_steps, the number of increments tried.  Blocks until the round is done.
+ * Returns ESTEPS if max_steps was reached first. */
+int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                        const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
+                        const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
+                        rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                        int32_t *h_steps);
+
+/* The whole path for one scheduling event: candidate table, mask, curves and greedy round for
+ * d_jobs[0..J), with the intermediate tables in context-owned scratch (grown on demand, kept
+ * between calls).  Outputs as rubick_greedy_round. */
+int rubick_schedule_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const rubick_cluster *h_cluster,
+                          int max_steps, rubick_assignment *d_out, rubick_node *d_node_out, int32_t *h_steps);
+
+/* Same with HOST buffers: copies h_jobs to the device, runs the round, copies the assignments
+ * (and node states, if h_node_out is not NULL) back.  h_jobs / h_out may be pageable or pinned. */
+int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J, const rubick_cluster *h_cluster,
+                               int max_steps, rubick_assignment *h_out, rubick_node *h_node_out, int32_t *h_steps);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RUBICK_H */

@@ -1,0 +1,389 @@
+// Host side of librubick: context, plan enumerator, validation and the extern "C" entry points.
+// Every entry point validates its arguments, then enqueues kernels on the context's stream.
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "rubick_internal.cuh"
+
+using namespace rubick;
+
+namespace rubick {
+
+int fail(rubick_ctx *ctx, int code, const char *msg)
+{
+    if (ctx) ctx->err = msg;
+    return code;
+}
+
+int cuda_fail(rubick_ctx *ctx, cudaError_t e, const char *what)
+{
+    if (ctx) {
+        ctx->err = std::string(what) + ": " + cudaGetErrorString(e);
+    }
+    return e == cudaErrorMemoryAllocation ? RUBICK_ENOMEM : RUBICK_ECUDA;
+}
+
+static bool is_pow2(int64_t x) { return x > 0 && (x & (x - 1)) == 0; }
+static int ilog2(int64_t x) { int n = 0; while ((int64_t(1) << (n + 1)) <= x) ++n; return n; }
+
+// grows a device buffer to at least `need` elements (contents are not preserved)
+template <typename T>
+static int ensure(rubick_ctx *ctx, T *&ptr, size_t &cap, size_t need)
+{
+    if (need <= cap) return RUBICK_OK;
+    if (ptr) { cudaFree(ptr); ptr = nullptr; cap = 0; }
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&ptr), need * sizeof(T));
+    if (e != cudaSuccess) { ptr = nullptr; return cuda_fail(ctx, e, "cudaMalloc (scratch)"); }
+    cap = need;
+    return RUBICK_OK;
+}
+
+}  // namespace rubick
+
+#define CHECK_CTX(ctx) do { if (!(ctx)) return RUBICK_EINVAL; } while (0)
+#define CUDA_TRY(ctx, call, what) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail(ctx, e_, what); } while (0)
+
+extern "C" {
+
+int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *cuda_stream)
+{
+    if (!out || !h_env) return RUBICK_EINVAL;
+    *out = nullptr;
+    const rubick_env &e = *h_env;
+    if (!(e.B_intra > 0) || !(e.B_inter > 0) || !(e.B_pcie > 0) || e.gpu_mem_bytes <= 0 || e.mem_per_node_bytes <= 0
+        || e.gpus_per_node <= 0 || e.cpus_per_node <= 0 || e.bytes_per_elem <= 0 || !is_pow2(e.gpus_per_node))
+        return RUBICK_EINVAL;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) return RUBICK_ECUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return RUBICK_ECUDA;
+    rubick_ctx *ctx = new (std::nothrow) rubick_ctx();
+    if (!ctx) return RUBICK_ENOMEM;
+    ctx->env = e;
+    ctx->device = device;
+    ctx->stream = static_cast<cudaStream_t>(cuda_stream);
+    ctx->has_space = false;
+    ctx->d_quads = nullptr; ctx->d_status = nullptr; ctx->d_steps = nullptr;
+    ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0;
+    ctx->d_thr = nullptr; ctx->d_feas = nullptr; ctx->d_cv = nullptr; ctx->d_cp = nullptr; ctx->d_cg = nullptr;
+    ctx->cap_thr = ctx->cap_feas = ctx->cap_curve = 0;
+    ctx->d_jobs_stage = nullptr; ctx->cap_jobs = 0;
+    ctx->d_out_stage = nullptr; ctx->cap_out = 0;
+    ctx->d_node_stage = nullptr; ctx->cap_node = 0;
+    ctx->tile_jobs = 256;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return RUBICK_ECUDA; }
+    ctx->num_sms = prop.multiProcessorCount;
+    if (cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 8) != cudaSuccess) { delete ctx; return RUBICK_ENOMEM; }
+    ctx->d_steps = reinterpret_cast<int32_t *>(ctx->d_status + 1);
+    if (cudaMemsetAsync(ctx->d_status, 0, 8, ctx->stream) != cudaSuccess) { cudaFree(ctx->d_status); delete ctx; return RUBICK_ECUDA; }
+    *out = ctx;
+    return RUBICK_OK;
+}
+
+void rubick_destroy(rubick_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->d_quads); cudaFree(ctx->d_status); cudaFree(ctx->d_round_scratch);
+    cudaFree(ctx->d_thr); cudaFree(ctx->d_feas); cudaFree(ctx->d_cv); cudaFree(ctx->d_cp); cudaFree(ctx->d_cg);
+    cudaFree(ctx->d_jobs_stage); cudaFree(ctx->d_out_stage); cudaFree(ctx->d_node_stage);
+    delete ctx;
+}
+
+const char *rubick_last_error(const rubick_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int rubick_sync(rubick_ctx *ctx)
+{
+    CHECK_CTX(ctx);
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+    uint32_t st = 0;
+    CUDA_TRY(ctx, cudaMemcpy(&st, ctx->d_status, 4, cudaMemcpyDeviceToHost), "read status");
+    if (st & DS_FEAS_NOT_THRESHOLD) {
+        cudaMemset(ctx->d_status, 0, 4);
+        return fail(ctx, RUBICK_ESTATE, "a feasibility word is not a threshold in the memory-level index");
+    }
+    return RUBICK_OK;
+}
+
+int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out, int cap, int *n_out,
+                           int32_t *h_group_off)
+{
+    if (!h_g_levels || nG < 1 || nG > RUBICK_MAX_G_LEVELS || !n_out || cap < 0 || (cap > 0 && !h_out)) return RUBICK_EINVAL;
+    for (int i = 0; i < nG; ++i)
+        if (h_g_levels[i] <= 0 || (i && h_g_levels[i] <= h_g_levels[i - 1])) return RUBICK_EINVAL;
+    int n = 0;
+    for (int gi = 0; gi < nG; ++gi) {
+        if (h_group_off) h_group_off[gi] = n;
+        const int g = h_g_levels[gi];
+        if (!is_pow2(g)) continue;            // only power-of-two GPU counts factor into (d, t, p)
+        const int lg = ilog2(g);
+        for (int lt = 0; lt <= lg; ++lt)
+            for (int lp = 0; lp + lt <= lg; ++lp)
+                for (int z = 0; z < 4; ++z)
+                    for (int v = 0; v < 4; ++v, ++n)
+                        if (n < cap) {
+                            rubick_plan &pl = h_out[n];
+                            pl.log2d = uint8_t(lg - lt - lp); pl.log2t = uint8_t(lt); pl.log2p = uint8_t(lp);
+                            pl.zero = uint8_t(z); pl.gc = uint8_t(v >> 1); pl.off = uint8_t(v & 1);
+                            pl.g_level = uint8_t(gi); pl.disabled = 0;
+                        }
+    }
+    if (h_group_off) h_group_off[nG] = n;
+    *n_out = n;
+    return RUBICK_OK;
+}
+
+int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const rubick_grid *h_grid)
+{
+    CHECK_CTX(ctx);
+    if (!h_plans || !h_grid || P <= 0 || (P & 3)) return fail(ctx, RUBICK_EINVAL, "plans: need a positive multiple of 4");
+    const rubick_grid &gr = *h_grid;
+    if (gr.nG < 1 || gr.nG > RUBICK_MAX_G_LEVELS || gr.nC < 1 || gr.nC > RUBICK_MAX_C_LEVELS || gr.nM < 1
+        || gr.nM > RUBICK_MAX_M_LEVELS || !gr.g_levels || !gr.c_levels || !gr.m_levels_bytes)
+        return fail(ctx, RUBICK_EINVAL, "grid: level counts out of range or null axes");
+    const int Gn = ctx->env.gpus_per_node;
+    for (int i = 0; i < gr.nG; ++i) {
+        const int g = gr.g_levels[i];
+        if (g <= 0 || (i && g <= gr.g_levels[i - 1]) || (g > Gn && g % Gn)) return fail(ctx, RUBICK_EINVAL, "grid: GPU levels must increase; levels above a node must be whole nodes");
+    }
+    for (int i = 0; i < gr.nC; ++i)
+        if (gr.c_levels[i] <= 0 || (i && gr.c_levels[i] <= gr.c_levels[i - 1])) return fail(ctx, RUBICK_EINVAL, "grid: CPU levels must be positive and increasing");
+    for (int i = 0; i < gr.nM; ++i)
+        if (gr.m_levels_bytes[i] <= 0 || (i && gr.m_levels_bytes[i] <= gr.m_levels_bytes[i - 1])) return fail(ctx, RUBICK_EINVAL, "grid: memory levels must be positive and increasing");
+
+    Space sp;
+    std::memset(&sp, 0, sizeof sp);
+    sp.P = P; sp.Q = P / 4; sp.nG = gr.nG; sp.nC = gr.nC; sp.nM = gr.nM;
+    sp.Gn = Gn; sp.log2Gn = ilog2(Gn); sp.Cn = ctx->env.cpus_per_node;
+    sp.strict = ctx->env.strict_zero_dp_only ? 1 : 0;
+    sp.e = float(ctx->env.bytes_per_elem);
+    sp.inv_B_intra = float(1.0 / ctx->env.B_intra);
+    sp.inv_B_inter = float(1.0 / ctx->env.B_inter);
+    sp.inv_B_pcie = float(1.0 / ctx->env.B_pcie);
+    sp.gpu_mem = ctx->env.gpu_mem_bytes; sp.Mn = ctx->env.mem_per_node_bytes;
+    for (int i = 0; i < gr.nG; ++i) { sp.g_levels[i] = gr.g_levels[i]; if (gr.g_levels[i] <= Gn) sp.n_small = i + 1; }
+    for (int i = 0; i < gr.nC; ++i) { sp.c_levels[i] = gr.c_levels[i]; sp.inv_c[i] = 1.0f / float(gr.c_levels[i]); }
+    for (int i = 0; i < gr.nM; ++i) sp.m_levels[i] = gr.m_levels_bytes[i];
+
+    // plans: ordered by level, quads of (gc, off), GPU count = the level's
+    std::vector<QuadDesc> quads(size_t(P) / 4);
+    int level = 0;
+    sp.group_off[0] = 0;
+    for (int i = 0; i < P; ++i) {
+        const rubick_plan &pl = h_plans[i];
+        if (pl.g_level >= gr.nG || pl.g_level < level) return fail(ctx, RUBICK_EINVAL, "plans: g_level out of range or not ascending");
+        if (pl.zero > 3 || pl.gc > 1 || pl.off > 1 || pl.log2d > 15 || pl.log2t > 15 || pl.log2p > 15
+            || int(pl.log2d) + pl.log2t + pl.log2p > 20)
+            return fail(ctx, RUBICK_EINVAL, "plans: field out of range");
+        if ((int64_t(1) << (pl.log2d + pl.log2t + pl.log2p)) != gr.g_levels[pl.g_level])
+            return fail(ctx, RUBICK_EINVAL, "plans: d*t*p differs from the GPU level");
+        if (pl.g_level > level) {
+            if (i & 3) return fail(ctx, RUBICK_EINVAL, "plans: a level must start on a quad boundary");
+            while (level < pl.g_level) sp.group_off[++level] = i;
+        }
+        const int v = i & 3;
+        if (pl.gc != (v >> 1) || pl.off != (v & 1)) return fail(ctx, RUBICK_EINVAL, "plans: quads must run (gc, off) = (0,0), (0,1), (1,0), (1,1)");
+        QuadDesc &q = quads[size_t(i) >> 2];
+        if (v == 0) {
+            q.log2d = pl.log2d; q.log2t = pl.log2t; q.log2p = pl.log2p; q.zero = pl.zero; q.g_level = pl.g_level;
+            q.flags = 0; q.disabled = 0; q.pad = 0;
+            const int64_t d = int64_t(1) << pl.log2d, t = int64_t(1) << pl.log2t, g = gr.g_levels[pl.g_level];
+            if (t <= Gn) q.flags |= QF_T_FITS_NODE;
+            if (d * t > Gn) q.flags |= QF_DP_INTER;
+            if (g > Gn) q.flags |= QF_PP_INTER;
+        } else if (q.log2d != pl.log2d || q.log2t != pl.log2t || q.log2p != pl.log2p || q.zero != pl.zero) {
+            return fail(ctx, RUBICK_EINVAL, "plans: the four plans of a quad must share d, t, p and the ZeRO stage");
+        }
+        if (pl.disabled) q.disabled |= uint8_t(1u << v);
+    }
+    while (level < gr.nG) sp.group_off[++level] = P;
+
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device), "cudaSetDevice");
+    if (ctx->d_quads) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_quads); ctx->d_quads = nullptr; }
+    CUDA_TRY(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->d_quads), quads.size() * sizeof(QuadDesc)), "cudaMalloc (plan table)");
+    CUDA_TRY(ctx, cudaMemcpy(ctx->d_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice), "upload plan table");
+    ctx->space = sp;
+    ctx->plans.assign(h_plans, h_plans + P);
+    ctx->has_space = true;
+    return RUBICK_OK;
+}
+
+static int check_ready(rubick_ctx *ctx, int J)
+{
+    if (!ctx->has_space) return fail(ctx, RUBICK_ESTATE, "no plan space: call rubick_set_space first");
+    if (J < 0) return fail(ctx, RUBICK_EINVAL, "negative job count");
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return fail(ctx, RUBICK_ECUDA, "cudaSetDevice failed");
+    return RUBICK_OK;
+}
+
+int rubick_eval_candidates(rubick_ctx *ctx, const rubick_job *d_jobs, int J, float *d_thr, uint32_t *d_feas)
+{
+    CHECK_CTX(ctx);
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (J == 0) return RUBICK_OK;
+    if (!d_jobs || !d_thr || !d_feas) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if ((reinterpret_cast<uintptr_t>(d_thr) & 15) || (reinterpret_cast<uintptr_t>(d_feas) & 15) || (reinterpret_cast<uintptr_t>(d_jobs) & 15))
+        return fail(ctx, RUBICK_EINVAL, "d_jobs, d_thr and d_feas must be 16-byte aligned");
+    if (int64_t(J) * ctx->space.Q >= (int64_t(1) << 31)) return fail(ctx, RUBICK_EINVAL, "J * P / 4 must stay below 2^31: evaluate in job tiles");
+    CUDA_TRY(ctx, launch_eval(ctx->space, ctx->d_quads, d_jobs, J, d_thr, d_feas, ctx->stream), "launch eval_candidates");
+    return RUBICK_OK;
+}
+
+int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
+                     float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g)
+{
+    CHECK_CTX(ctx);
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (J == 0) return RUBICK_OK;
+    if (!d_thr || !d_feas || !d_best_val || !d_best_plan || !d_best_g) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if (reinterpret_cast<uintptr_t>(d_thr) & 15) return fail(ctx, RUBICK_EINVAL, "d_thr must be 16-byte aligned");
+    if (flags & ~RUBICK_BEST_RAW) return fail(ctx, RUBICK_EINVAL, "unknown flag");
+    CUDA_TRY(ctx, launch_best(ctx->space, d_thr, d_feas, J, flags, d_best_val, d_best_plan, d_best_g, ctx->d_status, ctx->stream),
+             "launch best_plan");
+    return RUBICK_OK;
+}
+
+int rubick_marginal_gain(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_curve_val,
+                         const rubick_assignment *d_state,
+                         float *d_gain_gpu, float *d_gain_cpu, int32_t *d_next_g, int32_t *d_next_c)
+{
+    CHECK_CTX(ctx);
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (J == 0) return RUBICK_OK;
+    if (!d_jobs || !d_curve_val || !d_state || !d_gain_gpu || !d_gain_cpu || !d_next_g || !d_next_c) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    CUDA_TRY(ctx, launch_gain(ctx->space, d_jobs, J, d_curve_val, d_state, d_gain_gpu, d_gain_cpu, d_next_g, d_next_c, ctx->stream),
+             "launch marginal_gain");
+    return RUBICK_OK;
+}
+
+// enqueue the round and leave the step count in ctx->d_steps
+static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
+                         const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps, rubick_assignment *d_out,
+                         rubick_node *d_node_out, int32_t *d_step_log)
+{
+    const size_t need = round_scratch_need(ctx->space, J, N);
+    if (need > ctx->round_scratch_bytes) {
+        if (ctx->d_round_scratch) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_round_scratch); ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0; }
+        CUDA_TRY(ctx, cudaMalloc(&ctx->d_round_scratch, need), "cudaMalloc (round scratch)");
+        ctx->round_scratch_bytes = need;
+    }
+    CUDA_TRY(ctx, launch_round(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
+                               ctx->d_round_scratch, ctx->d_status, ctx->d_steps, ctx->stream),
+             "launch greedy_round");
+    return RUBICK_OK;
+}
+
+// wait for the round, fetch the step count and the cap flag
+static int finish_round(rubick_ctx *ctx, int32_t *h_steps)
+{
+    uint32_t two[2] = {0, 0};
+    CUDA_TRY(ctx, cudaMemcpyAsync(two, ctx->d_status, 8, cudaMemcpyDeviceToHost, ctx->stream), "read round status");
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
+    if (h_steps) *h_steps = int32_t(two[1]);
+    if (two[0] & DS_STEP_CAP) {
+        const uint32_t cleared = two[0] & ~DS_STEP_CAP;
+        cudaMemcpyAsync(ctx->d_status, &cleared, 4, cudaMemcpyHostToDevice, ctx->stream);
+        cudaStreamSynchronize(ctx->stream);
+        return fail(ctx, RUBICK_ESTEPS, "greedy round stopped at max_steps");
+    }
+    if (two[0] & DS_FEAS_NOT_THRESHOLD) {
+        cudaMemset(ctx->d_status, 0, 4);
+        return fail(ctx, RUBICK_ESTATE, "a feasibility word is not a threshold in the memory-level index");
+    }
+    return RUBICK_OK;
+}
+
+static int check_round_args(rubick_ctx *ctx, int J, const rubick_cluster *h_cluster, int max_steps)
+{
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (!h_cluster || h_cluster->n_nodes < 1 || h_cluster->n_nodes > RUBICK_MAX_NODES) return fail(ctx, RUBICK_EINVAL, "cluster: 1 .. RUBICK_MAX_NODES nodes");
+    if (max_steps < 0) return fail(ctx, RUBICK_EINVAL, "negative max_steps");
+    if (J >= (1 << 29)) return fail(ctx, RUBICK_EINVAL, "too many jobs");
+    return RUBICK_OK;
+}
+
+int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                        const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
+                        const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
+                        rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                        int32_t *h_steps)
+{
+    CHECK_CTX(ctx);
+    int rc = check_round_args(ctx, J, h_cluster, max_steps);
+    if (rc) return rc;
+    if (J > 0 && (!d_jobs || !d_curve_val || !d_curve_plan || !d_curve_g || !d_feas || !d_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    rc = enqueue_round(ctx, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, h_cluster->n_nodes, max_steps, d_out,
+                       d_node_out, d_step_log);
+    if (rc) return rc;
+    return finish_round(ctx, h_steps);
+}
+
+// candidate table, mask and curves for d_jobs[0..J) into context scratch, in job tiles whose
+// throughput rows are produced and consumed back to back
+static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
+{
+    const Space &sp = ctx->space;
+    const int tile = ctx->tile_jobs < J ? ctx->tile_jobs : J;
+    int rc;
+    if ((rc = ensure(ctx, ctx->d_thr, ctx->cap_thr, size_t(tile) * sp.nC * sp.P))) return rc;
+    if ((rc = ensure(ctx, ctx->d_feas, ctx->cap_feas, size_t(J) * sp.P))) return rc;
+    const size_t curve = size_t(J) * sp.nG * sp.nC * sp.nM;
+    if (curve > ctx->cap_curve) {
+        size_t c1 = ctx->cap_curve, c2 = ctx->cap_curve, c3 = ctx->cap_curve;
+        if ((rc = ensure(ctx, ctx->d_cv, c1, curve))) return rc;
+        if ((rc = ensure(ctx, ctx->d_cp, c2, curve))) return rc;
+        if ((rc = ensure(ctx, ctx->d_cg, c3, curve))) return rc;
+        ctx->cap_curve = curve;
+    }
+    const size_t per_job = size_t(sp.nG) * sp.nC * sp.nM;
+    for (int j0 = 0; j0 < J; j0 += tile) {
+        const int n = J - j0 < tile ? J - j0 : tile;
+        CUDA_TRY(ctx, launch_eval(sp, ctx->d_quads, d_jobs + j0, n, ctx->d_thr, ctx->d_feas + size_t(j0) * sp.P, ctx->stream), "launch eval_candidates");
+        CUDA_TRY(ctx, launch_best(sp, ctx->d_thr, ctx->d_feas + size_t(j0) * sp.P, n, 0u, ctx->d_cv + j0 * per_job,
+                                  ctx->d_cp + j0 * per_job, ctx->d_cg + j0 * per_job, ctx->d_status, ctx->stream),
+                 "launch best_plan");
+    }
+    return RUBICK_OK;
+}
+
+int rubick_schedule_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const rubick_cluster *h_cluster,
+                          int max_steps, rubick_assignment *d_out, rubick_node *d_node_out, int32_t *h_steps)
+{
+    CHECK_CTX(ctx);
+    int rc = check_round_args(ctx, J, h_cluster, max_steps);
+    if (rc) return rc;
+    if (J > 0 && (!d_jobs || !d_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if (J > 0 && (reinterpret_cast<uintptr_t>(d_jobs) & 15)) return fail(ctx, RUBICK_EINVAL, "d_jobs must be 16-byte aligned");
+    if ((rc = enqueue_tables(ctx, d_jobs, J))) return rc;
+    if ((rc = enqueue_round(ctx, d_jobs, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster->n_nodes, max_steps, d_out, d_node_out, nullptr))) return rc;
+    return finish_round(ctx, h_steps);
+}
+
+int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J, const rubick_cluster *h_cluster,
+                               int max_steps, rubick_assignment *h_out, rubick_node *h_node_out, int32_t *h_steps)
+{
+    CHECK_CTX(ctx);
+    int rc = check_round_args(ctx, J, h_cluster, max_steps);
+    if (rc) return rc;
+    if (J > 0 && (!h_jobs || !h_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    const int N = h_cluster->n_nodes;
+    if ((rc = ensure(ctx, ctx->d_jobs_stage, ctx->cap_jobs, size_t(J > 0 ? J : 1)))) return rc;
+    if ((rc = ensure(ctx, ctx->d_out_stage, ctx->cap_out, size_t(J > 0 ? J : 1)))) return rc;
+    if ((rc = ensure(ctx, ctx->d_node_stage, ctx->cap_node, size_t(N)))) return rc;
+    if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_jobs_stage, h_jobs, size_t(J) * sizeof(rubick_job), cudaMemcpyHostToDevice, ctx->stream), "copy jobs to device");
+    if ((rc = enqueue_tables(ctx, ctx->d_jobs_stage, J))) return rc;
+    if ((rc = enqueue_round(ctx, ctx->d_jobs_stage, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, N, max_steps, ctx->d_out_stage,
+                            ctx->d_node_stage, nullptr))) return rc;
+    if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_out_stage, size_t(J) * sizeof(rubick_assignment), cudaMemcpyDeviceToHost, ctx->stream), "copy assignments to host");
+    if (h_node_out) CUDA_TRY(ctx, cudaMemcpyAsync(h_node_out, ctx->d_node_stage, size_t(N) * sizeof(rubick_node), cudaMemcpyDeviceToHost, ctx->stream), "copy node states to host");
+    return finish_round(ctx, h_steps);
+}
+
+}  // extern "C"

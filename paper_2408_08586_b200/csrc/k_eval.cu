@@ -1,0 +1,224 @@
+// Candidate-grid evaluation: predicted throughput for every (job, plan, CPU level) and the
+// memory-feasibility word for every (job, plan).
+//
+// Mapping.  Plans come in quads: four consecutive plan indices share (d, t, p, ZeRO stage) and
+// differ in (gradient checkpointing, offload) = (0,0), (0,1), (1,0), (1,1).  One thread owns one
+// (job, quad): it reads the 128-byte job record once, computes everything that does not depend
+// on the CPU level once (forward / backward time, the three communication times, T_cc, the
+// non-offload optimizer time, the offload transfer time and its overlap with the gradient
+// ring), then walks the CPU levels and stores one float4 per level.  Consecutive threads own
+// consecutive quads, so a warp writes 512 contiguous bytes per level: the kernel is a pure
+// write stream of 4 bytes per candidate plus 4 / C bytes of mask.
+//
+// Model (paper Section 4):  THROUGHPUT = b / T_iter,  T_iter = T_cc + T_oo + k_const  (Eq. 1)
+//   T_fwd  = tau * mu / (t p) * (m + p - 1 if p > 1)                       forward, pipeline bubble
+//   T_bwd  = k_bwd T_fwd (+ T_fwd under gradient checkpointing)
+//   T_comm = V / B per dimension, V = 0 at degree 1;  V_dp ring all-reduce of the shard,
+//            V_tp four all-reduces per layer, V_pp stage boundaries of 1F1B
+//   T_cc   = a T_fwd + (a - 1) T_bwd + f^{k_sync}(T_bwd, T_dp) + T_tp + T_pp
+//   T_oo   = T_opt, or under ZeRO-Offload f^{k_off}(T_dp, T_off) + f^{k_swap}(T_opt(c), T_off)
+//   f^k(x, y) = (x^k + y^k)^(1/k)                                           (Section 4.3)
+// Arithmetic is single precision.  f^k is evaluated as M (1 + (m/M)^k)^(1/k) with M = max and
+// m = min, so that no power can overflow and the hardware log2 / exp2 approximations act on
+// arguments where their absolute error stays below 1e-6 relative to the result.
+//
+// Feasibility (integer bytes, exact): mixed-precision Adam model states (2 + 2 + 12 bytes per
+// shard parameter, ZeRO stage 1 / 2 / 3 dividing optimizer / + gradients / + parameters by d,
+// offload moving gradients and optimizer states to the host), activations of one stage's layers
+// for the micro-batches in flight, against the GPU memory; host need g * host_base (+ 14 P under
+// offload) against each host-memory level and its per-node share against the node.
+
+#include "rubick_internal.cuh"
+
+namespace rubick {
+
+__device__ __forceinline__ float lg2_approx(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// 2^-n for 0 <= n < 127, exact
+__device__ __forceinline__ float pow2_neg(int n) { return __int_as_float((127 - n) << 23); }
+
+// f^k(x, y) for x, y >= 0 with inv_k = 1 / k
+__device__ __forceinline__ float overlap(float k, float inv_k, float x, float y)
+{
+    float hi = fmaxf(x, y), lo = fminf(x, y);
+    if (lo == 0.0f) return hi;
+    float r = lo * rcp_approx(hi);               // in (0, 1]
+    float u = ex2_approx(k * lg2_approx(r));     // r^k in [0, 1]
+    return hi * ex2_approx(inv_k * lg2_approx(1.0f + u));
+}
+
+__device__ __forceinline__ int64_t cdiv_shift(int64_t x, int s) { return (x + ((int64_t(1) << s) - 1)) >> s; }
+
+struct JobRegs {
+    double P; int64_t host_base;
+    int32_t l, h, s, b, mu_cap, alpha;
+    float tau, k_bwd, k_sync, k_opt, k_opt_off, k_off, k_swap, k_const;
+};
+
+__device__ __forceinline__ JobRegs load_job(const rubick_job *jp)
+{
+    const int4 *v = reinterpret_cast<const int4 *>(jp);
+    int4 a = __ldg(v + 0), b = __ldg(v + 1), c = __ldg(v + 2), d = __ldg(v + 3), e = __ldg(v + 4);
+    JobRegs r;
+    r.P = __hiloint2double(a.y, a.x);
+    r.host_base = (int64_t(uint32_t(a.w)) << 32) | uint32_t(a.z);
+    r.l = b.x; r.h = b.y; r.s = b.z; r.b = b.w;
+    r.mu_cap = c.x; r.alpha = c.y; r.tau = __int_as_float(c.z); r.k_bwd = __int_as_float(c.w);
+    r.k_sync = __int_as_float(d.x); r.k_opt = __int_as_float(d.y); r.k_opt_off = __int_as_float(d.z);
+    r.k_off = __int_as_float(d.w);
+    r.k_swap = __int_as_float(e.x); r.k_const = __int_as_float(e.y);
+    return r;
+}
+
+// first level index whose value is >= need (nM if none); levels strictly increasing
+__device__ __forceinline__ int first_level(const Space &sp, int64_t need)
+{
+    int lo = 0, hi = sp.nM;
+    while (lo < hi) {
+        int mid = (lo + hi) >> 1;
+        if (sp.m_levels[mid] >= need) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
+__global__ void __launch_bounds__(256)
+eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads,
+                       const rubick_job *__restrict__ jobs, int J, float *__restrict__ thr,
+                       uint32_t *__restrict__ feas)
+{
+    // J * Q < 2^31 is checked by the host entry point
+    const uint32_t gid = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= uint32_t(J) * uint32_t(sp.Q)) return;
+    const int j = int(gid / uint32_t(sp.Q));
+    const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
+
+    const JobRegs jb = load_job(jobs + j);
+    const uint2 qraw = __ldg(reinterpret_cast<const uint2 *>(quads) + q);
+    const int ld = qraw.x & 0xff, lt = (qraw.x >> 8) & 0xff, lp = (qraw.x >> 16) & 0xff, z = (qraw.x >> 24) & 0xff;
+    const int qflags = (qraw.y >> 8) & 0xff, disabled = (qraw.y >> 16) & 0xff;
+    const int lg = ld + lt + lp;
+    const int d = 1 << ld, t = 1 << lt, p = 1 << lp;
+
+    // structural validity of the (d, t, p, z) part; offload additionally needs ZeRO stage >= 2
+    bool valid = (qflags & QF_T_FITS_NODE) && p <= jb.l && d <= jb.b && (jb.b & (d - 1)) == 0
+                 && (jb.h & (t - 1)) == 0 && !(sp.strict && z > 0 && (lt + lp) > 0);
+    const bool valid_off = valid && z >= 2;
+
+    // micro-batching
+    const int r = max(jb.b >> ld, 1);
+    const int mu = min(r, max(jb.mu_cap, 1));
+    const int n = (r + mu - 1) / mu;
+    const int m = p > 1 ? n : 1;
+    const int a = p > 1 ? 1 : n;
+
+    // ---- times that do not depend on the CPU level -------------------------------------------
+    const float inv_tp = pow2_neg(lt + lp);
+    float T_fwd = jb.tau * float(mu) * inv_tp;
+    if (p > 1) T_fwd *= float(n + p - 1);
+    const float T_bwd0 = jb.k_bwd * T_fwd;
+    const float T_bwd1 = T_bwd0 + T_fwd;
+
+    const float Pf = float(jb.P);
+    const float bsh = float(int64_t(jb.b) * jb.s * jb.h);
+    float T_dp = 0.0f, T_tp = 0.0f, T_pp = 0.0f;
+    if (d > 1) {
+        float V = sp.e * Pf * (float(d - 1) * pow2_neg(lg - 1));
+        if (z == 3) V *= 1.5f;
+        T_dp = V * ((qflags & QF_DP_INTER) ? sp.inv_B_inter : sp.inv_B_intra);
+    }
+    if (t > 1) T_tp = sp.e * 8.0f * float(t - 1) * bsh * float(jb.l) * pow2_neg(ld + lt) * sp.inv_B_intra;
+    if (p > 1) T_pp = sp.e * 2.0f * float(p) * bsh * pow2_neg(ld + lt) * ((qflags & QF_PP_INTER) ? sp.inv_B_inter : sp.inv_B_intra);
+
+    const float inv_ksync = 1.0f / jb.k_sync;
+    const float af = float(a);
+    const float fixed = af * T_fwd + T_tp + T_pp + jb.k_const;
+    const float cc0 = fixed + (af - 1.0f) * T_bwd0 + overlap(jb.k_sync, inv_ksync, T_bwd0, T_dp);
+    const float cc1 = fixed + (af - 1.0f) * T_bwd1 + overlap(jb.k_sync, inv_ksync, T_bwd1, T_dp);
+
+    const float Psi = Pf * inv_tp;
+    const float inv_d = pow2_neg(ld);
+    const float T_opt = jb.k_opt * Psi * (z >= 1 ? inv_d : 1.0f);
+    const float bf = float(jb.b);
+
+    float4 out;
+    out.x = (valid && !(disabled & 1)) ? bf / (cc0 + T_opt) : 0.0f;
+    out.z = (valid && !(disabled & 4)) ? bf / (cc1 + T_opt) : 0.0f;
+    out.y = 0.0f;
+    out.w = 0.0f;
+
+    // ---- feasibility words ---------------------------------------------------------------------
+    {
+        const int64_t Pi = int64_t(jb.P);
+        const int64_t Psi_i = cdiv_shift(Pi, lt + lp);
+        const int64_t params = 2 * cdiv_shift(Psi_i, z == 3 ? ld : 0);
+        const int64_t grads = 2 * cdiv_shift(Psi_i, z >= 2 ? ld : 0);
+        const int64_t opt = 12 * cdiv_shift(Psi_i, z >= 1 ? ld : 0);
+        const int64_t smh = int64_t(jb.s) * mu * jb.h;
+        const int64_t A = cdiv_shift(int64_t(jb.alpha) * smh, lt);
+        const int64_t Lq = cdiv_shift(jb.l, lp) * (p > 1 ? min(m, p) : 1);
+        const int64_t act0 = Lq * A;
+        const int64_t act1 = Lq * 2 * smh + A;
+        const int64_t st0 = params + grads + opt, st1 = params;
+        const int64_t need0 = jb.host_base << lg;
+        const int64_t need1 = need0 + 14 * Pi;
+        const int nshift = max(lg - sp.log2Gn, 0);
+        const uint32_t full = sp.nM >= 32 ? 0xffffffffu : ((1u << sp.nM) - 1u);
+        uint32_t w0 = 0u, w1 = 0u;
+        if (cdiv_shift(need0, nshift) <= sp.Mn) { int f = first_level(sp, need0); if (f < sp.nM) w0 = (full << f) & full; }
+        if (cdiv_shift(need1, nshift) <= sp.Mn) { int f = first_level(sp, need1); if (f < sp.nM) w1 = (full << f) & full; }
+        uint4 fw;
+        fw.x = (valid && !(disabled & 1) && st0 + act0 <= sp.gpu_mem) ? w0 : 0u;
+        fw.y = (valid_off && !(disabled & 2) && st1 + act0 <= sp.gpu_mem) ? w1 : 0u;
+        fw.z = (valid && !(disabled & 4) && st0 + act1 <= sp.gpu_mem) ? w0 : 0u;
+        fw.w = (valid_off && !(disabled & 8) && st1 + act1 <= sp.gpu_mem) ? w1 : 0u;
+        *reinterpret_cast<uint4 *>(feas + (size_t(j) * sp.P + 4 * size_t(q))) = fw;
+    }
+
+    // ---- walk the CPU levels -------------------------------------------------------------------
+    float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
+    const bool off0 = valid_off && !(disabled & 2), off1 = valid_off && !(disabled & 8);
+    if (!(off0 || off1)) {
+        for (int ci = 0; ci < sp.nC; ++ci, row += sp.P) __stcs(reinterpret_cast<float4 *>(row), out);
+    } else {
+        const float T_off = sp.e * Psi * inv_d * sp.inv_B_pcie;
+        const float inv_kswap = 1.0f / jb.k_swap;
+        const float f_off = overlap(jb.k_off, 1.0f / jb.k_off, T_dp, T_off);
+        const float base0 = cc0 + f_off, base1 = cc1 + f_off;
+        const float opt_c = jb.k_opt_off * Psi * inv_d;      // times 1 / c
+        for (int ci = 0; ci < sp.nC; ++ci, row += sp.P) {
+            const float f_swap = overlap(jb.k_swap, inv_kswap, opt_c * sp.inv_c[ci], T_off);
+            out.y = off0 ? bf / (base0 + f_swap) : 0.0f;
+            out.w = off1 ? bf / (base1 + f_swap) : 0.0f;
+            __stcs(reinterpret_cast<float4 *>(row), out);
+        }
+    }
+}
+
+cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J,
+                        float *d_thr, uint32_t *d_feas, cudaStream_t st)
+{
+    if (J == 0) return cudaSuccess;
+    const int64_t total = int64_t(J) * sp.Q;
+    const int block = 256;
+    const int64_t grid = (total + block - 1) / block;
+    eval_candidates_kernel<<<unsigned(grid), block, 0, st>>>(sp, d_quads, d_jobs, J, d_thr, d_feas);
+    return cudaGetLastError();
+}
+
+}  // namespace rubick

@@ -1,0 +1,503 @@
+// Marginal gains and the greedy scheduling round (paper Section 5.2, Algorithm 1 in
+// marginal-gain form).
+//
+// Gain ("slope") of a job = weighted curve gain per unit of added resource: for GPUs up to the
+// smallest level whose curve value strictly exceeds what the job has now, for CPU cores up to
+// the next core level, both read at the top host-memory level (memory is not searched, it is
+// allocated once the plan is known).  Gains are computed in single precision with one rounding
+// per operation (__fmul_rn / __fsub_rn / __fdiv_rn, never fused), so that any other
+// implementation of the same arithmetic reaches bit-identical decisions.
+//
+// The round is inherently sequential (every commit changes node capacities and one job's
+// gains), so it runs as ONE persistent CTA that keeps the cluster state and the per-job scan
+// state in shared memory and never returns to the host between increments:
+//   per step:  (1) all warps rebuild the first-fit table  node(g level, c level)  and the count of
+//                  empty nodes;
+//              (2) all threads scan their jobs: a candidate counts only if it can be placed;
+//              (3) block-wide argmax on a 64-bit key (gain bits << 32 | ~job), GPU gains before
+//                  CPU gains;
+//              (4) warp 0 commits the winner: placement, host-memory level, curve lookup
+//                  (GetBestPlan), memory of that plan (AllocMem), node bookkeeping, new gains.
+// The step count is bounded by max_steps; hitting it sets a status bit instead of spinning.
+
+#include "rubick_internal.cuh"
+
+namespace rubick {
+
+constexpr int ROUND_THREADS = 1024;
+constexpr int ROUND_WARPS = ROUND_THREADS / 32;
+
+// scan state of one job (16 bytes)
+struct HotA {
+    float gain_g, gain_c;     // 0 = no candidate
+    uint32_t packed;          // see pack()
+    int32_t node;             // node of a single-node job, lowest node of a multi-node job, -1 if none
+};
+// the rest of a job's state (16 bytes)
+struct HotB {
+    float val;                // predicted throughput of the present allocation
+    int32_t plan;
+    int32_t f_level;          // host-memory level allocated (first feasible level of the plan)
+    float w;
+};
+
+// packed: [5:0] present g level + 1 (0 = nothing held) | [12:6] c level (present, or where an
+// unallocated job would start) | [18:13] target g level + 1 (0 = none) | [19] pending |
+// [20] GPU increments frozen | [21] CPU increments frozen
+__device__ __forceinline__ uint32_t pack(int gi, int ci, int next_gi, bool pending, bool fz_g, bool fz_c)
+{
+    return uint32_t(gi + 1) | (uint32_t(ci) << 6) | (uint32_t(next_gi + 1) << 13) | (uint32_t(pending) << 19)
+           | (uint32_t(fz_g) << 20) | (uint32_t(fz_c) << 21);
+}
+__device__ __forceinline__ int pk_gi(uint32_t p) { return int(p & 63u) - 1; }
+__device__ __forceinline__ int pk_ci(uint32_t p) { return int((p >> 6) & 127u); }
+__device__ __forceinline__ int pk_next_gi(uint32_t p) { return int((p >> 13) & 63u) - 1; }
+__device__ __forceinline__ bool pk_pending(uint32_t p) { return (p >> 19) & 1u; }
+__device__ __forceinline__ bool pk_fz_g(uint32_t p) { return (p >> 20) & 1u; }
+__device__ __forceinline__ bool pk_fz_c(uint32_t p) { return (p >> 21) & 1u; }
+
+__device__ __forceinline__ size_t curve_idx(const Space &sp, int j, int gi, int ci, int mi)
+{
+    return ((size_t(j) * sp.nG + gi) * sp.nC + ci) * sp.nM + mi;
+}
+
+struct Gains { int next_g, next_c; float gain_g, gain_c; };
+
+// One thread computes the gains of one job from the curve table.
+__device__ Gains job_gains(const Space &sp, const float *__restrict__ cv, int j, float w, int gi, int ci, float val)
+{
+    Gains r; r.next_g = -1; r.next_c = -1; r.gain_g = 0.0f; r.gain_c = 0.0f;
+    const int mt = sp.nM - 1;
+    const bool alloc = gi >= 0;
+    const float cur = alloc ? val : 0.0f;
+    const float vcur = alloc ? __fmul_rn(w, cur) : 0.0f;
+    for (int g2 = gi + 1; g2 < sp.nG; ++g2) {
+        const float v = cv[curve_idx(sp, j, g2, ci, mt)];
+        if (v > cur) {
+            const float dg = float(sp.g_levels[g2] - (alloc ? sp.g_levels[gi] : 0));
+            r.next_g = g2;
+            r.gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, v), vcur), dg);
+            break;
+        }
+    }
+    if (alloc && ci + 1 < sp.nC) {
+        const float v = cv[curve_idx(sp, j, gi, ci + 1, mt)];
+        const float dc = float(sp.c_levels[ci + 1] - sp.c_levels[ci]);
+        const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(w, v), vcur), dc);
+        if (gn > 0.0f) { r.next_c = ci + 1; r.gain_c = gn; }
+    }
+    return r;
+}
+
+__device__ __forceinline__ int level_of_g(const Space &sp, int g)
+{
+    for (int i = 0; i < sp.nG; ++i) if (sp.g_levels[i] == g) return i;
+    return -1;
+}
+__device__ __forceinline__ int level_of_c(const Space &sp, int c)
+{
+    for (int i = 0; i < sp.nC; ++i) if (sp.c_levels[i] == c) return i;
+    return -1;
+}
+
+__global__ void marginal_gain_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
+                                     const float *__restrict__ cv, const rubick_assignment *__restrict__ state,
+                                     float *__restrict__ gain_gpu, float *__restrict__ gain_cpu,
+                                     int32_t *__restrict__ next_g, int32_t *__restrict__ next_c)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= J) return;
+    const rubick_assignment s = state[j];
+    int gi = -1, ci = jobs[j].cmin_idx > 0 ? jobs[j].cmin_idx : 0;
+    if (s.g > 0) { gi = level_of_g(sp, s.g); ci = level_of_c(sp, s.c); }
+    Gains r;
+    if (s.g > 0 && (gi < 0 || ci < 0)) { r.next_g = r.next_c = -1; r.gain_g = r.gain_c = 0.0f; }   // not on the grid
+    else r = job_gains(sp, cv, j, jobs[j].w, gi, min(ci, sp.nC - 1), s.thr);
+    gain_gpu[j] = r.gain_g; gain_cpu[j] = r.gain_c; next_g[j] = r.next_g; next_c[j] = r.next_c;
+}
+
+cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const float *d_curve_val,
+                        const rubick_assignment *d_state, float *d_gain_gpu, float *d_gain_cpu,
+                        int32_t *d_next_g, int32_t *d_next_c, cudaStream_t st)
+{
+    if (J == 0) return cudaSuccess;
+    marginal_gain_kernel<<<(J + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, d_curve_val, d_state, d_gain_gpu,
+                                                         d_gain_cpu, d_next_g, d_next_c);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
+// greedy round
+// ------------------------------------------------------------------------------------------------
+
+struct Cluster {           // views into shared memory
+    int32_t *free_g, *free_c, *owner;
+    int64_t *free_m;
+    int32_t *ff;           // [n_small][nC] first node that fits the whole job, -1 if none
+    int N;
+};
+
+__device__ __forceinline__ int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Can (g level gi2, c level ci2) be placed for a job that holds (gi, ci) on `node`?
+__device__ __forceinline__ bool placeable(const Space &sp, const Cluster &cl, int n_empty, int gi, int ci, int node,
+                                          int gi2, int ci2)
+{
+    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    const bool alloc = gi >= 0;
+    const int g = alloc ? sp.g_levels[gi] : 0, c = alloc ? sp.c_levels[ci] : 0;
+    if (g2 <= sp.Gn) {
+        if (alloc && cl.free_g[node] >= g2 - g && cl.free_c[node] >= c2 - c) return true;
+        return cl.ff[gi2 * sp.nC + ci2] >= 0;
+    }
+    const int k2 = g2 >> sp.log2Gn;
+    if ((c2 + k2 - 1) / k2 > sp.Cn) return false;
+    if (alloc && g >= sp.Gn) { const int k = g >> sp.log2Gn; return n_empty >= k2 - k; }
+    const int empty = n_empty + ((alloc && cl.free_g[node] + g == sp.Gn) ? 1 : 0);
+    return empty >= k2;
+}
+
+// warp-cooperative: first node with at least g free GPUs and c free cores, -1 if none
+__device__ int first_fit_warp(const Cluster &cl, int g, int c, int lane)
+{
+    for (int base = 0; base < cl.N; base += 32) {
+        const int n = base + lane;
+        const bool ok = n < cl.N && cl.free_g[n] >= g && cl.free_c[n] >= c;
+        const unsigned b = __ballot_sync(0xffffffffu, ok);
+        if (b) return base + __ffs(b) - 1;
+    }
+    return -1;
+}
+
+struct RoundShared {
+    unsigned long long red[2][ROUND_WARPS];
+    int n_empty;
+    int sel_j, sel_type;
+    int steps, capped;
+};
+
+// Commit job j to (gi2, ci2); executed by warp 0 (all lanes).  Returns true when the allocation
+// was made.  need_gain: the new value must strictly exceed the present one.
+__device__ bool commit_warp(const Space &sp, Cluster &cl, int n_empty, const float *__restrict__ cv,
+                            const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
+                            const uint32_t *__restrict__ feas, int j, HotA &ha, HotB &hb, int gi2, int ci2,
+                            bool need_gain, int lane)
+{
+    const int gi = pk_gi(ha.packed), ci = pk_ci(ha.packed);
+    const bool alloc = gi >= 0;
+    const int g = alloc ? sp.g_levels[gi] : 0, c = alloc ? sp.c_levels[ci] : 0;
+    const int64_t m_cur = alloc ? sp.m_levels[hb.f_level] : 0;
+    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    const int k = alloc ? max(g >> sp.log2Gn, 1) : 0;
+
+    // ---- placement -----------------------------------------------------------------------------
+    int k2 = 1, target = -1, need_new = 0;
+    bool stay = false;
+    if (g2 <= sp.Gn) {
+        if (alloc && cl.free_g[ha.node] >= g2 - g && cl.free_c[ha.node] >= c2 - c) { stay = true; target = ha.node; }
+        else target = first_fit_warp(cl, g2, c2, lane);
+        if (target < 0) return false;
+    } else {
+        k2 = g2 >> sp.log2Gn;
+        if ((c2 + k2 - 1) / k2 > sp.Cn) return false;
+        if (alloc && g >= sp.Gn) { stay = true; need_new = k2 - k; if (n_empty < need_new) return false; }
+        else {
+            need_new = k2;
+            const int empty = n_empty + ((alloc && cl.free_g[ha.node] + g == sp.Gn) ? 1 : 0);
+            if (empty < need_new) return false;
+        }
+    }
+
+    // ---- host-memory level that fits the target, curve lookup, memory of the plan ---------------
+    const int64_t avail = k2 > 1 ? sp.Mn : cl.free_m[target] + ((stay && alloc) ? m_cur : 0);
+    const bool fits = lane < sp.nM && cdiv64(sp.m_levels[lane < sp.nM ? lane : 0], k2) <= avail;
+    const unsigned fb = __ballot_sync(0xffffffffu, fits);
+    if (!fb) return false;
+    const int mi = 31 - __clz(fb);
+    const size_t o = curve_idx(sp, j, gi2, ci2, mi);
+    const float v = __ldg(cv + o);
+    const int plan = __ldg(cp + o), gu = __ldg(cg + o);
+    if (plan < 0 || !(v > 0.0f) || gu != g2) return false;
+    if (need_gain && alloc && !(v > hb.val)) return false;
+    const uint32_t word = __ldg(feas + size_t(j) * sp.P + plan);
+    const int f = __ffs(word) - 1;
+    if (f < 0 || f > mi) return false;
+    const int64_t m2 = sp.m_levels[f];
+
+    // ---- node bookkeeping ------------------------------------------------------------------------
+    int first = -1;
+    if (k2 == 1) {
+        if (lane == 0) {
+            if (alloc) { cl.free_g[ha.node] += g; cl.free_c[ha.node] += c; cl.free_m[ha.node] += m_cur; }
+            cl.free_g[target] -= g2; cl.free_c[target] -= c2; cl.free_m[target] -= m2;
+        }
+        first = target;
+    } else {
+        const int cs2 = (c2 + k2 - 1) / k2;
+        const int64_t ms2 = cdiv64(m2, k2);
+        if (stay) {
+            // whole nodes already held keep their GPUs; only the core / memory shares change
+            const int cs1 = (c + k - 1) / k;
+            const int64_t ms1 = cdiv64(m_cur, k);
+            if (k == 1) {
+                if (lane == 0) { cl.free_c[ha.node] += c - cs2; cl.free_m[ha.node] += m_cur - ms2; cl.owner[ha.node] = j; }
+            } else {
+                for (int n = lane; n < cl.N; n += 32)
+                    if (cl.owner[n] == j) { cl.free_c[n] += cs1 - cs2; cl.free_m[n] += ms1 - ms2; }
+            }
+            first = ha.node;
+        } else if (alloc && lane == 0) {
+            cl.free_g[ha.node] += g; cl.free_c[ha.node] += c; cl.free_m[ha.node] += m_cur;
+        }
+        __syncwarp();
+        int taken = 0;
+        for (int base = 0; base < cl.N && taken < need_new; base += 32) {
+            const int n = base + lane;
+            const bool empty = n < cl.N && cl.free_g[n] == sp.Gn;
+            const unsigned b = __ballot_sync(0xffffffffu, empty);
+            const int rank = __popc(b & ((1u << lane) - 1u));
+            if (empty && taken + rank < need_new) {
+                cl.free_g[n] = 0; cl.free_c[n] -= cs2; cl.free_m[n] -= ms2; cl.owner[n] = j;
+            }
+            if (b) { const int lowest = base + __ffs(b) - 1; if (first < 0 || lowest < first) first = lowest; }
+            taken += __popc(b);
+        }
+    }
+    __syncwarp();
+    ha.node = first;
+    ha.packed = pack(gi2, ci2, -1, false, pk_fz_g(ha.packed), pk_fz_c(ha.packed));
+    hb.val = v; hb.plan = plan; hb.f_level = f;
+    return true;
+}
+
+__global__ void __launch_bounds__(ROUND_THREADS, 1)
+greedy_round_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
+                    const float *__restrict__ cv, const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
+                    const uint32_t *__restrict__ feas, int N, int max_steps, rubick_assignment *__restrict__ out,
+                    rubick_node *__restrict__ node_out, int32_t *__restrict__ step_log, HotA *hotA_g, HotB *hotB_g,
+                    int hot_in_smem, uint32_t *__restrict__ status, int32_t *__restrict__ steps_out)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ RoundShared sh;
+
+    // shared layout: free_m [N] i64 | free_g [N] | free_c [N] | owner [N] | ff [n_small * nC] | hot arrays
+    Cluster cl;
+    cl.N = N;
+    cl.free_m = reinterpret_cast<int64_t *>(smem_raw);
+    cl.free_g = reinterpret_cast<int32_t *>(cl.free_m + N);
+    cl.free_c = cl.free_g + N;
+    cl.owner = cl.free_c + N;
+    cl.ff = cl.owner + N;
+    const int n_ff = sp.n_small * sp.nC;
+    size_t off = size_t(N) * 20 + size_t(n_ff) * 4;
+    off = (off + 15) & ~size_t(15);
+    HotA *hotA = hot_in_smem ? reinterpret_cast<HotA *>(smem_raw + off) : hotA_g;
+    HotB *hotB = hot_in_smem ? reinterpret_cast<HotB *>(smem_raw + off + size_t(J) * sizeof(HotA)) : hotB_g;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int mt = sp.nM - 1;
+
+    for (int n = tid; n < N; n += ROUND_THREADS) {
+        cl.free_g[n] = sp.Gn; cl.free_c[n] = sp.Cn; cl.free_m[n] = sp.Mn; cl.owner[n] = -1;
+    }
+    for (int j = tid; j < J; j += ROUND_THREADS) {
+        const rubick_job *jb = jobs + j;
+        const int gmin = jb->gmin_idx;
+        const int c0 = min(max(jb->cmin_idx, 0), sp.nC - 1);
+        HotA a; a.gain_g = 0.0f; a.gain_c = 0.0f; a.node = -1;
+        a.packed = pack(-1, c0, -1, gmin >= 0, false, false);
+        HotB b; b.val = 0.0f; b.plan = -1; b.f_level = -1; b.w = jb->w;
+        hotA[j] = a; hotB[j] = b;
+    }
+    if (tid == 0) { sh.steps = 0; sh.capped = 0; sh.n_empty = N; }
+    __syncthreads();
+
+    // ---- Phase A: guaranteed minima, in job order (warp 0) ----------------------------------------
+    if (warp == 0) {
+        int n_empty = N;
+        for (int base = 0; base < J; base += 32) {
+            const int jj = base + lane;
+            const bool want = jj < J && pk_pending(hotA[jj].packed);
+            unsigned todo = __ballot_sync(0xffffffffu, want);
+            while (todo) {
+                const int j = base + __ffs(todo) - 1;
+                todo &= todo - 1;
+                const rubick_job *jb = jobs + j;
+                const int gmin = jb->gmin_idx, cmin = max(jb->cmin_idx, 0);
+                if (gmin >= sp.nG || cmin >= sp.nC) continue;
+                const size_t o = curve_idx(sp, j, gmin, cmin, mt);
+                if (__ldg(cp + o) < 0) continue;
+                // the curve may reach this value with fewer GPUs than the level offers
+                const int gi = level_of_g(sp, __ldg(cg + o));
+                if (gi < 0) continue;
+                HotA a = hotA[j]; HotB b = hotB[j];
+                if (commit_warp(sp, cl, n_empty, cv, cp, cg, feas, j, a, b, gi, cmin, false, lane)) {
+                    if (lane == 0) { hotA[j] = a; hotB[j] = b; }
+                    // recount empty nodes
+                    int cnt = 0;
+                    for (int nb = 0; nb < N; nb += 32) {
+                        const int n = nb + lane;
+                        cnt += __popc(__ballot_sync(0xffffffffu, n < N && cl.free_g[n] == sp.Gn));
+                    }
+                    n_empty = cnt;
+                }
+                __syncwarp();
+            }
+        }
+    }
+    __syncthreads();
+
+    // initial gains of every job that may still grow
+    for (int j = tid; j < J; j += ROUND_THREADS) {
+        HotA a = hotA[j];
+        if (pk_pending(a.packed)) continue;
+        const Gains r = job_gains(sp, cv, j, hotB[j].w, pk_gi(a.packed), pk_ci(a.packed), hotB[j].val);
+        a.gain_g = r.gain_g; a.gain_c = r.gain_c;
+        a.packed = pack(pk_gi(a.packed), pk_ci(a.packed), r.next_g, false, false, false);
+        hotA[j] = a;
+    }
+    __syncthreads();
+
+    // ---- Phase B: greedy increments -----------------------------------------------------------------
+    for (;;) {
+        // (1) first-fit table and empty-node count
+        for (int e = warp; e <= n_ff; e += ROUND_WARPS) {
+            if (e == n_ff) {
+                int cnt = 0;
+                for (int nb = 0; nb < N; nb += 32) {
+                    const int n = nb + lane;
+                    cnt += __popc(__ballot_sync(0xffffffffu, n < N && cl.free_g[n] == sp.Gn));
+                }
+                if (lane == 0) sh.n_empty = cnt;
+            } else {
+                const int gi = e / sp.nC, ci = e - gi * sp.nC;
+                const int n = first_fit_warp(cl, sp.g_levels[gi], sp.c_levels[ci], lane);
+                if (lane == 0) cl.ff[e] = n;
+            }
+        }
+        __syncthreads();
+
+        // (2) scan: best placeable GPU increment and best placeable CPU increment of my jobs
+        const int n_empty = sh.n_empty;
+        unsigned long long best_g = 0ull, best_c = 0ull;
+        for (int j = tid; j < J; j += ROUND_THREADS) {
+            const HotA a = hotA[j];
+            const unsigned long long kg = (static_cast<unsigned long long>(__float_as_uint(a.gain_g)) << 32) | (0xffffffffu - uint32_t(j));
+            const unsigned long long kc = (static_cast<unsigned long long>(__float_as_uint(a.gain_c)) << 32) | (0xffffffffu - uint32_t(j));
+            const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+            if (a.gain_g > 0.0f && kg > best_g && placeable(sp, cl, n_empty, gi, ci, a.node, pk_next_gi(a.packed), ci)) best_g = kg;
+            if (a.gain_c > 0.0f && kc > best_c && placeable(sp, cl, n_empty, gi, ci, a.node, gi, ci + 1)) best_c = kc;
+        }
+        // (3) block argmax
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) {
+            const unsigned long long og = __shfl_xor_sync(0xffffffffu, best_g, s);
+            const unsigned long long oc = __shfl_xor_sync(0xffffffffu, best_c, s);
+            best_g = og > best_g ? og : best_g;
+            best_c = oc > best_c ? oc : best_c;
+        }
+        if (lane == 0) { sh.red[0][warp] = best_g; sh.red[1][warp] = best_c; }
+        __syncthreads();
+        if (warp == 0) {
+            unsigned long long bg = sh.red[0][lane], bc = sh.red[1][lane];
+#pragma unroll
+            for (int s = 16; s > 0; s >>= 1) {
+                const unsigned long long og = __shfl_xor_sync(0xffffffffu, bg, s);
+                const unsigned long long oc = __shfl_xor_sync(0xffffffffu, bc, s);
+                bg = og > bg ? og : bg;
+                bc = oc > bc ? oc : bc;
+            }
+            int sel_j = -1, sel_type = -1;
+            if (bg) { sel_j = int(0xffffffffu - uint32_t(bg)); sel_type = 0; }
+            else if (bc) { sel_j = int(0xffffffffu - uint32_t(bc)); sel_type = 1; }
+            if (sel_j >= 0 && sh.steps >= max_steps) { if (lane == 0) sh.capped = 1; sel_j = -1; }
+
+            // (4) commit
+            if (sel_j >= 0) {
+                const int j = sel_j;
+                HotA a = hotA[j]; HotB b = hotB[j];
+                const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                const int gi2 = sel_type == 0 ? pk_next_gi(a.packed) : gi;
+                const int ci2 = sel_type == 0 ? ci : ci + 1;
+                const bool ok = commit_warp(sp, cl, n_empty, cv, cp, cg, feas, j, a, b, gi2, ci2, true, lane);
+                bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+                if (!ok) { if (sel_type == 0) fz_g = true; else fz_c = true; }
+                const Gains r = job_gains(sp, cv, j, b.w, pk_gi(a.packed), pk_ci(a.packed), b.val);
+                a.gain_g = fz_g ? 0.0f : r.gain_g;
+                a.gain_c = fz_c ? 0.0f : r.gain_c;
+                a.packed = pack(pk_gi(a.packed), pk_ci(a.packed), r.next_g, false, fz_g, fz_c);
+                if (lane == 0) {
+                    hotA[j] = a; hotB[j] = b;
+                    if (step_log) step_log[sh.steps] = (j << 2) | (sel_type << 1) | int(ok);
+                    sh.steps += 1;
+                }
+            }
+            if (lane == 0) sh.sel_j = sel_j;
+        }
+        __syncthreads();
+        if (sh.sel_j < 0) break;
+    }
+
+    // ---- results ------------------------------------------------------------------------------------
+    for (int j = tid; j < J; j += ROUND_THREADS) {
+        const HotA a = hotA[j]; const HotB b = hotB[j];
+        const int gi = pk_gi(a.packed);
+        rubick_assignment r;
+        if (gi >= 0) {
+            r.g = sp.g_levels[gi]; r.c = sp.c_levels[pk_ci(a.packed)]; r.m_bytes = sp.m_levels[b.f_level];
+            r.plan = b.plan; r.first_node = a.node; r.n_nodes = max(r.g >> sp.log2Gn, 1);
+            r.thr = b.val; r.status = RUBICK_RUNNING; r.m_level = b.f_level;
+        } else {
+            r.g = 0; r.c = 0; r.m_bytes = 0; r.plan = -1; r.first_node = -1; r.n_nodes = 0; r.thr = 0.0f;
+            r.status = pk_pending(a.packed) ? RUBICK_PENDING : RUBICK_UNALLOCATED; r.m_level = -1;
+        }
+        out[j] = r;
+    }
+    if (node_out)
+        for (int n = tid; n < N; n += ROUND_THREADS) {
+            rubick_node nd;
+            nd.free_g = cl.free_g[n]; nd.free_c = cl.free_c[n]; nd.free_m = cl.free_m[n]; nd.owner = cl.owner[n];
+            nd.reserved = 0;
+            node_out[n] = nd;
+        }
+    if (tid == 0) {
+        *steps_out = sh.steps;
+        if (sh.capped) atomicOr(status, DS_STEP_CAP);
+    }
+}
+
+static size_t round_fixed_smem(const Space &sp, int N)
+{
+    size_t off = size_t(N) * 20 + size_t(sp.n_small) * sp.nC * 4;
+    return (off + 15) & ~size_t(15);
+}
+constexpr size_t ROUND_SMEM_LIMIT = 200 * 1024;
+
+static bool hot_fits_smem(const Space &sp, int J, int N)
+{
+    return round_fixed_smem(sp, N) + size_t(J) * (sizeof(HotA) + sizeof(HotB)) <= ROUND_SMEM_LIMIT;
+}
+
+size_t round_scratch_need(const Space &sp, int J, int N)
+{
+    return hot_fits_smem(sp, J, N) ? 0 : size_t(J) * (sizeof(HotA) + sizeof(HotB));
+}
+
+cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
+                         const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
+                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                         void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
+{
+    const bool in_smem = hot_fits_smem(sp, J, N);
+    const size_t smem = round_fixed_smem(sp, N) + (in_smem ? size_t(J) * (sizeof(HotA) + sizeof(HotB)) : 0);
+    cudaError_t e = cudaFuncSetAttribute(greedy_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ROUND_SMEM_LIMIT));
+    if (e != cudaSuccess) return e;
+    HotA *ha = reinterpret_cast<HotA *>(d_scratch);
+    HotB *hb = reinterpret_cast<HotB *>(reinterpret_cast<unsigned char *>(d_scratch) + size_t(J) * sizeof(HotA));
+    greedy_round_kernel<<<1, ROUND_THREADS, smem, st>>>(sp, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out,
+                                                        d_node_out, d_step_log, ha, hb, in_smem ? 1 : 0, d_status,
+                                                        d_steps);
+    return cudaGetLastError();
+}
+
+}  // namespace rubick

@@ -1,0 +1,99 @@
+// Internal declarations shared by the translation units of librubick (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "rubick.h"
+
+namespace rubick {
+
+// Per plan quad (four consecutive plans sharing d, t, p and the ZeRO stage), packed for the
+// evaluation kernel.  Built by rubick_set_space from the plan list and the environment.
+struct QuadDesc {
+    uint8_t log2d, log2t, log2p, zero;
+    uint8_t g_level;
+    uint8_t flags;      // QF_* bits
+    uint8_t disabled;   // bit i: plan 4q + i is disabled
+    uint8_t pad;
+};
+enum : uint8_t {
+    QF_T_FITS_NODE = 1,   // t <= gpus_per_node
+    QF_DP_INTER = 2,      // the data-parallel ring crosses nodes (d * t > gpus_per_node)
+    QF_PP_INTER = 4,      // the pipeline crosses nodes (g > gpus_per_node)
+};
+
+// Everything a kernel needs to know about the environment and the grid; passed by value as a
+// __grid_constant__ kernel parameter so that level lookups are uniform constant-bank reads.
+struct Space {
+    int32_t P, Q;                 // plans, quads (P / 4)
+    int32_t nG, nC, nM;
+    int32_t Gn, log2Gn, Cn;
+    int32_t strict;
+    int32_t n_small;              // number of GPU levels <= Gn (they come first)
+    float e;                      // bytes per element
+    float inv_B_intra, inv_B_inter, inv_B_pcie;
+    int64_t gpu_mem, Mn;
+    int32_t g_levels[RUBICK_MAX_G_LEVELS];
+    int32_t group_off[RUBICK_MAX_G_LEVELS + 1];
+    int32_t c_levels[RUBICK_MAX_C_LEVELS];
+    float inv_c[RUBICK_MAX_C_LEVELS];
+    int64_t m_levels[RUBICK_MAX_M_LEVELS];
+};
+
+// device status word bits (read back by rubick_sync / the round)
+enum : uint32_t {
+    DS_FEAS_NOT_THRESHOLD = 1u,
+    DS_STEP_CAP = 2u,
+};
+
+}  // namespace rubick
+
+struct rubick_ctx {
+    rubick_env env;
+    int device;
+    cudaStream_t stream;
+    bool has_space;
+    rubick::Space space;
+    std::vector<rubick_plan> plans;
+    rubick::QuadDesc *d_quads;          // [Q]
+    uint32_t *d_status;                 // one word, DS_* bits
+    int32_t *d_steps;                   // one word, steps of the last round
+    // scratch of the greedy round (hot per-job state when it does not fit shared memory)
+    void *d_round_scratch;
+    size_t round_scratch_bytes;
+    // scratch tables of rubick_schedule_round
+    float *d_thr; uint32_t *d_feas; float *d_cv; int32_t *d_cp; int32_t *d_cg;
+    size_t cap_thr, cap_feas, cap_curve;     // capacities in elements
+    rubick_job *d_jobs_stage; size_t cap_jobs;
+    rubick_assignment *d_out_stage; size_t cap_out;
+    rubick_node *d_node_stage; size_t cap_node;
+    int tile_jobs;                      // job tile of rubick_schedule_round
+    int num_sms;
+    std::string err;
+};
+
+namespace rubick {
+
+int fail(rubick_ctx *ctx, int code, const char *msg);
+int cuda_fail(rubick_ctx *ctx, cudaError_t e, const char *what);
+
+// launchers, one per translation unit
+cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J,
+                        float *d_thr, uint32_t *d_feas, cudaStream_t st);
+cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
+                        float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, uint32_t *d_status,
+                        cudaStream_t st);
+cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const float *d_curve_val,
+                        const rubick_assignment *d_state, float *d_gain_gpu, float *d_gain_cpu,
+                        int32_t *d_next_g, int32_t *d_next_c, cudaStream_t st);
+size_t round_scratch_need(const Space &sp, int J, int N);
+cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
+                         const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
+                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                         void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
+
+}  // namespace rubick
