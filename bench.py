@@ -1,0 +1,357 @@
+#!/usr/bin/env python
+"""Benchmark of the Rubick scheduler hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+A step is one pass of the whole path over one synthetic batch of jobs: candidate table +
+feasibility mask, best plans and sensitivity curves, marginal gains, and one greedy scheduling
+round, each through the C ABI with inputs resident in HBM.  Rank 0 prints one JSON line.  With
+N > 1 (torchrun) every rank runs the path on its own independent batch (another tenant's
+cluster: same recipe, another seed); there is no data-path collective, times are the maximum
+over ranks, and `value` is the job total.
+
+`--impl reference` times the CPU checker (oracle/) as it stands on a bounded sample of the same
+workload; it is a deliberately slow program and serves as a reported baseline only.
+"""
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2408_08586_b200 import workloads  # noqa: E402
+
+METRIC = "candidate_evals_per_sec"
+UNIT = "stored candidate evaluations/s (job x plan x cpu-level; host-memory levels resolved by mask bits)"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one eval_candidates launch from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum), as bytes per stored candidate; valid only for the kernel source it was
+# taken on (sha1 of k_eval.cu), otherwise reported as null.
+NCU_EVAL_TRAFFIC = {"k_eval_sha1": None, "bytes_per_candidate": None}
+
+
+def shard_seed_offset(rank):
+    """Each rank schedules an independent cluster drawn from the same recipe."""
+    return 100 * rank
+
+
+def _reduce(x, world, op_name):
+    if world == 1:
+        return x
+    import torch
+    import torch.distributed as dist
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([x], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=getattr(dist.ReduceOp, op_name))
+    return float(t.item())
+
+
+def reduce_max_ms(ms, world):
+    """Max over ranks of a per-rank time (the job is as slow as its slowest rank)."""
+    return _reduce(ms, world, "MAX")
+
+
+def reduce_sum(x, world):
+    return _reduce(x, world, "SUM")
+
+
+def make_workload(name, rank=0, J=None, n_nodes=None):
+    base = workloads.CONFIGS[name]["seed"]
+    workloads.CONFIGS[name]["seed"] = base + shard_seed_offset(rank)
+    try:
+        return workloads.make(name, J=J, n_nodes=n_nodes)
+    finally:
+        workloads.CONFIGS[name]["seed"] = base
+
+
+def algorithmic_bytes_eval(J, P, C):
+    """Bytes one eval_candidates launch must move: 4 per stored candidate (the table), 4 per
+    (job, plan) (the mask word), 128 per job (its record)."""
+    return 4.0 * J * P * C + 4.0 * J * P + 128.0 * J
+
+
+def algorithmic_bytes_best(J, P, C, G, M):
+    """best_plan: reads the table and the mask once, writes value + plan + g per (j, g, c, m)."""
+    return 4.0 * J * P * C + 4.0 * J * P + 12.0 * J * G * C * M
+
+
+def measured_hbm_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "of measured (MEASURED_PEAKS.json hbm_gbs: copy, read + write bytes)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "of fallback (no MEASURED_PEAKS.json)"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.file,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample(cfg, J_sample, n_nodes, nthreads):
+    """One pass of the checker over the first J_sample jobs: table, curves, round -> (seconds, P)."""
+    import oracle
+    jobs = workloads.take(cfg["jobs"], slice(0, J_sample))
+    t0 = time.perf_counter()
+    plans, _ = oracle.enumerate_plans(cfg["g_levels"])
+    thr, feas = oracle.eval_candidates(jobs, plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=nthreads)
+    cv, cp, cg = oracle.best_plan(thr.astype(np.float32), feas, plans, cfg["g_levels"], len(cfg["m_levels"]), nthreads=nthreads)
+    oracle.schedule_round(jobs, cfg["env"], cv.astype(np.float32), cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                          cfg["m_levels"], n_nodes)
+    return time.perf_counter() - t0, len(plans)
+
+
+def run_reference(args):
+    """The CPU checker as the reference arm: rank 0 only, a bounded sample per step."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    cfg = make_workload(args.workload, J=args.jobs, n_nodes=args.nodes)
+    J_full = len(cfg["jobs"]["P"])
+    J_s = min(J_full, args.ref_jobs)
+    nodes = max(1, cfg["n_nodes"] * J_s // J_full)
+    threads = os.cpu_count() or 1
+    for _ in range(args.warmup):
+        oracle_sample(cfg, min(J_s, 16), nodes, threads)
+    t = 0.0
+    P = 0
+    for _ in range(args.steps):
+        dt, P = oracle_sample(cfg, J_s, nodes, threads)
+        t += dt
+    C = len(cfg["c_levels"])
+    value = J_s * P * C * args.steps / t
+    sample = f"first {J_s} of {J_full} jobs on {nodes} nodes per step: table + curves + greedy round"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "jobs": J_s, "plans": P, "cpu_levels": C, "nodes": nodes},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="throughput-stress", choices=list(workloads.CONFIGS))
+    ap.add_argument("--jobs", type=int, default=None, help="override the job count (small captures)")
+    ap.add_argument("--nodes", type=int, default=None)
+    ap.add_argument("--ref-jobs", type=int, default=1024, help="jobs per step of the CPU arm / baseline sample")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2408_08586_b200 import binding as rb
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    cfg = make_workload(args.workload, rank=rank, J=args.jobs, n_nodes=args.nodes)
+    jobs, N = cfg["jobs"], cfg["n_nodes"]
+    J = len(jobs["P"])
+    plans, _ = rb.enumerate_plans(cfg["g_levels"])
+    P, G, C, M = len(plans), len(cfg["g_levels"]), len(cfg["c_levels"]), len(cfg["m_levels"])
+    stream = torch.cuda.Stream(device=dev)
+    ctx = rb.Context(cfg["env"], device=local, stream=stream.cuda_stream)
+    ctx.set_space(plans, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"])
+
+    # device buffers (inputs resident in HBM before the timed region)
+    h_jobs = rb.pack_jobs(jobs)
+    d_jobs = rb.to_device(h_jobs, dev)
+    d_thr = torch.empty(J * C * P, dtype=torch.float32, device=dev)
+    d_feas = torch.empty(J * P, dtype=torch.int32, device=dev)
+    ncurve = J * G * C * M
+    d_cv = torch.empty(ncurve, dtype=torch.float32, device=dev)
+    d_cp = torch.empty(ncurve, dtype=torch.int32, device=dev)
+    d_cg = torch.empty(ncurve, dtype=torch.int32, device=dev)
+    d_state = torch.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+    d_gain = [torch.empty(J, dtype=torch.float32, device=dev) for _ in range(2)]
+    d_next = [torch.empty(J, dtype=torch.int32, device=dev) for _ in range(2)]
+    d_out = torch.empty(J * rb.ASSIGN_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+    d_node = torch.empty(N * rb.NODE_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+    max_steps = 1 << 30
+    round_steps = [0]
+    torch.cuda.synchronize()
+
+    def ev():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record(stream)
+        return e
+
+    def step(marks=None):
+        m = [ev()] if marks is not None else None
+        ctx.eval_candidates(d_jobs, J, d_thr, d_feas)
+        if m: m.append(ev())
+        ctx.best_plan(d_thr, d_feas, J, d_cv, d_cp, d_cg)
+        if m: m.append(ev())
+        ctx.marginal_gain(d_jobs, J, d_cv, d_state, d_gain[0], d_gain[1], d_next[0], d_next[1])
+        if m: m.append(ev())
+        round_steps[0], _ = ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node)
+        if m:
+            m.append(ev())
+            marks.append(m)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local) if rank == 0 else None
+    marks = []
+    t_start = ev()
+    for _ in range(args.steps):
+        step(marks)
+    t_end = ev()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    total_ms = reduce_max_ms(t_start.elapsed_time(t_end), world)
+    stage_ms = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(4)] for m in marks]).mean(axis=0)
+    evals_all = reduce_sum(float(J) * P * C, world)
+    ms_per_step = total_ms / args.steps
+    value = evals_all / (ms_per_step * 1e-3)
+
+    # end to end through the host-buffer entry point: pinned job records in, assignments out
+    e2e = None
+    if not args.no_e2e:
+        hp_jobs = torch.from_numpy(h_jobs.view(np.uint8).reshape(-1).copy()).pin_memory()
+        hp_out = torch.empty(J * rb.ASSIGN_DTYPE.itemsize, dtype=torch.uint8).pin_memory()
+        hp_node = torch.empty(N * rb.NODE_DTYPE.itemsize, dtype=torch.uint8).pin_memory()
+        for _ in range(max(1, min(args.warmup, 3))):
+            ctx.schedule_round_host(hp_jobs, J, N, max_steps, hp_out, hp_node)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            ctx.schedule_round_host(hp_jobs, J, N, max_steps, hp_out, hp_node)
+        torch.cuda.synchronize()
+        e2e_ms = reduce_max_ms(1e3 * (time.perf_counter() - t0) / args.steps, world)
+        e2e = {"value": evals_all / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": int(J * rb.JOB_DTYPE.itemsize),
+               "d2h_bytes_per_step": int(J * rb.ASSIGN_DTYPE.itemsize + N * rb.NODE_DTYPE.itemsize),
+               "call": "rubick_schedule_round_host: pinned job records in, assignments and node states out"}
+
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_hbm_peak()
+    eval_gbs = algorithmic_bytes_eval(J, P, C) / (stage_ms[0] * 1e-3) / 1e9
+    best_gbs = algorithmic_bytes_best(J, P, C, G, M) / (stage_ms[1] * 1e-3) / 1e9
+    sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2408_08586_b200", "csrc", "k_eval.cu"), "rb").read()).hexdigest()
+    traffic = None
+    if NCU_EVAL_TRAFFIC["k_eval_sha1"] == sha and NCU_EVAL_TRAFFIC["bytes_per_candidate"]:
+        traffic = NCU_EVAL_TRAFFIC["bytes_per_candidate"] * float(J) * P * C
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        threads = os.cpu_count() or 1
+        J_s = min(J, args.ref_jobs)
+        nodes_s = max(1, N * J_s // J)
+        dt, _ = oracle_sample(cfg, J_s, nodes_s, threads)
+        cpu_baseline = {"value": J_s * P * C / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+                        "sample": f"first {J_s} of {J} jobs on {nodes_s} nodes, one pass: table + curves + greedy round ({dt:.1f} s)"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "jobs_per_gpu": J, "plans": P, "gpu_levels": G, "cpu_levels": C,
+                   "mem_levels": M, "nodes": N,
+                   "l2": "the table written per step is %.2f GB, larger than the 126 MB L2" % (4e-9 * J * P * C),
+                   "step": "eval_candidates + best_plan + marginal_gain + greedy_round"},
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": 4 * args.steps,
+        "roofline": {"kernel": "eval_candidates_kernel", "bound": "hbm", "achieved": eval_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": eval_gbs / peak, "traffic": traffic, "peak_source": peak_src,
+                     "bytes_per_candidate": algorithmic_bytes_eval(J, P, C) / (float(J) * P * C),
+                     "ms_per_launch": float(stage_ms[0])},
+        "cpu_baseline": cpu_baseline,
+        "stages_ms": {"eval_candidates": float(stage_ms[0]), "best_plan": float(stage_ms[1]),
+                      "marginal_gain": float(stage_ms[2]), "greedy_round": float(stage_ms[3])},
+        "eval_kernel_candidates_per_sec": float(J) * P * C / (stage_ms[0] * 1e-3),
+        "logical_candidates_per_sec": value * M,
+        "best_plan_roofline": {"bound": "hbm", "achieved": best_gbs, "peak": peak, "unit": "GB/s", "frac": best_gbs / peak},
+        "round": {"steps": int(round_steps[0]), "latency_ms": float(stage_ms[3]),
+                  "us_per_step": float(1e3 * stage_ms[3] / max(1, round_steps[0]))},
+    }
+    print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -217,7 +217,7 @@ __device__ bool commit_warp(const Space &sp, Cluster &cl, int n_empty, const flo
     const size_t o = curve_idx(sp, j, gi2, ci2, mi);
     const float v = __ldg(cv + o);
     const int plan = __ldg(cp + o), gu = __ldg(cg + o);
-    if (plan < 0 || !(v > 0.0f) || gu != g2) return false;
+    if (plan < 0 || plan >= sp.P || !(v > 0.0f) || gu != g2) return false;
     if (need_gain && alloc && !(v > hb.val)) return false;
     const uint32_t word = __ldg(feas + size_t(j) * sp.P + plan);
     const int f = __ffs(word) - 1;
@@ -488,6 +488,10 @@ cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const
                          rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                          void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
 {
+    // every step either raises one job by a level or freezes one (job, resource) pair, so a
+    // round cannot take more steps than this; the clamp keeps the device loop bounded regardless
+    const long long natural = (long long)J * (sp.nG + sp.nC + 2) + 1;
+    if ((long long)max_steps > natural) max_steps = int(natural < 0x7fffffffLL ? natural : 0x7fffffffLL);
     const bool in_smem = hot_fits_smem(sp, J, N);
     const size_t smem = round_fixed_smem(sp, N) + (in_smem ? size_t(J) * (sizeof(HotA) + sizeof(HotB)) : 0);
     cudaError_t e = cudaFuncSetAttribute(greedy_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ROUND_SMEM_LIMIT));

@@ -217,7 +217,7 @@ def test_marginal_gain_is_bit_exact(name, J):
         want = oracle.gain(cfg["jobs"], cv, cfg["g_levels"], cfg["c_levels"], g, c, val)
         for a, b in zip(outs, want):
             assert np.array_equal(a.cpu().numpy().view(np.uint32), b.view(np.uint32))
-        assert (want[0] > 0).any() and (want[1] > 0).any()
+        assert (want[0] > 0).any() and (name == "tiny" or (want[1] > 0).any())
 
 
 ROUND_CASES = [("tiny", None, None), ("paper-scale", None, None), ("cluster-512", 96, 24), ("cluster-512", 700, 64),
@@ -236,10 +236,13 @@ def test_greedy_round_on_the_oracle_tables_is_bit_exact(name, J, N):
     assert want["steps"] > 0
 
 
-def test_greedy_round_under_memory_pressure_and_small_nodes():
+@pytest.mark.parametrize("mem_gib,cpus", [(96, 40), (64, 96), (48, 96)])
+def test_greedy_round_under_memory_pressure_and_small_nodes(mem_gib, cpus):
     """Host memory tight enough that commits are rejected or pick a lower memory level."""
     cfg = workloads.make("cluster-512", J=200, n_nodes=12)
-    cfg["env"] = env(mem_per_node_bytes=160 * GIB, cpus_per_node=40)
+    cfg["jobs"]["gmin_idx"][:] = -1
+    cfg["jobs"]["cmin_idx"][:] = -1
+    cfg["env"] = env(mem_per_node_bytes=mem_gib * GIB, cpus_per_node=cpus)
     gpu = Gpu(cfg)
     plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
     want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
@@ -247,6 +250,7 @@ def test_greedy_round_under_memory_pressure_and_small_nodes():
     got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 12)
     assert_rounds_equal(got, want)
     assert (want["log"] & 1 == 0).any()                    # some increment was rejected and frozen
+    assert (want["n_nodes"] > 1).any()                     # and some job spans whole nodes
 
 
 def test_greedy_round_step_cap():
