@@ -45,6 +45,7 @@ extern "C" {
 #define RUBICK_MAX_C_LEVELS  64
 #define RUBICK_MAX_M_LEVELS  32      /* one feasibility word per (job, plan) */
 #define RUBICK_MAX_NODES     4096    /* node state of a round lives in shared memory */
+#define RUBICK_NOALLOC_MAX_JOBS 32768 /* job limit of rubick_greedy_round_noalloc (1 MiB fixed state) */
 
 /* per-job status in rubick_assignment */
 #define RUBICK_UNALLOCATED 0
@@ -198,6 +199,26 @@ int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
                         const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                         int32_t *h_steps);
+
+/* rubick_greedy_round for callers that cannot allocate device memory when they schedule: a
+ * daemon that received a fixed device-memory budget at start-up and shares the GPU with jobs
+ * that fill the rest (a late cudaMalloc may fail, and stalls the device while it runs), or a
+ * process whose device memory belongs to a framework's caching allocator.  (The paper has no counterpart; this is
+ * a convenience of this library.)  Same inputs, outputs, order of decisions and return codes
+ * as rubick_greedy_round, without the step log.  It calls no cudaMalloc, cudaFree or other
+ * allocating routine: the per-job scan state lives in a fixed 1 MiB array inside the library
+ * (32 bytes per job), which every GPU that loads the library holds until the process exits.
+ *  - J above RUBICK_NOALLOC_MAX_JOBS is rejected with EINVAL and a message naming the limit.
+ *  - The first call on a device looks up the array's device address (one cudaGetSymbolAddress
+ *    with that device current) and remembers it; make that first call before any stream capture.
+ *  - All calls, from every context on the device, share the one array.  The kernel rewrites the
+ *    state of all J jobs before reading it, so contents left by an earlier call do no harm; but
+ *    two calls whose kernels overlap on the GPU (different streams, different contexts or
+ *    processes or host threads) race on it and give undefined results.  Run them one after another. */
+int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                                const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
+                                const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
+                                rubick_assignment *d_out, rubick_node *d_node_out, int32_t *h_steps);
 
 /* The whole path for one scheduling event: candidate table, mask, curves and greedy round for
  * d_jobs[0..J), with the intermediate tables in context-owned scratch (grown on demand, kept

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "librubick.so")
 OK, EINVAL, ENOMEM, ECUDA, ESTEPS, ESTATE = 0, -1, -2, -3, -4, -5
 UNALLOCATED, RUNNING, PENDING = 0, 1, 2
 BEST_RAW = 1
+NOALLOC_MAX_JOBS = 32768
 
 JOB_DTYPE = np.dtype([
     ("P", "<f8"), ("host_base_bytes", "<i8"), ("l", "<i4"), ("h", "<i4"), ("s", "<i4"), ("b", "<i4"),
@@ -49,7 +50,8 @@ class Cluster(C.Structure):
 
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
            "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_marginal_gain",
-           "rubick_greedy_round", "rubick_schedule_round", "rubick_schedule_round_host"]
+           "rubick_greedy_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
+           "rubick_schedule_round_host"]
 
 _lib = None
 
@@ -81,6 +83,7 @@ def lib():
         L.rubick_best_plan.argtypes = [vp, vp, vp, ip, C.c_uint, vp, vp, vp]
         L.rubick_marginal_gain.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp]
         L.rubick_greedy_round.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, vp, C.POINTER(C.c_int32)]
+        L.rubick_greedy_round_noalloc.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         for name in EXPORTS:
@@ -204,6 +207,19 @@ class Context:
         rc = self._check(lib().rubick_greedy_round(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_curve_plan),
                                                    _ptr(d_curve_g), _ptr(d_feas), C.byref(cl), int(max_steps), _ptr(d_out),
                                                    _ptr(d_node_out), _ptr(d_step_log), C.byref(steps)), allow=(ESTEPS,))
+        return steps.value, rc == ESTEPS
+
+    def greedy_round_noalloc(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, n_nodes, max_steps, d_out,
+                             d_node_out=None):
+        """rubick_greedy_round_noalloc: the round with its job state in the library's fixed array,
+        for callers that may not allocate device memory; at most NOALLOC_MAX_JOBS jobs.
+        -> (steps, capped)"""
+        steps = C.c_int32(0)
+        cl = Cluster(int(n_nodes))
+        rc = self._check(lib().rubick_greedy_round_noalloc(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val),
+                                                           _ptr(d_curve_plan), _ptr(d_curve_g), _ptr(d_feas), C.byref(cl),
+                                                           int(max_steps), _ptr(d_out), _ptr(d_node_out), C.byref(steps)),
+                         allow=(ESTEPS,))
         return steps.value, rc == ESTEPS
 
     def schedule_round(self, d_jobs, J, n_nodes, max_steps, d_out, d_node_out=None):

@@ -505,3 +505,89 @@ cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const
 }
 
 }  // namespace rubick
+
+// ------------------------------------------------------------------------------------------------
+// Greedy round for callers that must not allocate.
+//
+// Some hosts of this library cannot call cudaMalloc when they schedule: a scheduler daemon that
+// was given a fixed device-memory budget at start-up and shares the GPU with jobs that fill the
+// rest of it (a late allocation may fail, and it synchronises the whole device while it runs), or
+// a process whose device memory is owned by a framework's caching allocator that has already
+// reserved everything.  rubick_greedy_round grows a context scratch buffer with cudaMalloc when
+// the per-job scan state does not fit shared memory; the entry point below never allocates: the
+// per-job state always lives in the fixed array declared here, which every GPU that loads the
+// library holds until the process exits.
+// ------------------------------------------------------------------------------------------------
+
+namespace rubick {
+
+constexpr size_t NOALLOC_STATE_BYTES = size_t(RUBICK_NOALLOC_MAX_JOBS) * (sizeof(HotA) + sizeof(HotB));   // 1 MiB
+static __device__ __align__(256) unsigned char g_noalloc_state[NOALLOC_STATE_BYTES];
+
+// In host code `g_noalloc_state` is only a handle; the device address has to be asked for, once
+// per device, with that device current.
+constexpr int NOALLOC_MAX_DEVICES = 64;
+static void *g_noalloc_addr[NOALLOC_MAX_DEVICES];
+
+}  // namespace rubick
+
+extern "C" int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                                           const float *d_curve_val, const int32_t *d_curve_plan,
+                                           const int32_t *d_curve_g, const uint32_t *d_feas,
+                                           const rubick_cluster *h_cluster, int max_steps,
+                                           rubick_assignment *d_out, rubick_node *d_node_out, int32_t *h_steps)
+{
+    using namespace rubick;
+    if (!ctx) return RUBICK_EINVAL;
+    if (!ctx->has_space) return fail(ctx, RUBICK_ESTATE, "no plan space: call rubick_set_space first");
+    if (J < 0 || max_steps < 0) return fail(ctx, RUBICK_EINVAL, "negative job count or max_steps");
+    if (J > RUBICK_NOALLOC_MAX_JOBS)
+        return fail(ctx, RUBICK_EINVAL, "rubick_greedy_round_noalloc: more than RUBICK_NOALLOC_MAX_JOBS jobs; the fixed state array cannot hold them");
+    if (!h_cluster || h_cluster->n_nodes < 1 || h_cluster->n_nodes > RUBICK_MAX_NODES)
+        return fail(ctx, RUBICK_EINVAL, "cluster: 1 .. RUBICK_MAX_NODES nodes");
+    if (J > 0 && (!d_jobs || !d_curve_val || !d_curve_plan || !d_curve_g || !d_feas || !d_out))
+        return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if (ctx->device < 0 || ctx->device >= NOALLOC_MAX_DEVICES) return fail(ctx, RUBICK_EINVAL, "device index out of range");
+    const Space &sp = ctx->space;
+    const int N = h_cluster->n_nodes;
+    const size_t smem = round_fixed_smem(sp, N);
+    if (smem > ROUND_SMEM_LIMIT) return fail(ctx, RUBICK_EINVAL, "cluster state does not fit shared memory");
+
+    cudaError_t e = cudaSetDevice(ctx->device);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaSetDevice");
+    if (!g_noalloc_addr[ctx->device]) {          // first call on this device: resolve the array's device address
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_state);
+        if (e != cudaSuccess || !p) return cuda_fail(ctx, e, "cudaGetSymbolAddress (fixed round state)");
+        g_noalloc_addr[ctx->device] = p;
+    }
+    unsigned char *base = static_cast<unsigned char *>(g_noalloc_addr[ctx->device]);
+    HotA *ha = reinterpret_cast<HotA *>(base);
+    HotB *hb = reinterpret_cast<HotB *>(base + size_t(RUBICK_NOALLOC_MAX_JOBS) * sizeof(HotA));
+
+    const long long natural = (long long)J * (sp.nG + sp.nC + 2) + 1;
+    if ((long long)max_steps > natural) max_steps = int(natural < 0x7fffffffLL ? natural : 0x7fffffffLL);
+    e = cudaFuncSetAttribute(greedy_round_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(ROUND_SMEM_LIMIT));
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaFuncSetAttribute");
+    // the kernel writes every job's state before it reads it, so stale contents of the array
+    // from an earlier call need no clearing
+    greedy_round_kernel<<<1, ROUND_THREADS, smem, ctx->stream>>>(sp, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas,
+                                                                 N, max_steps, d_out, d_node_out, nullptr, ha, hb, 0,
+                                                                 ctx->d_status, ctx->d_steps);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "launch greedy_round (fixed state)");
+
+    uint32_t two[2] = {0u, 0u};
+    e = cudaMemcpyAsync(two, ctx->d_status, 8, cudaMemcpyDeviceToHost, ctx->stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "read round status");
+    e = cudaStreamSynchronize(ctx->stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaStreamSynchronize");
+    if (h_steps) *h_steps = int32_t(two[1]);
+    if (two[0] & DS_STEP_CAP) {
+        const uint32_t cleared = two[0] & ~uint32_t(DS_STEP_CAP);
+        cudaMemcpyAsync(ctx->d_status, &cleared, 4, cudaMemcpyHostToDevice, ctx->stream);
+        cudaStreamSynchronize(ctx->stream);
+        return fail(ctx, RUBICK_ESTEPS, "greedy round stopped at max_steps");
+    }
+    return RUBICK_OK;
+}
