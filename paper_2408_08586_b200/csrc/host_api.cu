@@ -267,15 +267,21 @@ static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const
                          const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps, rubick_assignment *d_out,
                          rubick_node *d_node_out, int32_t *d_step_log)
 {
-    const size_t need = round_scratch_need(ctx->space, J, N);
+    const bool fast = round_fast_supported(ctx->space, J, N);
+    const size_t need = fast ? round_fast_scratch_need(ctx->space, J, N) : round_scratch_need(ctx->space, J, N);
     if (need > ctx->round_scratch_bytes) {
         if (ctx->d_round_scratch) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_round_scratch); ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0; }
         CUDA_TRY(ctx, cudaMalloc(&ctx->d_round_scratch, need), "cudaMalloc (round scratch)");
         ctx->round_scratch_bytes = need;
     }
-    CUDA_TRY(ctx, launch_round(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
-                               ctx->d_round_scratch, ctx->d_status, ctx->d_steps, ctx->stream),
-             "launch greedy_round");
+    if (fast)
+        CUDA_TRY(ctx, launch_round_fast(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
+                                        ctx->d_round_scratch, ctx->d_status, ctx->d_steps, ctx->stream),
+                 "launch greedy_round (fast path)");
+    else
+        CUDA_TRY(ctx, launch_round(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
+                                   ctx->d_round_scratch, ctx->d_status, ctx->d_steps, ctx->stream),
+                 "launch greedy_round");
     return RUBICK_OK;
 }
 

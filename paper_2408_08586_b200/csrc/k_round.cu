@@ -1,0 +1,812 @@
+// Greedy scheduling round, fast path (paper Section 5.2, Algorithm 1 in marginal-gain form).
+//
+// Same decisions, step for step, as the plain round in k_sched.cu (largest placeable positive
+// GPU gain first, CPU gain when no GPU increment is left, lowest job index on ties, commit with
+// the best plan and its host memory), organised so that one step costs about a microsecond:
+//
+//   prepare  (grid)   per (job, GPU level, CPU level): the curve entry at the top host-memory level
+//                     together with the first feasible memory level of its plan, 16 bytes.  A commit
+//                     whose node offers at least that level needs no further table look-up, because
+//                     the curve at any level >= the plan's first level equals the curve at the top.
+//   keys     (grid)   every best-effort job starts unallocated, and its first increment (smallest
+//                     GPU level with a non-zero curve at its starting CPU level) and gain are fixed
+//                     until it is allocated: one 64-bit key (class = target levels | gain | ~job).
+//                     Guaranteed jobs get their Phase-A target resolved here too.
+//   sort     (1 CTA)  bitonic sort of the keys: inside a class (same target levels = same placement
+//                     test) only the first unconsumed job can ever be selected.
+//   round    (1 CTA)  persistent loop.  Shared memory holds the node state, an incrementally
+//                     maintained first-fit table  node(g level, c level), the head of every class and
+//                     one 36-byte slot per RUNNING job.  A step scans class heads + running slots
+//                     (not all jobs), reduces a 64-bit key (type | gain | ~job) across the block, and
+//                     warp 0 commits: placement from the first-fit table, memory level by ballot,
+//                     node bookkeeping, table repair for the touched nodes, new gains with one
+//                     warp-wide load of the job's curve column.
+//
+// All gain arithmetic uses __fmul_rn / __fsub_rn / __fdiv_rn (one rounding per operation, never
+// fused) so that decisions are reproducible bit for bit.  Every loop is bounded (steps by
+// max_steps, scans by the node / level counts); nothing spins on memory.
+
+#include "rubick_internal.cuh"
+
+namespace rubick {
+namespace fastround {
+
+constexpr int RT = 1024;
+constexpr int RW = RT / 32;
+constexpr int TOUCH_CAP = 160;
+constexpr size_t SMEM_LIMIT = 200 * 1024;
+constexpr int SORT_SMEM_KEYS = 16384;
+
+typedef unsigned long long u64;
+
+struct HotCurve { float val; int32_t plan; int32_t f; int32_t ok; };                        // 16 bytes
+struct PhaseA { int32_t gi, ci; float val; int32_t plan; int32_t f; int32_t ok; float w; int32_t pad; };   // 32 bytes
+struct SlotA { float gain_g, gain_c; uint32_t packed; int32_t node; };
+struct SlotB { float val; int32_t plan; int32_t f_level; float w; };
+
+// sort key of an unallocated job: [63:53] class = gi2 * 64 + ci | [52:21] gain bits | [20:0] ~job
+constexpr int KEY_JOB_BITS = 21;
+constexpr u64 KEY_JOB_MASK = (1ull << KEY_JOB_BITS) - 1;
+__device__ __forceinline__ int key_job(u64 k) { return int(KEY_JOB_MASK - (k & KEY_JOB_MASK)); }
+__device__ __forceinline__ uint32_t key_gain_bits(u64 k) { return uint32_t(k >> KEY_JOB_BITS); }
+__device__ __forceinline__ int key_class(u64 k) { return int(k >> 53); }
+
+// selection key of a step: [63] 1 = GPU increment | [62:31] gain bits | [30:0] ~job
+__device__ __forceinline__ u64 sel_key(int type_gpu, uint32_t gain_bits, int j)
+{
+    return (u64(type_gpu) << 63) | (u64(gain_bits) << 31) | u64(0x7fffffffu - uint32_t(j));
+}
+__device__ __forceinline__ int sel_job(u64 k) { return int(0x7fffffffu - uint32_t(k & 0x7fffffffu)); }
+
+// slot.packed: [5:0] g level | [12:6] c level | [18:13] target g level + 1 | [20] GPU frozen | [21] CPU frozen
+__device__ __forceinline__ uint32_t pack(int gi, int ci, int next_gi, bool fz_g, bool fz_c)
+{
+    return uint32_t(gi) | (uint32_t(ci) << 6) | (uint32_t(next_gi + 1) << 13) | (uint32_t(fz_g) << 20) | (uint32_t(fz_c) << 21);
+}
+__device__ __forceinline__ int pk_gi(uint32_t p) { return int(p & 63u); }
+__device__ __forceinline__ int pk_ci(uint32_t p) { return int((p >> 6) & 127u); }
+__device__ __forceinline__ int pk_next_gi(uint32_t p) { return int((p >> 13) & 63u) - 1; }
+__device__ __forceinline__ bool pk_fz_g(uint32_t p) { return (p >> 20) & 1u; }
+__device__ __forceinline__ bool pk_fz_c(uint32_t p) { return (p >> 21) & 1u; }
+
+__device__ __forceinline__ size_t curve_idx(const Space &sp, int j, int gi, int ci, int mi)
+{
+    return ((size_t(j) * sp.nG + gi) * sp.nC + ci) * sp.nM + mi;
+}
+__device__ __forceinline__ size_t hc_idx(const Space &sp, int j, int gi, int ci) { return (size_t(j) * sp.nG + gi) * sp.nC + ci; }
+__device__ __forceinline__ int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+__device__ __forceinline__ HotCurve load_hc(const HotCurve *p)
+{
+    const int4 v = *reinterpret_cast<const int4 *>(p);
+    HotCurve h; h.val = __int_as_float(v.x); h.plan = v.y; h.f = v.z; h.ok = v.w;
+    return h;
+}
+
+// ---- prepare: curve entries at the top memory level with the plan's first feasible level ---------
+__global__ void round_prepare_kernel(const __grid_constant__ Space sp, const float *__restrict__ cv,
+                                     const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
+                                     const uint32_t *__restrict__ feas, int J, HotCurve *__restrict__ hc)
+{
+    const size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t per_job = size_t(sp.nG) * sp.nC;
+    if (i >= size_t(J) * per_job) return;
+    const int j = int(i / per_job);
+    const int gi = int((i - size_t(j) * per_job) / sp.nC);
+    const size_t o = i * sp.nM + (sp.nM - 1);
+    HotCurve h;
+    h.val = __ldg(cv + o); h.plan = __ldg(cp + o);
+    h.ok = __ldg(cg + o) == sp.g_levels[gi];
+    h.f = -1;
+    if (h.plan >= 0 && h.plan < sp.P) h.f = __ffs(__ldg(feas + size_t(j) * sp.P + h.plan)) - 1;
+    int4 v; v.x = __float_as_int(h.val); v.y = h.plan; v.z = h.f; v.w = h.ok;
+    reinterpret_cast<int4 *>(hc)[i] = v;
+}
+
+// ---- keys: first increment of every best-effort job, Phase-A target of every guaranteed job -------
+__global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
+                                  const HotCurve *__restrict__ hc, const int32_t *__restrict__ cp,
+                                  const int32_t *__restrict__ cg, u64 *__restrict__ keys, int n_pad,
+                                  PhaseA *__restrict__ pa)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n_pad) return;
+    u64 key = 0ull;
+    if (j < J) {
+        const rubick_job *jb = jobs + j;
+        const int gmin = jb->gmin_idx;
+        const float w = jb->w;
+        PhaseA a; a.gi = -2; a.ci = 0; a.val = 0.0f; a.plan = -1; a.f = -1; a.ok = 0; a.w = w; a.pad = 0;
+        if (gmin < 0) {
+            const int ci = min(max(jb->cmin_idx, 0), sp.nC - 1);
+            for (int gi = 0; gi < sp.nG; ++gi) {
+                const float v = hc[hc_idx(sp, j, gi, ci)].val;
+                if (v > 0.0f) {
+                    const float gain = __fdiv_rn(__fsub_rn(__fmul_rn(w, v), 0.0f), float(sp.g_levels[gi]));
+                    if (gain > 0.0f)
+                        key = (u64(gi * 64 + ci) << 53) | (u64(__float_as_uint(gain)) << KEY_JOB_BITS) | (KEY_JOB_MASK - u64(j));
+                    break;
+                }
+            }
+        } else {
+            // guaranteed: placed in Phase A at (gmin, cmin) with the GPU count the curve really uses
+            a.gi = -1;
+            const int cmin = max(jb->cmin_idx, 0);
+            if (gmin < sp.nG && cmin < sp.nC) {
+                const size_t o = curve_idx(sp, j, gmin, cmin, sp.nM - 1);
+                if (__ldg(cp + o) >= 0) {
+                    // the curve may reach this value with fewer GPUs than the level offers
+                    const int gu = __ldg(cg + o);
+                    int gi = -1;
+                    for (int i = 0; i < sp.nG; ++i) if (sp.g_levels[i] == gu) gi = i;
+                    if (gi >= 0) {
+                        const HotCurve h = load_hc(hc + hc_idx(sp, j, gi, cmin));
+                        a.gi = gi; a.ci = cmin; a.val = h.val; a.plan = h.plan; a.f = h.f; a.ok = h.ok;
+                    }
+                }
+            }
+        }
+        reinterpret_cast<int4 *>(pa + j)[0] = make_int4(a.gi, a.ci, __float_as_int(a.val), a.plan);
+        reinterpret_cast<int4 *>(pa + j)[1] = make_int4(a.f, a.ok, __float_as_int(a.w), 0);
+    }
+    keys[j] = key;
+}
+
+// ---- sort: descending bitonic sort of n (power of two) keys, then the weights in sorted order -----
+__global__ void __launch_bounds__(RT)
+round_sort_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ jobs, float *__restrict__ sorted_w,
+                  int in_smem)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    u64 *a = in_smem ? reinterpret_cast<u64 *>(smem_raw) : keys;
+    if (in_smem) {
+        for (int i = threadIdx.x; i < n; i += RT) a[i] = keys[i];
+        __syncthreads();
+    }
+    for (int k = 2; k <= n; k <<= 1)
+        for (int s = k >> 1; s > 0; s >>= 1) {
+            for (int i = threadIdx.x; i < n; i += RT) {
+                const int p = i ^ s;
+                if (p > i) {
+                    const u64 x = a[i], y = a[p];
+                    const bool desc = (i & k) == 0;
+                    if (desc ? (x < y) : (x > y)) { a[i] = y; a[p] = x; }
+                }
+            }
+            __syncthreads();
+        }
+    for (int i = threadIdx.x; i < n; i += RT) {
+        const u64 k = a[i];
+        if (in_smem) keys[i] = k;
+        sorted_w[i] = k ? jobs[key_job(k)].w : 0.0f;
+    }
+}
+
+// ---- the persistent round ---------------------------------------------------------------------------
+struct Views {
+    int64_t *free_m;
+    int32_t *free_g, *free_c, *owner, *ff, *touched;
+    int32_t *cls_ptr, *cls_end; u64 *cls_top; float *cls_w;
+    SlotA *sa; SlotB *sb; int32_t *sj;
+    int N;
+};
+
+struct Shared {
+    u64 red_key[RW];
+    uint32_t red_pay[RW];
+    int n_empty, n_slots, steps, capped, stop, nt, ff_full, n_guar;
+    int scan_cnt[RW];
+};
+
+__device__ int first_fit_from(const Views &v, int start, int g, int c, int lane)
+{
+    for (int base = start & ~31; base < v.N; base += 32) {
+        const int n = base + lane;
+        const bool ok = n >= start && n < v.N && v.free_g[n] >= g && v.free_c[n] >= c;
+        const unsigned b = __ballot_sync(0xffffffffu, ok);
+        if (b) return base + __ffs(b) - 1;
+    }
+    return -1;
+}
+
+// Repair the first-fit table after the nodes in v.touched[0..nt) changed (warp 0, all lanes).
+__device__ void ff_repair(const Space &sp, const Views &v, int nt, bool full, int lane)
+{
+    const int n_ff = sp.n_small * sp.nC;
+    for (int e0 = 0; e0 < n_ff; e0 += 32) {
+        const int e = e0 + lane;
+        const bool act = e < n_ff;
+        const int gi = act ? e / sp.nC : 0, ci = act ? e - gi * sp.nC : 0;
+        const int g = sp.g_levels[gi], c = sp.c_levels[ci];
+        int cur = act ? v.ff[e] : -1;
+        bool rescan = false;
+        int start = 0;
+        if (act) {
+            if (full) { rescan = true; start = 0; }
+            else {
+                int best_new = -1; bool lost = false;
+                for (int t = 0; t < nt; ++t) {
+                    const int n = v.touched[t];
+                    const bool fit = v.free_g[n] >= g && v.free_c[n] >= c;
+                    if (fit) { if (best_new < 0 || n < best_new) best_new = n; }
+                    else if (n == cur) lost = true;
+                }
+                if (best_new >= 0 && (cur < 0 || best_new < cur)) cur = best_new;
+                else if (lost) { rescan = true; start = cur + 1; }
+            }
+        }
+        unsigned need = __ballot_sync(0xffffffffu, rescan);
+        while (need) {
+            const int src = __ffs(need) - 1;
+            need &= need - 1;
+            const int g2 = __shfl_sync(0xffffffffu, g, src), c2 = __shfl_sync(0xffffffffu, c, src);
+            const int st = __shfl_sync(0xffffffffu, start, src);
+            const int r = first_fit_from(v, st, g2, c2, lane);
+            if (lane == src) cur = r;
+        }
+        if (act) v.ff[e] = cur;
+    }
+    __syncwarp();
+}
+
+struct Committed { int first; float val; int plan; int f; };
+
+// Commit job j to (gi2, ci2); warp 0, all lanes, uniform control flow.  `alloc`: the job holds
+// (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target
+// at the top memory level.  On success the node state, the touched list, the empty-node count and
+// the first-fit table are up to date.
+__device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const float *__restrict__ cv,
+                            const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
+                            const uint32_t *__restrict__ feas, int j, bool alloc, int gi, int ci, int node,
+                            float val_cur, int f_cur, int gi2, int ci2, HotCurve cand, bool need_gain, int lane,
+                            Committed &out)
+{
+    const int g = alloc ? sp.g_levels[gi] : 0, c = alloc ? sp.c_levels[ci] : 0;
+    const int64_t m_cur = alloc ? sp.m_levels[f_cur] : 0;
+    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    const int k = alloc ? max(g >> sp.log2Gn, 1) : 0;
+    const int n_empty = sh.n_empty;
+
+    int k2 = 1, target = -1, need_new = 0;
+    bool stay = false;
+    if (g2 <= sp.Gn) {
+        if (alloc && v.free_g[node] >= g2 - g && v.free_c[node] >= c2 - c) { stay = true; target = node; }
+        else target = v.ff[gi2 * sp.nC + ci2];
+        if (target < 0) return false;
+    } else {
+        k2 = g2 >> sp.log2Gn;
+        if ((c2 + k2 - 1) / k2 > sp.Cn) return false;
+        if (alloc && g >= sp.Gn) { stay = true; need_new = k2 - k; if (n_empty < need_new) return false; }
+        else {
+            need_new = k2;
+            const int empty = n_empty + ((alloc && v.free_g[node] + g == sp.Gn) ? 1 : 0);
+            if (empty < need_new) return false;
+        }
+    }
+
+    const int64_t avail = k2 > 1 ? sp.Mn : v.free_m[target] + ((stay && alloc) ? m_cur : 0);
+    const bool fits = lane < sp.nM && cdiv64(sp.m_levels[lane < sp.nM ? lane : 0], k2) <= avail;
+    const unsigned fb = __ballot_sync(0xffffffffu, fits);
+    if (!fb) return false;
+    const int mi = 31 - __clz(fb);
+
+    float val; int plan, f; bool okg;
+    if (cand.plan >= 0 && cand.f >= 0 && cand.f <= mi) {
+        // the top-level best plan is feasible at level mi, hence also the best one there
+        val = cand.val; plan = cand.plan; f = cand.f; okg = cand.ok != 0;
+    } else {
+        const size_t o = curve_idx(sp, j, gi2, ci2, mi);
+        val = __ldg(cv + o); plan = __ldg(cp + o); okg = __ldg(cg + o) == g2;
+        f = -1;
+        if (plan >= 0 && plan < sp.P) f = __ffs(__ldg(feas + size_t(j) * sp.P + plan)) - 1;
+    }
+    if (plan < 0 || plan >= sp.P || !(val > 0.0f) || !okg) return false;
+    if (need_gain && alloc && !(val > val_cur)) return false;
+    if (f < 0 || f > mi) return false;
+    const int64_t m2 = sp.m_levels[f];
+
+    // ---- node bookkeeping; every changed node goes on the touched list ---------------------------
+    int first = -1, nt = 0, d_empty = 0;
+    bool full = false;
+    if (k2 == 1) {
+        if (lane == 0) {
+            if (alloc && !stay) {
+                v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur;
+                v.touched[nt] = node;
+            }
+            if (stay) { v.free_g[target] -= g2 - g; v.free_c[target] -= c2 - c; v.free_m[target] -= m2 - m_cur; }
+            else { v.free_g[target] -= g2; v.free_c[target] -= c2; v.free_m[target] -= m2; }
+        }
+        __syncwarp();
+        if (alloc && !stay) { nt = 1; if (v.free_g[node] == sp.Gn) d_empty += 1; }
+        if (!stay && v.free_g[target] + g2 == sp.Gn) d_empty -= 1;
+        if (lane == 0) v.touched[nt] = target;
+        nt += 1;
+        first = target;
+    } else {
+        const int cs2 = (c2 + k2 - 1) / k2;
+        const int64_t ms2 = cdiv64(m2, k2);
+        if (stay) {
+            const int cs1 = (c + k - 1) / k;
+            const int64_t ms1 = cdiv64(m_cur, k);
+            if (k == 1) {
+                if (lane == 0) { v.free_c[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; v.touched[0] = node; }
+                nt = 1;
+            } else {
+                // cores only: GPU levels above a node change the node count, so this is a CPU step
+                for (int base = 0; base < v.N; base += 32) {
+                    const int n = base + lane;
+                    const bool mine = n < v.N && v.owner[n] == j;
+                    if (mine) { v.free_c[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
+                    const unsigned b = __ballot_sync(0xffffffffu, mine);
+                    if (mine) { const int pos = nt + __popc(b & ((1u << lane) - 1u)); if (pos < TOUCH_CAP) v.touched[pos] = n; }
+                    nt += __popc(b);
+                }
+            }
+            first = node;
+        } else if (alloc) {
+            if (lane == 0) { v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur; v.touched[0] = node; }
+            __syncwarp();
+            nt = 1;
+            if (v.free_g[node] == sp.Gn) d_empty += 1;
+        }
+        __syncwarp();
+        int taken = 0;
+        for (int base = 0; base < v.N && taken < need_new; base += 32) {
+            const int n = base + lane;
+            const bool empty = n < v.N && v.free_g[n] == sp.Gn;
+            const unsigned b = __ballot_sync(0xffffffffu, empty);
+            const int rank = __popc(b & ((1u << lane) - 1u));
+            if (empty && taken + rank < need_new) {
+                v.free_g[n] = 0; v.free_c[n] -= cs2; v.free_m[n] -= ms2; v.owner[n] = j;
+                const int pos = nt + rank;
+                if (pos < TOUCH_CAP) v.touched[pos] = n;
+            }
+            if (b) { const int lowest = base + __ffs(b) - 1; if (first < 0 || lowest < first) first = lowest; }
+            const int got = min(__popc(b), need_new - taken);
+            taken += got; nt += got;
+        }
+        d_empty -= need_new;
+        if (nt > TOUCH_CAP) full = true;
+    }
+    __syncwarp();
+    if (lane == 0) sh.n_empty = n_empty + d_empty;
+    ff_repair(sp, v, nt, full, lane);
+    out.first = first; out.val = val; out.plan = plan; out.f = f;
+    return true;
+}
+
+// New gains of a running job (warp-wide): one load per GPU level above the present one.
+__device__ void gains_warp(const Space &sp, const HotCurve *__restrict__ hc, int j, float w, int gi, int ci, float val,
+                           int lane, int &next_g, float &gain_g, int &next_c, float &gain_c)
+{
+    const float vcur = __fmul_rn(w, val);
+    const int lvl = gi + 1 + lane;
+    float v = 0.0f;
+    if (lvl < sp.nG) v = hc[hc_idx(sp, j, lvl, ci)].val;
+    float vc = 0.0f;
+    if (ci + 1 < sp.nC) vc = hc[hc_idx(sp, j, gi, ci + 1)].val;
+    const unsigned b = __ballot_sync(0xffffffffu, lvl < sp.nG && v > val);
+    next_g = -1; gain_g = 0.0f; next_c = -1; gain_c = 0.0f;
+    if (b) {
+        const int src = __ffs(b) - 1;
+        const float vv = __shfl_sync(0xffffffffu, v, src);
+        next_g = gi + 1 + src;
+        gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, vv), vcur), float(sp.g_levels[next_g] - sp.g_levels[gi]));
+    }
+    if (ci + 1 < sp.nC) {
+        const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(w, vc), vcur), float(sp.c_levels[ci + 1] - sp.c_levels[ci]));
+        if (gn > 0.0f) { next_c = ci + 1; gain_c = gn; }
+    }
+}
+
+// the same for one thread (initial gains of the jobs placed in Phase A)
+__device__ void gains_thread(const Space &sp, const HotCurve *__restrict__ hc, int j, float w, int gi, int ci, float val,
+                             int &next_g, float &gain_g, int &next_c, float &gain_c)
+{
+    const float vcur = __fmul_rn(w, val);
+    next_g = -1; gain_g = 0.0f; next_c = -1; gain_c = 0.0f;
+    for (int g2 = gi + 1; g2 < sp.nG; ++g2) {
+        const float v = hc[hc_idx(sp, j, g2, ci)].val;
+        if (v > val) {
+            next_g = g2;
+            gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, v), vcur), float(sp.g_levels[g2] - sp.g_levels[gi]));
+            break;
+        }
+    }
+    if (ci + 1 < sp.nC) {
+        const float v = hc[hc_idx(sp, j, gi, ci + 1)].val;
+        const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(w, v), vcur), float(sp.c_levels[ci + 1] - sp.c_levels[ci]));
+        if (gn > 0.0f) { next_c = ci + 1; gain_c = gn; }
+    }
+}
+
+__device__ __forceinline__ bool slot_placeable(const Space &sp, const Views &v, int n_empty, int gi, int ci, int node,
+                                               int gi2, int ci2)
+{
+    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    const int g = sp.g_levels[gi], c = sp.c_levels[ci];
+    if (g2 <= sp.Gn) {
+        if (v.free_g[node] >= g2 - g && v.free_c[node] >= c2 - c) return true;
+        return v.ff[gi2 * sp.nC + ci2] >= 0;
+    }
+    const int k2 = g2 >> sp.log2Gn;
+    if ((c2 + k2 - 1) / k2 > sp.Cn) return false;
+    if (g >= sp.Gn) return n_empty >= k2 - (g >> sp.log2Gn);
+    return n_empty + ((v.free_g[node] + g == sp.Gn) ? 1 : 0) >= k2;
+}
+
+__device__ __forceinline__ bool class_placeable(const Space &sp, const Views &v, int n_empty, int gi2, int ci2)
+{
+    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    if (g2 <= sp.Gn) return v.ff[gi2 * sp.nC + ci2] >= 0;
+    const int k2 = g2 >> sp.log2Gn;
+    return (c2 + k2 - 1) / k2 <= sp.Cn && n_empty >= k2;
+}
+
+struct RoundArgs {
+    const rubick_job *jobs; int J;
+    const float *cv; const int32_t *cp; const int32_t *cg; const uint32_t *feas;
+    int N, max_steps;
+    rubick_assignment *out; rubick_node *node_out; int32_t *step_log;
+    const HotCurve *hc; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
+    int32_t *glist;
+    SlotA *sa_g; SlotB *sb_g; int32_t *sj_g; int slots_in_smem; int slot_cap;
+    uint32_t *status; int32_t *steps_out;
+};
+
+__global__ void __launch_bounds__(RT, 1)
+greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant__ RoundArgs A)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    __shared__ Shared sh;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int N = A.N, J = A.J;
+    const int n_ff = sp.n_small * sp.nC, n_cls = sp.nG * sp.nC;
+
+    Views v;
+    v.N = N;
+    unsigned char *p = smem_raw;
+    v.free_m = reinterpret_cast<int64_t *>(p); p += size_t(N) * 8;
+    v.cls_top = reinterpret_cast<u64 *>(p); p += size_t(n_cls) * 8;
+    v.free_g = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
+    v.free_c = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
+    v.owner = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
+    v.ff = reinterpret_cast<int32_t *>(p); p += size_t(n_ff) * 4;
+    v.touched = reinterpret_cast<int32_t *>(p); p += size_t(TOUCH_CAP) * 4;
+    v.cls_ptr = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
+    v.cls_end = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
+    v.cls_w = reinterpret_cast<float *>(p); p += size_t(n_cls) * 4;
+    p = smem_raw + ((size_t(p - smem_raw) + 15) & ~size_t(15));
+    if (A.slots_in_smem) {
+        v.sa = reinterpret_cast<SlotA *>(p); p += size_t(A.slot_cap) * sizeof(SlotA);
+        v.sb = reinterpret_cast<SlotB *>(p); p += size_t(A.slot_cap) * sizeof(SlotB);
+        v.sj = reinterpret_cast<int32_t *>(p);
+    } else { v.sa = A.sa_g; v.sb = A.sb_g; v.sj = A.sj_g; }
+
+    // ---- set-up ---------------------------------------------------------------------------------
+    for (int n = tid; n < N; n += RT) { v.free_g[n] = sp.Gn; v.free_c[n] = sp.Cn; v.free_m[n] = sp.Mn; v.owner[n] = -1; }
+    for (int e = tid; e < n_ff; e += RT) v.ff[e] = 0;                      // every node is empty
+    for (int t = tid; t < n_cls; t += RT) { v.cls_ptr[t] = 0; v.cls_end[t] = 0; v.cls_top[t] = 0ull; v.cls_w[t] = 0.0f; }
+    if (tid == 0) { sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; }
+    __syncthreads();
+
+    // class segments of the sorted keys: a class starts where the class field changes
+    for (int i = tid; i < A.n_pad; i += RT) {
+        const u64 k = A.keys[i];
+        const u64 kp = i ? A.keys[i - 1] : 0ull;
+        if (k && (i == 0 || key_class(kp) != key_class(k))) {
+            const int cls = key_class(k);
+            const int t = (cls >> 6) * sp.nC + (cls & 63);
+            v.cls_ptr[t] = i; v.cls_top[t] = k; v.cls_w[t] = A.sorted_w[i];
+        }
+        if (i && kp && (!k || key_class(kp) != key_class(k))) {
+            const int cls = key_class(kp);
+            v.cls_end[(cls >> 6) * sp.nC + (cls & 63)] = i;
+        }
+        if (i == A.n_pad - 1 && k) {
+            const int cls = key_class(k);
+            v.cls_end[(cls >> 6) * sp.nC + (cls & 63)] = A.n_pad;
+        }
+    }
+    // default results and the ordered list of guaranteed jobs
+    {
+        const int chunk = (J + RT - 1) / RT;
+        const int j0 = min(tid * chunk, J), j1 = min(j0 + chunk, J);
+        int cnt = 0;
+        for (int j = j0; j < j1; ++j) {
+            const int gi = A.pa[j].gi;
+            cnt += gi != -2;
+            rubick_assignment r;
+            r.g = 0; r.c = 0; r.m_bytes = 0; r.plan = -1; r.first_node = -1; r.n_nodes = 0; r.thr = 0.0f;
+            r.status = gi != -2 ? RUBICK_PENDING : RUBICK_UNALLOCATED; r.m_level = -1;
+            A.out[j] = r;
+        }
+        // exclusive scan of cnt over the block
+        int incl = cnt;
+#pragma unroll
+        for (int s = 1; s < 32; s <<= 1) { const int o = __shfl_up_sync(0xffffffffu, incl, s); if (lane >= s) incl += o; }
+        if (lane == 31) sh.scan_cnt[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            int wsum = sh.scan_cnt[lane];
+#pragma unroll
+            for (int s = 1; s < 32; s <<= 1) { const int o = __shfl_up_sync(0xffffffffu, wsum, s); if (lane >= s) wsum += o; }
+            sh.scan_cnt[lane] = wsum;
+            if (lane == 31) sh.n_guar = wsum;
+        }
+        __syncthreads();
+        int pos = incl - cnt + (warp ? sh.scan_cnt[warp - 1] : 0);
+        for (int j = j0; j < j1; ++j)
+            if (A.pa[j].gi != -2) A.glist[pos++] = j;
+    }
+    __syncthreads();
+
+    // ---- Phase A: guaranteed minima in job order (warp 0) ------------------------------------------
+    if (warp == 0) {
+        const int ng = sh.n_guar;
+        for (int base = 0; base < ng; base += 32) {
+            // lanes fetch 32 list entries at once; they are used one after another
+            const int idx = base + lane;
+            int jl = -1; int4 a0 = make_int4(-1, 0, 0, -1), a1 = make_int4(-1, 0, 0, 0);
+            if (idx < ng) {
+                jl = A.glist[idx];
+                a0 = reinterpret_cast<const int4 *>(A.pa + jl)[0];
+                a1 = reinterpret_cast<const int4 *>(A.pa + jl)[1];
+            }
+            const int cnt = min(32, ng - base);
+            for (int i = 0; i < cnt; ++i) {
+                const int j = __shfl_sync(0xffffffffu, jl, i);
+                const int gi = __shfl_sync(0xffffffffu, a0.x, i), ci = __shfl_sync(0xffffffffu, a0.y, i);
+                HotCurve cand;
+                cand.val = __int_as_float(__shfl_sync(0xffffffffu, a0.z, i));
+                cand.plan = __shfl_sync(0xffffffffu, a0.w, i);
+                cand.f = __shfl_sync(0xffffffffu, a1.x, i);
+                cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
+                const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
+                if (gi < 0) continue;
+                Committed cm;
+                if (commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm)) {
+                    const int s = sh.n_slots;
+                    if (lane == 0) {
+                        SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
+                        SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
+                        v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
+                        sh.n_slots = s + 1;
+                    }
+                    __syncwarp();
+                }
+            }
+        }
+    }
+    __syncthreads();
+    // gains of the jobs placed in Phase A
+    for (int s = tid; s < sh.n_slots; s += RT) {
+        SlotA a = v.sa[s]; const SlotB b = v.sb[s];
+        int ng_, nc_; float gg, gc;
+        gains_thread(sp, A.hc, v.sj[s], b.w, pk_gi(a.packed), pk_ci(a.packed), b.val, ng_, gg, nc_, gc);
+        a.gain_g = gg; a.gain_c = gc; a.packed = pack(pk_gi(a.packed), pk_ci(a.packed), ng_, false, false);
+        v.sa[s] = a;
+    }
+    __syncthreads();
+
+    // ---- Phase B ---------------------------------------------------------------------------------------
+    for (;;) {
+        const int n_empty = sh.n_empty, n_slots = sh.n_slots;
+        u64 best = 0ull; uint32_t pay = 0u;
+        for (int t = tid; t < n_cls; t += RT) {
+            const u64 k = v.cls_top[t];
+            if (k) {
+                const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
+                if (class_placeable(sp, v, n_empty, gi2, ci2)) {
+                    const u64 sk = sel_key(1, key_gain_bits(k), key_job(k));
+                    if (sk > best) { best = sk; pay = 0x80000000u | uint32_t(t); }
+                }
+            }
+        }
+        for (int s = tid; s < n_slots; s += RT) {
+            const SlotA a = v.sa[s];
+            const int j = v.sj[s];
+            const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+            if (a.gain_g > 0.0f) {
+                const u64 sk = sel_key(1, __float_as_uint(a.gain_g), j);
+                if (sk > best && slot_placeable(sp, v, n_empty, gi, ci, a.node, pk_next_gi(a.packed), ci)) { best = sk; pay = uint32_t(s); }
+            }
+            if (a.gain_c > 0.0f) {
+                const u64 sk = sel_key(0, __float_as_uint(a.gain_c), j);
+                if (sk > best && slot_placeable(sp, v, n_empty, gi, ci, a.node, gi, ci + 1)) { best = sk; pay = uint32_t(s); }
+            }
+        }
+#pragma unroll
+        for (int s = 16; s > 0; s >>= 1) {
+            const u64 ok = __shfl_xor_sync(0xffffffffu, best, s);
+            const uint32_t op = __shfl_xor_sync(0xffffffffu, pay, s);
+            if (ok > best) { best = ok; pay = op; }
+        }
+        if (lane == 0) { sh.red_key[warp] = best; sh.red_pay[warp] = pay; }
+        __syncthreads();
+        if (warp == 0) {
+            best = sh.red_key[lane]; pay = sh.red_pay[lane];
+#pragma unroll
+            for (int s = 16; s > 0; s >>= 1) {
+                const u64 ok = __shfl_xor_sync(0xffffffffu, best, s);
+                const uint32_t op = __shfl_xor_sync(0xffffffffu, pay, s);
+                if (ok > best) { best = ok; pay = op; }
+            }
+            bool go = best != 0ull;
+            if (go && sh.steps >= A.max_steps) { if (lane == 0) sh.capped = 1; go = false; }
+            if (go) {
+                const int type_gpu = int(best >> 63);
+                const int j = sel_job(best);
+                bool ok;
+                if (pay & 0x80000000u) {
+                    // head of a class of unallocated jobs; consumed whether or not the commit succeeds
+                    const int t = int(pay & 0x7fffffffu);
+                    const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
+                    const float w = v.cls_w[t];
+                    const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
+                    Committed cm;
+                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
+                    const int ptr = v.cls_ptr[t] + 1;
+                    u64 nk = 0ull; float nw = 0.0f;
+                    if (ptr < v.cls_end[t]) { nk = A.keys[ptr]; nw = A.sorted_w[ptr]; }
+                    if (ok) {
+                        int ng_, nc_; float gg, gc;
+                        gains_warp(sp, A.hc, j, w, gi2, ci2, cm.val, lane, ng_, gg, nc_, gc);
+                        if (lane == 0) {
+                            const int s = sh.n_slots;
+                            SlotA sa; sa.gain_g = gg; sa.gain_c = gc; sa.packed = pack(gi2, ci2, ng_, false, false); sa.node = cm.first;
+                            SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
+                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
+                            sh.n_slots = s + 1;
+                        }
+                    }
+                    if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; }
+                } else {
+                    const int s = int(pay);
+                    SlotA a = v.sa[s]; SlotB b = v.sb[s];
+                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi;
+                    const int ci2 = type_gpu ? ci : ci + 1;
+                    const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
+                    Committed cm;
+                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, true, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, lane, cm);
+                    bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+                    if (ok) {
+                        int ng_, nc_; float gg, gc;
+                        gains_warp(sp, A.hc, j, b.w, gi2, ci2, cm.val, lane, ng_, gg, nc_, gc);
+                        a.gain_g = fz_g ? 0.0f : gg; a.gain_c = fz_c ? 0.0f : gc;
+                        a.packed = pack(gi2, ci2, ng_, fz_g, fz_c); a.node = cm.first;
+                        b.val = cm.val; b.plan = cm.plan; b.f_level = cm.f;
+                    } else {
+                        if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
+                        a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
+                    }
+                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; }
+                }
+                if (lane == 0) {
+                    if (A.step_log) A.step_log[sh.steps] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
+                    sh.steps += 1;
+                }
+            }
+            if (lane == 0) sh.stop = go ? 0 : 1;
+        }
+        __syncthreads();
+        if (sh.stop) break;
+    }
+
+    // ---- results -----------------------------------------------------------------------------------------
+    for (int s = tid; s < sh.n_slots; s += RT) {
+        const SlotA a = v.sa[s]; const SlotB b = v.sb[s];
+        rubick_assignment r;
+        r.g = sp.g_levels[pk_gi(a.packed)]; r.c = sp.c_levels[pk_ci(a.packed)]; r.m_bytes = sp.m_levels[b.f_level];
+        r.plan = b.plan; r.first_node = a.node; r.n_nodes = max(r.g >> sp.log2Gn, 1);
+        r.thr = b.val; r.status = RUBICK_RUNNING; r.m_level = b.f_level;
+        A.out[v.sj[s]] = r;
+    }
+    if (A.node_out)
+        for (int n = tid; n < N; n += RT) {
+            rubick_node nd;
+            nd.free_g = v.free_g[n]; nd.free_c = v.free_c[n]; nd.free_m = v.free_m[n]; nd.owner = v.owner[n]; nd.reserved = 0;
+            A.node_out[n] = nd;
+        }
+    if (tid == 0) {
+        *A.steps_out = sh.steps;
+        if (sh.capped) atomicOr(A.status, DS_STEP_CAP);
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------------
+struct Layout {
+    int n_pad, slot_cap, slots_in_smem;
+    size_t smem, off_hc, off_keys, off_w, off_pa, off_glist, off_sa, off_sb, off_sj, total;
+};
+
+static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+static Layout make_layout(const Space &sp, int J, int N)
+{
+    Layout L;
+    int n = 2;
+    while (n < J) n <<= 1;
+    L.n_pad = n;
+    const long long gpus = (long long)N * sp.Gn;
+    L.slot_cap = int(gpus < J ? gpus : J);
+    if (L.slot_cap < 1) L.slot_cap = 1;
+    const size_t n_cls = size_t(sp.nG) * sp.nC;
+    size_t fixed = size_t(N) * 20 + n_cls * 20 + size_t(sp.n_small) * sp.nC * 4 + size_t(TOUCH_CAP) * 4;
+    fixed = (fixed + 15) & ~size_t(15);
+    const size_t slots = size_t(L.slot_cap) * (sizeof(SlotA) + sizeof(SlotB) + 4);
+    L.slots_in_smem = fixed + slots <= SMEM_LIMIT;
+    L.smem = fixed + (L.slots_in_smem ? slots : 0);
+    size_t o = 0;
+    L.off_hc = o; o = align256(o + size_t(J) * sp.nG * sp.nC * sizeof(HotCurve));
+    L.off_keys = o; o = align256(o + size_t(n) * 8);
+    L.off_w = o; o = align256(o + size_t(n) * 4);
+    L.off_pa = o; o = align256(o + size_t(J) * sizeof(PhaseA));
+    L.off_glist = o; o = align256(o + size_t(J) * 4);
+    L.off_sa = o; o = align256(o + (L.slots_in_smem ? 0 : size_t(L.slot_cap) * sizeof(SlotA)));
+    L.off_sb = o; o = align256(o + (L.slots_in_smem ? 0 : size_t(L.slot_cap) * sizeof(SlotB)));
+    L.off_sj = o; o = align256(o + (L.slots_in_smem ? 0 : size_t(L.slot_cap) * 4));
+    L.total = o;
+    return L;
+}
+
+}  // namespace fastround
+
+bool round_fast_supported(const Space &sp, int J, int N)
+{
+    using namespace fastround;
+    if (J < 1 || J >= (1 << KEY_JOB_BITS)) return false;
+    const size_t n_cls = size_t(sp.nG) * sp.nC;
+    const size_t fixed = size_t(N) * 20 + n_cls * 20 + size_t(sp.n_small) * sp.nC * 4 + size_t(TOUCH_CAP) * 4 + 16;
+    return fixed <= SMEM_LIMIT;
+}
+
+size_t round_fast_scratch_need(const Space &sp, int J, int N)
+{
+    return fastround::make_layout(sp, J, N).total;
+}
+
+cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
+                              const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
+                              rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                              void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
+{
+    using namespace fastround;
+    const Layout L = make_layout(sp, J, N);
+    unsigned char *base = static_cast<unsigned char *>(d_scratch);
+    HotCurve *hc = reinterpret_cast<HotCurve *>(base + L.off_hc);
+    u64 *keys = reinterpret_cast<u64 *>(base + L.off_keys);
+    float *sw = reinterpret_cast<float *>(base + L.off_w);
+    PhaseA *pa = reinterpret_cast<PhaseA *>(base + L.off_pa);
+
+    const long long natural = (long long)J * (sp.nG + sp.nC + 2) + 1;
+    if ((long long)max_steps > natural) max_steps = int(natural < 0x7fffffffLL ? natural : 0x7fffffffLL);
+
+    const size_t n_hc = size_t(J) * sp.nG * sp.nC;
+    round_prepare_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_cv, d_cp, d_cg, d_feas, J, hc);
+    round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa);
+    const int sort_smem = L.n_pad <= SORT_SMEM_KEYS;
+    cudaError_t e;
+    if (sort_smem && size_t(L.n_pad) * 8 > 48 * 1024) {
+        e = cudaFuncSetAttribute(round_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SORT_SMEM_KEYS * 8);
+        if (e != cudaSuccess) return e;
+    }
+    round_sort_kernel<<<1, RT, sort_smem ? size_t(L.n_pad) * 8 : 0, st>>>(keys, L.n_pad, d_jobs, sw, sort_smem);
+
+    RoundArgs A;
+    A.jobs = d_jobs; A.J = J; A.cv = d_cv; A.cp = d_cp; A.cg = d_cg; A.feas = d_feas; A.N = N; A.max_steps = max_steps;
+    A.out = d_out; A.node_out = d_node_out; A.step_log = d_step_log;
+    A.hc = hc; A.keys = keys; A.sorted_w = sw; A.n_pad = L.n_pad; A.pa = pa;
+    A.glist = reinterpret_cast<int32_t *>(base + L.off_glist);
+    A.sa_g = reinterpret_cast<SlotA *>(base + L.off_sa); A.sb_g = reinterpret_cast<SlotB *>(base + L.off_sb);
+    A.sj_g = reinterpret_cast<int32_t *>(base + L.off_sj);
+    A.slots_in_smem = L.slots_in_smem; A.slot_cap = L.slot_cap;
+    A.status = d_status; A.steps_out = d_steps;
+    e = cudaFuncSetAttribute(greedy_round_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(SMEM_LIMIT));
+    if (e != cudaSuccess) return e;
+    greedy_round_fast_kernel<<<1, RT, L.smem, st>>>(sp, A);
+    return cudaGetLastError();
+}
+
+}  // namespace rubick

@@ -50,6 +50,13 @@ enum : uint32_t {
     DS_STEP_CAP = 2u,
 };
 
+bool round_fast_supported(const Space &sp, int J, int N);
+size_t round_fast_scratch_need(const Space &sp, int J, int N);
+cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
+                              const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
+                              rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                              void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
+
 }  // namespace rubick
 
 struct rubick_ctx {
