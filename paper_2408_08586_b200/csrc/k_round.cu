@@ -15,12 +15,13 @@
 //   sort     (1 CTA)  bitonic sort of the keys: inside a class (same target levels = same placement
 //                     test) only the first unconsumed job can ever be selected.
 //   round    (1 CTA)  persistent loop.  Shared memory holds the node state, an incrementally
-//                     maintained first-fit table  node(g level, c level), the head of every class and
-//                     one 36-byte slot per RUNNING job.  A step scans class heads + running slots
-//                     (not all jobs), reduces a 64-bit key (type | gain | ~job) across the block, and
-//                     warp 0 commits: placement from the first-fit table, memory level by ballot,
-//                     node bookkeeping, table repair for the touched nodes, new gains with one
-//                     warp-wide load of the job's curve column.
+//                     maintained table "most free cores among nodes with >= g free GPUs" (a job of g GPUs
+//                     and c cores fits some node exactly when that entry is >= c), the head of every class and
+//                     one 36-byte slot per RUNNING job (scan state + placement needs).  A step scans class heads + running slots
+//                     (not all jobs), selects (type | gain, lowest job) across the block with warp reduce instructions, and
+//                     warp 0 commits: placement (own node, else first fit by a warp scan), memory level
+//                     by ballot, node bookkeeping, table rebuild, new gains from one warp-wide load of
+//                     the job's curve column issued together with the target's entry.
 //
 // All gain arithmetic uses __fmul_rn / __fsub_rn / __fdiv_rn (one rounding per operation, never
 // fused) so that decisions are reproducible bit for bit.  Every loop is bounded (steps by
@@ -33,7 +34,6 @@ namespace fastround {
 
 constexpr int RT = 1024;
 constexpr int RW = RT / 32;
-constexpr int TOUCH_CAP = 160;
 constexpr size_t SMEM_LIMIT = 200 * 1024;
 constexpr int SORT_SMEM_KEYS = 16384;
 
@@ -182,68 +182,56 @@ round_sort_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ 
 }
 
 // ---- the persistent round ---------------------------------------------------------------------------
+
+// what a slot's two candidates need in order to be placeable, precomputed when its gains are
+struct SlotC {
+    uint8_t gkind, ckind;     // K_SINGLE / K_MULTI_WHOLE / K_MULTI_PART / K_NONE
+    uint8_t gidx, cidx;       // GPU level whose "most free cores" entry decides a migration
+    int16_t dg, need, dc;     // extra GPUs on the own node / empty nodes needed / extra cores on the own node
+    int16_t c, c2, g;         // cores held, cores wanted, GPUs held
+};
+enum : uint8_t { K_SINGLE = 0, K_MULTI_WHOLE = 1, K_MULTI_PART = 2, K_NONE = 3 };
+
 struct Views {
     int64_t *free_m;
-    int32_t *free_g, *free_c, *owner, *ff, *touched;
+    int32_t *free_g, *free_c, *owner;
+    int32_t *maxc;                // [n_small] most free cores among nodes with at least g_levels[i] free GPUs, -1 if none
     int32_t *cls_ptr, *cls_end; u64 *cls_top; float *cls_w;
-    SlotA *sa; SlotB *sb; int32_t *sj;
+    int32_t *ccls;                // compact list of the non-empty classes (dense class indices)
+    SlotA *sa; SlotB *sb; SlotC *sc; int32_t *sj;
+    const int32_t *gl, *clv;      // GPU / CPU level values in shared memory (lanes index them divergently)
     int N;
 };
 
 struct Shared {
-    u64 red_key[RW];
-    uint32_t red_pay[RW];
-    int n_empty, n_slots, steps, capped, stop, nt, ff_full, n_guar;
+    uint32_t red_key[RW]; int32_t red_j[RW]; uint32_t red_pay[RW];
+    int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
     int scan_cnt[RW];
 };
 
-__device__ int first_fit_from(const Views &v, int start, int g, int c, int lane)
+// warp-cooperative: first node with at least g free GPUs and c free cores, -1 if none
+__device__ int first_fit_warp(const Views &v, int g, int c, int lane)
 {
-    for (int base = start & ~31; base < v.N; base += 32) {
+    for (int base = 0; base < v.N; base += 32) {
         const int n = base + lane;
-        const bool ok = n >= start && n < v.N && v.free_g[n] >= g && v.free_c[n] >= c;
+        const bool ok = n < v.N && v.free_g[n] >= g && v.free_c[n] >= c;
         const unsigned b = __ballot_sync(0xffffffffu, ok);
         if (b) return base + __ffs(b) - 1;
     }
     return -1;
 }
 
-// Repair the first-fit table after the nodes in v.touched[0..nt) changed (warp 0, all lanes).
-__device__ void ff_repair(const Space &sp, const Views &v, int nt, bool full, int lane)
+// warp-cooperative: rebuild maxc[] from the node state.  A job of g GPUs and c cores fits some
+// node as a whole exactly when maxc[level of g] >= c.
+__device__ void rebuild_maxc(const Space &sp, const Views &v, int lane)
 {
-    const int n_ff = sp.n_small * sp.nC;
-    for (int e0 = 0; e0 < n_ff; e0 += 32) {
-        const int e = e0 + lane;
-        const bool act = e < n_ff;
-        const int gi = act ? e / sp.nC : 0, ci = act ? e - gi * sp.nC : 0;
-        const int g = sp.g_levels[gi], c = sp.c_levels[ci];
-        int cur = act ? v.ff[e] : -1;
-        bool rescan = false;
-        int start = 0;
-        if (act) {
-            if (full) { rescan = true; start = 0; }
-            else {
-                int best_new = -1; bool lost = false;
-                for (int t = 0; t < nt; ++t) {
-                    const int n = v.touched[t];
-                    const bool fit = v.free_g[n] >= g && v.free_c[n] >= c;
-                    if (fit) { if (best_new < 0 || n < best_new) best_new = n; }
-                    else if (n == cur) lost = true;
-                }
-                if (best_new >= 0 && (cur < 0 || best_new < cur)) cur = best_new;
-                else if (lost) { rescan = true; start = cur + 1; }
-            }
-        }
-        unsigned need = __ballot_sync(0xffffffffu, rescan);
-        while (need) {
-            const int src = __ffs(need) - 1;
-            need &= need - 1;
-            const int g2 = __shfl_sync(0xffffffffu, g, src), c2 = __shfl_sync(0xffffffffu, c, src);
-            const int st = __shfl_sync(0xffffffffu, start, src);
-            const int r = first_fit_from(v, st, g2, c2, lane);
-            if (lane == src) cur = r;
-        }
-        if (act) v.ff[e] = cur;
+    for (int gi = 0; gi < sp.n_small; ++gi) {
+        const int g = sp.g_levels[gi];
+        int m = -1;
+        for (int n = lane; n < v.N; n += 32)
+            if (v.free_g[n] >= g) m = max(m, v.free_c[n]);
+        m = __reduce_max_sync(0xffffffffu, m);
+        if (lane == 0) v.maxc[gi] = m;
     }
     __syncwarp();
 }
@@ -252,8 +240,7 @@ struct Committed { int first; float val; int plan; int f; };
 
 // Commit job j to (gi2, ci2); warp 0, all lanes, uniform control flow.  `alloc`: the job holds
 // (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target
-// at the top memory level.  On success the node state, the touched list, the empty-node count and
-// the first-fit table are up to date.
+// at the top memory level.  On success the node state, the empty-node count and maxc[] are current.
 __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const float *__restrict__ cv,
                             const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
                             const uint32_t *__restrict__ feas, int j, bool alloc, int gi, int ci, int node,
@@ -270,7 +257,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     bool stay = false;
     if (g2 <= sp.Gn) {
         if (alloc && v.free_g[node] >= g2 - g && v.free_c[node] >= c2 - c) { stay = true; target = node; }
-        else target = v.ff[gi2 * sp.nC + ci2];
+        else if (v.maxc[gi2] >= c2) target = first_fit_warp(v, g2, c2, lane);
         if (target < 0) return false;
     } else {
         k2 = g2 >> sp.log2Gn;
@@ -283,8 +270,9 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         }
     }
 
+    // highest memory level whose per-node share fits: ceil(m / k2) <= avail  <=>  m <= avail * k2
     const int64_t avail = k2 > 1 ? sp.Mn : v.free_m[target] + ((stay && alloc) ? m_cur : 0);
-    const bool fits = lane < sp.nM && cdiv64(sp.m_levels[lane < sp.nM ? lane : 0], k2) <= avail;
+    const bool fits = lane < sp.nM && sp.m_levels[lane < sp.nM ? lane : 0] <= avail * k2;
     const unsigned fb = __ballot_sync(0xffffffffu, fits);
     if (!fb) return false;
     const int mi = 31 - __clz(fb);
@@ -304,49 +292,37 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     if (f < 0 || f > mi) return false;
     const int64_t m2 = sp.m_levels[f];
 
-    // ---- node bookkeeping; every changed node goes on the touched list ---------------------------
-    int first = -1, nt = 0, d_empty = 0;
-    bool full = false;
+    // ---- node bookkeeping ------------------------------------------------------------------------
+    int first = -1, d_empty = 0;
     if (k2 == 1) {
         if (lane == 0) {
-            if (alloc && !stay) {
-                v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur;
-                v.touched[nt] = node;
-            }
             if (stay) { v.free_g[target] -= g2 - g; v.free_c[target] -= c2 - c; v.free_m[target] -= m2 - m_cur; }
-            else { v.free_g[target] -= g2; v.free_c[target] -= c2; v.free_m[target] -= m2; }
+            else {
+                if (alloc) { v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur; }
+                v.free_g[target] -= g2; v.free_c[target] -= c2; v.free_m[target] -= m2;
+            }
         }
         __syncwarp();
-        if (alloc && !stay) { nt = 1; if (v.free_g[node] == sp.Gn) d_empty += 1; }
+        if (alloc && !stay && v.free_g[node] == sp.Gn) d_empty += 1;
         if (!stay && v.free_g[target] + g2 == sp.Gn) d_empty -= 1;
-        if (lane == 0) v.touched[nt] = target;
-        nt += 1;
         first = target;
     } else {
         const int cs2 = (c2 + k2 - 1) / k2;
         const int64_t ms2 = cdiv64(m2, k2);
         if (stay) {
+            // whole nodes already held keep their GPUs; only the core / memory shares change
             const int cs1 = (c + k - 1) / k;
             const int64_t ms1 = cdiv64(m_cur, k);
             if (k == 1) {
-                if (lane == 0) { v.free_c[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; v.touched[0] = node; }
-                nt = 1;
+                if (lane == 0) { v.free_c[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; }
             } else {
-                // cores only: GPU levels above a node change the node count, so this is a CPU step
-                for (int base = 0; base < v.N; base += 32) {
-                    const int n = base + lane;
-                    const bool mine = n < v.N && v.owner[n] == j;
-                    if (mine) { v.free_c[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
-                    const unsigned b = __ballot_sync(0xffffffffu, mine);
-                    if (mine) { const int pos = nt + __popc(b & ((1u << lane) - 1u)); if (pos < TOUCH_CAP) v.touched[pos] = n; }
-                    nt += __popc(b);
-                }
+                for (int n = lane; n < v.N; n += 32)
+                    if (v.owner[n] == j) { v.free_c[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
             }
             first = node;
         } else if (alloc) {
-            if (lane == 0) { v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur; v.touched[0] = node; }
+            if (lane == 0) { v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur; }
             __syncwarp();
-            nt = 1;
             if (v.free_g[node] == sp.Gn) d_empty += 1;
         }
         __syncwarp();
@@ -356,40 +332,31 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
             const bool empty = n < v.N && v.free_g[n] == sp.Gn;
             const unsigned b = __ballot_sync(0xffffffffu, empty);
             const int rank = __popc(b & ((1u << lane) - 1u));
-            if (empty && taken + rank < need_new) {
-                v.free_g[n] = 0; v.free_c[n] -= cs2; v.free_m[n] -= ms2; v.owner[n] = j;
-                const int pos = nt + rank;
-                if (pos < TOUCH_CAP) v.touched[pos] = n;
-            }
+            if (empty && taken + rank < need_new) { v.free_g[n] = 0; v.free_c[n] -= cs2; v.free_m[n] -= ms2; v.owner[n] = j; }
             if (b) { const int lowest = base + __ffs(b) - 1; if (first < 0 || lowest < first) first = lowest; }
-            const int got = min(__popc(b), need_new - taken);
-            taken += got; nt += got;
+            taken += __popc(b);
         }
         d_empty -= need_new;
-        if (nt > TOUCH_CAP) full = true;
     }
     __syncwarp();
     if (lane == 0) sh.n_empty = n_empty + d_empty;
-    ff_repair(sp, v, nt, full, lane);
+    rebuild_maxc(sp, v, lane);
     out.first = first; out.val = val; out.plan = plan; out.f = f;
     return true;
 }
 
-// New gains of a running job (warp-wide): one load per GPU level above the present one.
-__device__ void gains_warp(const Space &sp, const HotCurve *__restrict__ hc, int j, float w, int gi, int ci, float val,
-                           int lane, int &next_g, float &gain_g, int &next_c, float &gain_c)
+// gains of a running job from the values of its curve column (lane i holds the value of GPU level
+// gi + 1 + i, vc the value at the next core level); identical on every lane
+__device__ __forceinline__ void gains_from_column(const Space &sp, float w, int gi, int ci, float val, float v_lane,
+                                                  float vc, int lane, int &next_g, float &gain_g, int &next_c, float &gain_c)
 {
     const float vcur = __fmul_rn(w, val);
     const int lvl = gi + 1 + lane;
-    float v = 0.0f;
-    if (lvl < sp.nG) v = hc[hc_idx(sp, j, lvl, ci)].val;
-    float vc = 0.0f;
-    if (ci + 1 < sp.nC) vc = hc[hc_idx(sp, j, gi, ci + 1)].val;
-    const unsigned b = __ballot_sync(0xffffffffu, lvl < sp.nG && v > val);
+    const unsigned b = __ballot_sync(0xffffffffu, lvl < sp.nG && v_lane > val);
     next_g = -1; gain_g = 0.0f; next_c = -1; gain_c = 0.0f;
     if (b) {
         const int src = __ffs(b) - 1;
-        const float vv = __shfl_sync(0xffffffffu, v, src);
+        const float vv = __shfl_sync(0xffffffffu, v_lane, src);
         next_g = gi + 1 + src;
         gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, vv), vcur), float(sp.g_levels[next_g] - sp.g_levels[gi]));
     }
@@ -420,25 +387,37 @@ __device__ void gains_thread(const Space &sp, const HotCurve *__restrict__ hc, i
     }
 }
 
-__device__ __forceinline__ bool slot_placeable(const Space &sp, const Views &v, int n_empty, int gi, int ci, int node,
-                                               int gi2, int ci2)
+// placement requirements of a slot's candidates (see SlotC)
+__device__ SlotC make_slotc(const Space &sp, int gi, int ci, int next_g, int next_c)
 {
-    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    SlotC s;
     const int g = sp.g_levels[gi], c = sp.c_levels[ci];
-    if (g2 <= sp.Gn) {
-        if (v.free_g[node] >= g2 - g && v.free_c[node] >= c2 - c) return true;
-        return v.ff[gi2 * sp.nC + ci2] >= 0;
+    s.gkind = K_NONE; s.ckind = K_NONE; s.gidx = 0; s.cidx = uint8_t(gi < sp.n_small ? gi : 0);
+    s.dg = 0; s.need = 0; s.dc = 0; s.c = int16_t(c); s.c2 = 0; s.g = int16_t(g);
+    if (next_g >= 0) {
+        const int g2 = sp.g_levels[next_g];
+        if (g2 <= sp.Gn) { s.gkind = K_SINGLE; s.dg = int16_t(g2 - g); s.gidx = uint8_t(next_g); }
+        else {
+            const int k2 = g2 >> sp.log2Gn;
+            if ((c + k2 - 1) / k2 <= sp.Cn) {
+                if (g >= sp.Gn) { s.gkind = K_MULTI_WHOLE; s.need = int16_t(k2 - (g >> sp.log2Gn)); }
+                else { s.gkind = K_MULTI_PART; s.need = int16_t(k2); }
+            }
+        }
     }
-    const int k2 = g2 >> sp.log2Gn;
-    if ((c2 + k2 - 1) / k2 > sp.Cn) return false;
-    if (g >= sp.Gn) return n_empty >= k2 - (g >> sp.log2Gn);
-    return n_empty + ((v.free_g[node] + g == sp.Gn) ? 1 : 0) >= k2;
+    if (next_c >= 0) {
+        const int c2 = sp.c_levels[next_c];
+        s.c2 = int16_t(c2);
+        if (g <= sp.Gn) { s.ckind = K_SINGLE; s.dc = int16_t(c2 - c); }
+        else { const int k = g >> sp.log2Gn; if ((c2 + k - 1) / k <= sp.Cn) s.ckind = K_MULTI_WHOLE; }
+    }
+    return s;
 }
 
 __device__ __forceinline__ bool class_placeable(const Space &sp, const Views &v, int n_empty, int gi2, int ci2)
 {
-    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
-    if (g2 <= sp.Gn) return v.ff[gi2 * sp.nC + ci2] >= 0;
+    const int g2 = v.gl[gi2], c2 = v.clv[ci2];
+    if (g2 <= sp.Gn) return v.maxc[gi2] >= c2;
     const int k2 = g2 >> sp.log2Gn;
     return (c2 + k2 - 1) / k2 <= sp.Cn && n_empty >= k2;
 }
@@ -450,9 +429,23 @@ struct RoundArgs {
     rubick_assignment *out; rubick_node *node_out; int32_t *step_log;
     const HotCurve *hc; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
     int32_t *glist;
-    SlotA *sa_g; SlotB *sb_g; int32_t *sj_g; int slots_in_smem; int slot_cap;
+    SlotA *sa_g; SlotB *sb_g; SlotC *sc_g; int32_t *sj_g; int slots_in_smem; int slot_cap;
     uint32_t *status; int32_t *steps_out;
 };
+
+constexpr int SLOT_BYTES = int(sizeof(SlotA) + sizeof(SlotC)) + 4;     // per running job in shared memory
+
+// block-wide selection: largest key32, lowest job among equal keys.  Per-thread triple in, the
+// winner (key 0 = none) out on every lane of warp 0.
+__device__ __forceinline__ void warp_select(uint32_t &key, int &j, uint32_t &pay)
+{
+    const uint32_t m = __reduce_max_sync(0xffffffffu, key);
+    const int jm = __reduce_min_sync(0xffffffffu, (key == m && m) ? j : 0x7fffffff);
+    const unsigned b = __ballot_sync(0xffffffffu, key == m && j == jm);
+    const int src = b ? __ffs(b) - 1 : 0;
+    pay = __shfl_sync(0xffffffffu, pay, src);
+    key = m; j = jm;
+}
 
 __global__ void __launch_bounds__(RT, 1)
 greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant__ RoundArgs A)
@@ -461,7 +454,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     __shared__ Shared sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
-    const int n_ff = sp.n_small * sp.nC, n_cls = sp.nG * sp.nC;
+    const int n_cls = sp.nG * sp.nC;
 
     Views v;
     v.N = N;
@@ -471,23 +464,29 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     v.free_g = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
     v.free_c = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
     v.owner = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
-    v.ff = reinterpret_cast<int32_t *>(p); p += size_t(n_ff) * 4;
-    v.touched = reinterpret_cast<int32_t *>(p); p += size_t(TOUCH_CAP) * 4;
     v.cls_ptr = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
     v.cls_end = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
     v.cls_w = reinterpret_cast<float *>(p); p += size_t(n_cls) * 4;
+    v.ccls = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
+    v.maxc = reinterpret_cast<int32_t *>(p); p += size_t(RUBICK_MAX_G_LEVELS) * 4;
+    int32_t *gl_s = reinterpret_cast<int32_t *>(p); p += size_t(RUBICK_MAX_G_LEVELS) * 4;
+    int32_t *cl_s = reinterpret_cast<int32_t *>(p); p += size_t(RUBICK_MAX_C_LEVELS) * 4;
+    v.gl = gl_s; v.clv = cl_s;
     p = smem_raw + ((size_t(p - smem_raw) + 15) & ~size_t(15));
     if (A.slots_in_smem) {
         v.sa = reinterpret_cast<SlotA *>(p); p += size_t(A.slot_cap) * sizeof(SlotA);
-        v.sb = reinterpret_cast<SlotB *>(p); p += size_t(A.slot_cap) * sizeof(SlotB);
+        v.sc = reinterpret_cast<SlotC *>(p); p += size_t(A.slot_cap) * sizeof(SlotC);
         v.sj = reinterpret_cast<int32_t *>(p);
-    } else { v.sa = A.sa_g; v.sb = A.sb_g; v.sj = A.sj_g; }
+    } else { v.sa = A.sa_g; v.sc = A.sc_g; v.sj = A.sj_g; }
+    v.sb = A.sb_g;          // value / plan / memory level / weight: touched only by commits, kept in global memory
 
     // ---- set-up ---------------------------------------------------------------------------------
     for (int n = tid; n < N; n += RT) { v.free_g[n] = sp.Gn; v.free_c[n] = sp.Cn; v.free_m[n] = sp.Mn; v.owner[n] = -1; }
-    for (int e = tid; e < n_ff; e += RT) v.ff[e] = 0;                      // every node is empty
     for (int t = tid; t < n_cls; t += RT) { v.cls_ptr[t] = 0; v.cls_end[t] = 0; v.cls_top[t] = 0ull; v.cls_w[t] = 0.0f; }
-    if (tid == 0) { sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; }
+    if (tid < sp.nG) gl_s[tid] = sp.g_levels[tid];
+    if (tid < sp.nC) cl_s[tid] = sp.c_levels[tid];
+    if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
+    if (tid == 0) { sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0; }
     __syncthreads();
 
     // class segments of the sorted keys: a class starts where the class field changes
@@ -521,7 +520,6 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             r.status = gi != -2 ? RUBICK_PENDING : RUBICK_UNALLOCATED; r.m_level = -1;
             A.out[j] = r;
         }
-        // exclusive scan of cnt over the block
         int incl = cnt;
 #pragma unroll
         for (int s = 1; s < 32; s <<= 1) { const int o = __shfl_up_sync(0xffffffffu, incl, s); if (lane >= s) incl += o; }
@@ -533,6 +531,16 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             for (int s = 1; s < 32; s <<= 1) { const int o = __shfl_up_sync(0xffffffffu, wsum, s); if (lane >= s) wsum += o; }
             sh.scan_cnt[lane] = wsum;
             if (lane == 31) sh.n_guar = wsum;
+            // compact list of the classes that have members
+            int n_c = 0;
+            for (int base = 0; base < n_cls; base += 32) {
+                const int t = base + lane;
+                const bool has = t < n_cls && v.cls_top[t] != 0ull;
+                const unsigned b = __ballot_sync(0xffffffffu, has);
+                if (has) v.ccls[n_c + __popc(b & ((1u << lane) - 1u))] = t;
+                n_c += __popc(b);
+            }
+            if (lane == 0) sh.n_ccls = n_c;
         }
         __syncthreads();
         int pos = incl - cnt + (warp ? sh.scan_cnt[warp - 1] : 0);
@@ -586,77 +594,86 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         gains_thread(sp, A.hc, v.sj[s], b.w, pk_gi(a.packed), pk_ci(a.packed), b.val, ng_, gg, nc_, gc);
         a.gain_g = gg; a.gain_c = gc; a.packed = pack(pk_gi(a.packed), pk_ci(a.packed), ng_, false, false);
         v.sa[s] = a;
+        v.sc[s] = make_slotc(sp, pk_gi(a.packed), pk_ci(a.packed), ng_, nc_);
     }
     __syncthreads();
 
     // ---- Phase B ---------------------------------------------------------------------------------------
     for (;;) {
-        const int n_empty = sh.n_empty, n_slots = sh.n_slots;
-        u64 best = 0ull; uint32_t pay = 0u;
-        for (int t = tid; t < n_cls; t += RT) {
+        const int n_empty = sh.n_empty, n_slots = sh.n_slots, n_ccls = sh.n_ccls;
+        uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
+        for (int i = tid; i < n_ccls; i += RT) {
+            const int t = v.ccls[i];
             const u64 k = v.cls_top[t];
             if (k) {
                 const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
-                if (class_placeable(sp, v, n_empty, gi2, ci2)) {
-                    const u64 sk = sel_key(1, key_gain_bits(k), key_job(k));
-                    if (sk > best) { best = sk; pay = 0x80000000u | uint32_t(t); }
+                const uint32_t k32 = 0x80000000u | key_gain_bits(k);
+                const int j = key_job(k);
+                if ((k32 > best || (k32 == best && j < best_j)) && class_placeable(sp, v, n_empty, gi2, ci2)) {
+                    best = k32; best_j = j; pay = 0x80000000u | uint32_t(t);
                 }
             }
         }
         for (int s = tid; s < n_slots; s += RT) {
             const SlotA a = v.sa[s];
+            const SlotC q = v.sc[s];
             const int j = v.sj[s];
-            const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
             if (a.gain_g > 0.0f) {
-                const u64 sk = sel_key(1, __float_as_uint(a.gain_g), j);
-                if (sk > best && slot_placeable(sp, v, n_empty, gi, ci, a.node, pk_next_gi(a.packed), ci)) { best = sk; pay = uint32_t(s); }
+                const uint32_t k32 = 0x80000000u | __float_as_uint(a.gain_g);
+                if (k32 > best || (k32 == best && j < best_j)) {
+                    bool ok;
+                    if (q.gkind == K_SINGLE) ok = v.free_g[a.node] >= q.dg || v.maxc[q.gidx] >= q.c;
+                    else if (q.gkind == K_MULTI_WHOLE) ok = n_empty >= q.need;
+                    else if (q.gkind == K_MULTI_PART) ok = n_empty + (v.free_g[a.node] + q.g == sp.Gn ? 1 : 0) >= q.need;
+                    else ok = false;
+                    if (ok) { best = k32; best_j = j; pay = uint32_t(s); }
+                }
             }
             if (a.gain_c > 0.0f) {
-                const u64 sk = sel_key(0, __float_as_uint(a.gain_c), j);
-                if (sk > best && slot_placeable(sp, v, n_empty, gi, ci, a.node, gi, ci + 1)) { best = sk; pay = uint32_t(s); }
+                const uint32_t k32 = __float_as_uint(a.gain_c);
+                if (k32 > best || (k32 == best && j < best_j)) {
+                    bool ok;
+                    if (q.ckind == K_SINGLE) ok = v.free_c[a.node] >= q.dc || v.maxc[q.cidx] >= q.c2;
+                    else ok = q.ckind == K_MULTI_WHOLE;
+                    if (ok) { best = k32; best_j = j; pay = uint32_t(s); }
+                }
             }
         }
-#pragma unroll
-        for (int s = 16; s > 0; s >>= 1) {
-            const u64 ok = __shfl_xor_sync(0xffffffffu, best, s);
-            const uint32_t op = __shfl_xor_sync(0xffffffffu, pay, s);
-            if (ok > best) { best = ok; pay = op; }
-        }
-        if (lane == 0) { sh.red_key[warp] = best; sh.red_pay[warp] = pay; }
+        warp_select(best, best_j, pay);
+        if (lane == 0) { sh.red_key[warp] = best; sh.red_j[warp] = best_j; sh.red_pay[warp] = pay; }
         __syncthreads();
         if (warp == 0) {
-            best = sh.red_key[lane]; pay = sh.red_pay[lane];
-#pragma unroll
-            for (int s = 16; s > 0; s >>= 1) {
-                const u64 ok = __shfl_xor_sync(0xffffffffu, best, s);
-                const uint32_t op = __shfl_xor_sync(0xffffffffu, pay, s);
-                if (ok > best) { best = ok; pay = op; }
-            }
-            bool go = best != 0ull;
+            best = sh.red_key[lane]; best_j = sh.red_j[lane]; pay = sh.red_pay[lane];
+            warp_select(best, best_j, pay);
+            bool go = best != 0u;
             if (go && sh.steps >= A.max_steps) { if (lane == 0) sh.capped = 1; go = false; }
             if (go) {
-                const int type_gpu = int(best >> 63);
-                const int j = sel_job(best);
+                const int type_gpu = int(best >> 31);
+                const int j = best_j;
                 bool ok;
                 if (pay & 0x80000000u) {
                     // head of a class of unallocated jobs; consumed whether or not the commit succeeds
                     const int t = int(pay & 0x7fffffffu);
                     const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
                     const float w = v.cls_w[t];
+                    // one round trip: the target's entry and the column the new gains will need
                     const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                    Committed cm;
-                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
+                    const int lvl = gi2 + 1 + lane;
+                    const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
+                    const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
                     const int ptr = v.cls_ptr[t] + 1;
                     u64 nk = 0ull; float nw = 0.0f;
                     if (ptr < v.cls_end[t]) { nk = A.keys[ptr]; nw = A.sorted_w[ptr]; }
+                    Committed cm;
+                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
                     if (ok) {
                         int ng_, nc_; float gg, gc;
-                        gains_warp(sp, A.hc, j, w, gi2, ci2, cm.val, lane, ng_, gg, nc_, gc);
+                        gains_from_column(sp, w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
                         if (lane == 0) {
                             const int s = sh.n_slots;
                             SlotA sa; sa.gain_g = gg; sa.gain_c = gc; sa.packed = pack(gi2, ci2, ng_, false, false); sa.node = cm.first;
                             SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
-                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
+                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j; v.sc[s] = make_slotc(sp, gi2, ci2, ng_, nc_);
                             sh.n_slots = s + 1;
                         }
                     }
@@ -668,15 +685,19 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi;
                     const int ci2 = type_gpu ? ci : ci + 1;
                     const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
+                    const int lvl = gi2 + 1 + lane;
+                    const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
+                    const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
                     Committed cm;
                     ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, true, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, lane, cm);
                     bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                     if (ok) {
                         int ng_, nc_; float gg, gc;
-                        gains_warp(sp, A.hc, j, b.w, gi2, ci2, cm.val, lane, ng_, gg, nc_, gc);
+                        gains_from_column(sp, b.w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
                         a.gain_g = fz_g ? 0.0f : gg; a.gain_c = fz_c ? 0.0f : gc;
                         a.packed = pack(gi2, ci2, ng_, fz_g, fz_c); a.node = cm.first;
                         b.val = cm.val; b.plan = cm.plan; b.f_level = cm.f;
+                        if (lane == 0) v.sc[s] = make_slotc(sp, gi2, ci2, ng_, nc_);
                     } else {
                         if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
                         a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
@@ -718,10 +739,17 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
 // ---- host side ------------------------------------------------------------------------------------------
 struct Layout {
     int n_pad, slot_cap, slots_in_smem;
-    size_t smem, off_hc, off_keys, off_w, off_pa, off_glist, off_sa, off_sb, off_sj, total;
+    size_t smem, off_hc, off_keys, off_w, off_pa, off_glist, off_sa, off_sb, off_sc, off_sj, total;
 };
 
 static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+static size_t fixed_smem(const Space &sp, int N)
+{
+    const size_t n_cls = size_t(sp.nG) * sp.nC;
+    const size_t fixed = size_t(N) * 20 + n_cls * 24 + size_t(2 * RUBICK_MAX_G_LEVELS + RUBICK_MAX_C_LEVELS) * 4;
+    return (fixed + 15) & ~size_t(15);
+}
 
 static Layout make_layout(const Space &sp, int J, int N)
 {
@@ -732,21 +760,21 @@ static Layout make_layout(const Space &sp, int J, int N)
     const long long gpus = (long long)N * sp.Gn;
     L.slot_cap = int(gpus < J ? gpus : J);
     if (L.slot_cap < 1) L.slot_cap = 1;
-    const size_t n_cls = size_t(sp.nG) * sp.nC;
-    size_t fixed = size_t(N) * 20 + n_cls * 20 + size_t(sp.n_small) * sp.nC * 4 + size_t(TOUCH_CAP) * 4;
-    fixed = (fixed + 15) & ~size_t(15);
-    const size_t slots = size_t(L.slot_cap) * (sizeof(SlotA) + sizeof(SlotB) + 4);
+    const size_t fixed = fixed_smem(sp, N);
+    const size_t slots = size_t(L.slot_cap) * SLOT_BYTES;
     L.slots_in_smem = fixed + slots <= SMEM_LIMIT;
     L.smem = fixed + (L.slots_in_smem ? slots : 0);
+    const size_t gs = L.slots_in_smem ? 0 : size_t(L.slot_cap);
     size_t o = 0;
     L.off_hc = o; o = align256(o + size_t(J) * sp.nG * sp.nC * sizeof(HotCurve));
     L.off_keys = o; o = align256(o + size_t(n) * 8);
     L.off_w = o; o = align256(o + size_t(n) * 4);
     L.off_pa = o; o = align256(o + size_t(J) * sizeof(PhaseA));
     L.off_glist = o; o = align256(o + size_t(J) * 4);
-    L.off_sa = o; o = align256(o + (L.slots_in_smem ? 0 : size_t(L.slot_cap) * sizeof(SlotA)));
-    L.off_sb = o; o = align256(o + (L.slots_in_smem ? 0 : size_t(L.slot_cap) * sizeof(SlotB)));
-    L.off_sj = o; o = align256(o + (L.slots_in_smem ? 0 : size_t(L.slot_cap) * 4));
+    L.off_sa = o; o = align256(o + gs * sizeof(SlotA));
+    L.off_sb = o; o = align256(o + size_t(L.slot_cap) * sizeof(SlotB));
+    L.off_sc = o; o = align256(o + gs * sizeof(SlotC));
+    L.off_sj = o; o = align256(o + gs * 4);
     L.total = o;
     return L;
 }
@@ -757,9 +785,8 @@ bool round_fast_supported(const Space &sp, int J, int N)
 {
     using namespace fastround;
     if (J < 1 || J >= (1 << KEY_JOB_BITS)) return false;
-    const size_t n_cls = size_t(sp.nG) * sp.nC;
-    const size_t fixed = size_t(N) * 20 + n_cls * 20 + size_t(sp.n_small) * sp.nC * 4 + size_t(TOUCH_CAP) * 4 + 16;
-    return fixed <= SMEM_LIMIT;
+    if (sp.Cn > 32767 || sp.g_levels[sp.nG - 1] > 32767 || sp.c_levels[sp.nC - 1] > 32767) return false;   // SlotC holds int16
+    return fixed_smem(sp, N) <= SMEM_LIMIT;
 }
 
 size_t round_fast_scratch_need(const Space &sp, int J, int N)
@@ -800,7 +827,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     A.hc = hc; A.keys = keys; A.sorted_w = sw; A.n_pad = L.n_pad; A.pa = pa;
     A.glist = reinterpret_cast<int32_t *>(base + L.off_glist);
     A.sa_g = reinterpret_cast<SlotA *>(base + L.off_sa); A.sb_g = reinterpret_cast<SlotB *>(base + L.off_sb);
-    A.sj_g = reinterpret_cast<int32_t *>(base + L.off_sj);
+    A.sc_g = reinterpret_cast<SlotC *>(base + L.off_sc); A.sj_g = reinterpret_cast<int32_t *>(base + L.off_sj);
     A.slots_in_smem = L.slots_in_smem; A.slot_cap = L.slot_cap;
     A.status = d_status; A.steps_out = d_steps;
     e = cudaFuncSetAttribute(greedy_round_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(SMEM_LIMIT));
