@@ -244,8 +244,8 @@ struct Committed { int first; float val; int plan; int f; };
 __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const float *__restrict__ cv,
                             const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
                             const uint32_t *__restrict__ feas, int j, bool alloc, int gi, int ci, int node,
-                            float val_cur, int f_cur, int gi2, int ci2, HotCurve cand, bool need_gain, int lane,
-                            Committed &out)
+                            float val_cur, int f_cur, int gi2, int ci2, HotCurve cand, bool need_gain, bool rebuild,
+                            int lane, Committed &out)
 {
     const int g = alloc ? sp.g_levels[gi] : 0, c = alloc ? sp.c_levels[ci] : 0;
     const int64_t m_cur = alloc ? sp.m_levels[f_cur] : 0;
@@ -340,7 +340,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     }
     __syncwarp();
     if (lane == 0) sh.n_empty = n_empty + d_empty;
-    rebuild_maxc(sp, v, lane);
+    if (rebuild) rebuild_maxc(sp, v, lane);
     out.first = first; out.val = val; out.plan = plan; out.f = f;
     return true;
 }
@@ -537,7 +537,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 const int t = base + lane;
                 const bool has = t < n_cls && v.cls_top[t] != 0ull;
                 const unsigned b = __ballot_sync(0xffffffffu, has);
-                if (has) v.ccls[n_c + __popc(b & ((1u << lane) - 1u))] = t;
+                if (has) v.ccls[n_c + __popc(b & ((1u << lane) - 1u))] = t | ((t / sp.nC) << 16) | ((t % sp.nC) << 24);
                 n_c += __popc(b);
             }
             if (lane == 0) sh.n_ccls = n_c;
@@ -573,7 +573,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
                 if (gi < 0) continue;
                 Committed cm;
-                if (commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm)) {
+                if (commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, true, lane, cm)) {
                     const int s = sh.n_slots;
                     if (lane == 0) {
                         SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
@@ -600,13 +600,23 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
 
     // ---- Phase B ---------------------------------------------------------------------------------------
     for (;;) {
+        // most free cores among the nodes with >= g free GPUs: one warp per small GPU level
+        if (warp < sp.n_small) {
+            const int g = sp.g_levels[warp];
+            int m = -1;
+#pragma unroll 4
+            for (int n = lane; n < N; n += 32) m = max(m, v.free_g[n] >= g ? v.free_c[n] : -1);
+            m = __reduce_max_sync(0xffffffffu, m);
+            if (lane == 0) v.maxc[warp] = m;
+        }
+        __syncthreads();
         const int n_empty = sh.n_empty, n_slots = sh.n_slots, n_ccls = sh.n_ccls;
         uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
         for (int i = tid; i < n_ccls; i += RT) {
-            const int t = v.ccls[i];
+            const int packed = v.ccls[i];
+            const int t = packed & 0xffff, gi2 = (packed >> 16) & 0xff, ci2 = (packed >> 24) & 0xff;
             const u64 k = v.cls_top[t];
             if (k) {
-                const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
                 const uint32_t k32 = 0x80000000u | key_gain_bits(k);
                 const int j = key_job(k);
                 if ((k32 > best || (k32 == best && j < best_j)) && class_placeable(sp, v, n_empty, gi2, ci2)) {
@@ -618,26 +628,17 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             const SlotA a = v.sa[s];
             const SlotC q = v.sc[s];
             const int j = v.sj[s];
-            if (a.gain_g > 0.0f) {
-                const uint32_t k32 = 0x80000000u | __float_as_uint(a.gain_g);
-                if (k32 > best || (k32 == best && j < best_j)) {
-                    bool ok;
-                    if (q.gkind == K_SINGLE) ok = v.free_g[a.node] >= q.dg || v.maxc[q.gidx] >= q.c;
-                    else if (q.gkind == K_MULTI_WHOLE) ok = n_empty >= q.need;
-                    else if (q.gkind == K_MULTI_PART) ok = n_empty + (v.free_g[a.node] + q.g == sp.Gn ? 1 : 0) >= q.need;
-                    else ok = false;
-                    if (ok) { best = k32; best_j = j; pay = uint32_t(s); }
-                }
-            }
-            if (a.gain_c > 0.0f) {
-                const uint32_t k32 = __float_as_uint(a.gain_c);
-                if (k32 > best || (k32 == best && j < best_j)) {
-                    bool ok;
-                    if (q.ckind == K_SINGLE) ok = v.free_c[a.node] >= q.dc || v.maxc[q.cidx] >= q.c2;
-                    else ok = q.ckind == K_MULTI_WHOLE;
-                    if (ok) { best = k32; best_j = j; pay = uint32_t(s); }
-                }
-            }
+            const int fg = v.free_g[a.node], fc = v.free_c[a.node];
+            const int mg = v.maxc[q.gidx], mc = v.maxc[q.cidx];
+            const bool part_empty = fg + q.g == sp.Gn;
+            const bool ok_g = a.gain_g > 0.0f
+                              && (q.gkind == K_SINGLE ? (fg >= q.dg || mg >= q.c)
+                                  : q.gkind == K_MULTI_WHOLE ? n_empty >= q.need
+                                  : q.gkind == K_MULTI_PART ? n_empty + int(part_empty) >= q.need : false);
+            const bool ok_c = a.gain_c > 0.0f && (q.ckind == K_SINGLE ? (fc >= q.dc || mc >= q.c2) : q.ckind == K_MULTI_WHOLE);
+            // a GPU increment outranks any CPU increment
+            const uint32_t k32 = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : ok_c ? __float_as_uint(a.gain_c) : 0u;
+            if (k32 > best || (k32 == best && k32 && j < best_j)) { best = k32; best_j = j; pay = uint32_t(s); }
         }
         warp_select(best, best_j, pay);
         if (lane == 0) { sh.red_key[warp] = best; sh.red_j[warp] = best_j; sh.red_pay[warp] = pay; }
@@ -665,7 +666,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     u64 nk = 0ull; float nw = 0.0f;
                     if (ptr < v.cls_end[t]) { nk = A.keys[ptr]; nw = A.sorted_w[ptr]; }
                     Committed cm;
-                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
+                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, false, lane, cm);
                     if (ok) {
                         int ng_, nc_; float gg, gc;
                         gains_from_column(sp, w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
@@ -689,7 +690,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
                     const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
                     Committed cm;
-                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, true, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, lane, cm);
+                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, true, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, false, lane, cm);
                     bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                     if (ok) {
                         int ng_, nc_; float gg, gc;
