@@ -192,55 +192,73 @@ struct SlotC {
 };
 enum : uint8_t { K_SINGLE = 0, K_MULTI_WHOLE = 1, K_MULTI_PART = 2, K_NONE = 3 };
 
+constexpr int SCAN_WARPS = RW - 1;          // warps 0 .. 30 scan running jobs, warp 31 the class heads
+constexpr int SCAN_T = SCAN_WARPS * 32;
+
+// node n: gc[n] = free GPUs << 16 | free cores (padding entries are 0: they never fit anything)
+__device__ __forceinline__ int fg_of(int w) { return w >> 16; }
+__device__ __forceinline__ int fc_of(int w) { return w & 0xffff; }
+
 struct Views {
     int64_t *free_m;
-    int32_t *free_g, *free_c, *owner;
+    int32_t *gc, *owner;
     int32_t *maxc;                // [n_small] most free cores among nodes with at least g_levels[i] free GPUs, -1 if none
     int32_t *cls_ptr, *cls_end; u64 *cls_top; float *cls_w;
-    int32_t *ccls;                // compact list of the non-empty classes (dense class indices)
+    int32_t *ccls;                // compact list of the non-empty classes: dense index | gi2 << 16 | ci2 << 24
     SlotA *sa; SlotB *sb; SlotC *sc; int32_t *sj;
     const int32_t *gl, *clv;      // GPU / CPU level values in shared memory (lanes index them divergently)
-    int N;
+    int N, N_pad;
 };
 
 struct Shared {
     uint32_t red_key[RW]; int32_t red_j[RW]; uint32_t red_pay[RW];
+    int dirty[RW];                // warp must rescan: one of its slots (or a class head) changed
     int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
+    int ver;                      // bumped whenever maxc[] or the empty-node count changes
+    int maxc_dirty;               // the last commit may have changed maxc[]
+    int t0, t1;                   // nodes whose free GPUs / cores the last commit changed (-1 = none)
     int scan_cnt[RW];
 };
 
 // warp-cooperative: first node with at least g free GPUs and c free cores, -1 if none
 __device__ int first_fit_warp(const Views &v, int g, int c, int lane)
 {
-    for (int base = 0; base < v.N; base += 32) {
-        const int n = base + lane;
-        const bool ok = n < v.N && v.free_g[n] >= g && v.free_c[n] >= c;
-        const unsigned b = __ballot_sync(0xffffffffu, ok);
-        if (b) return base + __ffs(b) - 1;
+    const int4 *w4 = reinterpret_cast<const int4 *>(v.gc);
+    for (int base = 0; base < v.N_pad; base += 128) {
+        const int4 x = w4[(base >> 2) + lane];
+        int first = -1;
+        if (fg_of(x.w) >= g && fc_of(x.w) >= c) first = 3;
+        if (fg_of(x.z) >= g && fc_of(x.z) >= c) first = 2;
+        if (fg_of(x.y) >= g && fc_of(x.y) >= c) first = 1;
+        if (fg_of(x.x) >= g && fc_of(x.x) >= c) first = 0;
+        const unsigned b = __ballot_sync(0xffffffffu, first >= 0);
+        if (b) return __shfl_sync(0xffffffffu, base + 4 * lane + first, __ffs(b) - 1);
     }
     return -1;
 }
 
-// warp-cooperative: rebuild maxc[] from the node state.  A job of g GPUs and c cores fits some
-// node as a whole exactly when maxc[level of g] >= c.
-__device__ void rebuild_maxc(const Space &sp, const Views &v, int lane)
+// warp-cooperative: most free cores among the nodes with at least g free GPUs (-1 if none).  A job of
+// g GPUs and c cores fits some node as a whole exactly when this is >= c.
+__device__ int max_cores_warp(const Views &v, int g, int lane)
 {
-    for (int gi = 0; gi < sp.n_small; ++gi) {
-        const int g = sp.g_levels[gi];
-        int m = -1;
-        for (int n = lane; n < v.N; n += 32)
-            if (v.free_g[n] >= g) m = max(m, v.free_c[n]);
-        m = __reduce_max_sync(0xffffffffu, m);
-        if (lane == 0) v.maxc[gi] = m;
+    const int4 *w4 = reinterpret_cast<const int4 *>(v.gc);
+    int m = -1;
+    for (int base = 0; base < v.N_pad; base += 128) {
+        const int4 x = w4[(base >> 2) + lane];
+        m = max(m, fg_of(x.x) >= g ? fc_of(x.x) : -1);
+        m = max(m, fg_of(x.y) >= g ? fc_of(x.y) : -1);
+        m = max(m, fg_of(x.z) >= g ? fc_of(x.z) : -1);
+        m = max(m, fg_of(x.w) >= g ? fc_of(x.w) : -1);
     }
-    __syncwarp();
+    return __reduce_max_sync(0xffffffffu, m);
 }
 
 struct Committed { int first; float val; int plan; int f; };
 
-// Commit job j to (gi2, ci2); warp 0, all lanes, uniform control flow.  `alloc`: the job holds
-// (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target
-// at the top memory level.  On success the node state, the empty-node count and maxc[] are current.
+// Commit job j to (gi2, ci2); one warp, all lanes, uniform control flow.  `alloc`: the job holds
+// (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target at
+// the top memory level.  On success node state and empty-node count are current; maxc[] is rebuilt
+// here when `rebuild`, otherwise sh.maxc_dirty / sh.ver / sh.t0 / sh.t1 tell the block what changed.
 __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const float *__restrict__ cv,
                             const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
                             const uint32_t *__restrict__ feas, int j, bool alloc, int gi, int ci, int node,
@@ -256,7 +274,8 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     int k2 = 1, target = -1, need_new = 0;
     bool stay = false;
     if (g2 <= sp.Gn) {
-        if (alloc && v.free_g[node] >= g2 - g && v.free_c[node] >= c2 - c) { stay = true; target = node; }
+        if (alloc) { const int w = v.gc[node]; stay = fg_of(w) >= g2 - g && fc_of(w) >= c2 - c; }
+        if (stay) target = node;
         else if (v.maxc[gi2] >= c2) target = first_fit_warp(v, g2, c2, lane);
         if (target < 0) return false;
     } else {
@@ -265,7 +284,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         if (alloc && g >= sp.Gn) { stay = true; need_new = k2 - k; if (n_empty < need_new) return false; }
         else {
             need_new = k2;
-            const int empty = n_empty + ((alloc && v.free_g[node] + g == sp.Gn) ? 1 : 0);
+            const int empty = n_empty + ((alloc && fg_of(v.gc[node]) + g == sp.Gn) ? 1 : 0);
             if (empty < need_new) return false;
         }
     }
@@ -294,18 +313,33 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
 
     // ---- node bookkeeping ------------------------------------------------------------------------
     int first = -1, d_empty = 0;
+    bool maxc_dirty = true;
+    int t0 = -1, t1 = -1;
     if (k2 == 1) {
+        const int moved = alloc && !stay;
+        const int w_old_n = moved ? v.gc[node] : 0, w_old_t = v.gc[target];
+        const int w_new_n = w_old_n + (g << 16) + c;
+        const int w_new_t = stay ? w_old_t - ((g2 - g) << 16) - (c2 - c) : w_old_t - (g2 << 16) - c2;
         if (lane == 0) {
-            if (stay) { v.free_g[target] -= g2 - g; v.free_c[target] -= c2 - c; v.free_m[target] -= m2 - m_cur; }
-            else {
-                if (alloc) { v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur; }
-                v.free_g[target] -= g2; v.free_c[target] -= c2; v.free_m[target] -= m2;
+            if (moved) { v.gc[node] = w_new_n; v.free_m[node] += m_cur; }
+            v.gc[target] = w_new_t;
+            v.free_m[target] -= stay ? m2 - m_cur : m2;
+        }
+        if (moved && fg_of(w_new_n) == sp.Gn) d_empty += 1;
+        if (!stay && fg_of(w_old_t) == sp.Gn) d_empty -= 1;
+        first = target; t1 = target; t0 = moved ? node : -1;
+        // can maxc[] have changed?  lane i answers for GPU level i
+        bool ch = false;
+        if (lane < sp.n_small) {
+            const int gl = sp.g_levels[lane], mx = v.maxc[lane];
+            const int ot = fg_of(w_old_t) >= gl ? fc_of(w_old_t) : -1, nt = fg_of(w_new_t) >= gl ? fc_of(w_new_t) : -1;
+            ch = (ot == mx && nt < ot) || nt > mx;
+            if (moved) {
+                const int on = fg_of(w_old_n) >= gl ? fc_of(w_old_n) : -1, nn = fg_of(w_new_n) >= gl ? fc_of(w_new_n) : -1;
+                ch = ch || (on == mx && nn < on) || nn > mx;
             }
         }
-        __syncwarp();
-        if (alloc && !stay && v.free_g[node] == sp.Gn) d_empty += 1;
-        if (!stay && v.free_g[target] + g2 == sp.Gn) d_empty -= 1;
-        first = target;
+        maxc_dirty = __any_sync(0xffffffffu, ch);
     } else {
         const int cs2 = (c2 + k2 - 1) / k2;
         const int64_t ms2 = cdiv64(m2, k2);
@@ -314,33 +348,44 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
             const int cs1 = (c + k - 1) / k;
             const int64_t ms1 = cdiv64(m_cur, k);
             if (k == 1) {
-                if (lane == 0) { v.free_c[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; }
+                if (lane == 0) { v.gc[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; }
             } else {
                 for (int n = lane; n < v.N; n += 32)
-                    if (v.owner[n] == j) { v.free_c[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
+                    if (v.owner[n] == j) { v.gc[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
             }
             first = node;
         } else if (alloc) {
-            if (lane == 0) { v.free_g[node] += g; v.free_c[node] += c; v.free_m[node] += m_cur; }
+            if (lane == 0) { v.gc[node] += (g << 16) + c; v.free_m[node] += m_cur; }
             __syncwarp();
-            if (v.free_g[node] == sp.Gn) d_empty += 1;
+            if (fg_of(v.gc[node]) == sp.Gn) d_empty += 1;
         }
         __syncwarp();
         int taken = 0;
         for (int base = 0; base < v.N && taken < need_new; base += 32) {
             const int n = base + lane;
-            const bool empty = n < v.N && v.free_g[n] == sp.Gn;
+            const bool empty = n < v.N && fg_of(v.gc[n]) == sp.Gn;
             const unsigned b = __ballot_sync(0xffffffffu, empty);
             const int rank = __popc(b & ((1u << lane) - 1u));
-            if (empty && taken + rank < need_new) { v.free_g[n] = 0; v.free_c[n] -= cs2; v.free_m[n] -= ms2; v.owner[n] = j; }
+            if (empty && taken + rank < need_new) { v.gc[n] -= (sp.Gn << 16) + cs2; v.free_m[n] -= ms2; v.owner[n] = j; }
             if (b) { const int lowest = base + __ffs(b) - 1; if (first < 0 || lowest < first) first = lowest; }
             taken += __popc(b);
         }
         d_empty -= need_new;
     }
     __syncwarp();
-    if (lane == 0) sh.n_empty = n_empty + d_empty;
-    if (rebuild) rebuild_maxc(sp, v, lane);
+    if (rebuild) {
+        for (int i = 0; i < sp.n_small; ++i) {
+            const int m = max_cores_warp(v, sp.g_levels[i], lane);
+            if (lane == 0) v.maxc[i] = m;
+        }
+        if (lane == 0) sh.n_empty = n_empty + d_empty;
+        __syncwarp();
+    } else if (lane == 0) {
+        sh.n_empty = n_empty + d_empty;
+        sh.maxc_dirty = maxc_dirty;
+        sh.t0 = t0; sh.t1 = t1;
+        if (d_empty != 0 || k2 > 1) sh.ver += 1;
+    }
     out.first = first; out.val = val; out.plan = plan; out.f = f;
     return true;
 }
@@ -414,14 +459,6 @@ __device__ SlotC make_slotc(const Space &sp, int gi, int ci, int next_g, int nex
     return s;
 }
 
-__device__ __forceinline__ bool class_placeable(const Space &sp, const Views &v, int n_empty, int gi2, int ci2)
-{
-    const int g2 = v.gl[gi2], c2 = v.clv[ci2];
-    if (g2 <= sp.Gn) return v.maxc[gi2] >= c2;
-    const int k2 = g2 >> sp.log2Gn;
-    return (c2 + k2 - 1) / k2 <= sp.Cn && n_empty >= k2;
-}
-
 struct RoundArgs {
     const rubick_job *jobs; int J;
     const float *cv; const int32_t *cp; const int32_t *cg; const uint32_t *feas;
@@ -435,8 +472,7 @@ struct RoundArgs {
 
 constexpr int SLOT_BYTES = int(sizeof(SlotA) + sizeof(SlotC)) + 4;     // per running job in shared memory
 
-// block-wide selection: largest key32, lowest job among equal keys.  Per-thread triple in, the
-// winner (key 0 = none) out on every lane of warp 0.
+// warp-wide selection: largest key, lowest job among equal keys (key 0 = nothing)
 __device__ __forceinline__ void warp_select(uint32_t &key, int &j, uint32_t &pay)
 {
     const uint32_t m = __reduce_max_sync(0xffffffffu, key);
@@ -457,12 +493,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     const int n_cls = sp.nG * sp.nC;
 
     Views v;
-    v.N = N;
+    v.N = N; v.N_pad = (N + 127) & ~127;
     unsigned char *p = smem_raw;
+    v.gc = reinterpret_cast<int32_t *>(p); p += size_t(v.N_pad) * 4;            // 16-byte aligned: read as int4
     v.free_m = reinterpret_cast<int64_t *>(p); p += size_t(N) * 8;
     v.cls_top = reinterpret_cast<u64 *>(p); p += size_t(n_cls) * 8;
-    v.free_g = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
-    v.free_c = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
     v.owner = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
     v.cls_ptr = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
     v.cls_end = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
@@ -481,12 +516,17 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     v.sb = A.sb_g;          // value / plan / memory level / weight: touched only by commits, kept in global memory
 
     // ---- set-up ---------------------------------------------------------------------------------
-    for (int n = tid; n < N; n += RT) { v.free_g[n] = sp.Gn; v.free_c[n] = sp.Cn; v.free_m[n] = sp.Mn; v.owner[n] = -1; }
+    for (int n = tid; n < v.N_pad; n += RT) v.gc[n] = n < N ? ((sp.Gn << 16) | sp.Cn) : 0;
+    for (int n = tid; n < N; n += RT) { v.free_m[n] = sp.Mn; v.owner[n] = -1; }
     for (int t = tid; t < n_cls; t += RT) { v.cls_ptr[t] = 0; v.cls_end[t] = 0; v.cls_top[t] = 0ull; v.cls_w[t] = 0.0f; }
     if (tid < sp.nG) gl_s[tid] = sp.g_levels[tid];
     if (tid < sp.nC) cl_s[tid] = sp.c_levels[tid];
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
-    if (tid == 0) { sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0; }
+    if (tid < RW) sh.dirty[tid] = 1;
+    if (tid == 0) {
+        sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
+        sh.ver = 0; sh.maxc_dirty = 1; sh.t0 = -1; sh.t1 = -1;
+    }
     __syncthreads();
 
     // class segments of the sorted keys: a class starts where the class field changes
@@ -599,55 +639,80 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     __syncthreads();
 
     // ---- Phase B ---------------------------------------------------------------------------------------
+    // Every warp remembers the best candidate among its own slots (warp 31: among the class heads) and
+    // looks again only when something it depends on changed: one of its slots, a node one of its slots
+    // sits on, maxc[] or the number of empty nodes.
+    uint32_t c_key = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
     for (;;) {
-        // most free cores among the nodes with >= g free GPUs: one warp per small GPU level
-        if (warp < sp.n_small) {
-            const int g = sp.g_levels[warp];
-            int m = -1;
-#pragma unroll 4
-            for (int n = lane; n < N; n += 32) m = max(m, v.free_g[n] >= g ? v.free_c[n] : -1);
-            m = __reduce_max_sync(0xffffffffu, m);
-            if (lane == 0) v.maxc[warp] = m;
+        if (sh.maxc_dirty) {                                   // uniform: written before the last barrier
+            if (warp < sp.n_small) {
+                const int m = max_cores_warp(v, sp.g_levels[warp], lane);
+                if (lane == 0 && m != v.maxc[warp]) { v.maxc[warp] = m; atomicAdd(&sh.ver, 1); }
+            }
+            __syncthreads();
         }
-        __syncthreads();
-        const int n_empty = sh.n_empty, n_slots = sh.n_slots, n_ccls = sh.n_ccls;
-        uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
-        for (int i = tid; i < n_ccls; i += RT) {
-            const int packed = v.ccls[i];
-            const int t = packed & 0xffff, gi2 = (packed >> 16) & 0xff, ci2 = (packed >> 24) & 0xff;
-            const u64 k = v.cls_top[t];
-            if (k) {
-                const uint32_t k32 = 0x80000000u | key_gain_bits(k);
-                const int j = key_job(k);
-                if ((k32 > best || (k32 == best && j < best_j)) && class_placeable(sp, v, n_empty, gi2, ci2)) {
-                    best = k32; best_j = j; pay = 0x80000000u | uint32_t(t);
+        const int n_empty = sh.n_empty, n_slots = sh.n_slots, ver = sh.ver;
+        bool rescan = ver != my_ver || sh.dirty[warp] != 0;
+        if (warp < SCAN_WARPS) {
+            if (!rescan) {
+                const int t0 = sh.t0, t1 = sh.t1;
+                bool hit = false;
+                for (int s = tid; s < n_slots; s += SCAN_T) { const int nd = v.sa[s].node; hit = hit || nd == t0 || nd == t1; }
+                rescan = __any_sync(0xffffffffu, hit);
+            }
+            if (rescan) {
+                uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
+                for (int s = tid; s < n_slots; s += SCAN_T) {
+                    const SlotA a = v.sa[s];
+                    const SlotC q = v.sc[s];
+                    const int j = v.sj[s];
+                    const int w = v.gc[a.node];
+                    const int fg = fg_of(w), fc = fc_of(w);
+                    const int mg = v.maxc[q.gidx], mc = v.maxc[q.cidx];
+                    const bool part_empty = fg + q.g == sp.Gn;
+                    const bool ok_g = a.gain_g > 0.0f
+                                      && (q.gkind == K_SINGLE ? (fg >= q.dg || mg >= q.c)
+                                          : q.gkind == K_MULTI_WHOLE ? n_empty >= q.need
+                                          : q.gkind == K_MULTI_PART ? n_empty + int(part_empty) >= q.need : false);
+                    const bool ok_c = a.gain_c > 0.0f && (q.ckind == K_SINGLE ? (fc >= q.dc || mc >= q.c2) : q.ckind == K_MULTI_WHOLE);
+                    // a GPU increment outranks any CPU increment
+                    const uint32_t k32 = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : ok_c ? __float_as_uint(a.gain_c) : 0u;
+                    if (k32 > best || (k32 == best && k32 && j < best_j)) { best = k32; best_j = j; pay = uint32_t(s); }
+                }
+                warp_select(best, best_j, pay);
+                c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
+                if (lane == 0) sh.dirty[warp] = 0;
+            }
+        } else if (rescan) {
+            uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
+            const int n_ccls = sh.n_ccls;
+            for (int i = lane; i < n_ccls; i += 32) {
+                const int packed = v.ccls[i];
+                const int t = packed & 0xffff, gi2 = (packed >> 16) & 0xff, ci2 = (packed >> 24) & 0xff;
+                const u64 k = v.cls_top[t];
+                if (k) {
+                    const int g2 = v.gl[gi2], c2 = v.clv[ci2];
+                    bool ok;
+                    if (g2 <= sp.Gn) ok = v.maxc[gi2] >= c2;
+                    else { const int k2 = g2 >> sp.log2Gn; ok = (c2 + k2 - 1) / k2 <= sp.Cn && n_empty >= k2; }
+                    const uint32_t k32 = ok ? (0x80000000u | key_gain_bits(k)) : 0u;
+                    const int j = key_job(k);
+                    if (k32 > best || (k32 == best && k32 && j < best_j)) { best = k32; best_j = j; pay = 0x80000000u | uint32_t(t); }
                 }
             }
+            warp_select(best, best_j, pay);
+            c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
+            if (lane == 0) sh.dirty[warp] = 0;
         }
-        for (int s = tid; s < n_slots; s += RT) {
-            const SlotA a = v.sa[s];
-            const SlotC q = v.sc[s];
-            const int j = v.sj[s];
-            const int fg = v.free_g[a.node], fc = v.free_c[a.node];
-            const int mg = v.maxc[q.gidx], mc = v.maxc[q.cidx];
-            const bool part_empty = fg + q.g == sp.Gn;
-            const bool ok_g = a.gain_g > 0.0f
-                              && (q.gkind == K_SINGLE ? (fg >= q.dg || mg >= q.c)
-                                  : q.gkind == K_MULTI_WHOLE ? n_empty >= q.need
-                                  : q.gkind == K_MULTI_PART ? n_empty + int(part_empty) >= q.need : false);
-            const bool ok_c = a.gain_c > 0.0f && (q.ckind == K_SINGLE ? (fc >= q.dc || mc >= q.c2) : q.ckind == K_MULTI_WHOLE);
-            // a GPU increment outranks any CPU increment
-            const uint32_t k32 = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : ok_c ? __float_as_uint(a.gain_c) : 0u;
-            if (k32 > best || (k32 == best && k32 && j < best_j)) { best = k32; best_j = j; pay = uint32_t(s); }
-        }
-        warp_select(best, best_j, pay);
-        if (lane == 0) { sh.red_key[warp] = best; sh.red_j[warp] = best_j; sh.red_pay[warp] = pay; }
+        if (lane == 0) { sh.red_key[warp] = c_key; sh.red_j[warp] = c_j; sh.red_pay[warp] = c_pay; }
         __syncthreads();
         if (warp == 0) {
-            best = sh.red_key[lane]; best_j = sh.red_j[lane]; pay = sh.red_pay[lane];
+            uint32_t best = sh.red_key[lane], pay = sh.red_pay[lane]; int best_j = sh.red_j[lane];
             warp_select(best, best_j, pay);
             bool go = best != 0u;
             if (go && sh.steps >= A.max_steps) { if (lane == 0) sh.capped = 1; go = false; }
+            if (lane == 0) { sh.maxc_dirty = 0; sh.t0 = -1; sh.t1 = -1; }
+            __syncwarp();
             if (go) {
                 const int type_gpu = int(best >> 31);
                 const int j = best_j;
@@ -676,9 +741,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
                             v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j; v.sc[s] = make_slotc(sp, gi2, ci2, ng_, nc_);
                             sh.n_slots = s + 1;
+                            sh.dirty[(s % SCAN_T) >> 5] = 1;
                         }
                     }
-                    if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; }
+                    if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[RW - 1] = 1; }
                 } else {
                     const int s = int(pay);
                     SlotA a = v.sa[s]; SlotB b = v.sb[s];
@@ -703,7 +769,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
                         a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
                     }
-                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; }
+                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; sh.dirty[(s % SCAN_T) >> 5] = 1; }
                 }
                 if (lane == 0) {
                     if (A.step_log) A.step_log[sh.steps] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
@@ -728,7 +794,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     if (A.node_out)
         for (int n = tid; n < N; n += RT) {
             rubick_node nd;
-            nd.free_g = v.free_g[n]; nd.free_c = v.free_c[n]; nd.free_m = v.free_m[n]; nd.owner = v.owner[n]; nd.reserved = 0;
+            nd.free_g = fg_of(v.gc[n]); nd.free_c = fc_of(v.gc[n]); nd.free_m = v.free_m[n]; nd.owner = v.owner[n]; nd.reserved = 0;
             A.node_out[n] = nd;
         }
     if (tid == 0) {
@@ -748,7 +814,8 @@ static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
 static size_t fixed_smem(const Space &sp, int N)
 {
     const size_t n_cls = size_t(sp.nG) * sp.nC;
-    const size_t fixed = size_t(N) * 20 + n_cls * 24 + size_t(2 * RUBICK_MAX_G_LEVELS + RUBICK_MAX_C_LEVELS) * 4;
+    const size_t n_pad = (size_t(N) + 127) & ~size_t(127);
+    const size_t fixed = n_pad * 4 + size_t(N) * 12 + n_cls * 24 + size_t(2 * RUBICK_MAX_G_LEVELS + RUBICK_MAX_C_LEVELS) * 4;
     return (fixed + 15) & ~size_t(15);
 }
 
@@ -786,7 +853,9 @@ bool round_fast_supported(const Space &sp, int J, int N)
 {
     using namespace fastround;
     if (J < 1 || J >= (1 << KEY_JOB_BITS)) return false;
-    if (sp.Cn > 32767 || sp.g_levels[sp.nG - 1] > 32767 || sp.c_levels[sp.nC - 1] > 32767) return false;   // SlotC holds int16
+    // node words and slot requirements hold 15 / 16-bit fields
+    if (sp.Cn > 32767 || sp.Gn > 16384 || sp.g_levels[sp.nG - 1] > 32767 || sp.c_levels[sp.nC - 1] > 32767) return false;
+    if (size_t(sp.nG) * sp.nC > 65535) return false;
     return fixed_smem(sp, N) <= SMEM_LIMIT;
 }
 
