@@ -185,7 +185,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="throughput-stress", choices=list(workloads.CONFIGS))
@@ -194,6 +194,7 @@ def main():
     ap.add_argument("--ref-jobs", type=int, default=1024, help="jobs per step of the CPU arm / baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--events", type=int, default=200, help="scheduling events of the event-driven run (0 = skip)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -263,10 +264,10 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    sampler = ClockSampler(local) if rank == 0 else None       # nvidia-smi needs a moment to start: launch it before the warm-up
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
     marks = []
     t_start = ev()
     for _ in range(args.steps):
@@ -299,6 +300,24 @@ def main():
                "d2h_bytes_per_step": int(J * rb.ASSIGN_DTYPE.itemsize + N * rb.NODE_DTYPE.itemsize),
                "call": "rubick_schedule_round_host: pinned job records in, assignments and node states out"}
 
+    # event-driven run: every arrival / completion re-plans all active jobs (rank 0 only)
+    events = None
+    if args.events > 0 and rank == 0:
+        from paper_2408_08586_b200 import events as ev_mod
+        ecfg = make_workload("events")
+        ectx = rb.Context(ecfg["env"], device=local, stream=stream.cuda_stream)
+        eplans, _ = rb.enumerate_plans(ecfg["g_levels"])
+        ectx.set_space(eplans, ecfg["g_levels"], ecfg["c_levels"], ecfg["m_levels"])
+        ev_mod.run_events(ectx, ecfg, n_events=5)                                    # warm-up: scratch allocation
+        r = ev_mod.run_events(ectx, ecfg, n_events=args.events)
+        events = {"events": int(len(r["latency_ms"])), "nodes": int(ecfg["n_nodes"]),
+                  "active_jobs_min": int(r["active"].min()), "active_jobs_max": int(r["active"].max()),
+                  "round_latency_ms_p50": float(np.percentile(r["latency_ms"], 50)),
+                  "round_latency_ms_p99": float(np.percentile(r["latency_ms"], 99)),
+                  "steps_per_round_mean": float(r["steps"].mean()),
+                  "what": "rubick_schedule_round_host per event: host job records in, table + curves + round on the GPU, assignments out"}
+        ectx.close()
+
     if rank != 0:
         if world > 1:
             import torch.distributed as dist
@@ -316,7 +335,7 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
-        J_s = min(J, args.ref_jobs)
+        J_s = min(J, 4 * args.ref_jobs)                         # a few seconds on all host cores
         nodes_s = max(1, N * J_s // J)
         dt, _ = oracle_sample(cfg, J_s, nodes_s, threads)
         cpu_baseline = {"value": J_s * P * C / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -343,6 +362,7 @@ def main():
         "eval_kernel_candidates_per_sec": float(J) * P * C / (stage_ms[0] * 1e-3),
         "logical_candidates_per_sec": value * M,
         "best_plan_roofline": {"bound": "hbm", "achieved": best_gbs, "peak": peak, "unit": "GB/s", "frac": best_gbs / peak},
+        "events": events,
         "round": {"steps": int(round_steps[0]), "latency_ms": float(stage_ms[3]),
                   "us_per_step": float(1e3 * stage_ms[3] / max(1, round_steps[0]))},
     }

@@ -1,0 +1,117 @@
+"""Parity at the benchmark's full size (16,384 jobs, 512 nodes), in the launch configuration
+bench.py times: sampled jobs against the oracle one by one, properties that hold at any size on
+everything else, and the two round implementations against each other."""
+import numpy as np
+import pytest
+
+import oracle
+from gpu_util import Gpu, assert_rounds_equal, has_cuda, unpack_round
+from paper_2408_08586_b200 import binding as rb
+from paper_2408_08586_b200 import workloads
+
+pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not has_cuda(), reason="needs a CUDA device")]
+
+
+@pytest.fixture(scope="module")
+def full():
+    cfg = workloads.make("throughput-stress")
+    gpu = Gpu(cfg)
+    J = len(cfg["jobs"]["P"])
+    d_jobs, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    d_cv, d_cp, d_cg = gpu.best(d_thr, d_feas, J)
+    return cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg
+
+
+def test_sampled_jobs_match_the_oracle(full):
+    cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg = full
+    rng = np.random.default_rng(7)
+    sample = np.unique(np.concatenate([[0, 1, J - 1, J - 2, 255, 256, 8191, 8192], rng.integers(0, J, 24)]))
+    jobs = workloads.take(cfg["jobs"], sample)
+    plans, _ = oracle.enumerate_plans(cfg["g_levels"])
+    thr, feas = oracle.eval_candidates(jobs, plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=8)
+    t = gpu.torch
+    idx = t.from_numpy(sample).cuda()
+    got_thr = d_thr.view(J, gpu.nC, gpu.P)[idx].cpu().numpy()
+    got_feas = d_feas.view(J, gpu.P)[idx].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got_feas, feas)
+    nz = thr > 0
+    assert np.array_equal(got_thr > 0, nz)
+    assert (np.abs(got_thr[nz] - thr[nz]) / thr[nz]).max() <= 1e-5
+    # curves of the sampled jobs: the GPU's arg-max over its own single-precision rows, replayed by the oracle's
+    # definition on the oracle's rows: values within tolerance, indices equal except at near ties
+    ov, op, og = oracle.best_plan(thr, feas, plans, cfg["g_levels"], gpu.nM, prefix=True, nthreads=8)
+    sh = (J, gpu.nG, gpu.nC, gpu.nM)
+    gv = d_cv.view(sh)[idx].cpu().numpy(); gp = d_cp.view(sh)[idx].cpu().numpy(); gg = d_cg.view(sh)[idx].cpu().numpy()
+    has = op >= 0
+    assert np.array_equal(gp >= 0, has)
+    assert (np.abs(gv[has] - ov[has]) / ov[has]).max() <= 1e-5
+    diff = has & (gp != op)
+    jj, _, cc, _ = np.nonzero(diff)
+    assert np.all(thr[jj, cc, gp[diff]] >= ov[diff] * (1 - 1e-6))
+    assert diff.mean() < 0.01 and np.array_equal(gg[~diff], og[~diff])
+
+
+def test_properties_of_the_whole_table(full):
+    cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg = full
+    t = gpu.torch
+    thr = d_thr.view(J, gpu.nC, gpu.P)
+    assert bool(t.isfinite(d_thr).all()) and float(d_thr.min()) >= 0
+    # cores matter only to offload plans (odd plan indices) and never hurt
+    assert bool((thr[:, 1:, 0::2] == thr[:, :-1, 0::2]).all())
+    assert bool((thr[:, 1:, 1::2] >= thr[:, :-1, 1::2]).all())
+    # an invalid plan is invalid at every core level
+    assert bool(((thr[:, 0, :] == 0) == (thr[:, -1, :] == 0)).all())
+    # feasibility words are thresholds in the level index
+    w = d_feas.view(J, gpu.P).to(t.int64) & 0xFFFFFFFF
+    low = w & (-w)
+    assert bool(((w == 0) | (w == (0xFFFFFFFF & ~(low - 1)))).all())
+    # curves: non-decreasing in GPUs, cores and host memory; the carried GPU count never exceeds the level
+    cv = d_cv.view(J, gpu.nG, gpu.nC, gpu.nM)
+    assert bool((cv[:, 1:] >= cv[:, :-1]).all()) and bool((cv[:, :, 1:] >= cv[:, :, :-1]).all())
+    assert bool((cv[:, :, :, 1:] >= cv[:, :, :, :-1]).all())
+    levels = t.tensor(cfg["g_levels"], device="cuda", dtype=t.int32).view(1, -1, 1, 1)
+    cg = d_cg.view(J, gpu.nG, gpu.nC, gpu.nM)
+    assert bool((cg <= levels).all()) and bool(((d_cp.view_as(cg) >= 0) == (cv > 0)).all())
+
+
+def test_round_at_full_size_is_a_valid_packing_and_both_kernels_agree(full):
+    cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg = full
+    t = gpu.torch
+    N = cfg["n_nodes"]
+    res = []
+    for call in (gpu.ctx.greedy_round, gpu.ctx.greedy_round_noalloc):       # fast path / plain single-kernel form
+        d_out = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_node = t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        steps, capped = call(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, 1 << 30, d_out, d_node)
+        res.append(unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped, None))
+    fast, plain = res
+    assert_rounds_equal(fast, plain)
+    r = fast
+    e = cfg["env"]
+    Gn, Cn, Mn = e["gpus_per_node"], e["cpus_per_node"], e["mem_per_node_bytes"]
+    run = r["status"] == rb.RUNNING
+    assert run.sum() > 500 and not r["capped"] and r["steps"] > 1000
+    used = np.zeros((N, 3), dtype=np.int64)
+    single = run & (r["n_nodes"] == 1)
+    np.add.at(used, r["first_node"][single], np.stack([r["g"][single], r["c"][single], r["m_bytes"][single]], axis=1))
+    for j in np.nonzero(run & (r["n_nodes"] > 1))[0]:
+        own = np.nonzero(r["node"][:, 3] == j)[0]
+        k = int(r["n_nodes"][j])
+        assert len(own) == k and own[0] == r["first_node"][j] and r["g"][j] == k * Gn
+        used[own] += (Gn, -(-int(r["c"][j]) // k), -(-int(r["m_bytes"][j]) // k))
+    assert np.all(used <= np.array([Gn, Cn, Mn]))
+    assert np.array_equal(r["node"][:, 0], Gn - used[:, 0]) and np.array_equal(r["node"][:, 1], Cn - used[:, 1])
+    assert np.array_equal(r["node"][:, 2], Mn - used[:, 2])
+    # the value of every running job is the curve's at its levels
+    cv = d_cv.view(J, gpu.nG, gpu.nC, gpu.nM).cpu().numpy()
+    gi = np.searchsorted(cfg["g_levels"], r["g"][run]); ci = np.searchsorted(cfg["c_levels"], r["c"][run])
+    assert np.all(r["thr"][run] <= cv[np.nonzero(run)[0], gi, ci, -1]) and np.all(r["thr"][run] > 0)
+
+
+def test_event_driven_rounds_run_and_stay_consistent():
+    from paper_2408_08586_b200 import events
+    cfg = workloads.make("events", J=400, n_nodes=16)
+    gpu = Gpu(cfg)
+    r = events.run_events(gpu.ctx, cfg, n_events=25, warm_jobs=120)
+    assert len(r["latency_ms"]) == 25 and (r["latency_ms"] > 0).all()
+    assert r["active"].min() >= 100 and r["active"].max() <= 150 and (r["steps"] > 0).all()
