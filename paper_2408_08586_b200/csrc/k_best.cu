@@ -2,47 +2,55 @@
 // curve (paper Section 5.2): an argmax over the plans of one GPU level that are feasible at a
 // memory level, lowest plan index on ties, then the running maximum along the GPU axis.
 //
-// One CTA owns one job.  Its feasibility words are turned once into "first feasible level" bytes
-// in shared memory (words are thresholds in the level index, so the first set bit says it all).
-// Each warp then takes CPU levels in turn: lanes stream the level's row of the throughput table
-// with 16-byte loads (four plans = one quad per load) and keep, per lane, a running maximum for
-// the (GPU level, first feasible level) pair they are currently seeing; when the pair changes the
-// run is pushed into a per-warp bucket array [GPU level][memory level] with a 64-bit shared-memory
-// max.  Candidates are ordered by the 64-bit key (value bits << 32 | ~plan index): positive floats
-// order like their bit patterns, and the inverted index makes the lowest plan win equal values.
-// After the row, lane m owns memory level m: a shuffle prefix-maximum over lanes turns buckets
-// into "best among plans feasible at level <= m", and a running maximum over GPU levels gives the
-// curve.  The table is read once (4 bytes per candidate); outputs are 12 bytes per (g, c, m).
+// One CTA owns one job.  Its feasibility words are turned once into 16-bit "slots" in shared memory:
+// slot = GPU level * 32 + first feasible memory level (words are thresholds in the level index, so
+// the first set bit says it all), 0xffff for a plan that is feasible nowhere.  Each warp then takes
+// two CPU levels at a time: lanes stream both rows of the throughput table with 16-byte loads (four
+// plans = one quad per load) and keep, per row and per plan parity (offload plans alternate with
+// the others and usually need another memory level), a running (value, index) maximum for the slot
+// they are currently seeing; a strict "greater" keeps the lowest index because a lane meets its
+// plans in ascending order.  When the slot changes, the run is pushed into a per-warp bucket array
+// [row][slot] with a 64-bit shared-memory max on (value bits << 32 | ~index): positive floats order
+// like their bit patterns and the inverted index makes the lowest plan win equal values across
+// lanes.  After the rows, lane m owns memory level m: the maximum over the occupied buckets at or
+// below m gives "best among plans feasible at level m", and a running maximum over GPU levels
+// gives the curve.  The table is read once (4 bytes per candidate); outputs are 12 bytes per
+// (g, c, m).
 
 #include "rubick_internal.cuh"
 
 namespace rubick {
 
-constexpr int BEST_WARPS = 8;
+constexpr int BEST_WARPS = 12;         // at most; fewer when the buckets of many GPU levels would not fit
+constexpr int BEST_ROWS = 2;          // CPU levels a warp processes together
 
-__device__ __forceinline__ unsigned long long make_key(float v, int idx)
+typedef unsigned long long u64;
+
+__device__ __forceinline__ u64 make_key(float v, int idx)
 {
-    return (static_cast<unsigned long long>(__float_as_uint(v)) << 32) | (0xffffffffu - uint32_t(idx));
+    return (static_cast<u64>(__float_as_uint(v)) << 32) | (0xffffffffu - uint32_t(idx));
 }
 
 struct Run {
-    unsigned long long key;   // 0 = empty
-    int slot;                 // g_level * 32 + first level
+    float v[BEST_ROWS]; int i[BEST_ROWS];
+    uint32_t slot;            // 0xffff = nothing yet
 };
 
-__device__ __forceinline__ void run_flush(Run &r, unsigned long long *bucket)
+__device__ __forceinline__ void run_flush(Run &r, u64 *bucket, int row_stride)
 {
-    if (r.key) atomicMax(bucket + r.slot, r.key);
-    r.key = 0ull;
+#pragma unroll
+    for (int k = 0; k < BEST_ROWS; ++k) {
+        if (r.v[k] > 0.0f) atomicMax(bucket + k * row_stride + r.slot, make_key(r.v[k], r.i[k]));
+        r.v[k] = 0.0f; r.i[k] = -1;
+    }
 }
 
-__device__ __forceinline__ void run_add(Run &r, unsigned long long *bucket, float v, int idx, int f, int grp)
+__device__ __forceinline__ void run_add(Run &r, u64 *bucket, int row_stride, uint32_t slot, int idx, float va, float vb)
 {
-    if (f == 255 || !(v > 0.0f)) return;
-    const int slot = grp * 32 + f;
-    const unsigned long long k = make_key(v, idx);
-    if (slot != r.slot) { run_flush(r, bucket); r.slot = slot; }
-    r.key = k > r.key ? k : r.key;
+    if (slot == 0xffffu) return;
+    if (slot != r.slot) { if (r.slot != 0xffffu) run_flush(r, bucket, row_stride); r.slot = slot; }
+    if (va > r.v[0]) { r.v[0] = va; r.i[0] = idx; }
+    if (vb > r.v[1]) { r.v[1] = vb; r.i[1] = idx; }
 }
 
 __global__ void __launch_bounds__(BEST_WARPS * 32)
@@ -50,11 +58,12 @@ best_plan_kernel(const __grid_constant__ Space sp, const float *__restrict__ thr
                  int J, unsigned flags, float *__restrict__ best_val, int32_t *__restrict__ best_plan,
                  int32_t *__restrict__ best_g, uint32_t *__restrict__ status)
 {
-    extern __shared__ unsigned char smem_raw[];
-    // layout: buckets [BEST_WARPS][nG][32] u64 | first level [P] u8 (padded to 4) | quad group [Q] u8
-    unsigned long long *buckets = reinterpret_cast<unsigned long long *>(smem_raw);
-    uint8_t *flevel = reinterpret_cast<uint8_t *>(buckets + BEST_WARPS * sp.nG * 32);
-    uint8_t *qgroup = flevel + ((sp.P + 15) & ~15);
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    // layout: buckets [BEST_WARPS][BEST_ROWS][nG * 32] u64 | slot of every plan [P] u16
+    const int row_stride = sp.nG * 32;
+    const int n_warps = blockDim.x >> 5;
+    u64 *buckets = reinterpret_cast<u64 *>(smem_raw);
+    uint16_t *pslot = reinterpret_cast<uint16_t *>(buckets + size_t(n_warps) * BEST_ROWS * row_stride);
 
     const int j = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -63,80 +72,102 @@ best_plan_kernel(const __grid_constant__ Space sp, const float *__restrict__ thr
     bool bad = false;
     for (int i = threadIdx.x; i < sp.P; i += blockDim.x) {
         const uint32_t w = __ldg(feas + size_t(j) * sp.P + i) & full;
-        int f = 255;
+        uint32_t s = 0xffffu;
         if (w) {
-            f = __ffs(w) - 1;
+            const int f = __ffs(w) - 1;
             bad |= (w != ((full << f) & full));
+            int g = 0;
+            while (g + 1 < sp.nG && i >= sp.group_off[g + 1]) ++g;
+            s = uint32_t(g * 32 + f);
         }
-        flevel[i] = uint8_t(f);
-    }
-    for (int q = threadIdx.x; q < sp.Q; q += blockDim.x) {
-        int g = 0;
-        while (g + 1 < sp.nG && 4 * q >= sp.group_off[g + 1]) ++g;
-        qgroup[q] = uint8_t(g);
+        pslot[i] = uint16_t(s);
     }
     if (bad) atomicOr(status, DS_FEAS_NOT_THRESHOLD);
     __syncthreads();
 
-    unsigned long long *bucket = buckets + warp * sp.nG * 32;
-    const uint32_t *flevel4 = reinterpret_cast<const uint32_t *>(flevel);
+    u64 *bucket = buckets + size_t(warp) * BEST_ROWS * row_stride;
+    const uint2 *pslot4 = reinterpret_cast<const uint2 *>(pslot);
     const bool raw = (flags & RUBICK_BEST_RAW) != 0;
+    const int n_pairs = (sp.nC + BEST_ROWS - 1) / BEST_ROWS;
 
-    for (int ci = warp; ci < sp.nC; ci += BEST_WARPS) {
-        for (int i = lane; i < sp.nG * 32; i += 32) bucket[i] = 0ull;
+    for (int pr = warp; pr < n_pairs; pr += n_warps) {
+        const int ca = pr * BEST_ROWS;
+        const bool has_b = ca + 1 < sp.nC;
+        const int cb = has_b ? ca + 1 : ca;
+        for (int i = lane; i < BEST_ROWS * row_stride; i += 32) bucket[i] = 0ull;
         __syncwarp();
 
-        const float4 *row = reinterpret_cast<const float4 *>(thr + (size_t(j) * sp.nC + ci) * sp.P);
-        Run even = {0ull, -1}, odd = {0ull, -1};   // plans 4q, 4q+2 (no offload) / 4q+1, 4q+3 (offload)
-        constexpr int UNROLL = 4;
+        const float4 *row_a = reinterpret_cast<const float4 *>(thr + (size_t(j) * sp.nC + ca) * sp.P);
+        const float4 *row_b = reinterpret_cast<const float4 *>(thr + (size_t(j) * sp.nC + cb) * sp.P);
+        Run even, odd;          // plans 4q, 4q+2 (no offload) / 4q+1, 4q+3 (offload)
+        even.slot = odd.slot = 0xffffu;
+#pragma unroll
+        for (int k = 0; k < BEST_ROWS; ++k) { even.v[k] = odd.v[k] = 0.0f; even.i[k] = odd.i[k] = -1; }
+
+        constexpr int UNROLL = 2;
         for (int q0 = lane; q0 < sp.Q; q0 += 32 * UNROLL) {
-            float4 v[UNROLL];
+            float4 va[UNROLL], vb[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int q = q0 + 32 * u;
-                v[u] = q < sp.Q ? __ldcs(row + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                const bool in = q < sp.Q;
+                va[u] = in ? __ldcs(row_a + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                vb[u] = in ? __ldcs(row_b + q) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int q = q0 + 32 * u;
                 if (q >= sp.Q) break;
-                const uint32_t f4 = flevel4[q];
-                const int grp = qgroup[q];
-                run_add(even, bucket, v[u].x, 4 * q + 0, f4 & 0xff, grp);
-                run_add(odd, bucket, v[u].y, 4 * q + 1, (f4 >> 8) & 0xff, grp);
-                run_add(even, bucket, v[u].z, 4 * q + 2, (f4 >> 16) & 0xff, grp);
-                run_add(odd, bucket, v[u].w, 4 * q + 3, f4 >> 24, grp);
+                const uint2 s4 = pslot4[q];
+                run_add(even, bucket, row_stride, s4.x & 0xffffu, 4 * q + 0, va[u].x, vb[u].x);
+                run_add(odd, bucket, row_stride, s4.x >> 16, 4 * q + 1, va[u].y, vb[u].y);
+                run_add(even, bucket, row_stride, s4.y & 0xffffu, 4 * q + 2, va[u].z, vb[u].z);
+                run_add(odd, bucket, row_stride, s4.y >> 16, 4 * q + 3, va[u].w, vb[u].w);
             }
         }
-        run_flush(even, bucket);
-        run_flush(odd, bucket);
+        if (even.slot != 0xffffu) run_flush(even, bucket, row_stride);
+        if (odd.slot != 0xffffu) run_flush(odd, bucket, row_stride);
         __syncwarp();
 
-        unsigned long long running = 0ull;
-        for (int g = 0; g < sp.nG; ++g) {
-            unsigned long long k = bucket[g * 32 + lane];
-            // inclusive prefix maximum over lanes: best among plans whose first level is <= lane
 #pragma unroll
-            for (int s = 1; s < 32; s <<= 1) {
-                const unsigned long long o = __shfl_up_sync(0xffffffffu, k, s);
-                if (lane >= s && o > k) k = o;
-            }
-            if (!raw) { running = k > running ? k : running; k = running; }
-            if (lane < sp.nM) {
-                const size_t o = ((size_t(j) * sp.nG + g) * sp.nC + ci) * sp.nM + lane;
-                const int plan = k ? int(0xffffffffu - uint32_t(k)) : -1;
-                best_val[o] = k ? __uint_as_float(uint32_t(k >> 32)) : 0.0f;
-                best_plan[o] = plan;
-                best_g[o] = plan >= 0 ? sp.g_levels[qgroup[plan >> 2]] : 0;
+        for (int k = 0; k < BEST_ROWS; ++k) {
+            if (k == 1 && !has_b) break;
+            const int ci = ca + k;
+            u64 running = 0ull;
+            for (int g = 0; g < sp.nG; ++g) {
+                const u64 mine = bucket[k * row_stride + g * 32 + lane];
+                // best among plans whose first level is <= lane: maximum over the occupied buckets at or below
+                unsigned occ = __ballot_sync(0xffffffffu, mine != 0ull);
+                u64 best = 0ull;
+                while (occ) {
+                    const int f = __ffs(occ) - 1;
+                    occ &= occ - 1;
+                    const u64 o = __shfl_sync(0xffffffffu, mine, f);
+                    if (lane >= f && o > best) best = o;
+                }
+                if (!raw) { running = best > running ? best : running; best = running; }
+                if (lane < sp.nM) {
+                    const size_t o = ((size_t(j) * sp.nG + g) * sp.nC + ci) * sp.nM + lane;
+                    const int plan = best ? int(0xffffffffu - uint32_t(best)) : -1;
+                    best_val[o] = best ? __uint_as_float(uint32_t(best >> 32)) : 0.0f;
+                    best_plan[o] = plan;
+                    best_g[o] = plan >= 0 ? sp.g_levels[pslot[plan] >> 5] : 0;
+                }
             }
         }
         __syncwarp();
     }
 }
 
-size_t best_smem_bytes(const Space &sp)
+static int best_warps(const Space &sp)
 {
-    return size_t(BEST_WARPS) * sp.nG * 32 * 8 + ((sp.P + 15) & ~15) + ((sp.Q + 15) & ~15);
+    const size_t budget = 200 * 1024, plan_bytes = (size_t(sp.P) * 2 + 15) & ~size_t(15);
+    const size_t per_warp = size_t(BEST_ROWS) * sp.nG * 32 * 8;
+    int w = plan_bytes < budget ? int((budget - plan_bytes) / per_warp) : 0;
+    const int pairs = (sp.nC + BEST_ROWS - 1) / BEST_ROWS;
+    if (w > BEST_WARPS) w = BEST_WARPS;
+    if (w > pairs) w = pairs;
+    return w;
 }
 
 cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
@@ -144,15 +175,14 @@ cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_f
                         cudaStream_t st)
 {
     if (J == 0) return cudaSuccess;
-    const size_t smem = best_smem_bytes(sp);
-    static size_t configured = 0;
-    if (smem > 48 * 1024 && smem > configured) {
+    const int warps = best_warps(sp);
+    if (warps < 1) return cudaErrorInvalidConfiguration;      // plan list too long for one CTA's shared memory
+    const size_t smem = size_t(warps) * BEST_ROWS * sp.nG * 32 * 8 + ((size_t(sp.P) * 2 + 15) & ~size_t(15));
+    if (smem > 48 * 1024) {
         cudaError_t e = cudaFuncSetAttribute(best_plan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (e != cudaSuccess) return e;
-        configured = smem;
     }
-    best_plan_kernel<<<J, BEST_WARPS * 32, smem, st>>>(sp, d_thr, d_feas, J, flags, d_best_val, d_best_plan,
-                                                       d_best_g, d_status);
+    best_plan_kernel<<<J, warps * 32, smem, st>>>(sp, d_thr, d_feas, J, flags, d_best_val, d_best_plan, d_best_g, d_status);
     return cudaGetLastError();
 }
 
