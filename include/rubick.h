@@ -155,7 +155,9 @@ int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out
  * 1 <= nM <= RUBICK_MAX_M_LEVELS, strictly increasing positive levels, GPU levels above
  * gpus_per_node multiples of it; P a positive multiple of 4; plans ordered by g_level and laid out
  * in runs of four that share (log2d, log2t, log2p, zero) with (gc, off) = (0,0), (0,1), (1,0), (1,1),
- * as rubick_enumerate_plans writes them; each plan's GPU count equals g_levels[g_level]. */
+ * and every (d, t, p) with its ZeRO stages 0, 1, 2, 3 in consecutive runs (so P is a multiple of 16),
+ * as rubick_enumerate_plans writes them; each plan's GPU count equals g_levels[g_level].  To
+ * restrict the space, set `disabled` on plans instead of dropping them. */
 int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const rubick_grid *h_grid);
 
 /* ---- the hot path ----------------------------------------------------------------------------- */

@@ -199,6 +199,13 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
         }
         if (pl.disabled) q.disabled |= uint8_t(1u << v);
     }
+    // four consecutive quads = ZeRO stages 0..3 of one (d, t, p) triple (the evaluation kernel's lanes rely on it)
+    if (quads.size() % 4) return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with all four ZeRO stages");
+    for (size_t i = 0; i < quads.size(); ++i) {
+        const QuadDesc &a = quads[i & ~size_t(3)], &b = quads[i];
+        if (b.zero != (i & 3) || a.log2d != b.log2d || a.log2t != b.log2t || a.log2p != b.log2p || a.g_level != b.g_level)
+            return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with ZeRO stages 0..3 in order (disable plans instead of dropping them)");
+    }
     while (level < gr.nG) sp.group_off[++level] = P;
 
     CUDA_TRY(ctx, cudaSetDevice(ctx->device), "cudaSetDevice");

@@ -8,7 +8,8 @@
 // non-offload optimizer time, the offload transfer time and its overlap with the gradient
 // ring), then walks the CPU levels and stores one float4 per level.  Consecutive threads own
 // consecutive quads, so a warp writes 512 contiguous bytes per level: the kernel is a pure
-// write stream of 4 bytes per candidate plus 4 / C bytes of mask.
+// write stream of 4 bytes per candidate plus 4 / C bytes of mask.  Four consecutive quads are the
+// ZeRO stages 0..3 of one (d, t, p) triple; their lanes split the per-level transcendental work.
 //
 // Model (paper Section 4):  THROUGHPUT = b / T_iter,  T_iter = T_cc + T_oo + k_const  (Eq. 1)
 //   T_fwd  = tau * mu / (t p) * (m + p - 1 if p > 1)                       forward, pipeline bubble
@@ -103,8 +104,12 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
                        uint32_t *__restrict__ feas)
 {
     // J * Q < 2^31 is checked by the host entry point
-    const uint32_t gid = blockIdx.x * blockDim.x + threadIdx.x;
-    if (gid >= uint32_t(J) * uint32_t(sp.Q)) return;
+    // Threads past the end mirror the last valid thread and store nothing: the CPU-level walk below
+    // exchanges values between the four lanes of a (d, t, p) triple, so whole warps stay converged.
+    const uint32_t total = uint32_t(J) * uint32_t(sp.Q);
+    const uint32_t gid_raw = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = gid_raw < total;
+    const uint32_t gid = active ? gid_raw : total - 1;
     const int j = int(gid / uint32_t(sp.Q));
     const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
 
@@ -187,25 +192,52 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
         fw.y = (valid_off && !(disabled & 2) && st1 + act0 <= sp.gpu_mem) ? w1 : 0u;
         fw.z = (valid && !(disabled & 4) && st0 + act1 <= sp.gpu_mem) ? w0 : 0u;
         fw.w = (valid_off && !(disabled & 8) && st1 + act1 <= sp.gpu_mem) ? w1 : 0u;
-        *reinterpret_cast<uint4 *>(feas + (size_t(j) * sp.P + 4 * size_t(q))) = fw;
+        if (active) *reinterpret_cast<uint4 *>(feas + (size_t(j) * sp.P + 4 * size_t(q))) = fw;
     }
 
     // ---- walk the CPU levels -------------------------------------------------------------------
+    // The four lanes of a triple (ZeRO stages 0..3 of the same d, t, p) share the work that depends on
+    // the core count: the swap overlap f^{k_swap}(T_opt(c), T_off) is the same for all four offload
+    // plans of the triple, so lane i evaluates it for core level 4n + i and the lanes trade results;
+    // then every lane divides for ONE offload plan (stage 2 + (lane >> 1), checkpointing = lane & 1)
+    // and the two lanes that own offload plans (stages 2 and 3) collect their pair.
     float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
     const bool off0 = valid_off && !(disabled & 2), off1 = valid_off && !(disabled & 8);
-    if (!(off0 || off1)) {
-        for (int ci = 0; ci < sp.nC; ++ci, row += sp.P) __stcs(reinterpret_cast<float4 *>(row), out);
-    } else {
-        const float T_off = sp.e * Psi * inv_d * sp.inv_B_pcie;
-        const float inv_kswap = 1.0f / jb.k_swap;
+    const unsigned FULL = 0xffffffffu;
+    if (!__any_sync(FULL, off0 || off1)) {
+        if (active)
+            for (int ci = 0; ci < sp.nC; ++ci, row += sp.P) __stcs(reinterpret_cast<float4 *>(row), out);
+        return;
+    }
+    const int lane = threadIdx.x & 31, gbase = lane & ~3, zl = lane & 3;
+    const float T_off = sp.e * Psi * inv_d * sp.inv_B_pcie;          // identical on the four lanes
+    const float opt_c = jb.k_opt_off * Psi * inv_d;                  // times 1 / c
+    const float inv_kswap = 1.0f / jb.k_swap;
+    float base0 = 0.0f, base1 = 0.0f;
+    if (valid_off) {
         const float f_off = overlap(jb.k_off, 1.0f / jb.k_off, T_dp, T_off);
-        const float base0 = cc0 + f_off, base1 = cc1 + f_off;
-        const float opt_c = jb.k_opt_off * Psi * inv_d;      // times 1 / c
-        for (int ci = 0; ci < sp.nC; ++ci, row += sp.P) {
-            const float f_swap = overlap(jb.k_swap, inv_kswap, opt_c * sp.inv_c[ci], T_off);
-            out.y = off0 ? bf / (base0 + f_swap) : 0.0f;
-            out.w = off1 ? bf / (base1 + f_swap) : 0.0f;
-            __stcs(reinterpret_cast<float4 *>(row), out);
+        base0 = cc0 + f_off; base1 = cc1 + f_off;
+    }
+    const int src = gbase + 2 + (zl >> 1);
+    const float sb0 = __shfl_sync(FULL, base0, src), sb1 = __shfl_sync(FULL, base1, src);
+    const int okbits = __shfl_sync(FULL, (off0 ? 1 : 0) | (off1 ? 2 : 0), src);
+    const float my_base = (zl & 1) ? sb1 : sb0;
+    const bool my_ok = (okbits >> (zl & 1)) & 1;
+    const int src_y = gbase + (zl == 3 ? 2 : 0), src_w = gbase + (zl == 3 ? 3 : 1);
+    for (int c0 = 0; c0 < sp.nC; c0 += 4) {
+        const int ci_mine = min(c0 + zl, sp.nC - 1);
+        const float fs_mine = overlap(jb.k_swap, inv_kswap, opt_c * sp.inv_c[ci_mine], T_off);
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+            const float fs = __shfl_sync(FULL, fs_mine, gbase + cc);
+            const float r = my_ok ? bf * rcp_approx(my_base + fs) : 0.0f;
+            const float ry = __shfl_sync(FULL, r, src_y), rw = __shfl_sync(FULL, r, src_w);
+            if (c0 + cc < sp.nC) {
+                out.y = zl >= 2 ? ry : 0.0f;
+                out.w = zl >= 2 ? rw : 0.0f;
+                if (active) __stcs(reinterpret_cast<float4 *>(row), out);
+                row += sp.P;
+            }
         }
     }
 }
