@@ -32,8 +32,9 @@
 namespace rubick {
 namespace fastround {
 
-constexpr int RT = 1024;
+constexpr int RT = 512;                 // threads of the persistent round kernel
 constexpr int RW = RT / 32;
+constexpr int SORT_T = 1024;            // threads of the sort kernel
 constexpr size_t SMEM_LIMIT = 200 * 1024;
 constexpr int SORT_SMEM_KEYS = 16384;
 
@@ -152,19 +153,19 @@ __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick
 }
 
 // ---- sort: descending bitonic sort of n (power of two) keys, then the weights in sorted order -----
-__global__ void __launch_bounds__(RT)
+__global__ void __launch_bounds__(SORT_T)
 round_sort_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ jobs, float *__restrict__ sorted_w,
                   int in_smem)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     u64 *a = in_smem ? reinterpret_cast<u64 *>(smem_raw) : keys;
     if (in_smem) {
-        for (int i = threadIdx.x; i < n; i += RT) a[i] = keys[i];
+        for (int i = threadIdx.x; i < n; i += SORT_T) a[i] = keys[i];
         __syncthreads();
     }
     for (int k = 2; k <= n; k <<= 1)
         for (int s = k >> 1; s > 0; s >>= 1) {
-            for (int i = threadIdx.x; i < n; i += RT) {
+            for (int i = threadIdx.x; i < n; i += SORT_T) {
                 const int p = i ^ s;
                 if (p > i) {
                     const u64 x = a[i], y = a[p];
@@ -174,7 +175,7 @@ round_sort_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ 
             }
             __syncthreads();
         }
-    for (int i = threadIdx.x; i < n; i += RT) {
+    for (int i = threadIdx.x; i < n; i += SORT_T) {
         const u64 k = a[i];
         if (in_smem) keys[i] = k;
         sorted_w[i] = k ? jobs[key_job(k)].w : 0.0f;
@@ -192,7 +193,7 @@ struct SlotC {
 };
 enum : uint8_t { K_SINGLE = 0, K_MULTI_WHOLE = 1, K_MULTI_PART = 2, K_NONE = 3 };
 
-constexpr int SCAN_WARPS = RW - 1;          // warps 0 .. 30 scan running jobs, warp 31 the class heads
+constexpr int SCAN_WARPS = RW - 1;          // all warps but the last scan running jobs, the last one the class heads
 constexpr int SCAN_T = SCAN_WARPS * 32;
 
 // node n: gc[n] = free GPUs << 16 | free cores (padding entries are 0: they never fit anything)
@@ -207,16 +208,18 @@ struct Views {
     int32_t *ccls;                // compact list of the non-empty classes: dense index | gi2 << 16 | ci2 << 24
     SlotA *sa; SlotB *sb; SlotC *sc; int32_t *sj;
     const int32_t *gl, *clv;      // GPU / CPU level values in shared memory (lanes index them divergently)
+    const int64_t *ml;            // memory level values, likewise
+    uint32_t *tb;                 // bit n set: the last iteration changed the free GPUs / cores of node n
     int N, N_pad;
 };
 
 struct Shared {
     uint32_t red_key[RW]; int32_t red_j[RW]; uint32_t red_pay[RW];
+    uint32_t red_key2[RW];        // second-best key of the warp (keys only: ties are resolved conservatively)
     int dirty[RW];                // warp must rescan: one of its slots (or a class head) changed
     int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
-    int t0, t1;                   // nodes whose free GPUs / cores the last commit changed (-1 = none)
     int scan_cnt[RW];
 };
 
@@ -383,7 +386,8 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     } else if (lane == 0) {
         sh.n_empty = n_empty + d_empty;
         sh.maxc_dirty = maxc_dirty;
-        sh.t0 = t0; sh.t1 = t1;
+        if (t0 >= 0) v.tb[t0 >> 5] |= 1u << (t0 & 31);
+        if (t1 >= 0) v.tb[t1 >> 5] |= 1u << (t1 & 31);
         if (d_empty != 0 || k2 > 1) sh.ver += 1;
     }
     out.first = first; out.val = val; out.plan = plan; out.f = f;
@@ -473,7 +477,7 @@ struct RoundArgs {
 constexpr int SLOT_BYTES = int(sizeof(SlotA) + sizeof(SlotC)) + 4;     // per running job in shared memory
 
 // warp-wide selection: largest key, lowest job among equal keys (key 0 = nothing)
-__device__ __forceinline__ void warp_select(uint32_t &key, int &j, uint32_t &pay)
+__device__ __forceinline__ int warp_select(uint32_t &key, int &j, uint32_t &pay)
 {
     const uint32_t m = __reduce_max_sync(0xffffffffu, key);
     const int jm = __reduce_min_sync(0xffffffffu, (key == m && m) ? j : 0x7fffffff);
@@ -481,6 +485,7 @@ __device__ __forceinline__ void warp_select(uint32_t &key, int &j, uint32_t &pay
     const int src = b ? __ffs(b) - 1 : 0;
     pay = __shfl_sync(0xffffffffu, pay, src);
     key = m; j = jm;
+    return src;                                   // the lane that held the winner
 }
 
 __global__ void __launch_bounds__(RT, 1)
@@ -498,6 +503,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     v.gc = reinterpret_cast<int32_t *>(p); p += size_t(v.N_pad) * 4;            // 16-byte aligned: read as int4
     v.free_m = reinterpret_cast<int64_t *>(p); p += size_t(N) * 8;
     v.cls_top = reinterpret_cast<u64 *>(p); p += size_t(n_cls) * 8;
+    int64_t *ml_s = reinterpret_cast<int64_t *>(p); p += size_t(RUBICK_MAX_M_LEVELS) * 8;
     v.owner = reinterpret_cast<int32_t *>(p); p += size_t(N) * 4;
     v.cls_ptr = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
     v.cls_end = reinterpret_cast<int32_t *>(p); p += size_t(n_cls) * 4;
@@ -506,7 +512,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     v.maxc = reinterpret_cast<int32_t *>(p); p += size_t(RUBICK_MAX_G_LEVELS) * 4;
     int32_t *gl_s = reinterpret_cast<int32_t *>(p); p += size_t(RUBICK_MAX_G_LEVELS) * 4;
     int32_t *cl_s = reinterpret_cast<int32_t *>(p); p += size_t(RUBICK_MAX_C_LEVELS) * 4;
-    v.gl = gl_s; v.clv = cl_s;
+    uint32_t *tb_s = reinterpret_cast<uint32_t *>(p); p += size_t(v.N_pad / 32) * 4;
+    v.gl = gl_s; v.clv = cl_s; v.ml = ml_s; v.tb = tb_s;
     p = smem_raw + ((size_t(p - smem_raw) + 15) & ~size_t(15));
     if (A.slots_in_smem) {
         v.sa = reinterpret_cast<SlotA *>(p); p += size_t(A.slot_cap) * sizeof(SlotA);
@@ -521,11 +528,13 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     for (int t = tid; t < n_cls; t += RT) { v.cls_ptr[t] = 0; v.cls_end[t] = 0; v.cls_top[t] = 0ull; v.cls_w[t] = 0.0f; }
     if (tid < sp.nG) gl_s[tid] = sp.g_levels[tid];
     if (tid < sp.nC) cl_s[tid] = sp.c_levels[tid];
+    if (tid < sp.nM) ml_s[tid] = sp.m_levels[tid];
+    for (int i = tid; i < v.N_pad / 32; i += RT) tb_s[i] = 0u;
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
     if (tid < RW) sh.dirty[tid] = 1;
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
-        sh.ver = 0; sh.maxc_dirty = 1; sh.t0 = -1; sh.t1 = -1;
+        sh.ver = 0; sh.maxc_dirty = 1;
     }
     __syncthreads();
 
@@ -566,10 +575,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         if (lane == 31) sh.scan_cnt[warp] = incl;
         __syncthreads();
         if (warp == 0) {
-            int wsum = sh.scan_cnt[lane];
+            int wsum = lane < RW ? sh.scan_cnt[lane] : 0;
 #pragma unroll
             for (int s = 1; s < 32; s <<= 1) { const int o = __shfl_up_sync(0xffffffffu, wsum, s); if (lane >= s) wsum += o; }
-            sh.scan_cnt[lane] = wsum;
+            if (lane < RW) sh.scan_cnt[lane] = wsum;
             if (lane == 31) sh.n_guar = wsum;
             // compact list of the classes that have members
             int n_c = 0;
@@ -642,7 +651,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // Every warp remembers the best candidate among its own slots (warp 31: among the class heads) and
     // looks again only when something it depends on changed: one of its slots, a node one of its slots
     // sits on, maxc[] or the number of empty nodes.
-    uint32_t c_key = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
+    uint32_t c_key = 0u, c_key2 = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
     for (;;) {
         if (sh.maxc_dirty) {                                   // uniform: written before the last barrier
             if (warp < sp.n_small) {
@@ -655,13 +664,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         bool rescan = ver != my_ver || sh.dirty[warp] != 0;
         if (warp < SCAN_WARPS) {
             if (!rescan) {
-                const int t0 = sh.t0, t1 = sh.t1;
                 bool hit = false;
-                for (int s = tid; s < n_slots; s += SCAN_T) { const int nd = v.sa[s].node; hit = hit || nd == t0 || nd == t1; }
+                for (int s = tid; s < n_slots; s += SCAN_T) { const int nd = v.sa[s].node; hit = hit || ((v.tb[nd >> 5] >> (nd & 31)) & 1u); }
                 rescan = __any_sync(0xffffffffu, hit);
             }
             if (rescan) {
-                uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
+                uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
                 for (int s = tid; s < n_slots; s += SCAN_T) {
                     const SlotA a = v.sa[s];
                     const SlotC q = v.sc[s];
@@ -675,16 +683,22 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                                           : q.gkind == K_MULTI_WHOLE ? n_empty >= q.need
                                           : q.gkind == K_MULTI_PART ? n_empty + int(part_empty) >= q.need : false);
                     const bool ok_c = a.gain_c > 0.0f && (q.ckind == K_SINGLE ? (fc >= q.dc || mc >= q.c2) : q.ckind == K_MULTI_WHOLE);
-                    // a GPU increment outranks any CPU increment
-                    const uint32_t k32 = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : ok_c ? __float_as_uint(a.gain_c) : 0u;
-                    if (k32 > best || (k32 == best && k32 && j < best_j)) { best = k32; best_j = j; pay = uint32_t(s); }
+                    // a GPU increment outranks any CPU increment; the job's other increment is only a runner-up
+                    const uint32_t kg = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : 0u;
+                    const uint32_t kc = ok_c ? __float_as_uint(a.gain_c) : 0u;
+                    const uint32_t k32 = ok_g ? kg : kc;
+                    if (k32 > best || (k32 == best && k32 && j < best_j)) { second = best; best = k32; best_j = j; pay = uint32_t(s); }
+                    else if (k32 > second) second = k32;
+                    if (ok_g && kc > second) second = kc;
                 }
-                warp_select(best, best_j, pay);
+                const uint32_t mine = best;
+                const int src = warp_select(best, best_j, pay);
+                c_key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
                 c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
                 if (lane == 0) sh.dirty[warp] = 0;
             }
         } else if (rescan) {
-            uint32_t best = 0u, pay = 0u; int best_j = 0x7fffffff;
+            uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
             const int n_ccls = sh.n_ccls;
             for (int i = lane; i < n_ccls; i += 32) {
                 const int packed = v.ccls[i];
@@ -697,23 +711,241 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     else { const int k2 = g2 >> sp.log2Gn; ok = (c2 + k2 - 1) / k2 <= sp.Cn && n_empty >= k2; }
                     const uint32_t k32 = ok ? (0x80000000u | key_gain_bits(k)) : 0u;
                     const int j = key_job(k);
-                    if (k32 > best || (k32 == best && k32 && j < best_j)) { best = k32; best_j = j; pay = 0x80000000u | uint32_t(t); }
+                    if (k32 > best || (k32 == best && k32 && j < best_j)) { second = best; best = k32; best_j = j; pay = 0x80000000u | uint32_t(t); }
+                    else if (k32 > second) second = k32;
                 }
             }
-            warp_select(best, best_j, pay);
+            const uint32_t mine = best;
+            const int src = warp_select(best, best_j, pay);
+            c_key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
             c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
             if (lane == 0) sh.dirty[warp] = 0;
         }
-        if (lane == 0) { sh.red_key[warp] = c_key; sh.red_j[warp] = c_j; sh.red_pay[warp] = c_pay; }
+        if (lane == 0) { sh.red_key[warp] = c_key; sh.red_j[warp] = c_j; sh.red_pay[warp] = c_pay; sh.red_key2[warp] = c_key2; }
         __syncthreads();
         if (warp == 0) {
-            uint32_t best = sh.red_key[lane], pay = sh.red_pay[lane]; int best_j = sh.red_j[lane];
+            const unsigned FULL = 0xffffffffu;
+            const uint32_t key = lane < RW ? sh.red_key[lane] : 0u, my_pay = lane < RW ? sh.red_pay[lane] : 0u;
+            const int my_j = lane < RW ? sh.red_j[lane] : 0x7fffffff;
+            uint32_t best = key, pay = my_pay; int best_j = my_j;
             warp_select(best, best_j, pay);
             bool go = best != 0u;
-            if (go && sh.steps >= A.max_steps) { if (lane == 0) sh.capped = 1; go = false; }
-            if (lane == 0) { sh.maxc_dirty = 0; sh.t0 = -1; sh.t1 = -1; }
+            const int steps0 = sh.steps, room = A.max_steps - steps0;
+            if (go && room <= 0) { if (lane == 0) sh.capped = 1; go = false; }
+            if (lane == 0) sh.maxc_dirty = 0;
+            for (int i = lane; i < v.N_pad / 32; i += 32) v.tb[i] = 0u;
             __syncwarp();
-            if (go) {
+
+            // ---- a batch of independent increments ---------------------------------------------------------
+            // Lane w holds the best candidate of warp w.  Increments that stay on their node, on pairwise
+            // different nodes, commute with everything except what happens on that node, so the next few
+            // picks of the sequential rule can be committed together as long as each of them still is the
+            // largest candidate: larger than every warp's runner-up (M), than the other warps' bests not yet
+            // taken, and than the new candidates of the jobs taken before it.  Each lane works out its own
+            // commit first (two global round trips for all lanes together instead of one per step).
+            int n_acc = 0;
+            // ---- a run of class heads that cannot be committed --------------------------------------------
+            // A rejected increment changes nothing but the head of its class, so as long as the heads of that
+            // class outrank every other candidate the sequential rule keeps trying them one after another
+            // against the same target and the same memory level: lane i settles the i-th entry of the
+            // class's sorted list, and everything before the first entry that would succeed is consumed.
+            if (go && (pay & 0x80000000u)) {
+                const int t = int(pay & 0x7fffffffu);
+                const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
+                const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+                const uint32_t B = __reduce_max_sync(FULL, lane < RW - 1 ? key : (lane == RW - 1 ? sh.red_key2[RW - 1] : 0u));
+                int k2 = 1; int64_t avail = -1;
+                if (g2 <= sp.Gn) {
+                    const int target = v.maxc[gi2] >= c2 ? first_fit_warp(v, g2, c2, lane) : -1;
+                    if (target >= 0) avail = v.free_m[target];
+                } else {
+                    k2 = g2 >> sp.log2Gn;
+                    if ((c2 + k2 - 1) / k2 <= sp.Cn && sh.n_empty >= k2) avail = sp.Mn;
+                }
+                if (avail >= 0) {
+                    const unsigned fb = __ballot_sync(FULL, lane < sp.nM && sp.m_levels[lane < sp.nM ? lane : 0] <= avail * k2);
+                    const int mi = fb ? 31 - __clz(fb) : -1;
+                    const int ptr = v.cls_ptr[t], end = v.cls_end[t];
+                    const int idx = ptr + lane;
+                    const u64 k = idx < end ? A.keys[idx] : 0ull;
+                    const bool in_run = k != 0ull && (0x80000000u | key_gain_bits(k)) > B;
+                    const int j = key_job(k);
+                    bool succ = false;
+                    if (in_run && mi >= 0) {
+                        const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
+                        float val; int plan, f; bool okg;
+                        if (cand.plan >= 0 && cand.f >= 0 && cand.f <= mi) { val = cand.val; plan = cand.plan; f = cand.f; okg = cand.ok != 0; }
+                        else {
+                            const size_t o = curve_idx(sp, j, gi2, ci2, mi);
+                            val = __ldg(A.cv + o); plan = __ldg(A.cp + o); okg = __ldg(A.cg + o) == g2;
+                            f = -1;
+                            if (plan >= 0 && plan < sp.P) f = __ffs(__ldg(A.feas + size_t(j) * sp.P + plan)) - 1;
+                        }
+                        succ = plan >= 0 && plan < sp.P && val > 0.0f && okg && f >= 0 && f <= mi;
+                    }
+                    // leading entries that are in the run and fail
+                    const unsigned stop = __ballot_sync(FULL, !in_run || succ);
+                    int n_fail = stop ? __ffs(stop) - 1 : 32;
+                    if (n_fail > room) n_fail = room;
+                    if (n_fail > 0) {
+                        if (lane < n_fail && A.step_log) A.step_log[steps0 + lane] = (j << 2) | 0;
+                        if (lane == 0) {
+                            const int np = ptr + n_fail;
+                            u64 nk = 0ull; float nw = 0.0f;
+                            if (np < end) { nk = A.keys[np]; nw = A.sorted_w[np]; }
+                            v.cls_ptr[t] = np; v.cls_top[t] = nk; v.cls_w[t] = nw;
+                            sh.dirty[RW - 1] = 1;
+                            sh.steps = steps0 + n_fail;
+                        }
+                        n_acc = n_fail;
+                    }
+                }
+            }
+            if (go && n_acc == 0) {
+                const uint32_t M = __reduce_max_sync(FULL, lane < RW ? sh.red_key2[lane] : 0u);
+                bool elig = false, s_ok = false, s_maxc = false, s_multi = false;
+                int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0;
+                int64_t s_dm = 0;
+                uint32_t s_bound = 0u;
+                SlotA na; SlotB nb; SlotC nq;
+                na.gain_g = na.gain_c = 0.0f; na.packed = 0u; na.node = -1;
+                nb.val = 0.0f; nb.plan = -1; nb.f_level = 0; nb.w = 0.0f;
+                nq.gkind = nq.ckind = K_NONE; nq.gidx = nq.cidx = 0; nq.dg = nq.need = nq.dc = nq.c = nq.c2 = nq.g = 0;
+                if (key != 0u && !(my_pay & 0x80000000u)) {
+                    const int s = int(my_pay), j = my_j;
+                    const SlotA a = v.sa[s];
+                    const int type_gpu = int(key >> 31);
+                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+                    const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+                    const int w_old = v.gc[a.node];
+                    // stays where it is: room on its own node, or more cores on the whole nodes it already holds
+                    const bool multi = g > sp.Gn;
+                    const int k = multi ? g >> sp.log2Gn : 1;
+                    const bool stays = multi ? (!type_gpu && (c2 + k - 1) / k <= sp.Cn)
+                                             : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
+                    if (stays) {
+                        // everything the commit and the new gains can need, in one wave of loads
+                        const SlotB b = v.sb[s];
+                        const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
+                        float col[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) col[u] = gi2 + 1 + u < sp.nG ? A.hc[hc_idx(sp, j, gi2 + 1 + u, ci2)].val : 0.0f;
+                        const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
+                        const int64_t m_cur = v.ml[b.f_level];
+                        const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
+                        int mi = -1;
+                        for (int i = 0; i < sp.nM; ++i) if (v.ml[i] <= avail) mi = i;
+                        s_multi = multi;
+                        bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+                        s_slot = s; s_node = a.node; s_type = type_gpu;
+                        if (mi < 0) { elig = true; s_ok = false; }
+                        else if (cand.plan >= 0 && cand.f >= 0 && cand.f <= mi) {
+                            elig = true;
+                            s_ok = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
+                        }
+                        if (elig && s_ok) {
+                            // new gains: first GPU level above gi2 whose curve value exceeds the new value
+                            const float val = cand.val, vcur = __fmul_rn(b.w, val);
+                            int ng_ = -1, nc_ = -1; float gg = 0.0f, gc = 0.0f;
+                            for (int base = gi2 + 1; base < sp.nG && ng_ < 0; base += 4) {
+                                if (base > gi2 + 1) {
+#pragma unroll
+                                    for (int u = 0; u < 4; ++u) col[u] = base + u < sp.nG ? A.hc[hc_idx(sp, j, base + u, ci2)].val : 0.0f;
+                                }
+#pragma unroll
+                                for (int u = 3; u >= 0; --u) if (base + u < sp.nG && col[u] > val) { ng_ = base + u; gg = col[u]; }
+                            }
+                            if (ng_ >= 0) gg = __fdiv_rn(__fsub_rn(__fmul_rn(b.w, gg), vcur), float(v.gl[ng_] - g2));
+                            if (ci2 + 1 < sp.nC) {
+                                const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(b.w, vc), vcur), float(v.clv[ci2 + 1] - c2));
+                                if (gn > 0.0f) { nc_ = ci2 + 1; gc = gn; }
+                            }
+                            na.gain_g = fz_g ? 0.0f : gg; na.gain_c = fz_c ? 0.0f : gc;
+                            na.packed = pack(gi2, ci2, ng_, fz_g, fz_c); na.node = a.node;
+                            nb.val = val; nb.plan = cand.plan; nb.f_level = cand.f; nb.w = b.w;
+                            nq = make_slotc(sp, gi2, ci2, ng_, nc_);
+                            if (multi) {
+                                // per-node shares of cores and memory on each of the k nodes (they hold no free GPU,
+                                // so maxc[] cannot change)
+                                s_dgc = (c2 + k - 1) / k - (c + k - 1) / k;
+                                s_dm = cdiv64(v.ml[cand.f], k) - cdiv64(m_cur, k);
+                            } else {
+                                s_dgc = ((g2 - g) << 16) + (c2 - c);
+                                s_dm = v.ml[cand.f] - m_cur;
+                            }
+                            // can maxc[] change?  (the node only loses GPUs / cores)
+                            const int w_new = w_old - s_dgc;
+                            for (int i = 0; i < sp.n_small && !multi; ++i) {
+                                const int glv = v.gl[i], mx = v.maxc[i];
+                                const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
+                                s_maxc = s_maxc || (ot == mx && nt < ot);
+                            }
+                        } else if (elig) {
+                            // rejected: the (job, type) pair is frozen, the other increment stays as it is
+                            if (type_gpu) { fz_g = true; } else { fz_c = true; }
+                            na = a; nb = b; nq = v.sc[s];
+                            if (type_gpu) na.gain_g = 0.0f; else na.gain_c = 0.0f;
+                            na.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
+                        }
+                        if (elig) {
+                            // the job's own next candidates, if they could be placed (maxc[] can only have
+                            // shrunk by then, so testing against the present table errs on the safe side)
+                            const int w_new = w_old - s_dgc;
+                            const int fg = fg_of(w_new), fc = fc_of(w_new);
+                            const int n_empty = sh.n_empty;
+                            const bool pg = na.gain_g > 0.0f
+                                            && (nq.gkind == K_SINGLE ? (fg >= nq.dg || v.maxc[nq.gidx] >= nq.c)
+                                                : nq.gkind == K_MULTI_WHOLE ? n_empty >= nq.need
+                                                : nq.gkind == K_MULTI_PART ? n_empty + int(fg + nq.g == sp.Gn) >= nq.need : false);
+                            const bool pc = na.gain_c > 0.0f && (nq.ckind == K_SINGLE ? (fc >= nq.dc || v.maxc[nq.cidx] >= nq.c2) : nq.ckind == K_MULTI_WHOLE);
+                            const uint32_t bg = pg ? (0x80000000u | __float_as_uint(na.gain_g)) : 0u;
+                            const uint32_t bc = pc ? __float_as_uint(na.gain_c) : 0u;
+                            s_bound = bg > bc ? bg : bc;
+                        }
+                    }
+                }
+                // take the candidates in the order the sequential rule would
+                uint32_t rem = key, T = M;
+                unsigned acc = 0u;
+                int my_order = -1;
+                while (n_acc < room) {
+                    uint32_t k = rem, src_lane = uint32_t(lane); int kj = my_j;
+                    warp_select(k, kj, src_lane);
+                    if (k == 0u || k <= T) break;
+                    const int wl = int(src_lane);
+                    if (!__shfl_sync(FULL, int(elig), wl)) break;
+                    const int nd = __shfl_sync(FULL, s_node, wl);
+                    if (__any_sync(FULL, ((acc >> lane) & 1u) && s_node == nd)) break;
+                    acc |= 1u << wl;
+                    if (lane == wl) { my_order = n_acc; rem = 0u; }
+                    const uint32_t bnd = __shfl_sync(FULL, s_bound, wl);
+                    T = bnd > T ? bnd : T;
+                    ++n_acc;
+                }
+                if (n_acc > 0) {
+                    if ((acc >> lane) & 1u) {
+                        if (s_ok && !s_multi) { v.gc[s_node] -= s_dgc; v.free_m[s_node] -= s_dm; }
+                        v.sa[s_slot] = na; v.sb[s_slot] = nb; v.sc[s_slot] = nq;
+                        sh.dirty[(s_slot % SCAN_T) >> 5] = 1;
+                        if (s_ok && !s_multi) atomicOr(&v.tb[s_node >> 5], 1u << (s_node & 31));
+                        if (A.step_log) A.step_log[steps0 + my_order] = (my_j << 2) | ((s_type ? 0 : 1) << 1) | int(s_ok);
+                    }
+                    // jobs on whole nodes: every node they own changes its share (no other job lives there)
+                    unsigned mm = __ballot_sync(FULL, ((acc >> lane) & 1u) && s_ok && s_multi);
+                    while (mm) {
+                        const int src = __ffs(mm) - 1;
+                        mm &= mm - 1;
+                        const int oj = __shfl_sync(FULL, my_j, src), dc = __shfl_sync(FULL, s_dgc, src);
+                        const long long dm = __shfl_sync(FULL, (long long)s_dm, src);
+                        for (int n = lane; n < N; n += 32)
+                            if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
+                    }
+                    const bool md = __any_sync(FULL, ((acc >> lane) & 1u) && s_ok && s_maxc);
+                    if (lane == 0) { sh.steps = steps0 + n_acc; sh.maxc_dirty = md ? 1 : 0; }
+                }
+            }
+            if (go && n_acc == 0) {
                 const int type_gpu = int(best >> 31);
                 const int j = best_j;
                 bool ok;
@@ -815,7 +1047,8 @@ static size_t fixed_smem(const Space &sp, int N)
 {
     const size_t n_cls = size_t(sp.nG) * sp.nC;
     const size_t n_pad = (size_t(N) + 127) & ~size_t(127);
-    const size_t fixed = n_pad * 4 + size_t(N) * 12 + n_cls * 24 + size_t(2 * RUBICK_MAX_G_LEVELS + RUBICK_MAX_C_LEVELS) * 4;
+    const size_t fixed = n_pad * 4 + size_t(N) * 12 + n_cls * 24 + size_t(2 * RUBICK_MAX_G_LEVELS + RUBICK_MAX_C_LEVELS) * 4
+                         + size_t(RUBICK_MAX_M_LEVELS) * 8 + n_pad / 8;
     return (fixed + 15) & ~size_t(15);
 }
 
@@ -889,7 +1122,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
         e = cudaFuncSetAttribute(round_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SORT_SMEM_KEYS * 8);
         if (e != cudaSuccess) return e;
     }
-    round_sort_kernel<<<1, RT, sort_smem ? size_t(L.n_pad) * 8 : 0, st>>>(keys, L.n_pad, d_jobs, sw, sort_smem);
+    round_sort_kernel<<<1, SORT_T, sort_smem ? size_t(L.n_pad) * 8 : 0, st>>>(keys, L.n_pad, d_jobs, sw, sort_smem);
 
     RoundArgs A;
     A.jobs = d_jobs; A.J = J; A.cv = d_cv; A.cp = d_cp; A.cg = d_cg; A.feas = d_feas; A.N = N; A.max_steps = max_steps;
