@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one eval_candidates launch from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), as bytes per stored candidate; valid only for the kernel source it was
 # taken on (sha1 of k_eval.cu), otherwise reported as null.
-NCU_EVAL_TRAFFIC = {"k_eval_sha1": None, "bytes_per_candidate": None}
+NCU_EVAL_TRAFFIC = {"k_eval_sha1": "be3bea64fb9d94bf621f04a5f1b0cff9846fb976", "bytes_per_candidate": 485.98554e6 / (2048 * 2640 * 24)}
 
 
 def shard_seed_offset(rank):
@@ -103,7 +103,7 @@ class ClockSampler:
         self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.file,
+                                          "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.file,
                                          stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
@@ -185,7 +185,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="throughput-stress", choices=list(workloads.CONFIGS))
