@@ -377,7 +377,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     }
     __syncwarp();
     if (rebuild) {
-        for (int i = 0; i < sp.n_small; ++i) {
+        for (int i = 0; i < sp.n_small && maxc_dirty; ++i) {
             const int m = max_cores_warp(v, sp.g_levels[i], lane);
             if (lane == 0) v.maxc[i] = m;
         }
@@ -437,14 +437,14 @@ __device__ void gains_thread(const Space &sp, const HotCurve *__restrict__ hc, i
 }
 
 // placement requirements of a slot's candidates (see SlotC)
-__device__ SlotC make_slotc(const Space &sp, int gi, int ci, int next_g, int next_c)
+__device__ SlotC make_slotc(const Space &sp, const int32_t *gl, const int32_t *clv, int gi, int ci, int next_g, int next_c)
 {
     SlotC s;
-    const int g = sp.g_levels[gi], c = sp.c_levels[ci];
+    const int g = gl[gi], c = clv[ci];
     s.gkind = K_NONE; s.ckind = K_NONE; s.gidx = 0; s.cidx = uint8_t(gi < sp.n_small ? gi : 0);
     s.dg = 0; s.need = 0; s.dc = 0; s.c = int16_t(c); s.c2 = 0; s.g = int16_t(g);
     if (next_g >= 0) {
-        const int g2 = sp.g_levels[next_g];
+        const int g2 = gl[next_g];
         if (g2 <= sp.Gn) { s.gkind = K_SINGLE; s.dg = int16_t(g2 - g); s.gidx = uint8_t(next_g); }
         else {
             const int k2 = g2 >> sp.log2Gn;
@@ -455,7 +455,7 @@ __device__ SlotC make_slotc(const Space &sp, int gi, int ci, int next_g, int nex
         }
     }
     if (next_c >= 0) {
-        const int c2 = sp.c_levels[next_c];
+        const int c2 = clv[next_c];
         s.c2 = int16_t(c2);
         if (g <= sp.Gn) { s.ckind = K_SINGLE; s.dc = int16_t(c2 - c); }
         else { const int k = g >> sp.log2Gn; if ((c2 + k - 1) / k <= sp.Cn) s.ckind = K_MULTI_WHOLE; }
@@ -643,7 +643,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         gains_thread(sp, A.hc, v.sj[s], b.w, pk_gi(a.packed), pk_ci(a.packed), b.val, ng_, gg, nc_, gc);
         a.gain_g = gg; a.gain_c = gc; a.packed = pack(pk_gi(a.packed), pk_ci(a.packed), ng_, false, false);
         v.sa[s] = a;
-        v.sc[s] = make_slotc(sp, pk_gi(a.packed), pk_ci(a.packed), ng_, nc_);
+        v.sc[s] = make_slotc(sp, v.gl, v.clv, pk_gi(a.packed), pk_ci(a.packed), ng_, nc_);
     }
     __syncthreads();
 
@@ -834,8 +834,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
                         const int64_t m_cur = v.ml[b.f_level];
                         const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
-                        int mi = -1;
-                        for (int i = 0; i < sp.nM; ++i) if (v.ml[i] <= avail) mi = i;
+                        int lo = 0, hi = sp.nM;                 // number of levels <= avail (levels ascend)
+                        while (lo < hi) { const int mid = (lo + hi) >> 1; if (v.ml[mid] <= avail) lo = mid + 1; else hi = mid; }
+                        const int mi = lo - 1;
                         s_multi = multi;
                         bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                         s_slot = s; s_node = a.node; s_type = type_gpu;
@@ -864,7 +865,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             na.gain_g = fz_g ? 0.0f : gg; na.gain_c = fz_c ? 0.0f : gc;
                             na.packed = pack(gi2, ci2, ng_, fz_g, fz_c); na.node = a.node;
                             nb.val = val; nb.plan = cand.plan; nb.f_level = cand.f; nb.w = b.w;
-                            nq = make_slotc(sp, gi2, ci2, ng_, nc_);
+                            nq = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                             if (multi) {
                                 // per-node shares of cores and memory on each of the k nodes (they hold no free GPU,
                                 // so maxc[] cannot change)
@@ -971,7 +972,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             const int s = sh.n_slots;
                             SlotA sa; sa.gain_g = gg; sa.gain_c = gc; sa.packed = pack(gi2, ci2, ng_, false, false); sa.node = cm.first;
                             SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
-                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j; v.sc[s] = make_slotc(sp, gi2, ci2, ng_, nc_);
+                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j; v.sc[s] = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                             sh.n_slots = s + 1;
                             sh.dirty[(s % SCAN_T) >> 5] = 1;
                         }
@@ -996,7 +997,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         a.gain_g = fz_g ? 0.0f : gg; a.gain_c = fz_c ? 0.0f : gc;
                         a.packed = pack(gi2, ci2, ng_, fz_g, fz_c); a.node = cm.first;
                         b.val = cm.val; b.plan = cm.plan; b.f_level = cm.f;
-                        if (lane == 0) v.sc[s] = make_slotc(sp, gi2, ci2, ng_, nc_);
+                        if (lane == 0) v.sc[s] = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                     } else {
                         if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
                         a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
