@@ -141,6 +141,7 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
     CHECK_CTX(ctx);
     if (!h_plans || !h_grid || P <= 0 || (P & 3)) return fail(ctx, RUBICK_EINVAL, "plans: need a positive multiple of 4");
     const rubick_grid &gr = *h_grid;
+    if (P > 65520) return fail(ctx, RUBICK_EINVAL, "plans: at most 65,520 plans (per-job plan tables live in shared memory)");
     if (gr.nG < 1 || gr.nG > RUBICK_MAX_G_LEVELS || gr.nC < 1 || gr.nC > RUBICK_MAX_C_LEVELS || gr.nM < 1
         || gr.nM > RUBICK_MAX_M_LEVELS || !gr.g_levels || !gr.c_levels || !gr.m_levels_bytes)
         return fail(ctx, RUBICK_EINVAL, "grid: level counts out of range or null axes");

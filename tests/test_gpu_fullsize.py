@@ -115,3 +115,23 @@ def test_event_driven_rounds_run_and_stay_consistent():
     r = events.run_events(gpu.ctx, cfg, n_events=25, warm_jobs=120)
     assert len(r["latency_ms"]) == 25 and (r["latency_ms"] > 0).all()
     assert r["active"].min() >= 100 and r["active"].max() <= 150 and (r["steps"] > 0).all()
+
+
+def test_round_with_slots_in_global_memory_matches_the_plain_kernel():
+    """2,048 nodes: more running-job slots than shared memory holds, so the fast round keeps them in
+    global scratch; the plain single-kernel round (itself checked against the oracle elsewhere) must
+    agree bit for bit."""
+    cfg = workloads.make("throughput-stress", J=9000, n_nodes=2048)
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    J, N = 9000, 2048
+    d_jobs, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    d_cv, d_cp, d_cg = gpu.best(d_thr, d_feas, J)
+    res = []
+    for call in (gpu.ctx.greedy_round, gpu.ctx.greedy_round_noalloc):
+        d_out = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_node = t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        steps, capped = call(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, 1 << 30, d_out, d_node)
+        res.append(unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped, None))
+    assert_rounds_equal(res[0], res[1])
+    assert (res[0]["status"] == rb.RUNNING).sum() > 2000 and (res[0]["n_nodes"] > 1).any()
