@@ -223,3 +223,24 @@ def bruteforce(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_leve
                                          _p(feas, C.c_uint32), C.c_int(feas.shape[1]), _p(gl, C.c_int64),
                                          C.c_int(len(gl)), _p(cl, C.c_int64), C.c_int(len(cl)),
                                          _p(ml, C.c_int64), C.c_int(len(ml))))
+
+
+def min_resources(thr, feas, curve_val, plans, g_levels, req):
+    """Minimum demand of guaranteed jobs.  req [J, 4] = requested g level, c level, m level, plan
+    (plan < 0: best effort) -> (gmin_idx, cmin_idx int32, baseline float64)."""
+    thr = _f64(thr)
+    feas = np.ascontiguousarray(feas, dtype=np.uint32)
+    cv = _f64(curve_val)
+    J, nC, Pn = thr.shape
+    nG, nM = cv.shape[1], cv.shape[3]
+    plans = _i32(plans)
+    gl = _i64(g_levels)
+    rq = _i64(req).reshape(J, 4)
+    gm = np.zeros(J, dtype=np.int32)
+    cm = np.zeros(J, dtype=np.int32)
+    base = np.zeros(J, dtype=np.float64)
+    lib().oracle_min_resources(_p(thr, C.c_double), _p(feas, C.c_uint32), _p(cv, C.c_double), C.c_int(J),
+                               _p(plans, C.c_int32), C.c_int(Pn), _p(gl, C.c_int64), C.c_int(nG), C.c_int(nC),
+                               C.c_int(nM), _p(rq, C.c_int64), _p(gm, C.c_int32), _p(cm, C.c_int32),
+                               _p(base, C.c_double))
+    return gm, cm, base

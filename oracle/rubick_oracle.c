@@ -347,6 +347,41 @@ void oracle_best_plan(const double *thr, const uint32_t *feas, int J, const int3
     (void)nthreads;
 }
 
+/* ---- minimum demand of a guaranteed job (Section 5.2, "Scheduling algorithm design") --------
+ * The job asked for (g_req, c_req, m_req) -- level indices -- with its original plan plan_req.
+ * Its guaranteed performance is what that plan predicts there (0 if the plan cannot run there).
+ * The minimum demand is the fewest resources, not above the request in any dimension, whose best
+ * plan reaches that performance and can run at all (non-zero curve); "fewest" is taken
+ * lexicographically, GPUs before cores.  If nothing qualifies the request itself is kept.
+ * plan_req < 0 marks a best-effort job: its minimum is nothing (-1, -1).
+ * req: [J][4] = g level, c level, m level, plan.  curve: running-maximum table [J][G][C][M]. */
+void oracle_min_resources(const double *thr, const uint32_t *feas, const double *curve_val, int J,
+                          const int32_t *plans, int P, const int64_t *g_levels, int nG, int nC, int nM,
+                          const int64_t *req, int32_t *gmin_idx, int32_t *cmin_idx, double *baseline)
+{
+    for (int j = 0; j < J; ++j) {
+        const int64_t *r = req + (size_t)j * 4;
+        int g_req = (int)r[0], c_req = (int)r[1], m_req = (int)r[2], plan = (int)r[3];
+        gmin_idx[j] = -1; cmin_idx[j] = -1; baseline[j] = 0.0;
+        if (plan < 0) continue;
+        double base = 0.0;
+        if (plan < P && g_req >= 0 && g_req < nG && c_req >= 0 && c_req < nC && m_req >= 0 && m_req < nM) {
+            const int32_t *pl = plans + (size_t)plan * PF_COUNT;
+            int64_t g = (int64_t)pl[PF_D] * pl[PF_T] * pl[PF_P];
+            if (g == g_levels[g_req] && ((feas[(size_t)j * P + plan] >> m_req) & 1u))
+                base = thr[((size_t)j * nC + c_req) * P + plan];
+        } else continue;
+        baseline[j] = base;
+        gmin_idx[j] = g_req; cmin_idx[j] = c_req;
+        int found = 0;
+        for (int gi = 0; gi <= g_req && !found; ++gi)
+            for (int ci = 0; ci <= c_req && !found; ++ci) {
+                double v = curve_val[(((size_t)j * nG + gi) * nC + ci) * nM + m_req];
+                if (v > 0.0 && v >= base) { gmin_idx[j] = gi; cmin_idx[j] = ci; found = 1; }
+            }
+    }
+}
+
 /* ======================================================================================
  * Scheduling: marginal gains and one greedy round.
  *

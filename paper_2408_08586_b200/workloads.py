@@ -71,6 +71,21 @@ def draw_jobs(rng, J, g_levels, n_c_levels, pmax=13e9, pmin=125e6, guaranteed_sh
     return jobs
 
 
+def draw_requests(seed, J, g_levels, n_c_levels, n_m_levels, guaranteed_share=0.5):
+    """What users asked for (Section 5.1: a requested amount of resources and an original plan):
+    level indices of GPUs / cores / host memory and `plan_rank` in [0, 1), the position of the
+    original plan among the plans of the requested GPU level (-1 marks a best-effort job).  Drawn
+    from a generator of its own so that the job fields above keep their values."""
+    rng = np.random.Generator(np.random.PCG64(seed + 2000))
+    pow2_idx = np.asarray([i for i, g in enumerate(g_levels) if g & (g - 1) == 0])
+    g_idx = rng.choice(pow2_idx, J)
+    c_idx = rng.integers(0, n_c_levels, J)
+    m_idx = rng.integers(n_m_levels // 2, n_m_levels, J)
+    rank = rng.uniform(0.0, 1.0, J)
+    guaranteed = rng.uniform(0.0, 1.0, J) < guaranteed_share
+    return dict(g_idx=g_idx, c_idx=c_idx, m_idx=m_idx, plan_rank=np.where(guaranteed, rank, -1.0))
+
+
 def make(name, J=None, n_nodes=None):
     """Build a named configuration; J / n_nodes override the size (same seed, same recipe)."""
     cfg = CONFIGS[name]

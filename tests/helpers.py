@@ -23,3 +23,15 @@ def env(**kw):
 
 def stack_jobs(*jobs):
     return {k: np.concatenate([np.asarray(j[k]) for j in jobs]) for k in jobs[0]}
+
+
+def requests_for(cfg, group_off, guaranteed_share=0.5):
+    """[J, 4] int64 requests (g level, c level, m level, original plan; plan -1 = best effort) from
+    the generator's draws; the plan is picked by rank inside the plans of the requested GPU level."""
+    J = len(cfg["jobs"]["P"])
+    rq = workloads.draw_requests(cfg["seed"], J, [int(g) for g in cfg["g_levels"]], len(cfg["c_levels"]),
+                                 len(cfg["m_levels"]), guaranteed_share)
+    off = np.asarray(group_off, dtype=np.int64)
+    size = off[rq["g_idx"] + 1] - off[rq["g_idx"]]
+    plan = np.where(rq["plan_rank"] >= 0, off[rq["g_idx"]] + np.floor(np.maximum(rq["plan_rank"], 0) * size).astype(np.int64), -1)
+    return np.stack([rq["g_idx"], rq["c_idx"], rq["m_idx"], plan], axis=1).astype(np.int64)

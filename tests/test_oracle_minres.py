@@ -1,0 +1,78 @@
+"""Pins of the oracle's minimum-demand search (paper Section 5.2: the fewest resources, not above
+the request in any dimension, whose best plan reaches the performance of the requested resources
+with the original plan and can run without running out of memory)."""
+import numpy as np
+import pytest
+
+import oracle
+from helpers import GIB, env, one_job, requests_for
+from paper_2408_08586_b200 import workloads
+
+
+def tables(cfg, nthreads=4):
+    plans, goff = oracle.enumerate_plans(cfg["g_levels"])
+    thr, feas = oracle.eval_candidates(cfg["jobs"], plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=nthreads)
+    cv, cp, cg = oracle.best_plan(thr, feas, plans, cfg["g_levels"], len(cfg["m_levels"]), prefix=True, nthreads=nthreads)
+    return plans, goff, thr, feas, cv
+
+
+def brute(thr, feas, cv, plans, g_levels, req):
+    J = thr.shape[0]
+    out = []
+    for j in range(J):
+        g, c, m, pl = (int(x) for x in req[j])
+        if pl < 0:
+            out.append((-1, -1, 0.0))
+            continue
+        runs = int(np.prod(plans[pl, :3])) == g_levels[g] and (feas[j, pl] >> m) & 1
+        base = float(thr[j, c, pl]) if runs else 0.0
+        ok = [(gi, ci) for gi in range(g + 1) for ci in range(c + 1) if cv[j, gi, ci, m] > 0 and cv[j, gi, ci, m] >= base]
+        out.append((*(min(ok) if ok else (g, c)), base))
+    return out
+
+
+@pytest.mark.parametrize("name", ["tiny", "paper-scale"])
+def test_minimum_demand_matches_an_exhaustive_scan(name):
+    cfg = workloads.make(name)
+    plans, goff, thr, feas, cv = tables(cfg)
+    req = requests_for(cfg, goff, guaranteed_share=0.8)
+    gm, cm, base = oracle.min_resources(thr, feas, cv, plans, cfg["g_levels"], req)
+    want = brute(thr, feas, cv, plans, cfg["g_levels"], req)
+    assert [(int(a), int(b), float(c)) for a, b, c in zip(gm, cm, base)] == want
+    guar = req[:, 3] >= 0
+    assert guar.any() and (name == "tiny" or (~guar).any())
+    assert np.all(gm[~guar] == -1) and np.all(cm[~guar] == -1)
+    # never above the request, and the guarantee holds at the minimum
+    assert np.all(gm[guar] <= req[guar, 0]) and np.all(cm[guar] <= req[guar, 1])
+    j = np.nonzero(guar)[0]
+    at_min = cv[j, gm[j], cm[j], req[j, 2]]
+    assert np.all(at_min >= base[j])
+    if name == "paper-scale":
+        # the point of the definition: the same performance with fewer resources under a better plan
+        assert ((gm[j] < req[j, 0]) & (base[j] > 0)).any()
+        assert (base[j] > 0).any() and (base[j] == 0).any()
+
+
+def test_hand_made_case():
+    # one job asking for 8 GPUs with pure data parallelism + gradient checkpointing + ZeRO-3 + offload
+    # (a slow plan): plain data parallelism on fewer GPUs already reaches that speed
+    cfg = workloads.make("tiny")
+    cfg["jobs"] = one_job(P=4e8, b=64, mu_cap=8, l=24, h=1024, s=512, k_opt_off=2e-7, k_off=1.0, k_swap=1.0)
+    plans, goff, thr, feas, cv = tables(cfg)
+    slow = [i for i, p in enumerate(plans) if tuple(p) == (8, 1, 1, 3, 1, 1)][0]
+    req = np.array([[7, 3, 2, slow]])
+    gm, cm, base = oracle.min_resources(thr, feas, cv, plans, cfg["g_levels"], req)
+    assert base[0] == thr[0, 3, slow] > 0
+    assert cfg["g_levels"][gm[0]] < 8 and cv[0, gm[0], cm[0], 2] >= base[0]
+    # one level less of either resource no longer reaches it (or cannot run)
+    if gm[0] > 0:
+        assert np.all(cv[0, :gm[0], :4, 2] < base[0])
+    if cm[0] > 0:
+        assert cv[0, gm[0], cm[0] - 1, 2] < base[0]
+    # a plan that cannot run at the request (wrong GPU count for the level) guarantees nothing: any runnable allocation will do
+    req = np.array([[3, 3, 2, slow]])
+    gm, cm, base = oracle.min_resources(thr, feas, cv, plans, cfg["g_levels"], req)
+    assert base[0] == 0 and (gm[0], cm[0]) == (0, 0)
+    # best effort
+    gm, cm, base = oracle.min_resources(thr, feas, cv, plans, cfg["g_levels"], np.array([[7, 3, 2, -1]]))
+    assert (gm[0], cm[0], base[0]) == (-1, -1, 0)
