@@ -114,6 +114,10 @@ typedef struct {
     int32_t m_level;             /* host-memory level index of m_bytes, -1 if none                  */
 } rubick_assignment;
 
+/* What a user asked for (paper Section 5.1): resource amounts as level indices and the original
+ * plan; plan < 0 marks a best-effort job. 16 bytes. */
+typedef struct { int32_t g_idx, c_idx, m_idx, plan; } rubick_request;
+
 /* Per-node state after a round. 24 bytes. */
 typedef struct {
     int32_t free_g, free_c;
@@ -187,6 +191,18 @@ int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas
 int rubick_marginal_gain(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_curve_val,
                          const rubick_assignment *d_state,
                          float *d_gain_gpu, float *d_gain_cpu, int32_t *d_next_g, int32_t *d_next_c);
+
+/* Minimum demand of guaranteed jobs (Section 5.2, "Scheduling algorithm design"): the job's
+ * guaranteed performance is what its original plan predicts at the requested resources
+ * (d_thr[j][c_idx][plan] if the plan uses g_levels[g_idx] GPUs and is feasible at memory level
+ * m_idx, else 0); its minimum demand is the lexicographically smallest (GPU level, core level), not
+ * above the request in either dimension, whose sensitivity-curve value at memory level m_idx is
+ * non-zero and reaches that performance; the request itself if there is none.  Writes the two
+ * level indices (the values rubick_job.gmin_idx / cmin_idx take) and the guaranteed performance;
+ * (-1, -1, 0) for best-effort jobs and for requests with indices off the grid.
+ * d_curve_val must be the running-maximum table of rubick_best_plan (not RUBICK_BEST_RAW). */
+int rubick_min_resources(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas, const float *d_curve_val, int J,
+                         const rubick_request *d_req, int32_t *d_gmin_idx, int32_t *d_cmin_idx, float *d_baseline);
 
 /* One greedy scheduling round (Section 5.2, Algorithm 1 in marginal-gain form) on given curve
  * tables, from an empty cluster, entirely on the device: guaranteed minima first, in job order;

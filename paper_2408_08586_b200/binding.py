@@ -27,6 +27,7 @@ PLAN_DTYPE = np.dtype([("log2d", "u1"), ("log2t", "u1"), ("log2p", "u1"), ("zero
                        ("off", "u1"), ("g_level", "u1"), ("disabled", "u1")])
 ASSIGN_DTYPE = np.dtype([("g", "<i4"), ("c", "<i4"), ("m_bytes", "<i8"), ("plan", "<i4"), ("first_node", "<i4"),
                          ("n_nodes", "<i4"), ("thr", "<f4"), ("status", "<i4"), ("m_level", "<i4")])
+REQUEST_DTYPE = np.dtype([("g_idx", "<i4"), ("c_idx", "<i4"), ("m_idx", "<i4"), ("plan", "<i4")])
 NODE_DTYPE = np.dtype([("free_g", "<i4"), ("free_c", "<i4"), ("free_m", "<i8"), ("owner", "<i4"), ("reserved", "<i4")])
 assert JOB_DTYPE.itemsize == 128 and PLAN_DTYPE.itemsize == 8
 assert ASSIGN_DTYPE.itemsize == 40 and NODE_DTYPE.itemsize == 24
@@ -50,6 +51,7 @@ class Cluster(C.Structure):
 
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
            "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_marginal_gain",
+           "rubick_min_resources",
            "rubick_greedy_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
            "rubick_schedule_round_host"]
 
@@ -82,6 +84,7 @@ def lib():
         L.rubick_eval_candidates.argtypes = [vp, vp, ip, vp, vp]
         L.rubick_best_plan.argtypes = [vp, vp, vp, ip, C.c_uint, vp, vp, vp]
         L.rubick_marginal_gain.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp]
+        L.rubick_min_resources.argtypes = [vp, vp, vp, vp, ip, vp, vp, vp, vp]
         L.rubick_greedy_round.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_greedy_round_noalloc.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
@@ -198,6 +201,10 @@ class Context:
     def marginal_gain(self, d_jobs, J, d_curve_val, d_state, d_gain_gpu, d_gain_cpu, d_next_g, d_next_c):
         return self._check(lib().rubick_marginal_gain(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_state),
                                                       _ptr(d_gain_gpu), _ptr(d_gain_cpu), _ptr(d_next_g), _ptr(d_next_c)))
+
+    def min_resources(self, d_thr, d_feas, d_curve_val, J, d_req, d_gmin_idx, d_cmin_idx, d_baseline):
+        return self._check(lib().rubick_min_resources(self._h, _ptr(d_thr), _ptr(d_feas), _ptr(d_curve_val), int(J), _ptr(d_req),
+                                                      _ptr(d_gmin_idx), _ptr(d_cmin_idx), _ptr(d_baseline)))
 
     def greedy_round(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, n_nodes, max_steps, d_out,
                      d_node_out=None, d_step_log=None):

@@ -270,6 +270,20 @@ int rubick_marginal_gain(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const
     return RUBICK_OK;
 }
 
+int rubick_min_resources(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas, const float *d_curve_val, int J,
+                         const rubick_request *d_req, int32_t *d_gmin_idx, int32_t *d_cmin_idx, float *d_baseline)
+{
+    CHECK_CTX(ctx);
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (J == 0) return RUBICK_OK;
+    if (!d_thr || !d_feas || !d_curve_val || !d_req || !d_gmin_idx || !d_cmin_idx || !d_baseline) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    CUDA_TRY(ctx, launch_min_resources(ctx->space, ctx->d_quads, d_thr, d_feas, d_curve_val, J, d_req, d_gmin_idx, d_cmin_idx,
+                                       d_baseline, ctx->stream),
+             "launch min_resources");
+    return RUBICK_OK;
+}
+
 // enqueue the round and leave the step count in ctx->d_steps
 static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps, rubick_assignment *d_out,

@@ -127,6 +127,46 @@ cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const 
 }
 
 // ------------------------------------------------------------------------------------------------
+// minimum demand of guaranteed jobs (paper Section 5.2): one thread per job walks the curve from the
+// smallest allocation upwards, GPUs before cores, and stops at the first one that runs and reaches
+// the performance the original plan predicts at the requested resources
+// ------------------------------------------------------------------------------------------------
+__global__ void min_resources_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads,
+                                     const float *__restrict__ thr, const uint32_t *__restrict__ feas,
+                                     const float *__restrict__ cv, int J, const rubick_request *__restrict__ req,
+                                     int32_t *__restrict__ gmin_idx, int32_t *__restrict__ cmin_idx,
+                                     float *__restrict__ baseline)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= J) return;
+    const rubick_request r = req[j];
+    int gm = -1, cm = -1; float base = 0.0f;
+    if (r.plan >= 0 && r.plan < sp.P && r.g_idx >= 0 && r.g_idx < sp.nG && r.c_idx >= 0 && r.c_idx < sp.nC
+        && r.m_idx >= 0 && r.m_idx < sp.nM) {
+        // the original plan runs at the request if it uses exactly that many GPUs and fits that much memory
+        const bool runs = quads[r.plan >> 2].g_level == r.g_idx && ((feas[size_t(j) * sp.P + r.plan] >> r.m_idx) & 1u);
+        if (runs) base = thr[(size_t(j) * sp.nC + r.c_idx) * sp.P + r.plan];
+        gm = r.g_idx; cm = r.c_idx;
+        bool found = false;
+        for (int gi = 0; gi <= r.g_idx && !found; ++gi)
+            for (int ci = 0; ci <= r.c_idx && !found; ++ci) {
+                const float v = cv[curve_idx(sp, j, gi, ci, r.m_idx)];
+                if (v > 0.0f && v >= base) { gm = gi; cm = ci; found = true; }
+            }
+    }
+    gmin_idx[j] = gm; cmin_idx[j] = cm; baseline[j] = base;
+}
+
+cudaError_t launch_min_resources(const Space &sp, const QuadDesc *d_quads, const float *d_thr, const uint32_t *d_feas,
+                                 const float *d_cv, int J, const rubick_request *d_req, int32_t *d_gmin, int32_t *d_cmin,
+                                 float *d_baseline, cudaStream_t st)
+{
+    if (J == 0) return cudaSuccess;
+    min_resources_kernel<<<(J + 127) / 128, 128, 0, st>>>(sp, d_quads, d_thr, d_feas, d_cv, J, d_req, d_gmin, d_cmin, d_baseline);
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------------
 // greedy round
 // ------------------------------------------------------------------------------------------------
 

@@ -97,6 +97,9 @@ cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_f
 cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const float *d_curve_val,
                         const rubick_assignment *d_state, float *d_gain_gpu, float *d_gain_cpu,
                         int32_t *d_next_g, int32_t *d_next_c, cudaStream_t st);
+cudaError_t launch_min_resources(const Space &sp, const QuadDesc *d_quads, const float *d_thr, const uint32_t *d_feas,
+                                 const float *d_cv, int J, const rubick_request *d_req, int32_t *d_gmin, int32_t *d_cmin,
+                                 float *d_baseline, cudaStream_t st);
 size_t round_scratch_need(const Space &sp, int J, int N);
 cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
