@@ -45,6 +45,7 @@ extern "C" {
 #define RUBICK_MAX_C_LEVELS  64
 #define RUBICK_MAX_M_LEVELS  32      /* one feasibility word per (job, plan) */
 #define RUBICK_MAX_NODES     4096    /* node state of a round lives in shared memory */
+#define RUBICK_MAX_TENANTS   256
 #define RUBICK_NOALLOC_MAX_JOBS 32768 /* job limit of rubick_greedy_round_noalloc (1 MiB fixed state) */
 
 /* per-job status in rubick_assignment */
@@ -80,7 +81,8 @@ typedef struct {
     float    w;                  /* weight of this job's throughput in the scheduling objective     */
     int32_t  gmin_idx, cmin_idx; /* guaranteed minimum as level indices; -1 = best effort / none    */
     uint32_t flags;              /* reserved, 0                                                     */
-    uint8_t  pad[40];
+    int32_t  tenant;             /* owner of the job for quota accounting, 0 .. n_tenants - 1       */
+    uint8_t  pad[36];
 } rubick_job;
 
 /* One execution plan (paper Section 3): DP / TP / PP degrees as log2, ZeRO stage 0..3, gradient
@@ -100,8 +102,17 @@ typedef struct {
     const int64_t *m_levels_bytes;   /* host memory in bytes [nM] */
 } rubick_grid;
 
-/* Homogeneous cluster: n_nodes nodes of the environment's shape, all free at the start of a round. */
-typedef struct { int32_t n_nodes; } rubick_cluster;
+/* Homogeneous cluster: n_nodes nodes of the environment's shape, all free at the start of a round.
+ * Tenant quotas (paper Section 5.1) are optional: with n_tenants > 0, a guaranteed job is placed in
+ * the first phase of a round only while its minimum demand (GPUs, cores) fits what is left of its
+ * tenant's quota, and uses that much of it once placed; jobs beyond the quota stay PENDING.
+ * n_tenants = 0 (pointers ignored): no quotas.  At most RUBICK_MAX_TENANTS tenants. */
+typedef struct {
+    int32_t n_nodes;
+    int32_t n_tenants;
+    const int32_t *quota_gpus;       /* host, [n_tenants] */
+    const int32_t *quota_cpus;       /* host, [n_tenants] */
+} rubick_cluster;
 
 /* Result (and input state) per job. 40 bytes. */
 typedef struct {
@@ -223,7 +234,7 @@ int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
  * that fill the rest (a late cudaMalloc may fail, and stalls the device while it runs), or a
  * process whose device memory belongs to a framework's caching allocator.  (The paper has no counterpart; this is
  * a convenience of this library.)  Same inputs, outputs, order of decisions and return codes
- * as rubick_greedy_round, without the step log.  It calls no cudaMalloc, cudaFree or other
+ * as rubick_greedy_round, without the step log and without tenant quotas (n_tenants must be 0).  It calls no cudaMalloc, cudaFree or other
  * allocating routine: the per-job scan state lives in a fixed 1 MiB array inside the library
  * (32 bytes per job), which every GPU that loads the library holds until the process exits.
  *  - J above RUBICK_NOALLOC_MAX_JOBS is rejected with EINVAL and a message naming the limit.

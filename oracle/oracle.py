@@ -16,7 +16,7 @@ _SRC = os.path.join(_HERE, "rubick_oracle.c")
 _SO = os.path.join(_HERE, "liboracle.so")
 
 JOB_FIELDS = ["P", "l", "h", "s", "b", "mu_cap", "alpha_act", "tau", "k_bwd", "k_sync", "k_opt",
-              "k_opt_off", "k_off", "k_swap", "k_const", "w", "gmin_idx", "cmin_idx", "host_base_bytes"]
+              "k_opt_off", "k_off", "k_swap", "k_const", "w", "gmin_idx", "cmin_idx", "host_base_bytes", "tenant"]
 ENV_FIELDS = ["B_intra", "B_inter", "B_pcie", "gpu_mem_bytes", "gpus_per_node", "cpus_per_node",
               "mem_per_node_bytes", "bytes_per_elem", "strict_zero_dp_only"]
 TERM_FIELDS = ["valid", "mu", "m", "a", "T_fwd", "T_bwd", "V_dp", "V_tp", "V_pp", "T_dp", "T_tp",
@@ -71,6 +71,8 @@ def job_rows(jobs):
     J = len(np.atleast_1d(jobs["P"]))
     rows = np.zeros((J, len(JOB_FIELDS)), dtype=np.float64)
     for i, k in enumerate(JOB_FIELDS):
+        if k == "tenant" and k not in jobs:
+            continue                                   # single tenant
         rows[:, i] = np.asarray(jobs[k], dtype=np.float64)
     return rows
 
@@ -178,7 +180,7 @@ def gain(jobs, curve_val, g_levels, c_levels, state_g, state_c, state_val):
 
 
 def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,
-                   n_nodes, max_steps=1 << 30, want_log=False):
+                   n_nodes, max_steps=1 << 30, want_log=False, quota=None):
     """One greedy round on single-precision curve tables.
 
     -> dict(g, c, m_bytes, plan, first_node, n_nodes, status, m_level, thr, node (N x 4:
@@ -195,10 +197,12 @@ def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_
     node = np.zeros((n_nodes, 4), dtype=np.int64)
     cap = int(min(max_steps, J * (len(gl) + len(cl) + 2) + 1))
     log = np.zeros(max(cap, 1), dtype=np.int32)
+    qt = None if quota is None else _i64(quota).reshape(-1, 2)      # per tenant: GPUs, cores
     r = lib().oracle_round(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double), _p(cv, C.c_float),
                            _p(cp, C.c_int32), _p(cg, C.c_int32), _p(feas, C.c_uint32), C.c_int(Pn),
                            _p(gl, C.c_int64), C.c_int(len(gl)), _p(cl, C.c_int64), C.c_int(len(cl)),
                            _p(ml, C.c_int64), C.c_int(len(ml)), C.c_int(n_nodes), C.c_int(cap),
+                           _p(qt, C.c_int64) if qt is not None else None, C.c_int(0 if qt is None else len(qt)),
                            _p(out_i, C.c_int64), _p(out_v, C.c_float), _p(node, C.c_int64),
                            _p(log, C.c_int32) if want_log else None)
     capped = r < 0

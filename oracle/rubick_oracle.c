@@ -54,6 +54,7 @@ enum {
     JF_GMIN,       /* guaranteed minimum GPU level index, -1 = best effort */
     JF_CMIN,       /* guaranteed minimum CPU level index, -1 = none        */
     JF_HOSTBASE,   /* host bytes per training process (one per GPU)      */
+    JF_TENANT,     /* tenant the job belongs to (quota accounting)       */
     JF_COUNT
 };
 
@@ -591,7 +592,10 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
 }
 
 /* One scheduling round from an empty cluster of N identical nodes.
- * Phase A: jobs with a guaranteed minimum, in index order, are placed at it.
+ * Phase A: jobs with a guaranteed minimum, in index order, are placed at it -- the paper's
+ * "privileged" jobs: with tenant quotas (n_tenants > 0; quota[t] = GPUs, cores) only while the
+ * minimum fits what is left of the job's tenant's quota, which a placed job then uses up
+ * (Section 5.2: "the quota usage of each job [is] its minimum demand"); others stay pending.
  * Phase B: repeatedly take, among increments that can be placed, the largest positive
  * GPU gain (lowest job index on ties); when there is none, the largest positive CPU gain;
  * stop when there is neither or after max_steps increments were tried.
@@ -604,6 +608,7 @@ int oracle_round(const double *jobs, int J, const double *env,
                  const uint32_t *feas, int P,
                  const int64_t *g_levels, int nG, const int64_t *c_levels, int nC,
                  const int64_t *m_levels, int nM, int N, int max_steps,
+                 const int64_t *quota, int n_tenants,
                  int64_t *out_i, float *out_val, int64_t *node_out, int32_t *step_log)
 {
     Sched S; memset(&S, 0, sizeof S);
@@ -621,6 +626,11 @@ int oracle_round(const double *jobs, int J, const double *env,
 
     /* Phase A: guaranteed minima */
     int mt = nM - 1;
+    int64_t *rem = NULL;
+    if (n_tenants > 0) {
+        rem = (int64_t *)malloc(sizeof(int64_t) * 2 * (size_t)n_tenants);
+        memcpy(rem, quota, sizeof(int64_t) * 2 * (size_t)n_tenants);
+    }
     for (int j = 0; j < J; ++j) {
         const double *job = jobs + (size_t)j * JF_COUNT;
         int gmin = (int)job[JF_GMIN];
@@ -634,11 +644,18 @@ int oracle_round(const double *jobs, int J, const double *env,
         int gi = -1;
         for (int i = 0; i < nG; ++i) if (g_levels[i] == (int64_t)curve_g[o]) gi = i;
         if (gi < 0) continue;
+        int t = (int)job[JF_TENANT];
+        if (n_tenants > 0) {
+            if (t < 0 || t >= n_tenants) continue;
+            if (rem[2 * t] < g_levels[gi] || rem[2 * t + 1] < c_levels[cmin]) continue;   /* beyond the quota: not privileged */
+        }
         Place pl = find_place(&S, &st[j], g_levels[gi], c_levels[cmin]);
         if (!pl.ok) continue;
         commit(&S, j, &st[j], gi, cmin, pl, 0);
         if (st[j].gi < 0) st[j].status = ST_PENDING;
+        else if (n_tenants > 0) { rem[2 * t] -= g_levels[gi]; rem[2 * t + 1] -= c_levels[cmin]; }
     }
+    free(rem);
 
     /* Phase B: greedy increments */
     int steps = 0, capped = 0;

@@ -22,7 +22,7 @@ JOB_DTYPE = np.dtype([
     ("P", "<f8"), ("host_base_bytes", "<i8"), ("l", "<i4"), ("h", "<i4"), ("s", "<i4"), ("b", "<i4"),
     ("mu_cap", "<i4"), ("alpha_act", "<i4"), ("tau", "<f4"), ("k_bwd", "<f4"), ("k_sync", "<f4"),
     ("k_opt", "<f4"), ("k_opt_off", "<f4"), ("k_off", "<f4"), ("k_swap", "<f4"), ("k_const", "<f4"),
-    ("w", "<f4"), ("gmin_idx", "<i4"), ("cmin_idx", "<i4"), ("flags", "<u4"), ("pad", "u1", (40,))])
+    ("w", "<f4"), ("gmin_idx", "<i4"), ("cmin_idx", "<i4"), ("flags", "<u4"), ("tenant", "<i4"), ("pad", "u1", (36,))])
 PLAN_DTYPE = np.dtype([("log2d", "u1"), ("log2t", "u1"), ("log2p", "u1"), ("zero", "u1"), ("gc", "u1"),
                        ("off", "u1"), ("g_level", "u1"), ("disabled", "u1")])
 ASSIGN_DTYPE = np.dtype([("g", "<i4"), ("c", "<i4"), ("m_bytes", "<i8"), ("plan", "<i4"), ("first_node", "<i4"),
@@ -46,7 +46,18 @@ class Grid(C.Structure):
 
 
 class Cluster(C.Structure):
-    _fields_ = [("n_nodes", C.c_int32)]
+    _fields_ = [("n_nodes", C.c_int32), ("n_tenants", C.c_int32), ("quota_gpus", C.POINTER(C.c_int32)),
+                ("quota_cpus", C.POINTER(C.c_int32))]
+
+
+def make_cluster(n_nodes, quota=None):
+    """rubick_cluster for n_nodes nodes; quota = None or an [n_tenants, 2] array of (GPUs, cores).
+    Returns (struct, keep-alive objects)."""
+    if quota is None:
+        return Cluster(int(n_nodes), 0, None, None), ()
+    q = np.ascontiguousarray(quota, dtype=np.int32).reshape(-1, 2)
+    qg, qc = np.ascontiguousarray(q[:, 0]), np.ascontiguousarray(q[:, 1])
+    return Cluster(int(n_nodes), len(q), qg.ctypes.data_as(C.POINTER(C.c_int32)), qc.ctypes.data_as(C.POINTER(C.c_int32))), (qg, qc)
 
 
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
@@ -125,7 +136,7 @@ def pack_jobs(jobs):
     J = len(np.atleast_1d(jobs["P"]))
     rec = np.zeros(J, dtype=JOB_DTYPE)
     for name in JOB_DTYPE.names:
-        if name in ("flags", "pad"):
+        if name in ("flags", "pad") or (name == "tenant" and name not in jobs):
             continue
         rec[name] = np.asarray(jobs[name])
     return rec
@@ -207,10 +218,10 @@ class Context:
                                                       _ptr(d_gmin_idx), _ptr(d_cmin_idx), _ptr(d_baseline)))
 
     def greedy_round(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, n_nodes, max_steps, d_out,
-                     d_node_out=None, d_step_log=None):
-        """-> (steps, capped)"""
+                     d_node_out=None, d_step_log=None, quota=None):
+        """-> (steps, capped); quota: None or [n_tenants, 2] (GPUs, cores)"""
         steps = C.c_int32(0)
-        cl = Cluster(int(n_nodes))
+        cl, _keep = make_cluster(n_nodes, quota)
         rc = self._check(lib().rubick_greedy_round(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_curve_plan),
                                                    _ptr(d_curve_g), _ptr(d_feas), C.byref(cl), int(max_steps), _ptr(d_out),
                                                    _ptr(d_node_out), _ptr(d_step_log), C.byref(steps)), allow=(ESTEPS,))
@@ -222,24 +233,24 @@ class Context:
         for callers that may not allocate device memory; at most NOALLOC_MAX_JOBS jobs.
         -> (steps, capped)"""
         steps = C.c_int32(0)
-        cl = Cluster(int(n_nodes))
+        cl, _keep = make_cluster(n_nodes)
         rc = self._check(lib().rubick_greedy_round_noalloc(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val),
                                                            _ptr(d_curve_plan), _ptr(d_curve_g), _ptr(d_feas), C.byref(cl),
                                                            int(max_steps), _ptr(d_out), _ptr(d_node_out), C.byref(steps)),
                          allow=(ESTEPS,))
         return steps.value, rc == ESTEPS
 
-    def schedule_round(self, d_jobs, J, n_nodes, max_steps, d_out, d_node_out=None):
+    def schedule_round(self, d_jobs, J, n_nodes, max_steps, d_out, d_node_out=None, quota=None):
         steps = C.c_int32(0)
-        cl = Cluster(int(n_nodes))
+        cl, _keep = make_cluster(n_nodes, quota)
         rc = self._check(lib().rubick_schedule_round(self._h, _ptr(d_jobs), int(J), C.byref(cl), int(max_steps), _ptr(d_out),
                                                      _ptr(d_node_out), C.byref(steps)), allow=(ESTEPS,))
         return steps.value, rc == ESTEPS
 
-    def schedule_round_host(self, h_jobs, J, n_nodes, max_steps, h_out, h_node_out=None):
+    def schedule_round_host(self, h_jobs, J, n_nodes, max_steps, h_out, h_node_out=None, quota=None):
         """h_jobs: JOB_DTYPE array (or pinned torch uint8 tensor); h_out: ASSIGN_DTYPE array / tensor."""
         steps = C.c_int32(0)
-        cl = Cluster(int(n_nodes))
+        cl, _keep = make_cluster(n_nodes, quota)
         rc = self._check(lib().rubick_schedule_round_host(self._h, _ptr(h_jobs), int(J), C.byref(cl), int(max_steps),
                                                           _ptr(h_out), _ptr(h_node_out), C.byref(steps)), allow=(ESTEPS,))
         return steps.value, rc == ESTEPS

@@ -75,8 +75,9 @@ int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *c
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return RUBICK_ECUDA; }
     ctx->num_sms = prop.multiProcessorCount;
-    if (cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 8) != cudaSuccess) { delete ctx; return RUBICK_ENOMEM; }
+    if (cudaMalloc(reinterpret_cast<void **>(&ctx->d_status), 8 + 8 * RUBICK_MAX_TENANTS) != cudaSuccess) { delete ctx; return RUBICK_ENOMEM; }
     ctx->d_steps = reinterpret_cast<int32_t *>(ctx->d_status + 1);
+    ctx->d_quota = reinterpret_cast<int32_t *>(ctx->d_status + 2);
     if (cudaMemsetAsync(ctx->d_status, 0, 8, ctx->stream) != cudaSuccess) { cudaFree(ctx->d_status); delete ctx; return RUBICK_ECUDA; }
     *out = ctx;
     return RUBICK_OK;
@@ -286,9 +287,17 @@ int rubick_min_resources(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_
 
 // enqueue the round and leave the step count in ctx->d_steps
 static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
-                         const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps, rubick_assignment *d_out,
-                         rubick_node *d_node_out, int32_t *d_step_log)
+                         const int32_t *d_cg, const uint32_t *d_feas, const rubick_cluster *cl, int max_steps,
+                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log)
 {
+    const int N = cl->n_nodes, T = cl->n_tenants;
+    if (T > 0) {
+        // interleave (GPUs, cores) per tenant; the staging vector lives in the context until the next round
+        cudaStreamSynchronize(ctx->stream);
+        ctx->h_quota.resize(size_t(2) * T);
+        for (int t = 0; t < T; ++t) { ctx->h_quota[2 * t] = cl->quota_gpus[t]; ctx->h_quota[2 * t + 1] = cl->quota_cpus[t]; }
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_quota, ctx->h_quota.data(), size_t(8) * T, cudaMemcpyHostToDevice, ctx->stream), "upload quotas");
+    }
     const bool fast = round_fast_supported(ctx->space, J, N);
     const size_t need = fast ? round_fast_scratch_need(ctx->space, J, N) : round_scratch_need(ctx->space, J, N);
     if (need > ctx->round_scratch_bytes) {
@@ -298,11 +307,11 @@ static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const
     }
     if (fast)
         CUDA_TRY(ctx, launch_round_fast(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
-                                        ctx->d_round_scratch, ctx->d_status, ctx->d_steps, ctx->stream),
+                                        ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream),
                  "launch greedy_round (fast path)");
     else
         CUDA_TRY(ctx, launch_round(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
-                                   ctx->d_round_scratch, ctx->d_status, ctx->d_steps, ctx->stream),
+                                   ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream),
                  "launch greedy_round");
     return RUBICK_OK;
 }
@@ -332,6 +341,8 @@ static int check_round_args(rubick_ctx *ctx, int J, const rubick_cluster *h_clus
     int rc = check_ready(ctx, J);
     if (rc) return rc;
     if (!h_cluster || h_cluster->n_nodes < 1 || h_cluster->n_nodes > RUBICK_MAX_NODES) return fail(ctx, RUBICK_EINVAL, "cluster: 1 .. RUBICK_MAX_NODES nodes");
+    if (h_cluster->n_tenants < 0 || h_cluster->n_tenants > RUBICK_MAX_TENANTS || (h_cluster->n_tenants > 0 && (!h_cluster->quota_gpus || !h_cluster->quota_cpus)))
+        return fail(ctx, RUBICK_EINVAL, "cluster: 0 .. RUBICK_MAX_TENANTS tenants with both quota arrays");
     if (max_steps < 0) return fail(ctx, RUBICK_EINVAL, "negative max_steps");
     if (J >= (1 << 29)) return fail(ctx, RUBICK_EINVAL, "too many jobs");
     return RUBICK_OK;
@@ -347,7 +358,7 @@ int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
     int rc = check_round_args(ctx, J, h_cluster, max_steps);
     if (rc) return rc;
     if (J > 0 && (!d_jobs || !d_curve_val || !d_curve_plan || !d_curve_g || !d_feas || !d_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
-    rc = enqueue_round(ctx, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, h_cluster->n_nodes, max_steps, d_out,
+    rc = enqueue_round(ctx, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, h_cluster, max_steps, d_out,
                        d_node_out, d_step_log);
     if (rc) return rc;
     return finish_round(ctx, h_steps);
@@ -390,7 +401,7 @@ int rubick_schedule_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, cons
     if (J > 0 && (!d_jobs || !d_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
     if (J > 0 && (reinterpret_cast<uintptr_t>(d_jobs) & 15)) return fail(ctx, RUBICK_EINVAL, "d_jobs must be 16-byte aligned");
     if ((rc = enqueue_tables(ctx, d_jobs, J))) return rc;
-    if ((rc = enqueue_round(ctx, d_jobs, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster->n_nodes, max_steps, d_out, d_node_out, nullptr))) return rc;
+    if ((rc = enqueue_round(ctx, d_jobs, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster, max_steps, d_out, d_node_out, nullptr))) return rc;
     return finish_round(ctx, h_steps);
 }
 
@@ -407,7 +418,7 @@ int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J,
     if ((rc = ensure(ctx, ctx->d_node_stage, ctx->cap_node, size_t(N)))) return rc;
     if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_jobs_stage, h_jobs, size_t(J) * sizeof(rubick_job), cudaMemcpyHostToDevice, ctx->stream), "copy jobs to device");
     if ((rc = enqueue_tables(ctx, ctx->d_jobs_stage, J))) return rc;
-    if ((rc = enqueue_round(ctx, ctx->d_jobs_stage, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, N, max_steps, ctx->d_out_stage,
+    if ((rc = enqueue_round(ctx, ctx->d_jobs_stage, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster, max_steps, ctx->d_out_stage,
                             ctx->d_node_stage, nullptr))) return rc;
     if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_out_stage, size_t(J) * sizeof(rubick_assignment), cudaMemcpyDeviceToHost, ctx->stream), "copy assignments to host");
     if (h_node_out) CUDA_TRY(ctx, cudaMemcpyAsync(h_node_out, ctx->d_node_stage, size_t(N) * sizeof(rubick_node), cudaMemcpyDeviceToHost, ctx->stream), "copy node states to host");

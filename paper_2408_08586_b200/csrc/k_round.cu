@@ -116,7 +116,7 @@ __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick
         const rubick_job *jb = jobs + j;
         const int gmin = jb->gmin_idx;
         const float w = jb->w;
-        PhaseA a; a.gi = -2; a.ci = 0; a.val = 0.0f; a.plan = -1; a.f = -1; a.ok = 0; a.w = w; a.pad = 0;
+        PhaseA a; a.gi = -2; a.ci = 0; a.val = 0.0f; a.plan = -1; a.f = -1; a.ok = 0; a.w = w; a.pad = jb->tenant;
         if (gmin < 0) {
             const int ci = min(max(jb->cmin_idx, 0), sp.nC - 1);
             for (int gi = 0; gi < sp.nG; ++gi) {
@@ -147,7 +147,7 @@ __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick
             }
         }
         reinterpret_cast<int4 *>(pa + j)[0] = make_int4(a.gi, a.ci, __float_as_int(a.val), a.plan);
-        reinterpret_cast<int4 *>(pa + j)[1] = make_int4(a.f, a.ok, __float_as_int(a.w), 0);
+        reinterpret_cast<int4 *>(pa + j)[1] = make_int4(a.f, a.ok, __float_as_int(a.w), a.pad);      // pad carries the tenant
     }
     keys[j] = key;
 }
@@ -471,6 +471,7 @@ struct RoundArgs {
     const HotCurve *hc; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
     int32_t *glist;
     SlotA *sa_g; SlotB *sb_g; SlotC *sc_g; int32_t *sj_g; int slots_in_smem; int slot_cap;
+    const int32_t *quota; int n_tenants;      // per tenant: GPUs, cores (n_tenants = 0: no quotas)
     uint32_t *status; int32_t *steps_out;
 };
 
@@ -493,6 +494,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Shared sh;
+    __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];      // what is left of every tenant's quota: GPUs, cores
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
     const int n_cls = sp.nG * sp.nC;
@@ -532,6 +534,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     for (int i = tid; i < v.N_pad / 32; i += RT) tb_s[i] = 0u;
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
     if (tid < RW) sh.dirty[tid] = 1;
+    for (int i = tid; i < 2 * A.n_tenants; i += RT) rem_q[i] = A.quota[i];
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
         sh.ver = 0; sh.maxc_dirty = 1;
@@ -620,7 +623,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 cand.f = __shfl_sync(0xffffffffu, a1.x, i);
                 cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
                 const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
+                const int tn = __shfl_sync(0xffffffffu, a1.w, i);
                 if (gi < 0) continue;
+                if (A.n_tenants > 0) {     // privileged only while the minimum fits the tenant's remaining quota
+                    if (tn < 0 || tn >= A.n_tenants) continue;
+                    if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[ci]) continue;
+                }
                 Committed cm;
                 if (commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, true, lane, cm)) {
                     const int s = sh.n_slots;
@@ -629,6 +637,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
                         v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
                         sh.n_slots = s + 1;
+                        if (A.n_tenants > 0) { rem_q[2 * tn] -= sp.g_levels[gi]; rem_q[2 * tn + 1] -= sp.c_levels[ci]; }
                     }
                     __syncwarp();
                 }
@@ -1101,7 +1110,8 @@ size_t round_fast_scratch_need(const Space &sp, int J, int N)
 cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                               const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                               rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
-                              void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
+                              void *d_scratch, const int32_t *d_quota, int n_tenants,
+                              uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
 {
     using namespace fastround;
     const Layout L = make_layout(sp, J, N);
@@ -1133,6 +1143,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     A.sa_g = reinterpret_cast<SlotA *>(base + L.off_sa); A.sb_g = reinterpret_cast<SlotB *>(base + L.off_sb);
     A.sc_g = reinterpret_cast<SlotC *>(base + L.off_sc); A.sj_g = reinterpret_cast<int32_t *>(base + L.off_sj);
     A.slots_in_smem = L.slots_in_smem; A.slot_cap = L.slot_cap;
+    A.quota = d_quota; A.n_tenants = n_tenants;
     A.status = d_status; A.steps_out = d_steps;
     e = cudaFuncSetAttribute(greedy_round_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(SMEM_LIMIT));
     if (e != cudaSuccess) return e;

@@ -315,10 +315,12 @@ greedy_round_kernel(const __grid_constant__ Space sp, const rubick_job *__restri
                     const float *__restrict__ cv, const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
                     const uint32_t *__restrict__ feas, int N, int max_steps, rubick_assignment *__restrict__ out,
                     rubick_node *__restrict__ node_out, int32_t *__restrict__ step_log, HotA *hotA_g, HotB *hotB_g,
-                    int hot_in_smem, uint32_t *__restrict__ status, int32_t *__restrict__ steps_out)
+                    int hot_in_smem, const int32_t *__restrict__ quota, int n_tenants,
+                    uint32_t *__restrict__ status, int32_t *__restrict__ steps_out)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ RoundShared sh;
+    __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];      // what is left of every tenant's quota: GPUs, cores
 
     // shared layout: free_m [N] i64 | free_g [N] | free_c [N] | owner [N] | ff [n_small * nC] | hot arrays
     Cluster cl;
@@ -350,6 +352,7 @@ greedy_round_kernel(const __grid_constant__ Space sp, const rubick_job *__restri
         hotA[j] = a; hotB[j] = b;
     }
     if (tid == 0) { sh.steps = 0; sh.capped = 0; sh.n_empty = N; }
+    for (int i = tid; i < 2 * n_tenants; i += ROUND_THREADS) rem_q[i] = quota[i];
     __syncthreads();
 
     // ---- Phase A: guaranteed minima, in job order (warp 0) ----------------------------------------
@@ -370,9 +373,16 @@ greedy_round_kernel(const __grid_constant__ Space sp, const rubick_job *__restri
                 // the curve may reach this value with fewer GPUs than the level offers
                 const int gi = level_of_g(sp, __ldg(cg + o));
                 if (gi < 0) continue;
+                const int tn = jb->tenant;
+                if (n_tenants > 0) {       // privileged only while the minimum fits the tenant's remaining quota
+                    if (tn < 0 || tn >= n_tenants) continue;
+                    if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[cmin]) continue;
+                }
                 HotA a = hotA[j]; HotB b = hotB[j];
                 if (commit_warp(sp, cl, n_empty, cv, cp, cg, feas, j, a, b, gi, cmin, false, lane)) {
                     if (lane == 0) { hotA[j] = a; hotB[j] = b; }
+                    if (lane == 0 && n_tenants > 0) { rem_q[2 * tn] -= sp.g_levels[gi]; rem_q[2 * tn + 1] -= sp.c_levels[cmin]; }
+                    __syncwarp();
                     // recount empty nodes
                     int cnt = 0;
                     for (int nb = 0; nb < N; nb += 32) {
@@ -526,7 +536,8 @@ size_t round_scratch_need(const Space &sp, int J, int N)
 cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                          rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
-                         void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
+                         void *d_scratch, const int32_t *d_quota, int n_tenants,
+                         uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
 {
     // every step either raises one job by a level or freezes one (job, resource) pair, so a
     // round cannot take more steps than this; the clamp keeps the device loop bounded regardless
@@ -539,8 +550,8 @@ cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const
     HotA *ha = reinterpret_cast<HotA *>(d_scratch);
     HotB *hb = reinterpret_cast<HotB *>(reinterpret_cast<unsigned char *>(d_scratch) + size_t(J) * sizeof(HotA));
     greedy_round_kernel<<<1, ROUND_THREADS, smem, st>>>(sp, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out,
-                                                        d_node_out, d_step_log, ha, hb, in_smem ? 1 : 0, d_status,
-                                                        d_steps);
+                                                        d_node_out, d_step_log, ha, hb, in_smem ? 1 : 0, d_quota, n_tenants,
+                                                        d_status, d_steps);
     return cudaGetLastError();
 }
 
@@ -585,6 +596,7 @@ extern "C" int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_
         return fail(ctx, RUBICK_EINVAL, "rubick_greedy_round_noalloc: more than RUBICK_NOALLOC_MAX_JOBS jobs; the fixed state array cannot hold them");
     if (!h_cluster || h_cluster->n_nodes < 1 || h_cluster->n_nodes > RUBICK_MAX_NODES)
         return fail(ctx, RUBICK_EINVAL, "cluster: 1 .. RUBICK_MAX_NODES nodes");
+    if (h_cluster->n_tenants != 0) return fail(ctx, RUBICK_EINVAL, "rubick_greedy_round_noalloc: tenant quotas are not supported (n_tenants must be 0)");
     if (J > 0 && (!d_jobs || !d_curve_val || !d_curve_plan || !d_curve_g || !d_feas || !d_out))
         return fail(ctx, RUBICK_EINVAL, "null pointer");
     if (ctx->device < 0 || ctx->device >= NOALLOC_MAX_DEVICES) return fail(ctx, RUBICK_EINVAL, "device index out of range");
@@ -613,7 +625,7 @@ extern "C" int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_
     // from an earlier call need no clearing
     greedy_round_kernel<<<1, ROUND_THREADS, smem, ctx->stream>>>(sp, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas,
                                                                  N, max_steps, d_out, d_node_out, nullptr, ha, hb, 0,
-                                                                 ctx->d_status, ctx->d_steps);
+                                                                 nullptr, 0, ctx->d_status, ctx->d_steps);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch greedy_round (fixed state)");
 

@@ -55,7 +55,8 @@ size_t round_fast_scratch_need(const Space &sp, int J, int N);
 cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                               const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                               rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
-                              void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
+                              void *d_scratch, const int32_t *d_quota, int n_tenants,
+                              uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
 
 }  // namespace rubick
 
@@ -69,6 +70,8 @@ struct rubick_ctx {
     rubick::QuadDesc *d_quads;          // [Q]
     uint32_t *d_status;                 // one word, DS_* bits
     int32_t *d_steps;                   // one word, steps of the last round
+    int32_t *d_quota;                   // [2 * RUBICK_MAX_TENANTS] per tenant: GPUs, cores (uploaded per round)
+    std::vector<int32_t> h_quota;       // staging copy that outlives the asynchronous upload
     // scratch of the greedy round (hot per-job state when it does not fit shared memory)
     void *d_round_scratch;
     size_t round_scratch_bytes;
@@ -104,6 +107,7 @@ size_t round_scratch_need(const Space &sp, int J, int N);
 cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                          rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
-                         void *d_scratch, uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
+                         void *d_scratch, const int32_t *d_quota, int n_tenants,
+                         uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
 
 }  // namespace rubick

@@ -59,7 +59,7 @@ class Gpu:
     def np_feas(self, d_feas, J):
         return d_feas.cpu().numpy().view(np.uint32).reshape(J, self.P)
 
-    def round_on_tables(self, jobs, cv, cp, cg, feas, n_nodes, max_steps=1 << 30, want_log=True):
+    def round_on_tables(self, jobs, cv, cp, cg, feas, n_nodes, max_steps=1 << 30, want_log=True, quota=None):
         """rubick_greedy_round on host-provided tables -> dict like the oracle's."""
         t = self.torch
         J = len(jobs["P"])
@@ -72,7 +72,7 @@ class Gpu:
         d_out = self.empty(max(J, 1) * rb.ASSIGN_DTYPE.itemsize, t.uint8)
         d_node = self.empty(n_nodes * rb.NODE_DTYPE.itemsize, t.uint8)
         d_log = self.empty(max(cap, 1), t.int32) if want_log else None
-        steps, capped = self.ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, n_nodes, cap, d_out, d_node, d_log)
+        steps, capped = self.ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, n_nodes, cap, d_out, d_node, d_log, quota=quota)
         return unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE)[:J], rb.from_device(d_node, rb.NODE_DTYPE), steps, capped,
                             d_log.cpu().numpy()[:steps] if want_log else None)
 

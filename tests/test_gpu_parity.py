@@ -380,3 +380,25 @@ def test_argument_validation():
     # the context stays usable after rejected calls
     _, d_thr, d_feas = gpu.eval(cfg["jobs"])
     assert gpu.np_thr(d_thr, 4).max() > 0
+
+
+@pytest.mark.parametrize("name,J,N", [("paper-scale", None, None), ("cluster-512", 500, 32)])
+def test_greedy_round_with_tenant_quotas_is_bit_exact(name, J, N):
+    cfg = workloads.make(name, J=J, n_nodes=N)
+    Jn = len(cfg["jobs"]["P"])
+    rng = np.random.default_rng(21)
+    cfg["jobs"]["tenant"] = rng.integers(0, 5, Jn)
+    cfg["jobs"]["gmin_idx"] = np.where(rng.uniform(size=Jn) < 0.6, rng.integers(0, 4, Jn), -1)
+    cfg["jobs"]["cmin_idx"] = np.where(cfg["jobs"]["gmin_idx"] >= 0, rng.integers(0, 3, Jn), -1)
+    quota = np.stack([rng.integers(4, 40, 5), rng.integers(16, 200, 5)], axis=1)
+    gpu = Gpu(cfg)
+    plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 cfg["n_nodes"], want_log=True, quota=quota)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], quota=quota)
+    assert_rounds_equal(got, want)
+    free = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 cfg["n_nodes"])
+    assert not np.array_equal(want["status"], free["status"])                # the quotas bite
+    with pytest.raises(rb.RubickError):
+        gpu.ctx.greedy_round(None, 0, None, None, None, None, 4, 10, None, quota=np.zeros((300, 2)))

@@ -39,7 +39,8 @@ def test_struct_sizes_match_the_header():
     assert rb.PLAN_DTYPE.itemsize == 8
     assert rb.ASSIGN_DTYPE.itemsize == 40 and rb.ASSIGN_DTYPE.fields["thr"][1] == 28
     assert rb.NODE_DTYPE.itemsize == 24
-    assert C.sizeof(rb.Env) == 56 and C.sizeof(rb.Grid) == 40
+    assert C.sizeof(rb.Env) == 56 and C.sizeof(rb.Grid) == 40 and C.sizeof(rb.Cluster) == 24
+    assert rb.JOB_DTYPE.fields["tenant"][1] == 88
 
 
 @pytest.mark.parametrize("levels", [[1, 2, 3, 4, 5, 6, 7, 8], [1, 2, 4, 8, 16, 32, 64], [1 << i for i in range(9)], [4, 12, 16]])

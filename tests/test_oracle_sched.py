@@ -199,3 +199,34 @@ def test_slope_aware_split_beats_the_equal_split():
         equal = float(sum(w[j] * cv[j, 3, ci[j], -1] for j in range(2)))     # 4 GPUs each
         wins += greedy >= equal * (1 - 1e-6)
     assert wins >= 18
+
+
+def test_tenant_quotas_limit_the_privileged_jobs():
+    """Section 5.1 / 5.2: a guaranteed job is placed first only while its minimum demand fits what is
+    left of its tenant's quota; the quota is used up by the minimum demand of the jobs placed."""
+    cfg = workloads.make("paper-scale")
+    J = 64
+    jobs = cfg["jobs"]
+    jobs["gmin_idx"] = np.full(J, 1)                 # every job is guaranteed 2 GPUs ...
+    jobs["cmin_idx"] = np.full(J, 0)                 # ... and 4 cores
+    jobs["tenant"] = np.arange(J) % 2
+    tb = tables(cfg)
+    plans, feas, cv, cp, cg = tb
+    kw = dict(want_log=True)
+    free = run_round(cfg, tb, **kw)
+    quota = np.array([[6, 12], [64, 4]])             # tenant 0: 6 GPUs; tenant 1: cores for one job only
+    lim = oracle.schedule_round(jobs, cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                cfg["n_nodes"], quota=quota, **kw)
+    check_invariants(cfg, tb, lim)
+    placed = lim["status"] == 1
+    t = jobs["tenant"]
+    # Phase A placed at most what the quotas allow, in job order; nobody beyond the quota runs at all
+    assert placed[t == 0].sum() <= 3 and placed[t == 1].sum() <= 1
+    first0 = np.nonzero((t == 0) & (cv[:, 1, 0, -1] > 0))[0][:3]
+    assert placed[first0].all()
+    assert (lim["status"][~placed] == 2).all() and placed.sum() < (free["status"] == 1).sum()
+    # without quotas the same call places more jobs; a generous quota changes nothing
+    big = oracle.schedule_round(jobs, cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                cfg["n_nodes"], quota=np.array([[10**6, 10**6]] * 2), **kw)
+    for k in ("g", "c", "plan", "status", "first_node"):
+        assert np.array_equal(big[k], free[k])
