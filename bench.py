@@ -201,8 +201,11 @@ def main():
 
     import torch
     from paper_2408_08586_b200 import binding as rb
+    from paper_2408_08586_b200 import build as rbuild
 
     rank = int(os.environ.get("RANK", "0"))
+    if not os.path.exists(rb.LIB_PATH) and int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        rbuild.build()                      # the library is built in-tree; compile it if this checkout has not been built yet
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
@@ -300,6 +303,26 @@ def main():
                "d2h_bytes_per_step": int(J * rb.ASSIGN_DTYPE.itemsize + N * rb.NODE_DTYPE.itemsize),
                "call": "rubick_schedule_round_host: pinned job records in, assignments and node states out"}
 
+    # minimum demand of guaranteed jobs on the same tables (first widening row; rank 0 only)
+    minres_ms = None
+    if rank == 0:
+        _, goff = rb.enumerate_plans(cfg["g_levels"])
+        rq = workloads.draw_requests(cfg["seed"], J, [int(g) for g in cfg["g_levels"]], C, M, 0.5)
+        size = goff[rq["g_idx"] + 1] - goff[rq["g_idx"]]
+        rec = np.zeros(J, dtype=rb.REQUEST_DTYPE)
+        rec["g_idx"], rec["c_idx"], rec["m_idx"] = rq["g_idx"], rq["c_idx"], rq["m_idx"]
+        rec["plan"] = np.where(rq["plan_rank"] >= 0, goff[rq["g_idx"]] + np.floor(np.maximum(rq["plan_rank"], 0) * size), -1)
+        d_req = rb.to_device(rec, dev)
+        d_gm, d_cm = torch.empty(J, dtype=torch.int32, device=dev), torch.empty(J, dtype=torch.int32, device=dev)
+        d_bl = torch.empty(J, dtype=torch.float32, device=dev)
+        ctx.min_resources(d_thr, d_feas, d_cv, J, d_req, d_gm, d_cm, d_bl)
+        a = ev()
+        for _ in range(10):
+            ctx.min_resources(d_thr, d_feas, d_cv, J, d_req, d_gm, d_cm, d_bl)
+        b = ev()
+        torch.cuda.synchronize()
+        minres_ms = a.elapsed_time(b) / 10
+
     # event-driven run: every arrival / completion re-plans all active jobs (rank 0 only)
     events = None
     if args.events > 0 and rank == 0:
@@ -363,6 +386,7 @@ def main():
         "logical_candidates_per_sec": value * M,
         "best_plan_roofline": {"bound": "hbm", "achieved": best_gbs, "peak": peak, "unit": "GB/s", "frac": best_gbs / peak},
         "events": events,
+        "min_resources_ms": minres_ms,
         "round": {"steps": int(round_steps[0]), "latency_ms": float(stage_ms[3]),
                   "us_per_step": float(1e3 * stage_ms[3] / max(1, round_steps[0]))},
     }
