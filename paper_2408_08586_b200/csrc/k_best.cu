@@ -134,7 +134,11 @@ best_plan_kernel(const __grid_constant__ Space sp, const float *__restrict__ thr
             if (k == 1 && !has_b) break;
             const int ci = ca + k;
             u64 running = 0ull;
-            for (int g = 0; g < sp.nG; ++g) {
+            int running_g = 0;
+            // outputs of (j, g, ci, lane) advance by nC * nM entries per GPU level
+            size_t o = (size_t(j) * sp.nG * sp.nC + ci) * sp.nM + lane;
+            const size_t o_step = size_t(sp.nC) * sp.nM;
+            for (int g = 0; g < sp.nG; ++g, o += o_step) {
                 const u64 mine = bucket[k * row_stride + g * 32 + lane];
                 // best among plans whose first level is <= lane: maximum over the occupied buckets at or below
                 unsigned occ = __ballot_sync(0xffffffffu, mine != 0ull);
@@ -142,16 +146,18 @@ best_plan_kernel(const __grid_constant__ Space sp, const float *__restrict__ thr
                 while (occ) {
                     const int f = __ffs(occ) - 1;
                     occ &= occ - 1;
-                    const u64 o = __shfl_sync(0xffffffffu, mine, f);
-                    if (lane >= f && o > best) best = o;
+                    const u64 ob = __shfl_sync(0xffffffffu, mine, f);
+                    if (lane >= f && ob > best) best = ob;
                 }
-                if (!raw) { running = best > running ? best : running; best = running; }
+                int best_gv = best ? sp.g_levels[g] : 0;       // the level's own plans use exactly its GPU count
+                if (!raw) {
+                    if (best > running) { running = best; running_g = best_gv; }
+                    best = running; best_gv = running_g;
+                }
                 if (lane < sp.nM) {
-                    const size_t o = ((size_t(j) * sp.nG + g) * sp.nC + ci) * sp.nM + lane;
-                    const int plan = best ? int(0xffffffffu - uint32_t(best)) : -1;
                     best_val[o] = best ? __uint_as_float(uint32_t(best >> 32)) : 0.0f;
-                    best_plan[o] = plan;
-                    best_g[o] = plan >= 0 ? sp.g_levels[pslot[plan] >> 5] : 0;
+                    best_plan[o] = best ? int(0xffffffffu - uint32_t(best)) : -1;
+                    best_g[o] = best_gv;
                 }
             }
         }
