@@ -737,7 +737,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             const uint32_t key = lane < RW ? sh.red_key[lane] : 0u, my_pay = lane < RW ? sh.red_pay[lane] : 0u;
             const int my_j = lane < RW ? sh.red_j[lane] : 0x7fffffff;
             uint32_t best = key, pay = my_pay; int best_j = my_j;
-            warp_select(best, best_j, pay);
+            const int top_lane = warp_select(best, best_j, pay);
             bool go = best != 0u;
             const int steps0 = sh.steps, room = A.max_steps - steps0;
             if (go && room <= 0) { if (lane == 0) sh.capped = 1; go = false; }
@@ -810,7 +810,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     }
                 }
             }
-            if (go && n_acc == 0) {
+            // the batch can only start with the overall best candidate: look at it first (shared memory only)
+            bool top_stays = false;
+            if (go && n_acc == 0 && !(pay & 0x80000000u)) {
+                bool st = false;
+                if (lane == top_lane) {
+                    const SlotA a = v.sa[int(my_pay)];
+                    const int type_gpu = int(key >> 31);
+                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+                    const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+                    const int w_old = v.gc[a.node];
+                    const int k = g > sp.Gn ? g >> sp.log2Gn : 1;
+                    st = g > sp.Gn ? (!type_gpu && (c2 + k - 1) / k <= sp.Cn)
+                                   : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
+                }
+                top_stays = __any_sync(FULL, st);
+            }
+            if (go && n_acc == 0 && top_stays) {
                 const uint32_t M = __reduce_max_sync(FULL, lane < RW ? sh.red_key2[lane] : 0u);
                 bool elig = false, s_ok = false, s_maxc = false, s_multi = false;
                 int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0;
