@@ -402,3 +402,31 @@ def test_greedy_round_with_tenant_quotas_is_bit_exact(name, J, N):
     assert not np.array_equal(want["status"], free["status"])                # the quotas bite
     with pytest.raises(rb.RubickError):
         gpu.ctx.greedy_round(None, 0, None, None, None, None, 4, 10, None, quota=np.zeros((300, 2)))
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_greedy_round_on_random_instances_is_bit_exact(seed):
+    """Random cluster shapes, job mixes and guarantees: the batched device round must replay the
+    oracle's one-step-at-a-time round exactly, step log included."""
+    rng = np.random.default_rng(1000 + seed)
+    name = ["paper-scale", "cluster-512", "events"][seed % 3]
+    J = int(rng.integers(40, 420))
+    N = int(rng.integers(3, 40))
+    cfg = workloads.make(name, J=J, n_nodes=N)
+    gn = int(rng.choice([4, 8]))
+    cfg["env"] = env(gpus_per_node=gn, cpus_per_node=int(rng.choice([32, 64, 96])),
+                     mem_per_node_bytes=int(rng.choice([128, 256, 512, 1024])) * GIB)
+    if gn == 4:
+        cfg["g_levels"] = np.array([g for g in cfg["g_levels"] if g <= 4 or g % 4 == 0])
+    share = float(rng.choice([0.0, 0.2, 0.6]))
+    guar = rng.uniform(size=J) < share
+    cfg["jobs"]["gmin_idx"] = np.where(guar, rng.integers(0, 4, J), -1)
+    cfg["jobs"]["cmin_idx"] = np.where(guar, rng.integers(0, 4, J), -1)
+    if seed % 4 == 0:
+        cfg["jobs"]["w"] = np.ones(J)                     # raw aggregated throughput instead of normalised
+    gpu = Gpu(cfg)
+    plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 N, want_log=True)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, N)
+    assert_rounds_equal(got, want)
