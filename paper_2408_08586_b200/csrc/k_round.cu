@@ -613,8 +613,18 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 a0 = reinterpret_cast<const int4 *>(A.pa + jl)[0];
                 a1 = reinterpret_cast<const int4 *>(A.pa + jl)[1];
             }
-            const int cnt = min(32, ng - base);
-            for (int i = 0; i < cnt; ++i) {
+            // Free resources only shrink during this phase, so a job that cannot be placed now never can:
+            // every lane tests its own job against the present tables and only the others take a turn.
+            bool may = false;
+            if (idx < ng && a0.x >= 0) {
+                const int g2 = v.gl[a0.x], c2 = v.clv[a0.y];
+                if (g2 <= sp.Gn) may = v.maxc[a0.x] >= c2;
+                else { const int k2 = g2 >> sp.log2Gn; may = (c2 + k2 - 1) / k2 <= sp.Cn && sh.n_empty >= k2; }
+            }
+            unsigned todo = __ballot_sync(0xffffffffu, may);
+            while (todo) {
+                const int i = __ffs(todo) - 1;
+                todo &= todo - 1;
                 const int j = __shfl_sync(0xffffffffu, jl, i);
                 const int gi = __shfl_sync(0xffffffffu, a0.x, i), ci = __shfl_sync(0xffffffffu, a0.y, i);
                 HotCurve cand;
