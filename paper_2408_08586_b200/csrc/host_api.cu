@@ -71,7 +71,7 @@ int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *c
     ctx->d_jobs_stage = nullptr; ctx->cap_jobs = 0;
     ctx->d_out_stage = nullptr; ctx->cap_out = 0;
     ctx->d_node_stage = nullptr; ctx->cap_node = 0;
-    ctx->tile_jobs = 256;
+    ctx->tile_jobs = 2048;            // 0.5 GB table tile at 2,640 plans x 24 core levels
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return RUBICK_ECUDA; }
     ctx->num_sms = prop.multiProcessorCount;
