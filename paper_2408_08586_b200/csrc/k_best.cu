@@ -5,7 +5,7 @@
 // One CTA owns one job.  Its feasibility words are turned once into 16-bit "slots" in shared memory:
 // slot = GPU level * 32 + first feasible memory level (words are thresholds in the level index, so
 // the first set bit says it all), 0xffff for a plan that is feasible nowhere.  Each warp then takes
-// two CPU levels at a time: lanes stream both rows of the throughput table with 16-byte loads (four
+// BEST_ROWS CPU levels at a time: lanes stream both rows of the throughput table with 16-byte loads (four
 // plans = one quad per load) and keep, per row and per plan parity (offload plans alternate with
 // the others and usually need another memory level), a running (value, index) maximum for the slot
 // they are currently seeing; a strict "greater" keeps the lowest index because a lane meets its
@@ -23,6 +23,7 @@ namespace rubick {
 
 constexpr int BEST_WARPS = 12;         // at most; fewer when the buckets of many GPU levels would not fit
 constexpr int BEST_ROWS = 2;          // CPU levels a warp processes together
+constexpr int BEST_UNROLL = 2;        // quads per lane in flight per row
 
 typedef unsigned long long u64;
 
@@ -45,12 +46,13 @@ __device__ __forceinline__ void run_flush(Run &r, u64 *bucket, int row_stride)
     }
 }
 
-__device__ __forceinline__ void run_add(Run &r, u64 *bucket, int row_stride, uint32_t slot, int idx, float va, float vb)
+__device__ __forceinline__ void run_add(Run &r, u64 *bucket, int row_stride, uint32_t slot, int idx, const float (&val)[BEST_ROWS])
 {
     if (slot == 0xffffu) return;
     if (slot != r.slot) { if (r.slot != 0xffffu) run_flush(r, bucket, row_stride); r.slot = slot; }
-    if (va > r.v[0]) { r.v[0] = va; r.i[0] = idx; }
-    if (vb > r.v[1]) { r.v[1] = vb; r.i[1] = idx; }
+#pragma unroll
+    for (int k = 0; k < BEST_ROWS; ++k)
+        if (val[k] > r.v[k]) { r.v[k] = val[k]; r.i[k] = idx; }
 }
 
 __global__ void __launch_bounds__(BEST_WARPS * 32)
@@ -92,37 +94,40 @@ best_plan_kernel(const __grid_constant__ Space sp, const float *__restrict__ thr
 
     for (int pr = warp; pr < n_pairs; pr += n_warps) {
         const int ca = pr * BEST_ROWS;
-        const bool has_b = ca + 1 < sp.nC;
-        const int cb = has_b ? ca + 1 : ca;
+        const int n_rows = min(BEST_ROWS, sp.nC - ca);          // the last group may be short
         for (int i = lane; i < BEST_ROWS * row_stride; i += 32) bucket[i] = 0ull;
         __syncwarp();
 
-        const float4 *row_a = reinterpret_cast<const float4 *>(thr + (size_t(j) * sp.nC + ca) * sp.P);
-        const float4 *row_b = reinterpret_cast<const float4 *>(thr + (size_t(j) * sp.nC + cb) * sp.P);
+        const float4 *row[BEST_ROWS];
+#pragma unroll
+        for (int k = 0; k < BEST_ROWS; ++k)
+            row[k] = reinterpret_cast<const float4 *>(thr + (size_t(j) * sp.nC + ca + (k < n_rows ? k : 0)) * sp.P);
         Run even, odd;          // plans 4q, 4q+2 (no offload) / 4q+1, 4q+3 (offload)
         even.slot = odd.slot = 0xffffu;
 #pragma unroll
         for (int k = 0; k < BEST_ROWS; ++k) { even.v[k] = odd.v[k] = 0.0f; even.i[k] = odd.i[k] = -1; }
 
-        constexpr int UNROLL = 2;
-        for (int q0 = lane; q0 < sp.Q; q0 += 32 * UNROLL) {
-            float4 va[UNROLL], vb[UNROLL];
+        for (int q0 = lane; q0 < sp.Q; q0 += 32 * BEST_UNROLL) {
+            float4 val[BEST_UNROLL][BEST_ROWS];
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
+            for (int u = 0; u < BEST_UNROLL; ++u) {
                 const int q = q0 + 32 * u;
-                const bool in = q < sp.Q;
-                va[u] = in ? __ldcs(row_a + q) : make_float4(0.f, 0.f, 0.f, 0.f);
-                vb[u] = in ? __ldcs(row_b + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int k = 0; k < BEST_ROWS; ++k)
+                    val[u][k] = q < sp.Q ? __ldcs(row[k] + q) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
+            for (int u = 0; u < BEST_UNROLL; ++u) {
                 const int q = q0 + 32 * u;
                 if (q >= sp.Q) break;
                 const uint2 s4 = pslot4[q];
-                run_add(even, bucket, row_stride, s4.x & 0xffffu, 4 * q + 0, va[u].x, vb[u].x);
-                run_add(odd, bucket, row_stride, s4.x >> 16, 4 * q + 1, va[u].y, vb[u].y);
-                run_add(even, bucket, row_stride, s4.y & 0xffffu, 4 * q + 2, va[u].z, vb[u].z);
-                run_add(odd, bucket, row_stride, s4.y >> 16, 4 * q + 3, va[u].w, vb[u].w);
+                float x[BEST_ROWS], y[BEST_ROWS], z[BEST_ROWS], w[BEST_ROWS];
+#pragma unroll
+                for (int k = 0; k < BEST_ROWS; ++k) { x[k] = val[u][k].x; y[k] = val[u][k].y; z[k] = val[u][k].z; w[k] = val[u][k].w; }
+                run_add(even, bucket, row_stride, s4.x & 0xffffu, 4 * q + 0, x);
+                run_add(odd, bucket, row_stride, s4.x >> 16, 4 * q + 1, y);
+                run_add(even, bucket, row_stride, s4.y & 0xffffu, 4 * q + 2, z);
+                run_add(odd, bucket, row_stride, s4.y >> 16, 4 * q + 3, w);
             }
         }
         if (even.slot != 0xffffu) run_flush(even, bucket, row_stride);
@@ -131,7 +136,7 @@ best_plan_kernel(const __grid_constant__ Space sp, const float *__restrict__ thr
 
 #pragma unroll
         for (int k = 0; k < BEST_ROWS; ++k) {
-            if (k == 1 && !has_b) break;
+            if (k >= n_rows) break;
             const int ci = ca + k;
             u64 running = 0ull;
             int running_g = 0;

@@ -1,6 +1,6 @@
 """Parity of the CUDA path with the oracle, element by element, through the C ABI.
 
-Tolerances (stated by the task's target and derived in the design notes):
+Tolerances:
   predicted throughput   1e-5 relative (single-precision kernel vs double-precision oracle)
   feasibility words      bit exact
   plan / allocation      bit exact when both sides see the same table; through the whole
