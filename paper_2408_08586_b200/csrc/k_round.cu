@@ -342,6 +342,8 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
                 ch = ch || (on == mx && nn < on) || nn > mx;
             }
         }
+        // while an empty node remains every entry equals the node's core count: nothing to recompute
+        if (n_empty + d_empty > 0) ch = lane < sp.n_small && v.maxc[lane] != sp.Cn;
         maxc_dirty = __any_sync(0xffffffffu, ch);
     } else {
         const int cs2 = (c2 + k2 - 1) / k2;
@@ -353,8 +355,15 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
             if (k == 1) {
                 if (lane == 0) { v.gc[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; }
             } else {
-                for (int n = lane; n < v.N; n += 32)
-                    if (v.owner[n] == j) { v.gc[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
+                // the k nodes of a job usually are node .. node + k - 1 (taken together from an empty stretch)
+                const int nn = node + lane;
+                const bool mine = lane < k && nn < v.N && v.owner[nn] == j;
+                if (__popc(__ballot_sync(0xffffffffu, mine)) == k) {
+                    if (mine) { v.gc[nn] += cs1 - cs2; v.free_m[nn] += ms1 - ms2; }
+                } else {
+                    for (int n = lane; n < v.N; n += 32)
+                        if (v.owner[n] == j) { v.gc[n] += cs1 - cs2; v.free_m[n] += ms1 - ms2; }
+                }
             }
             first = node;
         } else if (alloc) {
@@ -840,7 +849,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             if (go && n_acc == 0 && top_stays) {
                 const uint32_t M = __reduce_max_sync(FULL, lane < RW ? sh.red_key2[lane] : 0u);
                 bool elig = false, s_ok = false, s_maxc = false, s_multi = false;
-                int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0;
+                int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0, s_k = 1;
                 int64_t s_dm = 0;
                 uint32_t s_bound = 0u;
                 SlotA na; SlotB nb; SlotC nq;
@@ -873,7 +882,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         int lo = 0, hi = sp.nM;                 // number of levels <= avail (levels ascend)
                         while (lo < hi) { const int mid = (lo + hi) >> 1; if (v.ml[mid] <= avail) lo = mid + 1; else hi = mid; }
                         const int mi = lo - 1;
-                        s_multi = multi;
+                        s_multi = multi; s_k = k;
                         bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                         s_slot = s; s_node = a.node; s_type = type_gpu;
                         if (mi < 0) { elig = true; s_ok = false; }
@@ -913,7 +922,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             }
                             // can maxc[] change?  (the node only loses GPUs / cores)
                             const int w_new = w_old - s_dgc;
-                            for (int i = 0; i < sp.n_small && !multi; ++i) {
+                            bool saturated = sh.n_empty > 0;
+                            for (int i = 0; i < sp.n_small; ++i) saturated = saturated && v.maxc[i] == sp.Cn;
+                            for (int i = 0; i < sp.n_small && !multi && !saturated; ++i) {
                                 const int glv = v.gl[i], mx = v.maxc[i];
                                 const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
                                 s_maxc = s_maxc || (ot == mx && nt < ot);
@@ -975,8 +986,15 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         mm &= mm - 1;
                         const int oj = __shfl_sync(FULL, my_j, src), dc = __shfl_sync(FULL, s_dgc, src);
                         const long long dm = __shfl_sync(FULL, (long long)s_dm, src);
-                        for (int n = lane; n < N; n += 32)
-                            if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
+                        const int on = __shfl_sync(FULL, s_node, src), ok_ = __shfl_sync(FULL, s_k, src);
+                        const int nn = on + lane;
+                        const bool mine = lane < ok_ && nn < N && v.owner[nn] == oj;
+                        if (__popc(__ballot_sync(FULL, mine)) == ok_) {           // its nodes are on .. on + k - 1
+                            if (mine) { v.gc[nn] -= dc; v.free_m[nn] -= dm; }
+                        } else {
+                            for (int n = lane; n < N; n += 32)
+                                if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
+                        }
                     }
                     const bool md = __any_sync(FULL, ((acc >> lane) & 1u) && s_ok && s_maxc);
                     if (lane == 0) { sh.steps = steps0 + n_acc; sh.maxc_dirty = md ? 1 : 0; }
