@@ -294,7 +294,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
 
     // highest memory level whose per-node share fits: ceil(m / k2) <= avail  <=>  m <= avail * k2
     const int64_t avail = k2 > 1 ? sp.Mn : v.free_m[target] + ((stay && alloc) ? m_cur : 0);
-    const bool fits = lane < sp.nM && sp.m_levels[lane < sp.nM ? lane : 0] <= avail * k2;
+    const bool fits = lane < sp.nM && v.ml[lane < sp.nM ? lane : 0] <= avail * k2;
     const unsigned fb = __ballot_sync(0xffffffffu, fits);
     if (!fb) return false;
     const int mi = 31 - __clz(fb);
@@ -334,7 +334,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         // can maxc[] have changed?  lane i answers for GPU level i
         bool ch = false;
         if (lane < sp.n_small) {
-            const int gl = sp.g_levels[lane], mx = v.maxc[lane];
+            const int gl = v.gl[lane], mx = v.maxc[lane];
             const int ot = fg_of(w_old_t) >= gl ? fc_of(w_old_t) : -1, nt = fg_of(w_new_t) >= gl ? fc_of(w_new_t) : -1;
             ch = (ot == mx && nt < ot) || nt > mx;
             if (moved) {
@@ -791,7 +791,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if ((c2 + k2 - 1) / k2 <= sp.Cn && sh.n_empty >= k2) avail = sp.Mn;
                 }
                 if (avail >= 0) {
-                    const unsigned fb = __ballot_sync(FULL, lane < sp.nM && sp.m_levels[lane < sp.nM ? lane : 0] <= avail * k2);
+                    const unsigned fb = __ballot_sync(FULL, lane < sp.nM && v.ml[lane < sp.nM ? lane : 0] <= avail * k2);
                     const int mi = fb ? 31 - __clz(fb) : -1;
                     const int ptr = v.cls_ptr[t], end = v.cls_end[t];
                     const int idx = ptr + lane;
