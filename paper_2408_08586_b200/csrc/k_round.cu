@@ -2,7 +2,7 @@
 //
 // Same decisions, step for step, as the plain round in k_sched.cu (largest placeable positive
 // GPU gain first, CPU gain when no GPU increment is left, lowest job index on ties, commit with
-// the best plan and its host memory), organised so that one step costs about a microsecond:
+// the best plan and its host memory), organised so that one step costs about half a microsecond:
 //
 //   prepare  (grid)   per (job, GPU level, CPU level): the curve entry at the top host-memory level
 //                     together with the first feasible memory level of its plan, 16 bytes.  A commit
@@ -14,14 +14,26 @@
 //                     Guaranteed jobs get their Phase-A target resolved here too.
 //   sort     (1 CTA)  bitonic sort of the keys: inside a class (same target levels = same placement
 //                     test) only the first unconsumed job can ever be selected.
-//   round    (1 CTA)  persistent loop.  Shared memory holds the node state, an incrementally
-//                     maintained table "most free cores among nodes with >= g free GPUs" (a job of g GPUs
-//                     and c cores fits some node exactly when that entry is >= c), the head of every class and
-//                     one 36-byte slot per RUNNING job (scan state + placement needs).  A step scans class heads + running slots
-//                     (not all jobs), selects (type | gain, lowest job) across the block with warp reduce instructions, and
-//                     warp 0 commits: placement (own node, else first fit by a warp scan), memory level
-//                     by ballot, node bookkeeping, table rebuild, new gains from one warp-wide load of
-//                     the job's curve column issued together with the target's entry.
+//   round    (1 CTA)  persistent loop.  Shared memory holds one word per node (free GPUs << 16 | free
+//                     cores), free memory and whole-node owners, the table "most free cores among nodes
+//                     with >= g free GPUs" (a job of g GPUs and c cores fits some node exactly when that
+//                     entry is >= c), the head of every class, one 36-byte slot per RUNNING job (scan state
+//                     + what its two candidates need to be placeable) and a bitmap of the nodes the last
+//                     iteration changed.  Every warp caches the best candidate and the runner-up key of
+//                     its slots (the last warp: of the class heads) and looks again only when one of its
+//                     slots, a node under them, that table or the number of empty nodes changed.  Warp 0
+//                     picks (type | gain, lowest job) across the warps with warp reduce instructions and
+//                     commits, in the exact order of the one-step-at-a-time rule, as many steps as it can
+//                     prove independent of each other:
+//                       - a run of class heads that are rejected (a rejection changes nothing but the head
+//                         of its class; lane i settles the i-th entry of the class's sorted list);
+//                       - a batch of increments that stay on their own nodes (lane w works out the commit
+//                         of warp w's candidate; candidates are taken in descending order while each is
+//                         larger than every runner-up, every best not yet taken and every new candidate of
+//                         the jobs taken before it, and sits on another node);
+//                       - otherwise one general commit (migration, growth onto whole nodes, a class head
+//                         that succeeds): placement, memory level by ballot, node bookkeeping, new gains
+//                         from one warp-wide load of the job's curve column.
 //
 // All gain arithmetic uses __fmul_rn / __fsub_rn / __fdiv_rn (one rounding per operation, never
 // fused) so that decisions are reproducible bit for bit.  Every loop is bounded (steps by
@@ -52,12 +64,8 @@ __device__ __forceinline__ int key_job(u64 k) { return int(KEY_JOB_MASK - (k & K
 __device__ __forceinline__ uint32_t key_gain_bits(u64 k) { return uint32_t(k >> KEY_JOB_BITS); }
 __device__ __forceinline__ int key_class(u64 k) { return int(k >> 53); }
 
-// selection key of a step: [63] 1 = GPU increment | [62:31] gain bits | [30:0] ~job
-__device__ __forceinline__ u64 sel_key(int type_gpu, uint32_t gain_bits, int j)
-{
-    return (u64(type_gpu) << 63) | (u64(gain_bits) << 31) | u64(0x7fffffffu - uint32_t(j));
-}
-__device__ __forceinline__ int sel_job(u64 k) { return int(0x7fffffffu - uint32_t(k & 0x7fffffffu)); }
+// selection key of a step (32 bits): [31] 1 = GPU increment | [30:0] bits of the positive gain;
+// equal keys go to the lowest job index
 
 // slot.packed: [5:0] g level | [12:6] c level | [18:13] target g level + 1 | [20] GPU frozen | [21] CPU frozen
 __device__ __forceinline__ uint32_t pack(int gi, int ci, int next_gi, bool fz_g, bool fz_c)
