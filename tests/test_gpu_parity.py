@@ -430,3 +430,34 @@ def test_greedy_round_on_random_instances_is_bit_exact(seed):
                                  N, want_log=True)
     got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, N)
     assert_rounds_equal(got, want)
+
+
+def test_odd_grid_shapes_through_every_kernel():
+    """Five core levels (an odd count: the arg-max handles them in pairs), seven memory levels, five GPU
+    levels of which one is not a power of two, 4-GPU nodes: table, mask, curves, gains and round."""
+    cfg = workloads.make("paper-scale", J=37, n_nodes=9)
+    cfg["g_levels"] = np.array([1, 2, 4, 8, 12, 16])
+    cfg["c_levels"] = np.array([2, 6, 10, 30, 50])
+    cfg["m_levels"] = np.array([16, 48, 100, 200, 333, 512, 700]) * GIB
+    cfg["env"] = env(gpus_per_node=4, cpus_per_node=50, mem_per_node_bytes=700 * GIB)
+    cfg["jobs"]["gmin_idx"] = np.where(cfg["jobs"]["gmin_idx"] >= 0, 1, -1)
+    cfg["jobs"]["cmin_idx"] = np.where(cfg["jobs"]["gmin_idx"] >= 0, 2, -1)
+    gpu = Gpu(cfg)
+    J = 37
+    _, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
+    assert len(plans) == 16 * (1 + 3 + 6 + 10 + 15) and np.array_equal(gpu.np_feas(d_feas, J), feas)
+    check_thr(gpu.np_thr(d_thr, J), thr)
+    t = gpu.torch
+    d_thr32 = t.from_numpy(thr.astype(np.float32).reshape(-1)).cuda()
+    for raw in (False, True):
+        ov, op, og = oracle.best_plan(thr.astype(np.float32), feas, plans, cfg["g_levels"], gpu.nM, prefix=not raw, nthreads=4)
+        bv, bp, bg = gpu.best(d_thr32, d_feas, J, flags=rb.BEST_RAW if raw else 0)
+        sh = gpu.shape4(J)
+        assert np.array_equal(bv.cpu().numpy().reshape(sh), ov.astype(np.float32))
+        assert np.array_equal(bp.cpu().numpy().reshape(sh), op) and np.array_equal(bg.cpu().numpy().reshape(sh), og)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 9, want_log=True)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 9)
+    assert_rounds_equal(got, want)
+    assert want["steps"] > 5 and (want["n_nodes"] > 1).any()
