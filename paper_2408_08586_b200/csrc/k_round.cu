@@ -203,6 +203,9 @@ enum : uint8_t { K_SINGLE = 0, K_MULTI_WHOLE = 1, K_MULTI_PART = 2, K_NONE = 3 }
 
 constexpr int SCAN_WARPS = RW - 1;          // all warps but the last scan running jobs, the last one the class heads
 constexpr int SCAN_T = SCAN_WARPS * 32;
+constexpr int N_GROUPS = 2 * SCAN_WARPS + 1;   // candidates are cached per half warp (16 slots a pass) + one group for the class heads
+constexpr int CLS_G = N_GROUPS - 1;
+static_assert(N_GROUPS <= 32, "warp 0 holds one group per lane");
 
 // node n: gc[n] = free GPUs << 16 | free cores (padding entries are 0: they never fit anything)
 __device__ __forceinline__ int fg_of(int w) { return w >> 16; }
@@ -222,9 +225,9 @@ struct Views {
 };
 
 struct Shared {
-    uint32_t red_key[RW]; int32_t red_j[RW]; uint32_t red_pay[RW];
-    uint32_t red_key2[RW];        // second-best key of the warp (keys only: ties are resolved conservatively)
-    int dirty[RW];                // warp must rescan: one of its slots (or a class head) changed
+    uint32_t red_key[32]; int32_t red_j[32]; uint32_t red_pay[32];
+    uint32_t red_key2[32];        // second-best key of the group (keys only: ties are resolved conservatively)
+    int dirty[32];                // group must rescan: one of its slots (or a class head) changed
     int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
@@ -495,13 +498,13 @@ struct RoundArgs {
 constexpr int SLOT_BYTES = int(sizeof(SlotA) + sizeof(SlotC)) + 4;     // per running job in shared memory
 
 // warp-wide selection: largest key, lowest job among equal keys (key 0 = nothing)
-__device__ __forceinline__ int warp_select(uint32_t &key, int &j, uint32_t &pay)
+__device__ __forceinline__ int warp_select(uint32_t &key, int &j, uint32_t &pay, unsigned mask = 0xffffffffu)
 {
-    const uint32_t m = __reduce_max_sync(0xffffffffu, key);
-    const int jm = __reduce_min_sync(0xffffffffu, (key == m && m) ? j : 0x7fffffff);
-    const unsigned b = __ballot_sync(0xffffffffu, key == m && j == jm);
-    const int src = b ? __ffs(b) - 1 : 0;
-    pay = __shfl_sync(0xffffffffu, pay, src);
+    const uint32_t m = __reduce_max_sync(mask, key);
+    const int jm = __reduce_min_sync(mask, (key == m && m) ? j : 0x7fffffff);
+    const unsigned b = __ballot_sync(mask, key == m && j == jm);
+    const int src = b ? __ffs(b) - 1 : __ffs(mask) - 1;
+    pay = __shfl_sync(mask, pay, src);
     key = m; j = jm;
     return src;                                   // the lane that held the winner
 }
@@ -550,7 +553,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     if (tid < sp.nM) ml_s[tid] = sp.m_levels[tid];
     for (int i = tid; i < v.N_pad / 32; i += RT) tb_s[i] = 0u;
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
-    if (tid < RW) sh.dirty[tid] = 1;
+    if (tid < 32) sh.dirty[tid] = 1;
     for (int i = tid; i < 2 * A.n_tenants; i += RT) rem_q[i] = A.quota[i];
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
@@ -697,12 +700,14 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             __syncthreads();
         }
         const int n_empty = sh.n_empty, n_slots = sh.n_slots, ver = sh.ver;
-        bool rescan = ver != my_ver || sh.dirty[warp] != 0;
+        const unsigned hm = 0xffffu << (lane & 16);                   // my half of the warp
+        const int grp = warp < SCAN_WARPS ? 2 * warp + (lane >> 4) : CLS_G;
+        bool rescan = ver != my_ver || sh.dirty[grp] != 0;
         if (warp < SCAN_WARPS) {
             if (!rescan) {
                 bool hit = false;
                 for (int s = tid; s < n_slots; s += SCAN_T) { const int nd = v.sa[s].node; hit = hit || ((v.tb[nd >> 5] >> (nd & 31)) & 1u); }
-                rescan = __any_sync(0xffffffffu, hit);
+                rescan = __any_sync(hm, hit);
             }
             if (rescan) {
                 uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
@@ -728,10 +733,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if (ok_g && kc > second) second = kc;
                 }
                 const uint32_t mine = best;
-                const int src = warp_select(best, best_j, pay);
-                c_key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
+                const int src = warp_select(best, best_j, pay, hm);
+                c_key2 = __reduce_max_sync(hm, lane == src ? second : mine);
                 c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
-                if (lane == 0) sh.dirty[warp] = 0;
+                if ((lane & 15) == 0) sh.dirty[grp] = 0;
             }
         } else if (rescan) {
             uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
@@ -755,14 +760,16 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             const int src = warp_select(best, best_j, pay);
             c_key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
             c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
-            if (lane == 0) sh.dirty[warp] = 0;
+            if (lane == 0) sh.dirty[CLS_G] = 0;
         }
-        if (lane == 0) { sh.red_key[warp] = c_key; sh.red_j[warp] = c_j; sh.red_pay[warp] = c_pay; sh.red_key2[warp] = c_key2; }
+        if ((lane & 15) == 0 && (warp < SCAN_WARPS || lane == 0)) {
+            sh.red_key[grp] = c_key; sh.red_j[grp] = c_j; sh.red_pay[grp] = c_pay; sh.red_key2[grp] = c_key2;
+        }
         __syncthreads();
         if (warp == 0) {
             const unsigned FULL = 0xffffffffu;
-            const uint32_t key = lane < RW ? sh.red_key[lane] : 0u, my_pay = lane < RW ? sh.red_pay[lane] : 0u;
-            const int my_j = lane < RW ? sh.red_j[lane] : 0x7fffffff;
+            const uint32_t key = lane < N_GROUPS ? sh.red_key[lane] : 0u, my_pay = lane < N_GROUPS ? sh.red_pay[lane] : 0u;
+            const int my_j = lane < N_GROUPS ? sh.red_j[lane] : 0x7fffffff;
             uint32_t best = key, pay = my_pay; int best_j = my_j;
             const int top_lane = warp_select(best, best_j, pay);
             bool go = best != 0u;
@@ -789,7 +796,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 const int t = int(pay & 0x7fffffffu);
                 const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
                 const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
-                const uint32_t B = __reduce_max_sync(FULL, lane < RW - 1 ? key : (lane == RW - 1 ? sh.red_key2[RW - 1] : 0u));
+                const uint32_t B = __reduce_max_sync(FULL, lane < CLS_G ? key : (lane == CLS_G ? sh.red_key2[CLS_G] : 0u));
                 int k2 = 1; int64_t avail = -1;
                 if (g2 <= sp.Gn) {
                     const int target = v.maxc[gi2] >= c2 ? first_fit_warp(v, g2, c2, lane) : -1;
@@ -830,7 +837,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             u64 nk = 0ull; float nw = 0.0f;
                             if (np < end) { nk = A.keys[np]; nw = A.sorted_w[np]; }
                             v.cls_ptr[t] = np; v.cls_top[t] = nk; v.cls_w[t] = nw;
-                            sh.dirty[RW - 1] = 1;
+                            sh.dirty[CLS_G] = 1;
                             sh.steps = steps0 + n_fail;
                         }
                         n_acc = n_fail;
@@ -855,7 +862,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 top_stays = __any_sync(FULL, st);
             }
             if (go && n_acc == 0 && top_stays) {
-                const uint32_t M = __reduce_max_sync(FULL, lane < RW ? sh.red_key2[lane] : 0u);
+                const uint32_t M = __reduce_max_sync(FULL, lane < N_GROUPS ? sh.red_key2[lane] : 0u);
                 bool elig = false, s_ok = false, s_maxc = false, s_multi = false;
                 int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0, s_k = 1;
                 int64_t s_dm = 0;
@@ -983,7 +990,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if ((acc >> lane) & 1u) {
                         if (s_ok && !s_multi) { v.gc[s_node] -= s_dgc; v.free_m[s_node] -= s_dm; }
                         v.sa[s_slot] = na; v.sb[s_slot] = nb; v.sc[s_slot] = nq;
-                        sh.dirty[(s_slot % SCAN_T) >> 5] = 1;
+                        sh.dirty[(s_slot % SCAN_T) >> 4] = 1;
                         if (s_ok && !s_multi) atomicOr(&v.tb[s_node >> 5], 1u << (s_node & 31));
                         if (A.step_log) A.step_log[steps0 + my_order] = (my_j << 2) | ((s_type ? 0 : 1) << 1) | int(s_ok);
                     }
@@ -1036,10 +1043,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
                             v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j; v.sc[s] = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                             sh.n_slots = s + 1;
-                            sh.dirty[(s % SCAN_T) >> 5] = 1;
+                            sh.dirty[(s % SCAN_T) >> 4] = 1;
                         }
                     }
-                    if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[RW - 1] = 1; }
+                    if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[CLS_G] = 1; }
                 } else {
                     const int s = int(pay);
                     SlotA a = v.sa[s]; SlotB b = v.sb[s];
@@ -1064,7 +1071,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
                         a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
                     }
-                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; sh.dirty[(s % SCAN_T) >> 5] = 1; }
+                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; sh.dirty[(s % SCAN_T) >> 4] = 1; }
                 }
                 if (lane == 0) {
                     if (A.step_log) A.step_log[sh.steps] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
