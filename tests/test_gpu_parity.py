@@ -461,3 +461,24 @@ def test_odd_grid_shapes_through_every_kernel():
     got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 9)
     assert_rounds_equal(got, want)
     assert want["steps"] > 5 and (want["n_nodes"] > 1).any()
+
+
+def test_largest_supported_grid_and_cluster():
+    """64 core levels, 32 memory levels, 4,096 nodes (the limits of the shared-memory state)."""
+    cfg = workloads.make("paper-scale", J=48, n_nodes=4096)
+    cfg["c_levels"] = np.arange(1, 65)
+    cfg["env"] = env(cpus_per_node=64)
+    gpu = Gpu(cfg)
+    assert gpu.nC == 64 and gpu.nM == 32
+    _, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
+    assert np.array_equal(gpu.np_feas(d_feas, 48), feas)
+    check_thr(gpu.np_thr(d_thr, 48), thr)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 4096, want_log=True)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 4096)
+    assert_rounds_equal(got, want)
+    with pytest.raises(rb.RubickError):
+        gpu.ctx.greedy_round(None, 0, None, None, None, None, 4097, 10, None)
+    with pytest.raises(rb.RubickError):
+        gpu.ctx.set_space(gpu.plans, cfg["g_levels"], np.arange(1, 66), cfg["m_levels"])
