@@ -482,3 +482,39 @@ def test_largest_supported_grid_and_cluster():
         gpu.ctx.greedy_round(None, 0, None, None, None, None, 4097, 10, None)
     with pytest.raises(rb.RubickError):
         gpu.ctx.set_space(gpu.plans, cfg["g_levels"], np.arange(1, 66), cfg["m_levels"])
+
+
+def test_outputs_stay_inside_their_buffers():
+    """Every output buffer sits between two guard regions filled with a pattern; after the whole path has
+    run on a ragged job count the guards must be untouched."""
+    cfg = workloads.make("cluster-512", J=203, n_nodes=21)
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    J, N, G = 203, 21, 4096                                  # guard bytes on either side
+
+    def guarded(nbytes):
+        buf = t.full((nbytes + 2 * G,), 0xA5, dtype=t.uint8, device="cuda:0")
+        return buf, buf[G:G + nbytes]
+
+    d_jobs = gpu.jobs_to_device(cfg["jobs"])
+    thr_b, thr = guarded(J * gpu.nC * gpu.P * 4)
+    feas_b, feas = guarded(J * gpu.P * 4)
+    n = J * gpu.nG * gpu.nC * gpu.nM
+    cv_b, cv = guarded(n * 4); cp_b, cp = guarded(n * 4); cg_b, cg = guarded(n * 4)
+    out_b, out = guarded(J * rb.ASSIGN_DTYPE.itemsize); node_b, node = guarded(N * rb.NODE_DTYPE.itemsize)
+    log_b, log = guarded(4 * (J * (gpu.nG + gpu.nC + 2) + 1))
+    gains = [guarded(J * 4) for _ in range(4)]
+    req_out = [guarded(J * 4) for _ in range(3)]
+    gpu.ctx.eval_candidates(d_jobs, J, thr, feas)
+    gpu.ctx.best_plan(thr, feas, J, cv, cp, cg)
+    state = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    gpu.ctx.marginal_gain(d_jobs, J, cv, state, *[g[1] for g in gains])
+    rec = np.zeros(J, dtype=rb.REQUEST_DTYPE)
+    rec["g_idx"], rec["c_idx"], rec["m_idx"], rec["plan"] = 3, 5, 20, 170
+    gpu.ctx.min_resources(thr, feas, cv, J, rb.to_device(rec), *[r[1] for r in req_out])
+    steps, _ = gpu.ctx.greedy_round(d_jobs, J, cv, cp, cg, feas, N, J * (gpu.nG + gpu.nC + 2) + 1, out, node, log)
+    gpu.ctx.greedy_round_noalloc(d_jobs, J, cv, cp, cg, feas, N, 1 << 30, out, node)
+    gpu.ctx.sync()
+    assert steps > 0
+    for whole in [thr_b, feas_b, cv_b, cp_b, cg_b, out_b, node_b, log_b] + [g[0] for g in gains] + [r[0] for r in req_out]:
+        assert bool((whole[:G] == 0xA5).all()) and bool((whole[-G:] == 0xA5).all())
