@@ -188,9 +188,13 @@ int rubick_eval_candidates(rubick_ctx *ctx, const rubick_job *d_jobs, int J, flo
  * (Section 5.2: invalid GPU counts have zero throughput).  Unless RUBICK_BEST_RAW is given the
  * result is turned into the resource-sensitivity curve: the running maximum along the GPU axis,
  * carrying the plan and the GPU count actually used (Section 5.2, Fig. 6).
- * d_best_val / d_best_plan / d_best_g: J*G*C*M entries each.  Feasibility words must be
- * thresholds (bit i set implies every higher level bit set); a violation is reported by
- * rubick_sync as ESTATE. */
+ * d_best_val / d_best_plan / d_best_g: J*G*C*M entries each.  d_thr and d_feas must be 16-byte
+ * aligned; table entries must be finite and >= 0 (what rubick_eval_candidates writes).
+ * Feasibility words must be thresholds (bit i set implies every higher level bit set); a
+ * violation is reported by rubick_sync as ESTATE.  Masks in which the feasible plans of one GPU
+ * level share one first level per offload class (all masks of rubick_eval_candidates) take the
+ * streaming kernel; any other threshold mask is handled by a slower general kernel with the
+ * same results.  The context keeps J + 1 words of scratch (grown on demand with cudaMalloc). */
 int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
                      float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g);
 

@@ -71,6 +71,7 @@ int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *c
     ctx->d_jobs_stage = nullptr; ctx->cap_jobs = 0;
     ctx->d_out_stage = nullptr; ctx->cap_out = 0;
     ctx->d_node_stage = nullptr; ctx->cap_node = 0;
+    ctx->d_best_todo = nullptr; ctx->cap_best_todo = 0;
     ctx->tile_jobs = 2048;            // 0.5 GB table tile at 2,640 plans x 24 core levels
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return RUBICK_ECUDA; }
@@ -91,6 +92,7 @@ void rubick_destroy(rubick_ctx *ctx)
     cudaFree(ctx->d_quads); cudaFree(ctx->d_status); cudaFree(ctx->d_round_scratch);
     cudaFree(ctx->d_thr); cudaFree(ctx->d_feas); cudaFree(ctx->d_cv); cudaFree(ctx->d_cp); cudaFree(ctx->d_cg);
     cudaFree(ctx->d_jobs_stage); cudaFree(ctx->d_out_stage); cudaFree(ctx->d_node_stage);
+    cudaFree(ctx->d_best_todo);
     delete ctx;
 }
 
@@ -250,9 +252,12 @@ int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas
     if (rc) return rc;
     if (J == 0) return RUBICK_OK;
     if (!d_thr || !d_feas || !d_best_val || !d_best_plan || !d_best_g) return fail(ctx, RUBICK_EINVAL, "null pointer");
-    if (reinterpret_cast<uintptr_t>(d_thr) & 15) return fail(ctx, RUBICK_EINVAL, "d_thr must be 16-byte aligned");
+    if ((reinterpret_cast<uintptr_t>(d_thr) & 15) || (reinterpret_cast<uintptr_t>(d_feas) & 15))
+        return fail(ctx, RUBICK_EINVAL, "d_thr and d_feas must be 16-byte aligned");
     if (flags & ~RUBICK_BEST_RAW) return fail(ctx, RUBICK_EINVAL, "unknown flag");
-    CUDA_TRY(ctx, launch_best(ctx->space, d_thr, d_feas, J, flags, d_best_val, d_best_plan, d_best_g, ctx->d_status, ctx->stream),
+    if ((rc = ensure(ctx, ctx->d_best_todo, ctx->cap_best_todo, size_t(J) + 1))) return rc;
+    CUDA_TRY(ctx, launch_best(ctx->space, d_thr, d_feas, J, flags, d_best_val, d_best_plan, d_best_g, ctx->d_status,
+                              ctx->d_best_todo, ctx->num_sms, ctx->stream),
              "launch best_plan");
     return RUBICK_OK;
 }
@@ -373,6 +378,7 @@ static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
     int rc;
     if ((rc = ensure(ctx, ctx->d_thr, ctx->cap_thr, size_t(tile) * sp.nC * sp.P))) return rc;
     if ((rc = ensure(ctx, ctx->d_feas, ctx->cap_feas, size_t(J) * sp.P))) return rc;
+    if ((rc = ensure(ctx, ctx->d_best_todo, ctx->cap_best_todo, size_t(tile) + 1))) return rc;
     const size_t curve = size_t(J) * sp.nG * sp.nC * sp.nM;
     if (curve > ctx->cap_curve) {
         size_t c1 = ctx->cap_curve, c2 = ctx->cap_curve, c3 = ctx->cap_curve;
@@ -386,7 +392,8 @@ static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
         const int n = J - j0 < tile ? J - j0 : tile;
         CUDA_TRY(ctx, launch_eval(sp, ctx->d_quads, d_jobs + j0, n, ctx->d_thr, ctx->d_feas + size_t(j0) * sp.P, ctx->stream), "launch eval_candidates");
         CUDA_TRY(ctx, launch_best(sp, ctx->d_thr, ctx->d_feas + size_t(j0) * sp.P, n, 0u, ctx->d_cv + j0 * per_job,
-                                  ctx->d_cp + j0 * per_job, ctx->d_cg + j0 * per_job, ctx->d_status, ctx->stream),
+                                  ctx->d_cp + j0 * per_job, ctx->d_cg + j0 * per_job, ctx->d_status, ctx->d_best_todo,
+                                  ctx->num_sms, ctx->stream),
                  "launch best_plan");
     }
     return RUBICK_OK;

@@ -81,6 +81,7 @@ struct rubick_ctx {
     rubick_job *d_jobs_stage; size_t cap_jobs;
     rubick_assignment *d_out_stage; size_t cap_out;
     rubick_node *d_node_stage; size_t cap_node;
+    int32_t *d_best_todo; size_t cap_best_todo;     // rubick_best_plan: count + jobs left to the general kernel
     int tile_jobs;                      // job tile of rubick_schedule_round
     int num_sms;
     std::string err;
@@ -96,7 +97,7 @@ cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_j
                         float *d_thr, uint32_t *d_feas, cudaStream_t st);
 cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
                         float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, uint32_t *d_status,
-                        cudaStream_t st);
+                        int32_t *d_todo /* J + 1 words of scratch */, int num_sms, cudaStream_t st);
 cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const float *d_curve_val,
                         const rubick_assignment *d_state, float *d_gain_gpu, float *d_gain_cpu,
                         int32_t *d_next_g, int32_t *d_next_c, cudaStream_t st);
