@@ -151,6 +151,37 @@ def test_best_plan_with_scattered_feasibility_levels():
     assert np.array_equal(bg.cpu().numpy().reshape(sh), cg)
 
 
+@pytest.mark.parametrize("raw", [False, True])
+def test_best_plan_with_two_class_and_scattered_masks_in_one_batch(raw):
+    """Jobs whose masks have one first level per (GPU level, offload class) take the streaming
+    kernel, the others the general one; both in one call, with tie-heavy values, classes without
+    feasible plans, and either class lower than the other."""
+    cfg = workloads.make("paper-scale", J=24)
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    rng = np.random.default_rng(7)
+    plans, group_off = oracle.enumerate_plans(cfg["g_levels"])
+    J, nC, P, nM, nG = 24, gpu.nC, gpu.P, gpu.nM, gpu.nG
+    thr = rng.integers(0, 5, (J, nC, P)).astype(np.float32)
+    thr[:, :, ::7] *= 0.5
+    level_of = np.searchsorted(np.asarray(group_off[1:], dtype=np.int64), np.arange(P), side="right")
+    odd = (np.arange(P) & 1).astype(np.int64)
+    first = rng.integers(0, nM + 6, (J, nG, 2))                           # >= nM: the class has no feasible plan
+    f = first[np.arange(J)[:, None], level_of[None, :], odd[None, :]]
+    f = np.where(rng.uniform(size=(J, P)) < 0.4, nM, f)                   # plans that fit nowhere (GPU memory)
+    scattered = np.arange(J) % 3 == 1
+    f[scattered] = rng.integers(0, nM + 8, (int(scattered.sum()), P))
+    f[5, :] = nM                                                          # a job with nothing feasible
+    feas = np.where(f >= nM, 0, (0xFFFFFFFF << np.minimum(f, 31)) & 0xFFFFFFFF).astype(np.uint32)
+    cv, cp, cg = oracle.best_plan(thr, feas, plans, cfg["g_levels"], nM, prefix=not raw, nthreads=8)
+    bv, bp, bg = gpu.best(t.from_numpy(thr.reshape(-1)).cuda(), t.from_numpy(feas.view(np.int32).reshape(-1)).cuda(), J,
+                          flags=rb.BEST_RAW if raw else 0)
+    sh = gpu.shape4(J)
+    assert np.array_equal(bv.cpu().numpy().reshape(sh), cv.astype(np.float32))
+    assert np.array_equal(bp.cpu().numpy().reshape(sh), cp)
+    assert np.array_equal(bg.cpu().numpy().reshape(sh), cg)
+
+
 def test_non_threshold_feasibility_word_is_reported():
     cfg = workloads.make("tiny")
     gpu = Gpu(cfg)
