@@ -214,6 +214,60 @@ def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_
                 steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
 
 
+def schedule_round_incremental(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,
+                               n_nodes, prev, active=None, T=None, delta=None, nrec=None, theta=0.97,
+                               max_steps=1 << 30, want_log=False, quota=None):
+    """One incremental round (shrink / exchange step and reconfiguration gate) from `prev`, the dict a
+    previous round returned (None: an empty cluster).  active [J] marks used job slots; T, delta
+    (seconds) and nrec feed the gate.  -> dict like schedule_round; steps is None when `prev` does
+    not fit the grid or the cluster."""
+    rows = job_rows(jobs)
+    J = rows.shape[0]
+    cv = np.ascontiguousarray(curve_val, dtype=np.float32)
+    cp, cg = _i32(curve_plan), _i32(curve_g)
+    feas = np.ascontiguousarray(feas, dtype=np.uint32)
+    Pn = feas.shape[1] if feas.ndim == 2 else 0
+    gl, cl, ml = _i64(g_levels), _i64(c_levels), _i64(m_levels)
+    prev_i = np.zeros((max(J, 1), 8), dtype=np.int64)
+    prev_v = np.zeros(max(J, 1), dtype=np.float32)
+    prev_owner = np.full(n_nodes, -1, dtype=np.int32)
+    if prev is not None:
+        for col, key in enumerate(("g", "c", "m_bytes", "plan", "first_node", "n_nodes", "status", "m_level")):
+            prev_i[:J, col] = np.asarray(prev[key], dtype=np.int64)
+        prev_v[:J] = np.asarray(prev["thr"], dtype=np.float32)
+        prev_owner[:] = np.asarray(prev["node"], dtype=np.int64)[:, 3].astype(np.int32)
+    act = np.ones(max(J, 1), dtype=np.int32) if active is None else np.ascontiguousarray(active, dtype=np.int32)
+    Tt = np.full(max(J, 1), 1e9, dtype=np.float32) if T is None else np.ascontiguousarray(T, dtype=np.float32)
+    dl = np.zeros(max(J, 1), dtype=np.float32) if delta is None else np.ascontiguousarray(delta, dtype=np.float32)
+    nr = np.zeros(max(J, 1), dtype=np.int32) if nrec is None else np.ascontiguousarray(nrec, dtype=np.int32)
+    out_i = np.zeros((max(J, 1), 8), dtype=np.int64)
+    out_v = np.zeros(max(J, 1), dtype=np.float32)
+    node = np.zeros((n_nodes, 4), dtype=np.int64)
+    cap = int(min(max_steps, 2 * J * (len(gl) + len(cl) + 2) + 1))
+    log = np.zeros(max(cap, 1), dtype=np.int32)
+    qt = None if quota is None else _i64(quota).reshape(-1, 2)
+    f = lib().oracle_round_incremental
+    f.restype = C.c_int
+    r = f(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double), _p(cv, C.c_float),
+          _p(cp, C.c_int32), _p(cg, C.c_int32), _p(feas, C.c_uint32), C.c_int(Pn),
+          _p(gl, C.c_int64), C.c_int(len(gl)), _p(cl, C.c_int64), C.c_int(len(cl)),
+          _p(ml, C.c_int64), C.c_int(len(ml)), C.c_int(n_nodes), C.c_int(cap),
+          _p(qt, C.c_int64) if qt is not None else None, C.c_int(0 if qt is None else len(qt)),
+          _p(prev_i, C.c_int64), _p(prev_v, C.c_float), _p(prev_owner, C.c_int32), _p(act, C.c_int32),
+          _p(Tt, C.c_float), _p(dl, C.c_float), _p(nr, C.c_int32), C.c_float(theta),
+          _p(out_i, C.c_int64), _p(out_v, C.c_float), _p(node, C.c_int64),
+          _p(log, C.c_int32) if want_log else None)
+    if r == -2 ** 31:
+        return dict(steps=None)
+    capped = r < 0
+    steps = -r - 1 if capped else r
+    out_i = out_i[:J]
+    return dict(g=out_i[:, 0].copy(), c=out_i[:, 1].copy(), m_bytes=out_i[:, 2].copy(),
+                plan=out_i[:, 3].copy(), first_node=out_i[:, 4].copy(), n_nodes=out_i[:, 5].copy(),
+                status=out_i[:, 6].copy(), m_level=out_i[:, 7].copy(), thr=out_v[:J].copy(), node=node,
+                steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
+
+
 def bruteforce(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels):
     """Best total weighted throughput over all single-node assignments (tiny instances)."""
     rows = job_rows(jobs)

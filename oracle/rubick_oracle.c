@@ -4,8 +4,9 @@
  * A plain, slow, double-precision CPU statement of what the scheduler's data-parallel
  * path computes: the training-performance model (paper Section 4), the plan space and
  * the best-plan / resource-sensitivity-curve step (Section 5.2), the marginal-gain
- * ("slope") score and one greedy scheduling round (Section 5.2, Algorithm 1, in the
- * grow-only marginal-gain form), plus an exhaustive search used on tiny instances.
+ * ("slope") score, one greedy scheduling round (Section 5.2, Algorithm 1, in the
+ * grow-only marginal-gain form) and the incremental round with Algorithm 1's shrink step
+ * and the reconfiguration gate, plus an exhaustive search used on tiny instances.
  *
  * Only the test-suite, the smoke check and the CPU-baseline leg of the benchmark may
  * build or call this file.  It shares nothing with the CUDA library: no header, no
@@ -28,6 +29,9 @@
  *     implemented here is this project's reading; pinned by the exhaustive search
  *     (upper bound, equality on concave single-resource instances) and capacity
  *     invariants, otherwise "parity unpinned by the paper".
+ *   - incremental round: same status; pinned by its reductions (empty previous state =
+ *     the grow-only round; everything pinned = the previous state), the exhaustive search as
+ *     an upper bound, capacity / minimum-demand / gate invariants and hand-made exchanges.
  */
 #include <math.h>
 #include <stdint.h>
@@ -703,6 +707,330 @@ int oracle_round(const double *jobs, int J, const double *env,
             node_out[(size_t)n * 4 + 2] = S.free_m[n]; node_out[(size_t)n * 4 + 3] = S.owner[n];
         }
     free(S.free_g); free(S.free_c); free(S.free_m); free(S.owner); free(st);
+    return capped ? -steps - 1 : steps;
+}
+
+/* ======================================================================================
+ * Incremental round: Algorithm 1 with its shrink step, started from the previous allocation
+ * (Section 5.2 "Scheduling algorithm design" and "Incorporating reconfiguration penalty").
+ *
+ * Reading (the paper leaves the step size, the order of attempts and the roll-back open):
+ *  - Job slots keep their index between rounds; active[j] = 0 marks an empty slot.  A job
+ *    whose previous status is RUNNING keeps its GPUs, cores, memory, plan and node(s).
+ *  - Gate: a running job may be touched only if T > 0 and (T - (N + 1) * delta) / T > theta
+ *    (T seconds trained, N reconfigurations so far, delta seconds per checkpoint-resume; the
+ *    contemplated reconfiguration is counted).  Otherwise it is pinned: it neither grows nor
+ *    shrinks in this round.
+ *  - Minimum of a guaranteed job: the GPU count the curve really uses at (gmin, cmin), and cmin
+ *    cores.  Best-effort jobs have none.
+ *  - Shrink step of a running, unpinned single-node job ("over its minimum"): GPUs go down to the
+ *    next lower level whose own plans run (not below the minimum; a best-effort job without such
+ *    a level is preempted: everything released, back to the queue); cores go down one level (not
+ *    below the minimum, never to zero).  Its slope is the weighted value lost per unit given up,
+ *    read at the top memory level like the gains.  The shrunk job's plan and memory are
+ *    re-selected on its node (GetBestPlan / AllocMem); a step that does not fit is not offered.
+ *  - Exchange for an increment of job j on node n: while the node lacks GPUs (then cores) for
+ *    it, shrink the offered job on n with the lowest slope (lowest index on ties), provided the
+ *    slope is below j's gain for that resource, or unconditionally while j is a guaranteed job
+ *    being placed at its minimum.  A running job may reclaim only the resource of its
+ *    increment; a queued job pre-allocates GPUs and cores together, so its value per GPU and
+ *    per core are its two gains.  At most MAX_EXCHANGE shrink steps; then j is committed on n.  Any failure undoes the whole attempt.  Shrunk jobs do not grow again in the round.
+ *  - Phase A: queued guaranteed jobs in index order, within what their tenant's quota leaves
+ *    after the minima of its running guaranteed jobs, are placed at their minimum: free
+ *    resources first (first fit), else by exchange on the first node where it succeeds.
+ *  - Phase B: as in the grow-only round while some increment fits free resources.  When none
+ *    does, the largest-gain increment that is not frozen (GPU before CPU, lowest index on ties)
+ *    tries an exchange: a running single-node job on its own node, a queued job on the first node
+ *    where it succeeds; increments above one node never exchange.  Failure freezes (job, type).
+ *  step_log entry: (job << 3) | (by exchange << 2) | (type << 1) | accepted.
+ * ==================================================================================== */
+#define MAX_EXCHANGE 64
+
+typedef struct { int ok; int gi2, ci2; float slope; } Shrink;
+
+/* what job v would give up next of resource `type`, and at what loss per unit */
+static Shrink shrink_option(const Sched *S, int v, const JobState *js, int type, int guaranteed, int min_gi, int min_ci)
+{
+    Shrink sh; sh.ok = 0; sh.gi2 = -1; sh.ci2 = js->ci; sh.slope = 0.0f;
+    if (js->gi < 0 || js->k != 1) return sh;
+    const double *job = S->jobs + (size_t)v * JF_COUNT;
+    float w = (float)job[JF_W];
+    int mt = S->nM - 1;
+    float vcur = w * js->val;
+    if (type == 0) {
+        if (guaranteed && min_gi < 0) return sh;
+        int lo = guaranteed ? min_gi : 0;
+        for (int i = js->gi - 1; i >= lo; --i) {
+            size_t o = cidx(S, v, i, js->ci, mt);
+            if (S->cp[o] >= 0 && (int64_t)S->cg[o] == S->g_levels[i]) {
+                sh.ok = 1; sh.gi2 = i;
+                sh.slope = (vcur - w * S->cv[o]) / (float)(js->g - S->g_levels[i]);
+                return sh;
+            }
+        }
+        if (guaranteed) return sh;
+        sh.ok = 1; sh.gi2 = -1;                      /* preemption */
+        sh.slope = (vcur - w * 0.0f) / (float)js->g;
+        return sh;
+    }
+    int lo = guaranteed ? min_ci : 0;
+    if (js->ci - 1 < lo) return sh;
+    size_t o = cidx(S, v, js->gi, js->ci - 1, mt);
+    if (S->cp[o] < 0 || (int64_t)S->cg[o] != js->g) return sh;
+    sh.ok = 1; sh.gi2 = js->gi; sh.ci2 = js->ci - 1;
+    sh.slope = (vcur - w * S->cv[o]) / (float)(js->c - S->c_levels[js->ci - 1]);
+    return sh;
+}
+
+/* performs the shrink step (apply != 0) or only tells whether it fits (apply == 0) */
+static int do_shrink(Sched *S, int v, JobState *js, Shrink sh, int apply)
+{
+    if (sh.gi2 < 0) {
+        if (apply) {
+            release_job(S, v, js);
+            js->gi = -1; js->ci = 0; js->g = js->c = js->m = 0; js->plan = -1; js->node = -1; js->k = 0;
+            js->val = 0.0f; js->status = ST_UNALLOCATED;
+        }
+        return 1;
+    }
+    int n = js->node;
+    int64_t fg = S->free_g[n], fc = S->free_c[n], fm = S->free_m[n];
+    JobState keep = *js;
+    Place pl; pl.ok = 1; pl.k = 1; pl.stay = 1; pl.node = n; pl.need_new = 0;
+    int ok = commit(S, v, js, sh.gi2, sh.ci2, pl, 0);
+    if (!ok || !apply) { S->free_g[n] = fg; S->free_c[n] = fc; S->free_m[n] = fm; *js = keep; }
+    return ok;
+}
+
+typedef struct { const int *pinned, *guaranteed, *min_gi, *min_ci; } Roles;
+
+static int exchange(Sched *S, JobState *st, const Roles *R, int j, int gi2, int ci2, int n,
+                    int force, const float *cand_gain, int need_gain)
+{
+    int J = S->J, N = S->N;
+    JobState *st0 = (JobState *)malloc(sizeof(JobState) * (size_t)J);
+    int64_t *node0 = (int64_t *)malloc(sizeof(int64_t) * 3 * (size_t)N);
+    int32_t *own0 = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    memcpy(st0, st, sizeof(JobState) * (size_t)J);
+    memcpy(node0, S->free_g, sizeof(int64_t) * (size_t)N);
+    memcpy(node0 + N, S->free_c, sizeof(int64_t) * (size_t)N);
+    memcpy(node0 + 2 * N, S->free_m, sizeof(int64_t) * (size_t)N);
+    memcpy(own0, S->owner, sizeof(int32_t) * (size_t)N);
+
+    int on_n = st[j].gi >= 0 && st[j].k == 1 && st[j].node == n;
+    int64_t need[2];
+    need[0] = S->g_levels[gi2] - (on_n ? st[j].g : 0);
+    need[1] = S->c_levels[ci2] - (on_n ? st[j].c : 0);
+    int ok = 1, taken = 0;
+    for (int r = 0; r < 2 && ok; ++r) {
+        int64_t *free_r = r == 0 ? S->free_g : S->free_c;
+        while (free_r[n] < need[r]) {
+            if (!force && !(cand_gain[r] > 0.0f)) { ok = 0; break; }    /* this resource may not be reclaimed */
+            int best = -1; Shrink best_sh; best_sh.slope = 0.0f;
+            for (int v = 0; v < J; ++v) {
+                if (v == j || st[v].gi < 0 || st[v].k != 1 || st[v].node != n || R->pinned[v]) continue;
+                Shrink sh = shrink_option(S, v, &st[v], r, R->guaranteed[v], R->min_gi[v], R->min_ci[v]);
+                if (!sh.ok || !do_shrink(S, v, &st[v], sh, 0)) continue;
+                if (best < 0 || sh.slope < best_sh.slope) { best = v; best_sh = sh; }
+            }
+            if (best < 0) { ok = 0; break; }
+            if (!force && !(cand_gain[r] > best_sh.slope)) { ok = 0; break; }
+            if (++taken > MAX_EXCHANGE) { ok = 0; break; }
+            do_shrink(S, best, &st[best], best_sh, 1);
+            st[best].frozen[0] = st[best].frozen[1] = 1;
+        }
+    }
+    if (ok) {
+        Place pl; pl.ok = 1; pl.k = 1; pl.stay = on_n; pl.node = n; pl.need_new = 0;
+        ok = commit(S, j, &st[j], gi2, ci2, pl, need_gain);
+    }
+    if (!ok) {
+        memcpy(st, st0, sizeof(JobState) * (size_t)J);
+        memcpy(S->free_g, node0, sizeof(int64_t) * (size_t)N);
+        memcpy(S->free_c, node0 + N, sizeof(int64_t) * (size_t)N);
+        memcpy(S->free_m, node0 + 2 * N, sizeof(int64_t) * (size_t)N);
+        memcpy(S->owner, own0, sizeof(int32_t) * (size_t)N);
+    }
+    free(st0); free(node0); free(own0);
+    return ok;
+}
+
+/* prev_i [J][8], prev_val [J]: the previous round's out_i / out_val (status RUNNING = carried
+ * over); prev_owner [N]: its node owners; active [J]; T, delta [J] seconds; nrec [J]
+ * reconfigurations so far; theta: the gate's threshold (the paper uses 0.97).
+ * Outputs as oracle_round.  Returns the number of Phase-B steps, negated - 1 if capped;
+ * INT32_MIN when the previous state does not fit the grid or the cluster. */
+int oracle_round_incremental(const double *jobs, int J, const double *env,
+                             const float *curve_val, const int32_t *curve_plan, const int32_t *curve_g,
+                             const uint32_t *feas, int P,
+                             const int64_t *g_levels, int nG, const int64_t *c_levels, int nC,
+                             const int64_t *m_levels, int nM, int N, int max_steps,
+                             const int64_t *quota, int n_tenants,
+                             const int64_t *prev_i, const float *prev_val, const int32_t *prev_owner,
+                             const int32_t *active, const float *T, const float *delta, const int32_t *nrec,
+                             float theta,
+                             int64_t *out_i, float *out_val, int64_t *node_out, int32_t *step_log)
+{
+    Sched S; memset(&S, 0, sizeof S);
+    S.J = J; S.nG = nG; S.nC = nC; S.nM = nM; S.P = P; S.N = N;
+    S.cv = curve_val; S.cp = curve_plan; S.cg = curve_g; S.feas = feas; S.jobs = jobs;
+    S.g_levels = g_levels; S.c_levels = c_levels; S.m_levels = m_levels;
+    S.Gn = (int64_t)env[EF_GN]; S.Cn = (int64_t)env[EF_CN]; S.Mn = (int64_t)env[EF_MN];
+    S.free_g = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    S.free_c = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    S.free_m = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
+    S.owner = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    for (int n = 0; n < N; ++n) { S.free_g[n] = S.Gn; S.free_c[n] = S.Cn; S.free_m[n] = S.Mn; S.owner[n] = -1; }
+    size_t Jn = (size_t)(J > 0 ? J : 1);
+    JobState *st = (JobState *)calloc(Jn, sizeof(JobState));
+    int *pinned = (int *)calloc(Jn, sizeof(int)), *guaranteed = (int *)calloc(Jn, sizeof(int));
+    int *min_gi = (int *)calloc(Jn, sizeof(int)), *min_ci = (int *)calloc(Jn, sizeof(int));
+    Roles R; R.pinned = pinned; R.guaranteed = guaranteed; R.min_gi = min_gi; R.min_ci = min_ci;
+    int mt = nM - 1, bad = 0;
+
+    /* carried state, minima, gate */
+    for (int j = 0; j < J; ++j) {
+        const double *job = jobs + (size_t)j * JF_COUNT;
+        st[j].gi = -1; st[j].plan = -1; st[j].node = -1; st[j].status = ST_UNALLOCATED;
+        guaranteed[j] = (int)job[JF_GMIN] >= 0;
+        min_gi[j] = -1; min_ci[j] = start_ci(job);
+        if (guaranteed[j] && (int)job[JF_GMIN] < nG && min_ci[j] < nC) {
+            size_t o = cidx(&S, j, (int)job[JF_GMIN], min_ci[j], mt);
+            if (curve_plan[o] >= 0)
+                for (int i = 0; i < nG; ++i) if (g_levels[i] == (int64_t)curve_g[o]) min_gi[j] = i;
+        }
+        if (!active[j] || prev_i[(size_t)j * 8 + 6] != ST_RUNNING) continue;
+        const int64_t *pv = prev_i + (size_t)j * 8;
+        int gi = -1, ci = -1;
+        for (int i = 0; i < nG; ++i) if (g_levels[i] == pv[0]) gi = i;
+        for (int i = 0; i < nC; ++i) if (c_levels[i] == pv[1]) ci = i;
+        int k = (int)pv[5];
+        if (gi < 0 || ci < 0 || pv[3] < 0 || pv[3] >= P || pv[4] < 0 || pv[4] >= N || k < 1
+            || (k == 1 ? pv[0] > S.Gn : pv[0] != (int64_t)k * S.Gn)) { bad = 1; continue; }
+        st[j].gi = gi; st[j].ci = ci; st[j].g = pv[0]; st[j].c = pv[1]; st[j].m = pv[2];
+        st[j].plan = (int)pv[3]; st[j].node = (int)pv[4]; st[j].k = k; st[j].val = prev_val[j];
+        st[j].status = ST_RUNNING;
+        if (k == 1) {
+            int n = st[j].node;
+            S.free_g[n] -= st[j].g; S.free_c[n] -= st[j].c; S.free_m[n] -= st[j].m;
+        } else {
+            int cnt = 0;
+            for (int n = 0; n < N; ++n)
+                if (prev_owner[n] == j) {
+                    S.free_g[n] -= S.Gn; S.free_c[n] -= cdiv(st[j].c, k); S.free_m[n] -= cdiv(st[j].m, k);
+                    S.owner[n] = j; ++cnt;
+                }
+            if (cnt != k) bad = 1;
+        }
+        float t = T[j];
+        int pass = t > 0.0f && (t - (float)(nrec[j] + 1) * delta[j]) / t > theta;
+        pinned[j] = !pass;
+    }
+    for (int n = 0; n < N; ++n) if (S.free_g[n] < 0 || S.free_c[n] < 0 || S.free_m[n] < 0) bad = 1;
+    if (bad) {
+        free(S.free_g); free(S.free_c); free(S.free_m); free(S.owner); free(st);
+        free(pinned); free(guaranteed); free(min_gi); free(min_ci);
+        return INT32_MIN;
+    }
+
+    /* Phase A: queued guaranteed jobs within their tenant's remaining quota */
+    int64_t *rem = NULL;
+    if (n_tenants > 0) {
+        rem = (int64_t *)malloc(sizeof(int64_t) * 2 * (size_t)n_tenants);
+        memcpy(rem, quota, sizeof(int64_t) * 2 * (size_t)n_tenants);
+        for (int j = 0; j < J; ++j) {
+            int t = (int)jobs[(size_t)j * JF_COUNT + JF_TENANT];
+            if (st[j].gi >= 0 && guaranteed[j] && min_gi[j] >= 0 && t >= 0 && t < n_tenants) {
+                rem[2 * t] -= g_levels[min_gi[j]]; rem[2 * t + 1] -= c_levels[min_ci[j]];
+            }
+        }
+    }
+    for (int j = 0; j < J; ++j) {
+        if (!active[j] || !guaranteed[j] || st[j].gi >= 0) continue;
+        st[j].status = ST_PENDING;
+        if (min_gi[j] < 0) continue;
+        int gi = min_gi[j], cmin = min_ci[j];
+        int t = (int)jobs[(size_t)j * JF_COUNT + JF_TENANT];
+        if (n_tenants > 0) {
+            if (t < 0 || t >= n_tenants) continue;
+            if (rem[2 * t] < g_levels[gi] || rem[2 * t + 1] < c_levels[cmin]) continue;
+        }
+        Place pl = find_place(&S, &st[j], g_levels[gi], c_levels[cmin]);
+        int placed = pl.ok && commit(&S, j, &st[j], gi, cmin, pl, 0);
+        if (!placed && g_levels[gi] <= S.Gn)
+            for (int n = 0; n < N && !placed; ++n)
+                placed = exchange(&S, st, &R, j, gi, cmin, n, 1, NULL, 0);
+        if (!placed) { st[j].status = ST_PENDING; continue; }
+        if (n_tenants > 0) { rem[2 * t] -= g_levels[gi]; rem[2 * t + 1] -= c_levels[cmin]; }
+    }
+    free(rem);
+
+    /* Phase B */
+    int steps = 0, capped = 0;
+    for (;;) {
+        int best_j = -1, best_type = -1, best_next = -1, by_exchange = 0; float best_gain = 0.0f;
+        for (int pass = 0; pass < 2 && best_j < 0; ++pass)          /* 0: fits free resources; 1: any */
+            for (int type = 0; type < 2 && best_j < 0; ++type)
+                for (int j = 0; j < J; ++j) {
+                    if (!active[j] || pinned[j] || st[j].status == ST_PENDING || st[j].frozen[type]) continue;
+                    int32_t next[2]; float gain[2];
+                    job_gains(&S, j, &st[j], next, gain);
+                    if (next[type] < 0 || !(gain[type] > 0.0f)) continue;
+                    if (pass == 0) {
+                        int gi2 = type == 0 ? next[0] : st[j].gi;
+                        int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
+                        Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+                        if (!pl.ok) continue;
+                    }
+                    if (gain[type] > best_gain) { best_gain = gain[type]; best_j = j; best_type = type; best_next = next[type]; by_exchange = pass; }
+                }
+        if (best_j < 0) break;
+        if (steps >= max_steps) { capped = 1; break; }
+        int j = best_j;
+        int gi2 = best_type == 0 ? best_next : st[j].gi;
+        int ci2 = best_type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : best_next;
+        int ok = 0;
+        if (!by_exchange) {
+            Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+            ok = commit(&S, j, &st[j], gi2, ci2, pl, 1);
+        } else if (g_levels[gi2] <= S.Gn) {
+            /* what j gains per unit of each resource it would take from others: a running job only
+             * asks for the resource of its increment; a queued job pre-allocates GPUs and cores
+             * together, so its value counts per GPU and per core */
+            float cand[2] = {0.0f, 0.0f};
+            cand[best_type] = best_gain;
+            if (st[j].gi >= 0) {
+                if (st[j].k == 1) ok = exchange(&S, st, &R, j, gi2, ci2, st[j].node, 0, cand, 1);
+            } else {
+                float w = (float)jobs[(size_t)j * JF_COUNT + JF_W];
+                cand[1] = (w * curve_val[cidx(&S, j, gi2, ci2, mt)] - 0.0f) / (float)c_levels[ci2];
+                for (int n = 0; n < N && !ok; ++n)
+                    ok = exchange(&S, st, &R, j, gi2, ci2, n, 0, cand, 1);
+            }
+        }
+        if (!ok) st[j].frozen[best_type] = 1;
+        if (step_log) step_log[steps] = (int32_t)((j << 3) | (by_exchange << 2) | (best_type << 1) | ok);
+        ++steps;
+    }
+
+    for (int j = 0; j < J; ++j) {
+        int64_t *o = out_i + (size_t)j * 8;
+        int alloc = st[j].gi >= 0;
+        o[0] = alloc ? st[j].g : 0; o[1] = alloc ? st[j].c : 0; o[2] = alloc ? st[j].m : 0;
+        o[3] = alloc ? st[j].plan : -1; o[4] = alloc ? st[j].node : -1; o[5] = alloc ? st[j].k : 0;
+        o[6] = st[j].status;
+        int f = -1;
+        if (alloc) { uint32_t wd = feas[(size_t)j * P + st[j].plan]; f = 0; while (f < nM && !((wd >> f) & 1u)) ++f; }
+        o[7] = f;
+        out_val[j] = alloc ? st[j].val : 0.0f;
+    }
+    if (node_out)
+        for (int n = 0; n < N; ++n) {
+            node_out[(size_t)n * 4 + 0] = S.free_g[n]; node_out[(size_t)n * 4 + 1] = S.free_c[n];
+            node_out[(size_t)n * 4 + 2] = S.free_m[n]; node_out[(size_t)n * 4 + 3] = S.owner[n];
+        }
+    free(S.free_g); free(S.free_c); free(S.free_m); free(S.owner); free(st);
+    free(pinned); free(guaranteed); free(min_gi); free(min_ci);
     return capped ? -steps - 1 : steps;
 }
 
