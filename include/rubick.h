@@ -137,6 +137,15 @@ typedef struct {
     int32_t reserved;
 } rubick_node;
 
+/* What the reconfiguration gate of an incremental round needs to know about one job slot
+ * (paper Section 5.2, "Incorporating reconfiguration penalty"). 16 bytes. */
+typedef struct {
+    float   T;                   /* seconds the job has trained so far                               */
+    float   delta;               /* seconds one checkpoint-resume of the job costs                   */
+    int32_t n_reconf;            /* times the job has been reconfigured so far                       */
+    int32_t active;              /* 0: the slot is empty (job finished or never submitted)           */
+} rubick_reconf;
+
 /* ---- context ---------------------------------------------------------------------------------- */
 
 /* Creates a context bound to CUDA device `device` and to `cuda_stream` (a cudaStream_t passed as
@@ -232,6 +241,38 @@ int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
                         const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                         int32_t *h_steps);
+
+/* One incremental scheduling round (Section 5.2: Algorithm 1 with its shrink step, and
+ * "Incorporating reconfiguration penalty") on given curve tables, started from the allocation an
+ * earlier round left.  Job slots keep their index between rounds.
+ *  - d_prev / d_prev_nodes: the d_out and d_node_out of the earlier round on the same grid and
+ *    cluster (both NULL: an empty cluster).  A slot whose previous status is RUNNING keeps its
+ *    GPUs, cores, memory, plan and node(s); to retire a finished job clear its status (or mark the
+ *    slot inactive in d_reconf) before the call.
+ *  - d_reconf (NULL: every slot active, every job free to change): a running job may be touched in
+ *    this round only if T > 0 and (T - (n_reconf + 1) * delta) / T > theta (the paper uses 0.97);
+ *    otherwise it keeps its allocation and plan.
+ *  - A running, unpinned single-node job can be shrunk: GPUs to the next lower level whose own
+ *    plans run, cores by one level, never below its guaranteed minimum (the GPUs the curve uses at
+ *    (gmin_idx, cmin_idx), and cmin_idx cores); a best-effort job with no lower level is preempted
+ *    (status UNALLOCATED).  Jobs that span whole nodes are not shrunk.
+ *  - Queued guaranteed jobs are placed first at their minimum, within what their tenant's quota
+ *    leaves after the minima of its running guaranteed jobs: on free resources, else by shrinking
+ *    the lowest-slope jobs of the first node where that works.  Then increments are taken by
+ *    largest gain as in rubick_greedy_round while any fits free resources; when none does, the
+ *    largest-gain increment may take resources from the lowest-slope jobs on its node (a queued
+ *    job: the first node where it works) while its gain per unit exceeds their loss per unit.  An
+ *    exchange is all or nothing; a job shrunk in a round does not grow again in it.
+ * d_step_log entries: job << 3 | by exchange << 2 | type << 1 | accepted.  Returns ESTATE when the
+ * previous state does not fit the grid or the cluster (outputs are then not written), ESTEPS if
+ * max_steps was reached first.  gpus_per_node must not exceed 32.  Blocks until the round is done. */
+int rubick_incremental_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                             const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
+                             const uint32_t *d_feas, const rubick_cluster *h_cluster,
+                             const rubick_assignment *d_prev, const rubick_node *d_prev_nodes,
+                             const rubick_reconf *d_reconf, float theta, int max_steps,
+                             rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                             int32_t *h_steps);
 
 /* rubick_greedy_round for callers that cannot allocate device memory when they schedule: a
  * daemon that received a fixed device-memory budget at start-up and shares the GPU with jobs

@@ -906,7 +906,8 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
         for (int i = 0; i < nC; ++i) if (c_levels[i] == pv[1]) ci = i;
         int k = (int)pv[5];
         if (gi < 0 || ci < 0 || pv[3] < 0 || pv[3] >= P || pv[4] < 0 || pv[4] >= N || k < 1
-            || (k == 1 ? pv[0] > S.Gn : pv[0] != (int64_t)k * S.Gn)) { bad = 1; continue; }
+            || (k == 1 ? pv[0] > S.Gn : pv[0] != (int64_t)k * S.Gn)
+            || pv[7] < 0 || pv[7] >= nM || m_levels[pv[7]] != pv[2]) { bad = 1; continue; }
         st[j].gi = gi; st[j].ci = ci; st[j].g = pv[0]; st[j].c = pv[1]; st[j].m = pv[2];
         st[j].plan = (int)pv[3]; st[j].node = (int)pv[4]; st[j].k = k; st[j].val = prev_val[j];
         st[j].status = ST_RUNNING;

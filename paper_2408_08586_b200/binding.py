@@ -28,6 +28,7 @@ PLAN_DTYPE = np.dtype([("log2d", "u1"), ("log2t", "u1"), ("log2p", "u1"), ("zero
 ASSIGN_DTYPE = np.dtype([("g", "<i4"), ("c", "<i4"), ("m_bytes", "<i8"), ("plan", "<i4"), ("first_node", "<i4"),
                          ("n_nodes", "<i4"), ("thr", "<f4"), ("status", "<i4"), ("m_level", "<i4")])
 REQUEST_DTYPE = np.dtype([("g_idx", "<i4"), ("c_idx", "<i4"), ("m_idx", "<i4"), ("plan", "<i4")])
+RECONF_DTYPE = np.dtype([("T", "<f4"), ("delta", "<f4"), ("n_reconf", "<i4"), ("active", "<i4")])
 NODE_DTYPE = np.dtype([("free_g", "<i4"), ("free_c", "<i4"), ("free_m", "<i8"), ("owner", "<i4"), ("reserved", "<i4")])
 assert JOB_DTYPE.itemsize == 128 and PLAN_DTYPE.itemsize == 8
 assert ASSIGN_DTYPE.itemsize == 40 and NODE_DTYPE.itemsize == 24
@@ -63,7 +64,7 @@ def make_cluster(n_nodes, quota=None):
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
            "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_marginal_gain",
            "rubick_min_resources",
-           "rubick_greedy_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
+           "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
            "rubick_schedule_round_host"]
 
 _lib = None
@@ -97,6 +98,8 @@ def lib():
         L.rubick_marginal_gain.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp]
         L.rubick_min_resources.argtypes = [vp, vp, vp, vp, ip, vp, vp, vp, vp]
         L.rubick_greedy_round.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, vp, C.POINTER(C.c_int32)]
+        L.rubick_incremental_round.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), vp, vp, vp, C.c_float, ip, vp, vp, vp,
+                                               C.POINTER(C.c_int32)]
         L.rubick_greedy_round_noalloc.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
@@ -225,6 +228,20 @@ class Context:
         rc = self._check(lib().rubick_greedy_round(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_curve_plan),
                                                    _ptr(d_curve_g), _ptr(d_feas), C.byref(cl), int(max_steps), _ptr(d_out),
                                                    _ptr(d_node_out), _ptr(d_step_log), C.byref(steps)), allow=(ESTEPS,))
+        return steps.value, rc == ESTEPS
+
+    def incremental_round(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, n_nodes, max_steps, d_out,
+                          d_node_out=None, d_step_log=None, d_prev=None, d_prev_nodes=None, d_reconf=None, theta=0.97,
+                          quota=None):
+        """rubick_incremental_round -> (steps, capped); d_prev / d_prev_nodes: the previous round's
+        outputs (None: empty cluster); d_reconf: RECONF_DTYPE records (None: gate open)."""
+        steps = C.c_int32(0)
+        cl, _keep = make_cluster(n_nodes, quota)
+        rc = self._check(lib().rubick_incremental_round(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_curve_plan),
+                                                        _ptr(d_curve_g), _ptr(d_feas), C.byref(cl), _ptr(d_prev),
+                                                        _ptr(d_prev_nodes), _ptr(d_reconf), C.c_float(theta), int(max_steps),
+                                                        _ptr(d_out), _ptr(d_node_out), _ptr(d_step_log), C.byref(steps)),
+                         allow=(ESTEPS,))
         return steps.value, rc == ESTEPS
 
     def greedy_round_noalloc(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, n_nodes, max_steps, d_out,

@@ -338,6 +338,10 @@ static int finish_round(rubick_ctx *ctx, int32_t *h_steps)
         cudaMemset(ctx->d_status, 0, 4);
         return fail(ctx, RUBICK_ESTATE, "a feasibility word is not a threshold in the memory-level index");
     }
+    if (two[0] & DS_BAD_PREV) {
+        cudaMemset(ctx->d_status, 0, 4);
+        return fail(ctx, RUBICK_ESTATE, "incremental round: the previous allocation does not fit the grid or the cluster");
+    }
     return RUBICK_OK;
 }
 
@@ -366,6 +370,41 @@ int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
     rc = enqueue_round(ctx, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, h_cluster, max_steps, d_out,
                        d_node_out, d_step_log);
     if (rc) return rc;
+    return finish_round(ctx, h_steps);
+}
+
+int rubick_incremental_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                             const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
+                             const uint32_t *d_feas, const rubick_cluster *h_cluster,
+                             const rubick_assignment *d_prev, const rubick_node *d_prev_nodes,
+                             const rubick_reconf *d_reconf, float theta, int max_steps,
+                             rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
+                             int32_t *h_steps)
+{
+    CHECK_CTX(ctx);
+    int rc = check_round_args(ctx, J, h_cluster, max_steps);
+    if (rc) return rc;
+    if (J > 0 && (!d_jobs || !d_curve_val || !d_curve_plan || !d_curve_g || !d_feas || !d_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if ((d_prev == nullptr) != (d_prev_nodes == nullptr)) return fail(ctx, RUBICK_EINVAL, "d_prev and d_prev_nodes come together");
+    if (ctx->space.Gn > 32) return fail(ctx, RUBICK_EINVAL, "incremental round: at most 32 GPUs per node");
+    if (!(theta == theta)) return fail(ctx, RUBICK_EINVAL, "theta is not a number");
+    const int N = h_cluster->n_nodes, T = h_cluster->n_tenants;
+    if (T > 0) {
+        cudaStreamSynchronize(ctx->stream);
+        ctx->h_quota.resize(size_t(2) * T);
+        for (int t = 0; t < T; ++t) { ctx->h_quota[2 * t] = h_cluster->quota_gpus[t]; ctx->h_quota[2 * t + 1] = h_cluster->quota_cpus[t]; }
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_quota, ctx->h_quota.data(), size_t(8) * T, cudaMemcpyHostToDevice, ctx->stream), "upload quotas");
+    }
+    const size_t need = incr_scratch_need(ctx->space, J, N);
+    if (need > ctx->round_scratch_bytes) {
+        if (ctx->d_round_scratch) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_round_scratch); ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0; }
+        CUDA_TRY(ctx, cudaMalloc(&ctx->d_round_scratch, need), "cudaMalloc (round scratch)");
+        ctx->round_scratch_bytes = need;
+    }
+    CUDA_TRY(ctx, launch_round_incremental(ctx->space, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, N, max_steps,
+                                           d_prev, d_prev_nodes, d_reconf, theta, d_out, d_node_out, d_step_log,
+                                           ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream),
+             "launch incremental_round");
     return finish_round(ctx, h_steps);
 }
 

@@ -48,6 +48,7 @@ struct Space {
 enum : uint32_t {
     DS_FEAS_NOT_THRESHOLD = 1u,
     DS_STEP_CAP = 2u,
+    DS_BAD_PREV = 4u,             // incremental round: the previous state does not fit the grid or the cluster
 };
 
 bool round_fast_supported(const Space &sp, int J, int N);
@@ -105,6 +106,14 @@ cudaError_t launch_min_resources(const Space &sp, const QuadDesc *d_quads, const
                                  const float *d_cv, int J, const rubick_request *d_req, int32_t *d_gmin, int32_t *d_cmin,
                                  float *d_baseline, cudaStream_t st);
 size_t round_scratch_need(const Space &sp, int J, int N);
+size_t incr_scratch_need(const Space &sp, int J, int N);
+cudaError_t launch_round_incremental(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
+                                     const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
+                                     const rubick_assignment *d_prev, const rubick_node *d_prev_nodes,
+                                     const rubick_reconf *d_reconf, float theta, rubick_assignment *d_out,
+                                     rubick_node *d_node_out, int32_t *d_step_log, void *d_scratch,
+                                     const int32_t *d_quota, int n_tenants, uint32_t *d_status, int32_t *d_steps,
+                                     cudaStream_t st);
 cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                          rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,

@@ -77,6 +77,48 @@ class Gpu:
                             d_log.cpu().numpy()[:steps] if want_log else None)
 
 
+def pack_prev(prev, J, n_nodes):
+    """The dict a round returned -> (ASSIGN_DTYPE records, NODE_DTYPE records)."""
+    a = np.zeros(max(J, 1), dtype=rb.ASSIGN_DTYPE)
+    for k in ("g", "c", "m_bytes", "plan", "first_node", "n_nodes", "status", "m_level", "thr"):
+        a[k][:J] = np.asarray(prev[k])
+    nd = np.zeros(n_nodes, dtype=rb.NODE_DTYPE)
+    node = np.asarray(prev["node"])
+    nd["free_g"], nd["free_c"], nd["free_m"], nd["owner"] = node[:, 0], node[:, 1], node[:, 2], node[:, 3]
+    return a, nd
+
+
+def incremental_on_tables(gpu, jobs, cv, cp, cg, feas, n_nodes, prev, active=None, T=None, delta=None, nrec=None,
+                          theta=0.97, max_steps=1 << 30, quota=None):
+    """rubick_incremental_round on host-provided tables and previous state -> dict like the oracle's."""
+    t = gpu.torch
+    J = len(jobs["P"])
+    d_jobs = gpu.jobs_to_device(jobs)
+    d_cv = t.from_numpy(np.ascontiguousarray(cv, dtype=np.float32).reshape(-1)).cuda()
+    d_cp = t.from_numpy(np.ascontiguousarray(cp, dtype=np.int32).reshape(-1)).cuda()
+    d_cg = t.from_numpy(np.ascontiguousarray(cg, dtype=np.int32).reshape(-1)).cuda()
+    d_feas = t.from_numpy(np.ascontiguousarray(feas, dtype=np.uint32).view(np.int32).reshape(-1)).cuda()
+    cap = int(min(max_steps, 2 * J * (gpu.nG + gpu.nC + 2) + 1))
+    d_out = gpu.empty(max(J, 1) * rb.ASSIGN_DTYPE.itemsize, t.uint8)
+    d_node = gpu.empty(n_nodes * rb.NODE_DTYPE.itemsize, t.uint8)
+    d_log = gpu.empty(max(cap, 1), t.int32)
+    d_prev = d_prev_nodes = d_reconf = None
+    if prev is not None:
+        a, nd = pack_prev(prev, J, n_nodes)
+        d_prev, d_prev_nodes = rb.to_device(a), rb.to_device(nd)
+    if not (active is None and T is None and delta is None and nrec is None):
+        rc = np.zeros(max(J, 1), dtype=rb.RECONF_DTYPE)
+        rc["active"][:J] = 1 if active is None else np.asarray(active)
+        rc["T"][:J] = 1e9 if T is None else np.asarray(T, dtype=np.float32)
+        rc["delta"][:J] = 0 if delta is None else np.asarray(delta, dtype=np.float32)
+        rc["n_reconf"][:J] = 0 if nrec is None else np.asarray(nrec)
+        d_reconf = rb.to_device(rc)
+    steps, capped = gpu.ctx.incremental_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, n_nodes, cap, d_out, d_node, d_log,
+                                              d_prev=d_prev, d_prev_nodes=d_prev_nodes, d_reconf=d_reconf, theta=theta, quota=quota)
+    return unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE)[:J], rb.from_device(d_node, rb.NODE_DTYPE), steps, capped,
+                        d_log.cpu().numpy()[:steps])
+
+
 def unpack_round(out, node, steps, capped, log):
     return dict(g=out["g"].astype(np.int64), c=out["c"].astype(np.int64), m_bytes=out["m_bytes"].astype(np.int64),
                 plan=out["plan"].astype(np.int64), first_node=out["first_node"].astype(np.int64),

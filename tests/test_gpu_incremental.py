@@ -1,0 +1,142 @@
+"""rubick_incremental_round against the oracle's incremental round: same previous state, same tables,
+bit-exact allocations, node states and step logs (integer and single-precision work only)."""
+import numpy as np
+import pytest
+
+import oracle
+from gpu_util import Gpu, assert_rounds_equal, has_cuda, incremental_on_tables
+from helpers import GIB, env, one_job, stack_jobs
+from paper_2408_08586_b200 import binding as rb
+from paper_2408_08586_b200 import workloads
+from test_oracle_incremental import event_config, random_events
+from test_oracle_sched import concave_instance, tables
+
+pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not has_cuda(), reason="needs a CUDA device")]
+
+
+def both(gpu, cfg, tb, prev, **kw):
+    plans, feas, cv, cp, cg = tb
+    want = oracle.schedule_round_incremental(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                             cfg["m_levels"], cfg["n_nodes"], prev, want_log=True, **kw)
+    got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], prev, **kw)
+    return want, got
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_event_sequences_are_bit_exact(seed):
+    """Arrivals, completions, pinned jobs, guaranteed minima, exchanges and preemptions over eight rounds;
+    every round starts from the oracle's previous result on both sides."""
+    cfg, rng = event_config(seed)
+    tb = tables(cfg)
+    gpu = Gpu(cfg)
+    plans, feas, cv, cp, cg = tb
+    exchanges = 0
+    for inp, want in random_events(cfg, tb, 8, rng):
+        got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], inp["prev"], active=inp["active"],
+                                    T=inp["T"], delta=inp["delta"], nrec=inp["nrec"])
+        assert_rounds_equal(got, want)
+        exchanges += int((((want["log"] >> 2) & 1) & (want["log"] & 1)).sum())
+    if seed >= 2:
+        assert exchanges > 0
+
+
+def test_from_an_empty_cluster_and_with_quotas():
+    cfg = workloads.make("paper-scale")
+    J = 64
+    jobs = cfg["jobs"]
+    jobs["gmin_idx"] = np.where(np.arange(J) % 3 == 0, 1, -1)
+    jobs["cmin_idx"] = np.where(np.arange(J) % 3 == 0, 0, -1)
+    jobs["tenant"] = np.arange(J) % 2
+    tb = tables(cfg)
+    gpu = Gpu(cfg)
+    want, got = both(gpu, cfg, tb, None)
+    assert_rounds_equal(got, want)
+    quota = np.array([[6, 12], [64, 8]])
+    want_q, got_q = both(gpu, cfg, tb, None, quota=quota)
+    assert_rounds_equal(got_q, want_q)
+    assert (want_q["status"] == 2).any()
+    # second round on the first one's result: queued guaranteed jobs push in by exchange once the quota is lifted
+    want2, got2 = both(gpu, cfg, tb, want_q)
+    assert_rounds_equal(got2, want2)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_concave_exchanges_are_bit_exact(seed):
+    jobs, cv, cp, cg, feas = concave_instance(seed)
+    gl, cl, ml = np.arange(1, 9), np.array([4]), np.array([GIB])
+    cfg = dict(jobs=jobs, env=env(cpus_per_node=64), g_levels=gl, c_levels=cl, m_levels=ml, n_nodes=1)
+    plans, _ = rb.enumerate_plans(gl)
+    gpu = Gpu(cfg, plans=plans)
+    J = 4
+    hog = seed % J
+    prev = dict(g=np.zeros(J, np.int64), c=np.zeros(J, np.int64), m_bytes=np.zeros(J, np.int64), plan=np.full(J, -1),
+                first_node=np.full(J, -1), n_nodes=np.zeros(J, np.int64), status=np.zeros(J, np.int64),
+                m_level=np.full(J, -1), thr=np.zeros(J, np.float32), node=np.array([[0, 60, 0, -1]]))
+    prev["g"][hog], prev["c"][hog], prev["m_bytes"][hog], prev["plan"][hog] = 8, 4, GIB, 0
+    prev["first_node"][hog], prev["n_nodes"][hog], prev["status"][hog], prev["m_level"][hog] = 0, 1, 1, 0
+    prev["thr"][hog] = cv[hog, 7, 0, 0]
+    feas_full = np.zeros((J, gpu.P), dtype=np.uint32)
+    feas_full[:, 0] = 1
+    tb = (None, feas_full, cv, cp, cg)
+    want, got = both(gpu, cfg, tb, prev)
+    assert_rounds_equal(got, want)
+    assert ((want["log"] >> 2) & 1).all() and (want["log"] & 1).any()
+
+
+def test_multi_node_jobs_are_carried_over_and_never_shrunk():
+    cfg = workloads.make("cluster-512", J=96, n_nodes=24)
+    tb = tables(cfg, nthreads=8)
+    gpu = Gpu(cfg)
+    want, got = both(gpu, cfg, tb, None)
+    assert_rounds_equal(got, want)
+    assert (want["n_nodes"] > 1).any()
+    J = 96
+    rng = np.random.default_rng(5)
+    active = (rng.uniform(size=J) < 0.8).astype(np.int32)
+    prev = {k: (v.copy() if hasattr(v, "copy") else v) for k, v in want.items()}
+    prev["status"] = np.where(active == 1, prev["status"], 0)
+    T = rng.uniform(0.0, 4000.0, J).astype(np.float32)
+    delta = rng.uniform(5.0, 60.0, J).astype(np.float32)
+    want2, got2 = both(gpu, cfg, tb, prev, active=active, T=T, delta=delta, nrec=rng.integers(0, 3, J))
+    assert_rounds_equal(got2, want2)
+    multi = (prev["n_nodes"] > 1) & (prev["status"] == 1)
+    assert (want2["g"][multi] >= prev["g"][multi]).all()
+
+
+def test_inconsistent_previous_state_is_refused():
+    cfg = workloads.make("tiny")
+    tb = tables(cfg)
+    gpu = Gpu(cfg)
+    want, got = both(gpu, cfg, tb, None)
+    assert_rounds_equal(got, want)
+    bad = {k: (v.copy() if hasattr(v, "copy") else v) for k, v in want.items()}
+    j = int(np.nonzero(want["status"] == 1)[0][0])
+    bad["g"][j] = 1000
+    plans, feas, cv, cp, cg = tb
+    assert oracle.schedule_round_incremental(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                             cfg["m_levels"], cfg["n_nodes"], bad)["steps"] is None
+    with pytest.raises(rb.RubickError) as ei:
+        incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], bad)
+    assert ei.value.code == rb.ESTATE
+    # the context stays usable
+    again = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], want)
+    want2 = oracle.schedule_round_incremental(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                              cfg["m_levels"], cfg["n_nodes"], want, want_log=True)
+    assert_rounds_equal(again, want2)
+
+
+def test_step_cap_and_argument_validation():
+    cfg = workloads.make("paper-scale", J=32, n_nodes=2)
+    tb = tables(cfg)
+    gpu = Gpu(cfg)
+    want, got = both(gpu, cfg, tb, None, max_steps=5)
+    assert want["capped"] and got["capped"]
+    assert_rounds_equal(got, want)
+    t = gpu.torch
+    d = gpu.empty(64, t.uint8)
+    cl, _ = rb.make_cluster(2)
+    import ctypes as C
+    steps = C.c_int32(0)
+    rc = rb.lib().rubick_incremental_round(gpu.ctx._h, rb._ptr(d), 1, rb._ptr(d), rb._ptr(d), rb._ptr(d), rb._ptr(d), C.byref(cl),
+                                           rb._ptr(d), None, None, C.c_float(0.97), 10, rb._ptr(d), None, None, C.byref(steps))
+    assert rc == rb.EINVAL                       # previous assignments without the previous node states
