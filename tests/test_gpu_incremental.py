@@ -40,6 +40,64 @@ def test_event_sequences_are_bit_exact(seed):
         assert exchanges > 0
 
 
+@pytest.mark.parametrize("name,J,N,rounds", [("cluster-512", 320, 20, 6), ("paper-scale", 64, 2, 10)])
+def test_larger_event_sequences_with_quotas_are_bit_exact(name, J, N, rounds):
+    cfg, rng = event_config(11, name=name, J=J, n_nodes=N)
+    cfg["jobs"]["tenant"] = rng.integers(0, 3, J)
+    quota = np.array([[N * 3, N * 40], [N * 2, N * 30], [N, N * 10]])
+    tb = tables(cfg, nthreads=8)
+    gpu = Gpu(cfg)
+    plans, feas, cv, cp, cg = tb
+    active = np.zeros(J, dtype=np.int32)
+    prev = None
+    T = np.zeros(J, dtype=np.float32)
+    nrec = rng.integers(0, 2, J).astype(np.int32)
+    delta = rng.uniform(5.0, 60.0, J).astype(np.float32)
+    seen_exchange = seen_pending = False
+    for rnd in range(rounds):
+        arrive = rng.uniform(size=J) < (0.08 if rnd == 0 else 0.2)
+        leave = (rng.uniform(size=J) < 0.1) & (active == 1)
+        active = np.where(leave, 0, np.where(arrive, 1, active)).astype(np.int32)
+        if prev is not None:
+            T = np.where((prev["status"] == 1) & (active == 1), T + rng.uniform(100.0, 5000.0, J), 0).astype(np.float32)
+        kw = dict(active=active, T=T, delta=delta, nrec=nrec, quota=quota)
+        want = oracle.schedule_round_incremental(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                                 cfg["m_levels"], N, prev, want_log=True, **kw)
+        got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, N, prev, **kw)
+        assert want["steps"] is not None
+        assert_rounds_equal(got, want)
+        seen_exchange |= bool((((want["log"] >> 2) & 1) & (want["log"] & 1)).any())
+        seen_pending |= bool((want["status"] == 2).any())
+        prev = want
+    assert seen_exchange
+
+
+def test_small_nodes_and_few_levels_are_bit_exact():
+    """4-GPU nodes, three core levels, two memory levels: other list lengths, more preemptions."""
+    cfg = workloads.make("paper-scale", J=48, n_nodes=5)
+    cfg["env"] = env(gpus_per_node=4, cpus_per_node=24, mem_per_node_bytes=256 * GIB)
+    cfg["g_levels"] = np.array([1, 2, 4, 8, 16])
+    cfg["c_levels"] = np.array([2, 6, 12])
+    cfg["m_levels"] = np.array([64, 192]) * GIB
+    rng = np.random.default_rng(77)
+    cfg["jobs"]["gmin_idx"] = np.where(rng.uniform(size=48) < 0.3, rng.integers(0, 2, 48), -1)
+    cfg["jobs"]["cmin_idx"] = np.where(cfg["jobs"]["gmin_idx"] >= 0, 0, -1)
+    tb = tables(cfg, nthreads=8)
+    gpu = Gpu(cfg)
+    plans, feas, cv, cp, cg = tb
+    prev = None
+    active = np.zeros(48, dtype=np.int32)
+    for rnd in range(8):
+        active = np.where(rng.uniform(size=48) < 0.12, 0, np.where(rng.uniform(size=48) < 0.3, 1, active)).astype(np.int32)
+        T = rng.uniform(0.0, 3000.0, 48).astype(np.float32)
+        kw = dict(active=active, T=T, delta=np.full(48, 20.0, np.float32), nrec=rng.integers(0, 3, 48))
+        want = oracle.schedule_round_incremental(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                                 cfg["m_levels"], 5, prev, want_log=True, **kw)
+        got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, 5, prev, **kw)
+        assert_rounds_equal(got, want)
+        prev = want
+
+
 def test_from_an_empty_cluster_and_with_quotas():
     cfg = workloads.make("paper-scale")
     J = 64

@@ -171,11 +171,11 @@ def random_events(cfg, tb, rounds, rng):
         prev = r
 
 
-def event_config(seed):
-    cfg = workloads.make("paper-scale", J=40, n_nodes=3)
+def event_config(seed, name="paper-scale", J=40, n_nodes=3):
+    cfg = workloads.make(name, J=J, n_nodes=n_nodes)
     rng = np.random.default_rng(40 + seed)
-    cfg["jobs"]["gmin_idx"] = np.where(rng.uniform(size=40) < 0.4, rng.integers(0, 3, 40), -1)
-    cfg["jobs"]["cmin_idx"] = np.where(cfg["jobs"]["gmin_idx"] >= 0, rng.integers(0, 2, 40), -1)
+    cfg["jobs"]["gmin_idx"] = np.where(rng.uniform(size=J) < 0.4, rng.integers(0, 3, J), -1)
+    cfg["jobs"]["cmin_idx"] = np.where(cfg["jobs"]["gmin_idx"] >= 0, rng.integers(0, 2, J), -1)
     return cfg, rng
 
 
