@@ -339,6 +339,19 @@ def main():
                   "round_latency_ms_p99": float(np.percentile(r["latency_ms"], 99)),
                   "steps_per_round_mean": float(r["steps"].mean()),
                   "what": "rubick_schedule_round_host per event: host job records in, table + curves + round on the GPU, assignments out"}
+        # the same stream through the incremental round (previous allocation and tables kept on the device)
+        ev_mod.run_events_incremental(ectx, ecfg, n_events=5)
+        ri = ev_mod.run_events_incremental(ectx, ecfg, n_events=args.events)
+        inc_lat = ri["latency_ms"][1:] if len(ri["latency_ms"]) > 1 else ri["latency_ms"]      # event 0 builds every table
+        events["incremental"] = {
+            "events": int(len(ri["latency_ms"])), "slots": 4096,
+            "first_event_ms": float(ri["latency_ms"][0]),
+            "round_latency_ms_p50": float(np.percentile(inc_lat, 50)),
+            "round_latency_ms_p99": float(np.percentile(inc_lat, 99)),
+            "steps_per_round_mean": float(ri["steps"][1:].mean()) if len(ri["steps"]) > 1 else float(ri["steps"].mean()),
+            "reconfigured_per_round_mean": float(ri["reconfigured"][1:].mean()) if len(ri["reconfigured"]) > 1 else 0.0,
+            "what": "rubick_incremental_event_host per event: changed slot and gate inputs in, tables of that slot + incremental round "
+                    "(shrink / exchange step, reconfiguration gate at 0.97) on the GPU, assignments out"}
         ectx.close()
 
     if rank != 0:

@@ -274,6 +274,20 @@ int rubick_incremental_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
                              rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                              int32_t *h_steps);
 
+/* One scheduling event with state kept in the context: the incremental round on J job slots whose
+ * previous allocation, node states and curve tables stay on the device between calls (Section 5.2:
+ * curves are "cached for reuse").  h_jobs: all J records (host); only the slots listed in
+ * h_changed[0..n_changed) are uploaded and have their tables recomputed (a new arrival, a refitted
+ * model); n_changed < 0: all of them.  h_reconf: J gate / activity records (NULL: all active, gate
+ * open); clear `active` of a finished job's slot.  The first call, a call with another J or node
+ * count, a call after rubick_set_space or rubick_schedule_round*, or restart != 0 starts from an
+ * empty cluster with all tables recomputed.  Outputs (host): J assignments, optionally n_nodes
+ * node states and the step count.  Errors as rubick_incremental_round. */
+int rubick_incremental_event_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J, const rubick_cluster *h_cluster,
+                                  const int32_t *h_changed, int n_changed, const rubick_reconf *h_reconf, float theta,
+                                  int restart, int max_steps, rubick_assignment *h_out, rubick_node *h_node_out,
+                                  int32_t *h_steps);
+
 /* rubick_greedy_round for callers that cannot allocate device memory when they schedule: a
  * daemon that received a fixed device-memory budget at start-up and shares the GPU with jobs
  * that fill the rest (a late cudaMalloc may fail, and stalls the device while it runs), or a

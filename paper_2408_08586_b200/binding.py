@@ -65,7 +65,7 @@ EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error"
            "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_marginal_gain",
            "rubick_min_resources",
            "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
-           "rubick_schedule_round_host"]
+           "rubick_schedule_round_host", "rubick_incremental_event_host"]
 
 _lib = None
 
@@ -103,6 +103,8 @@ def lib():
         L.rubick_greedy_round_noalloc.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_schedule_round_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
+        L.rubick_incremental_event_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), vp, ip, vp, C.c_float, ip, ip, vp, vp,
+                                                    C.POINTER(C.c_int32)]
         for name in EXPORTS:
             if name not in ("rubick_destroy", "rubick_last_error"):
                 getattr(L, name).restype = ip
@@ -270,4 +272,21 @@ class Context:
         cl, _keep = make_cluster(n_nodes, quota)
         rc = self._check(lib().rubick_schedule_round_host(self._h, _ptr(h_jobs), int(J), C.byref(cl), int(max_steps),
                                                           _ptr(h_out), _ptr(h_node_out), C.byref(steps)), allow=(ESTEPS,))
+        return steps.value, rc == ESTEPS
+
+    def incremental_event_host(self, h_jobs, J, n_nodes, h_out, changed=None, h_reconf=None, theta=0.97, restart=False,
+                               max_steps=1 << 30, h_node_out=None, quota=None):
+        """rubick_incremental_event_host -> (steps, capped).  changed: slot indices whose records are new
+        (None: all); h_reconf: RECONF_DTYPE array (None: all active, gate open)."""
+        steps = C.c_int32(0)
+        cl, _keep = make_cluster(n_nodes, quota)
+        if changed is None:
+            ch, n_ch = None, -1
+        else:
+            ch = np.ascontiguousarray(changed, dtype=np.int32)
+            n_ch = len(ch)
+        rc = self._check(lib().rubick_incremental_event_host(self._h, _ptr(h_jobs), int(J), C.byref(cl), _ptr(ch) if n_ch > 0 else None,
+                                                             n_ch, _ptr(h_reconf), C.c_float(theta), int(bool(restart)),
+                                                             int(min(max_steps, 0x7fffffff)), _ptr(h_out), _ptr(h_node_out),
+                                                             C.byref(steps)), allow=(ESTEPS,))
         return steps.value, rc == ESTEPS

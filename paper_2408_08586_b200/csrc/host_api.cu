@@ -72,6 +72,9 @@ int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *c
     ctx->d_out_stage = nullptr; ctx->cap_out = 0;
     ctx->d_node_stage = nullptr; ctx->cap_node = 0;
     ctx->d_best_todo = nullptr; ctx->cap_best_todo = 0;
+    ctx->inc_J = 0; ctx->inc_N = 0; ctx->inc_cur = 0;
+    for (int i = 0; i < 2; ++i) { ctx->d_inc_state[i] = nullptr; ctx->d_inc_nodes[i] = nullptr; ctx->cap_inc_state[i] = 0; ctx->cap_inc_nodes[i] = 0; }
+    ctx->d_inc_reconf = nullptr; ctx->cap_inc_reconf = 0; ctx->d_inc_jobs = nullptr; ctx->cap_inc_jobs = 0;
     ctx->tile_jobs = 2048;            // 0.5 GB table tile at 2,640 plans x 24 core levels
     cudaDeviceProp prop;
     if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) { delete ctx; return RUBICK_ECUDA; }
@@ -93,6 +96,8 @@ void rubick_destroy(rubick_ctx *ctx)
     cudaFree(ctx->d_thr); cudaFree(ctx->d_feas); cudaFree(ctx->d_cv); cudaFree(ctx->d_cp); cudaFree(ctx->d_cg);
     cudaFree(ctx->d_jobs_stage); cudaFree(ctx->d_out_stage); cudaFree(ctx->d_node_stage);
     cudaFree(ctx->d_best_todo);
+    for (int i = 0; i < 2; ++i) { cudaFree(ctx->d_inc_state[i]); cudaFree(ctx->d_inc_nodes[i]); }
+    cudaFree(ctx->d_inc_reconf); cudaFree(ctx->d_inc_jobs);
     delete ctx;
 }
 
@@ -217,6 +222,7 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
     CUDA_TRY(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->d_quads), quads.size() * sizeof(QuadDesc)), "cudaMalloc (plan table)");
     CUDA_TRY(ctx, cudaMemcpy(ctx->d_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice), "upload plan table");
     ctx->space = sp;
+    ctx->inc_J = 0;
     ctx->plans.assign(h_plans, h_plans + P);
     ctx->has_space = true;
     return RUBICK_OK;
@@ -413,6 +419,7 @@ int rubick_incremental_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
 static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
 {
     const Space &sp = ctx->space;
+    ctx->inc_J = 0;                     // the table scratch is about to be rewritten
     const int tile = ctx->tile_jobs < J ? ctx->tile_jobs : J;
     int rc;
     if ((rc = ensure(ctx, ctx->d_thr, ctx->cap_thr, size_t(tile) * sp.nC * sp.P))) return rc;
@@ -469,6 +476,85 @@ int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J,
     if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_out_stage, size_t(J) * sizeof(rubick_assignment), cudaMemcpyDeviceToHost, ctx->stream), "copy assignments to host");
     if (h_node_out) CUDA_TRY(ctx, cudaMemcpyAsync(h_node_out, ctx->d_node_stage, size_t(N) * sizeof(rubick_node), cudaMemcpyDeviceToHost, ctx->stream), "copy node states to host");
     return finish_round(ctx, h_steps);
+}
+
+// tables of the listed slots only (the others keep what an earlier call computed)
+static int enqueue_tables_of(rubick_ctx *ctx, const rubick_job *d_jobs, const int32_t *h_slots, int n)
+{
+    const Space &sp = ctx->space;
+    const size_t per_job = size_t(sp.nG) * sp.nC * sp.nM;
+    for (int i = 0; i < n;) {
+        int run = 1;                    // consecutive slots go through the kernels together
+        while (i + run < n && h_slots[i + run] == h_slots[i] + run && run < ctx->tile_jobs) ++run;
+        const int s0 = h_slots[i];
+        CUDA_TRY(ctx, launch_eval(sp, ctx->d_quads, d_jobs + s0, run, ctx->d_thr, ctx->d_feas + size_t(s0) * sp.P, ctx->stream), "launch eval_candidates");
+        CUDA_TRY(ctx, launch_best(sp, ctx->d_thr, ctx->d_feas + size_t(s0) * sp.P, run, 0u, ctx->d_cv + s0 * per_job,
+                                  ctx->d_cp + s0 * per_job, ctx->d_cg + s0 * per_job, ctx->d_status, ctx->d_best_todo,
+                                  ctx->num_sms, ctx->stream),
+                 "launch best_plan");
+        i += run;
+    }
+    return RUBICK_OK;
+}
+
+int rubick_incremental_event_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J, const rubick_cluster *h_cluster,
+                                  const int32_t *h_changed, int n_changed, const rubick_reconf *h_reconf, float theta,
+                                  int restart, int max_steps, rubick_assignment *h_out, rubick_node *h_node_out,
+                                  int32_t *h_steps)
+{
+    CHECK_CTX(ctx);
+    int rc = check_round_args(ctx, J, h_cluster, max_steps);
+    if (rc) return rc;
+    if (J < 1 || !h_jobs || !h_out) return fail(ctx, RUBICK_EINVAL, "null pointer or no job slots");
+    if (n_changed > 0 && !h_changed) return fail(ctx, RUBICK_EINVAL, "n_changed > 0 without the slot list");
+    if (ctx->space.Gn > 32) return fail(ctx, RUBICK_EINVAL, "incremental round: at most 32 GPUs per node");
+    if (!(theta == theta)) return fail(ctx, RUBICK_EINVAL, "theta is not a number");
+    const int N = h_cluster->n_nodes, T = h_cluster->n_tenants;
+    const bool fresh = restart || ctx->inc_J != J || ctx->inc_N != N;
+    if (!fresh)
+        for (int i = 0; i < n_changed; ++i)
+            if (h_changed[i] < 0 || h_changed[i] >= J) return fail(ctx, RUBICK_EINVAL, "changed slot out of range");
+    for (int i = 0; i < 2; ++i) {
+        if ((rc = ensure(ctx, ctx->d_inc_state[i], ctx->cap_inc_state[i], size_t(J)))) return rc;
+        if ((rc = ensure(ctx, ctx->d_inc_nodes[i], ctx->cap_inc_nodes[i], size_t(N)))) return rc;
+    }
+    if ((rc = ensure(ctx, ctx->d_inc_jobs, ctx->cap_inc_jobs, size_t(J)))) return rc;
+    if ((rc = ensure(ctx, ctx->d_inc_reconf, ctx->cap_inc_reconf, size_t(J)))) return rc;
+    const bool all = fresh || n_changed < 0;
+    if (all) {
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_inc_jobs, h_jobs, size_t(J) * sizeof(rubick_job), cudaMemcpyHostToDevice, ctx->stream), "copy jobs to device");
+        if ((rc = enqueue_tables(ctx, ctx->d_inc_jobs, J))) return rc;
+    } else {
+        for (int i = 0; i < n_changed; ++i)
+            CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_inc_jobs + h_changed[i], h_jobs + h_changed[i], sizeof(rubick_job), cudaMemcpyHostToDevice, ctx->stream), "copy a job to device");
+        if ((rc = ensure(ctx, ctx->d_best_todo, ctx->cap_best_todo, size_t(ctx->tile_jobs) + 1))) return rc;
+        if ((rc = enqueue_tables_of(ctx, ctx->d_inc_jobs, h_changed, n_changed))) return rc;
+    }
+    if (h_reconf) CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_inc_reconf, h_reconf, size_t(J) * sizeof(rubick_reconf), cudaMemcpyHostToDevice, ctx->stream), "copy gate inputs to device");
+    if (T > 0) {
+        cudaStreamSynchronize(ctx->stream);
+        ctx->h_quota.resize(size_t(2) * T);
+        for (int t = 0; t < T; ++t) { ctx->h_quota[2 * t] = h_cluster->quota_gpus[t]; ctx->h_quota[2 * t + 1] = h_cluster->quota_cpus[t]; }
+        CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_quota, ctx->h_quota.data(), size_t(8) * T, cudaMemcpyHostToDevice, ctx->stream), "upload quotas");
+    }
+    const size_t need = incr_scratch_need(ctx->space, J, N);
+    if (need > ctx->round_scratch_bytes) {
+        if (ctx->d_round_scratch) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_round_scratch); ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0; }
+        CUDA_TRY(ctx, cudaMalloc(&ctx->d_round_scratch, need), "cudaMalloc (round scratch)");
+        ctx->round_scratch_bytes = need;
+    }
+    const int cur = ctx->inc_cur, nxt = 1 - cur;
+    CUDA_TRY(ctx, launch_round_incremental(ctx->space, ctx->d_inc_jobs, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, N, max_steps,
+                                           fresh ? nullptr : ctx->d_inc_state[cur], fresh ? nullptr : ctx->d_inc_nodes[cur],
+                                           h_reconf ? ctx->d_inc_reconf : nullptr, theta, ctx->d_inc_state[nxt], ctx->d_inc_nodes[nxt],
+                                           nullptr, ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream),
+             "launch incremental_round");
+    CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_inc_state[nxt], size_t(J) * sizeof(rubick_assignment), cudaMemcpyDeviceToHost, ctx->stream), "copy assignments to host");
+    if (h_node_out) CUDA_TRY(ctx, cudaMemcpyAsync(h_node_out, ctx->d_inc_nodes[nxt], size_t(N) * sizeof(rubick_node), cudaMemcpyDeviceToHost, ctx->stream), "copy node states to host");
+    rc = finish_round(ctx, h_steps);
+    if (rc == RUBICK_OK || rc == RUBICK_ESTEPS) { ctx->inc_cur = nxt; ctx->inc_J = J; ctx->inc_N = N; }
+    else ctx->inc_J = 0;
+    return rc;
 }
 
 }  // extern "C"

@@ -115,10 +115,15 @@ __device__ bool take_on_node(const Space &sp, const float *__restrict__ cv, cons
 
 struct IncrShared {
     unsigned long long red[4][ROUND_WARPS];
+    float redf[2][ROUND_WARPS];
+    int redi[3][ROUND_WARPS];
     int n_empty;
-    int sel_j;
+    int sel_j, which;         // the step's job and kind: 0 / 1 GPU / CPU increment on free resources, 2 / 3 by exchange
     int steps, capped;
-    int bad;
+    int changed;              // the last step changed the cluster: the first-fit table is stale
+    int batch;                // this iteration sorts out hopeless exchange candidates in bulk
+    float min_slope[2];       // lowest offered slope over all nodes, GPUs / cores
+    int max_free[2];          // most free GPUs / cores on any node
 };
 
 struct NodeLists {            // single-node jobs of every node
@@ -152,6 +157,40 @@ __device__ bool node_could_serve(const Space &sp, const Cluster &cl, const NodeL
     mov_g = __reduce_add_sync(0xffffffffu, mov_g) + cl.free_g[n];
     mov_c = __reduce_add_sync(0xffffffffu, mov_c) + cl.free_c[n];
     return mov_g >= g2 && mov_c >= c2;
+}
+
+// Lowest slope the single-node jobs of node n offer for GPUs and for cores (+inf when nobody offers).
+// An exchange that has to reclaim a resource on n fails at its first step unless the candidate's gain
+// exceeds this.  Warp-wide.
+__device__ void node_min_slopes(const Space &sp, const Cluster &cl, const NodeLists &nl, const float *__restrict__ cv,
+                                const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
+                                const uint32_t *__restrict__ feas, const HotA *hotA, const HotB *hotB, const uint32_t *roles,
+                                int n, int lane, float &ms_g, float &ms_c)
+{
+    const float inf = __int_as_float(0x7f800000);
+    float s[2] = {inf, inf};
+    if (lane < nl.cnt[n]) {
+        const int v = nl.jobs[size_t(n) * nl.Gn + lane];
+        const uint32_t vr = roles[v];
+        if (!rl_pinned(vr)) {
+            JobRegs vs; vs.a = hotA[v]; vs.b = hotB[v];
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                Offer of = shrink_offer(sp, cv, cp, cg, v, vs, vr, r);
+                if (of.ok && of.gi2 >= 0) {
+                    JobRegs t = vs; NodeFree tf; tf.g = cl.free_g[n]; tf.c = cl.free_c[n]; tf.m = cl.free_m[n];
+                    of.ok = take_on_node(sp, cv, cp, cg, feas, v, t, tf, n, true, of.gi2, of.ci2, false);
+                }
+                if (of.ok) s[r] = of.slope;
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 16; k > 0; k >>= 1) {
+        s[0] = fminf(s[0], __shfl_xor_sync(0xffffffffu, s[0], k));
+        s[1] = fminf(s[1], __shfl_xor_sync(0xffffffffu, s[1], k));
+    }
+    ms_g = s[0]; ms_c = s[1];
 }
 
 // Exchange attempt of job j for (gi2, ci2) on node n; warp 0, all lanes.  cand[r] = j's gain per unit
@@ -269,7 +308,8 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
     __shared__ IncrShared sh;
     __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];
 
-    // shared layout: free_m [N] i64 | free_g [N] | free_c [N] | owner [N] | list counts [N] | ff [n_small * nC]
+    // shared layout: free_m [N] i64 | free_g [N] | free_c [N] | owner [N] | list counts [N] | ff [n_small * nC] |
+    // min slopes [2][N] | dirty [N]
     Cluster cl;
     cl.N = N;
     cl.free_m = reinterpret_cast<int64_t *>(smem_raw);
@@ -282,6 +322,9 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
     nl.Gn = sp.Gn;
     cl.ff = nl.cnt + N;
     const int n_ff = sp.n_small * sp.nC;
+    float *ms_g = reinterpret_cast<float *>(cl.ff + n_ff);      // [N] lowest offered GPU slope on the node
+    float *ms_c = ms_g + N;                                     // [N] same for cores
+    int32_t *dirty = reinterpret_cast<int32_t *>(ms_c + N);     // [N] the node changed since its slopes were worked out
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int mt = sp.nM - 1;
@@ -291,7 +334,7 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
         cl.free_g[n] = sp.Gn; cl.free_c[n] = sp.Cn; cl.free_m[n] = sp.Mn; cl.owner[n] = -1; nl.cnt[n] = 0;
     }
     for (int j = tid; j < J; j += ROUND_THREADS) own_count[j] = 0;
-    if (tid == 0) { sh.steps = 0; sh.capped = 0; sh.n_empty = N; sh.bad = 0; }
+    if (tid == 0) { sh.steps = 0; sh.capped = 0; sh.n_empty = N; sh.changed = 1; sh.batch = 0; }
     for (int i = tid; i < 2 * n_tenants; i += ROUND_THREADS) rem_q[i] = quota[i];
     __syncthreads();
 
@@ -445,19 +488,27 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
     __syncthreads();
 
     // ---- Phase B ---------------------------------------------------------------------------------------------
+    for (int n = tid; n < N; n += ROUND_THREADS) dirty[n] = 1;
+    const float inf = __int_as_float(0x7f800000);
+    // With a step log every attempt is taken one at a time.  Without one, candidates whose exchange cannot
+    // get past its first step are frozen in bulk (same allocation, same step count).
+    const bool bulk = step_log == nullptr;
+    __syncthreads();
     for (;;) {
-        for (int e = warp; e <= n_ff; e += ROUND_WARPS) {
-            if (e == n_ff) {
-                int cnt = 0;
-                for (int nb = 0; nb < N; nb += 32) {
-                    const int n = nb + lane;
-                    cnt += __popc(__ballot_sync(0xffffffffu, n < N && cl.free_g[n] == sp.Gn));
+        if (sh.changed) {
+            for (int e = warp; e <= n_ff; e += ROUND_WARPS) {
+                if (e == n_ff) {
+                    int cnt = 0;
+                    for (int nb = 0; nb < N; nb += 32) {
+                        const int n = nb + lane;
+                        cnt += __popc(__ballot_sync(0xffffffffu, n < N && cl.free_g[n] == sp.Gn));
+                    }
+                    if (lane == 0) sh.n_empty = cnt;
+                } else {
+                    const int gi = e / sp.nC, ci = e - gi * sp.nC;
+                    const int n = first_fit_warp(cl, sp.g_levels[gi], sp.c_levels[ci], lane);
+                    if (lane == 0) cl.ff[e] = n;
                 }
-                if (lane == 0) sh.n_empty = cnt;
-            } else {
-                const int gi = e / sp.nC, ci = e - gi * sp.nC;
-                const int n = first_fit_warp(cl, sp.g_levels[gi], sp.c_levels[ci], lane);
-                if (lane == 0) cl.ff[e] = n;
             }
         }
         __syncthreads();
@@ -502,9 +553,139 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
             }
             int which = -1;
             for (int q = 0; q < 4 && which < 0; ++q) if (b4[q]) which = q;
-            int sel_j = which >= 0 ? int(0xffffffffu - uint32_t(b4[which])) : -1;
-            if (sel_j >= 0 && sh.steps >= max_steps) { if (lane == 0) sh.capped = 1; sel_j = -1; }
+            if (lane == 0) {
+                sh.which = which;
+                sh.sel_j = which >= 0 ? int(0xffffffffu - uint32_t(b4[which])) : -1;
+                sh.batch = bulk && which >= 2;
+            }
+        }
+        __syncthreads();
 
+        if (sh.batch) {
+            // (a) lowest offered slopes of the nodes that changed
+            for (int n = warp; n < N; n += ROUND_WARPS)
+                if (dirty[n]) {
+                    float g0, c0;
+                    node_min_slopes(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, n, lane, g0, c0);
+                    if (lane == 0) { ms_g[n] = g0; ms_c[n] = c0; dirty[n] = 0; }
+                }
+            __syncthreads();
+            // (b) over all nodes: lowest slopes, most free GPUs / cores
+            {
+                float lg = inf, lc = inf; int fg = 0, fc = 0;
+                for (int n = tid; n < N; n += ROUND_THREADS) {
+                    lg = fminf(lg, ms_g[n]); lc = fminf(lc, ms_c[n]);
+                    fg = max(fg, cl.free_g[n]); fc = max(fc, cl.free_c[n]);
+                }
+#pragma unroll
+                for (int k = 16; k > 0; k >>= 1) {
+                    lg = fminf(lg, __shfl_xor_sync(0xffffffffu, lg, k)); lc = fminf(lc, __shfl_xor_sync(0xffffffffu, lc, k));
+                    fg = max(fg, __shfl_xor_sync(0xffffffffu, fg, k)); fc = max(fc, __shfl_xor_sync(0xffffffffu, fc, k));
+                }
+                if (lane == 0) { sh.redf[0][warp] = lg; sh.redf[1][warp] = lc; sh.redi[0][warp] = fg; sh.redi[1][warp] = fc; }
+                __syncthreads();
+                if (warp == 0) {
+                    lg = sh.redf[0][lane]; lc = sh.redf[1][lane]; fg = sh.redi[0][lane]; fc = sh.redi[1][lane];
+#pragma unroll
+                    for (int k = 16; k > 0; k >>= 1) {
+                        lg = fminf(lg, __shfl_xor_sync(0xffffffffu, lg, k)); lc = fminf(lc, __shfl_xor_sync(0xffffffffu, lc, k));
+                        fg = max(fg, __shfl_xor_sync(0xffffffffu, fg, k)); fc = max(fc, __shfl_xor_sync(0xffffffffu, fc, k));
+                    }
+                    if (lane == 0) { sh.min_slope[0] = lg; sh.min_slope[1] = lc; sh.max_free[0] = fg; sh.max_free[1] = fc; }
+                }
+                __syncthreads();
+            }
+            // (c) a candidate is hopeless when its exchange is sure to fail at the first step: no node (its own
+            // node, for a running job) offers the resource below its gain.  Best candidate that is not hopeless:
+            const float all_g = sh.min_slope[0], all_c = sh.min_slope[1];
+            const int most_g = sh.max_free[0], most_c = sh.max_free[1];
+            auto hopeless = [&](int j, const HotA &a, int type) -> bool {
+                const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                const int gi2 = type == 0 ? pk_next_gi(a.packed) : gi;
+                if (sp.g_levels[gi2] > sp.Gn) return true;              // increments above one node never exchange
+                if (gi >= 0) {
+                    if (sp.g_levels[gi] > sp.Gn) return true;
+                    return type == 0 ? !(a.gain_g > ms_g[a.node]) : !(a.gain_c > ms_c[a.node]);
+                }
+                if (most_g < sp.g_levels[gi2] && !(a.gain_g > all_g)) return true;
+                if (most_c < sp.c_levels[ci]) {
+                    const float v2 = cv[curve_idx(sp, j, gi2, ci, mt)];
+                    const float cand_c = __fdiv_rn(__fsub_rn(__fmul_rn(hotB[j].w, v2), 0.0f), float(sp.c_levels[ci]));
+                    if (!(cand_c > all_c)) return true;
+                }
+                return false;
+            };
+            unsigned long long live[2] = {0ull, 0ull};
+            for (int j = tid; j < J; j += ROUND_THREADS) {
+                const HotA a = hotA[j];
+                const unsigned long long kg = (static_cast<unsigned long long>(__float_as_uint(a.gain_g)) << 32) | (0xffffffffu - uint32_t(j));
+                const unsigned long long kc = (static_cast<unsigned long long>(__float_as_uint(a.gain_c)) << 32) | (0xffffffffu - uint32_t(j));
+                if (a.gain_g > 0.0f && kg > live[0] && !hopeless(j, a, 0)) live[0] = kg;
+                if (a.gain_c > 0.0f && kc > live[1] && !hopeless(j, a, 1)) live[1] = kc;
+            }
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+#pragma unroll
+                for (int k = 16; k > 0; k >>= 1) {
+                    const unsigned long long o = __shfl_xor_sync(0xffffffffu, live[q], k);
+                    live[q] = o > live[q] ? o : live[q];
+                }
+                if (lane == 0) sh.red[q][warp] = live[q];
+            }
+            __syncthreads();
+            unsigned long long lv[2];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+                lv[q] = sh.red[q][lane];
+#pragma unroll
+                for (int k = 16; k > 0; k >>= 1) {
+                    const unsigned long long o = __shfl_xor_sync(0xffffffffu, lv[q], k);
+                    lv[q] = o > lv[q] ? o : lv[q];
+                }
+            }
+            __syncthreads();
+            // (d) hopeless candidates that come before it (GPU increments before CPU increments, larger key first)
+            // would each be tried, fail and be frozen: count them, freeze them
+            const int live_type = lv[0] ? 0 : (lv[1] ? 1 : 2);
+            int mine = 0;
+            for (int j = tid; j < J; j += ROUND_THREADS) {
+                HotA a = hotA[j];
+                const unsigned long long kg = (static_cast<unsigned long long>(__float_as_uint(a.gain_g)) << 32) | (0xffffffffu - uint32_t(j));
+                const unsigned long long kc = (static_cast<unsigned long long>(__float_as_uint(a.gain_c)) << 32) | (0xffffffffu - uint32_t(j));
+                bool fg = false, fc = false;
+                if (a.gain_g > 0.0f && (live_type > 0 || kg > lv[0]) && hopeless(j, a, 0)) fg = true;
+                if (a.gain_c > 0.0f && live_type > 0 && (live_type > 1 || kc > lv[1]) && hopeless(j, a, 1)) fc = true;
+                if (fg || fc) {
+                    mine += int(fg) + int(fc);
+                    if (fg) a.gain_g = 0.0f;
+                    if (fc) a.gain_c = 0.0f;
+                    a.packed = pack(pk_gi(a.packed), pk_ci(a.packed), pk_next_gi(a.packed), false, pk_fz_g(a.packed) || fg, pk_fz_c(a.packed) || fc);
+                    hotA[j] = a;
+                }
+            }
+            mine = __reduce_add_sync(0xffffffffu, mine);
+            if (lane == 0) sh.redi[2][warp] = mine;
+            __syncthreads();
+            if (warp == 0) {
+                const int frozen = __reduce_add_sync(0xffffffffu, sh.redi[2][lane]);
+                if (lane == 0) {
+                    if (sh.steps + frozen > max_steps) {               // the cap falls inside the run of failures
+                        sh.steps = max_steps; sh.capped = 1; sh.sel_j = -1; sh.which = -1;
+                    } else {
+                        sh.steps += frozen;
+                        sh.which = live_type < 2 ? 2 + live_type : -1;
+                        sh.sel_j = live_type < 2 ? int(0xffffffffu - uint32_t(lv[live_type])) : -1;
+                    }
+                }
+            }
+            __syncthreads();
+        }
+
+        if (warp == 0) {
+            const int which = sh.which;
+            int sel_j = sh.sel_j;
+            if (sel_j >= 0 && sh.steps >= max_steps) { if (lane == 0) sh.capped = 1; sel_j = -1; }
+            bool ok = false;
             if (sel_j >= 0) {
                 const int j = sel_j, type = which & 1;
                 const bool by_exchange = which >= 2;
@@ -513,14 +694,13 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
                 const int gi2 = type == 0 ? pk_next_gi(a.packed) : gi;
                 const int ci2 = type == 0 ? ci : ci + 1;
                 const float gain = type == 0 ? a.gain_g : a.gain_c;
-                bool ok = false;
+                const int old_node = a.node;
+                const bool was_single = gi >= 0 && sp.g_levels[gi] <= sp.Gn;
                 if (!by_exchange) {
-                    const int old_node = a.node;
-                    const bool was_single = gi >= 0 && sp.g_levels[gi] <= sp.Gn;
                     ok = commit_warp(sp, cl, n_empty, cv, cp, cg, feas, j, a, b, gi2, ci2, true, lane);
                     if (ok && lane == 0) {
-                        if (was_single) list_remove(nl, old_node, j);
-                        if (sp.g_levels[gi2] <= sp.Gn) list_add(nl, a.node, j);
+                        if (was_single) { list_remove(nl, old_node, j); dirty[old_node] = 1; }
+                        if (sp.g_levels[gi2] <= sp.Gn) { list_add(nl, a.node, j); dirty[a.node] = 1; }
                     }
                     __syncwarp();
                 } else if (sp.g_levels[gi2] <= sp.Gn) {
@@ -539,7 +719,7 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
                             ok = exchange_warp(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, j, gi2, ci2, n, false, cand_g, cand_c, true, lane);
                         }
                     }
-                    if (ok) { a = hotA[j]; b = hotB[j]; }
+                    if (ok) { a = hotA[j]; b = hotB[j]; if (lane == 0) dirty[a.node] = 1; }
                 }
                 bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                 if (!ok) { if (type == 0) fz_g = true; else fz_c = true; }
@@ -553,7 +733,7 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
                     sh.steps += 1;
                 }
             }
-            if (lane == 0) sh.sel_j = sel_j;
+            if (lane == 0) { sh.sel_j = sel_j; sh.changed = ok ? 1 : 0; }
         }
         __syncthreads();
         if (sh.sel_j < 0) break;
@@ -589,7 +769,7 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
 
 static size_t incr_smem(const Space &sp, int N)
 {
-    return (size_t(N) * 24 + size_t(sp.n_small) * sp.nC * 4 + 15) & ~size_t(15);
+    return (size_t(N) * 36 + size_t(sp.n_small) * sp.nC * 4 + 15) & ~size_t(15);
 }
 
 // scratch: HotA [J] | HotB [J] | roles [J] | whole-node counts [J] | node lists [N][Gn]

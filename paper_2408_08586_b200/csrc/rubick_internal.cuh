@@ -83,6 +83,11 @@ struct rubick_ctx {
     rubick_assignment *d_out_stage; size_t cap_out;
     rubick_node *d_node_stage; size_t cap_node;
     int32_t *d_best_todo; size_t cap_best_todo;     // rubick_best_plan: count + jobs left to the general kernel
+    // state that rubick_incremental_event_host carries from one event to the next
+    int inc_J, inc_N;                   // slots / nodes of the carried state and of the cached tables; inc_J = 0: none
+    int inc_cur;                        // which of the two state buffers holds the last result
+    rubick_assignment *d_inc_state[2]; rubick_node *d_inc_nodes[2]; rubick_reconf *d_inc_reconf; rubick_job *d_inc_jobs;
+    size_t cap_inc_state[2], cap_inc_nodes[2], cap_inc_reconf, cap_inc_jobs;
     int tile_jobs;                      // job tile of rubick_schedule_round
     int num_sms;
     std::string err;

@@ -1,4 +1,6 @@
-"""Event-driven harness: every job arrival or completion triggers one full scheduling round.
+"""Event-driven harness: every job arrival or completion triggers one scheduling round, either a full
+re-plan of all active jobs (``run_events``) or the incremental round that starts from the previous
+allocation (``run_events_incremental``).
 
 Host-side glue only (the paper's Section 7.4 uses a simulator for the same purpose): it keeps
 the set of active jobs, calls ``rubick_schedule_round_host`` on them at every event, advances each
@@ -68,3 +70,81 @@ def run_events(ctx, cfg, n_events=1000, warm_jobs=1500, max_steps=1 << 30, sync=
         if finished:
             active = [j for j in active if j not in finished]
     return dict(latency_ms=np.asarray(lat), active=np.asarray(act), steps=np.asarray(stp))
+
+
+def run_events_incremental(ctx, cfg, n_events=1000, warm_jobs=1500, slots=4096, theta=0.97, max_steps=1 << 30):
+    """The same event stream through ``rubick_incremental_event_host``: jobs live in `slots` fixed slots,
+    the previous allocation and the curve tables stay on the device, and an event uploads only the slot
+    that changed.  A job's checkpoint-resume cost is ``workloads.reconf_cost``; its trained time T and
+    reconfiguration count feed the gate of Section 5.2.
+    -> dict(latency_ms, active, steps, reconfigured [n_events])."""
+    jobs = cfg["jobs"]
+    pool = len(jobs["P"])
+    arrivals, lengths = workloads.draw_events(cfg["seed"], pool)
+    warm = min(warm_jobs, pool, slots)
+    arrivals = np.concatenate([np.zeros(warm), arrivals[: pool - warm] if pool > warm else []])
+    remaining = lengths.copy()
+    records = rb.pack_jobs(jobs)
+    N = cfg["n_nodes"]
+    w = np.asarray(jobs["w"], dtype=np.float64)
+    cost = workloads.reconf_cost(jobs)
+
+    slot_job = np.full(slots, -1, dtype=np.int64)          # pool index of the job in each slot
+    slot_job[:warm] = np.arange(warm)
+    free = list(range(slots - 1, warm - 1, -1))
+    h_jobs = np.zeros(slots, dtype=rb.JOB_DTYPE)
+    h_jobs[:warm] = records[:warm]
+    reconf = np.zeros(slots, dtype=rb.RECONF_DTYPE)
+    reconf["active"][:warm] = 1
+    reconf["delta"][:warm] = cost[:warm]
+    h_out = np.zeros(slots, dtype=rb.ASSIGN_DTYPE)
+    prev = np.zeros(slots, dtype=rb.ASSIGN_DTYPE)
+    next_arrival = warm
+    now = 0.0
+    changed = None                                          # first event: everything is new
+    lat, act, stp, rec = [], [], [], []
+    for _ in range(n_events):
+        live = np.nonzero(slot_job >= 0)[0]
+        if len(live) == 0 and next_arrival >= pool:
+            break
+        t0 = time.perf_counter()
+        steps, _ = ctx.incremental_event_host(h_jobs, slots, N, h_out, changed=changed, h_reconf=reconf, theta=theta,
+                                              restart=changed is None, max_steps=max_steps)
+        lat.append(1e3 * (time.perf_counter() - t0))
+        act.append(len(live))
+        stp.append(steps)
+        was = (prev["status"] == rb.RUNNING) & (slot_job >= 0)
+        moved = was & (h_out["status"] == rb.RUNNING) & ((h_out["g"] != prev["g"]) | (h_out["c"] != prev["c"]) | (h_out["plan"] != prev["plan"]))
+        reconf["n_reconf"] += moved.astype(np.int32)
+        rec.append(int(moved.sum()))
+        prev[:] = h_out
+        # advance to the next event
+        idx = slot_job[live]
+        rate = w[idx] * h_out["thr"][live].astype(np.float64)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            eta = np.where(rate > 0, remaining[idx] / rate, np.inf)
+        t_done = now + (eta.min() if len(eta) else np.inf)
+        t_arr = arrivals[next_arrival] if next_arrival < pool and free else np.inf
+        t_next = min(t_done, t_arr)
+        if not np.isfinite(t_next):
+            break
+        dt = t_next - now
+        remaining[idx] -= rate * dt
+        reconf["T"][live] = np.where(h_out["status"][live] == rb.RUNNING, reconf["T"][live] + dt, 0.0)
+        now = t_next
+        changed = []
+        if t_arr <= t_done:
+            s = free.pop()
+            slot_job[s] = next_arrival
+            h_jobs[s] = records[next_arrival]
+            reconf[s] = (0.0, cost[next_arrival], 0, 1)
+            changed.append(s)
+            next_arrival += 1
+        done = live[remaining[idx] <= 1e-9 * lengths[idx]]
+        if t_done <= t_arr and len(done) == 0:
+            done = live[[int(np.argmin(eta))]]
+        for s in done:
+            slot_job[s] = -1
+            reconf["active"][s] = 0
+            free.append(int(s))
+    return dict(latency_ms=np.asarray(lat), active=np.asarray(act), steps=np.asarray(stp), reconfigured=np.asarray(rec))

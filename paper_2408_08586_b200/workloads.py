@@ -104,6 +104,14 @@ def take(jobs, idx):
     return {k: np.asarray(v)[idx] for k, v in jobs.items()}
 
 
+def reconf_cost(jobs, fixed_s=20.0, bytes_per_param=14.0, storage_bytes_per_s=5e9):
+    """Checkpoint-resume seconds of each job (the delta of the reconfiguration gate, Section 5.2): a
+    fixed restart time plus the optimizer and model states written and read back once over the
+    checkpoint storage.  Generator constants; the paper prints no value."""
+    P = np.asarray(jobs["P"], dtype=np.float64)
+    return (fixed_s + 2.0 * bytes_per_param * P / storage_bytes_per_s).astype(np.float32)
+
+
 def draw_events(seed, n_jobs, mean_interarrival_s=30.0, median_len_s=7200.0, sigma=1.5):
     """Arrival times (Poisson process) and nominal lengths (log-normal) for an event-driven run."""
     rng = np.random.Generator(np.random.PCG64(seed + 1000))

@@ -89,8 +89,10 @@ def pack_prev(prev, J, n_nodes):
 
 
 def incremental_on_tables(gpu, jobs, cv, cp, cg, feas, n_nodes, prev, active=None, T=None, delta=None, nrec=None,
-                          theta=0.97, max_steps=1 << 30, quota=None):
-    """rubick_incremental_round on host-provided tables and previous state -> dict like the oracle's."""
+                          theta=0.97, max_steps=1 << 30, quota=None, want_log=True):
+    """rubick_incremental_round on host-provided tables and previous state -> dict like the oracle's.
+    Without a step log the library sorts out hopeless exchange candidates in bulk (another code path,
+    same allocation and step count)."""
     t = gpu.torch
     J = len(jobs["P"])
     d_jobs = gpu.jobs_to_device(jobs)
@@ -101,7 +103,7 @@ def incremental_on_tables(gpu, jobs, cv, cp, cg, feas, n_nodes, prev, active=Non
     cap = int(min(max_steps, 2 * J * (gpu.nG + gpu.nC + 2) + 1))
     d_out = gpu.empty(max(J, 1) * rb.ASSIGN_DTYPE.itemsize, t.uint8)
     d_node = gpu.empty(n_nodes * rb.NODE_DTYPE.itemsize, t.uint8)
-    d_log = gpu.empty(max(cap, 1), t.int32)
+    d_log = gpu.empty(max(cap, 1), t.int32) if want_log else None
     d_prev = d_prev_nodes = d_reconf = None
     if prev is not None:
         a, nd = pack_prev(prev, J, n_nodes)
@@ -116,7 +118,7 @@ def incremental_on_tables(gpu, jobs, cv, cp, cg, feas, n_nodes, prev, active=Non
     steps, capped = gpu.ctx.incremental_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, n_nodes, cap, d_out, d_node, d_log,
                                               d_prev=d_prev, d_prev_nodes=d_prev_nodes, d_reconf=d_reconf, theta=theta, quota=quota)
     return unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE)[:J], rb.from_device(d_node, rb.NODE_DTYPE), steps, capped,
-                        d_log.cpu().numpy()[:steps])
+                        d_log.cpu().numpy()[:steps] if want_log else None)
 
 
 def unpack_round(out, node, steps, capped, log):

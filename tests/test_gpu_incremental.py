@@ -35,6 +35,9 @@ def test_event_sequences_are_bit_exact(seed):
         got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], inp["prev"], active=inp["active"],
                                     T=inp["T"], delta=inp["delta"], nrec=inp["nrec"])
         assert_rounds_equal(got, want)
+        bulk = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, cfg["n_nodes"], inp["prev"], active=inp["active"],
+                                     T=inp["T"], delta=inp["delta"], nrec=inp["nrec"], want_log=False)
+        assert_rounds_equal(bulk, want)                  # no log: hopeless candidates frozen in bulk, same result and count
         exchanges += int((((want["log"] >> 2) & 1) & (want["log"] & 1)).sum())
     if seed >= 2:
         assert exchanges > 0
@@ -66,6 +69,7 @@ def test_larger_event_sequences_with_quotas_are_bit_exact(name, J, N, rounds):
         got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, N, prev, **kw)
         assert want["steps"] is not None
         assert_rounds_equal(got, want)
+        assert_rounds_equal(incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, N, prev, want_log=False, **kw), want)
         seen_exchange |= bool((((want["log"] >> 2) & 1) & (want["log"] & 1)).any())
         seen_pending |= bool((want["status"] == 2).any())
         prev = want
@@ -95,6 +99,15 @@ def test_small_nodes_and_few_levels_are_bit_exact():
                                                  cfg["m_levels"], 5, prev, want_log=True, **kw)
         got = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, 5, prev, **kw)
         assert_rounds_equal(got, want)
+        assert_rounds_equal(incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, 5, prev, want_log=False, **kw), want)
+        for cap in (3, 7, 15):                           # the step cap falls inside a run of bulk-frozen candidates
+            kc = dict(kw, max_steps=cap)
+            wc = oracle.schedule_round_incremental(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                                   cfg["m_levels"], 5, prev, want_log=True, **kc)
+            gc_ = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas, 5, prev, want_log=False, **kc)
+            assert gc_["steps"] == wc["steps"] and gc_["capped"] == wc["capped"]
+            if not wc["capped"]:
+                assert_rounds_equal(gc_, wc)
         prev = want
 
 
@@ -198,3 +211,62 @@ def test_step_cap_and_argument_validation():
     rc = rb.lib().rubick_incremental_round(gpu.ctx._h, rb._ptr(d), 1, rb._ptr(d), rb._ptr(d), rb._ptr(d), rb._ptr(d), C.byref(cl),
                                            rb._ptr(d), None, None, C.c_float(0.97), 10, rb._ptr(d), None, None, C.byref(steps))
     assert rc == rb.EINVAL                       # previous assignments without the previous node states
+
+
+def test_events_with_state_kept_in_the_context_match_the_oracle():
+    """rubick_incremental_event_host: slots, previous allocation and cached tables live in the context;
+    only changed slots are uploaded and re-evaluated.  The oracle replays every event on the tables the
+    library itself computes for the slots' current jobs."""
+    cfg, rng = event_config(5, J=48, n_nodes=3)
+    pool = workloads.make("paper-scale", J=200)["jobs"]               # jobs that arrive into the 48 slots
+    gpu = Gpu(cfg)
+    J, N = 48, 3
+    slot_jobs = {k: np.asarray(v).copy() for k, v in cfg["jobs"].items()}
+    records = rb.pack_jobs(slot_jobs)
+    h_out = np.zeros(J, dtype=rb.ASSIGN_DTYPE)
+    h_nodes = np.zeros(N, dtype=rb.NODE_DTYPE)
+    reconf = np.zeros(J, dtype=rb.RECONF_DTYPE)
+    reconf["delta"] = rng.uniform(5.0, 40.0, J)
+    prev = None
+    next_pool = 0
+    for rnd in range(8):
+        changed = []
+        for s in range(J):
+            if reconf["active"][s] and rng.uniform() < 0.12:
+                reconf["active"][s] = 0                                   # finished
+            elif not reconf["active"][s] and rng.uniform() < 0.25:
+                for k in slot_jobs:                                       # a new job takes the slot
+                    if k in pool:
+                        slot_jobs[k][s] = pool[k][next_pool]
+                slot_jobs["gmin_idx"][s] = int(rng.integers(0, 3)) if rng.uniform() < 0.4 else -1
+                slot_jobs["cmin_idx"][s] = 0 if slot_jobs["gmin_idx"][s] >= 0 else -1
+                next_pool += 1
+                reconf["active"][s] = 1
+                reconf["T"][s] = 0
+                reconf["n_reconf"][s] = 0
+                changed.append(s)
+        records = rb.pack_jobs(slot_jobs)
+        if prev is not None:
+            running = (prev["status"] == 1) & (reconf["active"] == 1)
+            reconf["T"] = np.where(running, reconf["T"] + rng.uniform(100.0, 4000.0, J), 0).astype(np.float32)
+        steps, capped = gpu.ctx.incremental_event_host(records, J, N, h_out, changed=None if rnd == 0 else changed,
+                                                       h_reconf=reconf, h_node_out=h_nodes)
+        # the oracle on the library's own tables of the current slot jobs
+        d_jobs, d_thr, d_feas = gpu.eval(slot_jobs)
+        bv, bp, bg = gpu.best(d_thr, d_feas, J)
+        sh = gpu.shape4(J)
+        cv, cp, cg = bv.cpu().numpy().reshape(sh), bp.cpu().numpy().reshape(sh), bg.cpu().numpy().reshape(sh)
+        feas = gpu.np_feas(d_feas, J)
+        want = oracle.schedule_round_incremental(slot_jobs, cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                                 cfg["m_levels"], N, prev, active=reconf["active"], T=reconf["T"],
+                                                 delta=reconf["delta"], nrec=reconf["n_reconf"])
+        assert want["steps"] == steps and not capped
+        for k in ("g", "c", "m_bytes", "plan", "first_node", "n_nodes", "status", "m_level"):
+            assert np.array_equal(h_out[k].astype(np.int64), want[k]), (rnd, k)
+        assert np.array_equal(h_out["thr"].view(np.uint32), want["thr"].view(np.uint32))
+        assert np.array_equal(np.stack([h_nodes["free_g"], h_nodes["free_c"], h_nodes["free_m"], h_nodes["owner"]], axis=1).astype(np.int64), want["node"])
+        if prev is not None:
+            was = (prev["status"] == 1) & (reconf["active"] == 1)
+            moved = was & (want["status"] == 1) & ((want["g"] != prev["g"]) | (want["c"] != prev["c"]) | (want["plan"] != prev["plan"]))
+            reconf["n_reconf"] += moved.astype(np.int32)
+        prev = want
