@@ -6,5 +6,5 @@ benchmark may import this package; the CUDA library and its Python binding never
 from .oracle import (  # noqa: F401
     JOB_FIELDS, ENV_FIELDS, TERM_FIELDS, MEM_FIELDS,
     build, lib, overlap, terms, memory, feas_word, enumerate_plans, eval_candidates,
-    best_plan, gain, schedule_round, schedule_round_incremental, bruteforce, min_resources,
+    best_plan, gain, schedule_round, schedule_round_incremental, bruteforce, min_resources, fit, FIT_NAMES,
 )

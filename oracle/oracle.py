@@ -268,6 +268,31 @@ def schedule_round_incremental(jobs, env, curve_val, curve_plan, curve_g, feas, 
                 steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
 
 
+FIT_NAMES = ("k_bwd", "k_sync", "k_opt", "k_opt_off", "k_off", "k_swap", "k_const")
+
+
+def fit(jobs, plans, env, sample_plan, sample_c, sample_thr, sweeps=14):
+    """Section 4.3 model fitting by RMSLE.  sample_plan [J, S] plan indices (-1: unused slot), sample_c
+    [J, S] cores, sample_thr [J, S] measured throughput; the start is the coefficients in `jobs`.
+    -> (theta [J, 7] in FIT_NAMES order, rmsle [J, 2] before / after, margin [J])."""
+    rows = job_rows(jobs)
+    J = rows.shape[0]
+    plans = _i32(plans)
+    spn = np.ascontiguousarray(sample_plan, dtype=np.int32).reshape(J, -1)
+    S = spn.shape[1]
+    scs = _i64(sample_c).reshape(J, S)
+    sth = _f64(sample_thr).reshape(J, S)
+    theta = np.zeros((J, 7), dtype=np.float64)
+    rmsle = np.zeros((J, 2), dtype=np.float64)
+    margin = np.zeros(J, dtype=np.float64)
+    f = lib().oracle_fit
+    f.restype = None
+    f(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double), _p(plans, C.c_int32), C.c_int(plans.shape[0]),
+      _p(spn, C.c_int32), _p(scs, C.c_int64), _p(sth, C.c_double), C.c_int(S), C.c_int(sweeps),
+      _p(theta, C.c_double), _p(rmsle, C.c_double), _p(margin, C.c_double))
+    return theta, rmsle, margin
+
+
 def bruteforce(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels):
     """Best total weighted throughput over all single-node assignments (tiny instances)."""
     rows = job_rows(jobs)

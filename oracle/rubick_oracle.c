@@ -1035,6 +1035,118 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
     return capped ? -steps - 1 : steps;
 }
 
+/* ======================================================================================
+ * Section 4.3, "Continuous model fitting": the seven fittable parameters of a model type
+ * (k_bwd, k_sync, k_opt, k_opt_off, k_off, k_swap, k_const) are chosen to minimise the root
+ * mean squared logarithmic error between the model and throughputs measured on sampled
+ * (plan, cores) configurations:  RMSLE = sqrt(mean_i (ln(1 + pred_i) - ln(1 + y_i))^2).
+ *
+ * The paper names no optimiser.  This project's reading is a derivative-free pattern search
+ * that two implementations can follow decision by decision:
+ *  - start from the coefficients in the job record (the previous fit), clamped to the bounds;
+ *  - `sweeps` sweeps; sweep r moves one parameter at a time, in Table 1's order, among the values
+ *    base * M_r^e, e = -4 .. 4, clamped, where M_0 = 2^(3/4) and M_(r+1) = sqrt(M_r); the other
+ *    six stay at their latest values; the candidate with the smallest error wins, the present
+ *    value on ties, then candidates in the order e = -1, +1, -2, +2, ... ;
+ *  - candidate values are built from correctly rounded operations only (sqrt, *, /), so they are
+ *    the same numbers everywhere; only the model's own pow / log may differ in the last bits.
+ * out_theta [J][7]; out_rmsle [J][2] = before, after; out_margin [J] = the smallest relative gap
+ * between the winning and the next distinct error over all decisions of the fit (a second
+ * implementation may only deviate where this is tiny).
+ * ==================================================================================== */
+enum { FIT_PARAMS = 7 };
+static const int fit_field[FIT_PARAMS] = {JF_KBWD, JF_KSYNC, JF_KOPT, JF_KOPTOFF, JF_KOFF, JF_KSWAP, JF_KCONST};
+static const double fit_lo[FIT_PARAMS] = {0.25, 1.0, 1e-13, 1e-10, 1.0, 1.0, 1e-4};
+static const double fit_hi[FIT_PARAMS] = {16.0, 16.0, 1e-9, 1e-6, 16.0, 16.0, 10.0};
+
+static double fit_sse(const double *row, const double *env, const int32_t *plans,
+                      const int32_t *s_plan, const int64_t *s_c, const double *s_thr, int S, int *n_out)
+{
+    double sse = 0.0; int n = 0;
+    for (int i = 0; i < S; ++i) {
+        if (s_plan[i] < 0) continue;
+        double out[TF_COUNT];
+        oracle_terms(row, env, plans + (size_t)s_plan[i] * PF_COUNT, (double)s_c[i], out);
+        double e = log1p(out[TF_THR]) - log1p(s_thr[i]);
+        sse += e * e; ++n;
+    }
+    if (n_out) *n_out = n;
+    return sse;
+}
+
+#define FIT_EPS 1e-9      /* a move must lower the squared error by more than this fraction */
+
+void oracle_fit(const double *jobs, int J, const double *env, const int32_t *plans, int P,
+                const int32_t *s_plan, const int64_t *s_c, const double *s_thr, int S, int sweeps,
+                double *out_theta, double *out_rmsle, double *out_margin)
+{
+    (void)P;
+    static const int order[8] = {-1, 1, -2, 2, -3, 3, -4, 4};
+    for (int j = 0; j < J; ++j) {
+        double row[JF_COUNT];
+        memcpy(row, jobs + (size_t)j * JF_COUNT, sizeof row);
+        const int32_t *sp = s_plan + (size_t)j * S; const int64_t *sc = s_c + (size_t)j * S; const double *sy = s_thr + (size_t)j * S;
+        for (int p = 0; p < FIT_PARAMS; ++p) {
+            double v = row[fit_field[p]];
+            if (!(v >= fit_lo[p])) v = fit_lo[p];
+            if (v > fit_hi[p]) v = fit_hi[p];
+            row[fit_field[p]] = v;
+        }
+        int n = 0;
+        double cur = fit_sse(row, env, plans, sp, sc, sy, S, &n);
+        double margin = INFINITY;
+        out_rmsle[2 * j] = n > 0 ? sqrt(cur / n) : 0.0;
+        double M = sqrt(2.0) * sqrt(sqrt(2.0));                 /* 2^(3/4) */
+        for (int r = 0; r < sweeps && n > 0; ++r) {
+            double mul[5]; mul[0] = 1.0; mul[1] = M; mul[2] = M * M; mul[3] = mul[2] * M; mul[4] = mul[2] * mul[2];
+            double before[FIT_PARAMS];
+            for (int p = 0; p < FIT_PARAMS; ++p) before[p] = row[fit_field[p]];
+            /* exploratory moves, one parameter at a time */
+            for (int p = 0; p < FIT_PARAMS; ++p) {
+                double base = row[fit_field[p]];
+                double best = cur, best_v = base;
+                for (int q = 0; q < 8; ++q) {
+                    int e = order[q];
+                    double v = e > 0 ? base * mul[e] : base / mul[-e];
+                    if (v < fit_lo[p]) v = fit_lo[p];
+                    if (v > fit_hi[p]) v = fit_hi[p];
+                    if (v == base) continue;
+                    row[fit_field[p]] = v;
+                    double sse = fit_sse(row, env, plans, sp, sc, sy, S, NULL);
+                    double bar = best * (1.0 - FIT_EPS);
+                    double gap = fabs(sse - bar) / (bar > 1e-300 ? bar : 1e-300);
+                    if (gap < margin) margin = gap;
+                    if (sse < bar) { best = sse; best_v = v; }
+                }
+                row[fit_field[p]] = best_v; cur = best;
+            }
+            /* pattern moves (Hooke and Jeeves): repeat the sweep's combined displacement while it pays */
+            for (int rep = 0; rep < 4; ++rep) {
+                double keep[FIT_PARAMS]; int moved = 0;
+                for (int p = 0; p < FIT_PARAMS; ++p) {
+                    keep[p] = row[fit_field[p]];
+                    double v = keep[p] * keep[p] / before[p];
+                    if (v < fit_lo[p]) v = fit_lo[p];
+                    if (v > fit_hi[p]) v = fit_hi[p];
+                    if (v != keep[p]) moved = 1;
+                    row[fit_field[p]] = v;
+                }
+                if (!moved) break;
+                double sse = fit_sse(row, env, plans, sp, sc, sy, S, NULL);
+                double bar = cur * (1.0 - FIT_EPS);
+                double gap = fabs(sse - bar) / (bar > 1e-300 ? bar : 1e-300);
+                if (gap < margin) margin = gap;
+                if (sse < bar) { cur = sse; for (int p = 0; p < FIT_PARAMS; ++p) before[p] = keep[p]; }
+                else { for (int p = 0; p < FIT_PARAMS; ++p) row[fit_field[p]] = keep[p]; break; }
+            }
+            if (r & 1) M = sqrt(M);                             /* the step halves every second sweep */
+        }
+        for (int p = 0; p < FIT_PARAMS; ++p) out_theta[(size_t)j * FIT_PARAMS + p] = row[fit_field[p]];
+        out_rmsle[2 * j + 1] = n > 0 ? sqrt(cur / n) : 0.0;
+        out_margin[j] = margin;
+    }
+}
+
 /* Exhaustive search on one node (tiny instances only): every job is either left out or
  * given one (g level, c level, m level); the allocation uses the GPUs of the curve entry,
  * the cores of the level and the memory of the entry's plan; sums must fit the node.

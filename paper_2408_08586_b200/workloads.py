@@ -112,6 +112,20 @@ def reconf_cost(jobs, fixed_s=20.0, bytes_per_param=14.0, storage_bytes_per_s=5e
     return (fixed_s + 2.0 * bytes_per_param * P / storage_bytes_per_s).astype(np.float32)
 
 
+FIT_NOMINAL = dict(k_bwd=2.0, k_sync=2.0, k_opt=1e-11, k_opt_off=2e-8, k_off=2.0, k_swap=2.0, k_const=0.05)
+
+
+def draw_fit_picks(seed, J, S, n_c_levels, noise_sigma=0.03):
+    """Random draws from which the tests and the benchmark build the measured samples of Section 4.3 for J
+    model types: per sample slot a rank in [0, 1) used to pick a plan among those the job can run (the
+    first third of the slots among offloading plans, as the paper asks for), a core-level index and a
+    log-normal measurement-noise factor.  No model arithmetic here: the throughputs come from whoever
+    uses the picks."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    return dict(rank=rng.uniform(0.0, 1.0, (J, S)), c_idx=rng.integers(0, n_c_levels, (J, S)),
+                noise=np.exp(rng.normal(0.0, noise_sigma, (J, S))))
+
+
 def draw_events(seed, n_jobs, mean_interarrival_s=30.0, median_len_s=7200.0, sigma=1.5):
     """Arrival times (Poisson process) and nominal lengths (log-normal) for an event-driven run."""
     rng = np.random.Generator(np.random.PCG64(seed + 1000))
