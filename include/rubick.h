@@ -146,6 +146,12 @@ typedef struct {
     int32_t active;              /* 0: the slot is empty (job finished or never submitted)           */
 } rubick_reconf;
 
+/* One measured configuration of a model type (Section 4.3): plan index, CPU cores and the throughput
+ * observed there; plan < 0 marks an unused slot. 16 bytes. */
+typedef struct { int32_t plan; int32_t cores; double thr; } rubick_sample;
+
+#define RUBICK_FIT_PARAMS 7      /* k_bwd, k_sync, k_opt, k_opt_off, k_off, k_swap, k_const (Table 1) */
+
 /* ---- context ---------------------------------------------------------------------------------- */
 
 /* Creates a context bound to CUDA device `device` and to `cuda_stream` (a cudaStream_t passed as
@@ -241,6 +247,19 @@ int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
                         const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                         int32_t *h_steps);
+
+/* Model fitting (Section 4.3, "Continuous model fitting"), for J model types at once: chooses the seven
+ * fittable parameters of each d_jobs[j] to minimise the root mean squared logarithmic error
+ * sqrt(mean_i (ln(1 + predicted throughput_i) - ln(1 + d_samples[j][i].thr))^2) over its S sample slots.
+ * The paper names no optimiser: this is a pattern search (exploratory moves on a geometric grid that
+ * halves every second sweep, then pattern moves) started from the coefficients in the job record and
+ * kept inside fixed bounds (k_bwd 0.25..16, the three overlap exponents 1..16, k_opt 1e-13..1e-9,
+ * k_opt_off 1e-10..1e-6, k_const 1e-4..10); `sweeps` sweeps (14 is a good default; at most 64).
+ * Double precision.  d_theta: J * 7 doubles in the order of RUBICK_FIT_PARAMS; d_rmsle: J * 2 doubles,
+ * the error before and after.  The job records themselves are not modified.  Plans refer to the
+ * plan list of rubick_set_space.  Enqueued on the context's stream; errors: EINVAL, ESTATE, ECUDA. */
+int rubick_fit_models(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const rubick_sample *d_samples, int S,
+                      int sweeps, double *d_theta, double *d_rmsle);
 
 /* One incremental scheduling round (Section 5.2: Algorithm 1 with its shrink step, and
  * "Incorporating reconfiguration penalty") on given curve tables, started from the allocation an

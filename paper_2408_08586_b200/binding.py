@@ -28,6 +28,8 @@ PLAN_DTYPE = np.dtype([("log2d", "u1"), ("log2t", "u1"), ("log2p", "u1"), ("zero
 ASSIGN_DTYPE = np.dtype([("g", "<i4"), ("c", "<i4"), ("m_bytes", "<i8"), ("plan", "<i4"), ("first_node", "<i4"),
                          ("n_nodes", "<i4"), ("thr", "<f4"), ("status", "<i4"), ("m_level", "<i4")])
 REQUEST_DTYPE = np.dtype([("g_idx", "<i4"), ("c_idx", "<i4"), ("m_idx", "<i4"), ("plan", "<i4")])
+SAMPLE_DTYPE = np.dtype([("plan", "<i4"), ("cores", "<i4"), ("thr", "<f8")])
+FIT_NAMES = ("k_bwd", "k_sync", "k_opt", "k_opt_off", "k_off", "k_swap", "k_const")
 RECONF_DTYPE = np.dtype([("T", "<f4"), ("delta", "<f4"), ("n_reconf", "<i4"), ("active", "<i4")])
 NODE_DTYPE = np.dtype([("free_g", "<i4"), ("free_c", "<i4"), ("free_m", "<i8"), ("owner", "<i4"), ("reserved", "<i4")])
 assert JOB_DTYPE.itemsize == 128 and PLAN_DTYPE.itemsize == 8
@@ -63,7 +65,7 @@ def make_cluster(n_nodes, quota=None):
 
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
            "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_marginal_gain",
-           "rubick_min_resources",
+           "rubick_min_resources", "rubick_fit_models",
            "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
            "rubick_schedule_round_host", "rubick_incremental_event_host"]
 
@@ -97,6 +99,7 @@ def lib():
         L.rubick_best_plan.argtypes = [vp, vp, vp, ip, C.c_uint, vp, vp, vp]
         L.rubick_marginal_gain.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp]
         L.rubick_min_resources.argtypes = [vp, vp, vp, vp, ip, vp, vp, vp, vp]
+        L.rubick_fit_models.argtypes = [vp, vp, ip, vp, ip, ip, vp, vp]
         L.rubick_greedy_round.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), ip, vp, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_incremental_round.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(Cluster), vp, vp, vp, C.c_float, ip, vp, vp, vp,
                                                C.POINTER(C.c_int32)]
@@ -221,6 +224,10 @@ class Context:
     def min_resources(self, d_thr, d_feas, d_curve_val, J, d_req, d_gmin_idx, d_cmin_idx, d_baseline):
         return self._check(lib().rubick_min_resources(self._h, _ptr(d_thr), _ptr(d_feas), _ptr(d_curve_val), int(J), _ptr(d_req),
                                                       _ptr(d_gmin_idx), _ptr(d_cmin_idx), _ptr(d_baseline)))
+
+    def fit_models(self, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle):
+        return self._check(lib().rubick_fit_models(self._h, _ptr(d_jobs), int(J), _ptr(d_samples), int(S), int(sweeps),
+                                                   _ptr(d_theta), _ptr(d_rmsle)))
 
     def greedy_round(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, n_nodes, max_steps, d_out,
                      d_node_out=None, d_step_log=None, quota=None):

@@ -296,6 +296,23 @@ int rubick_min_resources(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_
     return RUBICK_OK;
 }
 
+int rubick_fit_models(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const rubick_sample *d_samples, int S,
+                      int sweeps, double *d_theta, double *d_rmsle)
+{
+    CHECK_CTX(ctx);
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (J == 0) return RUBICK_OK;
+    if (!d_jobs || !d_samples || !d_theta || !d_rmsle) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if (S < 1 || S > 4096) return fail(ctx, RUBICK_EINVAL, "1 .. 4096 sample slots per model");
+    if (sweeps < 0 || sweeps > 64) return fail(ctx, RUBICK_EINVAL, "0 .. 64 sweeps");
+    if ((reinterpret_cast<uintptr_t>(d_samples) & 7) || (reinterpret_cast<uintptr_t>(d_theta) & 7) || (reinterpret_cast<uintptr_t>(d_rmsle) & 7))
+        return fail(ctx, RUBICK_EINVAL, "d_samples, d_theta and d_rmsle must be 8-byte aligned");
+    CUDA_TRY(ctx, launch_fit(ctx->env, ctx->d_quads, ctx->space.P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle, ctx->stream),
+             "launch fit_models");
+    return RUBICK_OK;
+}
+
 // enqueue the round and leave the step count in ctx->d_steps
 static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, const rubick_cluster *cl, int max_steps,
