@@ -323,6 +323,38 @@ def main():
         torch.cuda.synchronize()
         minres_ms = a.elapsed_time(b) / 10
 
+    # model fitting (Section 4.3) for the first model types of the batch: samples read off the candidate
+    # table this run just computed, with measurement noise; start from the generator's nominal coefficients
+    fit = None
+    if rank == 0 and J > 0:
+        Jf, S, sweeps = min(J, 1024), 16, 14
+        picks = workloads.draw_fit_picks(cfg["seed"], Jf, S, C)
+        thr_h = d_thr[: Jf * C * P].cpu().numpy().reshape(Jf, C, P)
+        feas_h = d_feas[: Jf * P].cpu().numpy().view(np.uint32).reshape(Jf, P)
+        pl6 = np.stack([1 << plans["log2d"].astype(np.int64), 1 << plans["log2t"].astype(np.int64), 1 << plans["log2p"].astype(np.int64),
+                        plans["zero"], plans["gc"], plans["off"]], axis=1)
+        sp_, sc_, sy_ = workloads.fit_samples(cfg, pl6, thr_h, feas_h, picks)
+        smp = np.zeros((Jf, S), dtype=rb.SAMPLE_DTYPE)
+        smp["plan"], smp["cores"], smp["thr"] = sp_, sc_, sy_
+        fj = workloads.take(jobs, slice(0, Jf))
+        for k_, v_ in workloads.FIT_NOMINAL.items():
+            fj[k_] = np.full(Jf, v_)
+        d_fj, d_smp = rb.to_device(rb.pack_jobs(fj), dev), rb.to_device(smp, dev)
+        d_theta = torch.empty(Jf * 7, dtype=torch.float64, device=dev)
+        d_rm = torch.empty(Jf * 2, dtype=torch.float64, device=dev)
+        ctx.fit_models(d_fj, Jf, d_smp, S, sweeps, d_theta, d_rm)
+        ctx.sync()
+        a = ev()
+        for _ in range(3):
+            ctx.fit_models(d_fj, Jf, d_smp, S, sweeps, d_theta, d_rm)
+        b = ev()
+        torch.cuda.synchronize()
+        rm = d_rm.cpu().numpy().reshape(Jf, 2)
+        fit_ms = a.elapsed_time(b) / 3
+        fit = {"model_types": Jf, "samples_per_model": S, "sweeps": sweeps, "ms": fit_ms, "fits_per_sec": Jf / (fit_ms * 1e-3),
+               "rmsle_before_median": float(np.median(rm[:, 0])), "rmsle_after_median": float(np.median(rm[:, 1])),
+               "what": "rubick_fit_models: 7 coefficients per model type by RMSLE over noisy samples (sigma 0.03) of this run's candidate table"}
+
     # event-driven run: every arrival / completion re-plans all active jobs (rank 0 only)
     events = None
     if args.events > 0 and rank == 0:
@@ -400,6 +432,7 @@ def main():
         "best_plan_roofline": {"bound": "hbm", "achieved": best_gbs, "peak": peak, "unit": "GB/s", "frac": best_gbs / peak},
         "events": events,
         "min_resources_ms": minres_ms,
+        "fit": fit,
         "round": {"steps": int(round_steps[0]), "latency_ms": float(stage_ms[3]),
                   "us_per_step": float(1e3 * stage_ms[3] / max(1, round_steps[0]))},
     }

@@ -13,17 +13,18 @@
 // they are the same numbers in any implementation; only pow / log inside the model may differ in the
 // last bits, which matters to a decision only when it sits within rounding of its threshold.
 //
-// Double precision throughout.  Eight lanes work on one model: lane q evaluates the q-th candidate of the
-// parameter being moved over all samples (sequential sum, sample order), lane 0 of the group then walks
-// the eight errors in order; a warp holds four models.  The work is a few thousand model evaluations
-// per fit, bound by the FP64 pipe and by pow / log.
+// Double precision throughout.  One warp per model: lane q + 8 * part evaluates the q-th of the eight
+// candidates of the parameter being moved on the samples i = part (mod 4); the four partial sums of a
+// candidate are added pairwise by two shuffles, then every lane walks the eight errors in candidate order.
+// The work is a few thousand model evaluations per fit, bound by latency of the FP64 pipe and pow / log.
 
 #include "rubick_internal.cuh"
 
 namespace rubick {
 
 constexpr int FIT_PARAMS = 7;
-constexpr int FIT_LANES = 8;          // candidates per parameter move = lanes per model
+constexpr int FIT_LANES = 8;          // candidates per parameter move
+constexpr int FIT_PARTS = 4;          // lanes that share the samples of one candidate
 constexpr double FIT_EPS = 1e-9;
 
 struct FitEnv {
@@ -84,21 +85,25 @@ __device__ double model_thr(const rubick_job &jb, const double *th, const FitEnv
     return bb / T_iter;
 }
 
+// Sum of squared log errors over all samples; the lanes that differ only in `part` hold the same th[] and
+// end up with the same total (pairwise sums of their partial sums).  Warp-wide.
 __device__ double sum_sq_log_err(const rubick_job &jb, const double *th, const FitEnv &ev, const QuadDesc *__restrict__ quads,
-                                 const rubick_sample *__restrict__ smp, int S, int P, int *n_out)
+                                 const rubick_sample *__restrict__ smp, int S, int P, int part, int *n_out)
 {
     double sse = 0.0; int n = 0;
-    for (int i = 0; i < S; ++i) {
+    for (int i = part; i < S; i += FIT_PARTS) {
         const rubick_sample x = smp[i];
         if (x.plan < 0 || x.plan >= P) continue;
         const double e = log1p(model_thr(jb, th, ev, quads, x.plan, double(x.cores))) - log1p(x.thr);
         sse += e * e; ++n;
     }
-    if (n_out) *n_out = n;
+    sse += __shfl_xor_sync(0xffffffffu, sse, 8);
+    sse += __shfl_xor_sync(0xffffffffu, sse, 16);
+    if (n_out) { n += __shfl_xor_sync(0xffffffffu, n, 8); n += __shfl_xor_sync(0xffffffffu, n, 16); *n_out = n; }
     return sse;
 }
 
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(64)
 fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict__ quads, int P,
                   const rubick_job *__restrict__ jobs, int J, const rubick_sample *__restrict__ samples, int S,
                   int sweeps, double *__restrict__ theta_out, double *__restrict__ rmsle_out)
@@ -107,8 +112,8 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
     const double hi[FIT_PARAMS] = {16.0, 16.0, 1e-9, 1e-6, 16.0, 16.0, 10.0};
     const int lane = threadIdx.x & 31;
     const int q = lane & (FIT_LANES - 1);                       // candidate this lane evaluates
-    const int group_base = lane & ~(FIT_LANES - 1);             // first lane of this model's group
-    const int j = (blockIdx.x * blockDim.x + threadIdx.x) / FIT_LANES;
+    const int part = lane >> 3;                                 // its share of the samples
+    const int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const bool live = j < J;
     const int jj = live ? j : 0;
     const rubick_job jb = jobs[jj];
@@ -122,7 +127,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
         if (th[p] > hi[p]) th[p] = hi[p];
     }
     int n = 0;
-    double cur = sum_sq_log_err(jb, th, ev, quads, smp, S, P, &n);
+    double cur = sum_sq_log_err(jb, th, ev, quads, smp, S, P, part, &n);
     const double rmsle0 = n > 0 ? sqrt(cur / n) : 0.0;
     double M = sqrt(2.0) * sqrt(sqrt(2.0));
     const int e_of_q = (q & 1) ? ((q >> 1) + 1) : -((q >> 1) + 1);     // q = 0..7 -> -1, +1, -2, +2, -3, +3, -4, +4
@@ -139,20 +144,21 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
             double v = e_of_q > 0 ? base * mul[e_of_q] : base / mul[-e_of_q];
             if (v < lo[p]) v = lo[p];
             if (v > hi[p]) v = hi[p];
-            double sse = 0.0;
-            if (v != base && n > 0) { th[p] = v; sse = sum_sq_log_err(jb, th, ev, quads, smp, S, P, nullptr); th[p] = base; }
+            th[p] = v;
+            const double sse = sum_sq_log_err(jb, th, ev, quads, smp, S, P, part, nullptr);
+            th[p] = base;
             // the eight errors in candidate order, as one after the other would see them
             double best = cur, best_v = base;
 #pragma unroll
             for (int k = 0; k < FIT_LANES; ++k) {
-                const double vk = __shfl_sync(0xffffffffu, v, group_base + k);
-                const double sk = __shfl_sync(0xffffffffu, sse, group_base + k);
+                const double vk = __shfl_sync(0xffffffffu, v, k);
+                const double sk = __shfl_sync(0xffffffffu, sse, k);
                 if (vk != base && n > 0 && sk < best * (1.0 - FIT_EPS)) { best = sk; best_v = vk; }
             }
             th[p] = best_v; cur = best;
         }
-        // pattern moves: every lane of the group computes the same thing
-        for (int rep = 0; rep < 4 && n > 0; ++rep) {
+        // pattern moves: every lane computes the same thing on its share of the samples
+        for (int rep = 0; rep < 4 && n > 0; ++rep) {        // (uniform over the warp: all lanes hold the same th and cur)
             double keep[FIT_PARAMS]; bool moved = false;
 #pragma unroll
             for (int p = 0; p < FIT_PARAMS; ++p) {
@@ -164,7 +170,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
                 th[p] = v;
             }
             if (!moved) break;
-            const double sse = sum_sq_log_err(jb, th, ev, quads, smp, S, P, nullptr);
+            const double sse = sum_sq_log_err(jb, th, ev, quads, smp, S, P, part, nullptr);
             if (sse < cur * (1.0 - FIT_EPS)) {
                 cur = sse;
 #pragma unroll
@@ -177,7 +183,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
         }
         if (r & 1) M = sqrt(M);
     }
-    if (live && q == 0) {
+    if (live && lane == 0) {
 #pragma unroll
         for (int p = 0; p < FIT_PARAMS; ++p) theta_out[size_t(j) * FIT_PARAMS + p] = th[p];
         rmsle_out[2 * size_t(j)] = rmsle0;
@@ -192,7 +198,7 @@ cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, int P, co
     FitEnv ev;
     ev.B_intra = env.B_intra; ev.B_inter = env.B_inter; ev.B_pcie = env.B_pcie; ev.e = double(env.bytes_per_elem);
     ev.Gn = env.gpus_per_node; ev.strict = env.strict_zero_dp_only ? 1 : 0;
-    const int threads = 128, per_block = threads / FIT_LANES;
+    const int threads = 64, per_block = threads / 32;
     fit_models_kernel<<<(J + per_block - 1) / per_block, threads, 0, st>>>(ev, d_quads, P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle);
     return cudaGetLastError();
 }

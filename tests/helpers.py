@@ -37,27 +37,4 @@ def requests_for(cfg, group_off, guaranteed_share=0.5):
     return np.stack([rq["g_idx"], rq["c_idx"], rq["m_idx"], plan], axis=1).astype(np.int64)
 
 
-def fit_samples(cfg, plans, thr, feas, picks, g_max=8, noisy=True):
-    """Measured samples for model fitting from a candidate table `thr` [J, C, P] (whoever computed it):
-    plans the job can run on at most g_max GPUs, the first third of the slots among offloading plans.
-    -> (plan [J, S] int32, cores [J, S] int64, throughput [J, S] float64); unused slots have plan -1."""
-    plans = np.asarray(plans)
-    J, S = picks["rank"].shape
-    g = plans[:, 0].astype(np.int64) * plans[:, 1] * plans[:, 2]
-    sp = np.full((J, S), -1, dtype=np.int32)
-    sc = np.zeros((J, S), dtype=np.int64)
-    sy = np.zeros((J, S), dtype=np.float64)
-    cl = np.asarray(cfg["c_levels"])
-    for j in range(J):
-        ok = (thr[j, 0] > 0) & (feas[j] != 0) & (g <= g_max)
-        off = np.nonzero(ok & (plans[:, 5] == 1))[0]
-        non = np.nonzero(ok & (plans[:, 5] == 0))[0]
-        for i in range(S):
-            pool = off if (i < S // 3 and len(off)) else non
-            if len(pool) == 0:
-                continue
-            pl = int(pool[min(int(picks["rank"][j, i] * len(pool)), len(pool) - 1)])
-            ci = int(picks["c_idx"][j, i])
-            sp[j, i], sc[j, i] = pl, cl[ci]
-            sy[j, i] = thr[j, ci, pl] * (picks["noise"][j, i] if noisy else 1.0)
-    return sp, sc, sy
+fit_samples = workloads.fit_samples
