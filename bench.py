@@ -194,7 +194,7 @@ def main():
     ap.add_argument("--ref-jobs", type=int, default=1024, help="jobs per step of the CPU arm / baseline sample")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--events", type=int, default=200, help="scheduling events of the event-driven run (0 = skip)")
+    ap.add_argument("--events", type=int, default=1000, help="scheduling events of the event-driven run (0 = skip)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -270,3 +270,25 @@ def test_events_with_state_kept_in_the_context_match_the_oracle():
             moved = was & (want["status"] == 1) & ((want["g"] != prev["g"]) | (want["c"] != prev["c"]) | (want["plan"] != prev["plan"]))
             reconf["n_reconf"] += moved.astype(np.int32)
         prev = want
+
+
+def test_degenerate_sizes():
+    """No jobs, no active slot, one node, and the largest cluster the node state supports."""
+    cfg = workloads.make("tiny")
+    tb = tables(cfg)
+    plans, feas, cv, cp, cg = tb
+    gpu = Gpu(cfg)
+    J = len(cfg["jobs"]["P"])
+    none = np.zeros(J, dtype=np.int32)
+    want, got = both(gpu, cfg, tb, None, active=none)
+    assert_rounds_equal(got, want)
+    assert want["steps"] == 0 and not want["g"].any()
+    t = gpu.torch
+    d_out = gpu.empty(64, t.uint8)
+    steps, capped = gpu.ctx.incremental_round(None, 0, None, None, None, None, 3, 10, d_out)
+    assert steps == 0 and not capped
+    big = dict(cfg, n_nodes=4096)
+    want, got = both(gpu, big, tb, None)
+    assert_rounds_equal(got, want)
+    again_w, again_g = both(gpu, big, tb, want, T=np.full(J, 1e6), delta=np.zeros(J), nrec=np.zeros(J))
+    assert_rounds_equal(again_g, again_w)

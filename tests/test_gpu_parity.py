@@ -545,7 +545,23 @@ def test_outputs_stay_inside_their_buffers():
     gpu.ctx.min_resources(thr, feas, cv, J, rb.to_device(rec), *[r[1] for r in req_out])
     steps, _ = gpu.ctx.greedy_round(d_jobs, J, cv, cp, cg, feas, N, J * (gpu.nG + gpu.nC + 2) + 1, out, node, log)
     gpu.ctx.greedy_round_noalloc(d_jobs, J, cv, cp, cg, feas, N, 1 << 30, out, node)
+    # the incremental round from that allocation (with and without a step log), and model fitting
+    out2_b, out2 = guarded(J * rb.ASSIGN_DTYPE.itemsize); node2_b, node2 = guarded(N * rb.NODE_DTYPE.itemsize)
+    log2_b, log2 = guarded(4 * (2 * J * (gpu.nG + gpu.nC + 2) + 1))
+    rc = np.zeros(J, dtype=rb.RECONF_DTYPE)
+    rc["active"], rc["T"], rc["delta"] = (np.arange(J) % 5 != 0), 5000.0, 20.0
+    d_rc = rb.to_device(rc)
+    gpu.ctx.incremental_round(d_jobs, J, cv, cp, cg, feas, N, 2 * J * (gpu.nG + gpu.nC + 2) + 1, out2, node2, log2,
+                              d_prev=out.clone(), d_prev_nodes=node.clone(), d_reconf=d_rc)
+    gpu.ctx.incremental_round(d_jobs, J, cv, cp, cg, feas, N, 1 << 30, out2, node2, None,
+                              d_prev=out.clone(), d_prev_nodes=node.clone(), d_reconf=d_rc)
+    S = 5
+    smp = np.zeros((J, S), dtype=rb.SAMPLE_DTYPE)
+    smp["plan"], smp["cores"], smp["thr"] = np.arange(J * S).reshape(J, S) % 64, 8, 1.0
+    th_b, th = guarded(J * 7 * 8); rm_b, rm = guarded(J * 2 * 8)
+    gpu.ctx.fit_models(d_jobs, J, rb.to_device(smp), S, 3, th, rm)
     gpu.ctx.sync()
     assert steps > 0
-    for whole in [thr_b, feas_b, cv_b, cp_b, cg_b, out_b, node_b, log_b] + [g[0] for g in gains] + [r[0] for r in req_out]:
+    for whole in [thr_b, feas_b, cv_b, cp_b, cg_b, out_b, node_b, log_b, out2_b, node2_b, log2_b, th_b, rm_b] \
+            + [g[0] for g in gains] + [r[0] for r in req_out]:
         assert bool((whole[:G] == 0xA5).all()) and bool((whole[-G:] == 0xA5).all())
