@@ -122,6 +122,7 @@ struct IncrShared {
     int steps, capped;
     int changed;              // the last step changed the cluster: the first-fit table is stale
     int batch;                // this iteration sorts out hopeless exchange candidates in bulk
+    int most_c[33];           // most free cores among the nodes with at least g free GPUs (g <= 32)
     float min_slope[2];       // lowest offered slope over all nodes, GPUs / cores
     int max_free[2];          // most free GPUs / cores on any node
 };
@@ -141,39 +142,48 @@ __device__ __forceinline__ void list_remove(NodeLists &nl, int n, int j)
         if (l[i] == j) { l[i] = l[c - 1]; nl.cnt[n] = c - 1; return; }
 }
 
-// An exchange for a queued job can only work on a node whose free amounts plus everything its
-// unpinned single-node jobs hold cover the job: a cheap test that spares hopeless attempts.  Warp-wide.
-__device__ bool node_could_serve(const Space &sp, const Cluster &cl, const NodeLists &nl, const HotA *hotA,
-                                 const uint32_t *roles, int n, int g2, int c2, int lane)
+// An exchange for a queued job can only work on a node whose free amounts plus everything its unpinned
+// single-node jobs hold cover the job: a cheap test that spares hopeless attempts.  Lane i looks at node
+// base + i; returns the ballot of the nodes that pass.
+__device__ unsigned nodes_could_serve(const Space &sp, const Cluster &cl, const NodeLists &nl, const HotA *hotA,
+                                      const uint32_t *roles, int base, int g2, int c2, int lane)
 {
-    int mov_g = 0, mov_c = 0;
-    if (lane < nl.cnt[n]) {
-        const int v = nl.jobs[size_t(n) * nl.Gn + lane];
-        if (!rl_pinned(roles[v])) {
-            const uint32_t pk = hotA[v].packed;
-            mov_g = sp.g_levels[pk_gi(pk)]; mov_c = sp.c_levels[pk_ci(pk)];
+    const int n = base + lane;
+    bool ok = false;
+    if (n < cl.N) {
+        int mov_g = cl.free_g[n], mov_c = cl.free_c[n];
+        if (mov_g < g2 || mov_c < c2) {
+            const int cnt = nl.cnt[n];
+            for (int i = 0; i < cnt; ++i) {
+                const int v = nl.jobs[size_t(n) * nl.Gn + i];
+                if (rl_pinned(roles[v])) continue;
+                const uint32_t pk = hotA[v].packed;
+                mov_g += sp.g_levels[pk_gi(pk)]; mov_c += sp.c_levels[pk_ci(pk)];
+            }
         }
+        ok = mov_g >= g2 && mov_c >= c2;
     }
-    mov_g = __reduce_add_sync(0xffffffffu, mov_g) + cl.free_g[n];
-    mov_c = __reduce_add_sync(0xffffffffu, mov_c) + cl.free_c[n];
-    return mov_g >= g2 && mov_c >= c2;
+    return __ballot_sync(0xffffffffu, ok);
 }
 
-// Lowest slope the single-node jobs of node n offer for GPUs and for cores (+inf when nobody offers).
-// An exchange that has to reclaim a resource on n fails at its first step unless the candidate's gain
-// exceeds this.  Warp-wide.
+// Lowest slope the single-node jobs of node n offer for GPUs and for cores (+inf when nobody offers), and
+// the GPUs and cores its unpinned single-node jobs hold.  An exchange whose first step has to reclaim a
+// resource on n fails there unless the candidate's gain exceeds the lowest slope, and it can never take
+// more than what those jobs hold.  Warp-wide.
 __device__ void node_min_slopes(const Space &sp, const Cluster &cl, const NodeLists &nl, const float *__restrict__ cv,
                                 const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
                                 const uint32_t *__restrict__ feas, const HotA *hotA, const HotB *hotB, const uint32_t *roles,
-                                int n, int lane, float &ms_g, float &ms_c)
+                                int n, int lane, float &ms_g, float &ms_c, int &held_g, int &held_c)
 {
     const float inf = __int_as_float(0x7f800000);
     float s[2] = {inf, inf};
+    int hg = 0, hc = 0;
     if (lane < nl.cnt[n]) {
         const int v = nl.jobs[size_t(n) * nl.Gn + lane];
         const uint32_t vr = roles[v];
         if (!rl_pinned(vr)) {
             JobRegs vs; vs.a = hotA[v]; vs.b = hotB[v];
+            hg = sp.g_levels[pk_gi(vs.a.packed)]; hc = sp.c_levels[pk_ci(vs.a.packed)];
 #pragma unroll
             for (int r = 0; r < 2; ++r) {
                 Offer of = shrink_offer(sp, cv, cp, cg, v, vs, vr, r);
@@ -191,6 +201,7 @@ __device__ void node_min_slopes(const Space &sp, const Cluster &cl, const NodeLi
         s[1] = fminf(s[1], __shfl_xor_sync(0xffffffffu, s[1], k));
     }
     ms_g = s[0]; ms_c = s[1];
+    held_g = __reduce_add_sync(0xffffffffu, hg); held_c = __reduce_add_sync(0xffffffffu, hc);
 }
 
 // Exchange attempt of job j for (gi2, ci2) on node n; warp 0, all lanes.  cand[r] = j's gain per unit
@@ -309,7 +320,7 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
     __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];
 
     // shared layout: free_m [N] i64 | free_g [N] | free_c [N] | owner [N] | list counts [N] | ff [n_small * nC] |
-    // min slopes [2][N] | dirty [N]
+    // min slopes [2][N] | dirty [N] | held [2][N]
     Cluster cl;
     cl.N = N;
     cl.free_m = reinterpret_cast<int64_t *>(smem_raw);
@@ -325,6 +336,8 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
     float *ms_g = reinterpret_cast<float *>(cl.ff + n_ff);      // [N] lowest offered GPU slope on the node
     float *ms_c = ms_g + N;                                     // [N] same for cores
     int32_t *dirty = reinterpret_cast<int32_t *>(ms_c + N);     // [N] the node changed since its slopes were worked out
+    int32_t *held_g = dirty + N;                                // [N] GPUs held by the node's unpinned single-node jobs
+    int32_t *held_c = held_g + N;                               // [N] their cores
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int mt = sp.nM - 1;
@@ -454,9 +467,14 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
                     }
                     __syncwarp();
                 } else if (sp.g_levels[gi] <= sp.Gn) {
-                    for (int n = 0; n < N && !placed; ++n)
-                        if (node_could_serve(sp, cl, nl, hotA, roles, n, sp.g_levels[gi], sp.c_levels[cmin], lane))
+                    for (int nb = 0; nb < N && !placed; nb += 32) {
+                        unsigned todo2 = nodes_could_serve(sp, cl, nl, hotA, roles, nb, sp.g_levels[gi], sp.c_levels[cmin], lane);
+                        while (todo2 && !placed) {
+                            const int n = nb + __ffs(todo2) - 1;
+                            todo2 &= todo2 - 1;
                             placed = exchange_warp(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, j, gi, cmin, n, true, 0.0f, 0.0f, false, lane);
+                        }
+                    }
                 }
                 if (placed) {
                     if (lane == 0 && n_tenants > 0) { rem_q[2 * tn] -= sp.g_levels[gi]; rem_q[2 * tn + 1] -= sp.c_levels[cmin]; }
@@ -496,19 +514,20 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
     __syncthreads();
     for (;;) {
         if (sh.changed) {
-            for (int e = warp; e <= n_ff; e += ROUND_WARPS) {
-                if (e == n_ff) {
-                    int cnt = 0;
-                    for (int nb = 0; nb < N; nb += 32) {
-                        const int n = nb + lane;
-                        cnt += __popc(__ballot_sync(0xffffffffu, n < N && cl.free_g[n] == sp.Gn));
-                    }
-                    if (lane == 0) sh.n_empty = cnt;
-                } else {
-                    const int gi = e / sp.nC, ci = e - gi * sp.nC;
-                    const int n = first_fit_warp(cl, sp.g_levels[gi], sp.c_levels[ci], lane);
-                    if (lane == 0) cl.ff[e] = n;
-                }
+            // an increment of (g, c) on one node fits somewhere exactly when the most free cores among the nodes
+            // with at least g free GPUs reach c; the table only has to say "fits" (>= 0) or not
+            for (int g = tid; g <= sp.Gn; g += ROUND_THREADS) sh.most_c[g] = -1;
+            if (tid == 0) sh.n_empty = 0;
+            __syncthreads();
+            for (int n = tid; n < N; n += ROUND_THREADS) {
+                const int fg = cl.free_g[n], fc = cl.free_c[n];
+                for (int g = 1; g <= fg; ++g) atomicMax(&sh.most_c[g], fc);
+                if (fg == sp.Gn) atomicAdd(&sh.n_empty, 1);
+            }
+            __syncthreads();
+            for (int e = tid; e < n_ff; e += ROUND_THREADS) {
+                const int gi = e / sp.nC, ci = e - gi * sp.nC;
+                cl.ff[e] = sh.most_c[sp.g_levels[gi]] >= sp.c_levels[ci] ? 0 : -1;
             }
         }
         __syncthreads();
@@ -565,9 +584,9 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
             // (a) lowest offered slopes of the nodes that changed
             for (int n = warp; n < N; n += ROUND_WARPS)
                 if (dirty[n]) {
-                    float g0, c0;
-                    node_min_slopes(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, n, lane, g0, c0);
-                    if (lane == 0) { ms_g[n] = g0; ms_c[n] = c0; dirty[n] = 0; }
+                    float g0, c0; int hg, hc;
+                    node_min_slopes(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, n, lane, g0, c0, hg, hc);
+                    if (lane == 0) { ms_g[n] = g0; ms_c[n] = c0; held_g[n] = hg; held_c[n] = hc; dirty[n] = 0; }
                 }
             __syncthreads();
             // (b) over all nodes: lowest slopes, most free GPUs / cores
@@ -597,8 +616,8 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
             }
             // (c) a candidate is hopeless when its exchange is sure to fail at the first step: no node (its own
             // node, for a running job) offers the resource below its gain.  Best candidate that is not hopeless:
-            const float all_g = sh.min_slope[0], all_c = sh.min_slope[1];
-            const int most_g = sh.max_free[0], most_c = sh.max_free[1];
+            const float all_g = sh.min_slope[0];
+            const int most_g = sh.max_free[0];
             auto hopeless = [&](int j, const HotA &a, int type) -> bool {
                 const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
                 const int gi2 = type == 0 ? pk_next_gi(a.packed) : gi;
@@ -607,13 +626,9 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
                     if (sp.g_levels[gi] > sp.Gn) return true;
                     return type == 0 ? !(a.gain_g > ms_g[a.node]) : !(a.gain_c > ms_c[a.node]);
                 }
-                if (most_g < sp.g_levels[gi2] && !(a.gain_g > all_g)) return true;
-                if (most_c < sp.c_levels[ci]) {
-                    const float v2 = cv[curve_idx(sp, j, gi2, ci, mt)];
-                    const float cand_c = __fdiv_rn(__fsub_rn(__fmul_rn(hotB[j].w, v2), 0.0f), float(sp.c_levels[ci]));
-                    if (!(cand_c > all_c)) return true;
-                }
-                return false;
+                // a queued job reclaims GPUs first: where every node lacks them, the first step decides.  (Its
+                // cores come second and may be freed by a preemption of the GPU phase: no shortcut there.)
+                return most_g < sp.g_levels[gi2] && !(a.gain_g > all_g);
             };
             unsigned long long live[2] = {0ull, 0ull};
             for (int j = tid; j < J; j += ROUND_THREADS) {
@@ -714,9 +729,24 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
                     } else {
                         const float v2 = cv[curve_idx(sp, j, gi2, ci2, mt)];
                         cand_c = __fdiv_rn(__fsub_rn(__fmul_rn(b.w, v2), 0.0f), float(sp.c_levels[ci2]));
-                        for (int n = 0; n < N && !ok; ++n) {
-                            if (!node_could_serve(sp, cl, nl, hotA, roles, n, sp.g_levels[gi2], sp.c_levels[ci2], lane)) continue;
-                            ok = exchange_warp(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, j, gi2, ci2, n, false, cand_g, cand_c, true, lane);
+                        const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+                        for (int nb = 0; nb < N && !ok; nb += 32) {
+                            unsigned todo;
+                            if (bulk) {
+                                // the per-node figures are fresh: enough free plus held amounts and, where GPUs
+                                // are short, a first offer below the gain
+                                const int n = nb + lane;
+                                const bool worth = n < N && cl.free_g[n] + held_g[n] >= g2 && cl.free_c[n] + held_c[n] >= c2
+                                                   && (cl.free_g[n] >= g2 || cand_g > ms_g[n]);
+                                todo = __ballot_sync(0xffffffffu, worth);
+                            } else {
+                                todo = nodes_could_serve(sp, cl, nl, hotA, roles, nb, g2, c2, lane);
+                            }
+                            while (todo && !ok) {
+                                const int n2 = nb + __ffs(todo) - 1;
+                                todo &= todo - 1;
+                                ok = exchange_warp(sp, cl, nl, cv, cp, cg, feas, hotA, hotB, roles, j, gi2, ci2, n2, false, cand_g, cand_c, true, lane);
+                            }
                         }
                     }
                     if (ok) { a = hotA[j]; b = hotB[j]; if (lane == 0) dirty[a.node] = 1; }
@@ -769,7 +799,7 @@ incremental_round_kernel(const __grid_constant__ Space sp, const rubick_job *__r
 
 static size_t incr_smem(const Space &sp, int N)
 {
-    return (size_t(N) * 36 + size_t(sp.n_small) * sp.nC * 4 + 15) & ~size_t(15);
+    return (size_t(N) * 44 + size_t(sp.n_small) * sp.nC * 4 + 15) & ~size_t(15);
 }
 
 // scratch: HotA [J] | HotB [J] | roles [J] | whole-node counts [J] | node lists [N][Gn]
