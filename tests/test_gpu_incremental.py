@@ -8,7 +8,7 @@ from gpu_util import Gpu, assert_rounds_equal, has_cuda, incremental_on_tables
 from helpers import GIB, env, one_job, stack_jobs
 from paper_2408_08586_b200 import binding as rb
 from paper_2408_08586_b200 import workloads
-from test_oracle_incremental import event_config, random_events
+from test_oracle_incremental import event_config, preemption_frees_cores_case, random_events
 from test_oracle_sched import concave_instance, tables
 
 pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not has_cuda(), reason="needs a CUDA device")]
@@ -292,3 +292,18 @@ def test_degenerate_sizes():
     assert_rounds_equal(got, want)
     again_w, again_g = both(gpu, big, tb, want, T=np.full(J, 1e6), delta=np.zeros(J), nrec=np.zeros(J))
     assert_rounds_equal(again_g, again_w)
+
+
+def test_cores_freed_by_a_preemption_are_seen_with_and_without_a_step_log():
+    cfg, tb, prev = preemption_frees_cores_case()
+    plans, feas, cv, cp, cg = tb
+    gpu_plans, _ = rb.enumerate_plans(cfg["g_levels"])
+    gpu = Gpu(cfg, plans=gpu_plans)
+    feas_full = np.zeros((2, gpu.P), dtype=np.uint32)
+    feas_full[:, 0] = 1
+    tb = (None, feas_full, cv, cp, cg)
+    want, got = both(gpu, cfg, tb, prev)
+    assert_rounds_equal(got, want)
+    assert list(want["status"]) == [0, 1]
+    bulk = incremental_on_tables(gpu, cfg["jobs"], cv, cp, cg, feas_full, 1, prev, want_log=False)
+    assert_rounds_equal(bulk, want)

@@ -231,3 +231,31 @@ def test_inconsistent_previous_state_is_refused(tiny):
     bad["status"][:] = first["status"]
     if (first["status"] == 1).sum() * 32 > tiny["env"]["cpus_per_node"]:
         assert incr(tiny, tb, bad)["steps"] is None
+
+
+def preemption_frees_cores_case():
+    """One node with 8 GPUs and 8 cores, all held by best-effort job 0, which runs on 8 GPUs only (value 8
+    with 8 cores, 2 with 4).  Queued job 1 wants 2 GPUs and 4 cores for a value of 6: 3 per GPU, 1.5 per core."""
+    cv = np.zeros((2, 4, 2, 1), dtype=np.float32)
+    cg = np.zeros((2, 4, 2, 1), dtype=np.int32)
+    cp = np.full((2, 4, 2, 1), -1, dtype=np.int32)
+    gl, cl, ml = np.array([1, 2, 4, 8]), np.array([4, 8]), np.array([GIB])
+    cv[0, 3, :, 0] = [2, 8]; cg[0, 3, :, 0] = 8; cp[0, 3, :, 0] = 0
+    cv[1, 1:, :, 0] = 6; cg[1, 1:, :, 0] = 2; cp[1, 1:, :, 0] = 0
+    feas = np.ones((2, 1), dtype=np.uint32)
+    jobs = stack_jobs(one_job(host_base_bytes=0), one_job(host_base_bytes=0))
+    cfg = dict(jobs=jobs, env=env(cpus_per_node=8), g_levels=gl, c_levels=cl, m_levels=ml, n_nodes=1)
+    prev = dict(g=np.array([8, 0]), c=np.array([8, 0]), m_bytes=np.array([GIB, 0]), plan=np.array([0, -1]),
+                first_node=np.array([0, -1]), n_nodes=np.array([1, 0]), status=np.array([1, 0]), m_level=np.array([0, -1]),
+                thr=np.array([8, 0], np.float32), node=np.array([[0, 0, 0, -1]]))
+    return cfg, (None, feas, cv, cp, cg), prev
+
+
+def test_a_preemption_in_the_gpu_phase_frees_the_cores_the_newcomer_needs():
+    """Job 0's cores cost 1.5 each, not below the newcomer's 1.5 per core, so cores alone could not be taken;
+    but its GPUs cost 1 each against a gain of 3, it has no smaller GPU count, so it is preempted, and its
+    cores come free with it."""
+    cfg, tb, prev = preemption_frees_cores_case()
+    r = incr(cfg, tb, prev, want_log=True)
+    assert list(r["status"]) == [0, 1] and list(r["g"]) == [0, 2] and list(r["c"]) == [0, 4]
+    assert r["log"][0] == (1 << 3) | (1 << 2) | 1
