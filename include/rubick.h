@@ -213,6 +213,14 @@ int rubick_eval_candidates(rubick_ctx *ctx, const rubick_job *d_jobs, int J, flo
 int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
                      float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g);
 
+/* rubick_eval_candidates followed by rubick_best_plan in one pass that never writes the candidate
+ * table: the mask (d_feas, J*P words) and the curves (d_best_*, J*G*C*M entries each) are bit-identical
+ * to what the two calls produce; only the J*C*P throughputs are not kept.  For callers that want the
+ * curves alone (a scheduling round): about 8 bytes per candidate of memory traffic less.
+ * d_jobs and d_feas 16-byte aligned; flags as rubick_best_plan. */
+int rubick_curves(rubick_ctx *ctx, const rubick_job *d_jobs, int J, unsigned flags, uint32_t *d_feas,
+                  float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g);
+
 /* Marginal gain ("slope", Section 5.2) of the next GPU and the next CPU increment of every job in
  * state d_state (fields g, c, thr are read; g == 0 means nothing held): the weighted curve gain
  * per added GPU up to the smallest level that strictly improves on the present value, and per

@@ -64,7 +64,7 @@ def make_cluster(n_nodes, quota=None):
 
 
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
-           "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_marginal_gain",
+           "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_curves", "rubick_marginal_gain",
            "rubick_min_resources", "rubick_fit_models",
            "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
            "rubick_schedule_round_host", "rubick_incremental_event_host"]
@@ -97,6 +97,7 @@ def lib():
         L.rubick_set_space.argtypes = [vp, vp, ip, C.POINTER(Grid)]
         L.rubick_eval_candidates.argtypes = [vp, vp, ip, vp, vp]
         L.rubick_best_plan.argtypes = [vp, vp, vp, ip, C.c_uint, vp, vp, vp]
+        L.rubick_curves.argtypes = [vp, vp, ip, C.c_uint, vp, vp, vp, vp]
         L.rubick_marginal_gain.argtypes = [vp, vp, ip, vp, vp, vp, vp, vp, vp]
         L.rubick_min_resources.argtypes = [vp, vp, vp, vp, ip, vp, vp, vp, vp]
         L.rubick_fit_models.argtypes = [vp, vp, ip, vp, ip, ip, vp, vp]
@@ -216,6 +217,10 @@ class Context:
     def best_plan(self, d_thr, d_feas, J, d_best_val, d_best_plan, d_best_g, flags=0):
         return self._check(lib().rubick_best_plan(self._h, _ptr(d_thr), _ptr(d_feas), int(J), int(flags),
                                                   _ptr(d_best_val), _ptr(d_best_plan), _ptr(d_best_g)))
+
+    def curves(self, d_jobs, J, d_feas, d_best_val, d_best_plan, d_best_g, flags=0):
+        return self._check(lib().rubick_curves(self._h, _ptr(d_jobs), int(J), int(flags), _ptr(d_feas), _ptr(d_best_val),
+                                               _ptr(d_best_plan), _ptr(d_best_g)))
 
     def marginal_gain(self, d_jobs, J, d_curve_val, d_state, d_gain_gpu, d_gain_cpu, d_next_g, d_next_c):
         return self._check(lib().rubick_marginal_gain(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_state),

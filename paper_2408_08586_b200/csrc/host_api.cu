@@ -268,6 +268,22 @@ int rubick_best_plan(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_feas
     return RUBICK_OK;
 }
 
+int rubick_curves(rubick_ctx *ctx, const rubick_job *d_jobs, int J, unsigned flags, uint32_t *d_feas,
+                  float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g)
+{
+    CHECK_CTX(ctx);
+    int rc = check_ready(ctx, J);
+    if (rc) return rc;
+    if (J == 0) return RUBICK_OK;
+    if (!d_jobs || !d_feas || !d_best_val || !d_best_plan || !d_best_g) return fail(ctx, RUBICK_EINVAL, "null pointer");
+    if ((reinterpret_cast<uintptr_t>(d_feas) & 15) || (reinterpret_cast<uintptr_t>(d_jobs) & 15))
+        return fail(ctx, RUBICK_EINVAL, "d_jobs and d_feas must be 16-byte aligned");
+    if (flags & ~RUBICK_BEST_RAW) return fail(ctx, RUBICK_EINVAL, "unknown flag");
+    CUDA_TRY(ctx, launch_curves(ctx->space, ctx->d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g, ctx->stream),
+             "launch curves");
+    return RUBICK_OK;
+}
+
 int rubick_marginal_gain(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_curve_val,
                          const rubick_assignment *d_state,
                          float *d_gain_gpu, float *d_gain_cpu, int32_t *d_next_g, int32_t *d_next_c)
@@ -431,17 +447,13 @@ int rubick_incremental_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
     return finish_round(ctx, h_steps);
 }
 
-// candidate table, mask and curves for d_jobs[0..J) into context scratch, in job tiles whose
-// throughput rows are produced and consumed back to back
+// mask and curves for d_jobs[0..J) into context scratch
 static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
 {
     const Space &sp = ctx->space;
     ctx->inc_J = 0;                     // the table scratch is about to be rewritten
-    const int tile = ctx->tile_jobs < J ? ctx->tile_jobs : J;
     int rc;
-    if ((rc = ensure(ctx, ctx->d_thr, ctx->cap_thr, size_t(tile) * sp.nC * sp.P))) return rc;
     if ((rc = ensure(ctx, ctx->d_feas, ctx->cap_feas, size_t(J) * sp.P))) return rc;
-    if ((rc = ensure(ctx, ctx->d_best_todo, ctx->cap_best_todo, size_t(tile) + 1))) return rc;
     const size_t curve = size_t(J) * sp.nG * sp.nC * sp.nM;
     if (curve > ctx->cap_curve) {
         size_t c1 = ctx->cap_curve, c2 = ctx->cap_curve, c3 = ctx->cap_curve;
@@ -450,15 +462,8 @@ static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
         if ((rc = ensure(ctx, ctx->d_cg, c3, curve))) return rc;
         ctx->cap_curve = curve;
     }
-    const size_t per_job = size_t(sp.nG) * sp.nC * sp.nM;
-    for (int j0 = 0; j0 < J; j0 += tile) {
-        const int n = J - j0 < tile ? J - j0 : tile;
-        CUDA_TRY(ctx, launch_eval(sp, ctx->d_quads, d_jobs + j0, n, ctx->d_thr, ctx->d_feas + size_t(j0) * sp.P, ctx->stream), "launch eval_candidates");
-        CUDA_TRY(ctx, launch_best(sp, ctx->d_thr, ctx->d_feas + size_t(j0) * sp.P, n, 0u, ctx->d_cv + j0 * per_job,
-                                  ctx->d_cp + j0 * per_job, ctx->d_cg + j0 * per_job, ctx->d_status, ctx->d_best_todo,
-                                  ctx->num_sms, ctx->stream),
-                 "launch best_plan");
-    }
+    // a round only needs the curves: the one-pass kernel never writes the candidate table
+    CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, d_jobs, J, 0u, ctx->d_feas, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->stream), "launch curves");
     return RUBICK_OK;
 }
 
@@ -501,14 +506,12 @@ static int enqueue_tables_of(rubick_ctx *ctx, const rubick_job *d_jobs, const in
     const Space &sp = ctx->space;
     const size_t per_job = size_t(sp.nG) * sp.nC * sp.nM;
     for (int i = 0; i < n;) {
-        int run = 1;                    // consecutive slots go through the kernels together
-        while (i + run < n && h_slots[i + run] == h_slots[i] + run && run < ctx->tile_jobs) ++run;
+        int run = 1;                    // consecutive slots go through the kernel together
+        while (i + run < n && h_slots[i + run] == h_slots[i] + run) ++run;
         const int s0 = h_slots[i];
-        CUDA_TRY(ctx, launch_eval(sp, ctx->d_quads, d_jobs + s0, run, ctx->d_thr, ctx->d_feas + size_t(s0) * sp.P, ctx->stream), "launch eval_candidates");
-        CUDA_TRY(ctx, launch_best(sp, ctx->d_thr, ctx->d_feas + size_t(s0) * sp.P, run, 0u, ctx->d_cv + s0 * per_job,
-                                  ctx->d_cp + s0 * per_job, ctx->d_cg + s0 * per_job, ctx->d_status, ctx->d_best_todo,
-                                  ctx->num_sms, ctx->stream),
-                 "launch best_plan");
+        CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, d_jobs + s0, run, 0u, ctx->d_feas + size_t(s0) * sp.P, ctx->d_cv + s0 * per_job,
+                                    ctx->d_cp + s0 * per_job, ctx->d_cg + s0 * per_job, ctx->stream),
+                 "launch curves");
         i += run;
     }
     return RUBICK_OK;
@@ -544,7 +547,6 @@ int rubick_incremental_event_host(rubick_ctx *ctx, const rubick_job *h_jobs, int
     } else {
         for (int i = 0; i < n_changed; ++i)
             CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_inc_jobs + h_changed[i], h_jobs + h_changed[i], sizeof(rubick_job), cudaMemcpyHostToDevice, ctx->stream), "copy a job to device");
-        if ((rc = ensure(ctx, ctx->d_best_todo, ctx->cap_best_todo, size_t(ctx->tile_jobs) + 1))) return rc;
         if ((rc = enqueue_tables_of(ctx, ctx->d_inc_jobs, h_changed, n_changed))) return rc;
     }
     if (h_reconf) CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_inc_reconf, h_reconf, size_t(J) * sizeof(rubick_reconf), cudaMemcpyHostToDevice, ctx->stream), "copy gate inputs to device");

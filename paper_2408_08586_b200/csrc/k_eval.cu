@@ -98,21 +98,16 @@ __device__ __forceinline__ int first_level(const Space &sp, int64_t need)
     return lo;
 }
 
-__global__ void __launch_bounds__(256)
-eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads,
-                       const rubick_job *__restrict__ jobs, int J, float *__restrict__ thr,
-                       uint32_t *__restrict__ feas)
+// Everything one thread does for (job j, quad q): the feasibility words (stored by active threads) and the
+// four throughputs of every CPU level, handed to emit(ci, float4, words) in ascending level order.  Whole warps
+// must call this together with the quads of a warp consecutive and starting at a multiple of four (the
+// four ZeRO stages of a (d, t, p) triple trade results); `active` = false for mirror threads past the end.
+// Returns the four feasibility words when KEEP_WORDS (zeros otherwise).
+template <bool KEEP_WORDS, class Emit>
+__device__ __forceinline__ uint4 eval_quad(const Space &sp, const QuadDesc *__restrict__ quads,
+                                           const rubick_job *__restrict__ jobs, int j, int q, bool active,
+                                           uint32_t *__restrict__ feas, Emit &&emit)
 {
-    // J * Q < 2^31 is checked by the host entry point
-    // Threads past the end mirror the last valid thread and store nothing: the CPU-level walk below
-    // exchanges values between the four lanes of a (d, t, p) triple, so whole warps stay converged.
-    const uint32_t total = uint32_t(J) * uint32_t(sp.Q);
-    const uint32_t gid_raw = blockIdx.x * blockDim.x + threadIdx.x;
-    const bool active = gid_raw < total;
-    const uint32_t gid = active ? gid_raw : total - 1;
-    const int j = int(gid / uint32_t(sp.Q));
-    const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
-
     const JobRegs jb = load_job(jobs + j);
     const uint2 qraw = __ldg(reinterpret_cast<const uint2 *>(quads) + q);
     const int ld = qraw.x & 0xff, lt = (qraw.x >> 8) & 0xff, lp = (qraw.x >> 16) & 0xff, z = (qraw.x >> 24) & 0xff;
@@ -161,6 +156,7 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
     const float T_opt = jb.k_opt * Psi * (z >= 1 ? inv_d : 1.0f);
     const float bf = float(jb.b);
 
+    uint4 fw_out = make_uint4(0u, 0u, 0u, 0u);
     float4 out;
     out.x = (valid && !(disabled & 1)) ? bf / (cc0 + T_opt) : 0.0f;
     out.z = (valid && !(disabled & 4)) ? bf / (cc1 + T_opt) : 0.0f;
@@ -193,6 +189,7 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
         fw.z = (valid && !(disabled & 4) && st0 + act1 <= sp.gpu_mem) ? w0 : 0u;
         fw.w = (valid_off && !(disabled & 8) && st1 + act1 <= sp.gpu_mem) ? w1 : 0u;
         if (active) *reinterpret_cast<uint4 *>(feas + (size_t(j) * sp.P + 4 * size_t(q))) = fw;
+        if (KEEP_WORDS) fw_out = fw;
     }
 
     // ---- walk the CPU levels -------------------------------------------------------------------
@@ -201,13 +198,11 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
     // plans of the triple, so lane i evaluates it for core level 4n + i and the lanes trade results;
     // then every lane divides for ONE offload plan (stage 2 + (lane >> 1), checkpointing = lane & 1)
     // and the two lanes that own offload plans (stages 2 and 3) collect their pair.
-    float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
     const bool off0 = valid_off && !(disabled & 2), off1 = valid_off && !(disabled & 8);
     const unsigned FULL = 0xffffffffu;
     if (!__any_sync(FULL, off0 || off1)) {
-        if (active)
-            for (int ci = 0; ci < sp.nC; ++ci, row += sp.P) __stcs(reinterpret_cast<float4 *>(row), out);
-        return;
+        for (int ci = 0; ci < sp.nC; ++ci) emit(ci, out, fw_out);
+        return fw_out;
     }
     const int lane = threadIdx.x & 31, gbase = lane & ~3, zl = lane & 3;
     const float T_off = sp.e * Psi * inv_d * sp.inv_B_pcie;          // identical on the four lanes
@@ -235,11 +230,148 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
             if (c0 + cc < sp.nC) {
                 out.y = zl >= 2 ? ry : 0.0f;
                 out.w = zl >= 2 ? rw : 0.0f;
-                if (active) __stcs(reinterpret_cast<float4 *>(row), out);
-                row += sp.P;
+                emit(c0 + cc, out, fw_out);
             }
         }
     }
+    return fw_out;
+}
+
+__global__ void __launch_bounds__(256)
+eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads,
+                       const rubick_job *__restrict__ jobs, int J, float *__restrict__ thr,
+                       uint32_t *__restrict__ feas)
+{
+    // J * Q < 2^31 is checked by the host entry point
+    // Threads past the end mirror the last valid thread and store nothing: the CPU-level walk
+    // exchanges values between the four lanes of a (d, t, p) triple, so whole warps stay converged.
+    const uint32_t total = uint32_t(J) * uint32_t(sp.Q);
+    const uint32_t gid_raw = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool active = gid_raw < total;
+    const uint32_t gid = active ? gid_raw : total - 1;
+    const int j = int(gid / uint32_t(sp.Q));
+    const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
+    float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
+    eval_quad<false>(sp, quads, jobs, j, q, active, feas, [&](int ci, const float4 &out, const uint4 &) {
+        if (active) __stcs(reinterpret_cast<float4 *>(row + size_t(ci) * sp.P), out);
+    });
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Curves without the table: the evaluation above and the best-plan / sensitivity-curve step (paper
+// Section 5.2) in one kernel, for callers that only want the curves (a scheduling round).  One CTA per
+// job; thread = quad as above, but each level's four throughputs go into a reduction instead of memory:
+// per class (plans without / with offload, which share one first feasible memory level per GPU level under
+// this library's memory rule) the lanes of a warp that sit in the same GPU level reduce the value with one
+// warp reduction, a vote names the lowest lane holding it, and that lane folds (value bits << 32 | ~index)
+// into a 64-bit shared-memory maximum per (GPU level, core level); plans without offload do not depend on
+// the core count and are reduced once per GPU level.  Then thread (c, m) combines the two
+// classes for memory level m, takes the running maximum over GPU levels and stores its three outputs.
+// Same values, same ties (lowest plan index) as best_plan on the table of eval_candidates: bit-identical.
+// Nothing but the mask (4 bytes per plan) and the curves is written: the kernel is bound by the FP32 and
+// transcendental pipes instead of the table's write and read streams.
+// ------------------------------------------------------------------------------------------------------
+constexpr int CURVES_THREADS = 128;      // small CTAs: the phases of the several CTAs of an SM overlap (704 threads: 2.4 ms, 128: 1.1 ms at 16,384 jobs)
+
+__global__ void __launch_bounds__(CURVES_THREADS)
+curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads, const rubick_job *__restrict__ jobs,
+              int J, unsigned flags, uint32_t *__restrict__ feas, float *__restrict__ best_val,
+              int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    unsigned long long *keys = reinterpret_cast<unsigned long long *>(smem_raw);      // [nG][nC + 1]: offload class per core level, then the other class
+    __shared__ int s_first[2 * RUBICK_MAX_G_LEVELS];        // first feasible memory level per (GPU level, class), nM = none
+    const int j = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const unsigned FULL = 0xffffffffu;
+
+    for (int i = tid; i < sp.nG * (sp.nC + 1); i += blockDim.x) keys[i] = 0ull;
+    if (tid < sp.nG) {
+        // host-memory need of the level's plans: g processes, plus the offloaded states (as in the mask above)
+        const rubick_job *jp = jobs + j;
+        const int g = sp.g_levels[tid];
+        const int lg = 31 - __clz(g);
+        const int64_t need0 = jp->host_base_bytes << lg, need1 = need0 + 14 * int64_t(jp->P);
+        const int nshift = max(lg - sp.log2Gn, 0);
+        int f0 = sp.nM, f1 = sp.nM;
+        if (cdiv_shift(need0, nshift) <= sp.Mn) f0 = first_level(sp, need0);
+        if (cdiv_shift(need1, nshift) <= sp.Mn) f1 = first_level(sp, need1);
+        s_first[2 * tid] = f0; s_first[2 * tid + 1] = f1;
+    }
+    __syncthreads();
+
+    for (int q0 = 0; q0 < sp.Q; q0 += blockDim.x) {
+        const int q_raw = q0 + tid;
+        const bool active = q_raw < sp.Q;
+        if (q0 + (tid & ~31) >= sp.Q) continue;                 // a whole warp past the end has nothing to mirror
+        const int q = active ? q_raw : sp.Q - 1;
+        const int level = reinterpret_cast<const uint8_t *>(quads + q)[4];             // QuadDesc::g_level
+        const unsigned peers = __match_any_sync(FULL, active ? level : -1);            // lanes of the same GPU level
+        unsigned long long *kq = keys + size_t(level) * (sp.nC + 1);
+        bool any_offload = false;                               // does a lane of my group own a feasible offloading plan?
+        eval_quad<true>(sp, quads, jobs, j, q, active, feas, [&](int ci, const float4 &o, const uint4 &words) {
+            // Infeasible plans count as 0.  Quads ascend with the lane and a lane's two plans of a class with
+            // their index, so among equal values the lowest lane holds the lowest plan index: one warp
+            // reduction for the value, one vote for who holds it, and that lane alone updates the key.
+            if (ci == 0) {
+                // plans without offload do not depend on the core count: one entry per GPU level
+                const float x = words.x ? o.x : 0.0f, z = words.z ? o.z : 0.0f;
+                const unsigned be = active ? __float_as_uint(fmaxf(x, z)) : 0u;
+                const unsigned me = __reduce_max_sync(peers, be);
+                const unsigned who = __ballot_sync(peers, be == me) & peers;
+                if (me && lane == __ffs(who) - 1)
+                    atomicMax(kq + sp.nC, (static_cast<unsigned long long>(me) << 32) | (FULL - (z > x ? 4u * q + 2u : 4u * q)));
+                any_offload = (__ballot_sync(peers, active && (words.y | words.w)) & peers) != 0u;
+            }
+            if (!any_offload) return;
+            const float y = words.y ? o.y : 0.0f, w = words.w ? o.w : 0.0f;
+            const unsigned bo = active ? __float_as_uint(fmaxf(y, w)) : 0u;
+            const unsigned mo = __reduce_max_sync(peers, bo);
+            if (mo) {
+                const unsigned who = __ballot_sync(peers, bo == mo) & peers;
+                if (lane == __ffs(who) - 1)
+                    atomicMax(kq + ci, (static_cast<unsigned long long>(mo) << 32) | (FULL - (w > y ? 4u * q + 3u : 4u * q + 1u)));
+            }
+        });
+    }
+    __syncthreads();
+
+    const bool raw = (flags & RUBICK_BEST_RAW) != 0;
+    for (int cm = tid; cm < sp.nC * sp.nM; cm += blockDim.x) {
+        const int ci = cm / sp.nM, m = cm - ci * sp.nM;
+        unsigned run_v = 0u, run_i = FULL; int run_g = 0;
+        size_t o = (size_t(j) * sp.nG * sp.nC + ci) * sp.nM + m;
+        for (int g = 0; g < sp.nG; ++g, o += size_t(sp.nC) * sp.nM) {
+            const unsigned long long ke = keys[size_t(g) * (sp.nC + 1) + sp.nC], ko = keys[size_t(g) * (sp.nC + 1) + ci];
+            const bool use_e = ke && m >= s_first[2 * g], use_o = ko && m >= s_first[2 * g + 1];
+            unsigned bv = use_e ? unsigned(ke >> 32) : 0u, bi = use_e ? FULL - unsigned(ke) : FULL;
+            const unsigned vo = unsigned(ko >> 32), io = FULL - unsigned(ko);
+            const bool odd_wins = use_o && (vo > bv || (vo == bv && io < bi));
+            bv = odd_wins ? vo : bv; bi = odd_wins ? io : bi;
+            int bg = bv ? sp.g_levels[g] : 0;
+            if (!raw) {
+                const bool up = bv > run_v;
+                run_v = up ? bv : run_v; run_i = up ? bi : run_i; run_g = up ? bg : run_g;
+                bv = run_v; bi = run_i; bg = run_g;
+            }
+            best_val[o] = __uint_as_float(bv);
+            best_plan[o] = int(bi);
+            best_g[o] = bg;
+        }
+    }
+}
+
+cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J, unsigned flags,
+                          uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, cudaStream_t st)
+{
+    if (J == 0) return cudaSuccess;
+    const size_t smem = size_t(sp.nG) * (sp.nC + 1) * sizeof(unsigned long long);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(curves_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        if (e != cudaSuccess) return e;
+    }
+    curves_kernel<<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J,

@@ -101,6 +101,8 @@ int cuda_fail(rubick_ctx *ctx, cudaError_t e, const char *what);
 // launchers, one per translation unit
 cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J,
                         float *d_thr, uint32_t *d_feas, cudaStream_t st);
+cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J, unsigned flags,
+                          uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, cudaStream_t st);
 cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
                         float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, uint32_t *d_status,
                         int32_t *d_todo /* J + 1 words of scratch */, int num_sms, cudaStream_t st);

@@ -182,6 +182,26 @@ def test_best_plan_with_two_class_and_scattered_masks_in_one_batch(raw):
     assert np.array_equal(bg.cpu().numpy().reshape(sh), cg)
 
 
+@pytest.mark.parametrize("name,J", [("tiny", None), ("paper-scale", None), ("cluster-512", 203)])
+@pytest.mark.parametrize("raw", [False, True])
+def test_curves_in_one_pass_equal_table_then_best_plan(name, J, raw):
+    """rubick_curves never writes the table; mask and curves must be bit-identical to the two-call path."""
+    cfg = workloads.make(name, J=J)
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    Jn = len(cfg["jobs"]["P"])
+    flags = rb.BEST_RAW if raw else 0
+    d_jobs, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    bv, bp, bg = gpu.best(d_thr, d_feas, Jn, flags=flags)
+    n = Jn * gpu.nG * gpu.nC * gpu.nM
+    f2 = gpu.empty(Jn * gpu.P, t.int32)
+    cv, cp, cg = gpu.empty(n, t.float32), gpu.empty(n, t.int32), gpu.empty(n, t.int32)
+    gpu.ctx.curves(d_jobs, Jn, f2, cv, cp, cg, flags=flags)
+    gpu.ctx.sync()
+    assert t.equal(f2, d_feas)
+    assert t.equal(cv.view(t.int32), bv.view(t.int32)) and t.equal(cp, bp) and t.equal(cg, bg)
+
+
 def test_non_threshold_feasibility_word_is_reported():
     cfg = workloads.make("tiny")
     gpu = Gpu(cfg)
