@@ -50,6 +50,21 @@ class Gpu:
         self.ctx.sync()
         return bv, bp, bg
 
+    def assert_one_pass_curves_match(self, jobs):
+        """rubick_curves against rubick_eval_candidates + rubick_best_plan on the same jobs: bit-identical."""
+        t = self.torch
+        J = len(jobs["P"])
+        d_jobs, d_thr, d_feas = self.eval(jobs)
+        n = J * self.nG * self.nC * self.nM
+        for flags in (0, rb.BEST_RAW):
+            bv, bp, bg = self.best(d_thr, d_feas, J, flags=flags)
+            f2 = self.empty(J * self.P, t.int32)
+            cv, cp, cg = self.empty(n, t.float32), self.empty(n, t.int32), self.empty(n, t.int32)
+            self.ctx.curves(d_jobs, J, f2, cv, cp, cg, flags=flags)
+            self.ctx.sync()
+            assert t.equal(f2, d_feas)
+            assert t.equal(cv.view(t.int32), bv.view(t.int32)) and t.equal(cp, bp) and t.equal(cg, bg)
+
     def shape4(self, J):
         return (J, self.nG, self.nC, self.nM)
 

@@ -73,6 +73,7 @@ def test_strict_zero_dp_only_and_other_environments():
         plans, thr, feas, *_ = oracle_tables(cfg)
         assert np.array_equal(gpu.np_feas(d_feas, 64), feas)
         check_thr(gpu.np_thr(d_thr, 64), thr)
+        gpu.assert_one_pass_curves_match(cfg["jobs"])
 
 
 def test_hand_made_jobs_with_odd_shapes():
@@ -99,6 +100,7 @@ def test_everything_infeasible_and_single_memory_level():
     plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
     assert not feas.any() and np.array_equal(gpu.np_feas(d_feas, 4), feas)
     check_thr(gpu.np_thr(d_thr, 4), thr)                   # predictions do not depend on memory
+    gpu.assert_one_pass_curves_match(cfg["jobs"])
     bv, bp, bg = gpu.best(d_thr, d_feas, 4)
     assert not bv.cpu().numpy().any() and (bp.cpu().numpy() == -1).all() and not bg.cpu().numpy().any()
     r = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 1)
@@ -403,6 +405,7 @@ def test_disabled_plans_are_never_chosen():
     oplans, othr, ofeas, *_ = oracle_tables(cfg)
     assert np.array_equal(feas[:, ~dis], ofeas[:, ~dis])
     check_thr(thr[:, :, ~dis], othr[:, :, ~dis])
+    gpu.assert_one_pass_curves_match(cfg["jobs"])
 
 
 def test_argument_validation():
@@ -512,6 +515,7 @@ def test_odd_grid_shapes_through_every_kernel():
     got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 9)
     assert_rounds_equal(got, want)
     assert want["steps"] > 5 and (want["n_nodes"] > 1).any()
+    gpu.assert_one_pass_curves_match(cfg["jobs"])
 
 
 def test_largest_supported_grid_and_cluster():
@@ -529,6 +533,7 @@ def test_largest_supported_grid_and_cluster():
                                  4096, want_log=True)
     got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, 4096)
     assert_rounds_equal(got, want)
+    gpu.assert_one_pass_curves_match(cfg["jobs"])
     with pytest.raises(rb.RubickError):
         gpu.ctx.greedy_round(None, 0, None, None, None, None, 4097, 10, None)
     with pytest.raises(rb.RubickError):
