@@ -403,7 +403,7 @@ def main():
     cpu_baseline = None
     if not args.no_cpu_baseline:
         threads = os.cpu_count() or 1
-        J_s = min(J, 4 * args.ref_jobs)                         # a few seconds on all host cores
+        J_s = min(J, 8 * args.ref_jobs)                         # about ten seconds on all host cores
         nodes_s = max(1, N * J_s // J)
         dt, _ = oracle_sample(cfg, J_s, nodes_s, threads)
         cpu_baseline = {"value": J_s * P * C / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
