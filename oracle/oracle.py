@@ -111,11 +111,18 @@ def feas_word(jobs, j, env, plan, m_levels):
                                       _p(_i32(plan), C.c_int32), _p(ml, C.c_int64), C.c_int(len(ml))))
 
 
-def enumerate_plans(g_levels):
-    """-> (plans [P, 6] int32 = d, t, p, z, gc, off; group_off [nG + 1] int32)."""
+def enumerate_plans(g_levels, any_degrees=False):
+    """-> (plans [P, 6] int32 = d, t, p, z, gc, off; group_off [nG + 1] int32).  any_degrees: every
+    factorisation of every GPU level instead of power-of-two degrees on power-of-two levels."""
     gl = _i64(g_levels)
     off = np.zeros(len(gl) + 1, dtype=np.int32)
     dummy = np.zeros((1, 6), dtype=np.int32)
+    if any_degrees:
+        f = lib().oracle_enumerate_plans_any
+        n = f(_p(gl, C.c_int64), C.c_int(len(gl)), _p(dummy, C.c_int32), C.c_int(0), _p(off, C.c_int32))
+        plans = np.zeros((max(n, 1), 6), dtype=np.int32)
+        f(_p(gl, C.c_int64), C.c_int(len(gl)), _p(plans, C.c_int32), C.c_int(n), _p(off, C.c_int32))
+        return plans[:n], off
     n = lib().oracle_enumerate_plans(_p(gl, C.c_int64), C.c_int(len(gl)), _p(dummy, C.c_int32), C.c_int(0),
                                      _p(off, C.c_int32))
     plans = np.zeros((max(n, 1), 6), dtype=np.int32)

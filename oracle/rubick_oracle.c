@@ -288,6 +288,39 @@ int oracle_enumerate_plans(const int64_t *g_levels, int nG, int32_t *plans, int 
     return n;
 }
 
+/* The wider plan space of the paper's own experiments (a 3-GPU tensor-parallel plan in Section 7.2,
+ * GPU counts such as 12 or 24 in Table 2): for EVERY GPU level g, all ordered factorisations
+ * g = d * t * p, TP degree ascending over the divisors of g, then PP degree ascending over the
+ * divisors of g / t, then ZeRO stage, gradient checkpointing, offload.  On power-of-two levels this
+ * is the list of oracle_enumerate_plans. */
+int oracle_enumerate_plans_any(const int64_t *g_levels, int nG, int32_t *plans, int cap, int32_t *group_off)
+{
+    int n = 0;
+    for (int gi = 0; gi < nG; ++gi) {
+        group_off[gi] = n;
+        int64_t g = g_levels[gi];
+        for (int64_t t = 1; t <= g; ++t) {
+            if (g % t != 0) continue;
+            for (int64_t p = 1; p <= g / t; ++p) {
+                if ((g / t) % p != 0) continue;
+                int64_t d = g / (t * p);
+                for (int z = 0; z < 4; ++z)
+                    for (int gc = 0; gc < 2; ++gc)
+                        for (int off = 0; off < 2; ++off) {
+                            if (n < cap) {
+                                int32_t *pl = plans + (size_t)n * PF_COUNT;
+                                pl[PF_D] = (int32_t)d; pl[PF_T] = (int32_t)t; pl[PF_P] = (int32_t)p;
+                                pl[PF_Z] = z; pl[PF_GC] = gc; pl[PF_OFF] = off;
+                            }
+                            ++n;
+                        }
+            }
+        }
+    }
+    group_off[nG] = n;
+    return n;
+}
+
 /* ---- candidate table: thr[J][C][P] and feas[J][P] ------------------------------------ */
 void oracle_eval(const double *jobs, int J, const int32_t *plans, int P, const double *env,
                  const int64_t *c_levels, int nC, const int64_t *m_levels, int nM,

@@ -120,3 +120,41 @@ def test_best_is_monotone_in_host_memory_and_cores(paper_scale):
     assert np.all(np.diff(bv, axis=3) >= 0)          # more host memory never hurts
     assert np.all(np.diff(bv, axis=2) >= 0)          # more cores never hurt
     assert (np.diff(bv, axis=2) > 0).any()           # and help where offload is the best plan
+
+
+def ordered_factorisations(g):
+    """Number of ordered triples (d, t, p) with d * t * p = g: multiplicative, C(a + 2, 2) per prime power."""
+    n, out, q = g, 1, 2
+    while n > 1:
+        a = 0
+        while n % q == 0:
+            n //= q
+            a += 1
+        out *= (a + 1) * (a + 2) // 2
+        q += 1
+    return out
+
+
+def test_any_degree_plan_space():
+    """The wider plan space (Section 7.2 uses a 3-GPU tensor-parallel plan, Table 2 GPU counts such as 12 and
+    24): every ordered factorisation of every GPU level, same canonical order; on power-of-two levels it is
+    the power-of-two list."""
+    levels = [1, 2, 3, 4, 6, 8, 12, 16, 24, 36]
+    plans, off = oracle.enumerate_plans(levels, any_degrees=True)
+    assert len(plans) == off[-1] == 16 * sum(ordered_factorisations(g) for g in levels)
+    for i, g in enumerate(levels):
+        grp = plans[off[i]:off[i + 1]]
+        assert len(grp) == 16 * ordered_factorisations(g)
+        assert np.all(grp[:, 0].astype(np.int64) * grp[:, 1] * grp[:, 2] == g)
+        triples = grp[::16, :3]
+        keys = [(int(t), int(p)) for d, t, p in triples]
+        assert keys == sorted(keys) and len(set(keys)) == len(keys)          # TP ascending, then PP ascending, no repeats
+        tail = grp[:16, 3:]
+        assert [tuple(r) for r in tail] == [(z, gc, o) for z in range(4) for gc in range(2) for o in range(2)]
+    pow2 = [1, 2, 4, 8, 16, 64]
+    a, oa = oracle.enumerate_plans(pow2, any_degrees=True)
+    b, ob = oracle.enumerate_plans(pow2)
+    assert np.array_equal(a, b) and np.array_equal(oa, ob)
+    # the 3-GPU tensor-parallel plan exists and is valid for a job whose hidden size divides by 3
+    p3 = plans[off[2]:off[3]]
+    assert any((r[:3] == [1, 3, 1]).all() for r in p3)
