@@ -93,6 +93,16 @@ typedef struct {
     uint8_t disabled;            /* non-zero: treat as invalid for every job */
 } rubick_plan;
 
+/* One plan of the wider plan space: degrees of any size (the paper's own experiments use a 3-GPU
+ * tensor-parallel plan and GPU counts such as 12 and 24).  12 bytes. */
+typedef struct {
+    uint16_t d, t, p;            /* data / tensor / pipeline parallel degrees, d * t * p = GPUs of the level */
+    uint8_t  zero, gc, off;
+    uint8_t  g_level;
+    uint8_t  disabled;           /* non-zero: treat as invalid for every job */
+    uint8_t  pad;
+} rubick_plan_wide;
+
 /* Resource grid: strictly increasing level values on each axis. */
 typedef struct {
     int32_t nG, nC, nM;
@@ -191,6 +201,19 @@ int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out
 int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const rubick_grid *h_grid);
 
 /* ---- the hot path ----------------------------------------------------------------------------- */
+
+/* The wider plan space: for EVERY GPU level g (not only powers of two) every ordered factorisation
+ * g = d * t * p, in the same canonical order (TP ascending over the divisors of g, then PP, then
+ * ZeRO stage, gradient checkpointing, offload); on power-of-two levels the list equals
+ * rubick_enumerate_plans'.  Same calling convention. */
+int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, rubick_plan_wide *h_out, int cap, int *n_out,
+                                int32_t *h_group_off);
+
+/* rubick_set_space for plans with degrees of any size.  The evaluation kernels then divide where
+ * the power-of-two space shifts (same model, same memory rule, same tolerances); everything
+ * downstream (best plan, curves, gains, rounds) is unchanged.  rubick_fit_models needs the
+ * power-of-two space.  GPU levels above a node must still be whole nodes. */
+int rubick_set_space_wide(rubick_ctx *ctx, const rubick_plan_wide *h_plans, int P, const rubick_grid *h_grid);
 
 /* Candidate table (paper Section 4, Eq. 1 with all its terms; THROUGHPUT = b / T_iter) and the
  * memory-feasibility mask, for jobs d_jobs[0..J).  d_thr: J*C*P floats, d_feas: J*P words, both

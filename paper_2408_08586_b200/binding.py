@@ -32,7 +32,9 @@ SAMPLE_DTYPE = np.dtype([("plan", "<i4"), ("cores", "<i4"), ("thr", "<f8")])
 FIT_NAMES = ("k_bwd", "k_sync", "k_opt", "k_opt_off", "k_off", "k_swap", "k_const")
 RECONF_DTYPE = np.dtype([("T", "<f4"), ("delta", "<f4"), ("n_reconf", "<i4"), ("active", "<i4")])
 NODE_DTYPE = np.dtype([("free_g", "<i4"), ("free_c", "<i4"), ("free_m", "<i8"), ("owner", "<i4"), ("reserved", "<i4")])
-assert JOB_DTYPE.itemsize == 128 and PLAN_DTYPE.itemsize == 8
+PLAN_WIDE_DTYPE = np.dtype([("d", "<u2"), ("t", "<u2"), ("p", "<u2"), ("zero", "u1"), ("gc", "u1"), ("off", "u1"),
+                            ("g_level", "u1"), ("disabled", "u1"), ("pad", "u1")])
+assert JOB_DTYPE.itemsize == 128 and PLAN_DTYPE.itemsize == 8 and PLAN_WIDE_DTYPE.itemsize == 12
 assert ASSIGN_DTYPE.itemsize == 40 and NODE_DTYPE.itemsize == 24
 
 
@@ -64,7 +66,7 @@ def make_cluster(n_nodes, quota=None):
 
 
 EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error", "rubick_enumerate_plans",
-           "rubick_set_space", "rubick_eval_candidates", "rubick_best_plan", "rubick_curves", "rubick_marginal_gain",
+           "rubick_set_space", "rubick_enumerate_plans_wide", "rubick_set_space_wide", "rubick_eval_candidates", "rubick_best_plan", "rubick_curves", "rubick_marginal_gain",
            "rubick_min_resources", "rubick_fit_models",
            "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
            "rubick_schedule_round_host", "rubick_incremental_event_host"]
@@ -95,6 +97,8 @@ def lib():
         L.rubick_last_error.restype = C.c_char_p
         L.rubick_enumerate_plans.argtypes = [vp, ip, vp, ip, C.POINTER(ip), vp]
         L.rubick_set_space.argtypes = [vp, vp, ip, C.POINTER(Grid)]
+        L.rubick_enumerate_plans_wide.argtypes = [vp, ip, vp, ip, C.POINTER(ip), vp]
+        L.rubick_set_space_wide.argtypes = [vp, vp, ip, C.POINTER(Grid)]
         L.rubick_eval_candidates.argtypes = [vp, vp, ip, vp, vp]
         L.rubick_best_plan.argtypes = [vp, vp, vp, ip, C.c_uint, vp, vp, vp]
         L.rubick_curves.argtypes = [vp, vp, ip, C.c_uint, vp, vp, vp, vp]
@@ -137,6 +141,21 @@ def enumerate_plans(g_levels):
     rc = lib().rubick_enumerate_plans(_ptr(gl), len(gl), _ptr(plans), n.value, C.byref(n), _ptr(off))
     if rc:
         raise RubickError(rc, "rubick_enumerate_plans")
+    return plans[:n.value], off
+
+
+def enumerate_plans_wide(g_levels):
+    """rubick_enumerate_plans_wide -> (plans as PLAN_WIDE_DTYPE array, group offsets [nG + 1] int32)."""
+    gl = np.ascontiguousarray(g_levels, dtype=np.int32)
+    n = C.c_int(0)
+    off = np.zeros(len(gl) + 1, dtype=np.int32)
+    rc = lib().rubick_enumerate_plans_wide(_ptr(gl), len(gl), None, 0, C.byref(n), _ptr(off))
+    if rc:
+        raise RubickError(rc, "rubick_enumerate_plans_wide")
+    plans = np.zeros(max(n.value, 1), dtype=PLAN_WIDE_DTYPE)
+    rc = lib().rubick_enumerate_plans_wide(_ptr(gl), len(gl), _ptr(plans), n.value, C.byref(n), _ptr(off))
+    if rc:
+        raise RubickError(rc, "rubick_enumerate_plans_wide")
     return plans[:n.value], off
 
 
@@ -202,13 +221,16 @@ class Context:
         return self._check(lib().rubick_sync(self._h))
 
     def set_space(self, plans, g_levels, c_levels, m_levels):
-        plans = np.ascontiguousarray(plans, dtype=PLAN_DTYPE)
+        """rubick_set_space, or rubick_set_space_wide when `plans` has PLAN_WIDE_DTYPE."""
+        wide = getattr(plans, "dtype", None) == PLAN_WIDE_DTYPE
+        plans = np.ascontiguousarray(plans, dtype=PLAN_WIDE_DTYPE if wide else PLAN_DTYPE)
         gl = np.ascontiguousarray(g_levels, dtype=np.int32)
         cl = np.ascontiguousarray(c_levels, dtype=np.int32)
         ml = np.ascontiguousarray(m_levels, dtype=np.int64)
         grid = Grid(len(gl), len(cl), len(ml), 0, gl.ctypes.data_as(C.POINTER(C.c_int32)),
                     cl.ctypes.data_as(C.POINTER(C.c_int32)), ml.ctypes.data_as(C.POINTER(C.c_int64)))
-        self._check(lib().rubick_set_space(self._h, _ptr(plans), len(plans), C.byref(grid)))
+        fn = lib().rubick_set_space_wide if wide else lib().rubick_set_space
+        self._check(fn(self._h, _ptr(plans), len(plans), C.byref(grid)))
         self.P, self.nG, self.nC, self.nM = len(plans), len(gl), len(cl), len(ml)
 
     def eval_candidates(self, d_jobs, J, d_thr, d_feas):

@@ -64,7 +64,7 @@ int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *c
     ctx->device = device;
     ctx->stream = static_cast<cudaStream_t>(cuda_stream);
     ctx->has_space = false;
-    ctx->d_quads = nullptr; ctx->d_status = nullptr; ctx->d_steps = nullptr;
+    ctx->d_quads = nullptr; ctx->d_wide_quads = nullptr; ctx->d_status = nullptr; ctx->d_steps = nullptr;
     ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0;
     ctx->d_thr = nullptr; ctx->d_feas = nullptr; ctx->d_cv = nullptr; ctx->d_cp = nullptr; ctx->d_cg = nullptr;
     ctx->cap_thr = ctx->cap_feas = ctx->cap_curve = 0;
@@ -92,7 +92,7 @@ void rubick_destroy(rubick_ctx *ctx)
     if (!ctx) return;
     cudaSetDevice(ctx->device);
     cudaStreamSynchronize(ctx->stream);
-    cudaFree(ctx->d_quads); cudaFree(ctx->d_status); cudaFree(ctx->d_round_scratch);
+    cudaFree(ctx->d_quads); cudaFree(ctx->d_wide_quads); cudaFree(ctx->d_status); cudaFree(ctx->d_round_scratch);
     cudaFree(ctx->d_thr); cudaFree(ctx->d_feas); cudaFree(ctx->d_cv); cudaFree(ctx->d_cp); cudaFree(ctx->d_cg);
     cudaFree(ctx->d_jobs_stage); cudaFree(ctx->d_out_stage); cudaFree(ctx->d_node_stage);
     cudaFree(ctx->d_best_todo);
@@ -144,10 +144,16 @@ int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out
     return RUBICK_OK;
 }
 
-int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const rubick_grid *h_grid)
+}  // extern "C"
+
+namespace {
+
+// one plan with its degrees written out (both plan record formats are brought to this form)
+struct NormPlan { int d, t, p, zero, gc, off, g_level, disabled; };
+
+int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_grid *h_grid, bool wide)
 {
-    CHECK_CTX(ctx);
-    if (!h_plans || !h_grid || P <= 0 || (P & 3)) return fail(ctx, RUBICK_EINVAL, "plans: need a positive multiple of 4");
+    if (!h_grid || P <= 0 || (P & 3)) return fail(ctx, RUBICK_EINVAL, "plans: need a positive multiple of 4");
     const rubick_grid &gr = *h_grid;
     if (P > 65520) return fail(ctx, RUBICK_EINVAL, "plans: at most 65,520 plans (per-job plan tables live in shared memory)");
     if (gr.nG < 1 || gr.nG > RUBICK_MAX_G_LEVELS || gr.nC < 1 || gr.nC > RUBICK_MAX_C_LEVELS || gr.nM < 1
@@ -168,6 +174,7 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
     sp.P = P; sp.Q = P / 4; sp.nG = gr.nG; sp.nC = gr.nC; sp.nM = gr.nM;
     sp.Gn = Gn; sp.log2Gn = ilog2(Gn); sp.Cn = ctx->env.cpus_per_node;
     sp.strict = ctx->env.strict_zero_dp_only ? 1 : 0;
+    sp.wide = wide ? 1 : 0;
     sp.e = float(ctx->env.bytes_per_elem);
     sp.inv_B_intra = float(1.0 / ctx->env.B_intra);
     sp.inv_B_inter = float(1.0 / ctx->env.B_inter);
@@ -179,16 +186,19 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
 
     // plans: ordered by level, quads of (gc, off), GPU count = the level's
     std::vector<QuadDesc> quads(size_t(P) / 4);
+    std::vector<WideQuad> wquads(wide ? size_t(P) / 4 : 0);
     int level = 0;
     sp.group_off[0] = 0;
     for (int i = 0; i < P; ++i) {
-        const rubick_plan &pl = h_plans[i];
+        const NormPlan &pl = h_plans[i];
         if (pl.g_level >= gr.nG || pl.g_level < level) return fail(ctx, RUBICK_EINVAL, "plans: g_level out of range or not ascending");
-        if (pl.zero > 3 || pl.gc > 1 || pl.off > 1 || pl.log2d > 15 || pl.log2t > 15 || pl.log2p > 15
-            || int(pl.log2d) + pl.log2t + pl.log2p > 20)
+        if (pl.zero < 0 || pl.zero > 3 || pl.gc < 0 || pl.gc > 1 || pl.off < 0 || pl.off > 1 || pl.d < 1 || pl.t < 1 || pl.p < 1
+            || pl.d > 32768 || pl.t > 32768 || pl.p > 32768 || int64_t(pl.d) * pl.t * pl.p > (int64_t(1) << 20))
             return fail(ctx, RUBICK_EINVAL, "plans: field out of range");
-        if ((int64_t(1) << (pl.log2d + pl.log2t + pl.log2p)) != gr.g_levels[pl.g_level])
+        if (int64_t(pl.d) * pl.t * pl.p != gr.g_levels[pl.g_level])
             return fail(ctx, RUBICK_EINVAL, "plans: d*t*p differs from the GPU level");
+        if (!wide && (!is_pow2(pl.d) || !is_pow2(pl.t) || !is_pow2(pl.p)))
+            return fail(ctx, RUBICK_EINVAL, "plans: degrees must be powers of two in this plan format");
         if (pl.g_level > level) {
             if (i & 3) return fail(ctx, RUBICK_EINVAL, "plans: a level must start on a quad boundary");
             while (level < pl.g_level) sp.group_off[++level] = i;
@@ -197,14 +207,17 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
         if (pl.gc != (v >> 1) || pl.off != (v & 1)) return fail(ctx, RUBICK_EINVAL, "plans: quads must run (gc, off) = (0,0), (0,1), (1,0), (1,1)");
         QuadDesc &q = quads[size_t(i) >> 2];
         if (v == 0) {
-            q.log2d = pl.log2d; q.log2t = pl.log2t; q.log2p = pl.log2p; q.zero = pl.zero; q.g_level = pl.g_level;
+            q.log2d = wide ? 0 : uint8_t(ilog2(pl.d)); q.log2t = wide ? 0 : uint8_t(ilog2(pl.t)); q.log2p = wide ? 0 : uint8_t(ilog2(pl.p));
+            q.zero = uint8_t(pl.zero); q.g_level = uint8_t(pl.g_level);
             q.flags = 0; q.disabled = 0; q.pad = 0;
-            const int64_t d = int64_t(1) << pl.log2d, t = int64_t(1) << pl.log2t, g = gr.g_levels[pl.g_level];
+            const int64_t d = pl.d, t = pl.t, g = gr.g_levels[pl.g_level];
             if (t <= Gn) q.flags |= QF_T_FITS_NODE;
             if (d * t > Gn) q.flags |= QF_DP_INTER;
             if (g > Gn) q.flags |= QF_PP_INTER;
-        } else if (q.log2d != pl.log2d || q.log2t != pl.log2t || q.log2p != pl.log2p || q.zero != pl.zero) {
-            return fail(ctx, RUBICK_EINVAL, "plans: the four plans of a quad must share d, t, p and the ZeRO stage");
+        } else {
+            const NormPlan &first = h_plans[i - v];
+            if (first.d != pl.d || first.t != pl.t || first.p != pl.p || first.zero != pl.zero)
+                return fail(ctx, RUBICK_EINVAL, "plans: the four plans of a quad must share d, t, p and the ZeRO stage");
         }
         if (pl.disabled) q.disabled |= uint8_t(1u << v);
     }
@@ -212,19 +225,91 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
     if (quads.size() % 4) return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with all four ZeRO stages");
     for (size_t i = 0; i < quads.size(); ++i) {
         const QuadDesc &a = quads[i & ~size_t(3)], &b = quads[i];
-        if (b.zero != (i & 3) || a.log2d != b.log2d || a.log2t != b.log2t || a.log2p != b.log2p || a.g_level != b.g_level)
+        const NormPlan &pa = h_plans[4 * (i & ~size_t(3))], &pb = h_plans[4 * i];
+        if (b.zero != (i & 3) || pa.d != pb.d || pa.t != pb.t || pa.p != pb.p || a.g_level != b.g_level)
             return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with ZeRO stages 0..3 in order (disable plans instead of dropping them)");
     }
     while (level < gr.nG) sp.group_off[++level] = P;
+    for (size_t i = 0; i < wquads.size(); ++i) {
+        const NormPlan &pl = h_plans[4 * i];
+        wquads[i].x = uint32_t(pl.d) | (uint32_t(pl.t) << 16);
+        wquads[i].y = uint32_t(pl.p) | (uint32_t(pl.zero) << 16);
+        wquads[i].z = uint32_t(quads[i].flags) | (uint32_t(quads[i].disabled) << 8);
+        wquads[i].w = 0u;
+    }
 
     CUDA_TRY(ctx, cudaSetDevice(ctx->device), "cudaSetDevice");
     if (ctx->d_quads) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_quads); ctx->d_quads = nullptr; }
     CUDA_TRY(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->d_quads), quads.size() * sizeof(QuadDesc)), "cudaMalloc (plan table)");
     CUDA_TRY(ctx, cudaMemcpy(ctx->d_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice), "upload plan table");
+    if (ctx->d_wide_quads) { cudaFree(ctx->d_wide_quads); ctx->d_wide_quads = nullptr; }
+    if (wide) {
+        CUDA_TRY(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->d_wide_quads), wquads.size() * sizeof(WideQuad)), "cudaMalloc (wide plan table)");
+        CUDA_TRY(ctx, cudaMemcpy(ctx->d_wide_quads, wquads.data(), wquads.size() * sizeof(WideQuad), cudaMemcpyHostToDevice), "upload wide plan table");
+    }
     ctx->space = sp;
     ctx->inc_J = 0;
-    ctx->plans.assign(h_plans, h_plans + P);
     ctx->has_space = true;
+    return RUBICK_OK;
+}
+
+
+}  // namespace
+
+extern "C" {
+
+int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const rubick_grid *h_grid)
+{
+    CHECK_CTX(ctx);
+    if (!h_plans || P <= 0) return fail(ctx, RUBICK_EINVAL, "plans: need a positive multiple of 4");
+    std::vector<NormPlan> np_list((size_t(P)));
+    for (int i = 0; i < P; ++i) {
+        const rubick_plan &pl = h_plans[i];
+        if (pl.log2d > 15 || pl.log2t > 15 || pl.log2p > 15) return fail(ctx, RUBICK_EINVAL, "plans: field out of range");
+        np_list[i] = NormPlan{1 << pl.log2d, 1 << pl.log2t, 1 << pl.log2p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled};
+    }
+    return install_space(ctx, np_list.data(), P, h_grid, false);
+}
+
+int rubick_set_space_wide(rubick_ctx *ctx, const rubick_plan_wide *h_plans, int P, const rubick_grid *h_grid)
+{
+    CHECK_CTX(ctx);
+    if (!h_plans || P <= 0) return fail(ctx, RUBICK_EINVAL, "plans: need a positive multiple of 4");
+    std::vector<NormPlan> np_list((size_t(P)));
+    for (int i = 0; i < P; ++i) {
+        const rubick_plan_wide &pl = h_plans[i];
+        np_list[i] = NormPlan{pl.d, pl.t, pl.p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled};
+    }
+    return install_space(ctx, np_list.data(), P, h_grid, true);
+}
+
+int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, rubick_plan_wide *h_out, int cap, int *n_out,
+                                int32_t *h_group_off)
+{
+    if (!h_g_levels || nG < 1 || nG > RUBICK_MAX_G_LEVELS || !n_out || cap < 0 || (cap > 0 && !h_out)) return RUBICK_EINVAL;
+    for (int i = 0; i < nG; ++i)
+        if (h_g_levels[i] <= 0 || h_g_levels[i] > 32768 || (i && h_g_levels[i] <= h_g_levels[i - 1])) return RUBICK_EINVAL;
+    int n = 0;
+    for (int gi = 0; gi < nG; ++gi) {
+        if (h_group_off) h_group_off[gi] = n;
+        const int g = h_g_levels[gi];
+        for (int t = 1; t <= g; ++t) {
+            if (g % t) continue;
+            for (int p = 1; p <= g / t; ++p) {
+                if ((g / t) % p) continue;
+                for (int z = 0; z < 4; ++z)
+                    for (int v = 0; v < 4; ++v, ++n)
+                        if (n < cap) {
+                            rubick_plan_wide &pl = h_out[n];
+                            pl.d = uint16_t(g / (t * p)); pl.t = uint16_t(t); pl.p = uint16_t(p);
+                            pl.zero = uint8_t(z); pl.gc = uint8_t(v >> 1); pl.off = uint8_t(v & 1);
+                            pl.g_level = uint8_t(gi); pl.disabled = 0; pl.pad = 0;
+                        }
+            }
+        }
+    }
+    if (h_group_off) h_group_off[nG] = n;
+    *n_out = n;
     return RUBICK_OK;
 }
 
@@ -246,7 +331,7 @@ int rubick_eval_candidates(rubick_ctx *ctx, const rubick_job *d_jobs, int J, flo
     if ((reinterpret_cast<uintptr_t>(d_thr) & 15) || (reinterpret_cast<uintptr_t>(d_feas) & 15) || (reinterpret_cast<uintptr_t>(d_jobs) & 15))
         return fail(ctx, RUBICK_EINVAL, "d_jobs, d_thr and d_feas must be 16-byte aligned");
     if (int64_t(J) * ctx->space.Q >= (int64_t(1) << 31)) return fail(ctx, RUBICK_EINVAL, "J * P / 4 must stay below 2^31: evaluate in job tiles");
-    CUDA_TRY(ctx, launch_eval(ctx->space, ctx->d_quads, d_jobs, J, d_thr, d_feas, ctx->stream), "launch eval_candidates");
+    CUDA_TRY(ctx, launch_eval(ctx->space, ctx->d_quads, ctx->d_wide_quads, d_jobs, J, d_thr, d_feas, ctx->stream), "launch eval_candidates");
     return RUBICK_OK;
 }
 
@@ -279,7 +364,7 @@ int rubick_curves(rubick_ctx *ctx, const rubick_job *d_jobs, int J, unsigned fla
     if ((reinterpret_cast<uintptr_t>(d_feas) & 15) || (reinterpret_cast<uintptr_t>(d_jobs) & 15))
         return fail(ctx, RUBICK_EINVAL, "d_jobs and d_feas must be 16-byte aligned");
     if (flags & ~RUBICK_BEST_RAW) return fail(ctx, RUBICK_EINVAL, "unknown flag");
-    CUDA_TRY(ctx, launch_curves(ctx->space, ctx->d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g, ctx->stream),
+    CUDA_TRY(ctx, launch_curves(ctx->space, ctx->d_quads, ctx->d_wide_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g, ctx->stream),
              "launch curves");
     return RUBICK_OK;
 }
@@ -322,6 +407,7 @@ int rubick_fit_models(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const ru
     if (!d_jobs || !d_samples || !d_theta || !d_rmsle) return fail(ctx, RUBICK_EINVAL, "null pointer");
     if (S < 1 || S > 4096) return fail(ctx, RUBICK_EINVAL, "1 .. 4096 sample slots per model");
     if (sweeps < 0 || sweeps > 64) return fail(ctx, RUBICK_EINVAL, "0 .. 64 sweeps");
+    if (ctx->space.wide) return fail(ctx, RUBICK_ESTATE, "model fitting works on the power-of-two plan space (rubick_set_space)");
     if ((reinterpret_cast<uintptr_t>(d_samples) & 7) || (reinterpret_cast<uintptr_t>(d_theta) & 7) || (reinterpret_cast<uintptr_t>(d_rmsle) & 7))
         return fail(ctx, RUBICK_EINVAL, "d_samples, d_theta and d_rmsle must be 8-byte aligned");
     CUDA_TRY(ctx, launch_fit(ctx->env, ctx->d_quads, ctx->space.P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle, ctx->stream),
@@ -463,7 +549,7 @@ static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
         ctx->cap_curve = curve;
     }
     // a round only needs the curves: the one-pass kernel never writes the candidate table
-    CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, d_jobs, J, 0u, ctx->d_feas, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->stream), "launch curves");
+    CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, ctx->d_wide_quads, d_jobs, J, 0u, ctx->d_feas, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->stream), "launch curves");
     return RUBICK_OK;
 }
 
@@ -509,7 +595,7 @@ static int enqueue_tables_of(rubick_ctx *ctx, const rubick_job *d_jobs, const in
         int run = 1;                    // consecutive slots go through the kernel together
         while (i + run < n && h_slots[i + run] == h_slots[i] + run) ++run;
         const int s0 = h_slots[i];
-        CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, d_jobs + s0, run, 0u, ctx->d_feas + size_t(s0) * sp.P, ctx->d_cv + s0 * per_job,
+        CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, ctx->d_wide_quads, d_jobs + s0, run, 0u, ctx->d_feas + size_t(s0) * sp.P, ctx->d_cv + s0 * per_job,
                                     ctx->d_cp + s0 * per_job, ctx->d_cg + s0 * per_job, ctx->stream),
                  "launch curves");
         i += run;

@@ -103,32 +103,48 @@ __device__ __forceinline__ int first_level(const Space &sp, int64_t need)
 // must call this together with the quads of a warp consecutive and starting at a multiple of four (the
 // four ZeRO stages of a (d, t, p) triple trade results); `active` = false for mirror threads past the end.
 // Returns the four feasibility words when KEEP_WORDS (zeros otherwise).
-template <bool KEEP_WORDS, class Emit>
-__device__ __forceinline__ uint4 eval_quad(const Space &sp, const QuadDesc *__restrict__ quads,
+// WIDE: degrees of any size from the wide quad table (divisions); otherwise powers of two from the
+// logarithms of the quad table (shifts, exact reciprocals).
+template <bool KEEP_WORDS, bool WIDE, class Emit>
+__device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restrict__ quads_any,
                                            const rubick_job *__restrict__ jobs, int j, int q, bool active,
                                            uint32_t *__restrict__ feas, Emit &&emit)
 {
     const JobRegs jb = load_job(jobs + j);
-    const uint2 qraw = __ldg(reinterpret_cast<const uint2 *>(quads) + q);
-    const int ld = qraw.x & 0xff, lt = (qraw.x >> 8) & 0xff, lp = (qraw.x >> 16) & 0xff, z = (qraw.x >> 24) & 0xff;
-    const int qflags = (qraw.y >> 8) & 0xff, disabled = (qraw.y >> 16) & 0xff;
-    const int lg = ld + lt + lp;
-    const int d = 1 << ld, t = 1 << lt, p = 1 << lp;
+    int ld = 0, lt = 0, lp = 0, lg = 0, d, t, p, z, qflags, disabled;
+    if constexpr (WIDE) {
+        const uint4 qraw = __ldg(reinterpret_cast<const uint4 *>(quads_any) + q);
+        d = qraw.x & 0xffff; t = qraw.x >> 16; p = qraw.y & 0xffff; z = (qraw.y >> 16) & 0xff;
+        qflags = qraw.z & 0xff; disabled = (qraw.z >> 8) & 0xff;
+    } else {
+        const uint2 qraw = __ldg(reinterpret_cast<const uint2 *>(quads_any) + q);
+        ld = qraw.x & 0xff; lt = (qraw.x >> 8) & 0xff; lp = (qraw.x >> 16) & 0xff; z = (qraw.x >> 24) & 0xff;
+        qflags = (qraw.y >> 8) & 0xff; disabled = (qraw.y >> 16) & 0xff;
+        lg = ld + lt + lp;
+        d = 1 << ld; t = 1 << lt; p = 1 << lp;
+    }
+    const int g = d * t * p;
+    // x / divisor rounded up; the divisor is 1 << shift in the power-of-two space
+    auto cdiv_by = [](int64_t x, int divisor, int shift) -> int64_t {
+        if constexpr (WIDE) return (x + divisor - 1) / divisor; else return cdiv_shift(x, shift);
+    };
 
     // structural validity of the (d, t, p, z) part; offload additionally needs ZeRO stage >= 2
-    bool valid = (qflags & QF_T_FITS_NODE) && p <= jb.l && d <= jb.b && (jb.b & (d - 1)) == 0
-                 && (jb.h & (t - 1)) == 0 && !(sp.strict && z > 0 && (lt + lp) > 0);
+    bool valid = (qflags & QF_T_FITS_NODE) && p <= jb.l && d <= jb.b && !(sp.strict && z > 0 && (t > 1 || p > 1));
+    if constexpr (WIDE) valid = valid && jb.b % d == 0 && jb.h % t == 0;
+    else valid = valid && (jb.b & (d - 1)) == 0 && (jb.h & (t - 1)) == 0;
     const bool valid_off = valid && z >= 2;
 
     // micro-batching
-    const int r = max(jb.b >> ld, 1);
+    const int r = max(WIDE ? jb.b / d : jb.b >> ld, 1);
     const int mu = min(r, max(jb.mu_cap, 1));
     const int n = (r + mu - 1) / mu;
     const int m = p > 1 ? n : 1;
     const int a = p > 1 ? 1 : n;
 
     // ---- times that do not depend on the CPU level -------------------------------------------
-    const float inv_tp = pow2_neg(lt + lp);
+    const float inv_tp = WIDE ? 1.0f / float(t * p) : pow2_neg(lt + lp);
+    const float inv_dt = WIDE ? 1.0f / float(d * t) : pow2_neg(ld + lt);
     float T_fwd = jb.tau * float(mu) * inv_tp;
     if (p > 1) T_fwd *= float(n + p - 1);
     const float T_bwd0 = jb.k_bwd * T_fwd;
@@ -138,12 +154,12 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const QuadDesc *__re
     const float bsh = float(int64_t(jb.b) * jb.s * jb.h);
     float T_dp = 0.0f, T_tp = 0.0f, T_pp = 0.0f;
     if (d > 1) {
-        float V = sp.e * Pf * (float(d - 1) * pow2_neg(lg - 1));
+        float V = sp.e * Pf * (WIDE ? 2.0f * float(d - 1) / float(g) : float(d - 1) * pow2_neg(lg - 1));
         if (z == 3) V *= 1.5f;
         T_dp = V * ((qflags & QF_DP_INTER) ? sp.inv_B_inter : sp.inv_B_intra);
     }
-    if (t > 1) T_tp = sp.e * 8.0f * float(t - 1) * bsh * float(jb.l) * pow2_neg(ld + lt) * sp.inv_B_intra;
-    if (p > 1) T_pp = sp.e * 2.0f * float(p) * bsh * pow2_neg(ld + lt) * ((qflags & QF_PP_INTER) ? sp.inv_B_inter : sp.inv_B_intra);
+    if (t > 1) T_tp = sp.e * 8.0f * float(t - 1) * bsh * float(jb.l) * inv_dt * sp.inv_B_intra;
+    if (p > 1) T_pp = sp.e * 2.0f * float(p) * bsh * inv_dt * ((qflags & QF_PP_INTER) ? sp.inv_B_inter : sp.inv_B_intra);
 
     const float inv_ksync = 1.0f / jb.k_sync;
     const float af = float(a);
@@ -152,7 +168,7 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const QuadDesc *__re
     const float cc1 = fixed + (af - 1.0f) * T_bwd1 + overlap(jb.k_sync, inv_ksync, T_bwd1, T_dp);
 
     const float Psi = Pf * inv_tp;
-    const float inv_d = pow2_neg(ld);
+    const float inv_d = WIDE ? 1.0f / float(d) : pow2_neg(ld);
     const float T_opt = jb.k_opt * Psi * (z >= 1 ? inv_d : 1.0f);
     const float bf = float(jb.b);
 
@@ -166,23 +182,25 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const QuadDesc *__re
     // ---- feasibility words ---------------------------------------------------------------------
     {
         const int64_t Pi = int64_t(jb.P);
-        const int64_t Psi_i = cdiv_shift(Pi, lt + lp);
-        const int64_t params = 2 * cdiv_shift(Psi_i, z == 3 ? ld : 0);
-        const int64_t grads = 2 * cdiv_shift(Psi_i, z >= 2 ? ld : 0);
-        const int64_t opt = 12 * cdiv_shift(Psi_i, z >= 1 ? ld : 0);
+        const int64_t Psi_i = cdiv_by(Pi, t * p, lt + lp);
+        const int64_t Psi_d = cdiv_by(Psi_i, d, ld);              // the shard of a ZeRO-partitioned state
+        const int64_t params = 2 * (z == 3 ? Psi_d : Psi_i);
+        const int64_t grads = 2 * (z >= 2 ? Psi_d : Psi_i);
+        const int64_t opt = 12 * (z >= 1 ? Psi_d : Psi_i);
         const int64_t smh = int64_t(jb.s) * mu * jb.h;
-        const int64_t A = cdiv_shift(int64_t(jb.alpha) * smh, lt);
-        const int64_t Lq = cdiv_shift(jb.l, lp) * (p > 1 ? min(m, p) : 1);
+        const int64_t A = cdiv_by(int64_t(jb.alpha) * smh, t, lt);
+        const int64_t Lq = cdiv_by(jb.l, p, lp) * (p > 1 ? min(m, p) : 1);
         const int64_t act0 = Lq * A;
         const int64_t act1 = Lq * 2 * smh + A;
         const int64_t st0 = params + grads + opt, st1 = params;
-        const int64_t need0 = jb.host_base << lg;
+        const int64_t need0 = WIDE ? jb.host_base * g : jb.host_base << lg;
         const int64_t need1 = need0 + 14 * Pi;
         const int nshift = max(lg - sp.log2Gn, 0);
+        const int nodes = g > sp.Gn ? g / sp.Gn : 1;
         const uint32_t full = sp.nM >= 32 ? 0xffffffffu : ((1u << sp.nM) - 1u);
         uint32_t w0 = 0u, w1 = 0u;
-        if (cdiv_shift(need0, nshift) <= sp.Mn) { int f = first_level(sp, need0); if (f < sp.nM) w0 = (full << f) & full; }
-        if (cdiv_shift(need1, nshift) <= sp.Mn) { int f = first_level(sp, need1); if (f < sp.nM) w1 = (full << f) & full; }
+        if (cdiv_by(need0, nodes, nshift) <= sp.Mn) { int f = first_level(sp, need0); if (f < sp.nM) w0 = (full << f) & full; }
+        if (cdiv_by(need1, nodes, nshift) <= sp.Mn) { int f = first_level(sp, need1); if (f < sp.nM) w1 = (full << f) & full; }
         uint4 fw;
         fw.x = (valid && !(disabled & 1) && st0 + act0 <= sp.gpu_mem) ? w0 : 0u;
         fw.y = (valid_off && !(disabled & 2) && st1 + act0 <= sp.gpu_mem) ? w1 : 0u;
@@ -237,8 +255,9 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const QuadDesc *__re
     return fw_out;
 }
 
+template <bool WIDE>
 __global__ void __launch_bounds__(256)
-eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads,
+eval_candidates_kernel(const __grid_constant__ Space sp, const void *__restrict__ quads,
                        const rubick_job *__restrict__ jobs, int J, float *__restrict__ thr,
                        uint32_t *__restrict__ feas)
 {
@@ -252,7 +271,7 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
     const int j = int(gid / uint32_t(sp.Q));
     const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
     float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
-    eval_quad<false>(sp, quads, jobs, j, q, active, feas, [&](int ci, const float4 &out, const uint4 &) {
+    eval_quad<false, WIDE>(sp, quads, jobs, j, q, active, feas, [&](int ci, const float4 &out, const uint4 &) {
         if (active) __stcs(reinterpret_cast<float4 *>(row + size_t(ci) * sp.P), out);
     });
 }
@@ -273,10 +292,11 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const QuadDesc *__restr
 // ------------------------------------------------------------------------------------------------------
 constexpr int CURVES_THREADS = 128;      // small CTAs: the phases of the several CTAs of an SM overlap (704 threads: 2.4 ms, 128: 1.1 ms at 16,384 jobs)
 
+template <bool WIDE>
 __global__ void __launch_bounds__(CURVES_THREADS)
-curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads, const rubick_job *__restrict__ jobs,
-              int J, unsigned flags, uint32_t *__restrict__ feas, float *__restrict__ best_val,
-              int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g)
+curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads, const void *__restrict__ quads_any,
+              const rubick_job *__restrict__ jobs, int J, unsigned flags, uint32_t *__restrict__ feas,
+              float *__restrict__ best_val, int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned long long *keys = reinterpret_cast<unsigned long long *>(smem_raw);      // [nG][nC + 1]: offload class per core level, then the other class
@@ -290,12 +310,11 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
         // host-memory need of the level's plans: g processes, plus the offloaded states (as in the mask above)
         const rubick_job *jp = jobs + j;
         const int g = sp.g_levels[tid];
-        const int lg = 31 - __clz(g);
-        const int64_t need0 = jp->host_base_bytes << lg, need1 = need0 + 14 * int64_t(jp->P);
-        const int nshift = max(lg - sp.log2Gn, 0);
+        const int64_t need0 = jp->host_base_bytes * g, need1 = need0 + 14 * int64_t(jp->P);
+        const int nodes = g > sp.Gn ? g / sp.Gn : 1;
         int f0 = sp.nM, f1 = sp.nM;
-        if (cdiv_shift(need0, nshift) <= sp.Mn) f0 = first_level(sp, need0);
-        if (cdiv_shift(need1, nshift) <= sp.Mn) f1 = first_level(sp, need1);
+        if ((need0 + nodes - 1) / nodes <= sp.Mn) f0 = first_level(sp, need0);
+        if ((need1 + nodes - 1) / nodes <= sp.Mn) f1 = first_level(sp, need1);
         s_first[2 * tid] = f0; s_first[2 * tid + 1] = f1;
     }
     __syncthreads();
@@ -309,7 +328,7 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
         const unsigned peers = __match_any_sync(FULL, active ? level : -1);            // lanes of the same GPU level
         unsigned long long *kq = keys + size_t(level) * (sp.nC + 1);
         bool any_offload = false;                               // does a lane of my group own a feasible offloading plan?
-        eval_quad<true>(sp, quads, jobs, j, q, active, feas, [&](int ci, const float4 &o, const uint4 &words) {
+        eval_quad<true, WIDE>(sp, quads_any, jobs, j, q, active, feas, [&](int ci, const float4 &o, const uint4 &words) {
             // Infeasible plans count as 0.  Quads ascend with the lane and a lane's two plans of a class with
             // their index, so among equal values the lowest lane holds the lowest plan index: one warp
             // reduction for the value, one vote for who holds it, and that lane alone updates the key.
@@ -361,27 +380,33 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
     }
 }
 
-cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J, unsigned flags,
-                          uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, cudaStream_t st)
+cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
+                          unsigned flags, uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g,
+                          cudaStream_t st)
 {
     if (J == 0) return cudaSuccess;
     const size_t smem = size_t(sp.nG) * (sp.nC + 1) * sizeof(unsigned long long);
     if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(curves_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+        cudaError_t e = sp.wide ? cudaFuncSetAttribute(curves_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))
+                                : cudaFuncSetAttribute(curves_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
         if (e != cudaSuccess) return e;
     }
-    curves_kernel<<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
+    if (sp.wide)
+        curves_kernel<true><<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_wide_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
+    else
+        curves_kernel<false><<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
     return cudaGetLastError();
 }
 
-cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J,
+cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
                         float *d_thr, uint32_t *d_feas, cudaStream_t st)
 {
     if (J == 0) return cudaSuccess;
     const int64_t total = int64_t(J) * sp.Q;
     const int block = 256;
     const int64_t grid = (total + block - 1) / block;
-    eval_candidates_kernel<<<unsigned(grid), block, 0, st>>>(sp, d_quads, d_jobs, J, d_thr, d_feas);
+    if (sp.wide) eval_candidates_kernel<true><<<unsigned(grid), block, 0, st>>>(sp, d_wide_quads, d_jobs, J, d_thr, d_feas);
+    else eval_candidates_kernel<false><<<unsigned(grid), block, 0, st>>>(sp, d_quads, d_jobs, J, d_thr, d_feas);
     return cudaGetLastError();
 }
 

@@ -26,6 +26,10 @@ enum : uint8_t {
     QF_PP_INTER = 4,      // the pipeline crosses nodes (g > gpus_per_node)
 };
 
+// A plan quad of the wide plan space (degrees of any size), 16 bytes, read as one uint4:
+// x = d | t << 16, y = p | ZeRO stage << 16, z = QF_* flags | disabled bits << 8, w = 0.
+struct WideQuad { uint32_t x, y, z, w; };
+
 // Everything a kernel needs to know about the environment and the grid; passed by value as a
 // __grid_constant__ kernel parameter so that level lookups are uniform constant-bank reads.
 struct Space {
@@ -33,6 +37,7 @@ struct Space {
     int32_t nG, nC, nM;
     int32_t Gn, log2Gn, Cn;
     int32_t strict;
+    int32_t wide;                 // plans with degrees of any size (wide quad table) instead of powers of two
     int32_t n_small;              // number of GPU levels <= Gn (they come first)
     float e;                      // bytes per element
     float inv_B_intra, inv_B_inter, inv_B_pcie;
@@ -69,6 +74,7 @@ struct rubick_ctx {
     rubick::Space space;
     std::vector<rubick_plan> plans;
     rubick::QuadDesc *d_quads;          // [Q]
+    rubick::WideQuad *d_wide_quads;     // [Q] only for a wide plan space
     uint32_t *d_status;                 // one word, DS_* bits
     int32_t *d_steps;                   // one word, steps of the last round
     int32_t *d_quota;                   // [2 * RUBICK_MAX_TENANTS] per tenant: GPUs, cores (uploaded per round)
@@ -99,10 +105,11 @@ int fail(rubick_ctx *ctx, int code, const char *msg);
 int cuda_fail(rubick_ctx *ctx, cudaError_t e, const char *what);
 
 // launchers, one per translation unit
-cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J,
+cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
                         float *d_thr, uint32_t *d_feas, cudaStream_t st);
-cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const rubick_job *d_jobs, int J, unsigned flags,
-                          uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, cudaStream_t st);
+cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
+                          unsigned flags, uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g,
+                          cudaStream_t st);
 cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
                         float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, uint32_t *d_status,
                         int32_t *d_todo /* J + 1 words of scratch */, int num_sms, cudaStream_t st);

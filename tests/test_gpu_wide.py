@@ -1,0 +1,111 @@
+"""The wider plan space (degrees of any size: the paper's 3-GPU tensor-parallel plan, 12- and 24-GPU jobs)
+through the CUDA path, against the oracle on the same plans: throughput within 1e-5 relative, masks and
+everything downstream bit-exact."""
+import numpy as np
+import pytest
+
+import oracle
+from gpu_util import Gpu, assert_rounds_equal, has_cuda
+from helpers import GIB, env
+from paper_2408_08586_b200 import binding as rb
+from paper_2408_08586_b200 import workloads
+from test_gpu_parity import check_thr
+
+pytestmark = [pytest.mark.gpu, pytest.mark.skipif(not has_cuda(), reason="needs a CUDA device")]
+
+
+def wide_config(J, levels, gpus_per_node, n_nodes, seed=6):
+    cfg = workloads.make("paper-scale", J=J, n_nodes=n_nodes)
+    rng = np.random.default_rng(seed)
+    cfg["g_levels"] = np.asarray(levels)
+    cfg["env"] = env(gpus_per_node=gpus_per_node)
+    jobs = cfg["jobs"]
+    # shapes that odd degrees divide: hidden sizes with a factor 3 or 5, batches with a factor 3
+    jobs["h"] = rng.choice([768, 1536, 3072, 1280, 2560, 1920, 1024], J)
+    jobs["b"] = rng.choice([48, 96, 24, 64, 30], J)
+    jobs["l"] = rng.integers(12, 49, J)
+    jobs["gmin_idx"] = np.where(rng.uniform(size=J) < 0.3, rng.integers(0, 3, J), -1)
+    jobs["cmin_idx"] = np.where(jobs["gmin_idx"] >= 0, 0, -1)
+    return cfg
+
+
+def oracle_wide(cfg, nthreads=8):
+    plans, goff = oracle.enumerate_plans(cfg["g_levels"], any_degrees=True)
+    thr, feas = oracle.eval_candidates(cfg["jobs"], plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=nthreads)
+    cv, cp, cg = oracle.best_plan(thr.astype(np.float32), feas, plans, cfg["g_levels"], len(cfg["m_levels"]), prefix=True, nthreads=nthreads)
+    return plans, goff, thr, feas, cv.astype(np.float32), cp, cg
+
+
+def test_wide_enumerators_agree():
+    for levels in ([1, 2, 3, 4, 5, 6, 7, 8], [1, 2, 3, 4, 6, 8, 16, 24, 48], [1, 2, 4, 8, 16]):
+        got, goff = rb.enumerate_plans_wide(levels)
+        want, woff = oracle.enumerate_plans(levels, any_degrees=True)
+        assert np.array_equal(goff, woff) and len(got) == len(want)
+        for col, name in enumerate(("d", "t", "p", "zero", "gc", "off")):
+            assert np.array_equal(got[name].astype(np.int64), want[:, col])
+        assert np.array_equal(got["g_level"], np.searchsorted(woff[1:], np.arange(len(want)), side="right"))
+
+
+@pytest.mark.parametrize("levels,gn,N", [([1, 2, 3, 4, 6, 8, 16, 24, 48], 8, 7), ([1, 2, 3, 4, 8, 12, 24], 4, 9)])
+def test_wide_plan_space_through_every_kernel(levels, gn, N):
+    J = 41
+    cfg = wide_config(J, levels, gn, N)
+    plans, goff, thr, feas, cv, cp, cg = oracle_wide(cfg)
+    gpu_plans, _ = rb.enumerate_plans_wide(levels)
+    gpu = Gpu(cfg, plans=gpu_plans)
+    assert gpu.P == len(plans)
+    _, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    assert np.array_equal(gpu.np_feas(d_feas, J), feas)
+    check_thr(gpu.np_thr(d_thr, J), thr)
+    odd = (plans[:, 0] % 3 == 0) | (plans[:, 1] % 3 == 0) | (plans[:, 2] % 3 == 0)
+    assert (thr[:, 0, odd] > 0).any() and feas[:, odd].any()               # plans with a degree of 3, 6, 12 ... do run
+    t = gpu.torch
+    d_thr32 = t.from_numpy(thr.astype(np.float32).reshape(-1)).cuda()
+    bv, bp, bg = gpu.best(d_thr32, d_feas, J)
+    sh = gpu.shape4(J)
+    assert np.array_equal(bv.cpu().numpy().reshape(sh), cv)
+    assert np.array_equal(bp.cpu().numpy().reshape(sh), cp) and np.array_equal(bg.cpu().numpy().reshape(sh), cg)
+    assert odd[cp[cp >= 0]].any()                                          # and win somewhere
+    gpu.assert_one_pass_curves_match(cfg["jobs"])
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 N, want_log=True)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, N)
+    assert_rounds_equal(got, want)
+    assert want["steps"] > 5
+    # the whole path on the library's own tables: allocations agree except after near ties of the two chains
+    d_out = gpu.empty(J * rb.ASSIGN_DTYPE.itemsize, t.uint8)
+    steps, capped = gpu.ctx.schedule_round(gpu.jobs_to_device(cfg["jobs"]), J, N, 1 << 30, d_out)
+    out = rb.from_device(d_out, rb.ASSIGN_DTYPE)
+    agree = (out["g"] == want["g"]) & (out["c"] == want["c"]) & (out["plan"] == want["plan"])
+    assert agree.mean() >= 0.9 and not capped
+
+
+def test_wide_space_validation_and_limits():
+    cfg = wide_config(8, [1, 2, 3, 4, 6, 8], 8, 2)
+    plans, _ = rb.enumerate_plans_wide(cfg["g_levels"])
+    gpu = Gpu(cfg, plans=plans)
+    bad = plans.copy()
+    bad["d"][0] = 2                                        # d * t * p no longer the level's GPU count
+    with pytest.raises(rb.RubickError):
+        gpu.ctx.set_space(bad, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"])
+    with pytest.raises(rb.RubickError):                    # 12 GPUs on 8-GPU nodes is not a whole number of nodes
+        gpu.ctx.set_space(*((lambda p: (p, [1, 2, 12], cfg["c_levels"], cfg["m_levels"]))(rb.enumerate_plans_wide([1, 2, 12])[0])))
+    # fitting needs the power-of-two space
+    t = gpu.torch
+    gpu.ctx.set_space(plans, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"])
+    d = gpu.empty(4096, t.float64)
+    with pytest.raises(rb.RubickError) as ei:
+        gpu.ctx.fit_models(d, 1, d, 4, 4, d, d)
+    assert ei.value.code == rb.ESTATE
+    # the power-of-two format refuses other degrees; the wide format on power-of-two levels equals it
+    p2, _ = rb.enumerate_plans([1, 2, 4, 8])
+    w2, _ = rb.enumerate_plans_wide([1, 2, 4, 8])
+    assert np.array_equal(1 << p2["log2d"].astype(np.int64), w2["d"]) and np.array_equal(1 << p2["log2t"].astype(np.int64), w2["t"])
+    cfg2 = workloads.make("tiny")
+    cfg2["g_levels"] = np.array([1, 2, 4, 8])
+    a = Gpu(cfg2, plans=p2)
+    b = Gpu(cfg2, plans=w2)
+    _, thr_a, feas_a = a.eval(cfg2["jobs"])
+    _, thr_b, feas_b = b.eval(cfg2["jobs"])
+    assert t.equal(feas_a, feas_b)
+    assert np.allclose(thr_a.cpu().numpy(), thr_b.cpu().numpy(), rtol=2e-6, atol=0)
