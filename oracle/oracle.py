@@ -35,6 +35,16 @@ def build(force=False):
     return _SO
 
 
+def _plans(plans):
+    """Plans as the C side reads them: rows of (d, t, p, ZeRO stage, gc, off, micro-batch halvings); a
+    six-column input (no explicit accumulation) gets a zero seventh column."""
+    a = np.atleast_2d(np.asarray(plans, dtype=np.int32))
+    if a.shape[1] == 6:
+        a = np.concatenate([a, np.zeros((a.shape[0], 1), dtype=np.int32)], axis=1)
+    assert a.shape[1] == 7
+    return np.ascontiguousarray(a)
+
+
 def _p(a, t):
     return a.ctypes.data_as(C.POINTER(t))
 
@@ -89,7 +99,7 @@ def terms(jobs, j, env, plan, c):
     """All model terms (TERM_FIELDS) of job j under plan = (d, t, p, z, gc, off) with c cores."""
     rows = job_rows(jobs)
     out = np.zeros(len(TERM_FIELDS))
-    pl = _i32(plan)
+    pl = _plans(plan).reshape(-1)
     lib().oracle_terms(_p(rows[j], C.c_double), _p(env_row(env), C.c_double), _p(pl, C.c_int32),
                        C.c_double(float(c)), _p(out, C.c_double))
     return dict(zip(TERM_FIELDS, out.tolist()))
@@ -98,7 +108,7 @@ def terms(jobs, j, env, plan, c):
 def memory(jobs, j, env, plan):
     rows = job_rows(jobs)
     out = np.zeros(len(MEM_FIELDS), dtype=np.int64)
-    pl = _i32(plan)
+    pl = _plans(plan).reshape(-1)
     lib().oracle_memory(_p(rows[j], C.c_double), _p(env_row(env), C.c_double), _p(pl, C.c_int32),
                         _p(out, C.c_int64))
     return dict(zip(MEM_FIELDS, out.tolist()))
@@ -108,24 +118,27 @@ def feas_word(jobs, j, env, plan, m_levels):
     rows = job_rows(jobs)
     ml = _i64(m_levels)
     return int(lib().oracle_feas_word(_p(rows[j], C.c_double), _p(env_row(env), C.c_double),
-                                      _p(_i32(plan), C.c_int32), _p(ml, C.c_int64), C.c_int(len(ml))))
+                                      _p(_plans(plan).reshape(-1), C.c_int32), _p(ml, C.c_int64), C.c_int(len(ml))))
 
 
-def enumerate_plans(g_levels, any_degrees=False):
-    """-> (plans [P, 6] int32 = d, t, p, z, gc, off; group_off [nG + 1] int32).  any_degrees: every
-    factorisation of every GPU level instead of power-of-two degrees on power-of-two levels."""
+def enumerate_plans(g_levels, any_degrees=False, accumulation_levels=1):
+    """-> (plans [P, 7] int32 = d, t, p, z, gc, off, micro-batch halvings; group_off [nG + 1] int32).
+    any_degrees: every factorisation of every GPU level instead of power-of-two degrees on power-of-two
+    levels; accumulation_levels > 1 (with any_degrees): the explicit accumulation axis, 0 .. levels - 1
+    halvings of the micro-batch."""
     gl = _i64(g_levels)
     off = np.zeros(len(gl) + 1, dtype=np.int32)
-    dummy = np.zeros((1, 6), dtype=np.int32)
+    dummy = np.zeros((1, 7), dtype=np.int32)
     if any_degrees:
         f = lib().oracle_enumerate_plans_any
-        n = f(_p(gl, C.c_int64), C.c_int(len(gl)), _p(dummy, C.c_int32), C.c_int(0), _p(off, C.c_int32))
-        plans = np.zeros((max(n, 1), 6), dtype=np.int32)
-        f(_p(gl, C.c_int64), C.c_int(len(gl)), _p(plans, C.c_int32), C.c_int(n), _p(off, C.c_int32))
+        n = f(_p(gl, C.c_int64), C.c_int(len(gl)), C.c_int(accumulation_levels), _p(dummy, C.c_int32), C.c_int(0), _p(off, C.c_int32))
+        plans = np.zeros((max(n, 1), 7), dtype=np.int32)
+        f(_p(gl, C.c_int64), C.c_int(len(gl)), C.c_int(accumulation_levels), _p(plans, C.c_int32), C.c_int(n), _p(off, C.c_int32))
         return plans[:n], off
+    assert accumulation_levels == 1
     n = lib().oracle_enumerate_plans(_p(gl, C.c_int64), C.c_int(len(gl)), _p(dummy, C.c_int32), C.c_int(0),
                                      _p(off, C.c_int32))
-    plans = np.zeros((max(n, 1), 6), dtype=np.int32)
+    plans = np.zeros((max(n, 1), 7), dtype=np.int32)
     lib().oracle_enumerate_plans(_p(gl, C.c_int64), C.c_int(len(gl)), _p(plans, C.c_int32), C.c_int(n),
                                  _p(off, C.c_int32))
     return plans[:n], off
@@ -135,7 +148,7 @@ def eval_candidates(jobs, plans, env, c_levels, m_levels, nthreads=1):
     """-> (thr [J, C, P] float64, feas [J, P] uint32)."""
     rows = job_rows(jobs)
     J = rows.shape[0]
-    plans = _i32(plans)
+    plans = _plans(plans)
     Pn = plans.shape[0]
     cl, ml = _i64(c_levels), _i64(m_levels)
     thr = np.zeros((J, len(cl), Pn), dtype=np.float64)
@@ -153,7 +166,7 @@ def best_plan(thr, feas, plans, g_levels, nM, prefix=True, nthreads=1):
     thr = _f64(thr)
     feas = np.ascontiguousarray(feas, dtype=np.uint32)
     J, nC, Pn = thr.shape
-    plans = _i32(plans)
+    plans = _plans(plans)
     gl = _i64(g_levels)
     nG = len(gl)
     bv = np.zeros((J, nG, nC, nM), dtype=np.float64)
@@ -284,7 +297,7 @@ def fit(jobs, plans, env, sample_plan, sample_c, sample_thr, sweeps=14):
     -> (theta [J, 7] in FIT_NAMES order, rmsle [J, 2] before / after, margin [J])."""
     rows = job_rows(jobs)
     J = rows.shape[0]
-    plans = _i32(plans)
+    plans = _plans(plans)
     spn = np.ascontiguousarray(sample_plan, dtype=np.int32).reshape(J, -1)
     S = spn.shape[1]
     scs = _i64(sample_c).reshape(J, S)
@@ -323,7 +336,7 @@ def min_resources(thr, feas, curve_val, plans, g_levels, req):
     cv = _f64(curve_val)
     J, nC, Pn = thr.shape
     nG, nM = cv.shape[1], cv.shape[3]
-    plans = _i32(plans)
+    plans = _plans(plans)
     gl = _i64(g_levels)
     rq = _i64(req).reshape(J, 4)
     gm = np.zeros(J, dtype=np.int32)

@@ -72,8 +72,10 @@ enum {
     EF_COUNT
 };
 
-/* one plan = 6 int32: d, t, p (degrees themselves), ZeRO stage z, gc, off */
-enum { PF_D = 0, PF_T, PF_P, PF_Z, PF_GC, PF_OFF, PF_COUNT };
+/* one plan = 7 int32: d, t, p (degrees themselves), ZeRO stage z, gc, off, and ga = how many times the
+ * micro-batch is halved below the largest one a replica may run (explicit gradient accumulation: Table 1
+ * lists the accumulation steps a among a plan's parameters; 0 = as few steps as possible) */
+enum { PF_D = 0, PF_T, PF_P, PF_Z, PF_GC, PF_OFF, PF_GA, PF_COUNT };
 
 /* terms returned by oracle_terms (for unit tests of the individual formulas) */
 enum {
@@ -118,6 +120,8 @@ static int plan_valid(const double *job, const double *env, const int32_t *pl)
     if (off && z < 2) return 0;           /* offload moves partitioned gradients       */
     if (h % t != 0) return 0;             /* the hidden dimension splits evenly        */
     if (env[EF_STRICT] != 0.0 && (z > 0 || off) && (t > 1 || p > 1)) return 0;
+    if (pl[PF_GA] < 0 || pl[PF_GA] > 30) return 0;
+    if ((imin(b / d, (int64_t)job[JF_MUCAP]) >> pl[PF_GA]) < 1) return 0;   /* a micro-batch holds at least one sample */
     return 1;
 }
 
@@ -128,7 +132,7 @@ static void micro_batching(const double *job, const int32_t *pl, int64_t *mu, in
 {
     int64_t b = (int64_t)job[JF_B], d = pl[PF_D], p = pl[PF_P];
     int64_t r = b / d;
-    *mu = imin(r, (int64_t)job[JF_MUCAP]);
+    *mu = imin(r, (int64_t)job[JF_MUCAP]) >> pl[PF_GA];
     int64_t n = cdiv(r, *mu);
     if (p > 1) { *m = n; *a = 1; } else { *m = 1; *a = n; }
 }
@@ -278,7 +282,7 @@ int oracle_enumerate_plans(const int64_t *g_levels, int nG, int32_t *plans, int 
                             if (n < cap) {
                                 int32_t *pl = plans + (size_t)n * PF_COUNT;
                                 pl[PF_D] = (int32_t)d; pl[PF_T] = (int32_t)t; pl[PF_P] = (int32_t)p;
-                                pl[PF_Z] = z; pl[PF_GC] = gc; pl[PF_OFF] = off;
+                                pl[PF_Z] = z; pl[PF_GC] = gc; pl[PF_OFF] = off; pl[PF_GA] = 0;
                             }
                             ++n;
                         }
@@ -291,9 +295,10 @@ int oracle_enumerate_plans(const int64_t *g_levels, int nG, int32_t *plans, int 
 /* The wider plan space of the paper's own experiments (a 3-GPU tensor-parallel plan in Section 7.2,
  * GPU counts such as 12 or 24 in Table 2): for EVERY GPU level g, all ordered factorisations
  * g = d * t * p, TP degree ascending over the divisors of g, then PP degree ascending over the
- * divisors of g / t, then ZeRO stage, gradient checkpointing, offload.  On power-of-two levels this
- * is the list of oracle_enumerate_plans. */
-int oracle_enumerate_plans_any(const int64_t *g_levels, int nG, int32_t *plans, int cap, int32_t *group_off)
+ * divisors of g / t, then n_ga accumulation settings (the micro-batch halved 0 .. n_ga - 1 times), then
+ * ZeRO stage, gradient checkpointing, offload.  With n_ga = 1 on power-of-two levels this is the list of
+ * oracle_enumerate_plans. */
+int oracle_enumerate_plans_any(const int64_t *g_levels, int nG, int n_ga, int32_t *plans, int cap, int32_t *group_off)
 {
     int n = 0;
     for (int gi = 0; gi < nG; ++gi) {
@@ -304,16 +309,17 @@ int oracle_enumerate_plans_any(const int64_t *g_levels, int nG, int32_t *plans, 
             for (int64_t p = 1; p <= g / t; ++p) {
                 if ((g / t) % p != 0) continue;
                 int64_t d = g / (t * p);
-                for (int z = 0; z < 4; ++z)
-                    for (int gc = 0; gc < 2; ++gc)
-                        for (int off = 0; off < 2; ++off) {
-                            if (n < cap) {
-                                int32_t *pl = plans + (size_t)n * PF_COUNT;
-                                pl[PF_D] = (int32_t)d; pl[PF_T] = (int32_t)t; pl[PF_P] = (int32_t)p;
-                                pl[PF_Z] = z; pl[PF_GC] = gc; pl[PF_OFF] = off;
+                for (int ga = 0; ga < n_ga; ++ga)
+                    for (int z = 0; z < 4; ++z)
+                        for (int gc = 0; gc < 2; ++gc)
+                            for (int off = 0; off < 2; ++off) {
+                                if (n < cap) {
+                                    int32_t *pl = plans + (size_t)n * PF_COUNT;
+                                    pl[PF_D] = (int32_t)d; pl[PF_T] = (int32_t)t; pl[PF_P] = (int32_t)p;
+                                    pl[PF_Z] = z; pl[PF_GC] = gc; pl[PF_OFF] = off; pl[PF_GA] = ga;
+                                }
+                                ++n;
                             }
-                            ++n;
-                        }
             }
         }
     }

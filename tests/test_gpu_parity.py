@@ -47,7 +47,7 @@ def test_plan_enumerators_agree():
         assert np.array_equal(aoff, boff)
         got = np.stack([1 << a["log2d"].astype(np.int64), 1 << a["log2t"].astype(np.int64),
                         1 << a["log2p"].astype(np.int64), a["zero"], a["gc"], a["off"]], axis=1)
-        assert np.array_equal(got, b)
+        assert np.array_equal(got, b[:, :6]) and not b[:, 6].any()
 
 
 @pytest.mark.parametrize("name,J", [("tiny", None), ("paper-scale", None), ("cluster-512", 1024), ("cluster-512", 77)])

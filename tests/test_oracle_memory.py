@@ -11,6 +11,7 @@ import pytest
 
 import oracle
 from helpers import GIB, env, one_job
+from paper_2408_08586_b200 import workloads
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_facts.txt")
 
@@ -56,7 +57,8 @@ def py_rule(job, e, plan, m_levels):
     offload moving gradients and optimizer to the host (14 bytes per parameter there),
     activations per layer alpha*s*mu*h/t (2*s*mu*h kept + one layer live under checkpointing)
     for the layers of one stage and the micro-batches in flight."""
-    d, t, p, z, gc, off = plan
+    d, t, p, z, gc, off = plan[:6]
+    ga = plan[6] if len(plan) > 6 else 0              # explicit accumulation: the micro-batch halved ga times
     g = {k: int(v[0]) for k, v in job.items() if k not in ("tau", "k_bwd", "k_sync", "k_opt", "k_opt_off",
                                                             "k_off", "k_swap", "k_const", "w")}
     cd = lambda a, b: -(-a // b)
@@ -64,7 +66,9 @@ def py_rule(job, e, plan, m_levels):
     if t > Gn or p > g["l"] or d > g["b"] or g["b"] % d or (off and z < 2) or g["h"] % t:
         return 0
     r = g["b"] // d
-    mu = min(r, g["mu_cap"])
+    mu = min(r, g["mu_cap"]) >> ga
+    if mu < 1:
+        return 0
     n = cd(r, mu)
     m = n if p > 1 else 1
     psi = cd(g["P"], t * p)
@@ -146,3 +150,33 @@ def test_memory_terms_by_hand():
     assert m0["act"] == 12 * A
     mg = oracle.memory(job, 0, env(), (4, 2, 2, 0, 1, 0))
     assert mg["act"] == 12 * 2 * 1024 * 4 * 2048 + A
+
+
+def test_rule_on_the_wider_plan_space_with_python_integers(paper_scale):
+    """Degrees of any size and the explicit accumulation axis: the same independent recomputation."""
+    cfg = dict(paper_scale)
+    cfg["g_levels"] = np.array([1, 2, 3, 4, 6, 8, 16, 24])
+    jobs = {k: np.asarray(v).copy() for k, v in cfg["jobs"].items()}
+    rng = np.random.default_rng(9)
+    jobs["h"] = rng.choice([768, 1536, 3072, 1920], 64)
+    jobs["b"] = rng.choice([48, 96, 24, 64], 64)
+    plans, _ = oracle.enumerate_plans(cfg["g_levels"], any_degrees=True, accumulation_levels=3)
+    assert len(plans) % 48 == 0 and set(plans[:, 6]) == {0, 1, 2}
+    _, feas = oracle.eval_candidates(jobs, plans, cfg["env"], cfg["c_levels"][:1], cfg["m_levels"])
+    seen_ga = 0
+    for _ in range(4000):
+        j, pi = int(rng.integers(64)), int(rng.integers(len(plans)))
+        job = workloads.take(jobs, [j])
+        want = py_rule(job, cfg["env"], tuple(int(x) for x in plans[pi]), [int(x) for x in cfg["m_levels"]])
+        assert int(feas[j, pi]) == want, (j, pi, plans[pi])
+        seen_ga += int(want != 0 and plans[pi, 6] > 0)
+    assert seen_ga > 50
+    # more accumulation never makes a plan that fits stop fitting in GPU memory, and lets some plans fit that did not
+    base = feas[:, plans[:, 6] == 0] != 0
+    more = feas[:, plans[:, 6] == 2] != 0
+    can_halve_twice = np.zeros_like(base)
+    for j in range(64):
+        r = jobs["b"][j] // np.maximum(plans[plans[:, 6] == 0, 0], 1)
+        can_halve_twice[j] = np.minimum(r, jobs["mu_cap"][j]) >= 4
+    assert not (base & ~more & can_halve_twice).any()
+    assert (more & ~base).any()

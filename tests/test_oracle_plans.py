@@ -35,8 +35,8 @@ def test_plans_are_exactly_the_power_of_two_factorisations():
                             for gc in range(2):
                                 for o in range(2):
                                     want.add((d, t, p, z, gc, o))
-    got = [tuple(int(x) for x in r) for r in plans]
-    assert len(got) == len(set(got)) == 320 and set(got) == want
+    got = [tuple(int(x) for x in r[:6]) for r in plans]
+    assert len(got) == len(set(got)) == 320 and set(got) == want and not plans[:, 6].any()
     # groups: level index i holds the plans using g_levels[i] GPUs; other levels are empty
     for i, g in enumerate(levels):
         grp = plans[off[i]:off[i + 1]]
@@ -149,7 +149,7 @@ def test_any_degree_plan_space():
         triples = grp[::16, :3]
         keys = [(int(t), int(p)) for d, t, p in triples]
         assert keys == sorted(keys) and len(set(keys)) == len(keys)          # TP ascending, then PP ascending, no repeats
-        tail = grp[:16, 3:]
+        tail = grp[:16, 3:6]
         assert [tuple(r) for r in tail] == [(z, gc, o) for z in range(4) for gc in range(2) for o in range(2)]
     pow2 = [1, 2, 4, 8, 16, 64]
     a, oa = oracle.enumerate_plans(pow2, any_degrees=True)
@@ -158,3 +158,41 @@ def test_any_degree_plan_space():
     # the 3-GPU tensor-parallel plan exists and is valid for a job whose hidden size divides by 3
     p3 = plans[off[2]:off[3]]
     assert any((r[:3] == [1, 3, 1]).all() for r in p3)
+
+
+def test_explicit_accumulation_axis():
+    """Table 1 lists the accumulation steps among a plan's parameters; the axis halves the micro-batch 0, 1, 2
+    ... times below the largest one a replica may run.  Pinned by the closed forms: the micro-batch halves, the
+    number of passes doubles, so the compute of an iteration (a forwards of mu samples each) is unchanged
+    without pipelining, the pipeline bubble shrinks with more micro-batches, the activation memory halves,
+    and a micro-batch below one sample does not exist."""
+    from helpers import env, one_job
+    levels = [1, 2, 3, 4, 6, 8]
+    base, boff = oracle.enumerate_plans(levels, any_degrees=True)
+    plans, off = oracle.enumerate_plans(levels, any_degrees=True, accumulation_levels=3)
+    assert len(plans) == 3 * len(base) and np.array_equal(off, 3 * boff)
+    keys = [(int(r[0] * r[1] * r[2]), int(r[1]), int(r[2]), int(r[6]), int(r[3]), int(r[4]), int(r[5])) for r in plans]
+    assert keys == sorted(keys)            # g, TP, PP, accumulation, ZeRO stage, GC, offload
+    assert np.array_equal(plans[plans[:, 6] == 0][:, :6], base[:, :6])
+    job = one_job(b=64, mu_cap=8, l=24, h=1536)
+    e = env()
+    t0 = oracle.terms(job, 0, e, (4, 1, 1, 0, 0, 0, 0), 8)          # r = 16, mu = 8, a = 2
+    t1 = oracle.terms(job, 0, e, (4, 1, 1, 0, 0, 0, 1), 8)          # mu = 4, a = 4
+    t2 = oracle.terms(job, 0, e, (4, 1, 1, 0, 0, 0, 3), 8)          # mu = 1, a = 16
+    assert (t0["mu"], t0["a"], t1["mu"], t1["a"], t2["mu"], t2["a"]) == (8, 2, 4, 4, 1, 16)
+    assert t1["T_fwd"] == pytest.approx(t0["T_fwd"] / 2, rel=1e-15) and t0["a"] * t0["T_fwd"] == pytest.approx(t1["a"] * t1["T_fwd"], rel=1e-15)
+    # only the overlapped last backward changes: T_cc differs by f(T_bwd, T_dp) evaluated at the smaller backward
+    k = float(job["k_sync"][0])
+    for tm in (t0, t1, t2):
+        want = tm["a"] * tm["T_fwd"] + (tm["a"] - 1) * tm["T_bwd"] + oracle.overlap(k, tm["T_bwd"], tm["T_dp"]) + tm["T_tp"] + tm["T_pp"]
+        assert tm["T_cc"] == pytest.approx(want, rel=1e-15)
+    assert oracle.terms(job, 0, e, (4, 1, 1, 0, 0, 0, 4), 8)["valid"] == 0          # 8 >> 4 = 0 samples
+    # pipelining: m micro-batches, bubble (m + p - 1) / m of the ideal time, smaller with more micro-batches
+    p0 = oracle.terms(job, 0, e, (1, 1, 4, 0, 0, 0, 0), 8)          # r = 64, mu = 8, m = 8
+    p1 = oracle.terms(job, 0, e, (1, 1, 4, 0, 0, 0, 2), 8)          # mu = 2, m = 32
+    assert (p0["m"], p1["m"]) == (8, 32)
+    assert p1["T_fwd"] / p0["T_fwd"] == pytest.approx((32 + 3) / 32 / ((8 + 3) / 8), rel=1e-12)
+    # activations: with checkpointing off they scale with the micro-batch
+    m0 = oracle.memory(job, 0, e, (4, 1, 1, 0, 0, 0, 0))
+    m1 = oracle.memory(job, 0, e, (4, 1, 1, 0, 0, 0, 1))
+    assert m1["act"] * 2 == m0["act"] and m1["params"] == m0["params"] and m1["opt"] == m0["opt"]
