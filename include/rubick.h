@@ -100,7 +100,8 @@ typedef struct {
     uint8_t  zero, gc, off;
     uint8_t  g_level;
     uint8_t  disabled;           /* non-zero: treat as invalid for every job */
-    uint8_t  pad;
+    uint8_t  accum;              /* explicit gradient accumulation (Table 1's a): the micro-batch is halved this
+                                    many times below the largest one a replica may run; 0 = fewest passes */
 } rubick_plan_wide;
 
 /* Resource grid: strictly increasing level values on each axis. */
@@ -204,10 +205,12 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
 
 /* The wider plan space: for EVERY GPU level g (not only powers of two) every ordered factorisation
  * g = d * t * p, in the same canonical order (TP ascending over the divisors of g, then PP, then
- * ZeRO stage, gradient checkpointing, offload); on power-of-two levels the list equals
- * rubick_enumerate_plans'.  Same calling convention. */
-int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, rubick_plan_wide *h_out, int cap, int *n_out,
-                                int32_t *h_group_off);
+ * n_accum accumulation settings 0 .. n_accum - 1, then ZeRO stage, gradient checkpointing,
+ * offload); with n_accum = 1 on power-of-two levels the list equals rubick_enumerate_plans'.
+ * A plan whose halved micro-batch would hold less than one sample is invalid for that job.
+ * Same calling convention; 1 <= n_accum <= 8. */
+int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, int n_accum, rubick_plan_wide *h_out, int cap,
+                                int *n_out, int32_t *h_group_off);
 
 /* rubick_set_space for plans with degrees of any size.  The evaluation kernels then divide where
  * the power-of-two space shifts (same model, same memory rule, same tolerances); everything

@@ -33,7 +33,7 @@ FIT_NAMES = ("k_bwd", "k_sync", "k_opt", "k_opt_off", "k_off", "k_swap", "k_cons
 RECONF_DTYPE = np.dtype([("T", "<f4"), ("delta", "<f4"), ("n_reconf", "<i4"), ("active", "<i4")])
 NODE_DTYPE = np.dtype([("free_g", "<i4"), ("free_c", "<i4"), ("free_m", "<i8"), ("owner", "<i4"), ("reserved", "<i4")])
 PLAN_WIDE_DTYPE = np.dtype([("d", "<u2"), ("t", "<u2"), ("p", "<u2"), ("zero", "u1"), ("gc", "u1"), ("off", "u1"),
-                            ("g_level", "u1"), ("disabled", "u1"), ("pad", "u1")])
+                            ("g_level", "u1"), ("disabled", "u1"), ("accum", "u1")])
 assert JOB_DTYPE.itemsize == 128 and PLAN_DTYPE.itemsize == 8 and PLAN_WIDE_DTYPE.itemsize == 12
 assert ASSIGN_DTYPE.itemsize == 40 and NODE_DTYPE.itemsize == 24
 
@@ -97,7 +97,7 @@ def lib():
         L.rubick_last_error.restype = C.c_char_p
         L.rubick_enumerate_plans.argtypes = [vp, ip, vp, ip, C.POINTER(ip), vp]
         L.rubick_set_space.argtypes = [vp, vp, ip, C.POINTER(Grid)]
-        L.rubick_enumerate_plans_wide.argtypes = [vp, ip, vp, ip, C.POINTER(ip), vp]
+        L.rubick_enumerate_plans_wide.argtypes = [vp, ip, ip, vp, ip, C.POINTER(ip), vp]
         L.rubick_set_space_wide.argtypes = [vp, vp, ip, C.POINTER(Grid)]
         L.rubick_eval_candidates.argtypes = [vp, vp, ip, vp, vp]
         L.rubick_best_plan.argtypes = [vp, vp, vp, ip, C.c_uint, vp, vp, vp]
@@ -144,16 +144,16 @@ def enumerate_plans(g_levels):
     return plans[:n.value], off
 
 
-def enumerate_plans_wide(g_levels):
+def enumerate_plans_wide(g_levels, accumulation_levels=1):
     """rubick_enumerate_plans_wide -> (plans as PLAN_WIDE_DTYPE array, group offsets [nG + 1] int32)."""
     gl = np.ascontiguousarray(g_levels, dtype=np.int32)
     n = C.c_int(0)
     off = np.zeros(len(gl) + 1, dtype=np.int32)
-    rc = lib().rubick_enumerate_plans_wide(_ptr(gl), len(gl), None, 0, C.byref(n), _ptr(off))
+    rc = lib().rubick_enumerate_plans_wide(_ptr(gl), len(gl), int(accumulation_levels), None, 0, C.byref(n), _ptr(off))
     if rc:
         raise RubickError(rc, "rubick_enumerate_plans_wide")
     plans = np.zeros(max(n.value, 1), dtype=PLAN_WIDE_DTYPE)
-    rc = lib().rubick_enumerate_plans_wide(_ptr(gl), len(gl), _ptr(plans), n.value, C.byref(n), _ptr(off))
+    rc = lib().rubick_enumerate_plans_wide(_ptr(gl), len(gl), int(accumulation_levels), _ptr(plans), n.value, C.byref(n), _ptr(off))
     if rc:
         raise RubickError(rc, "rubick_enumerate_plans_wide")
     return plans[:n.value], off

@@ -149,7 +149,7 @@ int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out
 namespace {
 
 // one plan with its degrees written out (both plan record formats are brought to this form)
-struct NormPlan { int d, t, p, zero, gc, off, g_level, disabled; };
+struct NormPlan { int d, t, p, zero, gc, off, g_level, disabled, accum; };
 
 int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_grid *h_grid, bool wide)
 {
@@ -193,7 +193,8 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
         const NormPlan &pl = h_plans[i];
         if (pl.g_level >= gr.nG || pl.g_level < level) return fail(ctx, RUBICK_EINVAL, "plans: g_level out of range or not ascending");
         if (pl.zero < 0 || pl.zero > 3 || pl.gc < 0 || pl.gc > 1 || pl.off < 0 || pl.off > 1 || pl.d < 1 || pl.t < 1 || pl.p < 1
-            || pl.d > 32768 || pl.t > 32768 || pl.p > 32768 || int64_t(pl.d) * pl.t * pl.p > (int64_t(1) << 20))
+            || pl.d > 32768 || pl.t > 32768 || pl.p > 32768 || int64_t(pl.d) * pl.t * pl.p > (int64_t(1) << 20)
+            || pl.accum < 0 || pl.accum > 30 || (!wide && pl.accum))
             return fail(ctx, RUBICK_EINVAL, "plans: field out of range");
         if (int64_t(pl.d) * pl.t * pl.p != gr.g_levels[pl.g_level])
             return fail(ctx, RUBICK_EINVAL, "plans: d*t*p differs from the GPU level");
@@ -216,7 +217,7 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
             if (g > Gn) q.flags |= QF_PP_INTER;
         } else {
             const NormPlan &first = h_plans[i - v];
-            if (first.d != pl.d || first.t != pl.t || first.p != pl.p || first.zero != pl.zero)
+            if (first.d != pl.d || first.t != pl.t || first.p != pl.p || first.zero != pl.zero || first.accum != pl.accum)
                 return fail(ctx, RUBICK_EINVAL, "plans: the four plans of a quad must share d, t, p and the ZeRO stage");
         }
         if (pl.disabled) q.disabled |= uint8_t(1u << v);
@@ -226,14 +227,14 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
     for (size_t i = 0; i < quads.size(); ++i) {
         const QuadDesc &a = quads[i & ~size_t(3)], &b = quads[i];
         const NormPlan &pa = h_plans[4 * (i & ~size_t(3))], &pb = h_plans[4 * i];
-        if (b.zero != (i & 3) || pa.d != pb.d || pa.t != pb.t || pa.p != pb.p || a.g_level != b.g_level)
+        if (b.zero != (i & 3) || pa.d != pb.d || pa.t != pb.t || pa.p != pb.p || pa.accum != pb.accum || a.g_level != b.g_level)
             return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with ZeRO stages 0..3 in order (disable plans instead of dropping them)");
     }
     while (level < gr.nG) sp.group_off[++level] = P;
     for (size_t i = 0; i < wquads.size(); ++i) {
         const NormPlan &pl = h_plans[4 * i];
         wquads[i].x = uint32_t(pl.d) | (uint32_t(pl.t) << 16);
-        wquads[i].y = uint32_t(pl.p) | (uint32_t(pl.zero) << 16);
+        wquads[i].y = uint32_t(pl.p) | (uint32_t(pl.zero) << 16) | (uint32_t(pl.accum) << 24);
         wquads[i].z = uint32_t(quads[i].flags) | (uint32_t(quads[i].disabled) << 8);
         wquads[i].w = 0u;
     }
@@ -266,7 +267,7 @@ int rubick_set_space(rubick_ctx *ctx, const rubick_plan *h_plans, int P, const r
     for (int i = 0; i < P; ++i) {
         const rubick_plan &pl = h_plans[i];
         if (pl.log2d > 15 || pl.log2t > 15 || pl.log2p > 15) return fail(ctx, RUBICK_EINVAL, "plans: field out of range");
-        np_list[i] = NormPlan{1 << pl.log2d, 1 << pl.log2t, 1 << pl.log2p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled};
+        np_list[i] = NormPlan{1 << pl.log2d, 1 << pl.log2t, 1 << pl.log2p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled, 0};
     }
     return install_space(ctx, np_list.data(), P, h_grid, false);
 }
@@ -278,15 +279,16 @@ int rubick_set_space_wide(rubick_ctx *ctx, const rubick_plan_wide *h_plans, int 
     std::vector<NormPlan> np_list((size_t(P)));
     for (int i = 0; i < P; ++i) {
         const rubick_plan_wide &pl = h_plans[i];
-        np_list[i] = NormPlan{pl.d, pl.t, pl.p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled};
+        np_list[i] = NormPlan{pl.d, pl.t, pl.p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled, pl.accum};
     }
     return install_space(ctx, np_list.data(), P, h_grid, true);
 }
 
-int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, rubick_plan_wide *h_out, int cap, int *n_out,
-                                int32_t *h_group_off)
+int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, int n_accum, rubick_plan_wide *h_out, int cap,
+                                int *n_out, int32_t *h_group_off)
 {
     if (!h_g_levels || nG < 1 || nG > RUBICK_MAX_G_LEVELS || !n_out || cap < 0 || (cap > 0 && !h_out)) return RUBICK_EINVAL;
+    if (n_accum < 1 || n_accum > 8) return RUBICK_EINVAL;
     for (int i = 0; i < nG; ++i)
         if (h_g_levels[i] <= 0 || h_g_levels[i] > 32768 || (i && h_g_levels[i] <= h_g_levels[i - 1])) return RUBICK_EINVAL;
     int n = 0;
@@ -297,14 +299,15 @@ int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, rubick_plan_w
             if (g % t) continue;
             for (int p = 1; p <= g / t; ++p) {
                 if ((g / t) % p) continue;
-                for (int z = 0; z < 4; ++z)
-                    for (int v = 0; v < 4; ++v, ++n)
-                        if (n < cap) {
-                            rubick_plan_wide &pl = h_out[n];
-                            pl.d = uint16_t(g / (t * p)); pl.t = uint16_t(t); pl.p = uint16_t(p);
-                            pl.zero = uint8_t(z); pl.gc = uint8_t(v >> 1); pl.off = uint8_t(v & 1);
-                            pl.g_level = uint8_t(gi); pl.disabled = 0; pl.pad = 0;
-                        }
+                for (int ga = 0; ga < n_accum; ++ga)
+                    for (int z = 0; z < 4; ++z)
+                        for (int v = 0; v < 4; ++v, ++n)
+                            if (n < cap) {
+                                rubick_plan_wide &pl = h_out[n];
+                                pl.d = uint16_t(g / (t * p)); pl.t = uint16_t(t); pl.p = uint16_t(p);
+                                pl.zero = uint8_t(z); pl.gc = uint8_t(v >> 1); pl.off = uint8_t(v & 1);
+                                pl.g_level = uint8_t(gi); pl.disabled = 0; pl.accum = uint8_t(ga);
+                            }
             }
         }
     }

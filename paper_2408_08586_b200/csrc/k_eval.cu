@@ -111,10 +111,10 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
                                            uint32_t *__restrict__ feas, Emit &&emit)
 {
     const JobRegs jb = load_job(jobs + j);
-    int ld = 0, lt = 0, lp = 0, lg = 0, d, t, p, z, qflags, disabled;
+    int ld = 0, lt = 0, lp = 0, lg = 0, accum = 0, d, t, p, z, qflags, disabled;
     if constexpr (WIDE) {
         const uint4 qraw = __ldg(reinterpret_cast<const uint4 *>(quads_any) + q);
-        d = qraw.x & 0xffff; t = qraw.x >> 16; p = qraw.y & 0xffff; z = (qraw.y >> 16) & 0xff;
+        d = qraw.x & 0xffff; t = qraw.x >> 16; p = qraw.y & 0xffff; z = (qraw.y >> 16) & 0xff; accum = qraw.y >> 24;
         qflags = qraw.z & 0xff; disabled = (qraw.z >> 8) & 0xff;
     } else {
         const uint2 qraw = __ldg(reinterpret_cast<const uint2 *>(quads_any) + q);
@@ -133,11 +133,13 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
     bool valid = (qflags & QF_T_FITS_NODE) && p <= jb.l && d <= jb.b && !(sp.strict && z > 0 && (t > 1 || p > 1));
     if constexpr (WIDE) valid = valid && jb.b % d == 0 && jb.h % t == 0;
     else valid = valid && (jb.b & (d - 1)) == 0 && (jb.h & (t - 1)) == 0;
-    const bool valid_off = valid && z >= 2;
-
     // micro-batching
     const int r = max(WIDE ? jb.b / d : jb.b >> ld, 1);
-    const int mu = min(r, max(jb.mu_cap, 1));
+    // explicit accumulation (wide space): the micro-batch halved `accum` times; it must still hold a sample
+    const int mu_most = min(r, max(jb.mu_cap, 1));
+    const int mu = max(mu_most >> accum, 1);
+    if constexpr (WIDE) valid = valid && (mu_most >> accum) >= 1;
+    const bool valid_off = valid && z >= 2;
     const int n = (r + mu - 1) / mu;
     const int m = p > 1 ? n : 1;
     const int a = p > 1 ? 1 : n;

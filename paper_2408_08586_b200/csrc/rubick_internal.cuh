@@ -27,7 +27,7 @@ enum : uint8_t {
 };
 
 // A plan quad of the wide plan space (degrees of any size), 16 bytes, read as one uint4:
-// x = d | t << 16, y = p | ZeRO stage << 16, z = QF_* flags | disabled bits << 8, w = 0.
+// x = d | t << 16, y = p | ZeRO stage << 16 | micro-batch halvings << 24, z = QF_* flags | disabled bits << 8, w = 0.
 struct WideQuad { uint32_t x, y, z, w; };
 
 // Everything a kernel needs to know about the environment and the grid; passed by value as a

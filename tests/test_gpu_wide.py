@@ -29,29 +29,32 @@ def wide_config(J, levels, gpus_per_node, n_nodes, seed=6):
     return cfg
 
 
-def oracle_wide(cfg, nthreads=8):
-    plans, goff = oracle.enumerate_plans(cfg["g_levels"], any_degrees=True)
+def oracle_wide(cfg, nthreads=8, accumulation_levels=1):
+    plans, goff = oracle.enumerate_plans(cfg["g_levels"], any_degrees=True, accumulation_levels=accumulation_levels)
     thr, feas = oracle.eval_candidates(cfg["jobs"], plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=nthreads)
     cv, cp, cg = oracle.best_plan(thr.astype(np.float32), feas, plans, cfg["g_levels"], len(cfg["m_levels"]), prefix=True, nthreads=nthreads)
     return plans, goff, thr, feas, cv.astype(np.float32), cp, cg
 
 
 def test_wide_enumerators_agree():
-    for levels in ([1, 2, 3, 4, 5, 6, 7, 8], [1, 2, 3, 4, 6, 8, 16, 24, 48], [1, 2, 4, 8, 16]):
-        got, goff = rb.enumerate_plans_wide(levels)
-        want, woff = oracle.enumerate_plans(levels, any_degrees=True)
+    for levels, n_acc in (([1, 2, 3, 4, 5, 6, 7, 8], 1), ([1, 2, 3, 4, 6, 8, 16, 24, 48], 3), ([1, 2, 4, 8, 16], 2)):
+        got, goff = rb.enumerate_plans_wide(levels, accumulation_levels=n_acc)
+        want, woff = oracle.enumerate_plans(levels, any_degrees=True, accumulation_levels=n_acc)
         assert np.array_equal(goff, woff) and len(got) == len(want)
-        for col, name in enumerate(("d", "t", "p", "zero", "gc", "off")):
+        for col, name in enumerate(("d", "t", "p", "zero", "gc", "off", "accum")):
             assert np.array_equal(got[name].astype(np.int64), want[:, col])
         assert np.array_equal(got["g_level"], np.searchsorted(woff[1:], np.arange(len(want)), side="right"))
 
 
-@pytest.mark.parametrize("levels,gn,N", [([1, 2, 3, 4, 6, 8, 16, 24, 48], 8, 7), ([1, 2, 3, 4, 8, 12, 24], 4, 9)])
-def test_wide_plan_space_through_every_kernel(levels, gn, N):
+@pytest.mark.parametrize("levels,gn,N,n_acc", [([1, 2, 3, 4, 6, 8, 16, 24, 48], 8, 7, 1), ([1, 2, 3, 4, 8, 12, 24], 4, 9, 1),
+                                               ([1, 2, 3, 4, 6, 8, 16], 8, 5, 3)])
+def test_wide_plan_space_through_every_kernel(levels, gn, N, n_acc):
     J = 41
     cfg = wide_config(J, levels, gn, N)
-    plans, goff, thr, feas, cv, cp, cg = oracle_wide(cfg)
-    gpu_plans, _ = rb.enumerate_plans_wide(levels)
+    if n_acc > 1:
+        cfg["env"]["gpu_mem_bytes"] = 24_000_000_000       # small GPUs: plans that only fit with smaller micro-batches
+    plans, goff, thr, feas, cv, cp, cg = oracle_wide(cfg, accumulation_levels=n_acc)
+    gpu_plans, _ = rb.enumerate_plans_wide(levels, accumulation_levels=n_acc)
     gpu = Gpu(cfg, plans=gpu_plans)
     assert gpu.P == len(plans)
     _, d_thr, d_feas = gpu.eval(cfg["jobs"])
@@ -66,6 +69,8 @@ def test_wide_plan_space_through_every_kernel(levels, gn, N):
     assert np.array_equal(bv.cpu().numpy().reshape(sh), cv)
     assert np.array_equal(bp.cpu().numpy().reshape(sh), cp) and np.array_equal(bg.cpu().numpy().reshape(sh), cg)
     assert odd[cp[cp >= 0]].any()                                          # and win somewhere
+    if n_acc > 1:
+        assert (plans[cp[cp >= 0], 6] > 0).any()                           # plans with extra accumulation win where memory is short
     gpu.assert_one_pass_curves_match(cfg["jobs"])
     want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
                                  N, want_log=True)
