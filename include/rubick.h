@@ -214,8 +214,8 @@ int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, int n_accum, 
 
 /* rubick_set_space for plans with degrees of any size.  The evaluation kernels then divide where
  * the power-of-two space shifts (same model, same memory rule, same tolerances); everything
- * downstream (best plan, curves, gains, rounds) is unchanged.  rubick_fit_models needs the
- * power-of-two space.  GPU levels above a node must still be whole nodes. */
+ * downstream (best plan, curves, gains, rounds, fitting) is unchanged.  GPU levels above a node
+ * must still be whole nodes. */
 int rubick_set_space_wide(rubick_ctx *ctx, const rubick_plan_wide *h_plans, int P, const rubick_grid *h_grid);
 
 /* Candidate table (paper Section 4, Eq. 1 with all its terms; THROUGHPUT = b / T_iter) and the

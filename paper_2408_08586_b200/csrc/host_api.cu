@@ -410,10 +410,9 @@ int rubick_fit_models(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const ru
     if (!d_jobs || !d_samples || !d_theta || !d_rmsle) return fail(ctx, RUBICK_EINVAL, "null pointer");
     if (S < 1 || S > 4096) return fail(ctx, RUBICK_EINVAL, "1 .. 4096 sample slots per model");
     if (sweeps < 0 || sweeps > 64) return fail(ctx, RUBICK_EINVAL, "0 .. 64 sweeps");
-    if (ctx->space.wide) return fail(ctx, RUBICK_ESTATE, "model fitting works on the power-of-two plan space (rubick_set_space)");
     if ((reinterpret_cast<uintptr_t>(d_samples) & 7) || (reinterpret_cast<uintptr_t>(d_theta) & 7) || (reinterpret_cast<uintptr_t>(d_rmsle) & 7))
         return fail(ctx, RUBICK_EINVAL, "d_samples, d_theta and d_rmsle must be 8-byte aligned");
-    CUDA_TRY(ctx, launch_fit(ctx->env, ctx->d_quads, ctx->space.P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle, ctx->stream),
+    CUDA_TRY(ctx, launch_fit(ctx->env, ctx->d_quads, ctx->space.wide ? ctx->d_wide_quads : nullptr, ctx->space.P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle, ctx->stream),
              "launch fit_models");
     return RUBICK_OK;
 }

@@ -42,18 +42,25 @@ __device__ __forceinline__ double overlap(double k, double x, double y)
 // Throughput of Eq. 1 for job jb with trial coefficients th[] under plan `idx` with c cores; 0 when the
 // plan is structurally invalid for the job.
 __device__ double model_thr(const rubick_job &jb, const double *th, const FitEnv &ev, const QuadDesc *__restrict__ quads,
-                            int idx, double c)
+                            const WideQuad *__restrict__ wide, int idx, double c)
 {
     const QuadDesc q = quads[idx >> 2];
     const int v = idx & 3, gc = v >> 1, off = v & 1, z = q.zero;
     if (q.disabled & (1u << v)) return 0.0;
-    const long long d = 1ll << q.log2d, t = 1ll << q.log2t, p = 1ll << q.log2p;
+    long long d = 1ll << q.log2d, t = 1ll << q.log2t, p = 1ll << q.log2p;
+    int accum = 0;
+    if (wide) {                         // degrees of any size and the accumulation setting
+        const WideQuad w = wide[idx >> 2];
+        d = w.x & 0xffff; t = w.x >> 16; p = w.y & 0xffff; accum = int(w.y >> 24);
+    }
     const long long b = jb.b, l = jb.l, h = jb.h;
     if (t > ev.Gn || p > l || d > b || b % d != 0 || (off && z < 2) || h % t != 0) return 0.0;
     if (ev.strict && (z > 0 || off) && (t > 1 || p > 1)) return 0.0;
 
     const long long r = b / d;
-    const long long mu_i = r < jb.mu_cap ? r : jb.mu_cap;
+    const long long mu_most = r < jb.mu_cap ? r : jb.mu_cap;
+    if ((mu_most >> accum) < 1) return 0.0;
+    const long long mu_i = mu_most >> accum;
     const long long n = (r + mu_i - 1) / mu_i;
     const double mu = double(mu_i), m = p > 1 ? double(n) : 1.0, a = p > 1 ? 1.0 : double(n);
     const double dd = double(d), tt = double(t), pp = double(p), g = dd * tt * pp;
@@ -88,13 +95,14 @@ __device__ double model_thr(const rubick_job &jb, const double *th, const FitEnv
 // Sum of squared log errors over all samples; the lanes that differ only in `part` hold the same th[] and
 // end up with the same total (pairwise sums of their partial sums).  Warp-wide.
 __device__ double sum_sq_log_err(const rubick_job &jb, const double *th, const FitEnv &ev, const QuadDesc *__restrict__ quads,
-                                 const rubick_sample *__restrict__ smp, int S, int P, int part, int *n_out)
+                                 const WideQuad *__restrict__ wide, const rubick_sample *__restrict__ smp, int S, int P,
+                                 int part, int *n_out)
 {
     double sse = 0.0; int n = 0;
     for (int i = part; i < S; i += FIT_PARTS) {
         const rubick_sample x = smp[i];
         if (x.plan < 0 || x.plan >= P) continue;
-        const double e = log1p(model_thr(jb, th, ev, quads, x.plan, double(x.cores))) - log1p(x.thr);
+        const double e = log1p(model_thr(jb, th, ev, quads, wide, x.plan, double(x.cores))) - log1p(x.thr);
         sse += e * e; ++n;
     }
     sse += __shfl_xor_sync(0xffffffffu, sse, 8);
@@ -104,7 +112,7 @@ __device__ double sum_sq_log_err(const rubick_job &jb, const double *th, const F
 }
 
 __global__ void __launch_bounds__(64)
-fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict__ quads, int P,
+fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict__ quads, const WideQuad *__restrict__ wide, int P,
                   const rubick_job *__restrict__ jobs, int J, const rubick_sample *__restrict__ samples, int S,
                   int sweeps, double *__restrict__ theta_out, double *__restrict__ rmsle_out)
 {
@@ -127,7 +135,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
         if (th[p] > hi[p]) th[p] = hi[p];
     }
     int n = 0;
-    double cur = sum_sq_log_err(jb, th, ev, quads, smp, S, P, part, &n);
+    double cur = sum_sq_log_err(jb, th, ev, quads, wide, smp, S, P, part, &n);
     const double rmsle0 = n > 0 ? sqrt(cur / n) : 0.0;
     double M = sqrt(2.0) * sqrt(sqrt(2.0));
     const int e_of_q = (q & 1) ? ((q >> 1) + 1) : -((q >> 1) + 1);     // q = 0..7 -> -1, +1, -2, +2, -3, +3, -4, +4
@@ -145,7 +153,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
             if (v < lo[p]) v = lo[p];
             if (v > hi[p]) v = hi[p];
             th[p] = v;
-            const double sse = sum_sq_log_err(jb, th, ev, quads, smp, S, P, part, nullptr);
+            const double sse = sum_sq_log_err(jb, th, ev, quads, wide, smp, S, P, part, nullptr);
             th[p] = base;
             // the eight errors in candidate order, as one after the other would see them
             double best = cur, best_v = base;
@@ -170,7 +178,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
                 th[p] = v;
             }
             if (!moved) break;
-            const double sse = sum_sq_log_err(jb, th, ev, quads, smp, S, P, part, nullptr);
+            const double sse = sum_sq_log_err(jb, th, ev, quads, wide, smp, S, P, part, nullptr);
             if (sse < cur * (1.0 - FIT_EPS)) {
                 cur = sse;
 #pragma unroll
@@ -191,7 +199,7 @@ fit_models_kernel(const __grid_constant__ FitEnv ev, const QuadDesc *__restrict_
     }
 }
 
-cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, int P, const rubick_job *d_jobs, int J,
+cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, const WideQuad *d_wide_quads, int P, const rubick_job *d_jobs, int J,
                        const rubick_sample *d_samples, int S, int sweeps, double *d_theta, double *d_rmsle, cudaStream_t st)
 {
     if (J == 0) return cudaSuccess;
@@ -199,7 +207,7 @@ cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, int P, co
     ev.B_intra = env.B_intra; ev.B_inter = env.B_inter; ev.B_pcie = env.B_pcie; ev.e = double(env.bytes_per_elem);
     ev.Gn = env.gpus_per_node; ev.strict = env.strict_zero_dp_only ? 1 : 0;
     const int threads = 64, per_block = threads / 32;
-    fit_models_kernel<<<(J + per_block - 1) / per_block, threads, 0, st>>>(ev, d_quads, P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle);
+    fit_models_kernel<<<(J + per_block - 1) / per_block, threads, 0, st>>>(ev, d_quads, d_wide_quads, P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle);
     return cudaGetLastError();
 }
 

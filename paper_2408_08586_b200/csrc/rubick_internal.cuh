@@ -119,7 +119,7 @@ cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const 
 cudaError_t launch_min_resources(const Space &sp, const QuadDesc *d_quads, const float *d_thr, const uint32_t *d_feas,
                                  const float *d_cv, int J, const rubick_request *d_req, int32_t *d_gmin, int32_t *d_cmin,
                                  float *d_baseline, cudaStream_t st);
-cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, int P, const rubick_job *d_jobs, int J,
+cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, const WideQuad *d_wide_quads, int P, const rubick_job *d_jobs, int J,
                        const rubick_sample *d_samples, int S, int sweeps, double *d_theta, double *d_rmsle, cudaStream_t st);
 size_t round_scratch_need(const Space &sp, int J, int N);
 size_t incr_scratch_need(const Space &sp, int J, int N);

@@ -95,14 +95,8 @@ def test_wide_space_validation_and_limits():
         gpu.ctx.set_space(bad, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"])
     with pytest.raises(rb.RubickError):                    # 12 GPUs on 8-GPU nodes is not a whole number of nodes
         gpu.ctx.set_space(*((lambda p: (p, [1, 2, 12], cfg["c_levels"], cfg["m_levels"]))(rb.enumerate_plans_wide([1, 2, 12])[0])))
-    # fitting needs the power-of-two space
-    t = gpu.torch
-    gpu.ctx.set_space(plans, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"])
-    d = gpu.empty(4096, t.float64)
-    with pytest.raises(rb.RubickError) as ei:
-        gpu.ctx.fit_models(d, 1, d, 4, 4, d, d)
-    assert ei.value.code == rb.ESTATE
     # the power-of-two format refuses other degrees; the wide format on power-of-two levels equals it
+    t = gpu.torch
     p2, _ = rb.enumerate_plans([1, 2, 4, 8])
     w2, _ = rb.enumerate_plans_wide([1, 2, 4, 8])
     assert np.array_equal(1 << p2["log2d"].astype(np.int64), w2["d"]) and np.array_equal(1 << p2["log2t"].astype(np.int64), w2["t"])
@@ -114,3 +108,24 @@ def test_wide_space_validation_and_limits():
     _, thr_b, feas_b = b.eval(cfg2["jobs"])
     assert t.equal(feas_a, feas_b)
     assert np.allclose(thr_a.cpu().numpy(), thr_b.cpu().numpy(), rtol=2e-6, atol=0)
+
+
+def test_model_fitting_on_the_wide_plan_space():
+    """Samples on plans with odd degrees and explicit accumulation; same decisions as the oracle's fit."""
+    from test_gpu_fit import gpu_fit
+    from test_oracle_fit import with_coefficients
+    J, S = 24, 16
+    cfg = wide_config(J, [1, 2, 3, 4, 6, 8], 8, 2)
+    plans, goff, thr, feas, *_ = oracle_wide(cfg, accumulation_levels=2)
+    picks = workloads.draw_fit_picks(5, J, S, len(cfg["c_levels"]))
+    sp, sc, sy = workloads.fit_samples(cfg, plans, thr, feas, picks)
+    assert ((plans[np.maximum(sp, 0), 1] == 3) & (sp >= 0)).any() and ((plans[np.maximum(sp, 0), 6] == 1) & (sp >= 0)).any()
+    start = with_coefficients(cfg["jobs"], {k: np.float32(v) for k, v in workloads.FIT_NOMINAL.items()})
+    want_theta, want_rmsle, margin = oracle.fit(start, plans, cfg["env"], sp, sc, sy, sweeps=10)
+    gpu_plans, _ = rb.enumerate_plans_wide(cfg["g_levels"], accumulation_levels=2)
+    gpu = Gpu(cfg, plans=gpu_plans)
+    theta, rmsle = gpu_fit(gpu, start, sp, sc, sy, sweeps=10)
+    assert np.allclose(rmsle, want_rmsle, rtol=1e-9, atol=1e-13)
+    firm = margin > 1e-11
+    assert firm.mean() > 0.8 and np.array_equal(theta[firm], want_theta[firm])
+    assert np.all(rmsle[:, 1] <= rmsle[:, 0]) and np.median(rmsle[:, 1]) < 0.5 * np.median(rmsle[:, 0])
