@@ -3,7 +3,10 @@
  * Rubick scheduler (arXiv 2408.08586): batched evaluation of the paper's training-performance
  * model over every (job x execution plan x resource allocation) candidate, the memory-feasibility
  * mask, the per-(job, allocation) best plan and resource-sensitivity curve, per-job marginal
- * gains, and a greedy allocation round that runs entirely on the device.
+ * gains, and a greedy allocation round that runs entirely on the device; further the minimum
+ * demand of guaranteed jobs and tenant quotas, the incremental round (shrink / exchange step,
+ * preemption, reconfiguration gate), batched fitting of the model's coefficients, and a wider plan
+ * space (degrees of any size, explicit gradient accumulation).
  *
  * Conventions
  *  - Every call returns an int: RUBICK_OK (0) or a negative error code.  Nothing throws, aborts
