@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM traffic of one eval_candidates launch from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum), as bytes per stored candidate; valid only for the kernel source it was
 # taken on (sha1 of k_eval.cu), otherwise reported as null.
-NCU_EVAL_TRAFFIC = {"k_eval_sha1": "be3bea64fb9d94bf621f04a5f1b0cff9846fb976", "bytes_per_candidate": 485.98554e6 / (2048 * 2640 * 24)}
+NCU_EVAL_TRAFFIC = {"k_eval_sha1": "782b20d6b0a3e6b89f7fd39fc5f12914d71aa5f6", "bytes_per_candidate": 483.89939e6 / (2048 * 2640 * 24)}
 
 
 def shard_seed_offset(rank):

@@ -273,8 +273,10 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const void *__restrict_
     const int j = int(gid / uint32_t(sp.Q));
     const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
     float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
-    eval_quad<false, WIDE>(sp, quads, jobs, j, q, active, feas, [&](int ci, const float4 &out, const uint4 &) {
-        if (active) __stcs(reinterpret_cast<float4 *>(row + size_t(ci) * sp.P), out);
+    // levels arrive in ascending order, one call each: the row pointer just advances
+    eval_quad<false, WIDE>(sp, quads, jobs, j, q, active, feas, [&](int, const float4 &out, const uint4 &) {
+        if (active) __stcs(reinterpret_cast<float4 *>(row), out);
+        row += sp.P;
     });
 }
 
