@@ -84,6 +84,9 @@ __device__ __forceinline__ size_t curve_idx(const Space &sp, int j, int gi, int 
 }
 __device__ __forceinline__ size_t hc_idx(const Space &sp, int j, int gi, int ci) { return (size_t(j) * sp.nG + gi) * sp.nC + ci; }
 __device__ __forceinline__ int64_t cdiv64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+// ceil(a / k), a >= 0, k >= 1: node counts of jobs on whole nodes usually are powers of two (a shift, no division)
+__device__ __forceinline__ int cdiv_k(int a, int k) { return (k & (k - 1)) ? (a + k - 1) / k : (a + k - 1) >> (__ffs(k) - 1); }
+__device__ __forceinline__ int64_t cdiv64_k(int64_t a, int k) { return (k & (k - 1)) ? (a + k - 1) / k : (a + k - 1) >> (__ffs(k) - 1); }
 __device__ __forceinline__ HotCurve load_hc(const HotCurve *p)
 {
     const int4 v = *reinterpret_cast<const int4 *>(p);
@@ -232,6 +235,7 @@ struct Shared {
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
     int scan_cnt[RW];
+    unsigned long long sel[32];   // batch selection: one ordering word per lane
 };
 
 // warp-cooperative: first node with at least g free GPUs and c free cores, -1 if none
@@ -249,6 +253,31 @@ __device__ int first_fit_warp(const Views &v, int g, int c, int lane)
         if (b) return __shfl_sync(0xffffffffu, base + 4 * lane + first, __ffs(b) - 1);
     }
     return -1;
+}
+
+// warp-cooperative: maxc[] for every level in one sweep over the node words (lane 0 stores).  Levels ascend, so
+// a node counts for the levels below the first one it has too few free GPUs for.
+__device__ void rebuild_maxc_warp(const Space &sp, const Views &v, int lane)
+{
+    const int4 *w4 = reinterpret_cast<const int4 *>(v.gc);
+    for (int i0 = 0; i0 < sp.n_small; i0 += 4) {
+        int g_[4], m_[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) { g_[u] = i0 + u < sp.n_small ? v.gl[i0 + u] : 0x7fffffff; m_[u] = -1; }
+        for (int base = 0; base < v.N_pad; base += 128) {
+            const int4 x = w4[(base >> 2) + lane];
+            const int w_[4] = { x.x, x.y, x.z, x.w };
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int u = 0; u < 4; ++u) m_[u] = max(m_[u], fg_of(w_[q]) >= g_[u] ? fc_of(w_[q]) : -1);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int m = __reduce_max_sync(0xffffffffu, m_[u]);
+            if (lane == 0 && i0 + u < sp.n_small) v.maxc[i0 + u] = m;
+        }
+    }
 }
 
 // warp-cooperative: most free cores among the nodes with at least g free GPUs (-1 if none).  A job of
@@ -269,14 +298,15 @@ __device__ int max_cores_warp(const Views &v, int g, int lane)
 
 struct Committed { int first; float val; int plan; int f; };
 
-// Commit job j to (gi2, ci2); one warp, all lanes, uniform control flow.  `alloc`: the job holds
+// Commit job j to (gi2, ci2); one warp, all lanes, uniform control flow.  `alloc` (compile time): the job holds
 // (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target at
 // the top memory level.  On success node state and empty-node count are current; maxc[] is rebuilt
 // here when `rebuild`, otherwise sh.maxc_dirty / sh.ver / sh.t0 / sh.t1 tell the block what changed.
+template <bool alloc, bool rebuild>
 __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const float *__restrict__ cv,
                             const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
-                            const uint32_t *__restrict__ feas, int j, bool alloc, int gi, int ci, int node,
-                            float val_cur, int f_cur, int gi2, int ci2, HotCurve cand, bool need_gain, bool rebuild,
+                            const uint32_t *__restrict__ feas, int j, int gi, int ci, int node,
+                            float val_cur, int f_cur, int gi2, int ci2, HotCurve cand, bool need_gain,
                             int lane, Committed &out)
 {
     const int g = alloc ? sp.g_levels[gi] : 0, c = alloc ? sp.c_levels[ci] : 0;
@@ -397,10 +427,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     }
     __syncwarp();
     if (rebuild) {
-        for (int i = 0; i < sp.n_small && maxc_dirty; ++i) {
-            const int m = max_cores_warp(v, sp.g_levels[i], lane);
-            if (lane == 0) v.maxc[i] = m;
-        }
+        if (maxc_dirty) rebuild_maxc_warp(sp, v, lane);
         if (lane == 0) sh.n_empty = n_empty + d_empty;
         __syncwarp();
     } else if (lane == 0) {
@@ -468,7 +495,7 @@ __device__ SlotC make_slotc(const Space &sp, const int32_t *gl, const int32_t *c
         if (g2 <= sp.Gn) { s.gkind = K_SINGLE; s.dg = int16_t(g2 - g); s.gidx = uint8_t(next_g); }
         else {
             const int k2 = g2 >> sp.log2Gn;
-            if ((c + k2 - 1) / k2 <= sp.Cn) {
+            if (cdiv_k(c, k2) <= sp.Cn) {
                 if (g >= sp.Gn) { s.gkind = K_MULTI_WHOLE; s.need = int16_t(k2 - (g >> sp.log2Gn)); }
                 else { s.gkind = K_MULTI_PART; s.need = int16_t(k2); }
             }
@@ -478,7 +505,7 @@ __device__ SlotC make_slotc(const Space &sp, const int32_t *gl, const int32_t *c
         const int c2 = clv[next_c];
         s.c2 = int16_t(c2);
         if (g <= sp.Gn) { s.ckind = K_SINGLE; s.dc = int16_t(c2 - c); }
-        else { const int k = g >> sp.log2Gn; if ((c2 + k - 1) / k <= sp.Cn) s.ckind = K_MULTI_WHOLE; }
+        else { const int k = g >> sp.log2Gn; if (cdiv_k(c2, k) <= sp.Cn) s.ckind = K_MULTI_WHOLE; }
     }
     return s;
 }
@@ -660,7 +687,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[ci]) continue;
                 }
                 Committed cm;
-                if (commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, true, lane, cm)) {
+                if (commit_warp<false, true>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm)) {
                     const int s = sh.n_slots;
                     if (lane == 0) {
                         SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
@@ -856,7 +883,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
                     const int w_old = v.gc[a.node];
                     const int k = g > sp.Gn ? g >> sp.log2Gn : 1;
-                    st = g > sp.Gn ? (!type_gpu && (c2 + k - 1) / k <= sp.Cn)
+                    st = g > sp.Gn ? (!type_gpu && cdiv_k(c2, k) <= sp.Cn)
                                    : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
                 }
                 top_stays = __any_sync(FULL, st);
@@ -871,6 +898,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 na.gain_g = na.gain_c = 0.0f; na.packed = 0u; na.node = -1;
                 nb.val = 0.0f; nb.plan = -1; nb.f_level = 0; nb.w = 0.0f;
                 nq.gkind = nq.ckind = K_NONE; nq.gidx = nq.cidx = 0; nq.dg = nq.need = nq.dc = nq.c = nq.c2 = nq.g = 0;
+                // the same for every lane: while an empty node remains and every maxc[] entry is the node's core
+                // count no commit that stays on its node can change maxc[]; the first four levels in registers
+                const bool saturated = sh.n_empty > 0 && __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
+                int mx_r[4], gl_r[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { mx_r[u] = u < sp.n_small ? v.maxc[u] : -2; gl_r[u] = u < sp.n_small ? v.gl[u] : 0x7fffffff; }
                 if (key != 0u && !(my_pay & 0x80000000u)) {
                     const int s = int(my_pay), j = my_j;
                     const SlotA a = v.sa[s];
@@ -882,26 +915,27 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     // stays where it is: room on its own node, or more cores on the whole nodes it already holds
                     const bool multi = g > sp.Gn;
                     const int k = multi ? g >> sp.log2Gn : 1;
-                    const bool stays = multi ? (!type_gpu && (c2 + k - 1) / k <= sp.Cn)
+                    const bool stays = multi ? (!type_gpu && cdiv_k(c2, k) <= sp.Cn)
                                              : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
                     if (stays) {
                         // everything the commit and the new gains can need, in one wave of loads
                         const SlotB b = v.sb[s];
                         const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                        float col[4];
+                        float col[8];
 #pragma unroll
-                        for (int u = 0; u < 4; ++u) col[u] = gi2 + 1 + u < sp.nG ? A.hc[hc_idx(sp, j, gi2 + 1 + u, ci2)].val : 0.0f;
+                        for (int u = 0; u < 8; ++u) col[u] = gi2 + 1 + u < sp.nG ? A.hc[hc_idx(sp, j, gi2 + 1 + u, ci2)].val : 0.0f;
                         const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
                         const int64_t m_cur = v.ml[b.f_level];
                         const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
-                        int lo = 0, hi = sp.nM;                 // number of levels <= avail (levels ascend)
-                        while (lo < hi) { const int mid = (lo + hi) >> 1; if (v.ml[mid] <= avail) lo = mid + 1; else hi = mid; }
-                        const int mi = lo - 1;
+                        // levels ascend: the highest level that fits is below 0 / at least cand.f exactly when
+                        // level 0 / level cand.f itself does not fit / fits
+                        const bool none_fits = v.ml[0] > avail;
+                        const bool cand_fits = cand.plan >= 0 && cand.f >= 0 && cand.f < sp.nM && v.ml[cand.f >= 0 && cand.f < sp.nM ? cand.f : 0] <= avail;
                         s_multi = multi; s_k = k;
                         bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                         s_slot = s; s_node = a.node; s_type = type_gpu;
-                        if (mi < 0) { elig = true; s_ok = false; }
-                        else if (cand.plan >= 0 && cand.f >= 0 && cand.f <= mi) {
+                        if (none_fits) { elig = true; s_ok = false; }
+                        else if (cand_fits) {
                             elig = true;
                             s_ok = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
                         }
@@ -909,13 +943,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             // new gains: first GPU level above gi2 whose curve value exceeds the new value
                             const float val = cand.val, vcur = __fmul_rn(b.w, val);
                             int ng_ = -1, nc_ = -1; float gg = 0.0f, gc = 0.0f;
-                            for (int base = gi2 + 1; base < sp.nG && ng_ < 0; base += 4) {
-                                if (base > gi2 + 1) {
 #pragma unroll
-                                    for (int u = 0; u < 4; ++u) col[u] = base + u < sp.nG ? A.hc[hc_idx(sp, j, base + u, ci2)].val : 0.0f;
-                                }
-#pragma unroll
-                                for (int u = 3; u >= 0; --u) if (base + u < sp.nG && col[u] > val) { ng_ = base + u; gg = col[u]; }
+                            for (int u = 7; u >= 0; --u) if (gi2 + 1 + u < sp.nG && col[u] > val) { ng_ = gi2 + 1 + u; gg = col[u]; }
+                            for (int lvl = gi2 + 9; lvl < sp.nG && ng_ < 0; ++lvl) {
+                                const float x = A.hc[hc_idx(sp, j, lvl, ci2)].val;
+                                if (x > val) { ng_ = lvl; gg = x; }
                             }
                             if (ng_ >= 0) gg = __fdiv_rn(__fsub_rn(__fmul_rn(b.w, gg), vcur), float(v.gl[ng_] - g2));
                             if (ci2 + 1 < sp.nC) {
@@ -929,20 +961,25 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             if (multi) {
                                 // per-node shares of cores and memory on each of the k nodes (they hold no free GPU,
                                 // so maxc[] cannot change)
-                                s_dgc = (c2 + k - 1) / k - (c + k - 1) / k;
-                                s_dm = cdiv64(v.ml[cand.f], k) - cdiv64(m_cur, k);
+                                s_dgc = cdiv_k(c2, k) - cdiv_k(c, k);
+                                s_dm = cdiv64_k(v.ml[cand.f], k) - cdiv64_k(m_cur, k);
                             } else {
                                 s_dgc = ((g2 - g) << 16) + (c2 - c);
                                 s_dm = v.ml[cand.f] - m_cur;
                             }
                             // can maxc[] change?  (the node only loses GPUs / cores)
                             const int w_new = w_old - s_dgc;
-                            bool saturated = sh.n_empty > 0;
-                            for (int i = 0; i < sp.n_small; ++i) saturated = saturated && v.maxc[i] == sp.Cn;
-                            for (int i = 0; i < sp.n_small && !multi && !saturated; ++i) {
-                                const int glv = v.gl[i], mx = v.maxc[i];
-                                const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
-                                s_maxc = s_maxc || (ot == mx && nt < ot);
+                            if (!multi && !saturated) {
+#pragma unroll
+                                for (int u = 0; u < 4; ++u) {
+                                    const int ot = fg_of(w_old) >= gl_r[u] ? fc_of(w_old) : -1, nt = fg_of(w_new) >= gl_r[u] ? fc_of(w_new) : -1;
+                                    s_maxc = s_maxc || (ot == mx_r[u] && nt < ot);
+                                }
+                                for (int i = 4; i < sp.n_small; ++i) {
+                                    const int glv = v.gl[i], mx = v.maxc[i];
+                                    const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
+                                    s_maxc = s_maxc || (ot == mx && nt < ot);
+                                }
                             }
                         } else if (elig) {
                             // rejected: the (job, type) pair is frozen, the other increment stays as it is
@@ -968,23 +1005,32 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         }
                     }
                 }
-                // take the candidates in the order the sequential rule would
-                uint32_t rem = key, T = M;
-                unsigned acc = 0u;
-                int my_order = -1;
-                while (n_acc < room) {
-                    uint32_t k = rem, src_lane = uint32_t(lane); int kj = my_j;
-                    warp_select(k, kj, src_lane);
-                    if (k == 0u || k <= T) break;
-                    const int wl = int(src_lane);
-                    if (!__shfl_sync(FULL, int(elig), wl)) break;
-                    const int nd = __shfl_sync(FULL, s_node, wl);
-                    if (__any_sync(FULL, ((acc >> lane) & 1u) && s_node == nd)) break;
-                    acc |= 1u << wl;
-                    if (lane == wl) { my_order = n_acc; rem = 0u; }
-                    const uint32_t bnd = __shfl_sync(FULL, s_bound, wl);
-                    T = bnd > T ? bnd : T;
-                    ++n_acc;
+                // Take the candidates in the order the sequential rule would: by descending key, lowest job first
+                // among equal keys.  The rule goes on while the next candidate could be worked out here, sits on a
+                // node of its own, and its key exceeds M and the bound of every candidate before it.  All of this
+                // holds for the candidates above one threshold t: the largest of M, the keys of the candidates that
+                // could not be worked out, the keys of those that share a node with a candidate ranked before them,
+                // and, among what is left, every bound (a bound at or above its own key: that key).  They form a
+                // prefix of the order, possibly a little shorter than the longest one; the rest waits a turn.
+                const u64 mine = (u64(key) << 32) | (key ? u64(uint32_t(KEY_JOB_MASK) - uint32_t(my_j)) << 5 : 0ull) | u64(31 - lane);
+                sh.sel[lane] = mine;                         // key, then lowest job, then lane: all words differ
+                __syncwarp();
+                const bool usable = key != 0u && elig;
+                uint32_t t = __reduce_max_sync(FULL, key != 0u && !elig ? key : 0u);
+                if (M > t) t = M;
+                bool lower = false;                          // a candidate ranked before this one sits on the same node
+                for (unsigned m = __match_any_sync(FULL, usable ? s_node : -1 - lane) & ~(1u << lane); m; m &= m - 1)
+                    lower = lower || sh.sel[__ffs(m) - 1] > mine;
+                const uint32_t t_node = __reduce_max_sync(FULL, lower ? key : 0u);
+                if (t_node > t) t = t_node;
+                const uint32_t t_bound = __reduce_max_sync(FULL, usable && key > t ? (s_bound < key ? s_bound : key) : 0u);
+                if (t_bound > t) t = t_bound;
+                unsigned acc = __ballot_sync(FULL, usable && key > t);
+                n_acc = __popc(acc);
+                int my_order = 0;                            // position among the taken ones (the step log wants it)
+                if (n_acc > room || A.step_log) {
+                    for (unsigned m = acc; m; m &= m - 1) my_order += int(sh.sel[__ffs(m) - 1] > mine);
+                    if (n_acc > room) { acc = __ballot_sync(FULL, ((acc >> lane) & 1u) && my_order < room); n_acc = room; }
                 }
                 if (n_acc > 0) {
                     if ((acc >> lane) & 1u) {
@@ -1033,7 +1079,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     u64 nk = 0ull; float nw = 0.0f;
                     if (ptr < v.cls_end[t]) { nk = A.keys[ptr]; nw = A.sorted_w[ptr]; }
                     Committed cm;
-                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, false, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, false, lane, cm);
+                    ok = commit_warp<false, false>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
                     if (ok) {
                         int ng_, nc_; float gg, gc;
                         gains_from_column(sp, w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
@@ -1058,7 +1104,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
                     const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
                     Committed cm;
-                    ok = commit_warp(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, true, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, false, lane, cm);
+                    ok = commit_warp<true, false>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, lane, cm);
                     bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                     if (ok) {
                         int ng_, nc_; float gg, gc;
