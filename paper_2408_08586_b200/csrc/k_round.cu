@@ -235,6 +235,7 @@ struct Shared {
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
     int scan_cnt[RW];
+    int ff_pos[RUBICK_MAX_G_LEVELS];   // Phase A: no node below this index has g_levels[i] free GPUs
     unsigned long long sel[32];   // batch selection: one ordering word per lane
 };
 
@@ -253,6 +254,26 @@ __device__ int first_fit_warp(const Views &v, int g, int c, int lane)
         if (b) return __shfl_sync(0xffffffffu, base + 4 * lane + first, __ffs(b) - 1);
     }
     return -1;
+}
+
+// The same while free GPUs only shrink (Phase A): ff_pos[gi] is a node index below which no node has g free
+// GPUs any more, so the search starts there, 32 nodes at a time, and moves the mark up to the first node that
+// still has them.
+__device__ int first_fit_from_mark(const Views &v, Shared &sh, int gi, int g, int c, int lane)
+{
+    const int need = (g << 16) | c;          // a word fits when it is at least `need` and its core field at least c
+    int first_g = -1, found = -1;
+    for (int pos = sh.ff_pos[gi]; pos < v.N && found < 0; pos += 32) {
+        const int n = pos + lane;
+        const int w = n < v.N_pad ? v.gc[n] : 0;
+        const unsigned bg = __ballot_sync(0xffffffffu, w >= (g << 16));
+        const unsigned bf = __ballot_sync(0xffffffffu, w >= need && fc_of(w) >= c);
+        if (first_g < 0 && bg) first_g = pos + __ffs(bg) - 1;
+        if (bf) found = pos + __ffs(bf) - 1;
+    }
+    __syncwarp();
+    if (lane == 0) sh.ff_pos[gi] = first_g >= 0 ? first_g : v.N;
+    return found;
 }
 
 // warp-cooperative: maxc[] for every level in one sweep over the node words (lane 0 stores).  Levels ascend, so
@@ -320,7 +341,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     if (g2 <= sp.Gn) {
         if (alloc) { const int w = v.gc[node]; stay = fg_of(w) >= g2 - g && fc_of(w) >= c2 - c; }
         if (stay) target = node;
-        else if (v.maxc[gi2] >= c2) target = first_fit_warp(v, g2, c2, lane);
+        else if (v.maxc[gi2] >= c2) target = rebuild ? first_fit_from_mark(v, sh, gi2, g2, c2, lane) : first_fit_warp(v, g2, c2, lane);
         if (target < 0) return false;
     } else {
         k2 = g2 >> sp.log2Gn;
@@ -581,6 +602,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     for (int i = tid; i < v.N_pad / 32; i += RT) tb_s[i] = 0u;
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
     if (tid < 32) sh.dirty[tid] = 1;
+    if (tid < RUBICK_MAX_G_LEVELS) sh.ff_pos[tid] = 0;
     for (int i = tid; i < 2 * A.n_tenants; i += RT) rem_q[i] = A.quota[i];
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
@@ -651,15 +673,17 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // ---- Phase A: guaranteed minima in job order (warp 0) ------------------------------------------
     if (warp == 0) {
         const int ng = sh.n_guar;
+        // lanes fetch 32 list entries at once; they are used one after another.  The records of the next 32 and
+        // the list entries of the 32 after them are requested before this batch is worked on.
+        int jl = lane < ng ? A.glist[lane] : -1;
+        int jl_next = 32 + lane < ng ? A.glist[32 + lane] : -1;
+        int4 a0 = make_int4(-1, 0, 0, -1), a1 = make_int4(-1, 0, 0, 0);
+        if (jl >= 0) { a0 = reinterpret_cast<const int4 *>(A.pa + jl)[0]; a1 = reinterpret_cast<const int4 *>(A.pa + jl)[1]; }
         for (int base = 0; base < ng; base += 32) {
-            // lanes fetch 32 list entries at once; they are used one after another
             const int idx = base + lane;
-            int jl = -1; int4 a0 = make_int4(-1, 0, 0, -1), a1 = make_int4(-1, 0, 0, 0);
-            if (idx < ng) {
-                jl = A.glist[idx];
-                a0 = reinterpret_cast<const int4 *>(A.pa + jl)[0];
-                a1 = reinterpret_cast<const int4 *>(A.pa + jl)[1];
-            }
+            int4 n0 = make_int4(-1, 0, 0, -1), n1 = make_int4(-1, 0, 0, 0);
+            if (jl_next >= 0) { n0 = reinterpret_cast<const int4 *>(A.pa + jl_next)[0]; n1 = reinterpret_cast<const int4 *>(A.pa + jl_next)[1]; }
+            const int jl_after = base + 64 + lane < ng ? A.glist[base + 64 + lane] : -1;
             // Free resources only shrink during this phase, so a job that cannot be placed now never can:
             // every lane tests its own job against the present tables and only the others take a turn.
             bool may = false;
@@ -699,6 +723,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     __syncwarp();
                 }
             }
+            jl = jl_next; a0 = n0; a1 = n1; jl_next = jl_after;
         }
     }
     __syncthreads();
