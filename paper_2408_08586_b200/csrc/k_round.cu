@@ -49,6 +49,7 @@ constexpr int RW = RT / 32;
 constexpr int SORT_T = 1024;            // threads of the sort kernel
 constexpr size_t SMEM_LIMIT = 200 * 1024;
 constexpr int SORT_SMEM_KEYS = 16384;
+constexpr int RUN_U = 4;                // a run of failing class heads settles up to 32 * RUN_U entries a turn
 
 typedef unsigned long long u64;
 
@@ -861,29 +862,44 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const unsigned fb = __ballot_sync(FULL, lane < sp.nM && v.ml[lane < sp.nM ? lane : 0] <= avail * k2);
                     const int mi = fb ? 31 - __clz(fb) : -1;
                     const int ptr = v.cls_ptr[t], end = v.cls_end[t];
-                    const int idx = ptr + lane;
-                    const u64 k = idx < end ? A.keys[idx] : 0ull;
-                    const bool in_run = k != 0ull && (0x80000000u | key_gain_bits(k)) > B;
-                    const int j = key_job(k);
-                    bool succ = false;
-                    if (in_run && mi >= 0) {
-                        const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                        float val; int plan, f; bool okg;
-                        if (cand.plan >= 0 && cand.f >= 0 && cand.f <= mi) { val = cand.val; plan = cand.plan; f = cand.f; okg = cand.ok != 0; }
-                        else {
-                            const size_t o = curve_idx(sp, j, gi2, ci2, mi);
-                            val = __ldg(A.cv + o); plan = __ldg(A.cp + o); okg = __ldg(A.cg + o) == g2;
-                            f = -1;
-                            if (plan >= 0 && plan < sp.P) f = __ffs(__ldg(A.feas + size_t(j) * sp.P + plan)) - 1;
-                        }
-                        succ = plan >= 0 && plan < sp.P && val > 0.0f && okg && f >= 0 && f <= mi;
+                    // RUN_U x 32 entries a turn: every lane looks at RUN_U of them, all loads of a kind in one wave
+                    u64 k[RUN_U]; bool in_run[RUN_U], succ[RUN_U]; HotCurve cand[RUN_U];
+#pragma unroll
+                    for (int u = 0; u < RUN_U; ++u) {
+                        const int idx = ptr + 32 * u + lane;
+                        k[u] = idx < end ? A.keys[idx] : 0ull;
                     }
-                    // leading entries that are in the run and fail
-                    const unsigned stop = __ballot_sync(FULL, !in_run || succ);
-                    int n_fail = stop ? __ffs(stop) - 1 : 32;
+#pragma unroll
+                    for (int u = 0; u < RUN_U; ++u) {
+                        in_run[u] = k[u] != 0ull && (0x80000000u | key_gain_bits(k[u])) > B;
+                        succ[u] = false;
+                        if (in_run[u] && mi >= 0) cand[u] = load_hc(A.hc + hc_idx(sp, key_job(k[u]), gi2, ci2));
+                    }
+                    int n_fail = 0; bool open_ = true;         // leading entries that are in the run and fail
+#pragma unroll
+                    for (int u = 0; u < RUN_U; ++u) {
+                        if (in_run[u] && mi >= 0) {
+                            const int j = key_job(k[u]);
+                            float val; int plan, f; bool okg;
+                            if (cand[u].plan >= 0 && cand[u].f >= 0 && cand[u].f <= mi) { val = cand[u].val; plan = cand[u].plan; f = cand[u].f; okg = cand[u].ok != 0; }
+                            else {
+                                const size_t o = curve_idx(sp, j, gi2, ci2, mi);
+                                val = __ldg(A.cv + o); plan = __ldg(A.cp + o); okg = __ldg(A.cg + o) == g2;
+                                f = -1;
+                                if (plan >= 0 && plan < sp.P) f = __ffs(__ldg(A.feas + size_t(j) * sp.P + plan)) - 1;
+                            }
+                            succ[u] = plan >= 0 && plan < sp.P && val > 0.0f && okg && f >= 0 && f <= mi;
+                        }
+                        const unsigned stop = __ballot_sync(FULL, !in_run[u] || succ[u]);
+                        if (open_) { n_fail += stop ? __ffs(stop) - 1 : 32; open_ = stop == 0u; }
+                    }
                     if (n_fail > room) n_fail = room;
                     if (n_fail > 0) {
-                        if (lane < n_fail && A.step_log) A.step_log[steps0 + lane] = (j << 2) | 0;
+                        if (A.step_log) {
+#pragma unroll
+                            for (int u = 0; u < RUN_U; ++u)
+                                if (32 * u + lane < n_fail) A.step_log[steps0 + 32 * u + lane] = (key_job(k[u]) << 2) | 0;
+                        }
                         if (lane == 0) {
                             const int np = ptr + n_fail;
                             u64 nk = 0ull; float nw = 0.0f;
