@@ -532,12 +532,52 @@ __device__ SlotC make_slotc(const Space &sp, const int32_t *gl, const int32_t *c
     return s;
 }
 
+// What a job wants next once it holds (gi, ci) with the curve's value there: its weighted gains, the GPU level
+// the GPU gain refers to and what both candidates need in order to be placeable.  None of it depends on the
+// cluster, so it is worked out for every (job, gi, ci) before the round and an increment that is committed in a
+// batch reads one 32-byte record instead of a column of the curve.
+struct __align__(16) Trans { float gain_g, gain_c; int32_t next_g, next_c; SlotC need; };
+static_assert(sizeof(Trans) == 32, "two 16-byte loads");
+
+__global__ void round_trans_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
+                                   const HotCurve *__restrict__ hc, Trans *__restrict__ tr)
+{
+    const size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t per_job = size_t(sp.nG) * sp.nC;
+    if (i >= size_t(J) * per_job) return;
+    const int j = int(i / per_job);
+    const int gi = int((i - size_t(j) * per_job) / sp.nC), ci = int(i - size_t(j) * per_job - size_t(gi) * sp.nC);
+    Trans t; t.gain_g = 0.0f; t.gain_c = 0.0f; t.next_g = -1; t.next_c = -1;
+    const float val = hc[i].val;
+    if (val > 0.0f) {
+        const float w = jobs[j].w, vcur = __fmul_rn(w, val);
+        for (int g2 = gi + 1; g2 < sp.nG; ++g2) {
+            const float x = hc[hc_idx(sp, j, g2, ci)].val;
+            if (x > val) {
+                t.next_g = g2;
+                t.gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, x), vcur), float(sp.g_levels[g2] - sp.g_levels[gi]));
+                break;
+            }
+        }
+        if (ci + 1 < sp.nC) {
+            const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(w, hc[i + 1].val), vcur), float(sp.c_levels[ci + 1] - sp.c_levels[ci]));
+            if (gn > 0.0f) { t.next_c = ci + 1; t.gain_c = gn; }
+        }
+    }
+    t.need = make_slotc(sp, sp.g_levels, sp.c_levels, gi, ci, t.next_g, t.next_c);
+    int4 lo, hi;
+    lo.x = __float_as_int(t.gain_g); lo.y = __float_as_int(t.gain_c); lo.z = t.next_g; lo.w = t.next_c;
+    hi = *reinterpret_cast<const int4 *>(&t.need);
+    reinterpret_cast<int4 *>(tr + i)[0] = lo;
+    reinterpret_cast<int4 *>(tr + i)[1] = hi;
+}
+
 struct RoundArgs {
     const rubick_job *jobs; int J;
     const float *cv; const int32_t *cp; const int32_t *cg; const uint32_t *feas;
     int N, max_steps;
     rubick_assignment *out; rubick_node *node_out; int32_t *step_log;
-    const HotCurve *hc; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
+    const HotCurve *hc; const Trans *tr; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
     int32_t *glist;
     SlotA *sa_g; SlotB *sb_g; SlotC *sc_g; int32_t *sj_g; int slots_in_smem; int slot_cap;
     const int32_t *quota; int n_tenants;      // per tenant: GPUs, cores (n_tenants = 0: no quotas)
@@ -962,10 +1002,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         // everything the commit and the new gains can need, in one wave of loads
                         const SlotB b = v.sb[s];
                         const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                        float col[8];
-#pragma unroll
-                        for (int u = 0; u < 8; ++u) col[u] = gi2 + 1 + u < sp.nG ? A.hc[hc_idx(sp, j, gi2 + 1 + u, ci2)].val : 0.0f;
-                        const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
+                        const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[0];
+                        const int4 t_hi = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[1];
                         const int64_t m_cur = v.ml[b.f_level];
                         const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
                         // levels ascend: the highest level that fits is below 0 / at least cand.f exactly when
@@ -981,24 +1019,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             s_ok = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
                         }
                         if (elig && s_ok) {
-                            // new gains: first GPU level above gi2 whose curve value exceeds the new value
-                            const float val = cand.val, vcur = __fmul_rn(b.w, val);
-                            int ng_ = -1, nc_ = -1; float gg = 0.0f, gc = 0.0f;
-#pragma unroll
-                            for (int u = 7; u >= 0; --u) if (gi2 + 1 + u < sp.nG && col[u] > val) { ng_ = gi2 + 1 + u; gg = col[u]; }
-                            for (int lvl = gi2 + 9; lvl < sp.nG && ng_ < 0; ++lvl) {
-                                const float x = A.hc[hc_idx(sp, j, lvl, ci2)].val;
-                                if (x > val) { ng_ = lvl; gg = x; }
-                            }
-                            if (ng_ >= 0) gg = __fdiv_rn(__fsub_rn(__fmul_rn(b.w, gg), vcur), float(v.gl[ng_] - g2));
-                            if (ci2 + 1 < sp.nC) {
-                                const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(b.w, vc), vcur), float(v.clv[ci2 + 1] - c2));
-                                if (gn > 0.0f) { nc_ = ci2 + 1; gc = gn; }
-                            }
-                            na.gain_g = fz_g ? 0.0f : gg; na.gain_c = fz_c ? 0.0f : gc;
-                            na.packed = pack(gi2, ci2, ng_, fz_g, fz_c); na.node = a.node;
-                            nb.val = val; nb.plan = cand.plan; nb.f_level = cand.f; nb.w = b.w;
-                            nq = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
+                            // the new gains and placement needs are those of the record of (gi2, ci2): the value
+                            // committed is the curve's
+                            na.gain_g = fz_g ? 0.0f : __int_as_float(t_lo.x); na.gain_c = fz_c ? 0.0f : __int_as_float(t_lo.y);
+                            na.packed = pack(gi2, ci2, t_lo.z, fz_g, fz_c); na.node = a.node;
+                            nb.val = cand.val; nb.plan = cand.plan; nb.f_level = cand.f; nb.w = b.w;
+                            nq = *reinterpret_cast<const SlotC *>(&t_hi);
                             if (multi) {
                                 // per-node shares of cores and memory on each of the k nodes (they hold no free GPU,
                                 // so maxc[] cannot change)
@@ -1195,7 +1221,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
 // ---- host side ------------------------------------------------------------------------------------------
 struct Layout {
     int n_pad, slot_cap, slots_in_smem;
-    size_t smem, off_hc, off_keys, off_w, off_pa, off_glist, off_sa, off_sb, off_sc, off_sj, total;
+    size_t smem, off_hc, off_tr, off_keys, off_w, off_pa, off_glist, off_sa, off_sb, off_sc, off_sj, total;
 };
 
 static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -1225,6 +1251,7 @@ static Layout make_layout(const Space &sp, int J, int N)
     const size_t gs = L.slots_in_smem ? 0 : size_t(L.slot_cap);
     size_t o = 0;
     L.off_hc = o; o = align256(o + size_t(J) * sp.nG * sp.nC * sizeof(HotCurve));
+    L.off_tr = o; o = align256(o + size_t(J) * sp.nG * sp.nC * sizeof(Trans));
     L.off_keys = o; o = align256(o + size_t(n) * 8);
     L.off_w = o; o = align256(o + size_t(n) * 4);
     L.off_pa = o; o = align256(o + size_t(J) * sizeof(PhaseA));
@@ -1273,6 +1300,8 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
 
     const size_t n_hc = size_t(J) * sp.nG * sp.nC;
     round_prepare_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_cv, d_cp, d_cg, d_feas, J, hc);
+    Trans *tr = reinterpret_cast<Trans *>(base + L.off_tr);
+    round_trans_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_jobs, J, hc, tr);
     round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa);
     const int sort_smem = L.n_pad <= SORT_SMEM_KEYS;
     cudaError_t e;
@@ -1285,7 +1314,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     RoundArgs A;
     A.jobs = d_jobs; A.J = J; A.cv = d_cv; A.cp = d_cp; A.cg = d_cg; A.feas = d_feas; A.N = N; A.max_steps = max_steps;
     A.out = d_out; A.node_out = d_node_out; A.step_log = d_step_log;
-    A.hc = hc; A.keys = keys; A.sorted_w = sw; A.n_pad = L.n_pad; A.pa = pa;
+    A.hc = hc; A.tr = tr; A.keys = keys; A.sorted_w = sw; A.n_pad = L.n_pad; A.pa = pa;
     A.glist = reinterpret_cast<int32_t *>(base + L.off_glist);
     A.sa_g = reinterpret_cast<SlotA *>(base + L.off_sa); A.sb_g = reinterpret_cast<SlotB *>(base + L.off_sb);
     A.sc_g = reinterpret_cast<SlotC *>(base + L.off_sc); A.sj_g = reinterpret_cast<int32_t *>(base + L.off_sj);
