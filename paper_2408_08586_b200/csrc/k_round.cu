@@ -177,13 +177,12 @@ round_sort_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ 
     }
     for (int k = 2; k <= n; k <<= 1)
         for (int s = k >> 1; s > 0; s >>= 1) {
-            for (int i = threadIdx.x; i < n; i += SORT_T) {
-                const int p = i ^ s;
-                if (p > i) {
-                    const u64 x = a[i], y = a[p];
-                    const bool desc = (i & k) == 0;
-                    if (desc ? (x < y) : (x > y)) { a[i] = y; a[p] = x; }
-                }
+            // one thread per pair (i, i + s): i has bit s clear
+            for (int t = threadIdx.x; t < (n >> 1); t += SORT_T) {
+                const int i = ((t & ~(s - 1)) << 1) | (t & (s - 1)), p = i | s;
+                const u64 x = a[i], y = a[p];
+                const bool desc = (i & k) == 0;
+                if (desc ? (x < y) : (x > y)) { a[i] = y; a[p] = x; }
             }
             __syncthreads();
         }
