@@ -419,7 +419,7 @@ def main():
                    "step": "eval_candidates + best_plan + marginal_gain + greedy_round"},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 8 * args.steps,   # eval, best_plan + its general-mask kernel, gain, prepare, keys, sort, round
+        "gpu_launches": 9 * args.steps,   # eval, best_plan + its general-mask kernel, gain, prepare, trans, keys, sort, round
         "roofline": {"kernel": "eval_candidates_kernel", "bound": "hbm", "achieved": eval_gbs, "peak": peak, "unit": "GB/s",
                      "frac": eval_gbs / peak, "traffic": traffic, "peak_source": peak_src,
                      "bytes_per_candidate": algorithmic_bytes_eval(J, P, C) / (float(J) * P * C),

@@ -8,6 +8,10 @@
 //                     together with the first feasible memory level of its plan, 16 bytes.  A commit
 //                     whose node offers at least that level needs no further table look-up, because
 //                     the curve at any level >= the plan's first level equals the curve at the top.
+//   trans    (grid)   per (job, GPU level, CPU level): the gains a job has once it holds that allocation with
+//                     the curve's value, the level its GPU gain refers to and what its two candidates need in
+//                     order to be placeable, 32 bytes.  A batched increment reads one record instead of a
+//                     column of the curve.
 //   keys     (grid)   every best-effort job starts unallocated, and its first increment (smallest
 //                     GPU level with a non-zero curve at its starting CPU level) and gain are fixed
 //                     until it is allocated: one 64-bit key (class = target levels | gain | ~job).
@@ -26,11 +30,12 @@
 //                     commits, in the exact order of the one-step-at-a-time rule, as many steps as it can
 //                     prove independent of each other:
 //                       - a run of class heads that are rejected (a rejection changes nothing but the head
-//                         of its class; lane i settles the i-th entry of the class's sorted list);
+//                         of its class; every lane settles four entries of the class's sorted list);
 //                       - a batch of increments that stay on their own nodes (lane w works out the commit
-//                         of warp w's candidate; candidates are taken in descending order while each is
-//                         larger than every runner-up, every best not yet taken and every new candidate of
-//                         the jobs taken before it, and sits on another node);
+//                         of group w's candidate; the candidates above one threshold - every runner-up,
+//                         every candidate that could not be worked out or shares a node with a better one,
+//                         every new candidate of the jobs taken - are a prefix of the sequential order
+//                         and are committed together);
 //                       - otherwise one general commit (migration, growth onto whole nodes, a class head
 //                         that succeeds): placement, memory level by ballot, node bookkeeping, new gains
 //                         from one warp-wide load of the job's curve column.
@@ -235,6 +240,7 @@ struct Shared {
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
     int scan_cnt[RW];
+    int empty_lo;                 // no node below this index is empty (whole multiples of 32 after a search)
     int ff_pos[RUBICK_MAX_G_LEVELS];   // Phase A: no node below this index has g_levels[i] free GPUs
     unsigned long long sel[32];   // batch selection: one ordering word per lane
 };
@@ -345,7 +351,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         if (target < 0) return false;
     } else {
         k2 = g2 >> sp.log2Gn;
-        if ((c2 + k2 - 1) / k2 > sp.Cn) return false;
+        if (cdiv_k(c2, k2) > sp.Cn) return false;
         if (alloc && g >= sp.Gn) { stay = true; need_new = k2 - k; if (n_empty < need_new) return false; }
         else {
             need_new = k2;
@@ -390,7 +396,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
             v.gc[target] = w_new_t;
             v.free_m[target] -= stay ? m2 - m_cur : m2;
         }
-        if (moved && fg_of(w_new_n) == sp.Gn) d_empty += 1;
+        if (moved && fg_of(w_new_n) == sp.Gn) { d_empty += 1; if (lane == 0 && node < sh.empty_lo) sh.empty_lo = node; }
         if (!stay && fg_of(w_old_t) == sp.Gn) d_empty -= 1;
         first = target; t1 = target; t0 = moved ? node : -1;
         // can maxc[] have changed?  lane i answers for GPU level i
@@ -408,12 +414,12 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         if (n_empty + d_empty > 0) ch = lane < sp.n_small && v.maxc[lane] != sp.Cn;
         maxc_dirty = __any_sync(0xffffffffu, ch);
     } else {
-        const int cs2 = (c2 + k2 - 1) / k2;
-        const int64_t ms2 = cdiv64(m2, k2);
+        const int cs2 = cdiv_k(c2, k2);
+        const int64_t ms2 = cdiv64_k(m2, k2);
         if (stay) {
             // whole nodes already held keep their GPUs; only the core / memory shares change
-            const int cs1 = (c + k - 1) / k;
-            const int64_t ms1 = cdiv64(m_cur, k);
+            const int cs1 = cdiv_k(c, alloc ? k : 1);
+            const int64_t ms1 = cdiv64_k(m_cur, alloc ? k : 1);
             if (k == 1) {
                 if (lane == 0) { v.gc[node] += c - cs2; v.free_m[node] += m_cur - ms2; v.owner[node] = j; }
             } else {
@@ -431,11 +437,11 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         } else if (alloc) {
             if (lane == 0) { v.gc[node] += (g << 16) + c; v.free_m[node] += m_cur; }
             __syncwarp();
-            if (fg_of(v.gc[node]) == sp.Gn) d_empty += 1;
+            if (fg_of(v.gc[node]) == sp.Gn) { d_empty += 1; if (lane == 0 && node < sh.empty_lo) sh.empty_lo = node; }
         }
         __syncwarp();
-        int taken = 0;
-        for (int base = 0; base < v.N && taken < need_new; base += 32) {
+        int taken = 0, base = sh.empty_lo & ~31;          // every empty node below the search's last look is taken
+        for (; base < v.N && taken < need_new; base += 32) {
             const int n = base + lane;
             const bool empty = n < v.N && fg_of(v.gc[n]) == sp.Gn;
             const unsigned b = __ballot_sync(0xffffffffu, empty);
@@ -444,6 +450,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
             if (b) { const int lowest = base + __ffs(b) - 1; if (first < 0 || lowest < first) first = lowest; }
             taken += __popc(b);
         }
+        if (lane == 0 && need_new > 0) sh.empty_lo = base - 32;
         d_empty -= need_new;
     }
     __syncwarp();
@@ -646,7 +653,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     for (int i = tid; i < 2 * A.n_tenants; i += RT) rem_q[i] = A.quota[i];
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
-        sh.ver = 0; sh.maxc_dirty = 1;
+        sh.ver = 0; sh.maxc_dirty = 1; sh.empty_lo = 0;
     }
     __syncthreads();
 
@@ -877,7 +884,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             // picks of the sequential rule can be committed together as long as each of them still is the
             // largest candidate: larger than every warp's runner-up (M), than the other warps' bests not yet
             // taken, and than the new candidates of the jobs taken before it.  Each lane works out its own
-            // commit first (two global round trips for all lanes together instead of one per step).
+            // commit first (one wave of global loads for all lanes together instead of several per step).
             int n_acc = 0;
             // ---- a run of class heads that cannot be committed --------------------------------------------
             // A rejected increment changes nothing but the head of its class, so as long as the heads of that
@@ -1141,19 +1148,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const int lvl = gi2 + 1 + lane;
                     const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
                     const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
+                    const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[0];
+                    const int4 t_hi = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[1];
                     const int ptr = v.cls_ptr[t] + 1;
                     u64 nk = 0ull; float nw = 0.0f;
                     if (ptr < v.cls_end[t]) { nk = A.keys[ptr]; nw = A.sorted_w[ptr]; }
                     Committed cm;
                     ok = commit_warp<false, false>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
                     if (ok) {
-                        int ng_, nc_; float gg, gc;
-                        gains_from_column(sp, w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
+                        // committed with the curve's own value (the usual case): the transition record has the rest
+                        const bool rec = cm.plan == cand.plan && cm.val == cand.val;
+                        int ng_ = t_lo.z, nc_ = t_lo.w; float gg = __int_as_float(t_lo.x), gc = __int_as_float(t_lo.y);
+                        if (!rec) gains_from_column(sp, w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
                         if (lane == 0) {
                             const int s = sh.n_slots;
                             SlotA sa; sa.gain_g = gg; sa.gain_c = gc; sa.packed = pack(gi2, ci2, ng_, false, false); sa.node = cm.first;
                             SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
-                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j; v.sc[s] = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
+                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
+                            v.sc[s] = rec ? *reinterpret_cast<const SlotC *>(&t_hi) : make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                             sh.n_slots = s + 1;
                             sh.dirty[(s % SCAN_T) >> 4] = 1;
                         }
@@ -1169,16 +1181,19 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const int lvl = gi2 + 1 + lane;
                     const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
                     const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
+                    const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[0];
+                    const int4 t_hi = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[1];
                     Committed cm;
                     ok = commit_warp<true, false>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, lane, cm);
                     bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
                     if (ok) {
-                        int ng_, nc_; float gg, gc;
-                        gains_from_column(sp, b.w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
+                        const bool rec = cm.plan == cand.plan && cm.val == cand.val;
+                        int ng_ = t_lo.z, nc_ = t_lo.w; float gg = __int_as_float(t_lo.x), gc = __int_as_float(t_lo.y);
+                        if (!rec) gains_from_column(sp, b.w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
                         a.gain_g = fz_g ? 0.0f : gg; a.gain_c = fz_c ? 0.0f : gc;
                         a.packed = pack(gi2, ci2, ng_, fz_g, fz_c); a.node = cm.first;
                         b.val = cm.val; b.plan = cm.plan; b.f_level = cm.f;
-                        if (lane == 0) v.sc[s] = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
+                        if (lane == 0) v.sc[s] = rec ? *reinterpret_cast<const SlotC *>(&t_hi) : make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                     } else {
                         if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
                         a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
