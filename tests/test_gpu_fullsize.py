@@ -108,6 +108,42 @@ def test_round_at_full_size_is_a_valid_packing_and_both_kernels_agree(full):
     assert np.all(r["thr"][run] <= cv[np.nonzero(run)[0], gi, ci, -1]) and np.all(r["thr"][run] > 0)
 
 
+@pytest.mark.parametrize("cap", [1, 31, 33, 127, 129, 700, 3001, 9000])
+def test_step_caps_inside_runs_and_batches_at_full_size(full, cap):
+    """The fast round commits several steps a turn (runs of failing class heads, batches of increments); a step
+    limit that falls inside one of them must stop it exactly where the one-step-at-a-time kernel stops."""
+    cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg = full
+    t = gpu.torch
+    N = cfg["n_nodes"]
+    res = []
+    for call in (gpu.ctx.greedy_round, gpu.ctx.greedy_round_noalloc):
+        d_out = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_node = t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        steps, capped = call(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, cap, d_out, d_node)
+        res.append(unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped, None))
+    assert res[0]["steps"] == cap and res[0]["capped"]
+    assert_rounds_equal(res[0], res[1])
+
+
+@pytest.mark.parametrize("n_jobs,n_nodes", [(1500, 512), (1500, 96), (600, 512)])
+def test_event_sized_rounds_agree_with_the_plain_kernel(n_jobs, n_nodes):
+    """The event-driven run's regime: a few hundred to 1,500 active jobs with large models (whole-node
+    jobs, migrations, growth onto empty nodes) on a cluster that is full, short of nodes, or half empty."""
+    cfg = workloads.make("events", J=n_jobs, n_nodes=n_nodes)
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    d_jobs, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    d_cv, d_cp, d_cg = gpu.best(d_thr, d_feas, n_jobs)
+    res = []
+    for call in (gpu.ctx.greedy_round, gpu.ctx.greedy_round_noalloc):
+        d_out = t.zeros(n_jobs * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_node = t.zeros(n_nodes * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        steps, capped = call(d_jobs, n_jobs, d_cv, d_cp, d_cg, d_feas, n_nodes, 1 << 30, d_out, d_node)
+        res.append(unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped, None))
+    assert_rounds_equal(res[0], res[1])
+    assert res[0]["steps"] > 300 and (n_nodes < 512 or (res[0]["n_nodes"] > 1).any())
+
+
 def test_event_driven_rounds_run_and_stay_consistent():
     from paper_2408_08586_b200 import events
     cfg = workloads.make("events", J=400, n_nodes=16)
