@@ -278,7 +278,9 @@ int rubick_min_resources(rubick_ctx *ctx, const float *d_thr, const uint32_t *d_
  * memory for the chosen node(s).  d_out: J assignments.  Optional (NULL to skip): d_node_out,
  * n_nodes entries; d_step_log, max_steps int32 entries (job << 2 | type << 1 | accepted);
  * h_steps, the number of increments tried.  Blocks until the round is done.
- * Returns ESTEPS if max_steps was reached first. */
+ * Returns ESTEPS if max_steps was reached first.  The context keeps the round's working tables in
+ * scratch of its own, grown on demand with cudaMalloc and kept for later rounds: about 48 bytes per
+ * (job, GPU level, core level) and 60 bytes per job. */
 int rubick_greedy_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
                         const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
                         const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,
