@@ -241,6 +241,7 @@ struct Shared {
     int maxc_dirty;               // the last commit may have changed maxc[]
     int scan_cnt[RW];
     int empty_lo;                 // no node below this index is empty (whole multiples of 32 after a search)
+    int4 pa_rec[32][2]; int pa_job[32];   // Phase A: the records of the 32 jobs being worked on
     int ff_pos[RUBICK_MAX_G_LEVELS];   // Phase A: no node below this index has g_levels[i] free GPUs
     unsigned long long sel[32];   // batch selection: one ordering word per lane
 };
@@ -336,9 +337,10 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
                             float val_cur, int f_cur, int gi2, int ci2, HotCurve cand, bool need_gain,
                             int lane, Committed &out)
 {
-    const int g = alloc ? sp.g_levels[gi] : 0, c = alloc ? sp.c_levels[ci] : 0;
-    const int64_t m_cur = alloc ? sp.m_levels[f_cur] : 0;
-    const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
+    // level values from their shared-memory copies (an indexed read of the constant bank takes longer)
+    const int g = alloc ? v.gl[gi] : 0, c = alloc ? v.clv[ci] : 0;
+    const int64_t m_cur = alloc ? v.ml[f_cur] : 0;
+    const int g2 = v.gl[gi2], c2 = v.clv[ci2];
     const int k = alloc ? max(g >> sp.log2Gn, 1) : 0;
     const int n_empty = sh.n_empty;
 
@@ -380,7 +382,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     if (plan < 0 || plan >= sp.P || !(val > 0.0f) || !okg) return false;
     if (need_gain && alloc && !(val > val_cur)) return false;
     if (f < 0 || f > mi) return false;
-    const int64_t m2 = sp.m_levels[f];
+    const int64_t m2 = v.ml[f];
 
     // ---- node bookkeeping ------------------------------------------------------------------------
     int first = -1, d_empty = 0;
@@ -740,18 +742,20 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 else { const int k2 = g2 >> sp.log2Gn; may = (c2 + k2 - 1) / k2 <= sp.Cn && sh.n_empty >= k2; }
             }
             unsigned todo = __ballot_sync(0xffffffffu, may);
+            // the records of the batch go through shared memory: one turn reads its job's with three loads
+            __syncwarp();
+            sh.pa_rec[lane][0] = a0; sh.pa_rec[lane][1] = a1; sh.pa_job[lane] = jl;
+            __syncwarp();
             while (todo) {
                 const int i = __ffs(todo) - 1;
                 todo &= todo - 1;
-                const int j = __shfl_sync(0xffffffffu, jl, i);
-                const int gi = __shfl_sync(0xffffffffu, a0.x, i), ci = __shfl_sync(0xffffffffu, a0.y, i);
+                const int4 r0 = sh.pa_rec[i][0], r1 = sh.pa_rec[i][1];
+                const int j = sh.pa_job[i];
+                const int gi = r0.x, ci = r0.y;
                 HotCurve cand;
-                cand.val = __int_as_float(__shfl_sync(0xffffffffu, a0.z, i));
-                cand.plan = __shfl_sync(0xffffffffu, a0.w, i);
-                cand.f = __shfl_sync(0xffffffffu, a1.x, i);
-                cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
-                const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
-                const int tn = __shfl_sync(0xffffffffu, a1.w, i);
+                cand.val = __int_as_float(r0.z); cand.plan = r0.w; cand.f = r1.x; cand.ok = r1.y;
+                const float w = __int_as_float(r1.z);
+                const int tn = r1.w;
                 if (gi < 0) continue;
                 if (A.n_tenants > 0) {     // privileged only while the minimum fits the tenant's remaining quota
                     if (tn < 0 || tn >= A.n_tenants) continue;
