@@ -74,6 +74,20 @@ def make_workload(name, rank=0, J=None, n_nodes=None):
         workloads.CONFIGS[name]["seed"] = base
 
 
+def sort_launches(J, tile=2048):
+    """Launches of the round's key sort: tiles of 2,048 keys are sorted in shared memory; every later stage of the
+    bitonic network takes one launch per stride of a tile or more and one for the strides inside the tiles."""
+    n = 2
+    while n < J:
+        n <<= 1
+    t = min(n, tile)
+    launches, k = 1, 2 * t
+    while k <= n:
+        launches += (k // 2).bit_length() - t.bit_length() + 1 + 1
+        k <<= 1
+    return launches
+
+
 def algorithmic_bytes_eval(J, P, C):
     """Bytes one eval_candidates launch must move: 4 per stored candidate (the table), 4 per
     (job, plan) (the mask word), 128 per job (its record)."""
@@ -419,7 +433,8 @@ def main():
                    "step": "eval_candidates + best_plan + marginal_gain + greedy_round"},
         "clocks": clocks,
         "e2e": e2e,
-        "gpu_launches": 9 * args.steps,   # eval, best_plan + its general-mask kernel, gain, prepare, trans, keys, sort, round
+        # eval, best_plan + its general-mask kernel, gain, prepare, trans, keys, the sort's launches, round
+        "gpu_launches": (8 + sort_launches(J)) * args.steps,
         "roofline": {"kernel": "eval_candidates_kernel", "bound": "hbm", "achieved": eval_gbs, "peak": peak, "unit": "GB/s",
                      "frac": eval_gbs / peak, "traffic": traffic, "peak_source": peak_src,
                      "bytes_per_candidate": algorithmic_bytes_eval(J, P, C) / (float(J) * P * C),

@@ -16,8 +16,9 @@
 //                     GPU level with a non-zero curve at its starting CPU level) and gain are fixed
 //                     until it is allocated: one 64-bit key (class = target levels | gain | ~job).
 //                     Guaranteed jobs get their Phase-A target resolved here too.
-//   sort     (1 CTA)  bitonic sort of the keys: inside a class (same target levels = same placement
-//                     test) only the first unconsumed job can ever be selected.
+//   sort     (grid)   bitonic sort of the keys, tiles in shared memory and wide strides in global memory: inside
+//                     a class (same target levels = same placement test) only the first unconsumed job can
+//                     ever be selected.
 //   round    (1 CTA)  persistent loop.  Shared memory holds one word per node (free GPUs << 16 | free
 //                     cores), free memory and whole-node owners, the table "most free cores among nodes
 //                     with >= g free GPUs" (a job of g GPUs and c cores fits some node exactly when that
@@ -51,9 +52,7 @@ namespace fastround {
 
 constexpr int RT = 512;                 // threads of the persistent round kernel
 constexpr int RW = RT / 32;
-constexpr int SORT_T = 1024;            // threads of the sort kernel
 constexpr size_t SMEM_LIMIT = 200 * 1024;
-constexpr int SORT_SMEM_KEYS = 16384;
 constexpr int RUN_U = 4;                // a run of failing class heads settles up to 32 * RUN_U entries a turn
 
 typedef unsigned long long u64;
@@ -170,32 +169,50 @@ __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick
 }
 
 // ---- sort: descending bitonic sort of n (power of two) keys, then the weights in sorted order -----
-__global__ void __launch_bounds__(SORT_T)
-round_sort_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ jobs, float *__restrict__ sorted_w,
-                  int in_smem)
+// Tiles of SORT_TILE keys live in shared memory, one CTA each: the stages up to the tile size run entirely there,
+// a later stage k does its passes with strides of a tile or more in global memory (one small launch each) and
+// the remaining ones in shared memory again.
+constexpr int SORT_TILE = 2048;
+constexpr int SORT_T = SORT_TILE / 2;   // one thread per compare-exchange pair of a tile
+
+__device__ __forceinline__ void sort_pair(u64 *a, int i, int p, bool desc)
 {
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    u64 *a = in_smem ? reinterpret_cast<u64 *>(smem_raw) : keys;
-    if (in_smem) {
-        for (int i = threadIdx.x; i < n; i += SORT_T) a[i] = keys[i];
-        __syncthreads();
-    }
-    for (int k = 2; k <= n; k <<= 1)
-        for (int s = k >> 1; s > 0; s >>= 1) {
-            // one thread per pair (i, i + s): i has bit s clear
-            for (int t = threadIdx.x; t < (n >> 1); t += SORT_T) {
-                const int i = ((t & ~(s - 1)) << 1) | (t & (s - 1)), p = i | s;
-                const u64 x = a[i], y = a[p];
-                const bool desc = (i & k) == 0;
-                if (desc ? (x < y) : (x > y)) { a[i] = y; a[p] = x; }
+    const u64 x = a[i], y = a[p];
+    if (desc ? (x < y) : (x > y)) { a[i] = y; a[p] = x; }
+}
+
+// stages k_from .. k_to of the tile starting at blockIdx.x * tile: for every stage the passes with stride
+// min(k / 2, tile / 2) down to 1.  last: also writes the weights in sorted order.
+__global__ void __launch_bounds__(SORT_T)
+round_sort_tile_kernel(u64 *__restrict__ keys, int n, int tile, int k_from, int k_to, int last,
+                       const rubick_job *__restrict__ jobs, float *__restrict__ sorted_w)
+{
+    __shared__ u64 a[SORT_TILE];
+    const int base = blockIdx.x * tile;
+    for (int i = threadIdx.x; i < tile; i += SORT_T) a[i] = keys[base + i];
+    __syncthreads();
+    for (int k = k_from; k <= k_to; k <<= 1)
+        for (int s = min(k >> 1, tile >> 1); s > 0; s >>= 1) {
+            for (int t = threadIdx.x; t < (tile >> 1); t += SORT_T) {
+                const int i = ((t & ~(s - 1)) << 1) | (t & (s - 1));
+                sort_pair(a, i, i | s, ((base + i) & k) == 0);
             }
             __syncthreads();
         }
-    for (int i = threadIdx.x; i < n; i += SORT_T) {
+    for (int i = threadIdx.x; i < tile; i += SORT_T) {
         const u64 k = a[i];
-        if (in_smem) keys[i] = k;
-        sorted_w[i] = k ? jobs[key_job(k)].w : 0.0f;
+        keys[base + i] = k;
+        if (last) sorted_w[base + i] = k ? jobs[key_job(k)].w : 0.0f;
     }
+}
+
+// one pass of stage k with stride s (a tile or more) in global memory; one thread per pair
+__global__ void round_sort_pass_kernel(u64 *__restrict__ keys, int n, int k, int s)
+{
+    const int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= (n >> 1)) return;
+    const int i = ((t & ~(s - 1)) << 1) | (t & (s - 1));
+    sort_pair(keys, i, i | s, (i & k) == 0);
 }
 
 // ---- the persistent round ---------------------------------------------------------------------------
@@ -1321,13 +1338,17 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     Trans *tr = reinterpret_cast<Trans *>(base + L.off_tr);
     round_trans_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_jobs, J, hc, tr);
     round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa);
-    const int sort_smem = L.n_pad <= SORT_SMEM_KEYS;
-    cudaError_t e;
-    if (sort_smem && size_t(L.n_pad) * 8 > 48 * 1024) {
-        e = cudaFuncSetAttribute(round_sort_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SORT_SMEM_KEYS * 8);
-        if (e != cudaSuccess) return e;
+    {
+        const int n = L.n_pad, tile = n < SORT_TILE ? n : SORT_TILE;
+        // every stage up to the tile size, tile by tile; then stage by stage: wide strides in global memory, the rest in tiles
+        round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, 2, tile, n == tile, d_jobs, sw);
+        for (int k = tile << 1; k <= n; k <<= 1) {
+            for (int s = k >> 1; s >= tile; s >>= 1)
+                round_sort_pass_kernel<<<((n >> 1) + 255) / 256, 256, 0, st>>>(keys, n, k, s);
+            round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, k, k, k == n, d_jobs, sw);
+        }
     }
-    round_sort_kernel<<<1, SORT_T, sort_smem ? size_t(L.n_pad) * 8 : 0, st>>>(keys, L.n_pad, d_jobs, sw, sort_smem);
+    cudaError_t e;
 
     RoundArgs A;
     A.jobs = d_jobs; A.J = J; A.cv = d_cv; A.cp = d_cp; A.cg = d_cg; A.feas = d_feas; A.N = N; A.max_steps = max_steps;
