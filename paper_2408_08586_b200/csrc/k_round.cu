@@ -123,7 +123,8 @@ __global__ void round_prepare_kernel(const __grid_constant__ Space sp, const flo
 __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
                                   const HotCurve *__restrict__ hc, const int32_t *__restrict__ cp,
                                   const int32_t *__restrict__ cg, u64 *__restrict__ keys, int n_pad,
-                                  PhaseA *__restrict__ pa)
+                                  PhaseA *__restrict__ pa, rubick_assignment *__restrict__ out,
+                                  int32_t *__restrict__ is_guar)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= n_pad) return;
@@ -164,6 +165,12 @@ __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick
         }
         reinterpret_cast<int4 *>(pa + j)[0] = make_int4(a.gi, a.ci, __float_as_int(a.val), a.plan);
         reinterpret_cast<int4 *>(pa + j)[1] = make_int4(a.f, a.ok, __float_as_int(a.w), a.pad);      // pad carries the tenant
+        // the result every job has until the round places it, and the mark the round builds its Phase-A list from
+        rubick_assignment r;
+        r.g = 0; r.c = 0; r.m_bytes = 0; r.plan = -1; r.first_node = -1; r.n_nodes = 0; r.thr = 0.0f;
+        r.status = a.gi != -2 ? RUBICK_PENDING : RUBICK_UNALLOCATED; r.m_level = -1;
+        out[j] = r;
+        is_guar[j] = a.gi != -2;
     }
     keys[j] = key;
 }
@@ -602,7 +609,7 @@ struct RoundArgs {
     const float *cv; const int32_t *cp; const int32_t *cg; const uint32_t *feas;
     int N, max_steps;
     rubick_assignment *out; rubick_node *node_out; int32_t *step_log;
-    const HotCurve *hc; const Trans *tr; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
+    const int32_t *is_guar; const HotCurve *hc; const Trans *tr; const u64 *keys; const float *sorted_w; int n_pad; const PhaseA *pa;
     int32_t *glist;
     SlotA *sa_g; SlotB *sb_g; SlotC *sc_g; int32_t *sj_g; int slots_in_smem; int slot_cap;
     const int32_t *quota; int n_tenants;      // per tenant: GPUs, cores (n_tenants = 0: no quotas)
@@ -694,23 +701,15 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             v.cls_end[(cls >> 6) * sp.nC + (cls & 63)] = A.n_pad;
         }
     }
-    // default results and the ordered list of guaranteed jobs
+    // the ordered list of guaranteed jobs: every warp owns a contiguous stretch of the job indices, counts its
+    // marks 32 at a time, and writes them behind those of the warps before it
     {
-        const int chunk = (J + RT - 1) / RT;
-        const int j0 = min(tid * chunk, J), j1 = min(j0 + chunk, J);
+        const int per_warp = (((J + RW - 1) / RW) + 31) & ~31;
+        const int w0 = min(warp * per_warp, J), w1 = min(w0 + per_warp, J);
         int cnt = 0;
-        for (int j = j0; j < j1; ++j) {
-            const int gi = A.pa[j].gi;
-            cnt += gi != -2;
-            rubick_assignment r;
-            r.g = 0; r.c = 0; r.m_bytes = 0; r.plan = -1; r.first_node = -1; r.n_nodes = 0; r.thr = 0.0f;
-            r.status = gi != -2 ? RUBICK_PENDING : RUBICK_UNALLOCATED; r.m_level = -1;
-            A.out[j] = r;
-        }
-        int incl = cnt;
-#pragma unroll
-        for (int s = 1; s < 32; s <<= 1) { const int o = __shfl_up_sync(0xffffffffu, incl, s); if (lane >= s) incl += o; }
-        if (lane == 31) sh.scan_cnt[warp] = incl;
+        for (int base = w0; base < w1; base += 32)
+            cnt += __popc(__ballot_sync(0xffffffffu, base + lane < w1 && A.is_guar[base + lane] != 0));
+        if (lane == 0) sh.scan_cnt[warp] = cnt;
         __syncthreads();
         if (warp == 0) {
             int wsum = lane < RW ? sh.scan_cnt[lane] : 0;
@@ -730,9 +729,13 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             if (lane == 0) sh.n_ccls = n_c;
         }
         __syncthreads();
-        int pos = incl - cnt + (warp ? sh.scan_cnt[warp - 1] : 0);
-        for (int j = j0; j < j1; ++j)
-            if (A.pa[j].gi != -2) A.glist[pos++] = j;
+        int pos = warp ? sh.scan_cnt[warp - 1] : 0;
+        for (int base = w0; base < w1; base += 32) {
+            const bool g = base + lane < w1 && A.is_guar[base + lane] != 0;
+            const unsigned b = __ballot_sync(0xffffffffu, g);
+            if (g) A.glist[pos + __popc(b & ((1u << lane) - 1u))] = base + lane;
+            pos += __popc(b);
+        }
     }
     __syncthreads();
 
@@ -1256,7 +1259,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
 // ---- host side ------------------------------------------------------------------------------------------
 struct Layout {
     int n_pad, slot_cap, slots_in_smem;
-    size_t smem, off_hc, off_tr, off_keys, off_w, off_pa, off_glist, off_sa, off_sb, off_sc, off_sj, total;
+    size_t smem, off_hc, off_tr, off_keys, off_w, off_pa, off_glist, off_isg, off_sa, off_sb, off_sc, off_sj, total;
 };
 
 static size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -1291,6 +1294,7 @@ static Layout make_layout(const Space &sp, int J, int N)
     L.off_w = o; o = align256(o + size_t(n) * 4);
     L.off_pa = o; o = align256(o + size_t(J) * sizeof(PhaseA));
     L.off_glist = o; o = align256(o + size_t(J) * 4);
+    L.off_isg = o; o = align256(o + size_t(J) * 4);
     L.off_sa = o; o = align256(o + gs * sizeof(SlotA));
     L.off_sb = o; o = align256(o + size_t(L.slot_cap) * sizeof(SlotB));
     L.off_sc = o; o = align256(o + gs * sizeof(SlotC));
@@ -1337,7 +1341,8 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     round_prepare_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_cv, d_cp, d_cg, d_feas, J, hc);
     Trans *tr = reinterpret_cast<Trans *>(base + L.off_tr);
     round_trans_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_jobs, J, hc, tr);
-    round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa);
+    round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa, d_out,
+                                                                reinterpret_cast<int32_t *>(base + L.off_isg));
     {
         const int n = L.n_pad, tile = n < SORT_TILE ? n : SORT_TILE;
         // every stage up to the tile size, tile by tile; then stage by stage: wide strides in global memory, the rest in tiles
@@ -1355,6 +1360,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     A.out = d_out; A.node_out = d_node_out; A.step_log = d_step_log;
     A.hc = hc; A.tr = tr; A.keys = keys; A.sorted_w = sw; A.n_pad = L.n_pad; A.pa = pa;
     A.glist = reinterpret_cast<int32_t *>(base + L.off_glist);
+    A.is_guar = reinterpret_cast<const int32_t *>(base + L.off_isg);
     A.sa_g = reinterpret_cast<SlotA *>(base + L.off_sa); A.sb_g = reinterpret_cast<SlotB *>(base + L.off_sb);
     A.sc_g = reinterpret_cast<SlotC *>(base + L.off_sc); A.sj_g = reinterpret_cast<int32_t *>(base + L.off_sj);
     A.slots_in_smem = L.slots_in_smem; A.slot_cap = L.slot_cap;
