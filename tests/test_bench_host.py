@@ -72,6 +72,29 @@ def test_algorithmic_byte_counts():
     assert bench.algorithmic_bytes_best(J, P, C, G, M) == 4.0 * J * P * C + 4.0 * J * P + 12.0 * J * G * C * M
 
 
+def test_sort_launch_count_follows_the_bitonic_network():
+    """Stages of a bitonic network over n keys with tiles of t keys: the stages up to t take one launch; stage k > t
+    takes log2(k / t) launches with strides of a tile or more and one for the strides inside the tiles."""
+    def brute(n, t=2048):
+        t = min(n, t)
+        launches, k = 1, 2
+        while k <= n:
+            if k > t:
+                s = k // 2
+                while s >= t:
+                    launches += 1
+                    s //= 2
+                launches += 1
+            k *= 2
+        return launches
+    for J in (1, 2, 64, 2048, 2049, 4096, 9000, 16384, 100000):
+        n = 2
+        while n < J:
+            n *= 2
+        assert bench.sort_launches(J) == brute(n)
+    assert bench.sort_launches(16384) == 10 and bench.sort_launches(1500) == 1
+
+
 def test_reference_arm_prints_one_json_line(capsys):
     import json
     import types
