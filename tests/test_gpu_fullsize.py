@@ -144,6 +144,22 @@ def test_event_sized_rounds_agree_with_the_plain_kernel(n_jobs, n_nodes):
     assert res[0]["steps"] > 300 and (n_nodes < 512 or (res[0]["n_nodes"] > 1).any())
 
 
+def test_round_repeats_bit_for_bit(full):
+    """The fast round uses shared-memory atomics (changed-node bitmap, version counter) and commits several steps a
+    turn; none of it may make the outcome depend on timing."""
+    cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg = full
+    t = gpu.torch
+    N = cfg["n_nodes"]
+    first = None
+    for _ in range(6):
+        d_out = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_node = t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        steps, capped = gpu.ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, 1 << 30, d_out, d_node)
+        cur = (steps, capped, d_out.cpu().numpy().tobytes(), d_node.cpu().numpy().tobytes())
+        first = first or cur
+        assert cur == first
+
+
 def test_event_driven_rounds_run_and_stay_consistent():
     from paper_2408_08586_b200 import events
     cfg = workloads.make("events", J=400, n_nodes=16)
