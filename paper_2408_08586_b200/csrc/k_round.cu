@@ -235,9 +235,11 @@ enum : uint8_t { K_SINGLE = 0, K_MULTI_WHOLE = 1, K_MULTI_PART = 2, K_NONE = 3 }
 
 constexpr int SCAN_WARPS = RW - 1;          // all warps but the last scan running jobs, the last one the class heads
 constexpr int SCAN_T = SCAN_WARPS * 32;
-constexpr int N_GROUPS = 2 * SCAN_WARPS + 1;   // candidates are cached per half warp (16 slots a pass) + one group for the class heads
+constexpr int N_GROUPS = 2 * SCAN_WARPS + 1;   // candidates seen by warp 0: the two best of every scanning warp + the best class head
 constexpr int CLS_G = N_GROUPS - 1;
-static_assert(N_GROUPS <= 32, "warp 0 holds one group per lane");
+static_assert(N_GROUPS <= 32, "warp 0 holds one candidate per lane");
+// the flag that makes the warp owning slot s look again (flags sit at the index of the warp's first candidate)
+__device__ __forceinline__ int dirty_of(int s) { return ((s % SCAN_T) >> 5) << 1; }
 
 // node n: gc[n] = free GPUs << 16 | free cores (padding entries are 0: they never fit anything)
 __device__ __forceinline__ int fg_of(int w) { return w >> 16; }
@@ -814,6 +816,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // looks again only when something it depends on changed: one of its slots, a node one of its slots
     // sits on, maxc[] or the number of empty nodes.
     uint32_t c_key = 0u, c_key2 = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
+    uint32_t c_keyB = 0u, c_payB = 0u; int c_jB = 0x7fffffff;          // scanning warps: their second candidate
     for (;;) {
         if (sh.maxc_dirty) {                                   // uniform: written before the last barrier
             if (warp < sp.n_small) {
@@ -823,8 +826,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             __syncthreads();
         }
         const int n_empty = sh.n_empty, n_slots = sh.n_slots, ver = sh.ver;
-        const unsigned hm = 0xffffu << (lane & 16);                   // my half of the warp
-        const int grp = warp < SCAN_WARPS ? 2 * warp + (lane >> 4) : CLS_G;
+        const unsigned hm = 0xffffffffu;
+        const int grp = warp < SCAN_WARPS ? 2 * warp : CLS_G;         // index of the warp's first candidate
         bool rescan = ver != my_ver || sh.dirty[grp] != 0;
         if (warp < SCAN_WARPS) {
             if (!rescan) {
@@ -833,7 +836,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 rescan = __any_sync(hm, hit);
             }
             if (rescan) {
-                uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
+                // the two best candidates of my slots in full, of everything else only the largest key
+                uint32_t k1 = 0u, k2 = 0u, rest = 0u, p1 = 0u, p2 = 0u; int j1 = 0x7fffffff, j2 = 0x7fffffff;
                 for (int s = tid; s < n_slots; s += SCAN_T) {
                     const SlotA a = v.sa[s];
                     const SlotC q = v.sc[s];
@@ -851,15 +855,23 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const uint32_t kg = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : 0u;
                     const uint32_t kc = ok_c ? __float_as_uint(a.gain_c) : 0u;
                     const uint32_t k32 = ok_g ? kg : kc;
-                    if (k32 > best || (k32 == best && k32 && j < best_j)) { second = best; best = k32; best_j = j; pay = uint32_t(s); }
-                    else if (k32 > second) second = k32;
-                    if (ok_g && kc > second) second = kc;
+                    if (k32 > k1 || (k32 == k1 && k32 && j < j1)) {
+                        rest = max(rest, k2); k2 = k1; j2 = j1; p2 = p1; k1 = k32; j1 = j; p1 = uint32_t(s);
+                    } else if (k32 > k2 || (k32 == k2 && k32 && j < j2)) {
+                        rest = max(rest, k2); k2 = k32; j2 = j; p2 = uint32_t(s);
+                    } else rest = max(rest, k32);
+                    if (ok_g) rest = max(rest, kc);
                 }
-                const uint32_t mine = best;
-                const int src = warp_select(best, best_j, pay, hm);
-                c_key2 = __reduce_max_sync(hm, lane == src ? second : mine);
-                c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
-                if ((lane & 15) == 0) sh.dirty[grp] = 0;
+                // the warp's best; then its second (the lane that gave the best offers its own second); then the
+                // largest key among what remains
+                uint32_t a_k = k1, a_p = p1; int a_j = j1;
+                const int src_a = warp_select(a_k, a_j, a_p, hm);
+                uint32_t b_k = lane == src_a ? k2 : k1, b_p = lane == src_a ? p2 : p1; int b_j = lane == src_a ? j2 : j1;
+                const int src_b = warp_select(b_k, b_j, b_p, hm);
+                const uint32_t left = lane == src_a ? (src_b == src_a ? 0u : k2) : (lane == src_b ? k2 : k1);
+                c_key2 = __reduce_max_sync(hm, max(rest, left));
+                c_key = a_k; c_j = a_j; c_pay = a_p; c_keyB = b_k; c_jB = b_j; c_payB = b_p; my_ver = ver;
+                if (lane == 0) sh.dirty[grp] = 0;
             }
         } else if (rescan) {
             uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
@@ -885,8 +897,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
             if (lane == 0) sh.dirty[CLS_G] = 0;
         }
-        if ((lane & 15) == 0 && (warp < SCAN_WARPS || lane == 0)) {
+        if (lane == 0) {
             sh.red_key[grp] = c_key; sh.red_j[grp] = c_j; sh.red_pay[grp] = c_pay; sh.red_key2[grp] = c_key2;
+            if (warp < SCAN_WARPS) { sh.red_key[grp + 1] = c_keyB; sh.red_j[grp + 1] = c_jB; sh.red_pay[grp + 1] = c_payB; sh.red_key2[grp + 1] = 0u; }
         }
         __syncthreads();
         if (warp == 0) {
@@ -1133,7 +1146,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if ((acc >> lane) & 1u) {
                         if (s_ok && !s_multi) { v.gc[s_node] -= s_dgc; v.free_m[s_node] -= s_dm; }
                         v.sa[s_slot] = na; v.sb[s_slot] = nb; v.sc[s_slot] = nq;
-                        sh.dirty[(s_slot % SCAN_T) >> 4] = 1;
+                        sh.dirty[dirty_of(s_slot)] = 1;
                         if (s_ok && !s_multi) atomicOr(&v.tb[s_node >> 5], 1u << (s_node & 31));
                         if (A.step_log) A.step_log[steps0 + my_order] = (my_j << 2) | ((s_type ? 0 : 1) << 1) | int(s_ok);
                     }
@@ -1191,7 +1204,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
                             v.sc[s] = rec ? *reinterpret_cast<const SlotC *>(&t_hi) : make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
                             sh.n_slots = s + 1;
-                            sh.dirty[(s % SCAN_T) >> 4] = 1;
+                            sh.dirty[dirty_of(s)] = 1;
                         }
                     }
                     if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[CLS_G] = 1; }
@@ -1222,7 +1235,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
                         a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
                     }
-                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; sh.dirty[(s % SCAN_T) >> 4] = 1; }
+                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; sh.dirty[dirty_of(s)] = 1; }
                 }
                 if (lane == 0) {
                     if (A.step_log) A.step_log[sh.steps] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
