@@ -24,10 +24,11 @@
 //                     with >= g free GPUs" (a job of g GPUs and c cores fits some node exactly when that
 //                     entry is >= c), the head of every class, one 36-byte slot per RUNNING job (scan state
 //                     + what its two candidates need to be placeable) and a bitmap of the nodes the last
-//                     iteration changed.  Every warp caches the best candidate and the runner-up key of
-//                     its slots (the last warp: of the class heads) and looks again only when one of its
-//                     slots, a node under them, that table or the number of empty nodes changed.  Warp 0
-//                     picks (type | gain, lowest job) across the warps with warp reduce instructions and
+//                     iteration changed.  Every warp caches the two best candidates of its slots and the
+//                     largest key among the rest (the last warp: the best class head and the runner-up key)
+//                     and looks again only when one of its slots, a node under them, that table or the
+//                     number of empty nodes changed.  Warp 0 holds one offered candidate per lane, picks
+//                     (type | gain, lowest job) across them with warp reduce instructions and
 //                     commits, in the exact order of the one-step-at-a-time rule, as many steps as it can
 //                     prove independent of each other:
 //                       - a run of class heads that are rejected (a rejection changes nothing but the head
@@ -812,7 +813,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     __syncthreads();
 
     // ---- Phase B ---------------------------------------------------------------------------------------
-    // Every warp remembers the best candidate among its own slots (warp 31: among the class heads) and
+    // Every warp remembers the two best candidates among its own slots (the last warp: the best class head) and
     // looks again only when something it depends on changed: one of its slots, a node one of its slots
     // sits on, maxc[] or the number of empty nodes.
     uint32_t c_key = 0u, c_key2 = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
@@ -916,10 +917,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             __syncwarp();
 
             // ---- a batch of independent increments ---------------------------------------------------------
-            // Lane w holds the best candidate of warp w.  Increments that stay on their node, on pairwise
+            // Every lane holds one candidate offered by the scanning warps.  Increments that stay on their node, on pairwise
             // different nodes, commute with everything except what happens on that node, so the next few
             // picks of the sequential rule can be committed together as long as each of them still is the
-            // largest candidate: larger than every warp's runner-up (M), than the other warps' bests not yet
+            // largest candidate: larger than every key that was not offered (M), than the offered ones not yet
             // taken, and than the new candidates of the jobs taken before it.  Each lane works out its own
             // commit first (one wave of global loads for all lanes together instead of several per step).
             int n_acc = 0;
