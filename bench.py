@@ -433,8 +433,8 @@ def main():
                    "step": "eval_candidates + best_plan + marginal_gain + greedy_round"},
         "clocks": clocks,
         "e2e": e2e,
-        # eval, best_plan + its general-mask kernel, gain, prepare, trans, keys, the sort's launches, round
-        "gpu_launches": (8 + sort_launches(J)) * args.steps,
+        # eval, best_plan + its general-mask kernel, gain, prepare, keys, the sort's launches, round
+        "gpu_launches": (7 + sort_launches(J)) * args.steps,
         "roofline": {"kernel": "eval_candidates_kernel", "bound": "hbm", "achieved": eval_gbs, "peak": peak, "unit": "GB/s",
                      "frac": eval_gbs / peak, "traffic": traffic, "peak_source": peak_src,
                      "bytes_per_candidate": algorithmic_bytes_eval(J, P, C) / (float(J) * P * C),

@@ -4,14 +4,14 @@
 // GPU gain first, CPU gain when no GPU increment is left, lowest job index on ties, commit with
 // the best plan and its host memory), organised so that one step costs about half a microsecond:
 //
-//   prepare  (grid)   per (job, GPU level, CPU level): the curve entry at the top host-memory level
-//                     together with the first feasible memory level of its plan, 16 bytes.  A commit
+//   prepare  (grid)   one CTA per job.  Per (job, GPU level, CPU level): the curve entry at the top host-memory
+//                     level together with the first feasible memory level of its plan, 16 bytes.  A commit
 //                     whose node offers at least that level needs no further table look-up, because
 //                     the curve at any level >= the plan's first level equals the curve at the top.
-//   trans    (grid)   per (job, GPU level, CPU level): the gains a job has once it holds that allocation with
-//                     the curve's value, the level its GPU gain refers to and what its two candidates need in
-//                     order to be placeable, 32 bytes.  A batched increment reads one record instead of a
-//                     column of the curve.
+//                     Then, from those values (kept in shared memory), a 32-byte transition record: the gains
+//                     a job has once it holds that allocation with the curve's value, the level its GPU gain
+//                     refers to and what its two candidates need in order to be placeable.  A batched
+//                     increment reads one record instead of a column of the curve.
 //   keys     (grid)   every best-effort job starts unallocated, and its first increment (smallest
 //                     GPU level with a non-zero curve at its starting CPU level) and gain are fixed
 //                     until it is allocated: one 64-bit key (class = target levels | gain | ~job).
@@ -98,26 +98,6 @@ __device__ __forceinline__ HotCurve load_hc(const HotCurve *p)
     const int4 v = *reinterpret_cast<const int4 *>(p);
     HotCurve h; h.val = __int_as_float(v.x); h.plan = v.y; h.f = v.z; h.ok = v.w;
     return h;
-}
-
-// ---- prepare: curve entries at the top memory level with the plan's first feasible level ---------
-__global__ void round_prepare_kernel(const __grid_constant__ Space sp, const float *__restrict__ cv,
-                                     const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
-                                     const uint32_t *__restrict__ feas, int J, HotCurve *__restrict__ hc)
-{
-    const size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    const size_t per_job = size_t(sp.nG) * sp.nC;
-    if (i >= size_t(J) * per_job) return;
-    const int j = int(i / per_job);
-    const int gi = int((i - size_t(j) * per_job) / sp.nC);
-    const size_t o = i * sp.nM + (sp.nM - 1);
-    HotCurve h;
-    h.val = __ldg(cv + o); h.plan = __ldg(cp + o);
-    h.ok = __ldg(cg + o) == sp.g_levels[gi];
-    h.f = -1;
-    if (h.plan >= 0 && h.plan < sp.P) h.f = __ffs(__ldg(feas + size_t(j) * sp.P + h.plan)) - 1;
-    int4 v; v.x = __float_as_int(h.val); v.y = h.plan; v.z = h.f; v.w = h.ok;
-    reinterpret_cast<int4 *>(hc)[i] = v;
 }
 
 // ---- keys: first increment of every best-effort job, Phase-A target of every guaranteed job -------
@@ -574,37 +554,57 @@ __device__ SlotC make_slotc(const Space &sp, const int32_t *gl, const int32_t *c
 struct __align__(16) Trans { float gain_g, gain_c; int32_t next_g, next_c; SlotC need; };
 static_assert(sizeof(Trans) == 32, "two 16-byte loads");
 
-__global__ void round_trans_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
-                                   const HotCurve *__restrict__ hc, Trans *__restrict__ tr)
+// ---- prepare: one CTA per job.  First the curve entries at the top memory level with the plan's first feasible
+// level (16 bytes each; their values also go to shared memory), then the transition records from those values.
+__global__ void __launch_bounds__(256)
+round_prepare_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, const float *__restrict__ cv,
+                     const int32_t *__restrict__ cp, const int32_t *__restrict__ cg, const uint32_t *__restrict__ feas,
+                     HotCurve *__restrict__ hc, Trans *__restrict__ tr)
 {
-    const size_t i = size_t(blockIdx.x) * blockDim.x + threadIdx.x;
-    const size_t per_job = size_t(sp.nG) * sp.nC;
-    if (i >= size_t(J) * per_job) return;
-    const int j = int(i / per_job);
-    const int gi = int((i - size_t(j) * per_job) / sp.nC), ci = int(i - size_t(j) * per_job - size_t(gi) * sp.nC);
-    Trans t; t.gain_g = 0.0f; t.gain_c = 0.0f; t.next_g = -1; t.next_c = -1;
-    const float val = hc[i].val;
-    if (val > 0.0f) {
-        const float w = jobs[j].w, vcur = __fmul_rn(w, val);
-        for (int g2 = gi + 1; g2 < sp.nG; ++g2) {
-            const float x = hc[hc_idx(sp, j, g2, ci)].val;
-            if (x > val) {
-                t.next_g = g2;
-                t.gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, x), vcur), float(sp.g_levels[g2] - sp.g_levels[gi]));
-                break;
+    __shared__ float sval[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS];
+    const int j = blockIdx.x;
+    const int per_job = sp.nG * sp.nC;
+    const size_t first = size_t(j) * per_job;
+    for (int e = threadIdx.x; e < per_job; e += blockDim.x) {
+        const int gi = e / sp.nC;
+        const size_t o = (first + e) * sp.nM + (sp.nM - 1);
+        HotCurve h;
+        h.val = __ldg(cv + o); h.plan = __ldg(cp + o);
+        h.ok = __ldg(cg + o) == sp.g_levels[gi];
+        h.f = -1;
+        if (h.plan >= 0 && h.plan < sp.P) h.f = __ffs(__ldg(feas + size_t(j) * sp.P + h.plan)) - 1;
+        int4 v; v.x = __float_as_int(h.val); v.y = h.plan; v.z = h.f; v.w = h.ok;
+        reinterpret_cast<int4 *>(hc)[first + e] = v;
+        sval[e] = h.val;
+    }
+    __syncthreads();
+    const float w = jobs[j].w;
+    for (int e = threadIdx.x; e < per_job; e += blockDim.x) {
+        const int gi = e / sp.nC, ci = e - gi * sp.nC;
+        Trans t; t.gain_g = 0.0f; t.gain_c = 0.0f; t.next_g = -1; t.next_c = -1;
+        const float val = sval[e];
+        if (val > 0.0f) {
+            const float vcur = __fmul_rn(w, val);
+            for (int g2 = gi + 1; g2 < sp.nG; ++g2) {
+                const float x = sval[g2 * sp.nC + ci];
+                if (x > val) {
+                    t.next_g = g2;
+                    t.gain_g = __fdiv_rn(__fsub_rn(__fmul_rn(w, x), vcur), float(sp.g_levels[g2] - sp.g_levels[gi]));
+                    break;
+                }
+            }
+            if (ci + 1 < sp.nC) {
+                const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(w, sval[e + 1]), vcur), float(sp.c_levels[ci + 1] - sp.c_levels[ci]));
+                if (gn > 0.0f) { t.next_c = ci + 1; t.gain_c = gn; }
             }
         }
-        if (ci + 1 < sp.nC) {
-            const float gn = __fdiv_rn(__fsub_rn(__fmul_rn(w, hc[i + 1].val), vcur), float(sp.c_levels[ci + 1] - sp.c_levels[ci]));
-            if (gn > 0.0f) { t.next_c = ci + 1; t.gain_c = gn; }
-        }
+        t.need = make_slotc(sp, sp.g_levels, sp.c_levels, gi, ci, t.next_g, t.next_c);
+        int4 lo, hi;
+        lo.x = __float_as_int(t.gain_g); lo.y = __float_as_int(t.gain_c); lo.z = t.next_g; lo.w = t.next_c;
+        hi = *reinterpret_cast<const int4 *>(&t.need);
+        reinterpret_cast<int4 *>(tr + first + e)[0] = lo;
+        reinterpret_cast<int4 *>(tr + first + e)[1] = hi;
     }
-    t.need = make_slotc(sp, sp.g_levels, sp.c_levels, gi, ci, t.next_g, t.next_c);
-    int4 lo, hi;
-    lo.x = __float_as_int(t.gain_g); lo.y = __float_as_int(t.gain_c); lo.z = t.next_g; lo.w = t.next_c;
-    hi = *reinterpret_cast<const int4 *>(&t.need);
-    reinterpret_cast<int4 *>(tr + i)[0] = lo;
-    reinterpret_cast<int4 *>(tr + i)[1] = hi;
 }
 
 struct RoundArgs {
@@ -1351,10 +1351,8 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     const long long natural = (long long)J * (sp.nG + sp.nC + 2) + 1;
     if ((long long)max_steps > natural) max_steps = int(natural < 0x7fffffffLL ? natural : 0x7fffffffLL);
 
-    const size_t n_hc = size_t(J) * sp.nG * sp.nC;
-    round_prepare_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_cv, d_cp, d_cg, d_feas, J, hc);
     Trans *tr = reinterpret_cast<Trans *>(base + L.off_tr);
-    round_trans_kernel<<<unsigned((n_hc + 255) / 256), 256, 0, st>>>(sp, d_jobs, J, hc, tr);
+    round_prepare_kernel<<<J, 256, 0, st>>>(sp, d_jobs, d_cv, d_cp, d_cg, d_feas, hc, tr);
     round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa, d_out,
                                                                 reinterpret_cast<int32_t *>(base + L.off_isg));
     {
