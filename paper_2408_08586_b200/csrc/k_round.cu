@@ -249,6 +249,7 @@ struct Shared {
     int scan_cnt[RW];
     int empty_lo;                 // no node below this index is empty (whole multiples of 32 after a search)
     int4 pa_rec[32][2]; int pa_job[32];   // Phase A: the records of the 32 jobs being worked on
+    int pa_commits;               // Phase A: jobs placed so far
     int ff_pos[RUBICK_MAX_G_LEVELS];   // Phase A: no node below this index has g_levels[i] free GPUs
     unsigned long long sel[32];   // batch selection: one ordering word per lane
 };
@@ -331,7 +332,7 @@ __device__ int max_cores_warp(const Views &v, int g, int lane)
     return __reduce_max_sync(0xffffffffu, m);
 }
 
-struct Committed { int first; float val; int plan; int f; };
+struct Committed { int first; float val; int plan; int f; };      // after a failure: first = -2 if no job with these target levels could have been placed
 
 // Commit job j to (gi2, ci2); one warp, all lanes, uniform control flow.  `alloc` (compile time): the job holds
 // (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target at
@@ -357,7 +358,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         if (alloc) { const int w = v.gc[node]; stay = fg_of(w) >= g2 - g && fc_of(w) >= c2 - c; }
         if (stay) target = node;
         else if (v.maxc[gi2] >= c2) target = rebuild ? first_fit_from_mark(v, sh, gi2, g2, c2, lane) : first_fit_warp(v, g2, c2, lane);
-        if (target < 0) return false;
+        if (target < 0) { out.first = -2; return false; }
     } else {
         k2 = g2 >> sp.log2Gn;
         if (cdiv_k(c2, k2) > sp.Cn) return false;
@@ -373,7 +374,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     const int64_t avail = k2 > 1 ? sp.Mn : v.free_m[target] + ((stay && alloc) ? m_cur : 0);
     const bool fits = lane < sp.nM && v.ml[lane < sp.nM ? lane : 0] <= avail * k2;
     const unsigned fb = __ballot_sync(0xffffffffu, fits);
-    if (!fb) return false;
+    if (!fb) { out.first = -2; return false; }      // the node found has too little memory for any level
     const int mi = 31 - __clz(fb);
 
     float val; int plan, f; bool okg;
@@ -638,6 +639,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     __shared__ Shared sh;
+    // Phase A: pa_fail[gi * nC + ci] = number of jobs placed when a job with these target levels last found no node
+    // or a node without memory for any level; while nothing else has been placed since, the next one fares the same
+    __shared__ int pa_fail[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS];
     __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];      // what is left of every tenant's quota: GPUs, cores
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
@@ -679,10 +683,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
     if (tid < 32) sh.dirty[tid] = 1;
     if (tid < RUBICK_MAX_G_LEVELS) sh.ff_pos[tid] = 0;
+    for (int t = tid; t < n_cls; t += RT) pa_fail[t] = -1;
     for (int i = tid; i < 2 * A.n_tenants; i += RT) rem_q[i] = A.quota[i];
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
-        sh.ver = 0; sh.maxc_dirty = 1; sh.empty_lo = 0;
+        sh.ver = 0; sh.maxc_dirty = 1; sh.empty_lo = 0; sh.pa_commits = 0;
     }
     __syncthreads();
 
@@ -763,6 +768,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 const int g2 = v.gl[a0.x], c2 = v.clv[a0.y];
                 if (g2 <= sp.Gn) may = v.maxc[a0.x] >= c2;
                 else { const int k2 = g2 >> sp.log2Gn; may = (c2 + k2 - 1) / k2 <= sp.Cn && sh.n_empty >= k2; }
+                may = may && pa_fail[a0.x * sp.nC + a0.y] != sh.pa_commits;
             }
             unsigned todo = __ballot_sync(0xffffffffu, may);
             // the records of the batch go through shared memory: one turn reads its job's with three loads
@@ -784,7 +790,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if (tn < 0 || tn >= A.n_tenants) continue;
                     if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[ci]) continue;
                 }
-                Committed cm;
+                if (pa_fail[gi * sp.nC + ci] == sh.pa_commits) continue;        // same levels, same cluster: same outcome
+                Committed cm; cm.first = -1;
                 if (commit_warp<false, true>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm)) {
                     const int s = sh.n_slots;
                     if (lane == 0) {
@@ -792,8 +799,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
                         v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
                         sh.n_slots = s + 1;
+                        sh.pa_commits += 1;
                         if (A.n_tenants > 0) { rem_q[2 * tn] -= sp.g_levels[gi]; rem_q[2 * tn + 1] -= sp.c_levels[ci]; }
                     }
+                    __syncwarp();
+                } else if (cm.first == -2) {
+                    if (lane == 0) pa_fail[gi * sp.nC + ci] = sh.pa_commits;
                     __syncwarp();
                 }
             }
