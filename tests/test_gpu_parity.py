@@ -306,6 +306,30 @@ def test_greedy_round_under_memory_pressure_and_small_nodes(mem_gib, cpus):
     assert (want["n_nodes"] > 1).any()                     # and some job spans whole nodes
 
 
+@pytest.mark.parametrize("mem_gib,share", [(48, 1.0), (64, 0.7), (160, 1.0)])
+def test_guaranteed_jobs_when_nodes_run_out_of_host_memory(mem_gib, share):
+    """Phase A under memory pressure: the node first fit finds has GPUs and cores left but no memory for any
+    level, so the job stays pending; jobs with the same minimum levels that follow fare the same until another
+    job is placed (the device round remembers such outcomes instead of trying again)."""
+    rng = np.random.default_rng(77)
+    J, N = 300, 6
+    cfg = workloads.make("cluster-512", J=J, n_nodes=N)
+    guar = rng.uniform(size=J) < share
+    cfg["jobs"]["gmin_idx"] = np.where(guar, rng.integers(0, 3, J), -1)
+    cfg["jobs"]["cmin_idx"] = np.where(guar, rng.integers(0, 3, J), -1)
+    cfg["env"] = env(mem_per_node_bytes=mem_gib * GIB)
+    gpu = Gpu(cfg)
+    plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 N, want_log=True)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, N)
+    assert_rounds_equal(got, want)
+    pending = want["status"] == rb.PENDING
+    assert pending.any() and (want["status"] == rb.RUNNING).any()
+    if mem_gib <= 64 and share == 1.0:
+        assert (want["node"][:, 0] > 0).any()              # GPUs are left over: memory is what ran out
+
+
 def test_greedy_round_step_cap():
     cfg = workloads.make("paper-scale")
     gpu = Gpu(cfg)
