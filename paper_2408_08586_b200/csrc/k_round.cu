@@ -957,6 +957,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const unsigned fb = __ballot_sync(FULL, lane < sp.nM && v.ml[lane < sp.nM ? lane : 0] <= avail * k2);
                     const int mi = fb ? 31 - __clz(fb) : -1;
                     const int ptr = v.cls_ptr[t], end = v.cls_end[t];
+                    int n_fail = 0;
+                    if (mi < 0) {
+                        // The node has no memory for any level: every head of the class that outranks the rest fails
+                        // the same way.  The class is sorted, so they are counted by a search with 32 probes a step.
+                        int lo = ptr, hi = end;          // entries before lo are in the run, entry hi (if any) is not
+                        while (lo < hi) {
+                            const int stride = (hi - lo + 31) / 32;
+                            const int idx = lo + lane * stride;
+                            const bool in = idx < hi && (0x80000000u | key_gain_bits(A.keys[idx])) > B;
+                            const int c = __popc(__ballot_sync(FULL, in));
+                            if (c == 0) break;
+                            hi = min(lo + c * stride, hi);
+                            lo += (c - 1) * stride + 1;
+                        }
+                        n_fail = min(lo - ptr, room);
+                        if (A.step_log)
+                            for (int i = lane; i < n_fail; i += 32) A.step_log[steps0 + i] = (key_job(A.keys[ptr + i]) << 2) | 0;
+                    } else {
                     // RUN_U x 32 entries a turn: every lane looks at RUN_U of them, all loads of a kind in one wave
                     u64 k[RUN_U]; bool in_run[RUN_U], succ[RUN_U]; HotCurve cand[RUN_U];
 #pragma unroll
@@ -970,7 +988,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         succ[u] = false;
                         if (in_run[u] && mi >= 0) cand[u] = load_hc(A.hc + hc_idx(sp, key_job(k[u]), gi2, ci2));
                     }
-                    int n_fail = 0; bool open_ = true;         // leading entries that are in the run and fail
+                    bool open_ = true;                          // leading entries that are in the run and fail
 #pragma unroll
                     for (int u = 0; u < RUN_U; ++u) {
                         if (in_run[u] && mi >= 0) {
@@ -989,12 +1007,13 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         if (open_) { n_fail += stop ? __ffs(stop) - 1 : 32; open_ = stop == 0u; }
                     }
                     if (n_fail > room) n_fail = room;
-                    if (n_fail > 0) {
-                        if (A.step_log) {
+                    if (A.step_log) {
 #pragma unroll
-                            for (int u = 0; u < RUN_U; ++u)
-                                if (32 * u + lane < n_fail) A.step_log[steps0 + 32 * u + lane] = (key_job(k[u]) << 2) | 0;
-                        }
+                        for (int u = 0; u < RUN_U; ++u)
+                            if (32 * u + lane < n_fail) A.step_log[steps0 + 32 * u + lane] = (key_job(k[u]) << 2) | 0;
+                    }
+                    }
+                    if (n_fail > 0) {
                         if (lane == 0) {
                             const int np = ptr + n_fail;
                             u64 nk = 0ull; float nw = 0.0f;
