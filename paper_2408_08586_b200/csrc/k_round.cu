@@ -642,6 +642,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // Phase A: pa_fail[gi * nC + ci] = number of jobs placed when a job with these target levels last found no node
     // or a node without memory for any level; while nothing else has been placed since, the next one fares the same
     __shared__ int pa_fail[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS];
+    // Phase B: bit t set = the last head of class t was placed; the next one is then tried directly instead of
+    // being looked at first as the start of a run of failing heads (either way gives the same steps)
+    __shared__ uint32_t cls_went[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS / 32];
     __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];      // what is left of every tenant's quota: GPUs, cores
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
@@ -684,6 +687,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     if (tid < 32) sh.dirty[tid] = 1;
     if (tid < RUBICK_MAX_G_LEVELS) sh.ff_pos[tid] = 0;
     for (int t = tid; t < n_cls; t += RT) pa_fail[t] = -1;
+    for (int t = tid; t < RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS / 32; t += RT) cls_went[t] = 0u;
     for (int i = tid; i < 2 * A.n_tenants; i += RT) rem_q[i] = A.quota[i];
     if (tid == 0) {
         sh.n_empty = N; sh.n_slots = 0; sh.steps = 0; sh.capped = 0; sh.stop = 0; sh.n_guar = 0; sh.n_ccls = 0;
@@ -940,7 +944,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             // class outrank every other candidate the sequential rule keeps trying them one after another
             // against the same target and the same memory level: lane i settles the i-th entry of the
             // class's sorted list, and everything before the first entry that would succeed is consumed.
-            if (go && (pay & 0x80000000u)) {
+            if (go && (pay & 0x80000000u) && !((cls_went[(pay & 0x7fffffffu) >> 5] >> (pay & 31u)) & 1u)) {
                 const int t = int(pay & 0x7fffffffu);
                 const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
                 const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
@@ -1238,7 +1242,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             sh.dirty[dirty_of(s)] = 1;
                         }
                     }
-                    if (lane == 0) { v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[CLS_G] = 1; }
+                    if (lane == 0) {
+                        v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[CLS_G] = 1;
+                        if (ok) cls_went[t >> 5] |= 1u << (t & 31); else cls_went[t >> 5] &= ~(1u << (t & 31));
+                    }
                 } else {
                     const int s = int(pay);
                     SlotA a = v.sa[s]; SlotB b = v.sb[s];
