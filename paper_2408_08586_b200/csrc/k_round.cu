@@ -462,6 +462,8 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         }
         if (lane == 0 && need_new > 0) sh.empty_lo = base - 32;
         d_empty -= need_new;
+        // while an empty node remains every entry of maxc[] equals the node's core count: nothing to recompute
+        if (n_empty + d_empty > 0) maxc_dirty = __any_sync(0xffffffffu, lane < sp.n_small && v.maxc[lane] != sp.Cn);
     }
     __syncwarp();
     if (rebuild) {
