@@ -2,7 +2,7 @@
 
 TEST INFRASTRUCTURE ONLY.  Builds ``liboracle.so`` beside the source with gcc on first use
 and marshals numpy arrays into the oracle's own plain layouts (jobs as rows of doubles,
-plans as rows of six int32, environment as a row of doubles).  Nothing here touches the
+plans as rows of seven int32, environment as a row of doubles).  Nothing here touches the
 CUDA library.
 """
 import ctypes as C
@@ -18,7 +18,7 @@ _SO = os.path.join(_HERE, "liboracle.so")
 JOB_FIELDS = ["P", "l", "h", "s", "b", "mu_cap", "alpha_act", "tau", "k_bwd", "k_sync", "k_opt",
               "k_opt_off", "k_off", "k_swap", "k_const", "w", "gmin_idx", "cmin_idx", "host_base_bytes", "tenant"]
 ENV_FIELDS = ["B_intra", "B_inter", "B_pcie", "gpu_mem_bytes", "gpus_per_node", "cpus_per_node",
-              "mem_per_node_bytes", "bytes_per_elem", "strict_zero_dp_only"]
+              "mem_per_node_bytes", "bytes_per_elem", "strict_zero_dp_only", "zero3_extra_volume"]
 TERM_FIELDS = ["valid", "mu", "m", "a", "T_fwd", "T_bwd", "V_dp", "V_tp", "V_pp", "T_dp", "T_tp",
                "T_pp", "T_cc", "T_opt", "T_off", "T_oo", "T_iter", "thr"]
 MEM_FIELDS = ["params", "grads", "opt", "act", "gpu_total", "gpu_ok", "host_need", "nodes"]
@@ -199,24 +199,34 @@ def gain(jobs, curve_val, g_levels, c_levels, state_g, state_c, state_val):
     return gg, gc, ng, nc
 
 
+CAND_FIELDS = ("gain", "next", "placeable", "v_cur", "v_next", "units", "shut", "m_commit", "v_commit", "g_commit")
+
+
 def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,
-                   n_nodes, max_steps=1 << 30, want_log=False, quota=None):
-    """One greedy round on single-precision curve tables.
+                   n_nodes, max_steps=1 << 30, want_log=False, quota=None, double_decisions=False, want_candidates=False):
+    """One greedy round.  Default: decisions in single precision on the curve table rounded to single
+    precision.  double_decisions: every decision in double precision on curve_val as given (float64).
+    want_candidates: also `cand`, a dict of [J, 2] arrays (CAND_FIELDS; axis 1 = GPU / CPU increment) with
+    what every job offered for the decision the round stopped at (the step `max_steps` cut off, or the
+    last look that found nothing to do).
 
     -> dict(g, c, m_bytes, plan, first_node, n_nodes, status, m_level, thr, node (N x 4:
-    free g, free c, free m, owner), steps, capped, log)."""
+    free g, free c, free m, owner), steps, capped, log[, cand])."""
     rows = job_rows(jobs)
     J = rows.shape[0]
     cv = np.ascontiguousarray(curve_val, dtype=np.float32)
+    cv64 = _f64(curve_val) if double_decisions else None
     cp, cg = _i32(curve_plan), _i32(curve_g)
     feas = np.ascontiguousarray(feas, dtype=np.uint32)
     Pn = feas.shape[1] if feas.ndim == 2 else 0
     gl, cl, ml = _i64(g_levels), _i64(c_levels), _i64(m_levels)
     out_i = np.zeros((max(J, 1), 8), dtype=np.int64)
     out_v = np.zeros(max(J, 1), dtype=np.float32)
+    out_v64 = np.zeros(max(J, 1), dtype=np.float64)
     node = np.zeros((n_nodes, 4), dtype=np.int64)
     cap = int(min(max_steps, J * (len(gl) + len(cl) + 2) + 1))
     log = np.zeros(max(cap, 1), dtype=np.int32)
+    cand = np.zeros((max(J, 1), 2, len(CAND_FIELDS)), dtype=np.float64)
     qt = None if quota is None else _i64(quota).reshape(-1, 2)      # per tenant: GPUs, cores
     r = lib().oracle_round(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double), _p(cv, C.c_float),
                            _p(cp, C.c_int32), _p(cg, C.c_int32), _p(feas, C.c_uint32), C.c_int(Pn),
@@ -224,14 +234,20 @@ def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_
                            _p(ml, C.c_int64), C.c_int(len(ml)), C.c_int(n_nodes), C.c_int(cap),
                            _p(qt, C.c_int64) if qt is not None else None, C.c_int(0 if qt is None else len(qt)),
                            _p(out_i, C.c_int64), _p(out_v, C.c_float), _p(node, C.c_int64),
-                           _p(log, C.c_int32) if want_log else None)
+                           _p(log, C.c_int32) if want_log else None,
+                           _p(cv64, C.c_double) if cv64 is not None else None, _p(out_v64, C.c_double),
+                           _p(cand, C.c_double) if want_candidates else None)
     capped = r < 0
     steps = -r - 1 if capped else r
     out_i = out_i[:J]
-    return dict(g=out_i[:, 0].copy(), c=out_i[:, 1].copy(), m_bytes=out_i[:, 2].copy(),
-                plan=out_i[:, 3].copy(), first_node=out_i[:, 4].copy(), n_nodes=out_i[:, 5].copy(),
-                status=out_i[:, 6].copy(), m_level=out_i[:, 7].copy(), thr=out_v[:J].copy(), node=node,
-                steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
+    res = dict(g=out_i[:, 0].copy(), c=out_i[:, 1].copy(), m_bytes=out_i[:, 2].copy(),
+               plan=out_i[:, 3].copy(), first_node=out_i[:, 4].copy(), n_nodes=out_i[:, 5].copy(),
+               status=out_i[:, 6].copy(), m_level=out_i[:, 7].copy(),
+               thr=out_v64[:J].copy() if double_decisions else out_v[:J].copy(), node=node,
+               steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
+    if want_candidates:
+        res["cand"] = {k: cand[:J, :, i].copy() for i, k in enumerate(CAND_FIELDS)}
+    return res
 
 
 def schedule_round_incremental(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,

@@ -69,6 +69,7 @@ enum {
     EF_GN, EF_CN, EF_MN,                /* GPUs, CPU cores, host bytes per node     */
     EF_E,                               /* bytes per element (2 = fp16)             */
     EF_STRICT,                          /* 1: ZeRO / offload only with t = p = 1    */
+    EF_Z3VOL,                           /* 1: ZeRO stage 3 moves 1.5 x V_dp (an option outside the paper; 0 = Section 4.1's rule) */
     EF_COUNT
 };
 
@@ -163,9 +164,12 @@ void oracle_terms(const double *job, const double *env, const int32_t *pl, doubl
     /* T_bwd = k_bwd * T_fwd, plus one recomputing forward under gradient checkpointing */
     double T_bwd = job[JF_KBWD] * T_fwd + (gc ? T_fwd : 0.0);
 
-    /* volumes in bytes; a degree of 1 sends nothing */
+    /* volumes in bytes; a degree of 1 sends nothing.  Section 4.1 ("Data Parallelism") gives
+     * V_dp = P 2(d-1)/(d t p) and applies it to the whole ZeRO series, so every stage uses it; the
+     * environment may switch on a factor 1.5 for stage 3 (parameter gathers on top of the gradient
+     * traffic), which is outside the paper and off by default. */
     double V_dp = 0.0, V_tp = 0.0, V_pp = 0.0;
-    if (d > 1) V_dp = e * P * 2.0 * (d - 1.0) / (d * t * p) * (z == 3 ? 1.5 : 1.0);
+    if (d > 1) V_dp = e * P * 2.0 * (d - 1.0) / (d * t * p) * ((z == 3 && env[EF_Z3VOL] != 0.0) ? 1.5 : 1.0);
     if (t > 1) V_tp = e * 4.0 * 2.0 * (t - 1.0) * b * s * h * l / (d * t);
     if (p > 1) V_pp = e * 2.0 * p * b * s * h / (d * t);
 
@@ -429,14 +433,18 @@ void oracle_min_resources(const double *thr, const uint32_t *feas, const double 
 /* ======================================================================================
  * Scheduling: marginal gains and one greedy round.
  *
- * All decisions are taken in single precision on the single-precision curve table, with
- * one rounding per operation in the order written (compile with -ffp-contract=off), so
- * that a second implementation can reproduce every comparison bit for bit.
+ * Two arithmetic forms of the same step list.  The default takes every decision in single
+ * precision on a single-precision curve table, with one rounding per operation in the order
+ * written (compile with -ffp-contract=off), so that a second implementation can reproduce every
+ * comparison bit for bit.  With a double-precision curve table (Sched.cv64) the same decisions
+ * are taken in double precision on it; the two forms may part only at a decision whose margin
+ * is within the rounding of the single-precision form (tests/test_oracle_sched.py).
  * ==================================================================================== */
 
 typedef struct {
     int J, nG, nC, nM, P, N;
     const float *cv;          /* curve value   [J][G][C][M] */
+    const double *cv64;       /* the same table in double precision: decisions in double (NULL: in single on cv) */
     const int32_t *cp;        /* curve plan    [J][G][C][M] */
     const int32_t *cg;        /* curve g used  [J][G][C][M] */
     const uint32_t *feas;     /* [J][P] */
@@ -452,7 +460,7 @@ typedef struct {
     int gi, ci;               /* level indices, gi = -1 when unallocated */
     int64_t g, c, m;          /* amounts held (m in bytes)               */
     int plan, node, k;        /* plan index, first node, node count      */
-    float val;                /* predicted throughput of the allocation  */
+    double val;               /* predicted throughput of the allocation (a float's value in the single-precision form) */
     int status;
     int frozen[2];            /* a rejected GPU / CPU increment is not retried this round */
 } JobState;
@@ -462,6 +470,17 @@ typedef struct { int ok; int k; int stay; int node; int need_new; } Place;
 static size_t cidx(const Sched *S, int j, int gi, int ci, int mi)
 {
     return (((size_t)j * S->nG + gi) * S->nC + ci) * S->nM + mi;
+}
+
+/* curve value at a table offset, in the precision the decisions are taken in */
+static double cval(const Sched *S, size_t o) { return S->cv64 ? S->cv64[o] : (double)S->cv[o]; }
+
+/* weighted gain per unit, (w v - w v_cur) / units, one rounding per operation */
+static double unit_gain(const Sched *S, double w, double v, double vcur, double units)
+{
+    if (S->cv64) return (w * v - w * vcur) / units;
+    float wf = (float)w;
+    return (double)((wf * (float)v - wf * (float)vcur) / (float)units);
 }
 
 static int count_empty(const Sched *S)
@@ -519,6 +538,19 @@ static void release_job(Sched *S, int j, JobState *js)
     }
 }
 
+/* highest host-memory level whose per-node share fits the node(s) of placement pl (-1: none) */
+static int commit_level(const Sched *S, const JobState *js, Place pl)
+{
+    int k2 = pl.k;
+    int64_t avail;
+    if (k2 > 1) avail = S->Mn;
+    else avail = S->free_m[pl.node] + ((pl.stay && js->gi >= 0) ? js->m : 0);
+    int mi = -1;
+    for (int i = 0; i < S->nM; ++i)
+        if (cdiv(S->m_levels[i], k2) <= avail) mi = i;
+    return mi;
+}
+
 /* Commit job j to (gi2, ci2) at placement pl: pick the host-memory level that fits the
  * target node(s), read the curve there (GetBestPlan), allocate that plan's memory
  * (AllocMem).  Returns 1 on success; 0 leaves everything unchanged.  need_gain != 0
@@ -527,16 +559,11 @@ static int commit(Sched *S, int j, JobState *js, int gi2, int ci2, Place pl, int
 {
     int64_t g2 = S->g_levels[gi2], c2 = S->c_levels[ci2];
     int k2 = pl.k;
-    int64_t avail;
-    if (k2 > 1) avail = S->Mn;
-    else avail = S->free_m[pl.node] + ((pl.stay && js->gi >= 0) ? js->m : 0);
-    int mi = -1;
-    for (int i = 0; i < S->nM; ++i)
-        if (cdiv(S->m_levels[i], k2) <= avail) mi = i;
+    int mi = commit_level(S, js, pl);
     if (mi < 0) return 0;
     size_t o = cidx(S, j, gi2, ci2, mi);
-    float v = S->cv[o]; int plan = S->cp[o]; int gu = S->cg[o];
-    if (plan < 0 || !(v > 0.0f)) return 0;
+    double v = cval(S, o); int plan = S->cp[o]; int gu = S->cg[o];
+    if (plan < 0 || !(v > 0.0)) return 0;
     if ((int64_t)gu != g2) return 0;              /* the level's own plans do not fit */
     if (need_gain && js->gi >= 0 && !(v > js->val)) return 0;
     uint32_t word = S->feas[(size_t)j * S->P + plan];
@@ -583,30 +610,27 @@ static int start_ci(const double *job) { return (int)job[JF_CMIN] > 0 ? (int)job
  * whose curve value, at the job's CPU level and the top host-memory level, strictly
  * exceeds the job's present value.  Target CPU level: the next one.  Returns through
  * next[0..1] the level indices (-1 = none) and through gain[0..1] the gains. */
-static void job_gains(const Sched *S, int j, const JobState *js, int32_t *next, float *gain)
+static void job_gains(const Sched *S, int j, const JobState *js, int32_t *next, double *gain)
 {
     const double *job = S->jobs + (size_t)j * JF_COUNT;
-    float w = (float)job[JF_W];
+    double w = job[JF_W];
     int mt = S->nM - 1;
     int allocated = js->gi >= 0;
     int ci = allocated ? js->ci : start_ci(job);
-    float cur = allocated ? js->val : 0.0f;
-    float vcur = allocated ? w * cur : 0.0f;
-    next[0] = next[1] = -1; gain[0] = gain[1] = 0.0f;
+    double cur = allocated ? js->val : 0.0;
+    next[0] = next[1] = -1; gain[0] = gain[1] = 0.0;
     for (int gi = js->gi + 1; gi < S->nG; ++gi) {
-        float v = S->cv[cidx(S, j, gi, ci, mt)];
+        double v = cval(S, cidx(S, j, gi, ci, mt));
         if (v > cur) {
-            float dg = (float)(S->g_levels[gi] - (allocated ? js->g : 0));
             next[0] = gi;
-            gain[0] = (w * v - vcur) / dg;
+            gain[0] = unit_gain(S, w, v, cur, (double)(S->g_levels[gi] - (allocated ? js->g : 0)));
             break;
         }
     }
     if (allocated && js->ci + 1 < S->nC) {
-        float v = S->cv[cidx(S, j, js->gi, js->ci + 1, mt)];
-        float dc = (float)(S->c_levels[js->ci + 1] - js->c);
-        float gn = (w * v - vcur) / dc;
-        if (gn > 0.0f) { next[1] = js->ci + 1; gain[1] = gn; }
+        double v = cval(S, cidx(S, j, js->gi, js->ci + 1, mt));
+        double gn = unit_gain(S, w, v, cur, (double)(S->c_levels[js->ci + 1] - js->c));
+        if (gn > 0.0) { next[1] = js->ci + 1; gain[1] = gn; }
     }
 }
 
@@ -628,9 +652,9 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
             for (int i = 0; i < nC; ++i) if (c_levels[i] == state_c[j]) js.ci = i;
             js.g = state_g[j]; js.c = state_c[j]; js.val = state_val[j];
         }
-        int32_t next[2]; float gain[2];
+        int32_t next[2]; double gain[2];
         job_gains(&S, j, &js, next, gain);
-        gain_gpu[j] = gain[0]; gain_cpu[j] = gain[1]; next_g[j] = next[0]; next_c[j] = next[1];
+        gain_gpu[j] = (float)gain[0]; gain_cpu[j] = (float)gain[1]; next_g[j] = next[0]; next_c[j] = next[1];
     }
 }
 
@@ -645,18 +669,29 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
  * out_i: [J][8] = g, c, m_bytes, plan, first node, node count, status, m level of plan
  * out_val: [J] predicted throughput; node_out: [N][4] = free g, free c, free m, owner
  * step_log (optional, length max_steps): (job << 2) | (type << 1) | accepted.
+ * curve_val64 (optional): the curve values in double precision; every decision is then taken in
+ * double on that table and out_val64 (optional) receives the values unrounded.
+ * cand_out (optional, [J][2][CAND_COUNT] doubles): what every job offered for the decision at which
+ * the round stopped (the step the cap cut off, or the last look that found nothing): per resource
+ * type the gain, the target level, whether it could be placed, the present and the target curve
+ * value, the units added, whether the job was shut out (pending or frozen for that type), and what a
+ * commit would read: the memory level that fits the target node(s) (-1: none), the curve value and
+ * the GPU count of the curve entry there.
  * Returns the number of Phase-B steps, negated - 1 if the cap was hit first. */
+enum { CAND_GAIN = 0, CAND_NEXT, CAND_PLACEABLE, CAND_VCUR, CAND_VNEXT, CAND_UNITS, CAND_SHUT, CAND_MCOMMIT, CAND_VCOMMIT, CAND_GCOMMIT, CAND_COUNT };
+
 int oracle_round(const double *jobs, int J, const double *env,
                  const float *curve_val, const int32_t *curve_plan, const int32_t *curve_g,
                  const uint32_t *feas, int P,
                  const int64_t *g_levels, int nG, const int64_t *c_levels, int nC,
                  const int64_t *m_levels, int nM, int N, int max_steps,
                  const int64_t *quota, int n_tenants,
-                 int64_t *out_i, float *out_val, int64_t *node_out, int32_t *step_log)
+                 int64_t *out_i, float *out_val, int64_t *node_out, int32_t *step_log,
+                 const double *curve_val64, double *out_val64, double *cand_out)
 {
     Sched S; memset(&S, 0, sizeof S);
     S.J = J; S.nG = nG; S.nC = nC; S.nM = nM; S.P = P; S.N = N;
-    S.cv = curve_val; S.cp = curve_plan; S.cg = curve_g; S.feas = feas; S.jobs = jobs;
+    S.cv = curve_val; S.cv64 = curve_val64; S.cp = curve_plan; S.cg = curve_g; S.feas = feas; S.jobs = jobs;
     S.g_levels = g_levels; S.c_levels = c_levels; S.m_levels = m_levels;
     S.Gn = (int64_t)env[EF_GN]; S.Cn = (int64_t)env[EF_CN]; S.Mn = (int64_t)env[EF_MN];
     S.free_g = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
@@ -703,13 +738,13 @@ int oracle_round(const double *jobs, int J, const double *env,
     /* Phase B: greedy increments */
     int steps = 0, capped = 0;
     for (;;) {
-        int best_j = -1, best_type = -1, best_next = -1; float best_gain = 0.0f;
+        int best_j = -1, best_type = -1, best_next = -1; double best_gain = 0.0;
         for (int type = 0; type < 2 && best_j < 0; ++type) {
             for (int j = 0; j < J; ++j) {
                 if (st[j].status == ST_PENDING || st[j].frozen[type]) continue;
-                int32_t next[2]; float gain[2];
+                int32_t next[2]; double gain[2];
                 job_gains(&S, j, &st[j], next, gain);
-                if (next[type] < 0 || !(gain[type] > 0.0f)) continue;
+                if (next[type] < 0 || !(gain[type] > 0.0)) continue;
                 int gi2 = type == 0 ? next[0] : st[j].gi;
                 int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
                 Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
@@ -729,6 +764,34 @@ int oracle_round(const double *jobs, int J, const double *env,
         ++steps;
     }
 
+    /* what every job offered for the decision the round stopped at */
+    if (cand_out)
+        for (int j = 0; j < J; ++j) {
+            int32_t next[2]; double gain[2];
+            job_gains(&S, j, &st[j], next, gain);
+            for (int type = 0; type < 2; ++type) {
+                double *c = cand_out + ((size_t)j * 2 + type) * CAND_COUNT;
+                for (int i = 0; i < CAND_COUNT; ++i) c[i] = 0.0;
+                c[CAND_GAIN] = gain[type]; c[CAND_NEXT] = next[type];
+                c[CAND_SHUT] = st[j].status == ST_PENDING || st[j].frozen[type];
+                c[CAND_VCUR] = st[j].gi >= 0 ? st[j].val : 0.0;
+                if (next[type] < 0) continue;
+                int gi2 = type == 0 ? next[0] : st[j].gi;
+                int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
+                Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+                c[CAND_PLACEABLE] = pl.ok;
+                c[CAND_MCOMMIT] = -1.0;
+                if (pl.ok && (pl.k > 1 || pl.node >= 0)) {
+                    int mi = commit_level(&S, &st[j], pl);
+                    c[CAND_MCOMMIT] = mi;
+                    if (mi >= 0) { c[CAND_VCOMMIT] = cval(&S, cidx(&S, j, gi2, ci2, mi)); c[CAND_GCOMMIT] = curve_g[cidx(&S, j, gi2, ci2, mi)]; }
+                }
+                c[CAND_VNEXT] = cval(&S, cidx(&S, j, gi2, ci2, mt));
+                c[CAND_UNITS] = type == 0 ? (double)(g_levels[gi2] - (st[j].gi >= 0 ? st[j].g : 0))
+                                          : (double)(c_levels[ci2] - st[j].c);
+            }
+        }
+
     for (int j = 0; j < J; ++j) {
         int64_t *o = out_i + (size_t)j * 8;
         int alloc = st[j].gi >= 0;
@@ -738,7 +801,8 @@ int oracle_round(const double *jobs, int J, const double *env,
         int f = -1;
         if (alloc) { uint32_t wd = feas[(size_t)j * P + st[j].plan]; f = 0; while (f < nM && !((wd >> f) & 1u)) ++f; }
         o[7] = f;
-        out_val[j] = alloc ? st[j].val : 0.0f;
+        out_val[j] = alloc ? (float)st[j].val : 0.0f;
+        if (out_val64) out_val64[j] = alloc ? st[j].val : 0.0;
     }
     if (node_out)
         for (int n = 0; n < N; ++n) {
@@ -795,7 +859,7 @@ static Shrink shrink_option(const Sched *S, int v, const JobState *js, int type,
     const double *job = S->jobs + (size_t)v * JF_COUNT;
     float w = (float)job[JF_W];
     int mt = S->nM - 1;
-    float vcur = w * js->val;
+    float vcur = w * (float)js->val;
     if (type == 0) {
         if (guaranteed && min_gi < 0) return sh;
         int lo = guaranteed ? min_gi : 0;
@@ -828,7 +892,7 @@ static int do_shrink(Sched *S, int v, JobState *js, Shrink sh, int apply)
         if (apply) {
             release_job(S, v, js);
             js->gi = -1; js->ci = 0; js->g = js->c = js->m = 0; js->plan = -1; js->node = -1; js->k = 0;
-            js->val = 0.0f; js->status = ST_UNALLOCATED;
+            js->val = 0.0; js->status = ST_UNALLOCATED;
         }
         return 1;
     }
@@ -1008,14 +1072,14 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
     /* Phase B */
     int steps = 0, capped = 0;
     for (;;) {
-        int best_j = -1, best_type = -1, best_next = -1, by_exchange = 0; float best_gain = 0.0f;
+        int best_j = -1, best_type = -1, best_next = -1, by_exchange = 0; double best_gain = 0.0;
         for (int pass = 0; pass < 2 && best_j < 0; ++pass)          /* 0: fits free resources; 1: any */
             for (int type = 0; type < 2 && best_j < 0; ++type)
                 for (int j = 0; j < J; ++j) {
                     if (!active[j] || pinned[j] || st[j].status == ST_PENDING || st[j].frozen[type]) continue;
-                    int32_t next[2]; float gain[2];
+                    int32_t next[2]; double gain[2];
                     job_gains(&S, j, &st[j], next, gain);
-                    if (next[type] < 0 || !(gain[type] > 0.0f)) continue;
+                    if (next[type] < 0 || !(gain[type] > 0.0)) continue;
                     if (pass == 0) {
                         int gi2 = type == 0 ? next[0] : st[j].gi;
                         int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
@@ -1038,7 +1102,7 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
              * asks for the resource of its increment; a queued job pre-allocates GPUs and cores
              * together, so its value counts per GPU and per core */
             float cand[2] = {0.0f, 0.0f};
-            cand[best_type] = best_gain;
+            cand[best_type] = (float)best_gain;
             if (st[j].gi >= 0) {
                 if (st[j].k == 1) ok = exchange(&S, st, &R, j, gi2, ci2, st[j].node, 0, cand, 1);
             } else {
@@ -1062,7 +1126,7 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
         int f = -1;
         if (alloc) { uint32_t wd = feas[(size_t)j * P + st[j].plan]; f = 0; while (f < nM && !((wd >> f) & 1u)) ++f; }
         o[7] = f;
-        out_val[j] = alloc ? st[j].val : 0.0f;
+        out_val[j] = alloc ? (float)st[j].val : 0.0f;
     }
     if (node_out)
         for (int n = 0; n < N; ++n) {

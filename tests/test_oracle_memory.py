@@ -152,6 +152,40 @@ def test_memory_terms_by_hand():
     assert mg["act"] == 12 * 2 * 1024 * 4 * 2048 + A
 
 
+def test_micro_batches_in_flight_and_layers_per_stage_by_hand():
+    """A pipelined plan with more micro-batches than stages: b = 64, d = 2 -> 32 samples per replica in
+    micro-batches of 2 -> m = 16 > p = 4, so 4 micro-batches are in flight (the smaller of the two);
+    26 layers over 4 stages -> 7 on the fullest stage (rounded up).  t = 2.
+    Per layer and micro-batch 34 * 1024 * 2 * 2048 / 2 = 71,303,168 bytes."""
+    job = one_job(P=1e9, l=26, h=2048, s=1024, b=64, mu_cap=2, alpha_act=34)
+    plain = oracle.memory(job, 0, env(), (2, 2, 4, 0, 0, 0))
+    assert plain["act"] == 1_996_488_704                      # 7 layers * 4 in flight * 71,303,168
+    ckpt = oracle.memory(job, 0, env(), (2, 2, 4, 0, 1, 0))
+    assert ckpt["act"] == 306_184_192                         # 28 * (2 * 1024 * 2 * 2048) + one live layer
+    # fewer micro-batches than stages: b = 8, d = 2, micro-batch 2 -> m = 2 < p = 4 -> 2 in flight
+    few = oracle.memory(one_job(P=1e9, l=26, h=2048, s=1024, b=8, mu_cap=2, alpha_act=34), 0, env(), (2, 2, 4, 0, 0, 0))
+    assert few["act"] == 998_244_352                          # 7 * 2 * 71,303,168
+    tm = oracle.terms(job, 0, env(), (2, 2, 4, 0, 0, 0), 8)
+    assert (tm["mu"], tm["m"], tm["a"]) == (2, 16, 1)
+
+
+def test_per_node_share_of_host_memory_on_a_multi_node_plan_by_hand():
+    """32 GPUs = 4 whole nodes, ZeRO-Offload: host need = 32 * 4 GiB + 14 * (1e11 + 1) = 1,537,438,953,486
+    bytes, a quarter of it per node = 384,359,738,371.5 -> 384,359,738,372 (rounded up).  The plan runs at a
+    memory level that covers the total only if a node also holds its share."""
+    job = one_job(P=100_000_000_001, l=24, h=2048, s=1024, b=16, mu_cap=1)
+    plan = (4, 8, 1, 2, 0, 1)
+    levels = [1400 * GIB, 1500 * GIB]                         # below / above the total need
+    mem = oracle.memory(job, 0, env(), plan)
+    assert mem["host_need"] == 1_537_438_953_486 and mem["nodes"] == 4 and mem["gpu_ok"] == 1
+    assert oracle.feas_word(job, 0, env(mem_per_node_bytes=384_359_738_372), plan, levels) == 0b10
+    assert oracle.feas_word(job, 0, env(mem_per_node_bytes=384_359_738_371), plan, levels) == 0
+    # on one node (8 GPUs) the whole need sits on that node
+    one = oracle.memory(job, 0, env(), (1, 8, 1, 2, 0, 1))
+    assert one["host_need"] == 8 * 4 * GIB + 1_400_000_000_014 and one["nodes"] == 1
+    assert oracle.feas_word(job, 0, env(mem_per_node_bytes=one["host_need"] - 1), (1, 8, 1, 2, 0, 1), [2048 * GIB]) == 0
+
+
 def test_rule_on_the_wider_plan_space_with_python_integers(paper_scale):
     """Degrees of any size and the explicit accumulation axis: the same independent recomputation."""
     cfg = dict(paper_scale)

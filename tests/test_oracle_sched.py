@@ -230,3 +230,81 @@ def test_tenant_quotas_limit_the_privileged_jobs():
                                 cfg["n_nodes"], quota=np.array([[10**6, 10**6]] * 2), **kw)
     for k in ("g", "c", "plan", "status", "first_node"):
         assert np.array_equal(big[k], free[k])
+
+
+# ---------------------------------------------------------------- single- against double-precision decisions
+def double_tables(cfg, nthreads=4):
+    """The oracle's chain without any rounding to single precision."""
+    plans, _ = oracle.enumerate_plans(cfg["g_levels"])
+    thr, feas = oracle.eval_candidates(cfg["jobs"], plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=nthreads)
+    cv, cp, cg = oracle.best_plan(thr, feas, plans, cfg["g_levels"], len(cfg["m_levels"]), prefix=True, nthreads=nthreads)
+    return plans, feas, cv, cp, cg
+
+
+def test_candidate_dump_reproduces_every_decision_of_a_round(paper_scale):
+    """The dump of what every job offered is the arbiter of the near-tie checks below: replaying the rule on it
+    must give the logged decision at every step of a round, and nothing after the last one."""
+    import near_tie
+    cfg = paper_scale
+    tb = tables(cfg)
+    full = run_round(cfg, tb, want_log=True)
+    assert full["steps"] > 20
+    for k in range(full["steps"] + 1):
+        r = run_round(cfg, tb, max_steps=k, want_log=True, want_candidates=True)
+        assert r["steps"] == k and np.array_equal(r["log"], full["log"][:k])
+        pick = near_tie.oracle_pick(r["cand"])
+        assert pick == (near_tie.decode(full["log"][k])[:2] if k < full["steps"] else None)
+        c = r["cand"]
+        has = c["next"] >= 0
+        # the gain is the weighted rise per unit, to single-precision rounding
+        w = np.asarray(cfg["jobs"]["w"])[:, None]
+        rise = (w * (c["v_next"] - c["v_cur"]))[has] / c["units"][has]
+        assert np.allclose(c["gain"][has], rise, rtol=0, atol=float((1e-6 * w * (c["v_next"] + c["v_cur"]))[has].max()))
+
+
+@pytest.mark.parametrize("name,J,N", [("tiny", None, None), ("paper-scale", None, None), ("cluster-512", 1024, 64),
+                                      ("events", 800, 64), ("throughput-stress", 2000, 64)])
+def test_single_precision_decisions_part_from_double_only_at_a_near_tie(name, J, N):
+    """The round decides in single precision on the curve table rounded to single precision (so that a GPU
+    kernel can follow it bit for bit); the method itself is stated in real numbers.  Deciding in double
+    precision on the unrounded table must give the same step log up to the first decision whose margin is
+    within the single-precision rounding of its gains; without such a near tie, the same round altogether."""
+    import near_tie
+    cfg = workloads.make(name, J=J, n_nodes=N)
+    plans, feas, cv, cp, cg = double_tables(cfg, nthreads=8)
+    args = (cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"], cfg["n_nodes"])
+    single = oracle.schedule_round(*args, want_log=True)
+    double = oracle.schedule_round(*args, want_log=True, double_decisions=True)
+    found = near_tie.assert_divergence_is_a_near_tie(
+        lambda k: oracle.schedule_round(*args, max_steps=k, want_log=True, double_decisions=True, want_candidates=True),
+        double["log"], single["log"], cfg["jobs"]["w"], tol=2.0 ** -24)
+    if found is None:
+        for key in ("g", "c", "m_bytes", "plan", "first_node", "n_nodes", "status", "node"):
+            assert np.array_equal(single[key], double[key]), key
+        assert np.allclose(single["thr"], double["thr"], rtol=2.0 ** -23, atol=0)
+    w = np.asarray(cfg["jobs"]["w"], dtype=np.float64)
+    assert float((w * single["thr"]).sum()) == pytest.approx(float((w * double["thr"]).sum()), rel=1e-4)
+
+
+def test_near_tie_check_refuses_a_planted_mistake():
+    """The check must not pass whatever it is given: a second chain that reads a table off by a tenth of a percent
+    for some jobs (a planted mistake, far outside rounding) parts from the oracle at a decision with a clear margin."""
+    import near_tie
+    cfg = workloads.make("cluster-512", J=600, n_nodes=48)
+    plans, feas, cv, cp, cg = double_tables(cfg, nthreads=8)
+    args = lambda table: (cfg["jobs"], cfg["env"], table, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"], cfg["n_nodes"])
+    good = oracle.schedule_round(*args(cv), want_log=True, double_decisions=True)
+    rng = np.random.default_rng(11)
+    refused = 0
+    for trial in range(6):
+        bad_table = cv * (1.0 + 1e-3 * rng.uniform(-1.0, 1.0, (cv.shape[0], 1, 1, 1)))
+        bad = oracle.schedule_round(*args(bad_table), want_log=True, double_decisions=True)
+        if near_tie.first_difference(good["log"], bad["log"]) is None:
+            continue
+        try:
+            near_tie.assert_divergence_is_a_near_tie(
+                lambda k: oracle.schedule_round(*args(cv), max_steps=k, want_log=True, double_decisions=True, want_candidates=True),
+                good["log"], bad["log"], cfg["jobs"]["w"], tol=2.0 ** -24)
+        except AssertionError:
+            refused += 1
+    assert refused >= 5
