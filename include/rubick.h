@@ -70,6 +70,10 @@ typedef struct {
     int32_t cpus_per_node;
     int32_t bytes_per_elem;             /* 2 = fp16 mixed precision                                  */
     int32_t strict_zero_dp_only;        /* 1: ZeRO stages / offload only for pure data parallelism   */
+    int32_t zero3_extra_volume;         /* 0: Section 4.1's V_dp for every ZeRO stage (the paper's rule);
+                                           1: stage 3 moves 1.5 x V_dp (parameter gathers on top of the
+                                           gradient ring; an option outside the paper)                */
+    int32_t reserved;                   /* 0                                                         */
 } rubick_env;
 
 /* One job: the model, batch and fitted coefficients of paper Table 1.  Exactly 128 bytes. */
@@ -356,11 +360,15 @@ int rubick_incremental_event_host(rubick_ctx *ctx, const rubick_job *h_jobs, int
  * (32 bytes per job), which every GPU that loads the library holds until the process exits.
  *  - J above RUBICK_NOALLOC_MAX_JOBS is rejected with EINVAL and a message naming the limit.
  *  - The first call on a device looks up the array's device address (one cudaGetSymbolAddress
- *    with that device current) and remembers it; make that first call before any stream capture.
- *  - All calls, from every context on the device, share the one array.  The kernel rewrites the
- *    state of all J jobs before reading it, so contents left by an earlier call do no harm; but
- *    two calls whose kernels overlap on the GPU (different streams, different contexts or
- *    processes or host threads) race on it and give undefined results.  Run them one after another. */
+ *    with that device current) and remembers it for the life of the process; make that first call
+ *    before any stream capture.  Two host threads may make their first calls at the same time (they
+ *    store the same address).  The address belongs to the device's primary context: do not call this
+ *    entry point on a device after a cudaDeviceReset of it.
+ *  - All calls of this process on the device, from every rubick context, share the one array (another
+ *    process has a copy of its own).  The kernel rewrites the state of all J jobs before reading it,
+ *    so contents left by an earlier call do no harm; but two calls whose kernels overlap on the GPU
+ *    (different streams, different rubick contexts or host threads) race on it and give undefined
+ *    results.  Run them one after another. */
 int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
                                 const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
                                 const uint32_t *d_feas, const rubick_cluster *h_cluster, int max_steps,

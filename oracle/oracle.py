@@ -199,7 +199,7 @@ def gain(jobs, curve_val, g_levels, c_levels, state_g, state_c, state_val):
     return gg, gc, ng, nc
 
 
-CAND_FIELDS = ("gain", "next", "placeable", "v_cur", "v_next", "units", "shut", "m_commit", "v_commit", "g_commit")
+CAND_FIELDS = ("gain", "next", "placeable", "v_cur", "v_next", "units", "shut", "m_commit", "v_commit", "g_commit", "gi", "ci")
 
 
 def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,

@@ -676,9 +676,9 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
  * type the gain, the target level, whether it could be placed, the present and the target curve
  * value, the units added, whether the job was shut out (pending or frozen for that type), and what a
  * commit would read: the memory level that fits the target node(s) (-1: none), the curve value and
- * the GPU count of the curve entry there.
+ * the GPU count of the curve entry there, and the (GPU level, core level) the increment leads to.
  * Returns the number of Phase-B steps, negated - 1 if the cap was hit first. */
-enum { CAND_GAIN = 0, CAND_NEXT, CAND_PLACEABLE, CAND_VCUR, CAND_VNEXT, CAND_UNITS, CAND_SHUT, CAND_MCOMMIT, CAND_VCOMMIT, CAND_GCOMMIT, CAND_COUNT };
+enum { CAND_GAIN = 0, CAND_NEXT, CAND_PLACEABLE, CAND_VCUR, CAND_VNEXT, CAND_UNITS, CAND_SHUT, CAND_MCOMMIT, CAND_VCOMMIT, CAND_GCOMMIT, CAND_GI, CAND_CI, CAND_COUNT };
 
 int oracle_round(const double *jobs, int J, const double *env,
                  const float *curve_val, const int32_t *curve_plan, const int32_t *curve_g,
@@ -779,7 +779,7 @@ int oracle_round(const double *jobs, int J, const double *env,
                 int gi2 = type == 0 ? next[0] : st[j].gi;
                 int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
                 Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
-                c[CAND_PLACEABLE] = pl.ok;
+                c[CAND_PLACEABLE] = pl.ok; c[CAND_GI] = gi2; c[CAND_CI] = ci2;
                 c[CAND_MCOMMIT] = -1.0;
                 if (pl.ok && (pl.k > 1 || pl.node >= 0)) {
                     int mi = commit_level(&S, &st[j], pl);

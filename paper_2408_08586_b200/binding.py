@@ -41,7 +41,8 @@ assert ASSIGN_DTYPE.itemsize == 40 and NODE_DTYPE.itemsize == 24
 class Env(C.Structure):
     _fields_ = [("B_intra", C.c_double), ("B_inter", C.c_double), ("B_pcie", C.c_double),
                 ("gpu_mem_bytes", C.c_int64), ("mem_per_node_bytes", C.c_int64), ("gpus_per_node", C.c_int32),
-                ("cpus_per_node", C.c_int32), ("bytes_per_elem", C.c_int32), ("strict_zero_dp_only", C.c_int32)]
+                ("cpus_per_node", C.c_int32), ("bytes_per_elem", C.c_int32), ("strict_zero_dp_only", C.c_int32),
+                ("zero3_extra_volume", C.c_int32), ("reserved", C.c_int32)]
 
 
 class Grid(C.Structure):
@@ -189,7 +190,8 @@ class Context:
     def __init__(self, env, device=0, stream=None):
         e = Env(float(env["B_intra"]), float(env["B_inter"]), float(env["B_pcie"]), int(env["gpu_mem_bytes"]),
                 int(env["mem_per_node_bytes"]), int(env["gpus_per_node"]), int(env["cpus_per_node"]),
-                int(env["bytes_per_elem"]), int(env.get("strict_zero_dp_only", 0)))
+                int(env["bytes_per_elem"]), int(env.get("strict_zero_dp_only", 0)),
+                int(env.get("zero3_extra_volume", 0)), 0)
         self._h = C.c_void_p()
         self.device = device
         rc = lib().rubick_create(C.byref(self._h), C.byref(e), int(device), C.c_void_p(stream) if stream else None)

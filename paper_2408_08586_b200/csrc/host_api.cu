@@ -174,6 +174,7 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
     sp.P = P; sp.Q = P / 4; sp.nG = gr.nG; sp.nC = gr.nC; sp.nM = gr.nM;
     sp.Gn = Gn; sp.log2Gn = ilog2(Gn); sp.Cn = ctx->env.cpus_per_node;
     sp.strict = ctx->env.strict_zero_dp_only ? 1 : 0;
+    sp.z3_volume = ctx->env.zero3_extra_volume ? 1.5f : 1.0f;
     sp.wide = wide ? 1 : 0;
     sp.e = float(ctx->env.bytes_per_elem);
     sp.inv_B_intra = float(1.0 / ctx->env.B_intra);
@@ -239,15 +240,24 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
         wquads[i].w = 0u;
     }
 
+    // the new tables are built beside the old ones and swapped in only when everything has succeeded: a failed
+    // allocation or upload leaves the context with the plan space it had
     CUDA_TRY(ctx, cudaSetDevice(ctx->device), "cudaSetDevice");
-    if (ctx->d_quads) { cudaStreamSynchronize(ctx->stream); cudaFree(ctx->d_quads); ctx->d_quads = nullptr; }
-    CUDA_TRY(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->d_quads), quads.size() * sizeof(QuadDesc)), "cudaMalloc (plan table)");
-    CUDA_TRY(ctx, cudaMemcpy(ctx->d_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice), "upload plan table");
-    if (ctx->d_wide_quads) { cudaFree(ctx->d_wide_quads); ctx->d_wide_quads = nullptr; }
-    if (wide) {
-        CUDA_TRY(ctx, cudaMalloc(reinterpret_cast<void **>(&ctx->d_wide_quads), wquads.size() * sizeof(WideQuad)), "cudaMalloc (wide plan table)");
-        CUDA_TRY(ctx, cudaMemcpy(ctx->d_wide_quads, wquads.data(), wquads.size() * sizeof(WideQuad), cudaMemcpyHostToDevice), "upload wide plan table");
+    QuadDesc *new_quads = nullptr;
+    WideQuad *new_wide = nullptr;
+    cudaError_t ce = cudaMalloc(reinterpret_cast<void **>(&new_quads), quads.size() * sizeof(QuadDesc));
+    if (ce == cudaSuccess) ce = cudaMemcpy(new_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess && wide) {
+        ce = cudaMalloc(reinterpret_cast<void **>(&new_wide), wquads.size() * sizeof(WideQuad));
+        if (ce == cudaSuccess) ce = cudaMemcpy(new_wide, wquads.data(), wquads.size() * sizeof(WideQuad), cudaMemcpyHostToDevice);
     }
+    if (ce != cudaSuccess) {
+        cudaFree(new_quads); cudaFree(new_wide);
+        return cuda_fail(ctx, ce, "plan tables (allocation or upload)");
+    }
+    cudaStreamSynchronize(ctx->stream);         // kernels of earlier calls may still read the old tables
+    cudaFree(ctx->d_quads); cudaFree(ctx->d_wide_quads);
+    ctx->d_quads = new_quads; ctx->d_wide_quads = new_wide;
     ctx->space = sp;
     ctx->inc_J = 0;
     ctx->has_space = true;
@@ -544,10 +554,15 @@ static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
     if ((rc = ensure(ctx, ctx->d_feas, ctx->cap_feas, size_t(J) * sp.P))) return rc;
     const size_t curve = size_t(J) * sp.nG * sp.nC * sp.nM;
     if (curve > ctx->cap_curve) {
+        // the three tables grow together; if one allocation fails none of them is kept, so that no later call
+        // (whose smaller J would skip this branch) can hand a freed or null table to a kernel
         size_t c1 = ctx->cap_curve, c2 = ctx->cap_curve, c3 = ctx->cap_curve;
-        if ((rc = ensure(ctx, ctx->d_cv, c1, curve))) return rc;
-        if ((rc = ensure(ctx, ctx->d_cp, c2, curve))) return rc;
-        if ((rc = ensure(ctx, ctx->d_cg, c3, curve))) return rc;
+        ctx->cap_curve = 0;
+        if ((rc = ensure(ctx, ctx->d_cv, c1, curve)) || (rc = ensure(ctx, ctx->d_cp, c2, curve)) || (rc = ensure(ctx, ctx->d_cg, c3, curve))) {
+            cudaFree(ctx->d_cv); cudaFree(ctx->d_cp); cudaFree(ctx->d_cg);
+            ctx->d_cv = nullptr; ctx->d_cp = nullptr; ctx->d_cg = nullptr;
+            return rc;
+        }
         ctx->cap_curve = curve;
     }
     // a round only needs the curves: the one-pass kernel never writes the candidate table
@@ -656,11 +671,13 @@ int rubick_incremental_event_host(rubick_ctx *ctx, const rubick_job *h_jobs, int
                                            h_reconf ? ctx->d_inc_reconf : nullptr, theta, ctx->d_inc_state[nxt], ctx->d_inc_nodes[nxt],
                                            nullptr, ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream),
              "launch incremental_round");
+    // the status first: a round that was refused has written no result, and the caller's buffers stay as they are
+    rc = finish_round(ctx, h_steps);
+    if (rc != RUBICK_OK && rc != RUBICK_ESTEPS) { ctx->inc_J = 0; return rc; }
+    ctx->inc_cur = nxt; ctx->inc_J = J; ctx->inc_N = N;
     CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_inc_state[nxt], size_t(J) * sizeof(rubick_assignment), cudaMemcpyDeviceToHost, ctx->stream), "copy assignments to host");
     if (h_node_out) CUDA_TRY(ctx, cudaMemcpyAsync(h_node_out, ctx->d_inc_nodes[nxt], size_t(N) * sizeof(rubick_node), cudaMemcpyDeviceToHost, ctx->stream), "copy node states to host");
-    rc = finish_round(ctx, h_steps);
-    if (rc == RUBICK_OK || rc == RUBICK_ESTEPS) { ctx->inc_cur = nxt; ctx->inc_J = J; ctx->inc_N = N; }
-    else ctx->inc_J = 0;
+    CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream), "cudaStreamSynchronize");
     return rc;
 }
 

@@ -14,7 +14,7 @@
 // Model (paper Section 4):  THROUGHPUT = b / T_iter,  T_iter = T_cc + T_oo + k_const  (Eq. 1)
 //   T_fwd  = tau * mu / (t p) * (m + p - 1 if p > 1)                       forward, pipeline bubble
 //   T_bwd  = k_bwd T_fwd (+ T_fwd under gradient checkpointing)
-//   T_comm = V / B per dimension, V = 0 at degree 1;  V_dp ring all-reduce of the shard,
+//   T_comm = V / B per dimension, V = 0 at degree 1;  V_dp ring all-reduce of the shard (every ZeRO stage),
 //            V_tp four all-reduces per layer, V_pp stage boundaries of 1F1B
 //   T_cc   = a T_fwd + (a - 1) T_bwd + f^{k_sync}(T_bwd, T_dp) + T_tp + T_pp
 //   T_oo   = T_opt, or under ZeRO-Offload f^{k_off}(T_dp, T_off) + f^{k_swap}(T_opt(c), T_off)
@@ -157,7 +157,7 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
     float T_dp = 0.0f, T_tp = 0.0f, T_pp = 0.0f;
     if (d > 1) {
         float V = sp.e * Pf * (WIDE ? 2.0f * float(d - 1) / float(g) : float(d - 1) * pow2_neg(lg - 1));
-        if (z == 3) V *= 1.5f;
+        if (z == 3) V *= sp.z3_volume;                   // 1 unless the environment asks for stage 3's parameter gathers
         T_dp = V * ((qflags & QF_DP_INTER) ? sp.inv_B_inter : sp.inv_B_intra);
     }
     if (t > 1) T_tp = sp.e * 8.0f * float(t - 1) * bsh * float(jb.l) * inv_dt * sp.inv_B_intra;

@@ -29,6 +29,7 @@ constexpr double FIT_EPS = 1e-9;
 
 struct FitEnv {
     double B_intra, B_inter, B_pcie, e;
+    double z3_volume;                 // factor on V_dp for ZeRO stage 3 (1 = Section 4.1's rule)
     int Gn, strict;
 };
 
@@ -71,7 +72,7 @@ __device__ double model_thr(const rubick_job &jb, const double *th, const FitEnv
     const double T_bwd = th[0] * T_fwd + (gc ? T_fwd : 0.0);
 
     double V_dp = 0.0, V_tp = 0.0, V_pp = 0.0;
-    if (d > 1) V_dp = ev.e * P * 2.0 * (dd - 1.0) / (dd * tt * pp) * (z == 3 ? 1.5 : 1.0);
+    if (d > 1) V_dp = ev.e * P * 2.0 * (dd - 1.0) / (dd * tt * pp) * (z == 3 ? ev.z3_volume : 1.0);
     if (t > 1) V_tp = ev.e * 4.0 * 2.0 * (tt - 1.0) * bb * s * hh * ll / (dd * tt);
     if (p > 1) V_pp = ev.e * 2.0 * pp * bb * s * hh / (dd * tt);
     const double B_dp = (dd * tt <= double(ev.Gn)) ? ev.B_intra : ev.B_inter;
@@ -205,7 +206,7 @@ cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, const Wid
     if (J == 0) return cudaSuccess;
     FitEnv ev;
     ev.B_intra = env.B_intra; ev.B_inter = env.B_inter; ev.B_pcie = env.B_pcie; ev.e = double(env.bytes_per_elem);
-    ev.Gn = env.gpus_per_node; ev.strict = env.strict_zero_dp_only ? 1 : 0;
+    ev.Gn = env.gpus_per_node; ev.strict = env.strict_zero_dp_only ? 1 : 0; ev.z3_volume = env.zero3_extra_volume ? 1.5 : 1.0;
     const int threads = 64, per_block = threads / 32;
     fit_models_kernel<<<(J + per_block - 1) / per_block, threads, 0, st>>>(ev, d_quads, d_wide_quads, P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle);
     return cudaGetLastError();

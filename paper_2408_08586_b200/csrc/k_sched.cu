@@ -20,6 +20,7 @@
 //                  (GetBestPlan), memory of that plan (AllocMem), node bookkeeping, new gains.
 // The step count is bounded by max_steps; hitting it sets a status bit instead of spinning.
 
+#include <atomic>
 #include "round_plain.cuh"
 
 namespace rubick {
@@ -360,9 +361,12 @@ constexpr size_t NOALLOC_STATE_BYTES = size_t(RUBICK_NOALLOC_MAX_JOBS) * (sizeof
 static __device__ __align__(256) unsigned char g_noalloc_state[NOALLOC_STATE_BYTES];
 
 // In host code `g_noalloc_state` is only a handle; the device address has to be asked for, once
-// per device, with that device current.
+// per device, with that device current.  The answer is kept for the life of the process (atomic: two
+// host threads making their first call on a device both store the same address).  It refers to the
+// device's primary context: after a cudaDeviceReset of that device the stored address is stale, so a
+// process that resets a device must not call this entry point on it afterwards.
 constexpr int NOALLOC_MAX_DEVICES = 64;
-static void *g_noalloc_addr[NOALLOC_MAX_DEVICES];
+static std::atomic<void *> g_noalloc_addr[NOALLOC_MAX_DEVICES];
 
 }  // namespace rubick
 
@@ -391,13 +395,13 @@ extern "C" int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_
 
     cudaError_t e = cudaSetDevice(ctx->device);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaSetDevice");
-    if (!g_noalloc_addr[ctx->device]) {          // first call on this device: resolve the array's device address
-        void *p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_noalloc_state);
-        if (e != cudaSuccess || !p) return cuda_fail(ctx, e, "cudaGetSymbolAddress (fixed round state)");
-        g_noalloc_addr[ctx->device] = p;
+    void *addr = g_noalloc_addr[ctx->device].load(std::memory_order_acquire);
+    if (!addr) {                                 // first call on this device: resolve the array's device address
+        e = cudaGetSymbolAddress(&addr, g_noalloc_state);
+        if (e != cudaSuccess || !addr) return cuda_fail(ctx, e, "cudaGetSymbolAddress (fixed round state)");
+        g_noalloc_addr[ctx->device].store(addr, std::memory_order_release);
     }
-    unsigned char *base = static_cast<unsigned char *>(g_noalloc_addr[ctx->device]);
+    unsigned char *base = static_cast<unsigned char *>(addr);
     HotA *ha = reinterpret_cast<HotA *>(base);
     HotB *hb = reinterpret_cast<HotB *>(base + size_t(RUBICK_NOALLOC_MAX_JOBS) * sizeof(HotA));
 

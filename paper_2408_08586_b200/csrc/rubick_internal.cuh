@@ -37,6 +37,7 @@ struct Space {
     int32_t nG, nC, nM;
     int32_t Gn, log2Gn, Cn;
     int32_t strict;
+    float z3_volume;              // factor on V_dp for ZeRO stage 3: 1 (Section 4.1's rule) or 1.5 (option)
     int32_t wide;                 // plans with degrees of any size (wide quad table) instead of powers of two
     int32_t n_small;              // number of GPU levels <= Gn (they come first)
     float e;                      // bytes per element

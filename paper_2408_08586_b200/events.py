@@ -17,11 +17,13 @@ from . import binding as rb
 from . import workloads
 
 
-def run_events(ctx, cfg, n_events=1000, warm_jobs=1500, max_steps=1 << 30, sync=None):
+def run_events(ctx, cfg, n_events=1000, warm_jobs=1500, max_steps=1 << 30, sync=None, on_round=None):
     """Replays n_events scheduling events.  -> dict(latency_ms [n_events], active [n_events], steps [n_events]).
 
     cfg: a workload dict whose jobs are the pool arrivals are drawn from, in order; the first
     `warm_jobs` of them are already in the system at time 0 so that rounds start at a realistic size.
+    on_round(event, pool_indices, h_jobs, h_out, h_nodes, steps), if given, sees every round's inputs and results
+    (outside the timed part); the node states are only fetched when it is given.
     """
     jobs = cfg["jobs"]
     pool = len(jobs["P"])
@@ -37,19 +39,22 @@ def run_events(ctx, cfg, n_events=1000, warm_jobs=1500, max_steps=1 << 30, sync=
     next_arrival = warm
     now = 0.0
     h_out = np.zeros(pool, dtype=rb.ASSIGN_DTYPE)
+    h_nodes = np.zeros(N, dtype=rb.NODE_DTYPE) if on_round is not None else None
     lat, act, stp = [], [], []
-    for _ in range(n_events):
+    for ev in range(n_events):
         if not active and next_arrival >= pool:
             break
         idx = np.asarray(active, dtype=np.int64)
         h_jobs = np.ascontiguousarray(records[idx])
         t0 = time.perf_counter()
-        steps, _ = ctx.schedule_round_host(h_jobs, len(idx), N, max_steps, h_out[: len(idx)])
+        steps, _ = ctx.schedule_round_host(h_jobs, len(idx), N, max_steps, h_out[: len(idx)], h_nodes)
         if sync is not None:
             sync()
         lat.append(1e3 * (time.perf_counter() - t0))
         act.append(len(idx))
         stp.append(steps)
+        if on_round is not None:
+            on_round(ev, idx, h_jobs, h_out[: len(idx)], h_nodes, steps)
         # advance to the next event: the earliest completion or the next arrival
         rate = w[idx] * h_out["thr"][: len(idx)].astype(np.float64)
         with np.errstate(divide="ignore", invalid="ignore"):
@@ -72,11 +77,12 @@ def run_events(ctx, cfg, n_events=1000, warm_jobs=1500, max_steps=1 << 30, sync=
     return dict(latency_ms=np.asarray(lat), active=np.asarray(act), steps=np.asarray(stp))
 
 
-def run_events_incremental(ctx, cfg, n_events=1000, warm_jobs=1500, slots=4096, theta=0.97, max_steps=1 << 30):
+def run_events_incremental(ctx, cfg, n_events=1000, warm_jobs=1500, slots=4096, theta=0.97, max_steps=1 << 30, on_round=None):
     """The same event stream through ``rubick_incremental_event_host``: jobs live in `slots` fixed slots,
     the previous allocation and the curve tables stay on the device, and an event uploads only the slot
     that changed.  A job's checkpoint-resume cost is ``workloads.reconf_cost``; its trained time T and
-    reconfiguration count feed the gate of Section 5.2.
+    reconfiguration count feed the gate of Section 5.2.  on_round(event, slot_job, h_jobs, reconf, changed, h_out,
+    h_nodes, steps), if given, sees every round's inputs and results (outside the timed part).
     -> dict(latency_ms, active, steps, reconfigured [n_events])."""
     jobs = cfg["jobs"]
     pool = len(jobs["P"])
@@ -102,17 +108,20 @@ def run_events_incremental(ctx, cfg, n_events=1000, warm_jobs=1500, slots=4096, 
     next_arrival = warm
     now = 0.0
     changed = None                                          # first event: everything is new
+    h_nodes = np.zeros(N, dtype=rb.NODE_DTYPE) if on_round is not None else None
     lat, act, stp, rec = [], [], [], []
-    for _ in range(n_events):
+    for ev in range(n_events):
         live = np.nonzero(slot_job >= 0)[0]
         if len(live) == 0 and next_arrival >= pool:
             break
         t0 = time.perf_counter()
         steps, _ = ctx.incremental_event_host(h_jobs, slots, N, h_out, changed=changed, h_reconf=reconf, theta=theta,
-                                              restart=changed is None, max_steps=max_steps)
+                                              restart=changed is None, max_steps=max_steps, h_node_out=h_nodes)
         lat.append(1e3 * (time.perf_counter() - t0))
         act.append(len(live))
         stp.append(steps)
+        if on_round is not None:
+            on_round(ev, slot_job, h_jobs, reconf, changed, h_out, h_nodes, steps)
         was = (prev["status"] == rb.RUNNING) & (slot_job >= 0)
         moved = was & (h_out["status"] == rb.RUNNING) & ((h_out["g"] != prev["g"]) | (h_out["c"] != prev["c"]) | (h_out["plan"] != prev["plan"]))
         reconf["n_reconf"] += moved.astype(np.int32)

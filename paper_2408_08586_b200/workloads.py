@@ -24,7 +24,7 @@ HOST_BASE = 4 * GIB                          # host bytes per training process
 
 ENV = dict(B_intra=400e9, B_inter=100e9, B_pcie=25e9, gpu_mem_bytes=80_000_000_000,
            gpus_per_node=8, cpus_per_node=96, mem_per_node_bytes=1024 * GIB, bytes_per_elem=2,
-           strict_zero_dp_only=0)
+           strict_zero_dp_only=0, zero3_extra_volume=0)
 
 CONFIGS = {
     # name: (seed, jobs, nodes, g levels, c levels, m levels [GiB], largest parameter count)

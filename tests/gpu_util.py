@@ -152,3 +152,83 @@ def assert_rounds_equal(a, b):
     assert a["steps"] == b["steps"] and a["capped"] == b["capped"]
     if a["log"] is not None and b["log"] is not None:
         assert np.array_equal(a["log"], b["log"])
+
+
+def assert_chain_parity(gpu, cfg, n_nodes, oracle_chain, got=None, tie_rtol=1e-6, thr_rtol=1e-5):
+    """The library's whole chain (its own single-precision table -> curves -> round) against the oracle's chain
+    (double-precision table rounded once -> curves -> round).  The two tables differ by rounding, so:
+      - masks are equal, curve values agree to thr_rtol, and the largest relative difference seen is `tol`;
+      - the step logs are identical up to the first decision that the oracle takes by a margin within what
+        `tol` can move (near_tie.assert_divergence_is_a_near_tie); up to there both sides hold the same GPUs
+        and cores on the same nodes, and plans differ only where the oracle rates the library's plan within
+        tie_rtol of its own;
+      - without such a near tie the two rounds are the same round.
+    oracle_chain = (plans, thr float64 [J, C, P], feas, cv float32, cp, cg) from the oracle; got (optional): the
+    result of the one-call path (rubick_schedule_round*), which must equal the logged round bit for bit.
+    Returns the description of the near tie, or None."""
+    import near_tie
+    import oracle
+    jobs = cfg["jobs"]
+    J = len(jobs["P"])
+    plans, thr, feas, cv, cp, cg = oracle_chain
+    d_jobs, d_thr, d_feas = gpu.eval(jobs)
+    bv, bp, bg = gpu.best(d_thr, d_feas, J)
+    sh = gpu.shape4(J)
+    gcv, gcp, gcg = bv.cpu().numpy().reshape(sh), bp.cpu().numpy().reshape(sh), bg.cpu().numpy().reshape(sh)
+    gfeas = gpu.np_feas(d_feas, J)
+    assert np.array_equal(gfeas, feas)
+    has = cv > 0
+    assert np.array_equal(gcv > 0, has)
+    tol = float((np.abs(gcv[has].astype(np.float64) - cv[has]) / cv[has]).max()) if has.any() else 0.0
+    assert tol <= thr_rtol, tol
+    logged = gpu.round_on_tables(jobs, gcv, gcp, gcg, gfeas, n_nodes)
+    if got is not None:
+        assert_rounds_equal(got, logged)
+    args = (jobs, cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"], n_nodes)
+    want = oracle.schedule_round(*args, want_log=True)
+    found = near_tie.assert_divergence_is_a_near_tie(
+        lambda k: oracle.schedule_round(*args, max_steps=k, want_log=True, want_candidates=True), want["log"], logged["log"],
+        jobs["w"], tol, lambda j, gi, ci, mi: gcp[j, gi, ci, mi] != cp[j, gi, ci, mi] or gcg[j, gi, ci, mi] != cg[j, gi, ci, mi])
+    if found is not None:
+        k = near_tie.first_difference(want["log"], logged["log"])
+        want = oracle.schedule_round(*args, max_steps=k, want_log=True)
+        logged = gpu.round_on_tables(jobs, gcv, gcp, gcg, gfeas, n_nodes, max_steps=k)
+        assert np.array_equal(want["log"], logged["log"])
+    for key in ("g", "c", "status", "first_node", "n_nodes"):
+        assert np.array_equal(want[key], logged[key]), key
+    assert np.array_equal(want["node"][:, [0, 1, 3]], logged["node"][:, [0, 1, 3]])
+    run = want["status"] == rb.RUNNING
+    assert np.allclose(logged["thr"][run], want["thr"][run], rtol=thr_rtol, atol=0)
+    other = np.nonzero(want["plan"] != logged["plan"])[0]
+    if len(other):
+        # another plan only where the oracle rates it as good as its own choice
+        ci = np.searchsorted(cfg["c_levels"], want["c"][other])
+        assert np.all(thr[other, ci, logged["plan"][other]] >= want["thr"][other].astype(np.float64) * (1 - tie_rtol - 2.0 ** -23))
+        assert len(other) <= max(2, J // 50)
+    same = want["plan"] == logged["plan"]
+    assert np.array_equal(want["m_bytes"][same], logged["m_bytes"][same])
+    if not len(other):
+        assert np.array_equal(want["node"], logged["node"])
+    return found
+
+
+def jobs_from_records(rec):
+    """JOB_DTYPE records -> the dict of per-job arrays the generators produce (exact: every field is a double,
+    an integer or a single-precision value)."""
+    return {k: np.asarray(rec[k], dtype=np.float64 if rec.dtype[k].kind == "f" else np.int64)
+            for k in rec.dtype.names if k not in ("flags", "pad")}
+
+
+def curves_of(gpu, records):
+    """The library's own mask and curve tables of the given job records (rubick_curves, the kernel the
+    scheduling entry points use) -> (cv [J, G, C, M] float32, cp, cg int32, feas [J, P] uint32)."""
+    t = gpu.torch
+    J = len(records)
+    n = J * gpu.nG * gpu.nC * gpu.nM
+    d_jobs = rb.to_device(records)
+    d_feas = gpu.empty(J * gpu.P, t.int32)
+    cv, cp, cg = gpu.empty(n, t.float32), gpu.empty(n, t.int32), gpu.empty(n, t.int32)
+    gpu.ctx.curves(d_jobs, J, d_feas, cv, cp, cg)
+    gpu.ctx.sync()
+    sh = gpu.shape4(J)
+    return cv.cpu().numpy().reshape(sh), cp.cpu().numpy().reshape(sh), cg.cpu().numpy().reshape(sh), gpu.np_feas(d_feas, J)

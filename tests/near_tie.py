@@ -77,9 +77,8 @@ def assert_divergence_is_a_near_tie(run_oracle, log_o, log_x, w, tol, entries_di
         # same increment, accepted by one chain only: the test v' > v at the commit level, or an entry the tables resolve differently
         vc, vcur = cand["v_commit"][jo, to], cand["v_cur"][jo, to]
         close = abs(vc - vcur) <= (tol + ARITH) * max(vc, vcur)
-        gi = int(cand["next"][jo, 0]) if to == 0 else -1
-        ci = int(cand["next"][jo, 1]) if to == 1 else -1
-        other = entries_differ is not None and entries_differ(jo, gi, ci, int(cand["m_commit"][jo, to]))
+        other = entries_differ is not None and cand["m_commit"][jo, to] >= 0 and entries_differ(
+            jo, int(cand["gi"][jo, to]), int(cand["ci"][jo, to]), int(cand["m_commit"][jo, to]))
         assert close or other, f"step {k}: job {jo} accepted by one chain only, with values {vc!r} against {vcur!r}"
         return f"step {k}: increment of job {jo} accepted by one chain only; deciding values within {tol + ARITH:.2g}"
     if to != tx:

@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 import oracle
-from gpu_util import Gpu, assert_rounds_equal, has_cuda, unpack_round
+from gpu_util import Gpu, assert_rounds_equal, curves_of, has_cuda, jobs_from_records, unpack_round
 from paper_2408_08586_b200 import binding as rb
 from paper_2408_08586_b200 import workloads
 
@@ -106,6 +106,104 @@ def test_round_at_full_size_is_a_valid_packing_and_both_kernels_agree(full):
     cv = d_cv.view(J, gpu.nG, gpu.nC, gpu.nM).cpu().numpy()
     gi = np.searchsorted(cfg["g_levels"], r["g"][run]); ci = np.searchsorted(cfg["c_levels"], r["c"][run])
     assert np.all(r["thr"][run] <= cv[np.nonzero(run)[0], gi, ci, -1]) and np.all(r["thr"][run] > 0)
+
+
+def test_round_at_full_size_matches_the_oracle_bit_for_bit(full):
+    """16,384 jobs on 512 nodes: the oracle's round on the library's own curve tables, step by step.  Every
+    decision of a round is an integer, so allocations, plans, memory, node states, values and the whole step
+    log must be identical.  (About a minute of single-threaded oracle work.)"""
+    cfg, gpu, J, d_jobs, d_thr, d_feas, d_cv, d_cp, d_cg = full
+    t = gpu.torch
+    N = cfg["n_nodes"]
+    sh = gpu.shape4(J)
+    cv, cp, cg = d_cv.cpu().numpy().reshape(sh), d_cp.cpu().numpy().reshape(sh), d_cg.cpu().numpy().reshape(sh)
+    feas = gpu.np_feas(d_feas, J)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"], N,
+                                 want_log=True)
+    cap = J * (gpu.nG + gpu.nC + 2) + 1
+    d_out = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    d_node = t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    d_log = t.zeros(cap, dtype=t.int32, device="cuda:0")
+    steps, capped = gpu.ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, cap, d_out, d_node, d_log)
+    got = unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped,
+                       d_log.cpu().numpy()[:steps])
+    assert want["steps"] > 5000 and not want["capped"]
+    assert_rounds_equal(got, want)
+    # and without a step log (the launch configuration the benchmark times)
+    d_out2 = t.zeros_like(d_out)
+    d_node2 = t.zeros_like(d_node)
+    steps2, capped2 = gpu.ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, 1 << 30, d_out2, d_node2)
+    assert (steps2, capped2) == (steps, capped) and t.equal(d_out2, d_out) and t.equal(d_node2, d_node)
+
+
+def _replay_in_threads(work, n_threads=8):
+    """Runs the oracle over the recorded rounds in threads (ctypes releases the interpreter lock during the C
+    call) and returns its results in order."""
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=n_threads) as pool:
+        return list(pool.map(lambda f: f(), work))
+
+
+def test_event_stream_full_replans_match_the_oracle():
+    """The event-driven run at 512 nodes through rubick_schedule_round_host: at each of 100 events the oracle
+    replays the round on the library's own tables of that event's active jobs; assignments, node states and
+    step counts must be identical."""
+    from paper_2408_08586_b200 import events
+    cfg = workloads.make("events")
+    gpu = Gpu(cfg)
+    side = Gpu(cfg)                                       # a second context computes the tables to hand to the oracle
+    N = cfg["n_nodes"]
+    seen, work = [], []
+
+    def on_round(ev, idx, h_jobs, h_out, h_nodes, steps):
+        cv, cp, cg, feas = curves_of(side, h_jobs)
+        jobs = jobs_from_records(h_jobs)
+        seen.append(unpack_round(h_out.copy(), h_nodes.copy(), steps, False, None))
+        work.append(lambda: oracle.schedule_round(jobs, cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
+                                                  cfg["m_levels"], N))
+
+    r = events.run_events(gpu.ctx, cfg, n_events=100, warm_jobs=900, on_round=on_round)
+    assert len(seen) == 100 and r["active"].min() > 600
+    for got, want in zip(seen, _replay_in_threads(work)):
+        assert_rounds_equal(got, want)
+    assert sum((g["n_nodes"] > 1).any() for g in seen) > 50           # whole-node jobs are part of the stream
+
+
+def test_event_stream_incremental_rounds_match_the_oracle():
+    """The same stream through rubick_incremental_event_host (state and tables kept in the context, one slot
+    uploaded per event): the oracle's incremental round, chained on its own previous result and fed the
+    library's tables of the slots' jobs, must give the identical allocation at each of 120 events."""
+    from paper_2408_08586_b200 import events
+    cfg = workloads.make("events")
+    gpu = Gpu(cfg)
+    side = Gpu(cfg)
+    N, slots = cfg["n_nodes"], 1536
+    tabs = {}
+    state = dict(prev=None, checked=0, moved=0)
+
+    def on_round(ev, slot_job, h_jobs, reconf, changed, h_out, h_nodes, steps):
+        fresh = range(slots) if changed is None else changed
+        if len(fresh):
+            sel = np.asarray(list(fresh), dtype=np.int64)
+            cv, cp, cg, feas = curves_of(side, np.ascontiguousarray(h_jobs[sel]))
+            if changed is None:
+                tabs.update(cv=cv, cp=cp, cg=cg, feas=feas)
+            else:
+                tabs["cv"][sel], tabs["cp"][sel], tabs["cg"][sel], tabs["feas"][sel] = cv, cp, cg, feas
+        want = oracle.schedule_round_incremental(jobs_from_records(h_jobs), cfg["env"], tabs["cv"], tabs["cp"], tabs["cg"], tabs["feas"],
+                                                 cfg["g_levels"], cfg["c_levels"], cfg["m_levels"], N, state["prev"],
+                                                 active=reconf["active"], T=reconf["T"], delta=reconf["delta"],
+                                                 nrec=reconf["n_reconf"], theta=0.97)
+        got = unpack_round(h_out.copy(), h_nodes.copy(), steps, False, None)
+        assert want["steps"] is not None
+        assert_rounds_equal(got, want)
+        if state["prev"] is not None:
+            state["moved"] += int(((state["prev"]["status"] == 1) & (want["status"] == 1) & (state["prev"]["g"] != want["g"])).sum())
+        state["prev"] = want
+        state["checked"] += 1
+
+    r = events.run_events_incremental(gpu.ctx, cfg, n_events=120, warm_jobs=900, slots=slots, on_round=on_round)
+    assert state["checked"] == 120 and r["active"].min() > 600 and state["moved"] > 0
 
 
 @pytest.mark.parametrize("cap", [1, 31, 33, 127, 129, 700, 3001, 9000])

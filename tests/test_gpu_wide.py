@@ -5,7 +5,7 @@ import numpy as np
 import pytest
 
 import oracle
-from gpu_util import Gpu, assert_rounds_equal, has_cuda
+from gpu_util import Gpu, assert_chain_parity, assert_rounds_equal, has_cuda, unpack_round
 from helpers import GIB, env
 from paper_2408_08586_b200 import binding as rb
 from paper_2408_08586_b200 import workloads
@@ -77,12 +77,13 @@ def test_wide_plan_space_through_every_kernel(levels, gn, N, n_acc):
     got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, N)
     assert_rounds_equal(got, want)
     assert want["steps"] > 5
-    # the whole path on the library's own tables: allocations agree except after near ties of the two chains
+    # the whole path in one call on the library's own tables: the same round up to the first near tie of the two chains
     d_out = gpu.empty(J * rb.ASSIGN_DTYPE.itemsize, t.uint8)
-    steps, capped = gpu.ctx.schedule_round(gpu.jobs_to_device(cfg["jobs"]), J, N, 1 << 30, d_out)
-    out = rb.from_device(d_out, rb.ASSIGN_DTYPE)
-    agree = (out["g"] == want["g"]) & (out["c"] == want["c"]) & (out["plan"] == want["plan"])
-    assert agree.mean() >= 0.9 and not capped
+    d_node = gpu.empty(N * rb.NODE_DTYPE.itemsize, t.uint8)
+    steps, capped = gpu.ctx.schedule_round(gpu.jobs_to_device(cfg["jobs"]), J, N, 1 << 30, d_out, d_node)
+    one_call = unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped, None)
+    assert_chain_parity(gpu, cfg, N, (plans, thr, feas, cv, cp, cg), got=one_call)
+    assert not capped
 
 
 def test_wide_space_validation_and_limits():

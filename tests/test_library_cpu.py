@@ -39,7 +39,7 @@ def test_struct_sizes_match_the_header():
     assert rb.PLAN_DTYPE.itemsize == 8
     assert rb.ASSIGN_DTYPE.itemsize == 40 and rb.ASSIGN_DTYPE.fields["thr"][1] == 28
     assert rb.NODE_DTYPE.itemsize == 24
-    assert C.sizeof(rb.Env) == 56 and C.sizeof(rb.Grid) == 40 and C.sizeof(rb.Cluster) == 24
+    assert C.sizeof(rb.Env) == 64 and C.sizeof(rb.Grid) == 40 and C.sizeof(rb.Cluster) == 24
     assert rb.JOB_DTYPE.fields["tenant"][1] == 88
 
 

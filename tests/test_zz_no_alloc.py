@@ -52,6 +52,34 @@ def test_noalloc_round_matches_the_ordinary_round_twice_in_a_row():
     assert not np.array_equal(want2["g"], want["g"][:len(want2["g"])])
 
 
+def test_noalloc_round_leaves_device_memory_as_it_found_it():
+    """What the entry point is for: in a fresh context, with 9,000 jobs (a count at which the ordinary entry point
+    has to grow its context's scratch with cudaMalloc), the call must not change the amount of free device memory
+    as the driver reports it, while the ordinary call on a fresh context does."""
+    cfg = workloads.make("throughput-stress", J=9000, n_nodes=48)
+    J, N = 9000, 48
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    d_jobs, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    d_cv, d_cp, d_cg = gpu.best(d_thr, d_feas, J)
+    d_out = t.zeros(J * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    d_node = t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    warm = Gpu(workloads.make("tiny"))                    # the library's kernels are loaded before anything is measured
+    tiny_out = t.zeros(4 * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    tj, tt, tf = warm.eval(warm.cfg["jobs"])
+    tv, tp, tg = warm.best(tt, tf, 4)
+    warm.ctx.greedy_round_noalloc(tj, 4, tv, tp, tg, tf, 1, 100, tiny_out)
+    warm.ctx.greedy_round(tj, 4, tv, tp, tg, tf, 1, 100, tiny_out)
+    t.cuda.synchronize()
+    free0 = t.cuda.mem_get_info()[0]
+    gpu.ctx.greedy_round_noalloc(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, 1 << 30, d_out, d_node)
+    t.cuda.synchronize()
+    assert t.cuda.mem_get_info()[0] == free0
+    gpu.ctx.greedy_round(d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, 1 << 30, d_out, d_node)
+    t.cuda.synchronize()
+    assert t.cuda.mem_get_info()[0] < free0               # the ordinary round allocated its scratch
+
+
 def test_noalloc_round_covers_job_counts_beyond_shared_memory_and_rejects_too_many():
     # 9000 jobs: the ordinary entry point moves the job state to allocated scratch here
     cfg = workloads.make("throughput-stress", J=9000, n_nodes=48)
