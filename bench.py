@@ -32,12 +32,24 @@ from paper_2408_08586_b200 import workloads  # noqa: E402
 
 METRIC = "candidate_evals_per_sec"
 UNIT = "stored candidate evaluations/s (job x plan x cpu-level; host-memory levels resolved by mask bits)"
+UNIT_E2E = "candidate evaluations/s (job x plan x cpu-level; evaluated inside the one-pass curves kernel, not stored)"
 FALLBACK_HBM_GBS = 6650.0
 
 # DRAM traffic of one eval_candidates launch from an ncu capture (dram__bytes_read.sum +
-# dram__bytes_write.sum), as bytes per stored candidate; valid only for the kernel source it was
-# taken on (sha1 of k_eval.cu), otherwise reported as null.
-NCU_EVAL_TRAFFIC = {"k_eval_sha1": "782b20d6b0a3e6b89f7fd39fc5f12914d71aa5f6", "bytes_per_candidate": 483.89939e6 / (2048 * 2640 * 24)}
+# dram__bytes_write.sum) on `jobs` jobs, as bytes per stored candidate; valid only for the kernel source it
+# was taken on (sha1 of k_eval.cu), otherwise reported as null.
+NCU_EVAL_TRAFFIC = {"k_eval_sha1": None, "jobs": 0, "bytes_per_candidate": None}
+
+# Single-precision and transcendental-unit instructions of the evaluation code per (job, plan quad), counted from
+# eval_quad in k_eval.cu (power-of-two instance): what does not depend on the core count (forward / backward,
+# three communication times, two overlaps with the gradient ring, two divisions into throughputs, their reciprocals
+# of exponents), the offload prelude (transfer time, one overlap, two reciprocals) and, per core level, a quarter of a
+# swap overlap plus one reciprocal-multiply.  A division counts as 1 transcendental + 7 single-precision instructions,
+# an overlap f^k as 5 + 5.
+def eval_quad_ops(C):
+    fp32 = 68 + 24 + 3.5 * C
+    xu = 13 + 7 + 2.25 * C
+    return fp32, xu
 
 
 def shard_seed_offset(rank):
@@ -66,12 +78,7 @@ def reduce_sum(x, world):
 
 
 def make_workload(name, rank=0, J=None, n_nodes=None):
-    base = workloads.CONFIGS[name]["seed"]
-    workloads.CONFIGS[name]["seed"] = base + shard_seed_offset(rank)
-    try:
-        return workloads.make(name, J=J, n_nodes=n_nodes)
-    finally:
-        workloads.CONFIGS[name]["seed"] = base
+    return workloads.make(name, J=J, n_nodes=n_nodes, seed=workloads.CONFIGS[name]["seed"] + shard_seed_offset(rank))
 
 
 def sort_launches(J, tile=2048):
@@ -155,16 +162,31 @@ class ClockSampler:
 
 
 def oracle_sample(cfg, J_sample, n_nodes, nthreads):
-    """One pass of the checker over the first J_sample jobs: table, curves, round -> (seconds, P)."""
+    """One pass of the checker over the first J_sample jobs: table, curves, round -> (seconds, P, seconds per stage).
+    The table and the curves run on `nthreads` threads (OpenMP over jobs); the round is sequential by nature and
+    always runs on one."""
     import oracle
     jobs = workloads.take(cfg["jobs"], slice(0, J_sample))
     t0 = time.perf_counter()
     plans, _ = oracle.enumerate_plans(cfg["g_levels"])
     thr, feas = oracle.eval_candidates(jobs, plans, cfg["env"], cfg["c_levels"], cfg["m_levels"], nthreads=nthreads)
+    t1 = time.perf_counter()
     cv, cp, cg = oracle.best_plan(thr.astype(np.float32), feas, plans, cfg["g_levels"], len(cfg["m_levels"]), nthreads=nthreads)
+    t2 = time.perf_counter()
     oracle.schedule_round(jobs, cfg["env"], cv.astype(np.float32), cp, cg, feas, cfg["g_levels"], cfg["c_levels"],
                           cfg["m_levels"], n_nodes)
-    return time.perf_counter() - t0, len(plans)
+    t3 = time.perf_counter()
+    return t3 - t0, len(plans), {"table": t1 - t0, "curves": t2 - t1, "round": t3 - t2}
+
+
+def baseline_record(cfg, J_s, nodes_s, threads, J_full):
+    dt, P, stages = oracle_sample(cfg, J_s, nodes_s, threads)
+    C = len(cfg["c_levels"])
+    return {"value": J_s * P * C / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "cores_per_stage": {"table": threads, "curves": threads, "round": 1},
+            "stages_s": {k: round(v, 3) for k, v in stages.items()},
+            "sample": f"first {J_s} of {J_full} jobs on {nodes_s} nodes, one pass: table + curves + greedy round ({dt:.1f} s); "
+                      "the round's cost grows faster than the job count, so the figure depends on the sample size"}
 
 
 def run_reference(args):
@@ -173,24 +195,30 @@ def run_reference(args):
         return
     cfg = make_workload(args.workload, J=args.jobs, n_nodes=args.nodes)
     J_full = len(cfg["jobs"]["P"])
-    J_s = min(J_full, args.ref_jobs)
+    threads = max(1, args.ref_threads)                    # single thread unless asked otherwise: the primary baseline
+    J_s = min(J_full, args.ref_jobs if args.ref_jobs else (96 if threads == 1 else 1024))
     nodes = max(1, cfg["n_nodes"] * J_s // J_full)
-    threads = os.cpu_count() or 1
     for _ in range(args.warmup):
         oracle_sample(cfg, min(J_s, 16), nodes, threads)
     t = 0.0
     P = 0
+    stages = {"table": 0.0, "curves": 0.0, "round": 0.0}
     for _ in range(args.steps):
-        dt, P = oracle_sample(cfg, J_s, nodes, threads)
+        dt, P, st = oracle_sample(cfg, J_s, nodes, threads)
         t += dt
+        for k in stages:
+            stages[k] += st[k]
     C = len(cfg["c_levels"])
     value = J_s * P * C * args.steps / t
-    sample = f"first {J_s} of {J_full} jobs on {nodes} nodes per step: table + curves + greedy round"
+    sample = (f"first {J_s} of {J_full} jobs on {nodes} nodes per step: table + curves + greedy round; the round's cost grows "
+              "faster than the job count, so the figure depends on the sample size")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": args.workload, "jobs": J_s, "plans": P, "cpu_levels": C, "nodes": nodes},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample,
+                             "cores_per_stage": {"table": threads, "curves": threads, "round": 1},
+                             "stages_s_per_step": {k: round(v / args.steps, 4) for k, v in stages.items()}},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -205,9 +233,11 @@ def main():
     ap.add_argument("--workload", default="throughput-stress", choices=list(workloads.CONFIGS))
     ap.add_argument("--jobs", type=int, default=None, help="override the job count (small captures)")
     ap.add_argument("--nodes", type=int, default=None)
-    ap.add_argument("--ref-jobs", type=int, default=1024, help="jobs per step of the CPU arm / baseline sample")
+    ap.add_argument("--ref-jobs", type=int, default=0, help="jobs per step of the CPU arm (0: 96 on one thread, 1024 on several)")
+    ap.add_argument("--ref-threads", type=int, default=1, help="threads of the CPU arm's table and curve stages (the round always runs on one)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-probes", action="store_true", help="skip the machine probes and the curves-kernel roofline")
     ap.add_argument("--events", type=int, default=1000, help="scheduling events of the event-driven run (0 = skip)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -286,11 +316,13 @@ def main():
         step()
     barrier()
     marks = []
+    launches_before = rb.kernel_launches()
     t_start = ev()
     for _ in range(args.steps):
         step(marks)
     t_end = ev()
     barrier()
+    gpu_launches = rb.kernel_launches() - launches_before        # counted by the library at every launch site
     clocks = sampler.stop() if sampler else None
     total_ms = reduce_max_ms(t_start.elapsed_time(t_end), world)
     stage_ms = np.array([[m[i].elapsed_time(m[i + 1]) for i in range(4)] for m in marks]).mean(axis=0)
@@ -312,10 +344,67 @@ def main():
             ctx.schedule_round_host(hp_jobs, J, N, max_steps, hp_out, hp_node)
         torch.cuda.synchronize()
         e2e_ms = reduce_max_ms(1e3 * (time.perf_counter() - t0) / args.steps, world)
-        e2e = {"value": evals_all / (e2e_ms * 1e-3), "unit": UNIT, "ms_per_step": e2e_ms,
+        e2e = {"value": evals_all / (e2e_ms * 1e-3), "unit": UNIT_E2E, "ms_per_step": e2e_ms,
                "h2d_bytes_per_step": int(J * rb.JOB_DTYPE.itemsize),
                "d2h_bytes_per_step": int(J * rb.ASSIGN_DTYPE.itemsize + N * rb.NODE_DTYPE.itemsize),
                "call": "rubick_schedule_round_host: pinned job records in, assignments and node states out"}
+
+    # the one-pass curves kernel (what the scheduling entry points run) on the same jobs, and the machine probes its
+    # roofline is quoted against: write-only and read-only streams, FP32 and transcendental-unit rates (rank 0 only)
+    curves_roofline = None
+    probes = None
+    if rank == 0 and not args.no_probes:
+        for _ in range(2):
+            ctx.curves(d_jobs, J, d_feas, d_cv, d_cp, d_cg)
+        reps = max(3, min(args.steps, 20))
+        cs = ClockSampler(local)
+        time.sleep(0.3)
+        a = ev()
+        for _ in range(reps):
+            ctx.curves(d_jobs, J, d_feas, d_cv, d_cp, d_cg)
+        b = ev()
+        torch.cuda.synchronize()
+        curves_ms = a.elapsed_time(b) / reps
+        curves_clk = cs.stop()
+
+        def timed_probe(kind, buf, iters, reps_):
+            ctx.probe(kind, buf, iters)                            # warm-up launch
+            s = ClockSampler(local)
+            time.sleep(0.3)
+            a_ = ev()
+            work = 0.0
+            for _ in range(reps_):
+                work += ctx.probe(kind, buf, iters)
+            b_ = ev()
+            torch.cuda.synchronize()
+            clk = s.stop()
+            return work / (a_.elapsed_time(b_) * 1e-3), clk["sm_mhz"]
+
+        wr, _ = timed_probe(rb.PROBE_WRITE, d_thr, 1, 20)
+        rd, _ = timed_probe(rb.PROBE_READ, d_thr, 1, 20)
+        fma, fma_mhz = timed_probe(rb.PROBE_FMA, d_thr, 1 << 17, 8)
+        xu, xu_mhz = timed_probe(rb.PROBE_XU, d_thr, 1 << 15, 8)
+        probes = {"write_only_gbs": wr / 1e9, "read_only_gbs": rd / 1e9, "fp32_fma_per_s": fma, "fp32_sm_mhz": fma_mhz,
+                  "xu_ops_per_s": xu, "xu_sm_mhz": xu_mhz,
+                  "what": "rubick_probe micro-kernels timed with CUDA events: float4 streaming stores / loads over the 4 GB table buffer, "
+                          "register-resident FMA chains, lg2/ex2/rcp chains; SM clock = median of nvidia-smi samples during the probe"}
+        fp_q, xu_q = eval_quad_ops(C)
+        quads = float(J) * (P // 4)
+        run_mhz = curves_clk["sm_mhz"]
+        scale = (lambda probe_mhz: (run_mhz / probe_mhz) if run_mhz and probe_mhz else 1.0)
+        out_bytes = 4.0 * J * P + 12.0 * J * G * C * M + 128.0 * J
+        floors = {"xu": quads * xu_q / (xu * scale(xu_mhz)), "fp32": quads * fp_q / (fma * scale(fma_mhz)), "hbm_write": out_bytes / wr}
+        bound = max(floors, key=floors.get)
+        curves_roofline = {"kernel": "curves_kernel", "ms_per_launch": curves_ms, "sm_mhz": run_mhz,
+                           "bound": {"xu": "alu", "fp32": "alu", "hbm_write": "hbm"}[bound], "binding_floor": bound,
+                           "floors_ms": {k: 1e3 * v for k, v in floors.items()},
+                           "frac": floors[bound] / (curves_ms * 1e-3),
+                           "fp32_instr_per_evaluation": fp_q / (4.0 * C), "xu_instr_per_evaluation": xu_q / (4.0 * C),
+                           "bytes_written_per_launch": out_bytes,
+                           "evaluations_per_sec": float(J) * P * C / (curves_ms * 1e-3),
+                           "what": "time the busiest unit would need at its probed rate (transcendental unit, FP32 pipe at the clock of this run, "
+                                   "or the write stream of mask + curves) over the measured time; the kernel itself is bound by instruction issue "
+                                   "(integer feasibility arithmetic, selects and reductions), see profiles/"}
 
     # minimum demand of guaranteed jobs on the same tables (first widening row; rank 0 only)
     minres_ms = None
@@ -414,14 +503,15 @@ def main():
     if NCU_EVAL_TRAFFIC["k_eval_sha1"] == sha and NCU_EVAL_TRAFFIC["bytes_per_candidate"]:
         traffic = NCU_EVAL_TRAFFIC["bytes_per_candidate"] * float(J) * P * C
 
+    # the checker as it stands on this machine's host cores: one thread (the primary figure), then all cores for the
+    # two stages that have a parallel loop (the round is sequential and stays on one)
     cpu_baseline = None
     if not args.no_cpu_baseline:
+        J1 = min(J, 512)                                        # about twelve seconds on one core
+        cpu_baseline = baseline_record(cfg, J1, max(1, N * J1 // J), 1, J)
         threads = os.cpu_count() or 1
-        J_s = min(J, 8 * args.ref_jobs)                         # about ten seconds on all host cores
-        nodes_s = max(1, N * J_s // J)
-        dt, _ = oracle_sample(cfg, J_s, nodes_s, threads)
-        cpu_baseline = {"value": J_s * P * C / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
-                        "sample": f"first {J_s} of {J} jobs on {nodes_s} nodes, one pass: table + curves + greedy round ({dt:.1f} s)"}
+        J2 = min(J, 4096)                                       # a few seconds on all cores
+        cpu_baseline["threaded"] = baseline_record(cfg, J2, max(1, N * J2 // J), threads, J)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -433,18 +523,25 @@ def main():
                    "step": "eval_candidates + best_plan + marginal_gain + greedy_round"},
         "clocks": clocks,
         "e2e": e2e,
-        # eval, best_plan + its general-mask kernel, gain, prepare, keys, the sort's launches, round
-        "gpu_launches": (7 + sort_launches(J)) * args.steps,
+        # per step: eval, best_plan + its general-mask kernel, gain, prepare, keys, the sort's launches, round
+        "gpu_launches": int(gpu_launches),
         "roofline": {"kernel": "eval_candidates_kernel", "bound": "hbm", "achieved": eval_gbs, "peak": peak, "unit": "GB/s",
                      "frac": eval_gbs / peak, "traffic": traffic, "peak_source": peak_src,
                      "bytes_per_candidate": algorithmic_bytes_eval(J, P, C) / (float(J) * P * C),
-                     "ms_per_launch": float(stage_ms[0])},
+                     "ms_per_launch": float(stage_ms[0]),
+                     "frac_of_write_only_probe": (eval_gbs / probes["write_only_gbs"]) if probes else None,
+                     "frac_of_8000_gbs_spec": eval_gbs / 8000.0,
+                     "traffic_source": (f"ncu capture on {NCU_EVAL_TRAFFIC['jobs']} jobs, scaled by the job count" if traffic else
+                                        "null: no capture of this kernel source")},
         "cpu_baseline": cpu_baseline,
         "stages_ms": {"eval_candidates": float(stage_ms[0]), "best_plan": float(stage_ms[1]),
                       "marginal_gain": float(stage_ms[2]), "greedy_round": float(stage_ms[3])},
         "eval_kernel_candidates_per_sec": float(J) * P * C / (stage_ms[0] * 1e-3),
         "logical_candidates_per_sec": value * M,
-        "best_plan_roofline": {"bound": "hbm", "achieved": best_gbs, "peak": peak, "unit": "GB/s", "frac": best_gbs / peak},
+        "best_plan_roofline": {"bound": "hbm", "achieved": best_gbs, "peak": peak, "unit": "GB/s", "frac": best_gbs / peak,
+                               "frac_of_read_only_probe": (best_gbs / probes["read_only_gbs"]) if probes else None},
+        "curves_roofline": curves_roofline,
+        "probes": probes,
         "events": events,
         "min_resources_ms": minres_ms,
         "fit": fit,

@@ -31,6 +31,7 @@
 #ifndef RUBICK_H
 #define RUBICK_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -384,6 +385,26 @@ int rubick_schedule_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, cons
  * (and node states, if h_node_out is not NULL) back.  h_jobs / h_out may be pageable or pinned. */
 int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J, const rubick_cluster *h_cluster,
                                int max_steps, rubick_assignment *h_out, rubick_node *h_node_out, int32_t *h_steps);
+
+/* ---- measurement aids (the paper has no counterpart) ------------------------------------------- */
+
+#define RUBICK_PROBE_WRITE 0   /* float4 streaming stores over d_buf:            work = bytes written        */
+#define RUBICK_PROBE_READ  1   /* float4 streaming loads over d_buf:             work = bytes read           */
+#define RUBICK_PROBE_FMA   2   /* single-precision fused multiply-adds in registers: work = FMAs issued      */
+#define RUBICK_PROBE_XU    3   /* lg2 / ex2 / rcp approximations in registers:   work = transcendental ops   */
+
+/* Enqueues ONE launch of a machine probe on the context's stream: a micro-kernel that measures the rate
+ * roofline fractions are quoted against on this GPU (a write-only and a read-only stream for the table
+ * kernels, FP32 and transcendental throughput for the one-pass curves kernel).  The caller times the
+ * launch with CUDA events on that stream.  d_buf: device scratch of `bytes` bytes (16-byte aligned, at
+ * least 4096; the streams cover all of it, the register probes write at most one word); iters: loop
+ * count of the register probes (ignored by the streams).  *h_work (optional) receives the amount of
+ * work the launch does, in the unit named above.  Errors: EINVAL, ECUDA. */
+int rubick_probe(rubick_ctx *ctx, int kind, void *d_buf, size_t bytes, int iters, double *h_work);
+
+/* Number of kernels this library has launched in this process so far (all contexts; every launch site
+ * counts itself).  The difference across a timed region is the number of launches inside it. */
+unsigned long long rubick_kernel_launches(void);
 
 #ifdef __cplusplus
 }

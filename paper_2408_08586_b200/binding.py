@@ -70,7 +70,7 @@ EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error"
            "rubick_set_space", "rubick_enumerate_plans_wide", "rubick_set_space_wide", "rubick_eval_candidates", "rubick_best_plan", "rubick_curves", "rubick_marginal_gain",
            "rubick_min_resources", "rubick_fit_models",
            "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
-           "rubick_schedule_round_host", "rubick_incremental_event_host"]
+           "rubick_schedule_round_host", "rubick_incremental_event_host", "rubick_probe", "rubick_kernel_launches"]
 
 _lib = None
 
@@ -114,8 +114,11 @@ def lib():
         L.rubick_schedule_round_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_incremental_event_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), vp, ip, vp, C.c_float, ip, ip, vp, vp,
                                                     C.POINTER(C.c_int32)]
+        L.rubick_probe.argtypes = [vp, ip, vp, C.c_size_t, ip, C.POINTER(C.c_double)]
+        L.rubick_kernel_launches.argtypes = []
+        L.rubick_kernel_launches.restype = C.c_ulonglong
         for name in EXPORTS:
-            if name not in ("rubick_destroy", "rubick_last_error"):
+            if name not in ("rubick_destroy", "rubick_last_error", "rubick_kernel_launches"):
                 getattr(L, name).restype = ip
         _lib = L
     return _lib
@@ -184,8 +187,24 @@ def from_device(t, dtype, shape=None):
     return a.reshape(shape) if shape is not None else a
 
 
+PROBE_WRITE, PROBE_READ, PROBE_FMA, PROBE_XU = 0, 1, 2, 3
+
+
+def kernel_launches():
+    """rubick_kernel_launches: kernels the library has launched in this process so far."""
+    return int(lib().rubick_kernel_launches())
+
+
 class Context:
     """Owns one rubick_ctx.  Methods carry the names of the C entry points they call."""
+
+    def probe(self, kind, d_buf, iters=1):
+        """rubick_probe: one launch of a machine probe on the context's stream -> the work it does
+        (bytes for the two streams, operations for the register probes)."""
+        work = C.c_double(0.0)
+        self._check(lib().rubick_probe(self._h, int(kind), _ptr(d_buf), int(d_buf.numel() * d_buf.element_size()), int(iters),
+                                       C.byref(work)))
+        return work.value
 
     def __init__(self, env, device=0, stream=None):
         e = Env(float(env["B_intra"]), float(env["B_inter"]), float(env["B_pcie"]), int(env["gpu_mem_bytes"]),

@@ -22,6 +22,9 @@ int cuda_fail(rubick_ctx *ctx, cudaError_t e, const char *what)
     if (ctx) {
         ctx->err = std::string(what) + ": " + cudaGetErrorString(e);
     }
+    // the runtime also remembers a failed call (a refused cudaMalloc, say) as its "last error"; take it out, or the
+    // next launch's own error check would report it
+    (void)cudaGetLastError();
     return e == cudaErrorMemoryAllocation ? RUBICK_ENOMEM : RUBICK_ECUDA;
 }
 

@@ -426,14 +426,14 @@ cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_f
     if (smem <= 200 * 1024) {
         e = cudaMemsetAsync(d_todo, 0, sizeof(int32_t), st);
         if (e != cudaSuccess) return e;
-        best_plan_kernel<<<J, warps * 32, smem, st>>>(sp, d_thr, d_feas, J, flags, d_best_val, d_best_plan, d_best_g, d_status, d_todo);
+        best_plan_kernel<<<J, warps * 32, smem, st>>>(sp, d_thr, d_feas, J, flags, d_best_val, d_best_plan, d_best_g, d_status, d_todo); count_launch();
     } else {
-        best_plan_todo_all_kernel<<<(J + 255) / 256, 256, 0, st>>>(d_todo, J);
+        best_plan_todo_all_kernel<<<(J + 255) / 256, 256, 0, st>>>(d_todo, J); count_launch();
     }
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int grid2 = J < 2 * num_sms ? J : 2 * num_sms;
-    best_plan_scattered_kernel<<<grid2, warps2 * 32, smem2, st>>>(sp, d_thr, d_feas, d_todo, flags, d_best_val, d_best_plan, d_best_g, d_status);
+    best_plan_scattered_kernel<<<grid2, warps2 * 32, smem2, st>>>(sp, d_thr, d_feas, d_todo, flags, d_best_val, d_best_plan, d_best_g, d_status); count_launch();
     return cudaGetLastError();
 }
 

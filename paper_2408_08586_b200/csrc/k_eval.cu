@@ -399,6 +399,7 @@ cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *
         curves_kernel<true><<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_wide_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
     else
         curves_kernel<false><<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -411,6 +412,7 @@ cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const void *d_
     const int64_t grid = (total + block - 1) / block;
     if (sp.wide) eval_candidates_kernel<true><<<unsigned(grid), block, 0, st>>>(sp, d_wide_quads, d_jobs, J, d_thr, d_feas);
     else eval_candidates_kernel<false><<<unsigned(grid), block, 0, st>>>(sp, d_quads, d_jobs, J, d_thr, d_feas);
+    count_launch();
     return cudaGetLastError();
 }
 

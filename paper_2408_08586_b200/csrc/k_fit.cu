@@ -208,7 +208,7 @@ cudaError_t launch_fit(const rubick_env &env, const QuadDesc *d_quads, const Wid
     ev.B_intra = env.B_intra; ev.B_inter = env.B_inter; ev.B_pcie = env.B_pcie; ev.e = double(env.bytes_per_elem);
     ev.Gn = env.gpus_per_node; ev.strict = env.strict_zero_dp_only ? 1 : 0; ev.z3_volume = env.zero3_extra_volume ? 1.5 : 1.0;
     const int threads = 64, per_block = threads / 32;
-    fit_models_kernel<<<(J + per_block - 1) / per_block, threads, 0, st>>>(ev, d_quads, d_wide_quads, P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle);
+    fit_models_kernel<<<(J + per_block - 1) / per_block, threads, 0, st>>>(ev, d_quads, d_wide_quads, P, d_jobs, J, d_samples, S, sweeps, d_theta, d_rmsle); count_launch();
     return cudaGetLastError();
 }
 

@@ -831,7 +831,7 @@ cudaError_t launch_round_incremental(const Space &sp, const rubick_job *d_jobs, 
     int32_t *lists = reinterpret_cast<int32_t *>(p);
     incremental_round_kernel<<<1, ROUND_THREADS, smem, st>>>(sp, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_prev,
                                                              d_prev_nodes, d_reconf, theta, d_out, d_node_out, d_step_log,
-                                                             ha, hb, roles, own, lists, d_quota, n_tenants, d_status, d_steps);
+                                                             ha, hb, roles, own, lists, d_quota, n_tenants, d_status, d_steps); count_launch();
     return cudaGetLastError();
 }
 

@@ -1391,17 +1391,19 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     if ((long long)max_steps > natural) max_steps = int(natural < 0x7fffffffLL ? natural : 0x7fffffffLL);
 
     Trans *tr = reinterpret_cast<Trans *>(base + L.off_tr);
-    round_prepare_kernel<<<J, 256, 0, st>>>(sp, d_jobs, d_cv, d_cp, d_cg, d_feas, hc, tr);
+    round_prepare_kernel<<<J, 256, 0, st>>>(sp, d_jobs, d_cv, d_cp, d_cg, d_feas, hc, tr); count_launch();
     round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa, d_out,
-                                                                reinterpret_cast<int32_t *>(base + L.off_isg));
+                                                                reinterpret_cast<int32_t *>(base + L.off_isg)); count_launch();
     {
         const int n = L.n_pad, tile = n < SORT_TILE ? n : SORT_TILE;
         // every stage up to the tile size, tile by tile; then stage by stage: wide strides in global memory, the rest in tiles
-        round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, 2, tile, n == tile, d_jobs, sw);
+        round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, 2, tile, n == tile, d_jobs, sw); count_launch();
         for (int k = tile << 1; k <= n; k <<= 1) {
-            for (int s = k >> 1; s >= tile; s >>= 1)
+            for (int s = k >> 1; s >= tile; s >>= 1) {
                 round_sort_pass_kernel<<<((n >> 1) + 255) / 256, 256, 0, st>>>(keys, n, k, s);
-            round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, k, k, k == n, d_jobs, sw);
+                count_launch();
+            }
+            round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, k, k, k == n, d_jobs, sw); count_launch();
         }
     }
     cudaError_t e;
@@ -1419,7 +1421,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     A.status = d_status; A.steps_out = d_steps;
     e = cudaFuncSetAttribute(greedy_round_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(SMEM_LIMIT));
     if (e != cudaSuccess) return e;
-    greedy_round_fast_kernel<<<1, RT, L.smem, st>>>(sp, A);
+    greedy_round_fast_kernel<<<1, RT, L.smem, st>>>(sp, A); count_launch();
     return cudaGetLastError();
 }
 

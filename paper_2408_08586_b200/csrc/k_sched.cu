@@ -47,7 +47,7 @@ cudaError_t launch_gain(const Space &sp, const rubick_job *d_jobs, int J, const 
 {
     if (J == 0) return cudaSuccess;
     marginal_gain_kernel<<<(J + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, d_curve_val, d_state, d_gain_gpu,
-                                                         d_gain_cpu, d_next_g, d_next_c);
+                                                         d_gain_cpu, d_next_g, d_next_c); count_launch();
     return cudaGetLastError();
 }
 
@@ -87,7 +87,7 @@ cudaError_t launch_min_resources(const Space &sp, const QuadDesc *d_quads, const
                                  float *d_baseline, cudaStream_t st)
 {
     if (J == 0) return cudaSuccess;
-    min_resources_kernel<<<(J + 127) / 128, 128, 0, st>>>(sp, d_quads, d_thr, d_feas, d_cv, J, d_req, d_gmin, d_cmin, d_baseline);
+    min_resources_kernel<<<(J + 127) / 128, 128, 0, st>>>(sp, d_quads, d_thr, d_feas, d_cv, J, d_req, d_gmin, d_cmin, d_baseline); count_launch();
     return cudaGetLastError();
 }
 
@@ -336,7 +336,7 @@ cudaError_t launch_round(const Space &sp, const rubick_job *d_jobs, int J, const
     HotB *hb = reinterpret_cast<HotB *>(reinterpret_cast<unsigned char *>(d_scratch) + size_t(J) * sizeof(HotA));
     greedy_round_kernel<<<1, ROUND_THREADS, smem, st>>>(sp, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out,
                                                         d_node_out, d_step_log, ha, hb, in_smem ? 1 : 0, d_quota, n_tenants,
-                                                        d_status, d_steps);
+                                                        d_status, d_steps); count_launch();
     return cudaGetLastError();
 }
 
@@ -413,7 +413,7 @@ extern "C" int rubick_greedy_round_noalloc(rubick_ctx *ctx, const rubick_job *d_
     // from an earlier call need no clearing
     greedy_round_kernel<<<1, ROUND_THREADS, smem, ctx->stream>>>(sp, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas,
                                                                  N, max_steps, d_out, d_node_out, nullptr, ha, hb, 0,
-                                                                 nullptr, 0, ctx->d_status, ctx->d_steps);
+                                                                 nullptr, 0, ctx->d_status, ctx->d_steps); count_launch();
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "launch greedy_round (fixed state)");
 

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
 #include <string>
 #include <vector>
 
@@ -56,6 +57,10 @@ enum : uint32_t {
     DS_STEP_CAP = 2u,
     DS_BAD_PREV = 4u,             // incremental round: the previous state does not fit the grid or the cluster
 };
+
+// kernels launched by this process so far (every launch site counts itself; read by rubick_kernel_launches)
+extern std::atomic<unsigned long long> g_kernel_launches;
+inline void count_launch(int n = 1) { g_kernel_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 bool round_fast_supported(const Space &sp, int J, int N);
 size_t round_fast_scratch_need(const Space &sp, int J, int N);

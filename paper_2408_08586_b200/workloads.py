@@ -86,13 +86,14 @@ def draw_requests(seed, J, g_levels, n_c_levels, n_m_levels, guaranteed_share=0.
     return dict(g_idx=g_idx, c_idx=c_idx, m_idx=m_idx, plan_rank=np.where(guaranteed, rank, -1.0))
 
 
-def make(name, J=None, n_nodes=None):
-    """Build a named configuration; J / n_nodes override the size (same seed, same recipe)."""
+def make(name, J=None, n_nodes=None, seed=None):
+    """Build a named configuration; J / n_nodes override the size and seed the configuration's seed (same recipe)."""
     cfg = CONFIGS[name]
-    rng = np.random.Generator(np.random.PCG64(cfg["seed"]))
+    seed = cfg["seed"] if seed is None else seed
+    rng = np.random.Generator(np.random.PCG64(seed))
     J = cfg["J"] if J is None else J
     jobs = draw_jobs(rng, J, cfg["g"], len(cfg["c"]), pmax=cfg["pmax"])
-    return dict(name=name, seed=cfg["seed"], jobs=jobs, env=dict(ENV),
+    return dict(name=name, seed=seed, jobs=jobs, env=dict(ENV),
                 g_levels=np.asarray(cfg["g"], dtype=np.int64),
                 c_levels=np.asarray(cfg["c"], dtype=np.int64),
                 m_levels=np.asarray(cfg["m"], dtype=np.int64) * GIB,

@@ -98,11 +98,12 @@ def test_sort_launch_count_follows_the_bitonic_network():
 def test_reference_arm_prints_one_json_line(capsys):
     import json
     import types
-    args = types.SimpleNamespace(workload="tiny", jobs=None, nodes=None, ref_jobs=4, warmup=1, steps=2, gpus=1)
+    args = types.SimpleNamespace(workload="tiny", jobs=None, nodes=None, ref_jobs=4, ref_threads=1, warmup=1, steps=2, gpus=1)
     os.environ.pop("RANK", None)
     bench.run_reference(args)
     line = json.loads(capsys.readouterr().out.strip())
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["cpu_baseline"]["cores"] == 1 and line["cpu_baseline"]["cores_per_stage"]["round"] == 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["metric"] == bench.METRIC
     os.environ["RANK"] = "1"
     try:
