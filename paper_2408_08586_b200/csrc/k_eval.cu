@@ -105,10 +105,17 @@ __device__ __forceinline__ int first_level(const Space &sp, int64_t need)
 // Returns the four feasibility words when KEEP_WORDS (zeros otherwise).
 // WIDE: degrees of any size from the wide quad table (divisions); otherwise powers of two from the
 // logarithms of the quad table (shifts, exact reciprocals).
-template <bool KEEP_WORDS, bool WIDE, class Emit>
+// LANE_PLANS: the caller wants no float4 per quad but the plans one by one, as the lanes compute them: head(out,
+// words, feasible) is called once with the two throughputs that do not depend on the core count (out.x, out.z), the
+// quad's four words and whether THIS LANE's offload plan -- ZeRO stage 2 + ((lane & 3) >> 1), checkpointing = lane & 1,
+// of the lane's (d, t, p) triple: plan index 4 * (first quad of the triple + 2 + ((lane & 3) >> 1)) + 1 + 2 * (lane & 1),
+// ascending with the lane -- may run at some memory level; then emit(ci, r) with that plan's throughput per core
+// level (0 when the plan is invalid; same bits as the float4 form).  emit is not called at all when no lane of the
+// warp holds a valid offload plan.
+template <bool KEEP_WORDS, bool WIDE, bool LANE_PLANS, class Head, class Emit>
 __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restrict__ quads_any,
                                            const rubick_job *__restrict__ jobs, int j, int q, bool active,
-                                           uint32_t *__restrict__ feas, Emit &&emit)
+                                           uint32_t *__restrict__ feas, Head &&head, Emit &&emit)
 {
     const JobRegs jb = load_job(jobs + j);
     int ld = 0, lt = 0, lp = 0, lg = 0, accum = 0, d, t, p, z, qflags, disabled;
@@ -220,11 +227,17 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
     // and the two lanes that own offload plans (stages 2 and 3) collect their pair.
     const bool off0 = valid_off && !(disabled & 2), off1 = valid_off && !(disabled & 8);
     const unsigned FULL = 0xffffffffu;
+    const int lane = threadIdx.x & 31, gbase = lane & ~3, zl = lane & 3;
+    if constexpr (LANE_PLANS) {
+        // may this lane's offload plan run at all?  its word sits with the lane that owns the quad
+        const uint32_t wy = __shfl_sync(FULL, fw_out.y, gbase + 2 + (zl >> 1)), ww = __shfl_sync(FULL, fw_out.w, gbase + 2 + (zl >> 1));
+        head(out, fw_out, ((zl & 1) ? ww : wy) != 0u);
+    }
     if (!__any_sync(FULL, off0 || off1)) {
-        for (int ci = 0; ci < sp.nC; ++ci) emit(ci, out, fw_out);
+        if constexpr (!LANE_PLANS)
+            for (int ci = 0; ci < sp.nC; ++ci) emit(ci, out, fw_out);
         return fw_out;
     }
-    const int lane = threadIdx.x & 31, gbase = lane & ~3, zl = lane & 3;
     const float T_off = sp.e * Psi * inv_d * sp.inv_B_pcie;          // identical on the four lanes
     const float opt_c = jb.k_opt_off * Psi * inv_d;                  // times 1 / c
     const float inv_kswap = 1.0f / jb.k_swap;
@@ -246,11 +259,15 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
         for (int cc = 0; cc < 4; ++cc) {
             const float fs = __shfl_sync(FULL, fs_mine, gbase + cc);
             const float r = my_ok ? bf * rcp_approx(my_base + fs) : 0.0f;
-            const float ry = __shfl_sync(FULL, r, src_y), rw = __shfl_sync(FULL, r, src_w);
-            if (c0 + cc < sp.nC) {
-                out.y = zl >= 2 ? ry : 0.0f;
-                out.w = zl >= 2 ? rw : 0.0f;
-                emit(c0 + cc, out, fw_out);
+            if constexpr (LANE_PLANS) {
+                if (c0 + cc < sp.nC) emit(c0 + cc, r);
+            } else {
+                const float ry = __shfl_sync(FULL, r, src_y), rw = __shfl_sync(FULL, r, src_w);
+                if (c0 + cc < sp.nC) {
+                    out.y = zl >= 2 ? ry : 0.0f;
+                    out.w = zl >= 2 ? rw : 0.0f;
+                    emit(c0 + cc, out, fw_out);
+                }
             }
         }
     }
@@ -274,7 +291,8 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const void *__restrict_
     const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
     float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
     // levels arrive in ascending order, one call each: the row pointer just advances
-    eval_quad<false, WIDE>(sp, quads, jobs, j, q, active, feas, [&](int, const float4 &out, const uint4 &) {
+    eval_quad<false, WIDE, false>(sp, quads, jobs, j, q, active, feas, [](const float4 &, const uint4 &, bool) {},
+                                  [&](int, const float4 &out, const uint4 &) {
         if (active) __stcs(reinterpret_cast<float4 *>(row), out);
         row += sp.P;
     });
@@ -283,18 +301,21 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const void *__restrict_
 // ------------------------------------------------------------------------------------------------------
 // Curves without the table: the evaluation above and the best-plan / sensitivity-curve step (paper
 // Section 5.2) in one kernel, for callers that only want the curves (a scheduling round).  One CTA per
-// job; thread = quad as above, but each level's four throughputs go into a reduction instead of memory:
-// per class (plans without / with offload, which share one first feasible memory level per GPU level under
-// this library's memory rule) the lanes of a warp that sit in the same GPU level reduce the value with one
-// warp reduction, a vote names the lowest lane holding it, and that lane folds (value bits << 32 | ~index)
-// into a 64-bit shared-memory maximum per (GPU level, core level); plans without offload do not depend on
-// the core count and are reduced once per GPU level.  Then thread (c, m) combines the two
-// classes for memory level m, takes the running maximum over GPU levels and stores its three outputs.
-// Same values, same ties (lowest plan index) as best_plan on the table of eval_candidates: bit-identical.
-// Nothing but the mask (4 bytes per plan) and the curves is written: the kernel is bound by the FP32 and
-// transcendental pipes instead of the table's write and read streams.
+// job; thread = quad as above, but nothing goes to memory: per class (plans without / with offload, which
+// share one first feasible memory level per GPU level under this library's memory rule) the lanes of a warp
+// that sit in the same GPU level reduce the value with one warp reduction, and a vote names the lowest lane
+// holding it.  Plans without offload do not depend on the core count and are reduced once per GPU level from
+// the quads' own two values; offload plans are reduced per core level straight from the lanes that computed
+// them (one plan per lane, plan index ascending with the lane, so the lowest lane holding the maximum holds
+// the lowest plan index).  The group's first lane folds (value bits << 32 | ~index) into a slot of its own warp
+// per (GPU level, core level) with a plain read-compare-write -- no atomics: a slot has one writer at a time, and
+// a warp synchronises between its passes over the quads.  After a CTA barrier the warps' slots are merged; then
+// thread (c, m) combines the two classes for memory level m, takes the running maximum over GPU levels and
+// stores its three outputs.  Same values, same ties (lowest plan index) as best_plan on the table of
+// eval_candidates: bit-identical.  Nothing but the mask (4 bytes per plan) and the curves is written.
 // ------------------------------------------------------------------------------------------------------
-constexpr int CURVES_THREADS = 128;      // small CTAs: the phases of the several CTAs of an SM overlap (704 threads: 2.4 ms, 128: 1.1 ms at 16,384 jobs)
+constexpr int CURVES_THREADS = 128;      // small CTAs: the phases of the several CTAs of an SM overlap
+constexpr int CURVES_WARPS = CURVES_THREADS / 32;
 
 template <bool WIDE>
 __global__ void __launch_bounds__(CURVES_THREADS)
@@ -303,13 +324,15 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
               float *__restrict__ best_val, int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    unsigned long long *keys = reinterpret_cast<unsigned long long *>(smem_raw);      // [nG][nC + 1]: offload class per core level, then the other class
+    // [warp][nG][nC + 1]: offload class per core level, then the other class; warp 0's copy receives the merge
+    unsigned long long *keys = reinterpret_cast<unsigned long long *>(smem_raw);
     __shared__ int s_first[2 * RUBICK_MAX_G_LEVELS];        // first feasible memory level per (GPU level, class), nM = none
     const int j = blockIdx.x;
-    const int tid = threadIdx.x, lane = tid & 31;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned FULL = 0xffffffffu;
+    const int per_warp = sp.nG * (sp.nC + 1);
 
-    for (int i = tid; i < sp.nG * (sp.nC + 1); i += blockDim.x) keys[i] = 0ull;
+    for (int i = tid; i < CURVES_WARPS * per_warp; i += blockDim.x) keys[i] = 0ull;
     if (tid < sp.nG) {
         // host-memory need of the level's plans: g processes, plus the offloaded states (as in the mask above)
         const rubick_job *jp = jobs + j;
@@ -323,6 +346,7 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
     }
     __syncthreads();
 
+    unsigned long long *mine = keys + size_t(warp) * per_warp;
     for (int q0 = 0; q0 < sp.Q; q0 += blockDim.x) {
         const int q_raw = q0 + tid;
         const bool active = q_raw < sp.Q;
@@ -330,32 +354,49 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
         const int q = active ? q_raw : sp.Q - 1;
         const int level = reinterpret_cast<const uint8_t *>(quads + q)[4];             // QuadDesc::g_level
         const unsigned peers = __match_any_sync(FULL, active ? level : -1);            // lanes of the same GPU level
-        unsigned long long *kq = keys + size_t(level) * (sp.nC + 1);
-        bool any_offload = false;                               // does a lane of my group own a feasible offloading plan?
-        eval_quad<true, WIDE>(sp, quads_any, jobs, j, q, active, feas, [&](int ci, const float4 &o, const uint4 &words) {
-            // Infeasible plans count as 0.  Quads ascend with the lane and a lane's two plans of a class with
-            // their index, so among equal values the lowest lane holds the lowest plan index: one warp
-            // reduction for the value, one vote for who holds it, and that lane alone updates the key.
-            if (ci == 0) {
-                // plans without offload do not depend on the core count: one entry per GPU level
+        const bool leader = active && lane == __ffs(peers) - 1;
+        const int q_lane0 = q_raw - lane;                       // quad of lane 0 (quads ascend with the lane)
+        unsigned long long *kq = mine + size_t(level) * (sp.nC + 1);
+        bool feasible = false;                                  // may this lane's offload plan run at some memory level?
+        eval_quad<true, WIDE, true>(sp, quads_any, jobs, j, q, active, feas,
+            [&](const float4 &o, const uint4 &words, bool lane_plan_feasible) {
+                // plans without offload: the quad's two values; infeasible plans count as 0.  Quads ascend with the
+                // lane and a quad's two plans with their index, so the lowest lane holding the maximum holds the
+                // lowest plan index.
+                feasible = active && lane_plan_feasible;
                 const float x = words.x ? o.x : 0.0f, z = words.z ? o.z : 0.0f;
                 const unsigned be = active ? __float_as_uint(fmaxf(x, z)) : 0u;
                 const unsigned me = __reduce_max_sync(peers, be);
                 const unsigned who = __ballot_sync(peers, be == me) & peers;
-                if (me && lane == __ffs(who) - 1)
-                    atomicMax(kq + sp.nC, (static_cast<unsigned long long>(me) << 32) | (FULL - (z > x ? 4u * q + 2u : 4u * q)));
-                any_offload = (__ballot_sync(peers, active && (words.y | words.w)) & peers) != 0u;
-            }
-            if (!any_offload) return;
-            const float y = words.y ? o.y : 0.0f, w = words.w ? o.w : 0.0f;
-            const unsigned bo = active ? __float_as_uint(fmaxf(y, w)) : 0u;
-            const unsigned mo = __reduce_max_sync(peers, bo);
-            if (mo) {
+                const unsigned second = __ballot_sync(peers, z > x);
+                if (me && leader) {
+                    const int wl = __ffs(who) - 1;
+                    const unsigned idx = 4u * unsigned(q_lane0 + wl) + (((second >> wl) & 1u) ? 2u : 0u);
+                    const unsigned long long key = (static_cast<unsigned long long>(me) << 32) | (FULL - idx);
+                    if (key > kq[sp.nC]) kq[sp.nC] = key;
+                }
+            },
+            [&](int ci, float r) {
+                const unsigned bo = feasible ? __float_as_uint(r) : 0u;
+                const unsigned mo = __reduce_max_sync(peers, bo);
                 const unsigned who = __ballot_sync(peers, bo == mo) & peers;
-                if (lane == __ffs(who) - 1)
-                    atomicMax(kq + ci, (static_cast<unsigned long long>(mo) << 32) | (FULL - (w > y ? 4u * q + 3u : 4u * q + 1u)));
-            }
-        });
+                if (mo && leader) {
+                    const int wl = __ffs(who) - 1;
+                    // lane wl computed plan (stage 2 + ((wl & 3) >> 1), checkpointing wl & 1) of its triple
+                    const unsigned idx = 4u * unsigned(q_lane0 + (wl & ~3) + 2 + ((wl & 3) >> 1)) + 1u + 2u * unsigned(wl & 1);
+                    const unsigned long long key = (static_cast<unsigned long long>(mo) << 32) | (FULL - idx);
+                    if (key > kq[ci]) kq[ci] = key;
+                }
+            });
+        __syncwarp();                                           // the next pass may have another leader for the same slot
+    }
+    __syncthreads();
+    // merge the warps' slots into warp 0's
+    for (int i = tid; i < per_warp; i += blockDim.x) {
+        unsigned long long k = keys[i];
+#pragma unroll
+        for (int w = 1; w < CURVES_WARPS; ++w) { const unsigned long long o = keys[size_t(w) * per_warp + i]; k = o > k ? o : k; }
+        keys[i] = k;
     }
     __syncthreads();
 
@@ -389,7 +430,7 @@ cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *
                           cudaStream_t st)
 {
     if (J == 0) return cudaSuccess;
-    const size_t smem = size_t(sp.nG) * (sp.nC + 1) * sizeof(unsigned long long);
+    const size_t smem = size_t(CURVES_WARPS) * sp.nG * (sp.nC + 1) * sizeof(unsigned long long);
     if (smem > 48 * 1024) {
         cudaError_t e = sp.wide ? cudaFuncSetAttribute(curves_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))
                                 : cudaFuncSetAttribute(curves_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
