@@ -98,6 +98,16 @@ __device__ __forceinline__ int first_level(const Space &sp, int64_t need)
     return lo;
 }
 
+// What the offload plans of a quad (stage >= 2: plans 4q + 1 and 4q + 3) need per core level c:
+//   throughput = bf * rcp(base_i + f^{k_swap}(opt_c / c, T_off)),  i = 0 without / 1 with gradient checkpointing
+struct OffloadTerms {
+    float T_off, opt_c;        // transfer time; optimizer time on one core (the same on the four quads of a triple)
+    float base0, base1;        // everything else in T_iter, per checkpointing setting
+    float k_swap, inv_kswap, bf;
+    bool ok0, ok1;             // plan 4q + 1 / 4q + 3 is structurally valid and not disabled
+    bool any;                  // some lane of the warp holds such a plan (warp-uniform)
+};
+
 // Everything one thread does for (job j, quad q): the feasibility words (stored by active threads) and the
 // four throughputs of every CPU level, handed to emit(ci, float4, words) in ascending level order.  Whole warps
 // must call this together with the quads of a warp consecutive and starting at a multiple of four (the
@@ -105,14 +115,10 @@ __device__ __forceinline__ int first_level(const Space &sp, int64_t need)
 // Returns the four feasibility words when KEEP_WORDS (zeros otherwise).
 // WIDE: degrees of any size from the wide quad table (divisions); otherwise powers of two from the
 // logarithms of the quad table (shifts, exact reciprocals).
-// LANE_PLANS: the caller wants no float4 per quad but the plans one by one, as the lanes compute them: head(out,
-// words, feasible) is called once with the two throughputs that do not depend on the core count (out.x, out.z), the
-// quad's four words and whether THIS LANE's offload plan -- ZeRO stage 2 + ((lane & 3) >> 1), checkpointing = lane & 1,
-// of the lane's (d, t, p) triple: plan index 4 * (first quad of the triple + 2 + ((lane & 3) >> 1)) + 1 + 2 * (lane & 1),
-// ascending with the lane -- may run at some memory level; then emit(ci, r) with that plan's throughput per core
-// level (0 when the plan is invalid; same bits as the float4 form).  emit is not called at all when no lane of the
-// warp holds a valid offload plan.
-template <bool KEEP_WORDS, bool WIDE, bool LANE_PLANS, class Head, class Emit>
+// TERMS_ONLY: the caller walks the core levels itself: head(out, words, terms) is called once with the two
+// throughputs that do not depend on the core count (out.x, out.z), the quad's four words and the quad's terms of the
+// offload plans (OffloadTerms; the same bits the float4 form uses), and emit is never called.
+template <bool KEEP_WORDS, bool WIDE, bool TERMS_ONLY, class Head, class Emit>
 __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restrict__ quads_any,
                                            const rubick_job *__restrict__ jobs, int j, int q, bool active,
                                            uint32_t *__restrict__ feas, Head &&head, Emit &&emit)
@@ -228,14 +234,10 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
     const bool off0 = valid_off && !(disabled & 2), off1 = valid_off && !(disabled & 8);
     const unsigned FULL = 0xffffffffu;
     const int lane = threadIdx.x & 31, gbase = lane & ~3, zl = lane & 3;
-    if constexpr (LANE_PLANS) {
-        // may this lane's offload plan run at all?  its word sits with the lane that owns the quad
-        const uint32_t wy = __shfl_sync(FULL, fw_out.y, gbase + 2 + (zl >> 1)), ww = __shfl_sync(FULL, fw_out.w, gbase + 2 + (zl >> 1));
-        head(out, fw_out, ((zl & 1) ? ww : wy) != 0u);
-    }
-    if (!__any_sync(FULL, off0 || off1)) {
-        if constexpr (!LANE_PLANS)
-            for (int ci = 0; ci < sp.nC; ++ci) emit(ci, out, fw_out);
+    const bool any_off = __any_sync(FULL, off0 || off1);
+    if (!any_off) {
+        if constexpr (TERMS_ONLY) head(out, fw_out, OffloadTerms{0.0f, 0.0f, 0.0f, 0.0f, 1.0f, 1.0f, bf, false, false, false});
+        else for (int ci = 0; ci < sp.nC; ++ci) emit(ci, out, fw_out);
         return fw_out;
     }
     const float T_off = sp.e * Psi * inv_d * sp.inv_B_pcie;          // identical on the four lanes
@@ -245,6 +247,10 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
     if (valid_off) {
         const float f_off = overlap(jb.k_off, 1.0f / jb.k_off, T_dp, T_off);
         base0 = cc0 + f_off; base1 = cc1 + f_off;
+    }
+    if constexpr (TERMS_ONLY) {
+        head(out, fw_out, OffloadTerms{T_off, opt_c, base0, base1, jb.k_swap, inv_kswap, bf, off0, off1, true});
+        return fw_out;
     }
     const int src = gbase + 2 + (zl >> 1);
     const float sb0 = __shfl_sync(FULL, base0, src), sb1 = __shfl_sync(FULL, base1, src);
@@ -259,15 +265,11 @@ __device__ __forceinline__ uint4 eval_quad(const Space &sp, const void *__restri
         for (int cc = 0; cc < 4; ++cc) {
             const float fs = __shfl_sync(FULL, fs_mine, gbase + cc);
             const float r = my_ok ? bf * rcp_approx(my_base + fs) : 0.0f;
-            if constexpr (LANE_PLANS) {
-                if (c0 + cc < sp.nC) emit(c0 + cc, r);
-            } else {
-                const float ry = __shfl_sync(FULL, r, src_y), rw = __shfl_sync(FULL, r, src_w);
-                if (c0 + cc < sp.nC) {
-                    out.y = zl >= 2 ? ry : 0.0f;
-                    out.w = zl >= 2 ? rw : 0.0f;
-                    emit(c0 + cc, out, fw_out);
-                }
+            const float ry = __shfl_sync(FULL, r, src_y), rw = __shfl_sync(FULL, r, src_w);
+            if (c0 + cc < sp.nC) {
+                out.y = zl >= 2 ? ry : 0.0f;
+                out.w = zl >= 2 ? rw : 0.0f;
+                emit(c0 + cc, out, fw_out);
             }
         }
     }
@@ -291,7 +293,7 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const void *__restrict_
     const int q = int(gid - uint32_t(j) * uint32_t(sp.Q));
     float *row = thr + (size_t(j) * sp.nC * sp.P + 4 * size_t(q));
     // levels arrive in ascending order, one call each: the row pointer just advances
-    eval_quad<false, WIDE, false>(sp, quads, jobs, j, q, active, feas, [](const float4 &, const uint4 &, bool) {},
+    eval_quad<false, WIDE, false>(sp, quads, jobs, j, q, active, feas, [](const float4 &, const uint4 &, const OffloadTerms &) {},
                                   [&](int, const float4 &out, const uint4 &) {
         if (active) __stcs(reinterpret_cast<float4 *>(row), out);
         row += sp.P;
@@ -301,24 +303,32 @@ eval_candidates_kernel(const __grid_constant__ Space sp, const void *__restrict_
 // ------------------------------------------------------------------------------------------------------
 // Curves without the table: the evaluation above and the best-plan / sensitivity-curve step (paper
 // Section 5.2) in one kernel, for callers that only want the curves (a scheduling round).  One CTA per
-// job; thread = quad as above, but nothing goes to memory: per class (plans without / with offload, which
-// share one first feasible memory level per GPU level under this library's memory rule) the lanes of a warp
-// that sit in the same GPU level reduce the value with one warp reduction, and a vote names the lowest lane
-// holding it.  Plans without offload do not depend on the core count and are reduced once per GPU level from
-// the quads' own two values; offload plans are reduced per core level straight from the lanes that computed
-// them (one plan per lane, plan index ascending with the lane, so the lowest lane holding the maximum holds
-// the lowest plan index).  The group's first lane folds (value bits << 32 | ~index) into a slot of its own warp
-// per (GPU level, core level) with a plain read-compare-write -- no atomics: a slot has one writer at a time, and
-// a warp synchronises between its passes over the quads.  After a CTA barrier the warps' slots are merged; then
-// thread (c, m) combines the two classes for memory level m, takes the running maximum over GPU levels and
-// stores its three outputs.  Same values, same ties (lowest plan index) as best_plan on the table of
-// eval_candidates: bit-identical.  Nothing but the mask (4 bytes per plan) and the curves is written.
+// job, and nothing but the mask (4 bytes per plan) and the curves goes to memory.
+//
+// Pass over 32 quads per warp, in two parts.  (1) Lane = quad, as in the table kernel: the feasibility words and
+// everything that does not depend on the core count.  Plans without offload do not depend on it at all: per
+// GPU level their maximum is one warp reduction over the quads' two values and a vote that names the lowest lane
+// holding it (quads ascend with the lane, so that is the lowest plan index).  (2) Lane = core level: the eight
+// (d, t, p) triples of the pass are walked one after the other, their terms handed round by shuffles; every
+// lane evaluates the triple's four offload plans at its own core level, in plan order, and keeps the running
+// maximum and its plan index in registers (strictly greater replaces: lowest index on ties).  No reduction
+// across lanes is needed, and the values are the same bits as the table kernel's.  Where the GPU level
+// changes inside a pass, and at its end, lane c folds its (value bits << 32 | ~index) into the slot
+// (GPU level, core level c) of its warp with a plain read-compare-write: a slot of the offload class only ever
+// has that one writer.
+//
+// After a CTA barrier the warps' slots are merged; then the output phase combines the two classes per memory
+// level (under this library's memory rule the plans of a class share one first feasible memory level per GPU
+// level), takes the running maximum over GPU levels and stores value, plan and GPU count: four memory levels per
+// thread with 16-byte stores when the layout allows it.  Same values, same ties (lowest plan index) as best_plan
+// on the table of eval_candidates: bit-identical.
 // ------------------------------------------------------------------------------------------------------
 constexpr int CURVES_THREADS = 128;      // small CTAs: the phases of the several CTAs of an SM overlap
 constexpr int CURVES_WARPS = CURVES_THREADS / 32;
+constexpr int CURVES_MIN_CTAS = 10;      // registers capped at 48 a thread: 40 warps an SM hide the shuffle and reciprocal latencies (0.57 ms against 0.89 ms uncapped)
 
-template <bool WIDE>
-__global__ void __launch_bounds__(CURVES_THREADS)
+template <bool WIDE, bool VEC4>
+__global__ void __launch_bounds__(CURVES_THREADS, WIDE ? 8 : CURVES_MIN_CTAS)       // the wide instance needs 64 registers
 curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads, const void *__restrict__ quads_any,
               const rubick_job *__restrict__ jobs, int J, unsigned flags, uint32_t *__restrict__ feas,
               float *__restrict__ best_val, int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g)
@@ -327,12 +337,14 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
     // [warp][nG][nC + 1]: offload class per core level, then the other class; warp 0's copy receives the merge
     unsigned long long *keys = reinterpret_cast<unsigned long long *>(smem_raw);
     __shared__ int s_first[2 * RUBICK_MAX_G_LEVELS];        // first feasible memory level per (GPU level, class), nM = none
+    __shared__ float s_inv_c[RUBICK_MAX_C_LEVELS];          // lane-indexed look-ups: not from the constant bank
     const int j = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned FULL = 0xffffffffu;
     const int per_warp = sp.nG * (sp.nC + 1);
 
     for (int i = tid; i < CURVES_WARPS * per_warp; i += blockDim.x) keys[i] = 0ull;
+    if (tid < sp.nC) s_inv_c[tid] = sp.inv_c[tid];
     if (tid < sp.nG) {
         // host-memory need of the level's plans: g processes, plus the offloaded states (as in the mask above)
         const rubick_job *jp = jobs + j;
@@ -354,41 +366,69 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
         const int q = active ? q_raw : sp.Q - 1;
         const int level = reinterpret_cast<const uint8_t *>(quads + q)[4];             // QuadDesc::g_level
         const unsigned peers = __match_any_sync(FULL, active ? level : -1);            // lanes of the same GPU level
-        const bool leader = active && lane == __ffs(peers) - 1;
         const int q_lane0 = q_raw - lane;                       // quad of lane 0 (quads ascend with the lane)
-        unsigned long long *kq = mine + size_t(level) * (sp.nC + 1);
-        bool feasible = false;                                  // may this lane's offload plan run at some memory level?
+        OffloadTerms ot;
+        unsigned has1 = 0u, has3 = 0u;                          // lanes whose plan 4q + 1 / 4q + 3 may run at some memory level
         eval_quad<true, WIDE, true>(sp, quads_any, jobs, j, q, active, feas,
-            [&](const float4 &o, const uint4 &words, bool lane_plan_feasible) {
-                // plans without offload: the quad's two values; infeasible plans count as 0.  Quads ascend with the
-                // lane and a quad's two plans with their index, so the lowest lane holding the maximum holds the
-                // lowest plan index.
-                feasible = active && lane_plan_feasible;
+            [&](const float4 &o, const uint4 &words, const OffloadTerms &terms) {
+                // plans without offload: the quad's two values; infeasible plans count as 0
+                ot = terms;
                 const float x = words.x ? o.x : 0.0f, z = words.z ? o.z : 0.0f;
                 const unsigned be = active ? __float_as_uint(fmaxf(x, z)) : 0u;
                 const unsigned me = __reduce_max_sync(peers, be);
                 const unsigned who = __ballot_sync(peers, be == me) & peers;
                 const unsigned second = __ballot_sync(peers, z > x);
-                if (me && leader) {
+                if (me && lane == __ffs(peers) - 1) {
                     const int wl = __ffs(who) - 1;
                     const unsigned idx = 4u * unsigned(q_lane0 + wl) + (((second >> wl) & 1u) ? 2u : 0u);
                     const unsigned long long key = (static_cast<unsigned long long>(me) << 32) | (FULL - idx);
-                    if (key > kq[sp.nC]) kq[sp.nC] = key;
+                    unsigned long long *slot = mine + size_t(level) * (sp.nC + 1) + sp.nC;
+                    if (key > *slot) *slot = key;
                 }
+                has1 = __ballot_sync(FULL, active && terms.ok0 && words.y != 0u);
+                has3 = __ballot_sync(FULL, active && terms.ok1 && words.w != 0u);
             },
-            [&](int ci, float r) {
-                const unsigned bo = feasible ? __float_as_uint(r) : 0u;
-                const unsigned mo = __reduce_max_sync(peers, bo);
-                const unsigned who = __ballot_sync(peers, bo == mo) & peers;
-                if (mo && leader) {
-                    const int wl = __ffs(who) - 1;
-                    // lane wl computed plan (stage 2 + ((wl & 3) >> 1), checkpointing wl & 1) of its triple
-                    const unsigned idx = 4u * unsigned(q_lane0 + (wl & ~3) + 2 + ((wl & 3) >> 1)) + 1u + 2u * unsigned(wl & 1);
-                    const unsigned long long key = (static_cast<unsigned long long>(mo) << 32) | (FULL - idx);
-                    if (key > kq[ci]) kq[ci] = key;
+            [](int, const float4 &, const uint4 &) {});
+        if (ot.any && ((has1 | has3) != 0u)) {
+            // lane = core level: walk the pass's triples (lanes 4 tau .. 4 tau + 3 hold ZeRO stages 0..3; the offload
+            // plans are those of stages 2 and 3)
+            for (int cb = 0; cb < sp.nC; cb += 32) {
+                const int ci = cb + lane;
+                const bool have = ci < sp.nC;
+                const float inv_c = s_inv_c[have ? ci : 0];
+                float run_v = 0.0f; unsigned run_i = 0u;
+                int cur = __shfl_sync(FULL, level, 0);
+                auto flush = [&](int lvl) {
+                    if (have && run_v > 0.0f) {
+                        const unsigned long long key = (static_cast<unsigned long long>(__float_as_uint(run_v)) << 32) | (FULL - run_i);
+                        unsigned long long *slot = mine + size_t(lvl) * (sp.nC + 1) + ci;
+                        if (key > *slot) *slot = key;
+                    }
+                    run_v = 0.0f;
+                };
+#pragma unroll 2
+                for (int tau = 0; tau < 8; ++tau) {
+                    const int l0 = 4 * tau;
+                    const unsigned bits = (((has1 >> (l0 + 2)) & 1u)) | (((has3 >> (l0 + 2)) & 1u) << 1)
+                                        | (((has1 >> (l0 + 3)) & 1u) << 2) | (((has3 >> (l0 + 3)) & 1u) << 3);     // warp-uniform
+                    const int lvl = __shfl_sync(FULL, level, l0);
+                    if (lvl != cur) { flush(cur); cur = lvl; }
+                    if (!bits) continue;
+                    const float T_off = __shfl_sync(FULL, ot.T_off, l0 + 2), opt_c = __shfl_sync(FULL, ot.opt_c, l0 + 2);
+                    const float b20 = __shfl_sync(FULL, ot.base0, l0 + 2), b21 = __shfl_sync(FULL, ot.base1, l0 + 2);
+                    const float b30 = __shfl_sync(FULL, ot.base0, l0 + 3), b31 = __shfl_sync(FULL, ot.base1, l0 + 3);
+                    const float fs = overlap(ot.k_swap, ot.inv_kswap, opt_c * inv_c, T_off);
+                    const unsigned p2 = 4u * unsigned(q_lane0 + l0 + 2), p3 = p2 + 4u;
+                    // the four plans in index order; strictly greater replaces
+                    if (bits & 1u) { const float r = ot.bf * rcp_approx(b20 + fs); if (r > run_v) { run_v = r; run_i = p2 + 1u; } }
+                    if (bits & 2u) { const float r = ot.bf * rcp_approx(b21 + fs); if (r > run_v) { run_v = r; run_i = p2 + 3u; } }
+                    if (bits & 4u) { const float r = ot.bf * rcp_approx(b30 + fs); if (r > run_v) { run_v = r; run_i = p3 + 1u; } }
+                    if (bits & 8u) { const float r = ot.bf * rcp_approx(b31 + fs); if (r > run_v) { run_v = r; run_i = p3 + 3u; } }
                 }
-            });
-        __syncwarp();                                           // the next pass may have another leader for the same slot
+                flush(cur);
+            }
+        }
+        __syncwarp();                                           // the slot of the other class may have another writer in the next pass
     }
     __syncthreads();
     // merge the warps' slots into warp 0's
@@ -401,26 +441,61 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
     __syncthreads();
 
     const bool raw = (flags & RUBICK_BEST_RAW) != 0;
-    for (int cm = tid; cm < sp.nC * sp.nM; cm += blockDim.x) {
-        const int ci = cm / sp.nM, m = cm - ci * sp.nM;
-        unsigned run_v = 0u, run_i = FULL; int run_g = 0;
-        size_t o = (size_t(j) * sp.nG * sp.nC + ci) * sp.nM + m;
-        for (int g = 0; g < sp.nG; ++g, o += size_t(sp.nC) * sp.nM) {
-            const unsigned long long ke = keys[size_t(g) * (sp.nC + 1) + sp.nC], ko = keys[size_t(g) * (sp.nC + 1) + ci];
-            const bool use_e = ke && m >= s_first[2 * g], use_o = ko && m >= s_first[2 * g + 1];
-            unsigned bv = use_e ? unsigned(ke >> 32) : 0u, bi = use_e ? FULL - unsigned(ke) : FULL;
-            const unsigned vo = unsigned(ko >> 32), io = FULL - unsigned(ko);
-            const bool odd_wins = use_o && (vo > bv || (vo == bv && io < bi));
-            bv = odd_wins ? vo : bv; bi = odd_wins ? io : bi;
-            int bg = bv ? sp.g_levels[g] : 0;
-            if (!raw) {
-                const bool up = bv > run_v;
-                run_v = up ? bv : run_v; run_i = up ? bi : run_i; run_g = up ? bg : run_g;
-                bv = run_v; bi = run_i; bg = run_g;
+    // what (GPU level g, core level ci) offers at memory level m: the better of the two classes that may run there
+    auto entry = [&](int g, unsigned long long ke, unsigned long long ko, int fe, int fo, int m, unsigned &bv, unsigned &bi, int &bg) {
+        const bool use_e = ke && m >= fe, use_o = ko && m >= fo;
+        bv = use_e ? unsigned(ke >> 32) : 0u; bi = use_e ? FULL - unsigned(ke) : FULL;
+        const unsigned vo = unsigned(ko >> 32), io = FULL - unsigned(ko);
+        const bool odd_wins = use_o && (vo > bv || (vo == bv && io < bi));
+        bv = odd_wins ? vo : bv; bi = odd_wins ? io : bi;
+        bg = bv ? sp.g_levels[g] : 0;
+    };
+    if constexpr (VEC4) {
+        // nM is a multiple of 4 and the three tables are 16-byte aligned: one thread = four memory levels
+        const int m4 = sp.nM >> 2;
+        for (int item = tid; item < sp.nC * m4; item += blockDim.x) {
+            const int ci = item / m4, mb = (item - ci * m4) << 2;
+            unsigned run_v[4] = {0u, 0u, 0u, 0u}, run_i[4] = {FULL, FULL, FULL, FULL}; int run_g[4] = {0, 0, 0, 0};
+            size_t o = (size_t(j) * sp.nG * sp.nC + ci) * sp.nM + mb;
+            for (int g = 0; g < sp.nG; ++g, o += size_t(sp.nC) * sp.nM) {
+                const unsigned long long ke = keys[size_t(g) * (sp.nC + 1) + sp.nC], ko = keys[size_t(g) * (sp.nC + 1) + ci];
+                const int fe = s_first[2 * g], fo = s_first[2 * g + 1];
+                uint4 v; int4 pi, gg;
+                unsigned *vv = reinterpret_cast<unsigned *>(&v); int *pp = reinterpret_cast<int *>(&pi), *gp = reinterpret_cast<int *>(&gg);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    unsigned bv, bi; int bg;
+                    entry(g, ke, ko, fe, fo, mb + k, bv, bi, bg);
+                    if (!raw) {
+                        const bool up = bv > run_v[k];
+                        run_v[k] = up ? bv : run_v[k]; run_i[k] = up ? bi : run_i[k]; run_g[k] = up ? bg : run_g[k];
+                        bv = run_v[k]; bi = run_i[k]; bg = run_g[k];
+                    }
+                    vv[k] = bv; pp[k] = int(bi); gp[k] = bg;
+                }
+                *reinterpret_cast<uint4 *>(best_val + o) = v;
+                *reinterpret_cast<int4 *>(best_plan + o) = pi;
+                *reinterpret_cast<int4 *>(best_g + o) = gg;
             }
-            best_val[o] = __uint_as_float(bv);
-            best_plan[o] = int(bi);
-            best_g[o] = bg;
+        }
+    } else {
+        for (int cm = tid; cm < sp.nC * sp.nM; cm += blockDim.x) {
+            const int ci = cm / sp.nM, m = cm - ci * sp.nM;
+            unsigned run_v = 0u, run_i = FULL; int run_g = 0;
+            size_t o = (size_t(j) * sp.nG * sp.nC + ci) * sp.nM + m;
+            for (int g = 0; g < sp.nG; ++g, o += size_t(sp.nC) * sp.nM) {
+                const unsigned long long ke = keys[size_t(g) * (sp.nC + 1) + sp.nC], ko = keys[size_t(g) * (sp.nC + 1) + ci];
+                unsigned bv, bi; int bg;
+                entry(g, ke, ko, s_first[2 * g], s_first[2 * g + 1], m, bv, bi, bg);
+                if (!raw) {
+                    const bool up = bv > run_v;
+                    run_v = up ? bv : run_v; run_i = up ? bi : run_i; run_g = up ? bg : run_g;
+                    bv = run_v; bi = run_i; bg = run_g;
+                }
+                best_val[o] = __uint_as_float(bv);
+                best_plan[o] = int(bi);
+                best_g[o] = bg;
+            }
         }
     }
 }
@@ -431,17 +506,20 @@ cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *
 {
     if (J == 0) return cudaSuccess;
     const size_t smem = size_t(CURVES_WARPS) * sp.nG * (sp.nC + 1) * sizeof(unsigned long long);
-    if (smem > 48 * 1024) {
-        cudaError_t e = sp.wide ? cudaFuncSetAttribute(curves_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem))
-                                : cudaFuncSetAttribute(curves_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
-        if (e != cudaSuccess) return e;
-    }
-    if (sp.wide)
-        curves_kernel<true><<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_wide_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
-    else
-        curves_kernel<false><<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, d_quads, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
-    count_launch();
-    return cudaGetLastError();
+    // 16-byte stores of four memory levels need rows that start on 16-byte boundaries
+    const bool vec4 = (sp.nM & 3) == 0 && ((reinterpret_cast<uintptr_t>(d_best_val) | reinterpret_cast<uintptr_t>(d_best_plan)
+                                            | reinterpret_cast<uintptr_t>(d_best_g)) & 15) == 0;
+    auto launch = [&](auto kernel, const void *quads_any) -> cudaError_t {
+        if (smem > 48 * 1024) {
+            cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
+            if (e != cudaSuccess) return e;
+        }
+        kernel<<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, quads_any, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
+        count_launch();
+        return cudaGetLastError();
+    };
+    if (sp.wide) return vec4 ? launch(curves_kernel<true, true>, d_wide_quads) : launch(curves_kernel<true, false>, d_wide_quads);
+    return vec4 ? launch(curves_kernel<false, true>, d_quads) : launch(curves_kernel<false, false>, d_quads);
 }
 
 cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
