@@ -286,8 +286,7 @@ __device__ int first_fit_from_mark(const Views &v, Shared &sh, int gi, int g, in
         if (first_g < 0 && bg) first_g = pos + __ffs(bg) - 1;
         if (bf) found = pos + __ffs(bf) - 1;
     }
-    __syncwarp();
-    if (lane == 0) sh.ff_pos[gi] = first_g >= 0 ? first_g : v.N;
+    sh.ff_pos[gi] = first_g >= 0 ? first_g : v.N;       // the same value from every lane: each sees its own store afterwards
     return found;
 }
 
@@ -777,45 +776,86 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 may = may && pa_fail[a0.x * sp.nC + a0.y] != sh.pa_commits;
             }
             unsigned todo = __ballot_sync(0xffffffffu, may);
-            // the records of the batch go through shared memory: one turn reads its job's with three loads
-            __syncwarp();
-            sh.pa_rec[lane][0] = a0; sh.pa_rec[lane][1] = a1; sh.pa_job[lane] = jl;
-            __syncwarp();
+            // what a turn needs of its job beyond the cluster's state, worked out by the job's lane: is the curve entry
+            // of the target usable as it stands (a plan that runs, with the level's own GPU count), and the memory it takes
+            const bool entry_ok = a0.w >= 0 && a0.w < sp.P && __int_as_float(a0.z) > 0.0f && a1.y != 0 && a1.x >= 0 && a1.x < sp.nM;
+            const long long m_need_l = entry_ok ? v.ml[a1.x] : 0;
+            // Turns run on all lanes alike (shuffles hand out the job's record, every lane reads and writes the same
+            // shared-memory words, so each lane sees its own stores and the warp never has to synchronise).  The
+            // usual turn -- a job that fits one node, whose curve entry is usable and whose memory fits the node found
+            // -- touches five words: the failure mark of its levels, the first-fit mark, the node's GPUs / cores and
+            // memory.  Anything else (whole-node minima, an entry that needs the table) goes through commit_warp.
             while (todo) {
                 const int i = __ffs(todo) - 1;
                 todo &= todo - 1;
-                const int4 r0 = sh.pa_rec[i][0], r1 = sh.pa_rec[i][1];
-                const int j = sh.pa_job[i];
-                const int gi = r0.x, ci = r0.y;
-                HotCurve cand;
-                cand.val = __int_as_float(r0.z); cand.plan = r0.w; cand.f = r1.x; cand.ok = r1.y;
-                const float w = __int_as_float(r1.z);
-                const int tn = r1.w;
+                const int gi = __shfl_sync(0xffffffffu, a0.x, i), ci = __shfl_sync(0xffffffffu, a0.y, i);
+                const int j = __shfl_sync(0xffffffffu, jl, i);
+                const int tn = __shfl_sync(0xffffffffu, a1.w, i);
+                const int usable = __shfl_sync(0xffffffffu, int(entry_ok), i);
+                const long long m_need = __shfl_sync(0xffffffffu, m_need_l, i);
                 if (gi < 0) continue;
                 if (A.n_tenants > 0) {     // privileged only while the minimum fits the tenant's remaining quota
                     if (tn < 0 || tn >= A.n_tenants) continue;
                     if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[ci]) continue;
                 }
-                if (pa_fail[gi * sp.nC + ci] == sh.pa_commits) continue;        // same levels, same cluster: same outcome
-                Committed cm; cm.first = -1;
-                if (commit_warp<false, true>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm)) {
-                    const int s = sh.n_slots;
-                    if (lane == 0) {
-                        SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
-                        SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
-                        v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
-                        sh.n_slots = s + 1;
-                        sh.pa_commits += 1;
-                        if (A.n_tenants > 0) { rem_q[2 * tn] -= sp.g_levels[gi]; rem_q[2 * tn + 1] -= sp.c_levels[ci]; }
+                const int commits = sh.pa_commits;
+                if (pa_fail[gi * sp.nC + ci] == commits) continue;              // same levels, same cluster: same outcome
+                const int g2 = v.gl[gi], c2 = v.clv[ci];
+                int placed_on = -1;
+                bool settled = false;
+                if (g2 <= sp.Gn && usable) {
+                    // no node below the mark has g2 free GPUs: if the node at the mark fits, it is the first fit
+                    int target = sh.ff_pos[gi];
+                    int w_old = target < N ? v.gc[target] : 0;
+                    if (!(fg_of(w_old) >= g2 && fc_of(w_old) >= c2)) {
+                        target = first_fit_from_mark(v, sh, gi, g2, c2, lane);
+                        w_old = target >= 0 ? v.gc[target] : 0;
                     }
+                    if (target < 0) { pa_fail[gi * sp.nC + ci] = commits; continue; }      // no node for these levels
+                    const int64_t fm = v.free_m[target];
+                    if (m_need <= fm) {
+                        // the highest memory level that fits the node is at or above the plan's own: the entry stands
+                        v.gc[target] = w_old - ((g2 << 16) + c2);
+                        v.free_m[target] = fm - m_need;
+                        if (fg_of(w_old) == sp.Gn) sh.n_empty = sh.n_empty - 1;
+                        placed_on = target; settled = true;
+                    } else if (v.ml[0] > fm) { pa_fail[gi * sp.nC + ci] = commits; continue; }   // the node found has memory for no level
+                }
+                const float val_e = __int_as_float(__shfl_sync(0xffffffffu, a0.z, i));
+                const int plan_e = __shfl_sync(0xffffffffu, a0.w, i), f_e = __shfl_sync(0xffffffffu, a1.x, i);
+                const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
+                Committed cm; cm.first = placed_on; cm.val = val_e; cm.plan = plan_e; cm.f = f_e;
+                if (!settled) {
+                    HotCurve cand;
+                    cand.val = val_e; cand.plan = plan_e; cand.f = f_e; cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
+                    cm.first = -1;
                     __syncwarp();
-                } else if (cm.first == -2) {
-                    if (lane == 0) pa_fail[gi * sp.nC + ci] = sh.pa_commits;
+                    settled = commit_warp<false, true>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm);
                     __syncwarp();
+                    if (!settled) {
+                        if (cm.first == -2) pa_fail[gi * sp.nC + ci] = commits;
+                        continue;
+                    }
+                }
+                const int s = sh.n_slots;
+                if (lane == 0) {
+                    SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
+                    SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
+                    v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
+                }
+                sh.n_slots = s + 1;
+                sh.pa_commits = commits + 1;
+                if (A.n_tenants > 0) {
+                    const int qg = rem_q[2 * tn], qc = rem_q[2 * tn + 1];
+                    rem_q[2 * tn] = qg - sp.g_levels[gi]; rem_q[2 * tn + 1] = qc - sp.c_levels[ci];
                 }
             }
             jl = jl_next; a0 = n0; a1 = n1; jl_next = jl_after;
         }
+        // During this phase maxc[] only served as a hint that errs on the generous side (the usual turn does not
+        // maintain it; free resources only shrink, so an old entry is never too small): make it exact again.
+        __syncwarp();
+        rebuild_maxc_warp(sp, v, lane);
     }
     __syncthreads();
     // gains of the jobs placed in Phase A
