@@ -224,6 +224,82 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_strong(args, cfg, rank, world, local, dev):
+    """One problem on all GPUs (paper Section 5.2: the curves of different jobs are independent and "can be computed
+    in parallel"): rank r builds mask and curves of its contiguous job tile with rubick_curves, one all-gather per
+    table brings every tile into every rank's HBM, and every rank runs the same greedy round on the full tables
+    (a round needs a global arg-max per step, so it is replicated, not sharded).  All ranks must reach the same
+    allocation; that is checked after the timed region."""
+    import torch
+    import torch.distributed as dist
+    from paper_2408_08586_b200 import binding as rb
+    from paper_2408_08586_b200 import sharding
+    jobs, N = cfg["jobs"], cfg["n_nodes"]
+    J = len(jobs["P"])
+    plans, _ = rb.enumerate_plans(cfg["g_levels"])
+    P, G, C, M = len(plans), len(cfg["g_levels"]), len(cfg["c_levels"]), len(cfg["m_levels"])
+    stream = torch.cuda.Stream(device=dev)
+    ctx = rb.Context(cfg["env"], device=local, stream=stream.cuda_stream)
+    ctx.set_space(plans, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"])
+    d_jobs = rb.to_device(rb.pack_jobs(jobs), dev)
+    rows = sharding.table_rows(P, G, C, M)
+    cap = sharding.tile_capacity(J, world)
+    start, count = sharding.job_tile(J, world, rank)
+    tile = {k: torch.zeros(cap * n, dtype=dt, device=dev) for k, (n, dt) in rows.items()}
+    full = {k: torch.empty(J * n, dtype=dt, device=dev) for k, (n, dt) in rows.items()}
+    d_out = torch.empty(J * rb.ASSIGN_DTYPE.itemsize + N * rb.NODE_DTYPE.itemsize, dtype=torch.uint8, device=dev)
+    d_assign, d_node = d_out[: J * rb.ASSIGN_DTYPE.itemsize], d_out[J * rb.ASSIGN_DTYPE.itemsize:]
+    compute = sharding.curves_tile_fn(ctx, d_jobs, rb.JOB_DTYPE.itemsize)
+    steps_taken = [0]
+
+    def step():
+        with torch.cuda.stream(stream):
+            if count:
+                compute(start, count, tile)
+            for k, (n, _) in rows.items():
+                sharding.gather_tiles(tile[k], J, world, n, full[k])
+            steps_taken[0], _ = ctx.greedy_round(d_jobs, J, full["cv"], full["cp"], full["cg"], full["feas"], N, 1 << 30, d_assign, d_node)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local) if rank == 0 else None
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches_before = rb.kernel_launches()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(args.steps):
+        step()
+    b.record(stream)
+    barrier()
+    gpu_launches = rb.kernel_launches() - launches_before
+    clocks = sampler.stop() if sampler else None
+    ms_per_step = reduce_max_ms(a.elapsed_time(b), world) / args.steps
+    agree = sharding.assignments_agree(d_out, world)
+    if not agree:
+        raise SystemExit("the ranks reached different allocations from the same tables")
+    if rank == 0:
+        gathered = sum(J * n * torch.empty(0, dtype=dt).element_size() for n, dt in rows.values())
+        line = {"metric": METRIC, "value": float(J) * P * C / (ms_per_step * 1e-3), "unit": UNIT_E2E, "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": args.workload, "jobs": J, "jobs_per_gpu_tile": cap, "plans": P, "gpu_levels": G, "cpu_levels": C,
+                           "mem_levels": M, "nodes": N,
+                           "step": "rubick_curves on this rank's job tile + all-gather of mask and curve tables + greedy_round (replicated)",
+                           "l2": "the tables gathered per step are %.2f GB, larger than the 126 MB L2" % (gathered / 1e9)},
+                "clocks": clocks, "gpu_launches": int(gpu_launches), "all_gather_bytes_per_rank": int(gathered),
+                "ranks_agree": True, "round": {"steps": int(steps_taken[0])},
+                "roofline": None, "cpu_baseline": None, "e2e": None}
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -239,6 +315,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-probes", action="store_true", help="skip the machine probes and the curves-kernel roofline")
     ap.add_argument("--events", type=int, default=1000, help="scheduling events of the event-driven run (0 = skip)")
+    ap.add_argument("--scaling", default="weak", choices=["weak", "strong"],
+                    help="weak: one independent problem per GPU; strong: ONE problem, curves built in job tiles across the GPUs, "
+                         "all-gathered, the round replicated")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -260,7 +339,9 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
-    cfg = make_workload(args.workload, rank=rank, J=args.jobs, n_nodes=args.nodes)
+    cfg = make_workload(args.workload, rank=0 if args.scaling == "strong" else rank, J=args.jobs, n_nodes=args.nodes)
+    if args.scaling == "strong":
+        return run_strong(args, cfg, rank, world, local, dev)
     jobs, N = cfg["jobs"], cfg["n_nodes"]
     J = len(jobs["P"])
     plans, _ = rb.enumerate_plans(cfg["g_levels"])
