@@ -18,7 +18,7 @@ _SO = os.path.join(_HERE, "liboracle.so")
 JOB_FIELDS = ["P", "l", "h", "s", "b", "mu_cap", "alpha_act", "tau", "k_bwd", "k_sync", "k_opt",
               "k_opt_off", "k_off", "k_swap", "k_const", "w", "gmin_idx", "cmin_idx", "host_base_bytes", "tenant"]
 ENV_FIELDS = ["B_intra", "B_inter", "B_pcie", "gpu_mem_bytes", "gpus_per_node", "cpus_per_node",
-              "mem_per_node_bytes", "bytes_per_elem", "strict_zero_dp_only", "zero3_extra_volume"]
+              "mem_per_node_bytes", "bytes_per_elem", "strict_zero_dp_only", "zero3_extra_volume", "spread_align"]
 TERM_FIELDS = ["valid", "mu", "m", "a", "T_fwd", "T_bwd", "V_dp", "V_tp", "V_pp", "T_dp", "T_tp",
                "T_pp", "T_cc", "T_opt", "T_off", "T_oo", "T_iter", "thr"]
 MEM_FIELDS = ["params", "grads", "opt", "act", "gpu_total", "gpu_ok", "host_need", "nodes"]
@@ -202,10 +202,17 @@ def gain(jobs, curve_val, g_levels, c_levels, state_g, state_c, state_val):
 CAND_FIELDS = ("gain", "next", "placeable", "v_cur", "v_next", "units", "shut", "m_commit", "v_commit", "g_commit", "gi", "ci")
 
 
+MAX_PIECES = 32
+
+
 def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_levels, m_levels,
-                   n_nodes, max_steps=1 << 30, want_log=False, quota=None, double_decisions=False, want_candidates=False):
+                   n_nodes, max_steps=1 << 30, want_log=False, quota=None, double_decisions=False, want_candidates=False,
+                   spread=None):
     """One greedy round.  Default: decisions in single precision on the curve table rounded to single
     precision.  double_decisions: every decision in double precision on curve_val as given (float64).
+    spread: None, or a list of (align, curve_val, curve_plan, curve_g, feas) -- the tables of spread placement classes
+    (pieces of `align` GPUs on several nodes), widest pieces first; the result then carries `pieces` [J, 32]
+    (node << 8 | GPUs, -1 = unused) and `cls` [J] (-1 = packed).
     want_candidates: also `cand`, a dict of [J, 2] arrays (CAND_FIELDS; axis 1 = GPU / CPU increment) with
     what every job offered for the decision the round stopped at (the step `max_steps` cut off, or the
     last look that found nothing to do).
@@ -228,6 +235,19 @@ def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_
     log = np.zeros(max(cap, 1), dtype=np.int32)
     cand = np.zeros((max(J, 1), 2, len(CAND_FIELDS)), dtype=np.float64)
     qt = None if quota is None else _i64(quota).reshape(-1, 2)      # per tenant: GPUs, cores
+    nK = 0 if not spread else len(spread)
+    keep = []
+    if nK:
+        al = _i64([int(x[0]) for x in spread])
+        tabs = [(np.ascontiguousarray(x[1], dtype=np.float32), _i32(x[2]), _i32(x[3]), np.ascontiguousarray(x[4], dtype=np.uint32)) for x in spread]
+        keep = [al, tabs]
+        ptr = lambda i, t: (C.POINTER(t) * nK)(*[_p(tb[i], t) for tb in tabs])
+        k_val, k_plan, k_g, k_feas = ptr(0, C.c_float), ptr(1, C.c_int32), ptr(2, C.c_int32), ptr(3, C.c_uint32)
+        al_p = _p(al, C.c_int64)
+    else:
+        k_val = k_plan = k_g = k_feas = al_p = None
+    pieces = np.full((max(J, 1), MAX_PIECES), -1, dtype=np.int32)
+    cls = np.full(max(J, 1), -1, dtype=np.int32)
     r = lib().oracle_round(_p(rows, C.c_double), C.c_int(J), _p(env_row(env), C.c_double), _p(cv, C.c_float),
                            _p(cp, C.c_int32), _p(cg, C.c_int32), _p(feas, C.c_uint32), C.c_int(Pn),
                            _p(gl, C.c_int64), C.c_int(len(gl)), _p(cl, C.c_int64), C.c_int(len(cl)),
@@ -236,7 +256,9 @@ def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_
                            _p(out_i, C.c_int64), _p(out_v, C.c_float), _p(node, C.c_int64),
                            _p(log, C.c_int32) if want_log else None,
                            _p(cv64, C.c_double) if cv64 is not None else None, _p(out_v64, C.c_double),
-                           _p(cand, C.c_double) if want_candidates else None)
+                           _p(cand, C.c_double) if want_candidates else None,
+                           C.c_int(nK), al_p, k_val, k_plan, k_g, k_feas, _p(pieces, C.c_int32), _p(cls, C.c_int32))
+    del keep
     capped = r < 0
     steps = -r - 1 if capped else r
     out_i = out_i[:J]
@@ -247,6 +269,8 @@ def schedule_round(jobs, env, curve_val, curve_plan, curve_g, feas, g_levels, c_
                steps=steps, capped=capped, log=log[:steps].copy() if want_log else None)
     if want_candidates:
         res["cand"] = {k: cand[:J, :, i].copy() for i, k in enumerate(CAND_FIELDS)}
+    if nK:
+        res["pieces"], res["cls"] = pieces[:J].copy(), cls[:J].copy()
     return res
 
 

@@ -70,6 +70,9 @@ enum {
     EF_E,                               /* bytes per element (2 = fp16)             */
     EF_STRICT,                          /* 1: ZeRO / offload only with t = p = 1    */
     EF_Z3VOL,                           /* 1: ZeRO stage 3 moves 1.5 x V_dp (an option outside the paper; 0 = Section 4.1's rule) */
+    EF_SPREAD,                          /* placement class of the prediction: 0 = packed (one node, or whole nodes);
+                                           a > 0 = spread over several nodes in pieces of a GPUs (Section 4.1: groups
+                                           whose GPUs sit on several nodes communicate at the inter-node bandwidth) */
     EF_COUNT
 };
 
@@ -121,6 +124,12 @@ static int plan_valid(const double *job, const double *env, const int32_t *pl)
     if (off && z < 2) return 0;           /* offload moves partitioned gradients       */
     if (h % t != 0) return 0;             /* the hidden dimension splits evenly        */
     if (env[EF_STRICT] != 0.0 && (z > 0 || off) && (t > 1 || p > 1)) return 0;
+    if (env[EF_SPREAD] != 0.0) {
+        /* spread in pieces of a GPUs: only jobs that one node could hold are spread, in at least two pieces,
+         * and a tensor-parallel group never straddles two pieces */
+        int64_t a = (int64_t)env[EF_SPREAD], g = d * t * p;
+        if (g > Gn || g <= a || g % a != 0 || a % t != 0) return 0;
+    }
     if (pl[PF_GA] < 0 || pl[PF_GA] > 30) return 0;
     if ((imin(b / d, (int64_t)job[JF_MUCAP]) >> pl[PF_GA]) < 1) return 0;   /* a micro-batch holds at least one sample */
     return 1;
@@ -178,6 +187,13 @@ void oracle_terms(const double *job, const double *env, const int32_t *pl, doubl
     double B_tp = env[EF_BINTRA];
     double B_dp = (d * t <= Gn) ? env[EF_BINTRA] : env[EF_BINTER];
     double B_pp = (g <= Gn) ? env[EF_BINTRA] : env[EF_BINTER];
+    if (env[EF_SPREAD] != 0.0) {
+        /* pieces of a GPUs on different nodes: a data-parallel group stays inside a piece only if its d * t
+         * consecutive ranks divide the piece; pipeline stages of different pieces talk across nodes */
+        double a = env[EF_SPREAD];
+        B_dp = fmod(a, d * t) == 0.0 ? env[EF_BINTRA] : env[EF_BINTER];
+        B_pp = env[EF_BINTER];
+    }
     double T_dp = V_dp / B_dp, T_tp = V_tp / B_tp, T_pp = V_pp / B_pp;
 
     /* T_cc: a forwards, a-1 plain backwards, the last backward overlapped with the
@@ -454,7 +470,13 @@ typedef struct {
     /* cluster state */
     int64_t *free_g, *free_c, *free_m;
     int32_t *owner;           /* job holding the whole node as part of a multi-node set, or -1 */
+    /* spread placement classes (none: nK = 0): tables predicted for pieces of align[k] GPUs on several nodes */
+    int nK;
+    const int64_t *align;
+    const float *const *kcv; const int32_t *const *kcp; const int32_t *const *kcg; const uint32_t *const *kfeas;
 } Sched;
+
+#define MAX_PIECES 32         /* a spread job sits on at most this many nodes (gpus per node <= 32) */
 
 typedef struct {
     int gi, ci;               /* level indices, gi = -1 when unallocated */
@@ -463,9 +485,11 @@ typedef struct {
     double val;               /* predicted throughput of the allocation (a float's value in the single-precision form) */
     int status;
     int frozen[2];            /* a rejected GPU / CPU increment is not retried this round */
+    int cls;                  /* -1: packed placement; k >= 0: spread in pieces of align[k] GPUs */
+    int np; int pn[MAX_PIECES], pq[MAX_PIECES];   /* spread: nodes used (ascending) and pieces on each */
 } JobState;
 
-typedef struct { int ok; int k; int stay; int node; int need_new; } Place;
+typedef struct { int ok; int k; int stay; int node; int need_new; int cls; int np; int pn[MAX_PIECES], pq[MAX_PIECES]; } Place;
 
 static size_t cidx(const Sched *S, int j, int gi, int ci, int mi)
 {
@@ -496,15 +520,45 @@ static int count_empty(const Sched *S)
  * lowest-numbered empty ones, with ceil(c2 / k) cores on each. */
 static Place find_place(const Sched *S, const JobState *js, int64_t g2, int64_t c2)
 {
-    Place pl; pl.ok = 0; pl.k = 1; pl.stay = 0; pl.node = -1; pl.need_new = 0;
+    Place pl; pl.ok = 0; pl.k = 1; pl.stay = 0; pl.node = -1; pl.need_new = 0; pl.cls = -1; pl.np = 0;
     int allocated = js->gi >= 0;
+    int spread = allocated && js->cls >= 0;
     if (g2 <= S->Gn) {
-        if (allocated && js->k == 1
+        if (allocated && !spread && js->k == 1
             && S->free_g[js->node] >= g2 - js->g && S->free_c[js->node] >= c2 - js->c) {
             pl.ok = 1; pl.stay = 1; pl.node = js->node; return pl;
         }
+        if (spread && g2 == js->g) {
+            /* more cores for a spread job: it stays where it is when every node it uses has the extra cores */
+            int64_t a = S->align[js->cls];
+            int64_t extra = cdiv(c2 * a, g2) - cdiv(js->c * a, js->g);
+            int fits = 1;
+            for (int i = 0; i < js->np; ++i) if (S->free_c[js->pn[i]] < extra * js->pq[i]) fits = 0;
+            if (fits) {
+                pl.ok = 1; pl.stay = 1; pl.cls = js->cls; pl.np = js->np; pl.node = js->pn[0];
+                for (int i = 0; i < js->np; ++i) { pl.pn[i] = js->pn[i]; pl.pq[i] = js->pq[i]; }
+                return pl;
+            }
+        }
         for (int n = 0; n < S->N; ++n)
             if (S->free_g[n] >= g2 && S->free_c[n] >= c2) { pl.ok = 1; pl.node = n; return pl; }
+        /* No node takes the whole job: assemble it from free pieces on several nodes, in node order, for the
+         * first spread class (they come with the widest pieces first) that finds enough of them.  A piece is
+         * a GPUs with the job's cores shared out evenly, ceil(c a / g) a piece.  What the job holds now is not
+         * counted: it is given back only once the new placement stands. */
+        for (int kx = 0; kx < S->nK; ++kx) {
+            int64_t a = S->align[kx];
+            if (a <= 0 || g2 % a != 0 || g2 <= a) continue;
+            int64_t want = g2 / a, cpp = cdiv(c2 * a, g2);
+            int np = 0; int64_t left = want;
+            for (int n = 0; n < S->N && left > 0 && np < MAX_PIECES; ++n) {
+                int64_t q = imin(S->free_g[n] / a, S->free_c[n] / cpp);
+                if (q <= 0) continue;
+                if (q > left) q = left;
+                pl.pn[np] = n; pl.pq[np] = (int)q; ++np; left -= q;
+            }
+            if (left == 0) { pl.ok = 1; pl.cls = kx; pl.np = np; pl.node = pl.pn[0]; return pl; }
+        }
         return pl;
     }
     if (g2 % S->Gn != 0) return pl;
@@ -512,13 +566,13 @@ static Place find_place(const Sched *S, const JobState *js, int64_t g2, int64_t 
     pl.k = k2;
     if (cdiv(c2, k2) > S->Cn) return pl;
     int empty = count_empty(S);
-    if (allocated && js->g >= S->Gn) {            /* holds whole nodes already */
+    if (allocated && !spread && js->g >= S->Gn) {            /* holds whole nodes already */
         if (k2 == js->k) { pl.ok = 1; pl.stay = 1; pl.node = js->node; return pl; }
         pl.need_new = k2 - js->k;
         pl.stay = 1;
     } else {
         pl.need_new = k2;
-        if (allocated && S->free_g[js->node] + js->g == S->Gn) empty += 1; /* its node empties */
+        if (allocated && !spread && S->free_g[js->node] + js->g == S->Gn) empty += 1; /* its node empties */
     }
     pl.ok = empty >= pl.need_new;
     return pl;
@@ -527,6 +581,16 @@ static Place find_place(const Sched *S, const JobState *js, int64_t g2, int64_t 
 static void release_job(Sched *S, int j, JobState *js)
 {
     if (js->gi < 0) return;
+    if (js->cls >= 0) {
+        /* spread: every piece gives back a GPUs and its even share of the cores and of the memory */
+        int64_t a = S->align[js->cls];
+        int64_t cpp = cdiv(js->c * a, js->g), mpp = cdiv(js->m * a, js->g);
+        for (int i = 0; i < js->np; ++i) {
+            int n = js->pn[i];
+            S->free_g[n] += a * js->pq[i]; S->free_c[n] += cpp * js->pq[i]; S->free_m[n] += mpp * js->pq[i];
+        }
+        return;
+    }
     if (js->k == 1) {
         S->free_g[js->node] += js->g; S->free_c[js->node] += js->c; S->free_m[js->node] += js->m;
     } else {
@@ -539,8 +603,22 @@ static void release_job(Sched *S, int j, JobState *js)
 }
 
 /* highest host-memory level whose per-node share fits the node(s) of placement pl (-1: none) */
-static int commit_level(const Sched *S, const JobState *js, Place pl)
+static int commit_level(const Sched *S, const JobState *js, Place pl, int64_t g2)
 {
+    if (pl.cls >= 0) {
+        /* spread: a level fits when every node holds the share of its pieces, ceil(m a / g) a piece (a job
+         * that stays has its present share of that node on top of what is free) */
+        int64_t a = S->align[pl.cls];
+        int64_t own = (pl.stay && js->gi >= 0) ? cdiv(js->m * a, js->g) : 0;
+        int mi = -1;
+        for (int i = 0; i < S->nM; ++i) {
+            int64_t mpp = cdiv(S->m_levels[i] * a, g2);
+            int fits = 1;
+            for (int q = 0; q < pl.np; ++q) if (mpp * pl.pq[q] > S->free_m[pl.pn[q]] + own * pl.pq[q]) fits = 0;
+            if (fits) mi = i;
+        }
+        return mi;
+    }
     int k2 = pl.k;
     int64_t avail;
     if (k2 > 1) avail = S->Mn;
@@ -559,14 +637,17 @@ static int commit(Sched *S, int j, JobState *js, int gi2, int ci2, Place pl, int
 {
     int64_t g2 = S->g_levels[gi2], c2 = S->c_levels[ci2];
     int k2 = pl.k;
-    int mi = commit_level(S, js, pl);
+    int mi = commit_level(S, js, pl, g2);
     if (mi < 0) return 0;
     size_t o = cidx(S, j, gi2, ci2, mi);
+    /* GetBestPlan for the placement found: a spread placement reads the tables of its class */
     double v = cval(S, o); int plan = S->cp[o]; int gu = S->cg[o];
+    const uint32_t *feas_tab = S->feas;
+    if (pl.cls >= 0) { v = (double)S->kcv[pl.cls][o]; plan = S->kcp[pl.cls][o]; gu = S->kcg[pl.cls][o]; feas_tab = S->kfeas[pl.cls]; }
     if (plan < 0 || !(v > 0.0)) return 0;
     if ((int64_t)gu != g2) return 0;              /* the level's own plans do not fit */
     if (need_gain && js->gi >= 0 && !(v > js->val)) return 0;
-    uint32_t word = S->feas[(size_t)j * S->P + plan];
+    uint32_t word = feas_tab[(size_t)j * S->P + plan];
     int f = 0; while (f < S->nM && !((word >> f) & 1u)) ++f;
     if (f > mi) return 0;
     int64_t m2 = S->m_levels[f];
@@ -579,7 +660,16 @@ static int commit(Sched *S, int j, JobState *js, int gi2, int ci2, Place pl, int
         else for (int n = 0; n < S->N; ++n) if (S->owner[n] == j) keep[nkeep++] = n;
     }
     release_job(S, j, js);
-    if (k2 == 1) {
+    if (pl.cls >= 0) {
+        int64_t a = S->align[pl.cls];
+        int64_t cpp = cdiv(c2 * a, g2), mpp = cdiv(m2 * a, g2);
+        for (int i = 0; i < pl.np; ++i) {
+            int n = pl.pn[i];
+            S->free_g[n] -= a * pl.pq[i]; S->free_c[n] -= cpp * pl.pq[i]; S->free_m[n] -= mpp * pl.pq[i];
+            js->pn[i] = n; js->pq[i] = pl.pq[i];
+        }
+        js->np = pl.np; js->node = pl.pn[0];
+    } else if (k2 == 1) {
         S->free_g[pl.node] -= g2; S->free_c[pl.node] -= c2; S->free_m[pl.node] -= m2;
         js->node = pl.node;
     } else {
@@ -598,7 +688,7 @@ static int commit(Sched *S, int j, JobState *js, int gi2, int ci2, Place pl, int
     }
     free(keep);
     js->gi = gi2; js->ci = ci2; js->g = g2; js->c = c2; js->m = m2;
-    js->plan = plan; js->k = k2; js->val = v; js->status = ST_RUNNING;
+    js->plan = plan; js->k = pl.cls >= 0 ? pl.np : k2; js->val = v; js->status = ST_RUNNING; js->cls = pl.cls;
     return 1;
 }
 
@@ -646,7 +736,7 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
     S.g_levels = g_levels; S.c_levels = c_levels;
     for (int j = 0; j < J; ++j) {
         JobState js; memset(&js, 0, sizeof js);
-        js.gi = -1; js.ci = 0;
+        js.gi = -1; js.ci = 0; js.cls = -1;
         if (state_g[j] > 0) {
             for (int i = 0; i < nG; ++i) if (g_levels[i] == state_g[j]) js.gi = i;
             for (int i = 0; i < nC; ++i) if (c_levels[i] == state_c[j]) js.ci = i;
@@ -669,6 +759,12 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
  * out_i: [J][8] = g, c, m_bytes, plan, first node, node count, status, m level of plan
  * out_val: [J] predicted throughput; node_out: [N][4] = free g, free c, free m, owner
  * step_log (optional, length max_steps): (job << 2) | (type << 1) | accepted.
+ * Spread placement (optional, n_spread > 0; Section 5.2: a job's placement is a list of per-node allocations and
+ * the plan is chosen for the placement found): when no single node takes a job of at most one node's GPUs, it is
+ * assembled from free pieces of spread_align[k] GPUs on several nodes, in node order, for the first class k
+ * that finds enough of them; the commit then reads class k's tables (predicted with the inter-node
+ * bandwidth for every group that leaves a piece).  Gains keep coming from the packed curves, as the cached
+ * slopes of the paper do.  out_pieces [J][32] / out_cls [J] report where such jobs sit.
  * curve_val64 (optional): the curve values in double precision; every decision is then taken in
  * double on that table and out_val64 (optional) receives the values unrounded.
  * cand_out (optional, [J][2][CAND_COUNT] doubles): what every job offered for the decision at which
@@ -687,20 +783,24 @@ int oracle_round(const double *jobs, int J, const double *env,
                  const int64_t *m_levels, int nM, int N, int max_steps,
                  const int64_t *quota, int n_tenants,
                  int64_t *out_i, float *out_val, int64_t *node_out, int32_t *step_log,
-                 const double *curve_val64, double *out_val64, double *cand_out)
+                 const double *curve_val64, double *out_val64, double *cand_out,
+                 int n_spread, const int64_t *spread_align, const float *const *spread_val,
+                 const int32_t *const *spread_plan, const int32_t *const *spread_g, const uint32_t *const *spread_feas,
+                 int32_t *out_pieces, int32_t *out_cls)
 {
     Sched S; memset(&S, 0, sizeof S);
     S.J = J; S.nG = nG; S.nC = nC; S.nM = nM; S.P = P; S.N = N;
     S.cv = curve_val; S.cv64 = curve_val64; S.cp = curve_plan; S.cg = curve_g; S.feas = feas; S.jobs = jobs;
     S.g_levels = g_levels; S.c_levels = c_levels; S.m_levels = m_levels;
     S.Gn = (int64_t)env[EF_GN]; S.Cn = (int64_t)env[EF_CN]; S.Mn = (int64_t)env[EF_MN];
+    S.nK = n_spread; S.align = spread_align; S.kcv = spread_val; S.kcp = spread_plan; S.kcg = spread_g; S.kfeas = spread_feas;
     S.free_g = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
     S.free_c = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
     S.free_m = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
     S.owner = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
     for (int n = 0; n < N; ++n) { S.free_g[n] = S.Gn; S.free_c[n] = S.Cn; S.free_m[n] = S.Mn; S.owner[n] = -1; }
     JobState *st = (JobState *)calloc((size_t)(J > 0 ? J : 1), sizeof(JobState));
-    for (int j = 0; j < J; ++j) { st[j].gi = -1; st[j].plan = -1; st[j].node = -1; st[j].status = ST_UNALLOCATED; }
+    for (int j = 0; j < J; ++j) { st[j].gi = -1; st[j].plan = -1; st[j].node = -1; st[j].status = ST_UNALLOCATED; st[j].cls = -1; }
 
     /* Phase A: guaranteed minima */
     int mt = nM - 1;
@@ -782,9 +882,10 @@ int oracle_round(const double *jobs, int J, const double *env,
                 c[CAND_PLACEABLE] = pl.ok; c[CAND_GI] = gi2; c[CAND_CI] = ci2;
                 c[CAND_MCOMMIT] = -1.0;
                 if (pl.ok && (pl.k > 1 || pl.node >= 0)) {
-                    int mi = commit_level(&S, &st[j], pl);
+                    int mi = commit_level(&S, &st[j], pl, g_levels[gi2]);
                     c[CAND_MCOMMIT] = mi;
-                    if (mi >= 0) { c[CAND_VCOMMIT] = cval(&S, cidx(&S, j, gi2, ci2, mi)); c[CAND_GCOMMIT] = curve_g[cidx(&S, j, gi2, ci2, mi)]; }
+                    if (mi >= 0 && pl.cls < 0) { c[CAND_VCOMMIT] = cval(&S, cidx(&S, j, gi2, ci2, mi)); c[CAND_GCOMMIT] = curve_g[cidx(&S, j, gi2, ci2, mi)]; }
+                    if (mi >= 0 && pl.cls >= 0) { c[CAND_VCOMMIT] = spread_val[pl.cls][cidx(&S, j, gi2, ci2, mi)]; c[CAND_GCOMMIT] = spread_g[pl.cls][cidx(&S, j, gi2, ci2, mi)]; }
                 }
                 c[CAND_VNEXT] = cval(&S, cidx(&S, j, gi2, ci2, mt));
                 c[CAND_UNITS] = type == 0 ? (double)(g_levels[gi2] - (st[j].gi >= 0 ? st[j].g : 0))
@@ -803,6 +904,12 @@ int oracle_round(const double *jobs, int J, const double *env,
         o[7] = f;
         out_val[j] = alloc ? (float)st[j].val : 0.0f;
         if (out_val64) out_val64[j] = alloc ? st[j].val : 0.0;
+        /* where a spread job sits: node << 8 | GPUs there, ascending nodes; -1 = unused entry */
+        if (out_cls) out_cls[j] = alloc ? st[j].cls : -1;
+        if (out_pieces)
+            for (int i = 0; i < MAX_PIECES; ++i)
+                out_pieces[(size_t)j * MAX_PIECES + i] = (alloc && st[j].cls >= 0 && i < st[j].np)
+                    ? (int32_t)((st[j].pn[i] << 8) | (int)(st[j].pq[i] * spread_align[st[j].cls])) : -1;
     }
     if (node_out)
         for (int n = 0; n < N; ++n) {
@@ -891,7 +998,7 @@ static int do_shrink(Sched *S, int v, JobState *js, Shrink sh, int apply)
     if (sh.gi2 < 0) {
         if (apply) {
             release_job(S, v, js);
-            js->gi = -1; js->ci = 0; js->g = js->c = js->m = 0; js->plan = -1; js->node = -1; js->k = 0;
+            js->gi = -1; js->ci = 0; js->g = js->c = js->m = 0; js->plan = -1; js->node = -1; js->k = 0; js->cls = -1;
             js->val = 0.0; js->status = ST_UNALLOCATED;
         }
         return 1;
@@ -899,7 +1006,7 @@ static int do_shrink(Sched *S, int v, JobState *js, Shrink sh, int apply)
     int n = js->node;
     int64_t fg = S->free_g[n], fc = S->free_c[n], fm = S->free_m[n];
     JobState keep = *js;
-    Place pl; pl.ok = 1; pl.k = 1; pl.stay = 1; pl.node = n; pl.need_new = 0;
+    Place pl; pl.ok = 1; pl.k = 1; pl.stay = 1; pl.node = n; pl.need_new = 0; pl.cls = -1; pl.np = 0;
     int ok = commit(S, v, js, sh.gi2, sh.ci2, pl, 0);
     if (!ok || !apply) { S->free_g[n] = fg; S->free_c[n] = fc; S->free_m[n] = fm; *js = keep; }
     return ok;
@@ -944,7 +1051,7 @@ static int exchange(Sched *S, JobState *st, const Roles *R, int j, int gi2, int 
         }
     }
     if (ok) {
-        Place pl; pl.ok = 1; pl.k = 1; pl.stay = on_n; pl.node = n; pl.need_new = 0;
+        Place pl; pl.ok = 1; pl.k = 1; pl.stay = on_n; pl.node = n; pl.need_new = 0; pl.cls = -1; pl.np = 0;
         ok = commit(S, j, &st[j], gi2, ci2, pl, need_gain);
     }
     if (!ok) {
@@ -994,7 +1101,7 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
     /* carried state, minima, gate */
     for (int j = 0; j < J; ++j) {
         const double *job = jobs + (size_t)j * JF_COUNT;
-        st[j].gi = -1; st[j].plan = -1; st[j].node = -1; st[j].status = ST_UNALLOCATED;
+        st[j].gi = -1; st[j].plan = -1; st[j].node = -1; st[j].status = ST_UNALLOCATED; st[j].cls = -1;
         guaranteed[j] = (int)job[JF_GMIN] >= 0;
         min_gi[j] = -1; min_ci[j] = start_ci(job);
         if (guaranteed[j] && (int)job[JF_GMIN] < nG && min_ci[j] < nC) {
