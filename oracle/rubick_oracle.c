@@ -498,6 +498,12 @@ static size_t cidx(const Sched *S, int j, int gi, int ci, int mi)
 
 /* curve value at a table offset, in the precision the decisions are taken in */
 static double cval(const Sched *S, size_t o) { return S->cv64 ? S->cv64[o] : (double)S->cv[o]; }
+/* the same on the curve of the placement class a job holds (a spread job's next steps are measured on the
+ * predictions of its own class, so that an increment is not credited with merely undoing the spreading) */
+static double cval_of(const Sched *S, const JobState *js, size_t o)
+{
+    return (js->gi >= 0 && js->cls >= 0) ? (double)S->kcv[js->cls][o] : cval(S, o);
+}
 
 /* weighted gain per unit, (w v - w v_cur) / units, one rounding per operation */
 static double unit_gain(const Sched *S, double w, double v, double vcur, double units)
@@ -710,7 +716,7 @@ static void job_gains(const Sched *S, int j, const JobState *js, int32_t *next, 
     double cur = allocated ? js->val : 0.0;
     next[0] = next[1] = -1; gain[0] = gain[1] = 0.0;
     for (int gi = js->gi + 1; gi < S->nG; ++gi) {
-        double v = cval(S, cidx(S, j, gi, ci, mt));
+        double v = cval_of(S, js, cidx(S, j, gi, ci, mt));
         if (v > cur) {
             next[0] = gi;
             gain[0] = unit_gain(S, w, v, cur, (double)(S->g_levels[gi] - (allocated ? js->g : 0)));
@@ -718,7 +724,7 @@ static void job_gains(const Sched *S, int j, const JobState *js, int32_t *next, 
         }
     }
     if (allocated && js->ci + 1 < S->nC) {
-        double v = cval(S, cidx(S, j, js->gi, js->ci + 1, mt));
+        double v = cval_of(S, js, cidx(S, j, js->gi, js->ci + 1, mt));
         double gn = unit_gain(S, w, v, cur, (double)(S->c_levels[js->ci + 1] - js->c));
         if (gn > 0.0) { next[1] = js->ci + 1; gain[1] = gn; }
     }
@@ -763,8 +769,8 @@ void oracle_gain(const double *jobs, int J, const float *curve_val,
  * the plan is chosen for the placement found): when no single node takes a job of at most one node's GPUs, it is
  * assembled from free pieces of spread_align[k] GPUs on several nodes, in node order, for the first class k
  * that finds enough of them; the commit then reads class k's tables (predicted with the inter-node
- * bandwidth for every group that leaves a piece).  Gains keep coming from the packed curves, as the cached
- * slopes of the paper do.  out_pieces [J][32] / out_cls [J] report where such jobs sit.
+ * bandwidth for every group that leaves a piece).  The gains of a job that sits in pieces are read off the
+ * curves of its class; everybody else's off the packed curves.  out_pieces [J][32] / out_cls [J] report where such jobs sit.
  * curve_val64 (optional): the curve values in double precision; every decision is then taken in
  * double on that table and out_val64 (optional) receives the values unrounded.
  * cand_out (optional, [J][2][CAND_COUNT] doubles): what every job offered for the decision at which

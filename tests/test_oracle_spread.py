@@ -155,31 +155,33 @@ def test_without_need_the_spread_round_is_the_packed_round(paper_scale):
 
 
 def test_a_job_assembled_from_two_half_free_nodes_by_hand():
-    """Two nodes of 8 GPUs.  Jobs 0 and 1 are guaranteed 6 GPUs each (one node each, 2 GPUs left on either).  Job 2,
-    best effort, gains up to 4 GPUs; no node has 4 free.  Without spread classes it stops at 2 GPUs on node 0; with
-    pieces of 2 it gets 2 + 2 on nodes 0 and 1, at the spread table's value, with cores and memory shared out evenly."""
+    """Two nodes of 8 GPUs.  Jobs 0 and 1 are guaranteed 6 GPUs each and gain nothing beyond (one node each, 2 GPUs
+    left on either).  Job 2, best effort, needs at least 4 GPUs to run at all; no node has 4 free.  Without spread
+    classes it stays in the queue; with pieces of 2 it gets 2 + 2 on nodes 0 and 1, at the spread table's value,
+    with cores and memory shared out evenly."""
     g_levels = np.array([1, 2, 4, 6, 8]); c_levels = np.array([4, 8]); m_levels = np.array([64, 128]) * GIB
     jobs = stack_jobs(one_job(gmin_idx=3, cmin_idx=0), one_job(gmin_idx=3, cmin_idx=0), one_job())
     J, nG, nC, nM, P = 3, 5, 2, 2, 8
-    val = np.array([1.0, 2.0, 3.5, 5.0, 6.0], dtype=np.float32)               # concave in GPUs, flat in cores and memory
-    cv = np.broadcast_to(val[None, :, None, None], (J, nG, nC, nM)).copy()
-    cp = np.broadcast_to(np.arange(nG, dtype=np.int32)[None, :, None, None], (J, nG, nC, nM)).copy()     # plan i serves level i
-    cg = np.broadcast_to(g_levels.astype(np.int32)[None, :, None, None], (J, nG, nC, nM)).copy()
+    # curves (running maximum over GPUs, flat in cores and memory) with the plan and the GPU count they really use
+    val = np.array([[1.0, 2.0, 3.5, 5.0, 5.0], [1.0, 2.0, 3.5, 5.0, 5.0], [0.0, 0.0, 3.5, 3.5, 3.5]], dtype=np.float32)
+    plan = np.array([[0, 1, 2, 3, 3], [0, 1, 2, 3, 3], [-1, -1, 2, 2, 2]], dtype=np.int32)
+    used = np.array([[1, 2, 4, 6, 6], [1, 2, 4, 6, 6], [0, 0, 4, 4, 4]], dtype=np.int32)
+    full = lambda x: np.broadcast_to(x[:, :, None, None], (J, nG, nC, nM)).copy()
+    cv, cp, cg = full(val), full(plan), full(used)
     feas = np.full((J, P), 0b11, dtype=np.uint32)
-    sv = cv * np.float32(0.75)                                                # spread predictions: three quarters of packed
-    sv[:, [0, 1]] = 0                                                         # 1 or 2 GPUs are not spread in pieces of 2
-    sp_, sg = cp.copy(), cg.copy()
-    sp_[:, [0, 1]] = -1; sg[:, [0, 1]] = 0
-    e = env()
-    args = (jobs, e, cv, cp, cg, feas, g_levels, c_levels, m_levels, 2)
+    # spread predictions for pieces of 2: three quarters of the packed value, for 4 GPUs and more
+    sv, sp_, sg = full(val * np.float32(0.75)), full(plan), full(used)
+    sv[:, :2] = 0; sp_[:, :2] = -1; sg[:, :2] = 0
+    args = (jobs, env(), cv, cp, cg, feas, g_levels, c_levels, m_levels, 2)
     plain = oracle.schedule_round(*args, want_log=True)
-    assert list(plain["g"]) == [6, 6, 2] and list(plain["first_node"]) == [0, 1, 0]
+    assert list(plain["g"]) == [6, 6, 0] and list(plain["first_node"]) == [0, 1, -1] and plain["steps"] == 0
     r = oracle.schedule_round(*args, want_log=True, spread=[(2, sv, sp_, sg, feas)])
-    assert list(r["g"]) == [6, 6, 4] and list(r["cls"]) == [-1, -1, 0] and r["n_nodes"][2] == 2
+    assert list(r["g"]) == [6, 6, 4] and list(r["cls"]) == [-1, -1, 0] and r["n_nodes"][2] == 2 and r["first_node"][2] == 0
     assert [int(x) for x in r["pieces"][2] if x >= 0] == [(0 << 8) | 2, (1 << 8) | 2]
-    assert r["thr"][2] == np.float32(3.5 * 0.75) and r["plan"][2] == 2
-    # 4 cores in two pieces: 2 a piece; 64 GiB in two pieces: 32 GiB a piece; the guaranteed jobs hold 6 GPUs and 4 cores each
+    assert r["thr"][2] == np.float32(3.5 * 0.75) and r["plan"][2] == 2 and list(r["log"]) == [(2 << 2) | 1]
+    # 4 cores in two pieces: 2 a piece; 64 GiB in two pieces: 32 GiB a piece; the guaranteed jobs hold 6 GPUs, 4 cores, 64 GiB each
     assert list(r["node"][:, 0]) == [0, 0] and list(r["node"][:, 1]) == [96 - 4 - 2, 96 - 4 - 2]
     assert list(r["node"][:, 2]) == [1024 * GIB - 64 * GIB - 32 * GIB] * 2
-    # the increment from 2 to 4 GPUs was accepted although its value (2.625) is what the packed curve promised less a quarter
-    assert r["steps"] >= plain["steps"]
+    # pieces of 4 cannot be found (2 free GPUs a node): the job stays in the queue
+    none = oracle.schedule_round(*args, want_log=True, spread=[(4, sv, sp_, sg, feas)])
+    assert list(none["g"]) == [6, 6, 0] and (none["cls"] < 0).all()
