@@ -51,6 +51,8 @@ extern "C" {
 #define RUBICK_MAX_NODES     4096    /* node state of a round lives in shared memory */
 #define RUBICK_MAX_TENANTS   256
 #define RUBICK_NOALLOC_MAX_JOBS 32768 /* job limit of rubick_greedy_round_noalloc (1 MiB fixed state) */
+#define RUBICK_MAX_PIECES    32      /* nodes a spread job may sit on (gpus_per_node <= 32 for spread placement) */
+#define RUBICK_MAX_SPREAD_CLASSES 4
 
 /* per-job status in rubick_assignment */
 #define RUBICK_UNALLOCATED 0
@@ -385,6 +387,51 @@ int rubick_schedule_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, cons
  * (and node states, if h_node_out is not NULL) back.  h_jobs / h_out may be pageable or pinned. */
 int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J, const rubick_cluster *h_cluster,
                                int max_steps, rubick_assignment *h_out, rubick_node *h_node_out, int32_t *h_steps);
+
+/* ---- spread placement (Section 4.1: groups whose GPUs sit on several nodes communicate at the inter-node
+ *      bandwidth; Section 5.2 / Algorithm 1: a job's placement is a list of per-node allocations found node by
+ *      node, and the plan is chosen for the placement found) ----------------------------------------------- */
+
+/* Placement class of everything evaluated from now on (rubick_eval_candidates, rubick_curves, rubick_fit_models
+ * and the calls built on them).  align = 0 (the default after rubick_set_space*): packed -- a job of at most
+ * gpus_per_node GPUs on one node, a larger one on whole nodes.  align = a > 0 (a power of two below
+ * gpus_per_node): spread over several nodes in pieces of a GPUs.  Only jobs that one node could hold are spread,
+ * in at least two pieces (a < g <= gpus_per_node, a divides g); a tensor-parallel group never straddles pieces
+ * (t divides a); a data-parallel group stays inside a piece only if d * t divides a, otherwise its ring runs at
+ * B_inter; pipeline traffic always runs at B_inter.  Plans that cannot be spread are invalid in the class
+ * (throughput 0, empty mask).  Host call; the plan tables on the device are rebuilt.  Errors: ESTATE (no plan
+ * space), EINVAL, ENOMEM, ECUDA. */
+int rubick_set_placement(rubick_ctx *ctx, int align);
+
+/* The tables of one spread class, as rubick_curves (or rubick_eval_candidates + rubick_best_plan) wrote them while
+ * rubick_set_placement(ctx, align) was in force.  Device pointers, J * G * C * M entries / J * P words. */
+typedef struct {
+    const float *d_curve_val; const int32_t *d_curve_plan; const int32_t *d_curve_g; const uint32_t *d_feas;
+    int32_t align;
+    int32_t reserved;
+} rubick_spread_class;
+
+/* rubick_greedy_round with spread placement.  The packed tables drive the round as before.  When no node takes a
+ * job of at most gpus_per_node GPUs whole (its own node has no room for the increment and no other node fits
+ * it), the job is assembled from FREE pieces on several nodes: classes in the order given (widest pieces first),
+ * nodes in index order, node n offering min(free GPUs / a, free cores / ceil(c a / g)) pieces, until g / a pieces
+ * are found; what the job holds is given back only once the new placement stands.  The commit then takes the
+ * highest memory level whose per-piece share ceil(m a / g) fits every node used and reads plan and value from
+ * that class's tables; a value that does not improve on the present one rejects the increment as usual.  A job
+ * that sits in pieces measures its next increments on its own class's curves; more cores for it stay on its
+ * nodes when each has them, otherwise it is placed anew (one node, pieces, or whole nodes from empty ones).
+ * d_pieces: J * RUBICK_MAX_PIECES words, node << 8 | GPUs there in ascending node order, -1 = unused;
+ * d_class: J words, -1 = packed, k = spread in the k-th class.  For such a job d_out has first_node = its lowest
+ * node and n_nodes = the number of nodes used; m_bytes is the plan's memory, shared out evenly over the pieces.
+ * n_classes = 0 gives rubick_greedy_round's result.  1 <= gpus_per_node <= 32, no tenant quotas (n_tenants = 0);
+ * one single-CTA kernel that rescans every job per step: meant for clusters of a few hundred jobs.
+ * The context keeps 32 bytes per job of scratch (grown on demand with cudaMalloc). */
+int rubick_greedy_round_spread(rubick_ctx *ctx, const rubick_job *d_jobs, int J,
+                               const float *d_curve_val, const int32_t *d_curve_plan, const int32_t *d_curve_g,
+                               const uint32_t *d_feas, const rubick_spread_class *h_classes, int n_classes,
+                               const rubick_cluster *h_cluster, int max_steps, rubick_assignment *d_out,
+                               rubick_node *d_node_out, int32_t *d_step_log, int32_t *d_pieces, int32_t *d_class,
+                               int32_t *h_steps);
 
 /* ---- measurement aids (the paper has no counterpart) ------------------------------------------- */
 

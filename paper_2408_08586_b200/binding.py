@@ -51,6 +51,14 @@ class Grid(C.Structure):
                 ("m_levels_bytes", C.POINTER(C.c_int64))]
 
 
+class SpreadClass(C.Structure):
+    _fields_ = [("d_curve_val", C.c_void_p), ("d_curve_plan", C.c_void_p), ("d_curve_g", C.c_void_p), ("d_feas", C.c_void_p),
+                ("align", C.c_int32), ("reserved", C.c_int32)]
+
+
+MAX_PIECES = 32
+
+
 class Cluster(C.Structure):
     _fields_ = [("n_nodes", C.c_int32), ("n_tenants", C.c_int32), ("quota_gpus", C.POINTER(C.c_int32)),
                 ("quota_cpus", C.POINTER(C.c_int32))]
@@ -70,7 +78,8 @@ EXPORTS = ["rubick_create", "rubick_destroy", "rubick_sync", "rubick_last_error"
            "rubick_set_space", "rubick_enumerate_plans_wide", "rubick_set_space_wide", "rubick_eval_candidates", "rubick_best_plan", "rubick_curves", "rubick_marginal_gain",
            "rubick_min_resources", "rubick_fit_models",
            "rubick_greedy_round", "rubick_incremental_round", "rubick_greedy_round_noalloc", "rubick_schedule_round",
-           "rubick_schedule_round_host", "rubick_incremental_event_host", "rubick_probe", "rubick_kernel_launches"]
+           "rubick_schedule_round_host", "rubick_incremental_event_host", "rubick_probe", "rubick_kernel_launches",
+           "rubick_set_placement", "rubick_greedy_round_spread"]
 
 _lib = None
 
@@ -114,6 +123,9 @@ def lib():
         L.rubick_schedule_round_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), ip, vp, vp, C.POINTER(C.c_int32)]
         L.rubick_incremental_event_host.argtypes = [vp, vp, ip, C.POINTER(Cluster), vp, ip, vp, C.c_float, ip, ip, vp, vp,
                                                     C.POINTER(C.c_int32)]
+        L.rubick_set_placement.argtypes = [vp, ip]
+        L.rubick_greedy_round_spread.argtypes = [vp, vp, ip, vp, vp, vp, vp, C.POINTER(SpreadClass), ip, C.POINTER(Cluster), ip, vp, vp, vp,
+                                                 vp, vp, C.POINTER(C.c_int32)]
         L.rubick_probe.argtypes = [vp, ip, vp, C.c_size_t, ip, C.POINTER(C.c_double)]
         L.rubick_kernel_launches.argtypes = []
         L.rubick_kernel_launches.restype = C.c_ulonglong
@@ -312,6 +324,25 @@ class Context:
                                                            _ptr(d_curve_plan), _ptr(d_curve_g), _ptr(d_feas), C.byref(cl),
                                                            int(max_steps), _ptr(d_out), _ptr(d_node_out), C.byref(steps)),
                          allow=(ESTEPS,))
+        return steps.value, rc == ESTEPS
+
+    def set_placement(self, align):
+        """rubick_set_placement: 0 = packed, a > 0 = spread over several nodes in pieces of a GPUs."""
+        return self._check(lib().rubick_set_placement(self._h, int(align)))
+
+    def greedy_round_spread(self, d_jobs, J, d_curve_val, d_curve_plan, d_curve_g, d_feas, classes, n_nodes, max_steps, d_out,
+                            d_pieces, d_class, d_node_out=None, d_step_log=None):
+        """rubick_greedy_round_spread.  classes: list of (align, d_curve_val, d_curve_plan, d_curve_g, d_feas) device tensors,
+        widest pieces first.  -> (steps, capped)"""
+        steps = C.c_int32(0)
+        cl, _keep = make_cluster(n_nodes)
+        arr = (SpreadClass * max(len(classes), 1))()
+        for i, (a, v, p, g, f) in enumerate(classes):
+            arr[i] = SpreadClass(_ptr(v), _ptr(p), _ptr(g), _ptr(f), int(a), 0)
+        rc = self._check(lib().rubick_greedy_round_spread(self._h, _ptr(d_jobs), int(J), _ptr(d_curve_val), _ptr(d_curve_plan),
+                                                          _ptr(d_curve_g), _ptr(d_feas), arr if classes else None, len(classes), C.byref(cl),
+                                                          int(max_steps), _ptr(d_out), _ptr(d_node_out), _ptr(d_step_log), _ptr(d_pieces),
+                                                          _ptr(d_class), C.byref(steps)), allow=(ESTEPS,))
         return steps.value, rc == ESTEPS
 
     def schedule_round(self, d_jobs, J, n_nodes, max_steps, d_out, d_node_out=None, quota=None):

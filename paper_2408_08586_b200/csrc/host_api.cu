@@ -151,8 +151,71 @@ int rubick_enumerate_plans(const int32_t *h_g_levels, int nG, rubick_plan *h_out
 
 namespace {
 
-// one plan with its degrees written out (both plan record formats are brought to this form)
-struct NormPlan { int d, t, p, zero, gc, off, g_level, disabled, accum; };
+// Quad tables of a plan list for a placement class (align = 0: packed; a > 0: spread in pieces of a GPUs).
+// Section 4.1: a group whose GPUs sit on several nodes talks at the inter-node bandwidth.  Packed: a job of at
+// most one node's GPUs sits on one node, a larger one on whole nodes (TP fastest, then DP, then PP).  Spread:
+// only jobs one node could hold, in at least two pieces; a tensor-parallel group never straddles pieces (t
+// divides a), a data-parallel group stays inside a piece only if d * t divides it, pipeline stages of different
+// pieces are on different nodes.  Plans that cannot be spread are disabled for the class.
+void build_quads(const std::vector<NormPlan> &plans, const int32_t *g_levels, int Gn, bool wide, int align,
+                 std::vector<QuadDesc> &quads, std::vector<WideQuad> &wquads)
+{
+    const size_t Q = plans.size() / 4;
+    quads.assign(Q, QuadDesc());
+    wquads.assign(wide ? Q : 0, WideQuad());
+    for (size_t i = 0; i < plans.size(); ++i) {
+        const NormPlan &pl = plans[i];
+        const int v = int(i & 3);
+        QuadDesc &q = quads[i >> 2];
+        if (v == 0) {
+            q.log2d = wide ? 0 : uint8_t(ilog2(pl.d)); q.log2t = wide ? 0 : uint8_t(ilog2(pl.t)); q.log2p = wide ? 0 : uint8_t(ilog2(pl.p));
+            q.zero = uint8_t(pl.zero); q.g_level = uint8_t(pl.g_level);
+            q.flags = 0; q.disabled = 0; q.pad = 0;
+            const int64_t d = pl.d, t = pl.t, g = g_levels[pl.g_level];
+            if (align == 0) {
+                if (t <= Gn) q.flags |= QF_T_FITS_NODE;
+                if (d * t > Gn) q.flags |= QF_DP_INTER;
+                if (g > Gn) q.flags |= QF_PP_INTER;
+            } else {
+                const bool may = g <= Gn && g > align && g % align == 0 && align % t == 0;
+                if (may) q.flags |= QF_T_FITS_NODE;
+                if (align % (d * t) != 0) q.flags |= QF_DP_INTER;
+                q.flags |= QF_PP_INTER;
+                if (!may) q.disabled = 0xf;
+            }
+        }
+        if (pl.disabled) q.disabled |= uint8_t(1u << v);
+    }
+    for (size_t i = 0; i < wquads.size(); ++i) {
+        const NormPlan &pl = plans[4 * i];
+        wquads[i].x = uint32_t(pl.d) | (uint32_t(pl.t) << 16);
+        wquads[i].y = uint32_t(pl.p) | (uint32_t(pl.zero) << 16) | (uint32_t(pl.accum) << 24);
+        wquads[i].z = uint32_t(quads[i].flags) | (uint32_t(quads[i].disabled) << 8);
+        wquads[i].w = 0u;
+    }
+}
+
+// uploads quad tables beside the old ones and swaps them in only when everything has succeeded
+int upload_quads(rubick_ctx *ctx, const std::vector<QuadDesc> &quads, const std::vector<WideQuad> &wquads)
+{
+    CUDA_TRY(ctx, cudaSetDevice(ctx->device), "cudaSetDevice");
+    QuadDesc *new_quads = nullptr;
+    WideQuad *new_wide = nullptr;
+    cudaError_t ce = cudaMalloc(reinterpret_cast<void **>(&new_quads), quads.size() * sizeof(QuadDesc));
+    if (ce == cudaSuccess) ce = cudaMemcpy(new_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice);
+    if (ce == cudaSuccess && !wquads.empty()) {
+        ce = cudaMalloc(reinterpret_cast<void **>(&new_wide), wquads.size() * sizeof(WideQuad));
+        if (ce == cudaSuccess) ce = cudaMemcpy(new_wide, wquads.data(), wquads.size() * sizeof(WideQuad), cudaMemcpyHostToDevice);
+    }
+    if (ce != cudaSuccess) {
+        cudaFree(new_quads); cudaFree(new_wide);
+        return cuda_fail(ctx, ce, "plan tables (allocation or upload)");
+    }
+    cudaStreamSynchronize(ctx->stream);         // kernels of earlier calls may still read the old tables
+    cudaFree(ctx->d_quads); cudaFree(ctx->d_wide_quads);
+    ctx->d_quads = new_quads; ctx->d_wide_quads = new_wide;
+    return RUBICK_OK;
+}
 
 int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_grid *h_grid, bool wide)
 {
@@ -189,8 +252,6 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
     for (int i = 0; i < gr.nM; ++i) sp.m_levels[i] = gr.m_levels_bytes[i];
 
     // plans: ordered by level, quads of (gc, off), GPU count = the level's
-    std::vector<QuadDesc> quads(size_t(P) / 4);
-    std::vector<WideQuad> wquads(wide ? size_t(P) / 4 : 0);
     int level = 0;
     sp.group_off[0] = 0;
     for (int i = 0; i < P; ++i) {
@@ -210,57 +271,28 @@ int install_space(rubick_ctx *ctx, const NormPlan *h_plans, int P, const rubick_
         }
         const int v = i & 3;
         if (pl.gc != (v >> 1) || pl.off != (v & 1)) return fail(ctx, RUBICK_EINVAL, "plans: quads must run (gc, off) = (0,0), (0,1), (1,0), (1,1)");
-        QuadDesc &q = quads[size_t(i) >> 2];
-        if (v == 0) {
-            q.log2d = wide ? 0 : uint8_t(ilog2(pl.d)); q.log2t = wide ? 0 : uint8_t(ilog2(pl.t)); q.log2p = wide ? 0 : uint8_t(ilog2(pl.p));
-            q.zero = uint8_t(pl.zero); q.g_level = uint8_t(pl.g_level);
-            q.flags = 0; q.disabled = 0; q.pad = 0;
-            const int64_t d = pl.d, t = pl.t, g = gr.g_levels[pl.g_level];
-            if (t <= Gn) q.flags |= QF_T_FITS_NODE;
-            if (d * t > Gn) q.flags |= QF_DP_INTER;
-            if (g > Gn) q.flags |= QF_PP_INTER;
-        } else {
+        if (v != 0) {
             const NormPlan &first = h_plans[i - v];
             if (first.d != pl.d || first.t != pl.t || first.p != pl.p || first.zero != pl.zero || first.accum != pl.accum)
                 return fail(ctx, RUBICK_EINVAL, "plans: the four plans of a quad must share d, t, p and the ZeRO stage");
         }
-        if (pl.disabled) q.disabled |= uint8_t(1u << v);
     }
     // four consecutive quads = ZeRO stages 0..3 of one (d, t, p) triple (the evaluation kernel's lanes rely on it)
-    if (quads.size() % 4) return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with all four ZeRO stages");
-    for (size_t i = 0; i < quads.size(); ++i) {
-        const QuadDesc &a = quads[i & ~size_t(3)], &b = quads[i];
-        const NormPlan &pa = h_plans[4 * (i & ~size_t(3))], &pb = h_plans[4 * i];
-        if (b.zero != (i & 3) || pa.d != pb.d || pa.t != pb.t || pa.p != pb.p || pa.accum != pb.accum || a.g_level != b.g_level)
+    if ((P / 4) % 4) return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with all four ZeRO stages");
+    for (int i = 0; i < P / 4; ++i) {
+        const NormPlan &pa = h_plans[4 * (i & ~3)], &pb = h_plans[4 * i];
+        if (pb.zero != (i & 3) || pa.d != pb.d || pa.t != pb.t || pa.p != pb.p || pa.accum != pb.accum || pa.g_level != pb.g_level)
             return fail(ctx, RUBICK_EINVAL, "plans: every (d, t, p) must come with ZeRO stages 0..3 in order (disable plans instead of dropping them)");
     }
     while (level < gr.nG) sp.group_off[++level] = P;
-    for (size_t i = 0; i < wquads.size(); ++i) {
-        const NormPlan &pl = h_plans[4 * i];
-        wquads[i].x = uint32_t(pl.d) | (uint32_t(pl.t) << 16);
-        wquads[i].y = uint32_t(pl.p) | (uint32_t(pl.zero) << 16) | (uint32_t(pl.accum) << 24);
-        wquads[i].z = uint32_t(quads[i].flags) | (uint32_t(quads[i].disabled) << 8);
-        wquads[i].w = 0u;
-    }
-
-    // the new tables are built beside the old ones and swapped in only when everything has succeeded: a failed
-    // allocation or upload leaves the context with the plan space it had
-    CUDA_TRY(ctx, cudaSetDevice(ctx->device), "cudaSetDevice");
-    QuadDesc *new_quads = nullptr;
-    WideQuad *new_wide = nullptr;
-    cudaError_t ce = cudaMalloc(reinterpret_cast<void **>(&new_quads), quads.size() * sizeof(QuadDesc));
-    if (ce == cudaSuccess) ce = cudaMemcpy(new_quads, quads.data(), quads.size() * sizeof(QuadDesc), cudaMemcpyHostToDevice);
-    if (ce == cudaSuccess && wide) {
-        ce = cudaMalloc(reinterpret_cast<void **>(&new_wide), wquads.size() * sizeof(WideQuad));
-        if (ce == cudaSuccess) ce = cudaMemcpy(new_wide, wquads.data(), wquads.size() * sizeof(WideQuad), cudaMemcpyHostToDevice);
-    }
-    if (ce != cudaSuccess) {
-        cudaFree(new_quads); cudaFree(new_wide);
-        return cuda_fail(ctx, ce, "plan tables (allocation or upload)");
-    }
-    cudaStreamSynchronize(ctx->stream);         // kernels of earlier calls may still read the old tables
-    cudaFree(ctx->d_quads); cudaFree(ctx->d_wide_quads);
-    ctx->d_quads = new_quads; ctx->d_wide_quads = new_wide;
+    std::vector<NormPlan> kept(h_plans, h_plans + P);
+    std::vector<QuadDesc> quads;
+    std::vector<WideQuad> wquads;
+    build_quads(kept, sp.g_levels, Gn, wide, 0, quads, wquads);
+    int rc = upload_quads(ctx, quads, wquads);
+    if (rc) return rc;
+    ctx->norm_plans.swap(kept);
+    ctx->placement_align = 0;
     ctx->space = sp;
     ctx->inc_J = 0;
     ctx->has_space = true;
@@ -295,6 +327,21 @@ int rubick_set_space_wide(rubick_ctx *ctx, const rubick_plan_wide *h_plans, int 
         np_list[i] = NormPlan{pl.d, pl.t, pl.p, pl.zero, pl.gc, pl.off, pl.g_level, pl.disabled, pl.accum};
     }
     return install_space(ctx, np_list.data(), P, h_grid, true);
+}
+
+int rubick_set_placement(rubick_ctx *ctx, int align)
+{
+    CHECK_CTX(ctx);
+    if (!ctx->has_space) return fail(ctx, RUBICK_ESTATE, "no plan space: call rubick_set_space first");
+    if (align < 0 || align >= ctx->space.Gn || (align & (align - 1))) return fail(ctx, RUBICK_EINVAL, "placement: align must be 0 or a power of two below gpus_per_node");
+    std::vector<QuadDesc> quads;
+    std::vector<WideQuad> wquads;
+    build_quads(ctx->norm_plans, ctx->space.g_levels, ctx->space.Gn, ctx->space.wide != 0, align, quads, wquads);
+    int rc = upload_quads(ctx, quads, wquads);
+    if (rc) return rc;
+    ctx->placement_align = align;
+    ctx->inc_J = 0;                     // cached tables of the incremental events belong to the other class
+    return RUBICK_OK;
 }
 
 int rubick_enumerate_plans_wide(const int32_t *h_g_levels, int nG, int n_accum, rubick_plan_wide *h_out, int cap,

@@ -72,6 +72,9 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
 
 }  // namespace rubick
 
+// one plan with its degrees written out (both plan record formats are brought to this form)
+struct NormPlan { int d, t, p, zero, gc, off, g_level, disabled, accum; };
+
 struct rubick_ctx {
     rubick_env env;
     int device;
@@ -79,6 +82,8 @@ struct rubick_ctx {
     bool has_space;
     rubick::Space space;
     std::vector<rubick_plan> plans;
+    std::vector<NormPlan> norm_plans;   // the installed plan list (rubick_set_placement rebuilds the quad tables from it)
+    int placement_align;                // placement class of the quad tables on the device: 0 packed, a > 0 spread
     rubick::QuadDesc *d_quads;          // [Q]
     rubick::WideQuad *d_wide_quads;     // [Q] only for a wide plan space
     uint32_t *d_status;                 // one word, DS_* bits
