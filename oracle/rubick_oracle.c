@@ -474,6 +474,7 @@ typedef struct {
     int nK;
     const int64_t *align;
     const float *const *kcv; const int32_t *const *kcp; const int32_t *const *kcg; const uint32_t *const *kfeas;
+    int *piece_n, *piece_q;   /* [J][MAX_PIECES], only with spread classes */
 } Sched;
 
 #define MAX_PIECES 32         /* a spread job sits on at most this many nodes (gpus per node <= 32) */
@@ -486,7 +487,8 @@ typedef struct {
     int status;
     int frozen[2];            /* a rejected GPU / CPU increment is not retried this round */
     int cls;                  /* -1: packed placement; k >= 0: spread in pieces of align[k] GPUs */
-    int np; int pn[MAX_PIECES], pq[MAX_PIECES];   /* spread: nodes used (ascending) and pieces on each */
+    int np;                   /* spread: number of nodes used; the nodes (ascending) and the pieces on each are in
+                                 Sched.piece_n / piece_q [job][MAX_PIECES] */
 } JobState;
 
 typedef struct { int ok; int k; int stay; int node; int need_new; int cls; int np; int pn[MAX_PIECES], pq[MAX_PIECES]; } Place;
@@ -524,8 +526,9 @@ static int count_empty(const Sched *S)
  * node when the increment fits there, else the first node (index order) with room for the
  * whole job.  Otherwise g2 / Gn whole nodes: those it already holds entirely plus the
  * lowest-numbered empty ones, with ceil(c2 / k) cores on each. */
-static Place find_place(const Sched *S, const JobState *js, int64_t g2, int64_t c2)
+static Place find_place_of(const Sched *S, int j, const JobState *js, int64_t g2, int64_t c2)
 {
+    const int *jpn = S->piece_n ? S->piece_n + (size_t)j * MAX_PIECES : NULL, *jpq = S->piece_q ? S->piece_q + (size_t)j * MAX_PIECES : NULL;
     Place pl; pl.ok = 0; pl.k = 1; pl.stay = 0; pl.node = -1; pl.need_new = 0; pl.cls = -1; pl.np = 0;
     int allocated = js->gi >= 0;
     int spread = allocated && js->cls >= 0;
@@ -539,10 +542,10 @@ static Place find_place(const Sched *S, const JobState *js, int64_t g2, int64_t 
             int64_t a = S->align[js->cls];
             int64_t extra = cdiv(c2 * a, g2) - cdiv(js->c * a, js->g);
             int fits = 1;
-            for (int i = 0; i < js->np; ++i) if (S->free_c[js->pn[i]] < extra * js->pq[i]) fits = 0;
+            for (int i = 0; i < js->np; ++i) if (S->free_c[jpn[i]] < extra * jpq[i]) fits = 0;
             if (fits) {
-                pl.ok = 1; pl.stay = 1; pl.cls = js->cls; pl.np = js->np; pl.node = js->pn[0];
-                for (int i = 0; i < js->np; ++i) { pl.pn[i] = js->pn[i]; pl.pq[i] = js->pq[i]; }
+                pl.ok = 1; pl.stay = 1; pl.cls = js->cls; pl.np = js->np; pl.node = jpn[0];
+                for (int i = 0; i < js->np; ++i) { pl.pn[i] = jpn[i]; pl.pq[i] = jpq[i]; }
                 return pl;
             }
         }
@@ -591,9 +594,10 @@ static void release_job(Sched *S, int j, JobState *js)
         /* spread: every piece gives back a GPUs and its even share of the cores and of the memory */
         int64_t a = S->align[js->cls];
         int64_t cpp = cdiv(js->c * a, js->g), mpp = cdiv(js->m * a, js->g);
+        const int *jpn = S->piece_n + (size_t)j * MAX_PIECES, *jpq = S->piece_q + (size_t)j * MAX_PIECES;
         for (int i = 0; i < js->np; ++i) {
-            int n = js->pn[i];
-            S->free_g[n] += a * js->pq[i]; S->free_c[n] += cpp * js->pq[i]; S->free_m[n] += mpp * js->pq[i];
+            int n = jpn[i];
+            S->free_g[n] += a * jpq[i]; S->free_c[n] += cpp * jpq[i]; S->free_m[n] += mpp * jpq[i];
         }
         return;
     }
@@ -672,7 +676,7 @@ static int commit(Sched *S, int j, JobState *js, int gi2, int ci2, Place pl, int
         for (int i = 0; i < pl.np; ++i) {
             int n = pl.pn[i];
             S->free_g[n] -= a * pl.pq[i]; S->free_c[n] -= cpp * pl.pq[i]; S->free_m[n] -= mpp * pl.pq[i];
-            js->pn[i] = n; js->pq[i] = pl.pq[i];
+            S->piece_n[(size_t)j * MAX_PIECES + i] = n; S->piece_q[(size_t)j * MAX_PIECES + i] = pl.pq[i];
         }
         js->np = pl.np; js->node = pl.pn[0];
     } else if (k2 == 1) {
@@ -800,6 +804,10 @@ int oracle_round(const double *jobs, int J, const double *env,
     S.g_levels = g_levels; S.c_levels = c_levels; S.m_levels = m_levels;
     S.Gn = (int64_t)env[EF_GN]; S.Cn = (int64_t)env[EF_CN]; S.Mn = (int64_t)env[EF_MN];
     S.nK = n_spread; S.align = spread_align; S.kcv = spread_val; S.kcp = spread_plan; S.kcg = spread_g; S.kfeas = spread_feas;
+    if (n_spread > 0) {
+        S.piece_n = (int *)calloc((size_t)(J > 0 ? J : 1) * MAX_PIECES, sizeof(int));
+        S.piece_q = (int *)calloc((size_t)(J > 0 ? J : 1) * MAX_PIECES, sizeof(int));
+    }
     S.free_g = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
     S.free_c = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
     S.free_m = (int64_t *)malloc(sizeof(int64_t) * (size_t)N);
@@ -833,7 +841,7 @@ int oracle_round(const double *jobs, int J, const double *env,
             if (t < 0 || t >= n_tenants) continue;
             if (rem[2 * t] < g_levels[gi] || rem[2 * t + 1] < c_levels[cmin]) continue;   /* beyond the quota: not privileged */
         }
-        Place pl = find_place(&S, &st[j], g_levels[gi], c_levels[cmin]);
+        Place pl = find_place_of(&S, j, &st[j], g_levels[gi], c_levels[cmin]);
         if (!pl.ok) continue;
         commit(&S, j, &st[j], gi, cmin, pl, 0);
         if (st[j].gi < 0) st[j].status = ST_PENDING;
@@ -853,7 +861,7 @@ int oracle_round(const double *jobs, int J, const double *env,
                 if (next[type] < 0 || !(gain[type] > 0.0)) continue;
                 int gi2 = type == 0 ? next[0] : st[j].gi;
                 int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
-                Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+                Place pl = find_place_of(&S, j, &st[j], g_levels[gi2], c_levels[ci2]);
                 if (!pl.ok) continue;
                 if (gain[type] > best_gain) { best_gain = gain[type]; best_j = j; best_type = type; best_next = next[type]; }
             }
@@ -863,7 +871,7 @@ int oracle_round(const double *jobs, int J, const double *env,
         int j = best_j;
         int gi2 = best_type == 0 ? best_next : st[j].gi;
         int ci2 = best_type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : best_next;
-        Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+        Place pl = find_place_of(&S, j, &st[j], g_levels[gi2], c_levels[ci2]);
         int ok = commit(&S, j, &st[j], gi2, ci2, pl, 1);
         if (!ok) st[j].frozen[best_type] = 1;
         if (step_log) step_log[steps] = (int32_t)((j << 2) | (best_type << 1) | ok);
@@ -884,7 +892,7 @@ int oracle_round(const double *jobs, int J, const double *env,
                 if (next[type] < 0) continue;
                 int gi2 = type == 0 ? next[0] : st[j].gi;
                 int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
-                Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+                Place pl = find_place_of(&S, j, &st[j], g_levels[gi2], c_levels[ci2]);
                 c[CAND_PLACEABLE] = pl.ok; c[CAND_GI] = gi2; c[CAND_CI] = ci2;
                 c[CAND_MCOMMIT] = -1.0;
                 if (pl.ok && (pl.k > 1 || pl.node >= 0)) {
@@ -915,14 +923,14 @@ int oracle_round(const double *jobs, int J, const double *env,
         if (out_pieces)
             for (int i = 0; i < MAX_PIECES; ++i)
                 out_pieces[(size_t)j * MAX_PIECES + i] = (alloc && st[j].cls >= 0 && i < st[j].np)
-                    ? (int32_t)((st[j].pn[i] << 8) | (int)(st[j].pq[i] * spread_align[st[j].cls])) : -1;
+                    ? (int32_t)((S.piece_n[(size_t)j * MAX_PIECES + i] << 8) | (int)(S.piece_q[(size_t)j * MAX_PIECES + i] * spread_align[st[j].cls])) : -1;
     }
     if (node_out)
         for (int n = 0; n < N; ++n) {
             node_out[(size_t)n * 4 + 0] = S.free_g[n]; node_out[(size_t)n * 4 + 1] = S.free_c[n];
             node_out[(size_t)n * 4 + 2] = S.free_m[n]; node_out[(size_t)n * 4 + 3] = S.owner[n];
         }
-    free(S.free_g); free(S.free_c); free(S.free_m); free(S.owner); free(st);
+    free(S.free_g); free(S.free_c); free(S.free_m); free(S.owner); free(st); free(S.piece_n); free(S.piece_q);
     return capped ? -steps - 1 : steps;
 }
 
@@ -1172,7 +1180,7 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
             if (t < 0 || t >= n_tenants) continue;
             if (rem[2 * t] < g_levels[gi] || rem[2 * t + 1] < c_levels[cmin]) continue;
         }
-        Place pl = find_place(&S, &st[j], g_levels[gi], c_levels[cmin]);
+        Place pl = find_place_of(&S, j, &st[j], g_levels[gi], c_levels[cmin]);
         int placed = pl.ok && commit(&S, j, &st[j], gi, cmin, pl, 0);
         if (!placed && g_levels[gi] <= S.Gn)
             for (int n = 0; n < N && !placed; ++n)
@@ -1196,7 +1204,7 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
                     if (pass == 0) {
                         int gi2 = type == 0 ? next[0] : st[j].gi;
                         int ci2 = type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : next[1];
-                        Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+                        Place pl = find_place_of(&S, j, &st[j], g_levels[gi2], c_levels[ci2]);
                         if (!pl.ok) continue;
                     }
                     if (gain[type] > best_gain) { best_gain = gain[type]; best_j = j; best_type = type; best_next = next[type]; by_exchange = pass; }
@@ -1208,7 +1216,7 @@ int oracle_round_incremental(const double *jobs, int J, const double *env,
         int ci2 = best_type == 0 ? (st[j].gi >= 0 ? st[j].ci : start_ci(jobs + (size_t)j * JF_COUNT)) : best_next;
         int ok = 0;
         if (!by_exchange) {
-            Place pl = find_place(&S, &st[j], g_levels[gi2], c_levels[ci2]);
+            Place pl = find_place_of(&S, j, &st[j], g_levels[gi2], c_levels[ci2]);
             ok = commit(&S, j, &st[j], gi2, ci2, pl, 1);
         } else if (g_levels[gi2] <= S.Gn) {
             /* what j gains per unit of each resource it would take from others: a running job only
