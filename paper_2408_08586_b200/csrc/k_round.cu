@@ -818,6 +818,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         v.gc[target] = w_old - ((g2 << 16) + c2);
                         v.free_m[target] = fm - m_need;
                         if (fg_of(w_old) == sp.Gn) sh.n_empty = sh.n_empty - 1;
+                        // the node at the mark has just lost the GPUs the next job of these levels would need: the mark
+                        // moves on at once, and that job looks at the following node without a search
+                        if (sh.ff_pos[gi] == target && fg_of(w_old) - g2 < g2) sh.ff_pos[gi] = target + 1;
                         placed_on = target; settled = true;
                     } else if (v.ml[0] > fm) { pa_fail[gi * sp.nC + ci] = commits; continue; }   // the node found has memory for no level
                 }
