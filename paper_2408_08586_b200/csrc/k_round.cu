@@ -755,6 +755,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // ---- Phase A: guaranteed minima in job order (warp 0) ------------------------------------------
     if (warp == 0) {
         const int ng = sh.n_guar;
+        // the phase's counters live in registers (every lane holds the same values) and go back to shared memory
+        // around the calls that use them there and at the end
+        int commits = sh.pa_commits, n_slots_r = sh.n_slots, n_empty_r = sh.n_empty;
         // lanes fetch 32 list entries at once; they are used one after another.  The records of the next 32 and
         // the list entries of the 32 after them are requested before this batch is worked on.
         int jl = lane < ng ? A.glist[lane] : -1;
@@ -769,11 +772,13 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             // Free resources only shrink during this phase, so a job that cannot be placed now never can:
             // every lane tests its own job against the present tables and only the others take a turn.
             bool may = false;
+            int need_l = 0, cls_l = 0;              // (GPUs << 16 | cores) of the job's minimum; index of its failure mark
             if (idx < ng && a0.x >= 0) {
                 const int g2 = v.gl[a0.x], c2 = v.clv[a0.y];
+                need_l = (g2 << 16) | c2; cls_l = a0.x * sp.nC + a0.y;
                 if (g2 <= sp.Gn) may = v.maxc[a0.x] >= c2;
-                else { const int k2 = g2 >> sp.log2Gn; may = (c2 + k2 - 1) / k2 <= sp.Cn && sh.n_empty >= k2; }
-                may = may && pa_fail[a0.x * sp.nC + a0.y] != sh.pa_commits;
+                else { const int k2 = g2 >> sp.log2Gn; may = (c2 + k2 - 1) / k2 <= sp.Cn && n_empty_r >= k2; }
+                may = may && pa_fail[cls_l] != commits;
             }
             unsigned todo = __ballot_sync(0xffffffffu, may);
             // what a turn needs of its job beyond the cluster's state, worked out by the job's lane: is the curve entry
@@ -790,17 +795,17 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 todo &= todo - 1;
                 const int gi = __shfl_sync(0xffffffffu, a0.x, i), ci = __shfl_sync(0xffffffffu, a0.y, i);
                 const int j = __shfl_sync(0xffffffffu, jl, i);
-                const int tn = __shfl_sync(0xffffffffu, a1.w, i);
+                const int need = __shfl_sync(0xffffffffu, need_l, i), cls = __shfl_sync(0xffffffffu, cls_l, i);
                 const int usable = __shfl_sync(0xffffffffu, int(entry_ok), i);
                 const long long m_need = __shfl_sync(0xffffffffu, m_need_l, i);
-                if (gi < 0) continue;
+                int tn = 0;
                 if (A.n_tenants > 0) {     // privileged only while the minimum fits the tenant's remaining quota
+                    tn = __shfl_sync(0xffffffffu, a1.w, i);
                     if (tn < 0 || tn >= A.n_tenants) continue;
                     if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[ci]) continue;
                 }
-                const int commits = sh.pa_commits;
-                if (pa_fail[gi * sp.nC + ci] == commits) continue;              // same levels, same cluster: same outcome
-                const int g2 = v.gl[gi], c2 = v.clv[ci];
+                if (pa_fail[cls] == commits) continue;              // same levels, same cluster: same outcome
+                const int g2 = need >> 16, c2 = need & 0xffff;
                 int placed_on = -1;
                 bool settled = false;
                 if (g2 <= sp.Gn && usable) {
@@ -811,18 +816,18 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         target = first_fit_from_mark(v, sh, gi, g2, c2, lane);
                         w_old = target >= 0 ? v.gc[target] : 0;
                     }
-                    if (target < 0) { pa_fail[gi * sp.nC + ci] = commits; continue; }      // no node for these levels
+                    if (target < 0) { pa_fail[cls] = commits; continue; }      // no node for these levels
                     const int64_t fm = v.free_m[target];
                     if (m_need <= fm) {
                         // the highest memory level that fits the node is at or above the plan's own: the entry stands
-                        v.gc[target] = w_old - ((g2 << 16) + c2);
+                        v.gc[target] = w_old - need;
                         v.free_m[target] = fm - m_need;
-                        if (fg_of(w_old) == sp.Gn) sh.n_empty = sh.n_empty - 1;
+                        if (fg_of(w_old) == sp.Gn) --n_empty_r;
                         // the node at the mark has just lost the GPUs the next job of these levels would need: the mark
                         // moves on at once, and that job looks at the following node without a search
                         if (sh.ff_pos[gi] == target && fg_of(w_old) - g2 < g2) sh.ff_pos[gi] = target + 1;
                         placed_on = target; settled = true;
-                    } else if (v.ml[0] > fm) { pa_fail[gi * sp.nC + ci] = commits; continue; }   // the node found has memory for no level
+                    } else if (v.ml[0] > fm) { pa_fail[cls] = commits; continue; }   // the node found has memory for no level
                 }
                 const float val_e = __int_as_float(__shfl_sync(0xffffffffu, a0.z, i));
                 const int plan_e = __shfl_sync(0xffffffffu, a0.w, i), f_e = __shfl_sync(0xffffffffu, a1.x, i);
@@ -832,22 +837,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     HotCurve cand;
                     cand.val = val_e; cand.plan = plan_e; cand.f = f_e; cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
                     cm.first = -1;
+                    sh.n_empty = n_empty_r;
                     __syncwarp();
                     settled = commit_warp<false, true>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm);
                     __syncwarp();
+                    n_empty_r = sh.n_empty;
                     if (!settled) {
-                        if (cm.first == -2) pa_fail[gi * sp.nC + ci] = commits;
+                        if (cm.first == -2) pa_fail[cls] = commits;
                         continue;
                     }
                 }
-                const int s = sh.n_slots;
+                const int s = n_slots_r;
                 if (lane == 0) {
                     SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
                     SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
                     v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
                 }
-                sh.n_slots = s + 1;
-                sh.pa_commits = commits + 1;
+                n_slots_r = s + 1;
+                ++commits;
                 if (A.n_tenants > 0) {
                     const int qg = rem_q[2 * tn], qc = rem_q[2 * tn + 1];
                     rem_q[2 * tn] = qg - sp.g_levels[gi]; rem_q[2 * tn + 1] = qc - sp.c_levels[ci];
@@ -857,6 +864,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         }
         // During this phase maxc[] only served as a hint that errs on the generous side (the usual turn does not
         // maintain it; free resources only shrink, so an old entry is never too small): make it exact again.
+        sh.pa_commits = commits; sh.n_slots = n_slots_r; sh.n_empty = n_empty_r;
         __syncwarp();
         rebuild_maxc_warp(sp, v, lane);
     }
