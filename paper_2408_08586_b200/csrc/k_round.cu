@@ -241,7 +241,8 @@ struct Views {
 
 struct Shared {
     uint32_t red_key[32]; int32_t red_j[32]; uint32_t red_pay[32];
-    uint32_t red_key2[32];        // second-best key of the group (keys only: ties are resolved conservatively)
+    uint32_t red_key2[32];        // even entries: largest key a group did not offer (keys only: ties are resolved conservatively);
+                                  // odd entries: largest key among the increments its warp found without a place
     int dirty[32];                // group must rescan: one of its slots (or a class head) changed
     int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
@@ -331,13 +332,28 @@ __device__ int max_cores_warp(const Views &v, int g, int lane)
     return __reduce_max_sync(0xffffffffu, m);
 }
 
-struct Committed { int first; float val; int plan; int f; };      // after a failure: first = -2 if no job with these target levels could have been placed
+struct Committed { int first; float val; int plan; int f; int freed; };      // after a failure: first = -2 if no job with these target levels could have been placed; freed: the job left a node
+
+// warp-cooperative: rebuilds maxc[] like rebuild_maxc_warp and tells whether an entry changed (same answer on every lane)
+__device__ bool rebuild_maxc_changed(const Space &sp, const Views &v, int lane)
+{
+    const int old = lane < sp.n_small ? v.maxc[lane] : 0;
+    __syncwarp();
+    rebuild_maxc_warp(sp, v, lane);
+    __syncwarp();
+    return __any_sync(0xffffffffu, lane < sp.n_small && v.maxc[lane] != old);
+}
+
+// How the caller of commit_warp keeps the derived state current:
+//   COMMIT_TURN   one commit a turn: sh.maxc_dirty / sh.ver and the bitmap of changed nodes tell the block what changed
+//   COMMIT_PHASE_A free resources only shrink: the search starts at the first-fit marks, maxc[] is rebuilt here
+//   COMMIT_CHAIN  several commits a turn: maxc[] is rebuilt here, sh.ver and the bitmap as for COMMIT_TURN
+enum { COMMIT_TURN = 0, COMMIT_PHASE_A = 1, COMMIT_CHAIN = 2 };
 
 // Commit job j to (gi2, ci2); one warp, all lanes, uniform control flow.  `alloc` (compile time): the job holds
 // (gi, ci) on `node` with value val_cur and memory level f_cur.  cand = curve entry of the target at
-// the top memory level.  On success node state and empty-node count are current; maxc[] is rebuilt
-// here when `rebuild`, otherwise sh.maxc_dirty / sh.ver / sh.t0 / sh.t1 tell the block what changed.
-template <bool alloc, bool rebuild>
+// the top memory level.  On success node state and empty-node count are current.
+template <bool alloc, int mode>
 __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const float *__restrict__ cv,
                             const int32_t *__restrict__ cp, const int32_t *__restrict__ cg,
                             const uint32_t *__restrict__ feas, int j, int gi, int ci, int node,
@@ -356,7 +372,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     if (g2 <= sp.Gn) {
         if (alloc) { const int w = v.gc[node]; stay = fg_of(w) >= g2 - g && fc_of(w) >= c2 - c; }
         if (stay) target = node;
-        else if (v.maxc[gi2] >= c2) target = rebuild ? first_fit_from_mark(v, sh, gi2, g2, c2, lane) : first_fit_warp(v, g2, c2, lane);
+        else if (v.maxc[gi2] >= c2) target = mode == COMMIT_PHASE_A ? first_fit_from_mark(v, sh, gi2, g2, c2, lane) : first_fit_warp(v, g2, c2, lane);
         if (target < 0) { out.first = -2; return false; }
     } else {
         k2 = g2 >> sp.log2Gn;
@@ -395,6 +411,7 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
     int first = -1, d_empty = 0;
     bool maxc_dirty = true;
     int t0 = -1, t1 = -1;
+    out.freed = alloc && !stay;
     if (k2 == 1) {
         const int moved = alloc && !stay;
         const int w_old_n = moved ? v.gc[node] : 0, w_old_t = v.gc[target];
@@ -465,9 +482,18 @@ __device__ bool commit_warp(const Space &sp, const Views &v, Shared &sh, const f
         if (n_empty + d_empty > 0) maxc_dirty = __any_sync(0xffffffffu, lane < sp.n_small && v.maxc[lane] != sp.Cn);
     }
     __syncwarp();
-    if (rebuild) {
+    if (mode == COMMIT_PHASE_A) {
         if (maxc_dirty) rebuild_maxc_warp(sp, v, lane);
         if (lane == 0) sh.n_empty = n_empty + d_empty;
+        __syncwarp();
+    } else if (mode == COMMIT_CHAIN) {
+        const bool changed = maxc_dirty && rebuild_maxc_changed(sp, v, lane);
+        if (lane == 0) {
+            sh.n_empty = n_empty + d_empty;
+            if (t0 >= 0) v.tb[t0 >> 5] |= 1u << (t0 & 31);
+            if (t1 >= 0) v.tb[t1 >> 5] |= 1u << (t1 & 31);
+            if (d_empty != 0 || k2 > 1 || changed) sh.ver += 1;
+        }
         __syncwarp();
     } else if (lane == 0) {
         sh.n_empty = n_empty + d_empty;
@@ -609,6 +635,39 @@ round_prepare_kernel(const __grid_constant__ Space sp, const rubick_job *__restr
     }
 }
 
+// The two increments of a running job under the present cluster state: the keys of those that have a place
+// (0 = none) and the larger key among those that have a gain but no place.  w_node = the word of the job's node.
+__device__ __forceinline__ void slot_keys(const Space &sp, const Views &v, int n_empty, const SlotA &a, const SlotC &q, int w_node,
+                                          uint32_t &kg, uint32_t &kc, uint32_t &blocked)
+{
+    const int fg = fg_of(w_node), fc = fc_of(w_node);
+    const int mg = v.maxc[q.gidx], mc = v.maxc[q.cidx];
+    const bool part_empty = fg + q.g == sp.Gn;
+    const bool ok_g = a.gain_g > 0.0f
+                      && (q.gkind == K_SINGLE ? (fg >= q.dg || mg >= q.c)
+                          : q.gkind == K_MULTI_WHOLE ? n_empty >= q.need
+                          : q.gkind == K_MULTI_PART ? n_empty + int(part_empty) >= q.need : false);
+    const bool ok_c = a.gain_c > 0.0f && (q.ckind == K_SINGLE ? (fc >= q.dc || mc >= q.c2) : q.ckind == K_MULTI_WHOLE);
+    kg = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : 0u;
+    kc = ok_c ? __float_as_uint(a.gain_c) : 0u;
+    blocked = 0u;
+    if (!ok_g && a.gain_g > 0.0f) blocked = 0x80000000u | __float_as_uint(a.gain_g);
+    if (!ok_c && a.gain_c > 0.0f) blocked = max(blocked, __float_as_uint(a.gain_c));
+}
+
+// One candidate staged for a chain of commits: everything its commit and its new gains can need.
+//   a, b    the job's slot (class entries: b.w = the job's weight)
+//   cand    curve entry of the target at the top memory level;  t_lo: first half of the target's transition record
+//   m       x = selection key | y = job | z = slot (-1: an unallocated job) | w = target gi | ci << 8 | GPU increment << 16
+//           | the usual commit applies << 17
+//   cur     x = what the job holds, y = what it wants (GPUs << 16 | cores), z = its node (-1: none)
+//   mem     x = memory it holds, y = memory of the target's entry (0 when that entry names no level)
+//   q       the job's present placement needs;  na, nb, nq: its slot once the target's entry is committed as it stands
+struct __align__(16) ChainRec { int4 m, cur; longlong2 mem; int4 na, nb, nq, q, a, b, cand, t_lo; };
+constexpr int CHAIN_SLOTS = N_GROUPS - 1;    // the candidates the scanning warps offer
+constexpr int CHAIN_CLS = 16;                // entries of the best class of unallocated jobs staged per turn
+static_assert(CHAIN_CLS < 32, "lane CHAIN_CLS fetches the key behind the staged entries");
+
 struct RoundArgs {
     const rubick_job *jobs; int J;
     const float *cv; const int32_t *cp; const int32_t *cg; const uint32_t *feas;
@@ -647,6 +706,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // being looked at first as the start of a run of failing heads (either way gives the same steps)
     __shared__ uint32_t cls_went[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS / 32];
     __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];      // what is left of every tenant's quota: GPUs, cores
+    __shared__ ChainRec chain[CHAIN_SLOTS + CHAIN_CLS];    // Phase B: the candidates of a chain of commits, in the rule's order
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
     const int n_cls = sp.nG * sp.nC;
@@ -839,7 +899,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     cm.first = -1;
                     sh.n_empty = n_empty_r;
                     __syncwarp();
-                    settled = commit_warp<false, true>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm);
+                    settled = commit_warp<false, COMMIT_PHASE_A>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm);
                     __syncwarp();
                     n_empty_r = sh.n_empty;
                     if (!settled) {
@@ -886,6 +946,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // sits on, maxc[] or the number of empty nodes.
     uint32_t c_key = 0u, c_key2 = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
     uint32_t c_keyB = 0u, c_payB = 0u; int c_jB = 0x7fffffff;          // scanning warps: their second candidate
+    uint32_t c_blk = 0u;               // largest key among the increments that have a gain but no place at present
     for (;;) {
         if (sh.maxc_dirty) {                                   // uniform: written before the last barrier
             if (warp < sp.n_small) {
@@ -906,7 +967,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             }
             if (rescan) {
                 // the two best candidates of my slots in full, of everything else only the largest key
-                uint32_t k1 = 0u, k2 = 0u, rest = 0u, p1 = 0u, p2 = 0u; int j1 = 0x7fffffff, j2 = 0x7fffffff;
+                uint32_t k1 = 0u, k2 = 0u, rest = 0u, p1 = 0u, p2 = 0u, blk = 0u; int j1 = 0x7fffffff, j2 = 0x7fffffff;
                 for (int s = tid; s < n_slots; s += SCAN_T) {
                     const SlotA a = v.sa[s];
                     const SlotC q = v.sc[s];
@@ -924,6 +985,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     const uint32_t kg = ok_g ? (0x80000000u | __float_as_uint(a.gain_g)) : 0u;
                     const uint32_t kc = ok_c ? __float_as_uint(a.gain_c) : 0u;
                     const uint32_t k32 = ok_g ? kg : kc;
+                    if (!ok_g && a.gain_g > 0.0f) blk = max(blk, 0x80000000u | __float_as_uint(a.gain_g));
+                    if (!ok_c && a.gain_c > 0.0f) blk = max(blk, __float_as_uint(a.gain_c));
                     if (k32 > k1 || (k32 == k1 && k32 && j < j1)) {
                         rest = max(rest, k2); k2 = k1; j2 = j1; p2 = p1; k1 = k32; j1 = j; p1 = uint32_t(s);
                     } else if (k32 > k2 || (k32 == k2 && k32 && j < j2)) {
@@ -939,11 +1002,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 const int src_b = warp_select(b_k, b_j, b_p, hm);
                 const uint32_t left = lane == src_a ? (src_b == src_a ? 0u : k2) : (lane == src_b ? k2 : k1);
                 c_key2 = __reduce_max_sync(hm, max(rest, left));
+                c_blk = __reduce_max_sync(hm, blk);
                 c_key = a_k; c_j = a_j; c_pay = a_p; c_keyB = b_k; c_jB = b_j; c_payB = b_p; my_ver = ver;
                 if (lane == 0) sh.dirty[grp] = 0;
             }
         } else if (rescan) {
-            uint32_t best = 0u, second = 0u, pay = 0u; int best_j = 0x7fffffff;
+            uint32_t best = 0u, second = 0u, pay = 0u, blk = 0u; int best_j = 0x7fffffff;
             const int n_ccls = sh.n_ccls;
             for (int i = lane; i < n_ccls; i += 32) {
                 const int packed = v.ccls[i];
@@ -955,6 +1019,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if (g2 <= sp.Gn) ok = v.maxc[gi2] >= c2;
                     else { const int k2 = g2 >> sp.log2Gn; ok = (c2 + k2 - 1) / k2 <= sp.Cn && n_empty >= k2; }
                     const uint32_t k32 = ok ? (0x80000000u | key_gain_bits(k)) : 0u;
+                    if (!ok) blk = max(blk, 0x80000000u | key_gain_bits(k));
                     const int j = key_job(k);
                     if (k32 > best || (k32 == best && k32 && j < best_j)) { second = best; best = k32; best_j = j; pay = 0x80000000u | uint32_t(t); }
                     else if (k32 > second) second = k32;
@@ -963,12 +1028,14 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             const uint32_t mine = best;
             const int src = warp_select(best, best_j, pay);
             c_key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
+            c_blk = __reduce_max_sync(0xffffffffu, blk);
             c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
             if (lane == 0) sh.dirty[CLS_G] = 0;
         }
         if (lane == 0) {
             sh.red_key[grp] = c_key; sh.red_j[grp] = c_j; sh.red_pay[grp] = c_pay; sh.red_key2[grp] = c_key2;
-            if (warp < SCAN_WARPS) { sh.red_key[grp + 1] = c_keyB; sh.red_j[grp + 1] = c_jB; sh.red_pay[grp + 1] = c_payB; sh.red_key2[grp + 1] = 0u; }
+            if (warp < SCAN_WARPS) { sh.red_key[grp + 1] = c_keyB; sh.red_j[grp + 1] = c_jB; sh.red_pay[grp + 1] = c_payB; }
+            sh.red_key2[grp + 1] = c_blk;            // the odd entries: what each warp found blocked
         }
         __syncthreads();
         if (warp == 0) {
@@ -1101,7 +1168,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 top_stays = __any_sync(FULL, st);
             }
             if (go && n_acc == 0 && top_stays) {
-                const uint32_t M = __reduce_max_sync(FULL, lane < N_GROUPS ? sh.red_key2[lane] : 0u);
+                const uint32_t M = __reduce_max_sync(FULL, !(lane & 1) ? sh.red_key2[lane] : 0u);
                 bool elig = false, s_ok = false, s_maxc = false, s_multi = false;
                 int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0, s_k = 1;
                 int64_t s_dm = 0;
@@ -1259,81 +1326,264 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if (lane == 0) { sh.steps = steps0 + n_acc; sh.maxc_dirty = md ? 1 : 0; }
                 }
             }
+            // ---- a chain of general commits ------------------------------------------------------------------
+            // Whatever the top candidate needs (a migration, growth onto whole nodes, the first placement of an
+            // unallocated job), its commit is worked out by the whole warp on the real cluster state, and so is
+            // every candidate after it for which the order of the sequential rule can be proved: all offered
+            // candidates and the first entries of the best class are fetched in one wave of loads and staged in
+            // shared memory in the rule's order (key, then lowest job); the next one is committed while its key
+            // exceeds every key that was not offered (M), every new candidate of the jobs committed before it in
+            // this turn and, once a commit has given resources back, every increment that had no place before
+            // (it might have one now).  A candidate whose own increment changed under the commits before it
+            // ends the chain, and so does a class that lost its place.
+            // Each lane prepares its candidate for the usual commit -- a job on one node whose target's curve entry
+            // is usable as it stands: what it holds and wants as node words, the memory of both, the slot it will
+            // have afterwards -- so that such a commit only has to find the node, compare the memory and store.
+            // Everything else (whole nodes, an entry that needs the table, too little memory) goes through commit_warp.
             if (go && n_acc == 0) {
-                const int type_gpu = int(best >> 31);
-                const int j = best_j;
-                bool ok;
-                if (pay & 0x80000000u) {
-                    // head of a class of unallocated jobs; consumed whether or not the commit succeeds
-                    const int t = int(pay & 0x7fffffffu);
-                    const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
-                    const float w = v.cls_w[t];
-                    // one round trip: the target's entry and the column the new gains will need
-                    const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                    const int lvl = gi2 + 1 + lane;
-                    const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
-                    const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
-                    const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[0];
-                    const int4 t_hi = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[1];
-                    const int ptr = v.cls_ptr[t] + 1;
-                    u64 nk = 0ull; float nw = 0.0f;
-                    if (ptr < v.cls_end[t]) { nk = A.keys[ptr]; nw = A.sorted_w[ptr]; }
-                    Committed cm;
-                    ok = commit_warp<false, false>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
-                    if (ok) {
-                        // committed with the curve's own value (the usual case): the transition record has the rest
-                        const bool rec = cm.plan == cand.plan && cm.val == cand.val;
-                        int ng_ = t_lo.z, nc_ = t_lo.w; float gg = __int_as_float(t_lo.x), gc = __int_as_float(t_lo.y);
-                        if (!rec) gains_from_column(sp, w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
-                        if (lane == 0) {
-                            const int s = sh.n_slots;
-                            SlotA sa; sa.gain_g = gg; sa.gain_c = gc; sa.packed = pack(gi2, ci2, ng_, false, false); sa.node = cm.first;
-                            SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
-                            v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
-                            v.sc[s] = rec ? *reinterpret_cast<const SlotC *>(&t_hi) : make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
-                            sh.n_slots = s + 1;
-                            sh.dirty[dirty_of(s)] = 1;
+                const uint32_t M = __reduce_max_sync(FULL, !(lane & 1) ? sh.red_key2[lane] : 0u);
+                const uint32_t Mblk = __reduce_max_sync(FULL, (lane & 1) ? sh.red_key2[lane] : 0u);
+                // -- stage the offered candidates of running jobs
+                const bool is_slot = lane < CLS_G && key != 0u;
+                const u64 mine = is_slot ? ((u64(key) << 32) | (u64(uint32_t(KEY_JOB_MASK) - uint32_t(my_j)) << 5) | u64(31 - lane)) : 0ull;
+                sh.sel[lane] = mine;
+                __syncwarp();
+                const int n_sc = __popc(__ballot_sync(FULL, is_slot));
+                if (is_slot) {
+                    int rank = 0;
+#pragma unroll
+                    for (int i = 0; i < CLS_G; ++i) rank += int(sh.sel[i] > mine);
+                    const int s = int(my_pay);
+                    const SlotA a = v.sa[s];
+                    const int type_gpu = int(key >> 31);
+                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+                    const size_t o = hc_idx(sp, my_j, gi2, ci2);
+                    ChainRec &r = chain[rank];
+                    const int4 b4 = *reinterpret_cast<const int4 *>(v.sb + s);
+                    const int4 c4 = *reinterpret_cast<const int4 *>(A.hc + o);
+                    const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + o)[0];
+                    r.nq = reinterpret_cast<const int4 *>(A.tr + o)[1];
+                    r.q = *reinterpret_cast<const int4 *>(&v.sc[s]);
+                    const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+                    const bool f_ok = c4.z >= 0 && c4.z < sp.nM;
+                    const bool cand_ok = c4.y >= 0 && c4.y < sp.P && f_ok && __int_as_float(c4.x) > 0.0f && c4.w != 0
+                                         && __int_as_float(c4.x) > __int_as_float(b4.x);
+                    const bool lean = cand_ok && g <= sp.Gn && g2 <= sp.Gn;
+                    const bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+                    r.a = make_int4(__float_as_int(a.gain_g), __float_as_int(a.gain_c), int(a.packed), a.node);
+                    r.b = b4; r.cand = c4; r.t_lo = t_lo;
+                    r.cur = make_int4((g << 16) | c, (g2 << 16) | c2, a.node, 0);
+                    r.mem = make_longlong2(v.ml[b4.z], f_ok ? v.ml[c4.z] : 0);
+                    r.na = make_int4(fz_g ? 0 : t_lo.x, fz_c ? 0 : t_lo.y, int(pack(gi2, ci2, t_lo.z, fz_g, fz_c)), -1);
+                    r.nb = make_int4(c4.x, c4.y, c4.z, b4.w);
+                    r.m = make_int4(int(key), my_j, s, gi2 | (ci2 << 8) | (type_gpu << 16) | (int(lean) << 17));
+                }
+                // -- and the first entries of the best class of unallocated jobs (its head is the candidate of lane CLS_G)
+                const uint32_t cls_key = __shfl_sync(FULL, key, CLS_G), cls_pay = __shfl_sync(FULL, my_pay, CLS_G);
+                int n_ce = 0, cls_t = -1, cls_ptr0 = 0, cls_end0 = 0;
+                u64 ce_k = 0ull; float ce_w = 0.0f;          // lane i: key and weight of entry i of the class (i <= CHAIN_CLS)
+                if (cls_key != 0u) {
+                    cls_t = int(cls_pay & 0x7fffffffu);
+                    const int gi2 = cls_t / sp.nC, ci2 = cls_t - gi2 * sp.nC;
+                    cls_ptr0 = v.cls_ptr[cls_t]; cls_end0 = v.cls_end[cls_t];
+                    n_ce = min(cls_end0 - cls_ptr0, CHAIN_CLS);
+                    const int idx = cls_ptr0 + lane;
+                    if (lane <= CHAIN_CLS && idx < cls_end0) { ce_k = A.keys[idx]; ce_w = A.sorted_w[idx]; }
+                    if (lane < n_ce) {
+                        const int j = key_job(ce_k);
+                        const size_t o = hc_idx(sp, j, gi2, ci2);
+                        ChainRec &r = chain[CHAIN_SLOTS + lane];
+                        const int4 c4 = *reinterpret_cast<const int4 *>(A.hc + o);
+                        const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + o)[0];
+                        r.nq = reinterpret_cast<const int4 *>(A.tr + o)[1];
+                        const int g2 = v.gl[gi2], c2 = v.clv[ci2];
+                        const bool f_ok = c4.z >= 0 && c4.z < sp.nM;
+                        const bool lean = c4.y >= 0 && c4.y < sp.P && f_ok && __int_as_float(c4.x) > 0.0f && c4.w != 0 && g2 <= sp.Gn;
+                        r.a = make_int4(0, 0, 0, -1);
+                        r.b = make_int4(0, -1, 0, __float_as_int(ce_w));
+                        r.cand = c4; r.t_lo = t_lo; r.q = make_int4(0, 0, 0, 0);
+                        r.cur = make_int4(0, (g2 << 16) | c2, -1, 0);
+                        r.mem = make_longlong2(0, f_ok ? v.ml[c4.z] : 0);
+                        r.na = make_int4(t_lo.x, t_lo.y, int(pack(gi2, ci2, t_lo.z, false, false)), -1);
+                        r.nb = make_int4(c4.x, c4.y, c4.z, __float_as_int(ce_w));
+                        r.m = make_int4(int(0x80000000u | key_gain_bits(ce_k)), j, -1, gi2 | (ci2 << 8) | (1 << 16) | (int(lean) << 17));
+                    }
+                }
+                const uint32_t ce_key32 = ce_k ? (0x80000000u | key_gain_bits(ce_k)) : 0u;
+                __syncwarp();
+
+                int i_s = 0, i_c = 0, done = 0;
+                int ne = sh.n_empty, n_sl = sh.n_slots;          // the same on every lane; shared memory follows every change
+                uint32_t b_new = 0u, b_blk = 0u;       // new candidates of the jobs committed in this turn: with / without a place
+                bool freed = false, last_cls_ok = false;
+                bool cls_open = true;                  // entries of the class are taken until one of them is rejected: a run of
+                                                       // rejections is settled faster by the turn that looks for one
+                while (done < room) {
+                    const bool c_avail = cls_open && i_c < n_ce;
+                    const int4 ms = i_s < n_sc ? chain[i_s].m : make_int4(0, 0x7fffffff, 0, 0);
+                    const int4 mc = c_avail ? chain[CHAIN_SLOTS + i_c].m : make_int4(0, 0x7fffffff, 0, 0);
+                    const bool take_c = uint32_t(mc.x) > uint32_t(ms.x) || (mc.x == ms.x && mc.y < ms.y);
+                    const int4 mx = take_c ? mc : ms;
+                    const uint32_t kx = uint32_t(mx.x);
+                    if (kx == 0u) break;
+                    if (done > 0) {
+                        uint32_t T = max(M, b_new);
+                        if (freed) T = max(T, max(Mblk, b_blk));
+                        // the class's next entry when it is not among the stream heads (not staged, or held back)
+                        if (!c_avail) T = max(T, __shfl_sync(FULL, ce_key32, i_c & 31));
+                        if (!(kx > T)) break;
+                    }
+                    const ChainRec *r = &chain[take_c ? CHAIN_SLOTS + i_c : i_s];
+                    const int j = mx.y, gi2 = mx.w & 0xff, ci2 = (mx.w >> 8) & 0xff, type_gpu = (mx.w >> 16) & 1;
+                    const int4 cur = r->cur;
+                    const int need_old = cur.x, need_new = cur.y, node = cur.z;
+                    const int g2 = need_new >> 16, c2 = need_new & 0xffff;
+                    const int s = take_c ? n_sl : mx.z;
+                    const int w_n = node >= 0 ? v.gc[node] : 0;
+                    SlotA na; SlotC nq;
+                    {
+                        const int4 x = r->na, y = r->nq;
+                        na.gain_g = __int_as_float(x.x); na.gain_c = __int_as_float(x.y); na.packed = uint32_t(x.z); na.node = -1;
+                        nq = *reinterpret_cast<const SlotC *>(&y);
+                    }
+                    if (done > 0) {
+                        if (take_c) {                    // has the class still got a place?
+                            bool has;
+                            if (g2 <= sp.Gn) has = v.maxc[gi2] >= c2;
+                            else { const int k2 = g2 >> sp.log2Gn; has = (c2 + k2 - 1) / k2 <= sp.Cn && ne >= k2; }
+                            if (!has) break;
+                        } else {                         // is this still the job's best increment that has a place?
+                            const int4 ra = r->a, rq = r->q;
+                            SlotA a0; a0.gain_g = __int_as_float(ra.x); a0.gain_c = __int_as_float(ra.y); a0.packed = uint32_t(ra.z); a0.node = node;
+                            uint32_t kg, kc, blk;
+                            slot_keys(sp, v, ne, a0, *reinterpret_cast<const SlotC *>(&rq), w_n, kg, kc, blk);
+                            if ((kg ? kg : kc) != kx) break;
                         }
                     }
-                    if (lane == 0) {
-                        v.cls_ptr[t] = ptr; v.cls_top[t] = nk; v.cls_w[t] = nw; sh.dirty[CLS_G] = 1;
-                        if (ok) cls_went[t >> 5] |= 1u << (t & 31); else cls_went[t >> 5] &= ~(1u << (t & 31));
+                    bool ok = false, settled = false;
+                    int w_new_t = 0;
+                    if ((mx.w >> 17) & 1) {
+                        const int d = need_new - need_old;          // (extra GPUs << 16) + extra cores: neither is negative
+                        const bool stay = node >= 0 && fg_of(w_n) >= (d >> 16) && fc_of(w_n) >= (d & 0xffff);
+                        const int target = stay ? node : (v.maxc[gi2] >= c2 ? first_fit_warp(v, g2, c2, lane) : -1);
+                        if (target >= 0) {
+                            const longlong2 mm = r->mem;            // x = memory held, y = memory of the target's entry
+                            const int w_t = stay ? w_n : v.gc[target];
+                            const int64_t fm = v.free_m[target] + (stay ? mm.x : 0);
+                            if (mm.y <= fm) {
+                                // the highest memory level that fits the node is at or above the plan's own: the entry stands
+                                const bool moved = node >= 0 && !stay;
+                                const int w_new_n = w_n + need_old;
+                                w_new_t = w_t - (stay ? d : need_new);
+                                const int ne0 = ne;
+                                if (moved) {
+                                    v.gc[node] = w_new_n; v.free_m[node] = v.free_m[node] + mm.x;
+                                    if (fg_of(w_new_n) == sp.Gn) { ++ne; if (node < sh.empty_lo) sh.empty_lo = node; }
+                                }
+                                v.gc[target] = w_new_t; v.free_m[target] = fm - mm.y;
+                                if (!stay && fg_of(w_t) == sp.Gn) --ne;
+                                if (lane == 0) {
+                                    if (moved) atomicOr(&v.tb[node >> 5], 1u << (node & 31));
+                                    atomicOr(&v.tb[target >> 5], 1u << (target & 31));
+                                }
+                                // can maxc[] have changed?  lane i answers for GPU level i
+                                bool ch = false;
+                                if (lane < sp.n_small) {
+                                    const int gl = v.gl[lane], mxc = v.maxc[lane];
+                                    const int ot = fg_of(w_t) >= gl ? fc_of(w_t) : -1, nt = fg_of(w_new_t) >= gl ? fc_of(w_new_t) : -1;
+                                    ch = (ot == mxc && nt < ot) || nt > mxc;
+                                    if (moved) {
+                                        const int on = fg_of(w_n) >= gl ? fc_of(w_n) : -1, nn = fg_of(w_new_n) >= gl ? fc_of(w_new_n) : -1;
+                                        ch = ch || (on == mxc && nn < on) || nn > mxc;
+                                    }
+                                    // while an empty node remains every entry equals the node's core count: nothing to recompute
+                                    if (ne > 0) ch = mxc != sp.Cn;
+                                }
+                                bool changed = false;
+                                if (__any_sync(FULL, ch)) { __syncwarp(); changed = rebuild_maxc_changed(sp, v, lane); }
+                                sh.n_empty = ne;
+                                if (lane == 0 && (ne != ne0 || changed)) sh.ver += 1;
+                                na.node = target;
+                                if (lane == 0) {
+                                    v.sa[s] = na; *reinterpret_cast<int4 *>(v.sb + s) = r->nb; v.sc[s] = nq;
+                                    if (take_c) v.sj[s] = j;
+                                    sh.dirty[dirty_of(s)] = 1;
+                                }
+                                if (take_c) { ++n_sl; sh.n_slots = n_sl; }
+                                freed = freed || moved;
+                                ok = true; settled = true;
+                            }
+                        }
                     }
-                } else {
-                    const int s = int(pay);
-                    SlotA a = v.sa[s]; SlotB b = v.sb[s];
-                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
-                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi;
-                    const int ci2 = type_gpu ? ci : ci + 1;
-                    const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                    const int lvl = gi2 + 1 + lane;
-                    const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
-                    const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
-                    const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[0];
-                    const int4 t_hi = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[1];
-                    Committed cm;
-                    ok = commit_warp<true, false>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, gi, ci, a.node, b.val, b.f_level, gi2, ci2, cand, true, lane, cm);
-                    bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+                    if (!settled) {
+                        const int4 rc = r->cand, t_lo = r->t_lo;
+                        HotCurve cand; cand.val = __int_as_float(rc.x); cand.plan = rc.y; cand.f = rc.z; cand.ok = rc.w;
+                        const int4 ra = r->a, rb = r->b;
+                        SlotA a0; a0.gain_g = __int_as_float(ra.x); a0.gain_c = __int_as_float(ra.y); a0.packed = uint32_t(ra.z); a0.node = node;
+                        SlotB nb; nb.val = __int_as_float(rb.x); nb.plan = rb.y; nb.f_level = rb.z; nb.w = __int_as_float(rb.w);
+                        bool fz_g = pk_fz_g(a0.packed), fz_c = pk_fz_c(a0.packed);
+                        Committed cm;
+                        __syncwarp();
+                        if (take_c) ok = commit_warp<false, COMMIT_CHAIN>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi2, ci2, cand, true, lane, cm);
+                        else ok = commit_warp<true, COMMIT_CHAIN>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, pk_gi(a0.packed), pk_ci(a0.packed), node,
+                                                                  nb.val, nb.f_level, gi2, ci2, cand, true, lane, cm);
+                        __syncwarp();
+                        ne = sh.n_empty;
+                        if (ok) {
+                            // committed with the curve's own value (the usual case): the transition record has the rest
+                            const bool rec = cm.plan == cand.plan && cm.val == cand.val;
+                            int ng_ = t_lo.z, nc_ = t_lo.w; float gg = __int_as_float(t_lo.x), gc = __int_as_float(t_lo.y);
+                            if (!rec) {
+                                const int lvl = gi2 + 1 + lane;
+                                const float v_lane = lvl < sp.nG ? A.hc[hc_idx(sp, j, lvl, ci2)].val : 0.0f;
+                                const float vc = ci2 + 1 < sp.nC ? A.hc[hc_idx(sp, j, gi2, ci2 + 1)].val : 0.0f;
+                                gains_from_column(sp, nb.w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
+                                nq = make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
+                            }
+                            na.gain_g = fz_g ? 0.0f : gg; na.gain_c = fz_c ? 0.0f : gc;
+                            na.packed = pack(gi2, ci2, ng_, fz_g, fz_c); na.node = cm.first;
+                            nb.val = cm.val; nb.plan = cm.plan; nb.f_level = cm.f;
+                            if (lane == 0) {
+                                v.sa[s] = na; v.sb[s] = nb; v.sc[s] = nq;
+                                if (take_c) v.sj[s] = j;
+                                sh.dirty[dirty_of(s)] = 1;
+                            }
+                            if (take_c) { ++n_sl; sh.n_slots = n_sl; }
+                            w_new_t = v.gc[na.node];
+                            freed = freed || cm.freed != 0;
+                        } else if (!take_c) {
+                            // rejected: the (job, type) pair is frozen, the other increment stays as it is
+                            if (type_gpu) { fz_g = true; a0.gain_g = 0.0f; } else { fz_c = true; a0.gain_c = 0.0f; }
+                            a0.packed = pack(pk_gi(a0.packed), pk_ci(a0.packed), pk_next_gi(a0.packed), fz_g, fz_c);
+                            if (lane == 0) { v.sa[s] = a0; sh.dirty[dirty_of(s)] = 1; }
+                        }
+                    }
                     if (ok) {
-                        const bool rec = cm.plan == cand.plan && cm.val == cand.val;
-                        int ng_ = t_lo.z, nc_ = t_lo.w; float gg = __int_as_float(t_lo.x), gc = __int_as_float(t_lo.y);
-                        if (!rec) gains_from_column(sp, b.w, gi2, ci2, cm.val, v_lane, vc, lane, ng_, gg, nc_, gc);
-                        a.gain_g = fz_g ? 0.0f : gg; a.gain_c = fz_c ? 0.0f : gc;
-                        a.packed = pack(gi2, ci2, ng_, fz_g, fz_c); a.node = cm.first;
-                        b.val = cm.val; b.plan = cm.plan; b.f_level = cm.f;
-                        if (lane == 0) v.sc[s] = rec ? *reinterpret_cast<const SlotC *>(&t_hi) : make_slotc(sp, v.gl, v.clv, gi2, ci2, ng_, nc_);
-                    } else {
-                        if (type_gpu) { fz_g = true; a.gain_g = 0.0f; } else { fz_c = true; a.gain_c = 0.0f; }
-                        a.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
+                        // what the job wants next, for the candidates after it in this turn
+                        uint32_t kg, kc, blk;
+                        slot_keys(sp, v, ne, na, nq, w_new_t, kg, kc, blk);
+                        b_new = max(b_new, max(kg, kc)); b_blk = max(b_blk, blk);
                     }
-                    if (lane == 0) { v.sa[s] = a; v.sb[s] = b; sh.dirty[dirty_of(s)] = 1; }
+                    if (take_c) { last_cls_ok = ok; if (!ok) cls_open = false; ++i_c; } else ++i_s;
+                    if (lane == 0 && A.step_log) A.step_log[steps0 + done] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
+                    ++done;
                 }
+                // the class moves on past the entries used (consumed whether or not their commits succeeded)
+                const u64 nk = __shfl_sync(FULL, ce_k, i_c & 31);
+                const float nw = __shfl_sync(FULL, ce_w, i_c & 31);
                 if (lane == 0) {
-                    if (A.step_log) A.step_log[sh.steps] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
-                    sh.steps += 1;
+                    if (i_c > 0) {
+                        const int np = cls_ptr0 + i_c;
+                        v.cls_ptr[cls_t] = np; v.cls_top[cls_t] = np < cls_end0 ? nk : 0ull; v.cls_w[cls_t] = np < cls_end0 ? nw : 0.0f;
+                        sh.dirty[CLS_G] = 1;
+                        if (last_cls_ok) cls_went[cls_t >> 5] |= 1u << (cls_t & 31); else cls_went[cls_t >> 5] &= ~(1u << (cls_t & 31));
+                    }
+                    sh.steps = steps0 + done;
                 }
+                n_acc = done;
             }
-            if (lane == 0) sh.stop = go ? 0 : 1;
+            if (lane == 0) sh.stop = (go && n_acc > 0) ? 0 : 1;      // a turn always settles at least one step
         }
         __syncthreads();
         if (sh.stop) break;
