@@ -1447,7 +1447,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         na.gain_g = __int_as_float(x.x); na.gain_c = __int_as_float(x.y); na.packed = uint32_t(x.z); na.node = -1;
                         nq = *reinterpret_cast<const SlotC *>(&y);
                     }
-                    if (done > 0) {
+                    if (done > 0 && !((mx.w >> 17) & 1)) {     // (the usual commit sees by itself whether its increment still has a place)
                         if (take_c) {                    // has the class still got a place?
                             bool has;
                             if (g2 <= sp.Gn) has = v.maxc[gi2] >= c2;
@@ -1466,7 +1466,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if ((mx.w >> 17) & 1) {
                         const int d = need_new - need_old;          // (extra GPUs << 16) + extra cores: neither is negative
                         const bool stay = node >= 0 && fg_of(w_n) >= (d >> 16) && fc_of(w_n) >= (d & 0xffff);
-                        const int target = stay ? node : (v.maxc[gi2] >= c2 ? first_fit_warp(v, g2, c2, lane) : -1);
+                        const bool has = stay || v.maxc[gi2] >= c2;
+                        // The commits before it may have taken the place this increment had.  (An increment of the job that
+                        // had no place can only have got one after resources were given back, and then its key is among
+                        // those the candidate had to exceed.)
+                        if (!has && done > 0) break;
+                        const int target = stay ? node : (has ? first_fit_warp(v, g2, c2, lane) : -1);
                         if (target >= 0) {
                             const longlong2 mm = r->mem;            // x = memory held, y = memory of the target's entry
                             const int w_t = stay ? w_n : v.gc[target];
