@@ -655,6 +655,30 @@ __device__ __forceinline__ void slot_keys(const Space &sp, const Views &v, int n
     if (!ok_c && a.gain_c > 0.0f) blocked = max(blocked, __float_as_uint(a.gain_c));
 }
 
+// The same for values every lane holds alike (a chain of commits): the branches are uniform, so only the tests the
+// job's kinds of increment need are executed.
+__device__ __forceinline__ void slot_keys_uniform(const Space &sp, const Views &v, int n_empty, const SlotA &a, const SlotC &q, int w_node,
+                                                  uint32_t &placed, uint32_t &blocked)
+{
+    placed = 0u; blocked = 0u;
+    const int fg = fg_of(w_node), fc = fc_of(w_node);
+    if (a.gain_g > 0.0f) {
+        bool ok = false;
+        if (q.gkind == K_SINGLE) ok = fg >= q.dg || v.maxc[q.gidx] >= q.c;
+        else if (q.gkind == K_MULTI_PART) ok = n_empty + int(fg + q.g == sp.Gn) >= q.need;
+        else if (q.gkind == K_MULTI_WHOLE) ok = n_empty >= q.need;
+        const uint32_t k = 0x80000000u | __float_as_uint(a.gain_g);
+        if (ok) placed = k; else blocked = k;
+    }
+    if (a.gain_c > 0.0f) {
+        bool ok = false;
+        if (q.ckind == K_SINGLE) ok = fc >= q.dc || v.maxc[q.cidx] >= q.c2;
+        else ok = q.ckind == K_MULTI_WHOLE;
+        const uint32_t k = __float_as_uint(a.gain_c);
+        if (ok) placed = max(placed, k); else blocked = max(blocked, k);
+    }
+}
+
 // One candidate staged for a chain of commits: everything its commit and its new gains can need.
 //   a, b    the job's slot (class entries: b.w = the job's weight)
 //   cand    curve entry of the target at the top memory level;  t_lo: first half of the target's transition record
@@ -1414,7 +1438,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 __syncwarp();
 
                 int i_s = 0, i_c = 0, done = 0;
-                int ne = sh.n_empty, n_sl = sh.n_slots;          // the same on every lane; shared memory follows every change
+                // counters of the block, the same on every lane; shared memory follows every change
+                int ne = sh.n_empty, n_sl = sh.n_slots, e_lo = sh.empty_lo, ver_r = sh.ver;
+                // while an empty node remains and every maxc[] entry is the node's core count no commit on single nodes changes maxc[]
+                bool all_max = __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
+                const int gl_l = lane < sp.n_small ? v.gl[lane] : 0x7fff;      // lane i answers for GPU level i when maxc[] is checked
                 uint32_t b_new = 0u, b_blk = 0u;       // new candidates of the jobs committed in this turn: with / without a place
                 bool freed = false, last_cls_ok = false;
                 bool cls_open = true;                  // entries of the class are taken until one of them is rejected: a run of
@@ -1436,21 +1464,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     }
                     const ChainRec *r = &chain[take_c ? CHAIN_SLOTS + i_c : i_s];
                     const int j = mx.y, gi2 = mx.w & 0xff, ci2 = (mx.w >> 8) & 0xff, type_gpu = (mx.w >> 16) & 1;
+                    const bool lean = (mx.w >> 17) & 1;
+                    // everything the usual commit reads of the record, in one wave
                     const int4 cur = r->cur;
+                    const longlong2 mm = r->mem;            // x = memory held, y = memory of the target's entry
+                    const int4 na4 = r->na, nq4 = r->nq;
                     const int need_old = cur.x, need_new = cur.y, node = cur.z;
                     const int g2 = need_new >> 16, c2 = need_new & 0xffff;
                     const int s = take_c ? n_sl : mx.z;
                     const int w_n = node >= 0 ? v.gc[node] : 0;
+                    const int64_t fm_n = node >= 0 ? v.free_m[node] : 0;
+                    const int mx_t = g2 <= sp.Gn ? v.maxc[gi2] : -1;
                     SlotA na; SlotC nq;
-                    {
-                        const int4 x = r->na, y = r->nq;
-                        na.gain_g = __int_as_float(x.x); na.gain_c = __int_as_float(x.y); na.packed = uint32_t(x.z); na.node = -1;
-                        nq = *reinterpret_cast<const SlotC *>(&y);
-                    }
-                    if (done > 0 && !((mx.w >> 17) & 1)) {     // (the usual commit sees by itself whether its increment still has a place)
+                    na.gain_g = __int_as_float(na4.x); na.gain_c = __int_as_float(na4.y); na.packed = uint32_t(na4.z); na.node = -1;
+                    nq = *reinterpret_cast<const SlotC *>(&nq4);
+                    if (done > 0 && !lean) {             // (the usual commit sees by itself whether its increment still has a place)
                         if (take_c) {                    // has the class still got a place?
                             bool has;
-                            if (g2 <= sp.Gn) has = v.maxc[gi2] >= c2;
+                            if (g2 <= sp.Gn) has = mx_t >= c2;
                             else { const int k2 = g2 >> sp.log2Gn; has = (c2 + k2 - 1) / k2 <= sp.Cn && ne >= k2; }
                             if (!has) break;
                         } else {                         // is this still the job's best increment that has a place?
@@ -1463,19 +1494,19 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     }
                     bool ok = false, settled = false;
                     int w_new_t = 0;
-                    if ((mx.w >> 17) & 1) {
+                    if (lean) {
                         const int d = need_new - need_old;          // (extra GPUs << 16) + extra cores: neither is negative
                         const bool stay = node >= 0 && fg_of(w_n) >= (d >> 16) && fc_of(w_n) >= (d & 0xffff);
-                        const bool has = stay || v.maxc[gi2] >= c2;
+                        const bool has = stay || mx_t >= c2;
                         // The commits before it may have taken the place this increment had.  (An increment of the job that
                         // had no place can only have got one after resources were given back, and then its key is among
                         // those the candidate had to exceed.)
                         if (!has && done > 0) break;
                         const int target = stay ? node : (has ? first_fit_warp(v, g2, c2, lane) : -1);
                         if (target >= 0) {
-                            const longlong2 mm = r->mem;            // x = memory held, y = memory of the target's entry
                             const int w_t = stay ? w_n : v.gc[target];
-                            const int64_t fm = v.free_m[target] + (stay ? mm.x : 0);
+                            const int64_t fm = stay ? fm_n + mm.x : v.free_m[target];
+                            const int mxc = lane < sp.n_small ? v.maxc[lane] : -1;
                             if (mm.y <= fm) {
                                 // the highest memory level that fits the node is at or above the plan's own: the entry stands
                                 const bool moved = node >= 0 && !stay;
@@ -1483,39 +1514,41 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                                 w_new_t = w_t - (stay ? d : need_new);
                                 const int ne0 = ne;
                                 if (moved) {
-                                    v.gc[node] = w_new_n; v.free_m[node] = v.free_m[node] + mm.x;
-                                    if (fg_of(w_new_n) == sp.Gn) { ++ne; if (node < sh.empty_lo) sh.empty_lo = node; }
+                                    v.gc[node] = w_new_n; v.free_m[node] = fm_n + mm.x;
+                                    if (fg_of(w_new_n) == sp.Gn) { ++ne; if (node < e_lo) { e_lo = node; sh.empty_lo = node; } }
                                 }
                                 v.gc[target] = w_new_t; v.free_m[target] = fm - mm.y;
                                 if (!stay && fg_of(w_t) == sp.Gn) --ne;
+                                // can maxc[] have changed?
+                                bool ch;
+                                if (ne > 0) ch = !all_max;          // (then every entry is the node's core count)
+                                else {
+                                    const int ot = fg_of(w_t) >= gl_l ? fc_of(w_t) : -1, nt = fg_of(w_new_t) >= gl_l ? fc_of(w_new_t) : -1;
+                                    bool c1 = (ot == mxc && nt < ot) || nt > mxc;
+                                    if (moved) {
+                                        const int on = fg_of(w_n) >= gl_l ? fc_of(w_n) : -1, nn = fg_of(w_new_n) >= gl_l ? fc_of(w_new_n) : -1;
+                                        c1 = c1 || (on == mxc && nn < on) || nn > mxc;
+                                    }
+                                    ch = __any_sync(FULL, c1);
+                                }
+                                bool changed = false;
+                                if (ch) {
+                                    __syncwarp();
+                                    changed = rebuild_maxc_changed(sp, v, lane);
+                                    all_max = __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
+                                }
+                                if (ne != ne0) sh.n_empty = ne;
+                                if (ne != ne0 || changed) { ++ver_r; sh.ver = ver_r; }
+                                na.node = target;
+                                if (take_c) { ++n_sl; sh.n_slots = n_sl; }
                                 if (lane == 0) {
                                     if (moved) atomicOr(&v.tb[node >> 5], 1u << (node & 31));
                                     atomicOr(&v.tb[target >> 5], 1u << (target & 31));
-                                }
-                                // can maxc[] have changed?  lane i answers for GPU level i
-                                bool ch = false;
-                                if (lane < sp.n_small) {
-                                    const int gl = v.gl[lane], mxc = v.maxc[lane];
-                                    const int ot = fg_of(w_t) >= gl ? fc_of(w_t) : -1, nt = fg_of(w_new_t) >= gl ? fc_of(w_new_t) : -1;
-                                    ch = (ot == mxc && nt < ot) || nt > mxc;
-                                    if (moved) {
-                                        const int on = fg_of(w_n) >= gl ? fc_of(w_n) : -1, nn = fg_of(w_new_n) >= gl ? fc_of(w_new_n) : -1;
-                                        ch = ch || (on == mxc && nn < on) || nn > mxc;
-                                    }
-                                    // while an empty node remains every entry equals the node's core count: nothing to recompute
-                                    if (ne > 0) ch = mxc != sp.Cn;
-                                }
-                                bool changed = false;
-                                if (__any_sync(FULL, ch)) { __syncwarp(); changed = rebuild_maxc_changed(sp, v, lane); }
-                                sh.n_empty = ne;
-                                if (lane == 0 && (ne != ne0 || changed)) sh.ver += 1;
-                                na.node = target;
-                                if (lane == 0) {
                                     v.sa[s] = na; *reinterpret_cast<int4 *>(v.sb + s) = r->nb; v.sc[s] = nq;
                                     if (take_c) v.sj[s] = j;
                                     sh.dirty[dirty_of(s)] = 1;
+                                    if (A.step_log) A.step_log[steps0 + done] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | 1;
                                 }
-                                if (take_c) { ++n_sl; sh.n_slots = n_sl; }
                                 freed = freed || moved;
                                 ok = true; settled = true;
                             }
@@ -1534,7 +1567,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         else ok = commit_warp<true, COMMIT_CHAIN>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, pk_gi(a0.packed), pk_ci(a0.packed), node,
                                                                   nb.val, nb.f_level, gi2, ci2, cand, true, lane, cm);
                         __syncwarp();
-                        ne = sh.n_empty;
+                        ne = sh.n_empty; e_lo = sh.empty_lo; ver_r = sh.ver;
+                        all_max = __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
                         if (ok) {
                             // committed with the curve's own value (the usual case): the transition record has the rest
                             const bool rec = cm.plan == cand.plan && cm.val == cand.val;
@@ -1563,15 +1597,15 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             a0.packed = pack(pk_gi(a0.packed), pk_ci(a0.packed), pk_next_gi(a0.packed), fz_g, fz_c);
                             if (lane == 0) { v.sa[s] = a0; sh.dirty[dirty_of(s)] = 1; }
                         }
+                        if (lane == 0 && A.step_log) A.step_log[steps0 + done] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
                     }
                     if (ok) {
                         // what the job wants next, for the candidates after it in this turn
-                        uint32_t kg, kc, blk;
-                        slot_keys(sp, v, ne, na, nq, w_new_t, kg, kc, blk);
-                        b_new = max(b_new, max(kg, kc)); b_blk = max(b_blk, blk);
+                        uint32_t kp, blk;
+                        slot_keys_uniform(sp, v, ne, na, nq, w_new_t, kp, blk);
+                        b_new = max(b_new, kp); b_blk = max(b_blk, blk);
                     }
                     if (take_c) { last_cls_ok = ok; if (!ok) cls_open = false; ++i_c; } else ++i_s;
-                    if (lane == 0 && A.step_log) A.step_log[steps0 + done] = (j << 2) | ((type_gpu ? 0 : 1) << 1) | int(ok);
                     ++done;
                 }
                 // the class moves on past the entries used (consumed whether or not their commits succeeded)
