@@ -100,6 +100,15 @@ __device__ __forceinline__ HotCurve load_hc(const HotCurve *p)
     return h;
 }
 
+// Requests the curve entry and the transition record of (j, gi, ci) into the L1 cache: the job that was just committed
+// may offer this allocation as its next candidate, and the turn that works the candidate out then finds them near.
+__device__ __forceinline__ void prefetch_target(const Space &sp, const HotCurve *hc, const void *tr32, int j, int gi, int ci)
+{
+    const size_t o = hc_idx(sp, j, gi, ci);
+    asm volatile("prefetch.global.L1 [%0];" :: "l"(hc + o));
+    asm volatile("prefetch.global.L1 [%0];" :: "l"(static_cast<const char *>(tr32) + o * 32));
+}
+
 // ---- keys: first increment of every best-effort job, Phase-A target of every guaranteed job -------
 __global__ void round_keys_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, int J,
                                   const HotCurve *__restrict__ hc, const int32_t *__restrict__ cp,
@@ -758,7 +767,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         v.sc = reinterpret_cast<SlotC *>(p); p += size_t(A.slot_cap) * sizeof(SlotC);
         v.sj = reinterpret_cast<int32_t *>(p);
     } else { v.sa = A.sa_g; v.sc = A.sc_g; v.sj = A.sj_g; }
-    v.sb = A.sb_g;          // value / plan / memory level / weight: touched only by commits, kept in global memory
+    // value / plan / memory level / weight: touched only by commits, kept in global memory (shared memory taken for them
+    // would come out of the L1 cache the curve entries and transition records are requested into)
+    v.sb = A.sb_g;
 
     // ---- set-up ---------------------------------------------------------------------------------
     for (int n = tid; n < v.N_pad; n += RT) v.gc[n] = n < N ? ((sp.Gn << 16) | sp.Cn) : 0;
@@ -1328,6 +1339,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         sh.dirty[dirty_of(s_slot)] = 1;
                         if (s_ok && !s_multi) atomicOr(&v.tb[s_node >> 5], 1u << (s_node & 31));
                         if (A.step_log) A.step_log[steps0 + my_order] = (my_j << 2) | ((s_type ? 0 : 1) << 1) | int(s_ok);
+                        if (s_ok) {
+                            const int ng_ = pk_next_gi(na.packed), gi_ = pk_gi(na.packed), ci_ = pk_ci(na.packed);
+                            if (na.gain_g > 0.0f && ng_ >= 0) prefetch_target(sp, A.hc, A.tr, my_j, ng_, ci_);
+                            if (na.gain_c > 0.0f && ci_ + 1 < sp.nC) prefetch_target(sp, A.hc, A.tr, my_j, gi_, ci_ + 1);
+                        }
                     }
                     // jobs on whole nodes: every node they own changes its share (no other job lives there)
                     unsigned mm = __ballot_sync(FULL, ((acc >> lane) & 1u) && s_ok && s_multi);
@@ -1604,6 +1620,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         uint32_t kp, blk;
                         slot_keys_uniform(sp, v, ne, na, nq, w_new_t, kp, blk);
                         b_new = max(b_new, kp); b_blk = max(b_blk, blk);
+
                     }
                     if (take_c) { last_cls_ok = ok; if (!ok) cls_open = false; ++i_c; } else ++i_s;
                     ++done;
