@@ -225,11 +225,13 @@ enum : uint8_t { K_SINGLE = 0, K_MULTI_WHOLE = 1, K_MULTI_PART = 2, K_NONE = 3 }
 
 constexpr int SCAN_WARPS = RW - 1;          // all warps but the last scan running jobs, the last one the class heads
 constexpr int SCAN_T = SCAN_WARPS * 32;
-constexpr int N_GROUPS = 2 * SCAN_WARPS + 1;   // candidates seen by warp 0: the two best of every scanning warp + the best class head
+constexpr int OFFER = 4;                    // candidates every scanning warp offers
+constexpr int N_GROUPS = OFFER * SCAN_WARPS + 1;   // candidates seen by warp 0: the best OFFER of every scanning warp + the best class head
 constexpr int CLS_G = N_GROUPS - 1;
-static_assert(N_GROUPS <= 32, "warp 0 holds one candidate per lane");
+constexpr int N_CAND = 64;                  // warp 0 holds two candidates per lane: lane l those of index l and l + 32
+static_assert(N_GROUPS <= N_CAND, "warp 0 holds two candidates per lane");
 // the flag that makes the warp owning slot s look again (flags sit at the index of the warp's first candidate)
-__device__ __forceinline__ int dirty_of(int s) { return ((s % SCAN_T) >> 5) << 1; }
+__device__ __forceinline__ int dirty_of(int s) { return ((s % SCAN_T) >> 5) * OFFER; }
 
 // node n: gc[n] = free GPUs << 16 | free cores (padding entries are 0: they never fit anything)
 __device__ __forceinline__ int fg_of(int w) { return w >> 16; }
@@ -249,10 +251,10 @@ struct Views {
 };
 
 struct Shared {
-    uint32_t red_key[32]; int32_t red_j[32]; uint32_t red_pay[32];
-    uint32_t red_key2[32];        // even entries: largest key a group did not offer (keys only: ties are resolved conservatively);
-                                  // odd entries: largest key among the increments its warp found without a place
-    int dirty[32];                // group must rescan: one of its slots (or a class head) changed
+    uint32_t red_key[N_CAND]; int32_t red_j[N_CAND]; uint32_t red_pay[N_CAND];   // the offered candidates; they stay until their warp looks again
+    uint32_t red_key2[N_CAND];    // at a warp's first index: largest key it did not offer (keys only: ties are resolved conservatively);
+                                  // at the next: largest key among the increments it found without a place
+    int dirty[N_CAND];            // (at a warp's first index) must look again: one of its slots (or a class head) changed
     int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
@@ -261,7 +263,7 @@ struct Shared {
     int4 pa_rec[32][2]; int pa_job[32];   // Phase A: the records of the 32 jobs being worked on
     int pa_commits;               // Phase A: jobs placed so far
     int ff_pos[RUBICK_MAX_G_LEVELS];   // Phase A: no node below this index has g_levels[i] free GPUs
-    unsigned long long sel[32];   // batch selection: one ordering word per lane
+    alignas(16) unsigned long long sel[N_CAND];   // batch selection: one ordering word per candidate (read two at a time)
 };
 
 // warp-cooperative: first node with at least g free GPUs and c free cores, -1 if none
@@ -689,15 +691,16 @@ __device__ __forceinline__ void slot_keys_uniform(const Space &sp, const Views &
 }
 
 // One candidate staged for a chain of commits: everything its commit and its new gains can need.
-//   a, b    the job's slot (class entries: b.w = the job's weight)
+//   b       value, plan, memory level and weight the job has (class entries: only the weight)
 //   cand    curve entry of the target at the top memory level;  t_lo: first half of the target's transition record
 //   m       x = selection key | y = job | z = slot (-1: an unallocated job) | w = target gi | ci << 8 | GPU increment << 16
 //           | the usual commit applies << 17
 //   cur     x = what the job holds, y = what it wants (GPUs << 16 | cores), z = its node (-1: none)
 //   mem     x = memory it holds, y = memory of the target's entry (0 when that entry names no level)
-//   q       the job's present placement needs;  na, nb, nq: its slot once the target's entry is committed as it stands
-struct __align__(16) ChainRec { int4 m, cur; longlong2 mem; int4 na, nb, nq, q, a, b, cand, t_lo; };
+//   na, nb, nq   its slot once the target's entry is committed as it stands
+struct __align__(16) ChainRec { int4 m, cur; longlong2 mem; int4 na, nb, nq, b, cand, t_lo; };
 constexpr int CHAIN_SLOTS = N_GROUPS - 1;    // the candidates the scanning warps offer
+constexpr int CLAIMS = 512;                  // entries of the table that finds candidates of a batch on the same node
 constexpr int CHAIN_CLS = 16;                // entries of the best class of unallocated jobs staged per turn
 static_assert(CHAIN_CLS < 32, "lane CHAIN_CLS fetches the key behind the staged entries");
 
@@ -734,12 +737,21 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     __shared__ Shared sh;
     // Phase A: pa_fail[gi * nC + ci] = number of jobs placed when a job with these target levels last found no node
     // or a node without memory for any level; while nothing else has been placed since, the next one fares the same
-    __shared__ int pa_fail[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS];
+    // (shares its memory with what only Phase B uses)
+    constexpr size_t PA_BYTES = (size_t(RUBICK_MAX_G_LEVELS) * RUBICK_MAX_C_LEVELS + 2 * RUBICK_MAX_TENANTS) * 4;
+    constexpr size_t PB_BYTES = sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS) + size_t(N_CAND) * 48 + size_t(CLAIMS) * 8;
+    __shared__ __align__(16) unsigned char phase_buf[PA_BYTES > PB_BYTES ? PA_BYTES : PB_BYTES];
+    int *pa_fail = reinterpret_cast<int *>(phase_buf);
     // Phase B: bit t set = the last head of class t was placed; the next one is then tried directly instead of
     // being looked at first as the start of a run of failing heads (either way gives the same steps)
     __shared__ uint32_t cls_went[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS / 32];
-    __shared__ int32_t rem_q[2 * RUBICK_MAX_TENANTS];      // what is left of every tenant's quota: GPUs, cores
-    __shared__ ChainRec chain[CHAIN_SLOTS + CHAIN_CLS];    // Phase B: the candidates of a chain of commits, in the rule's order
+    int32_t *rem_q = pa_fail + RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS;      // what is left of every tenant's quota: GPUs, cores
+    // Phase B: the candidates of a chain of commits, in the rule's order; the slots the candidates of a batch will have;
+    // the table that finds candidates of a batch on the same node (highest key, lowest job among equal keys)
+    ChainRec *chain = reinterpret_cast<ChainRec *>(phase_buf);
+    int4 *bst = reinterpret_cast<int4 *>(phase_buf + sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS));
+    uint32_t *claim_k = reinterpret_cast<uint32_t *>(phase_buf + sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS) + size_t(N_CAND) * 48);
+    int32_t *claim_j = reinterpret_cast<int32_t *>(claim_k + CLAIMS);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
     const int n_cls = sp.nG * sp.nC;
@@ -780,7 +792,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     if (tid < sp.nM) ml_s[tid] = sp.m_levels[tid];
     for (int i = tid; i < v.N_pad / 32; i += RT) tb_s[i] = 0u;
     if (tid < sp.n_small) v.maxc[tid] = sp.Cn;                              // every node is empty
-    if (tid < 32) sh.dirty[tid] = 1;
+    if (tid < N_CAND) { sh.dirty[tid] = 1; sh.red_key[tid] = 0u; sh.red_j[tid] = 0x7fffffff; sh.red_pay[tid] = 0u; sh.red_key2[tid] = 0u; }
     if (tid < RUBICK_MAX_G_LEVELS) sh.ff_pos[tid] = 0;
     for (int t = tid; t < n_cls; t += RT) pa_fail[t] = -1;
     for (int t = tid; t < RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS / 32; t += RT) cls_went[t] = 0u;
@@ -964,6 +976,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         rebuild_maxc_warp(sp, v, lane);
     }
     __syncthreads();
+    for (int i = tid; i < CLAIMS; i += RT) { claim_k[i] = 0u; claim_j[i] = 0x7fffffff; }
     // gains of the jobs placed in Phase A
     for (int s = tid; s < sh.n_slots; s += RT) {
         SlotA a = v.sa[s]; const SlotB b = v.sb[s];
@@ -976,12 +989,10 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     __syncthreads();
 
     // ---- Phase B ---------------------------------------------------------------------------------------
-    // Every warp remembers the two best candidates among its own slots (the last warp: the best class head) and
-    // looks again only when something it depends on changed: one of its slots, a node one of its slots
+    // Every warp leaves the best OFFER candidates among its own slots in shared memory (the last warp: the best class
+    // head) and looks again only when something it depends on changed: one of its slots, a node one of its slots
     // sits on, maxc[] or the number of empty nodes.
-    uint32_t c_key = 0u, c_key2 = 0u, c_pay = 0u; int c_j = 0x7fffffff; int my_ver = -1;
-    uint32_t c_keyB = 0u, c_payB = 0u; int c_jB = 0x7fffffff;          // scanning warps: their second candidate
-    uint32_t c_blk = 0u;               // largest key among the increments that have a gain but no place at present
+    int my_ver = -1;
     for (;;) {
         if (sh.maxc_dirty) {                                   // uniform: written before the last barrier
             if (warp < sp.n_small) {
@@ -992,7 +1003,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
         }
         const int n_empty = sh.n_empty, n_slots = sh.n_slots, ver = sh.ver;
         const unsigned hm = 0xffffffffu;
-        const int grp = warp < SCAN_WARPS ? 2 * warp : CLS_G;         // index of the warp's first candidate
+        const int grp = warp < SCAN_WARPS ? OFFER * warp : CLS_G;     // index of the warp's first candidate
         bool rescan = ver != my_ver || sh.dirty[grp] != 0;
         if (warp < SCAN_WARPS) {
             if (!rescan) {
@@ -1029,16 +1040,23 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     } else rest = max(rest, k32);
                     if (ok_g) rest = max(rest, kc);
                 }
-                // the warp's best; then its second (the lane that gave the best offers its own second); then the
-                // largest key among what remains
-                uint32_t a_k = k1, a_p = p1; int a_j = j1;
-                const int src_a = warp_select(a_k, a_j, a_p, hm);
-                uint32_t b_k = lane == src_a ? k2 : k1, b_p = lane == src_a ? p2 : p1; int b_j = lane == src_a ? j2 : j1;
-                const int src_b = warp_select(b_k, b_j, b_p, hm);
-                const uint32_t left = lane == src_a ? (src_b == src_a ? 0u : k2) : (lane == src_b ? k2 : k1);
-                c_key2 = __reduce_max_sync(hm, max(rest, left));
-                c_blk = __reduce_max_sync(hm, blk);
-                c_key = a_k; c_j = a_j; c_pay = a_p; c_keyB = b_k; c_jB = b_j; c_payB = b_p; my_ver = ver;
+                // the warp's best OFFER candidates one after another (the lane that gave one puts up its own second;
+                // a third of the same lane counts with what remains); then the largest key among what remains
+                uint32_t o_k = 0u, o_p = 0u; int o_j = 0x7fffffff;          // lane r keeps the warp's r-th candidate
+#pragma unroll
+                for (int r = 0; r < OFFER; ++r) {
+                    uint32_t w_k = k1, w_p = p1; int w_j = j1;
+                    const int src = warp_select(w_k, w_j, w_p, hm);
+                    if (lane == r) { o_k = w_k; o_j = w_j; o_p = w_p; }
+                    if (lane == src && w_k != 0u) { k1 = k2; j1 = j2; p1 = p2; k2 = 0u; j2 = 0x7fffffff; }
+                }
+                const uint32_t key2 = __reduce_max_sync(hm, max(rest, max(k1, k2)));
+                const uint32_t blkw = __reduce_max_sync(hm, blk);
+                if (lane < OFFER) {
+                    sh.red_key[grp + lane] = o_k; sh.red_j[grp + lane] = o_j; sh.red_pay[grp + lane] = o_p;
+                    sh.red_key2[grp + lane] = lane == 0 ? key2 : (lane == 1 ? blkw : 0u);
+                }
+                my_ver = ver;
                 if (lane == 0) sh.dirty[grp] = 0;
             }
         } else if (rescan) {
@@ -1062,22 +1080,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             }
             const uint32_t mine = best;
             const int src = warp_select(best, best_j, pay);
-            c_key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
-            c_blk = __reduce_max_sync(0xffffffffu, blk);
-            c_key = best; c_j = best_j; c_pay = pay; my_ver = ver;
-            if (lane == 0) sh.dirty[CLS_G] = 0;
-        }
-        if (lane == 0) {
-            sh.red_key[grp] = c_key; sh.red_j[grp] = c_j; sh.red_pay[grp] = c_pay; sh.red_key2[grp] = c_key2;
-            if (warp < SCAN_WARPS) { sh.red_key[grp + 1] = c_keyB; sh.red_j[grp + 1] = c_jB; sh.red_pay[grp + 1] = c_payB; }
-            sh.red_key2[grp + 1] = c_blk;            // the odd entries: what each warp found blocked
+            const uint32_t key2 = __reduce_max_sync(0xffffffffu, lane == src ? second : mine);
+            const uint32_t blkw = __reduce_max_sync(0xffffffffu, blk);
+            my_ver = ver;
+            if (lane == 0) {
+                sh.red_key[CLS_G] = best; sh.red_j[CLS_G] = best_j; sh.red_pay[CLS_G] = pay;
+                sh.red_key2[CLS_G] = key2; sh.red_key2[CLS_G + 1] = blkw;
+                sh.dirty[CLS_G] = 0;
+            }
         }
         __syncthreads();
         if (warp == 0) {
             const unsigned FULL = 0xffffffffu;
-            const uint32_t key = lane < N_GROUPS ? sh.red_key[lane] : 0u, my_pay = lane < N_GROUPS ? sh.red_pay[lane] : 0u;
-            const int my_j = lane < N_GROUPS ? sh.red_j[lane] : 0x7fffffff;
-            uint32_t best = key, pay = my_pay; int best_j = my_j;
+            // two candidates a lane: those of index lane and lane + 32 (the class head is the second one of lane CLS_G - 32)
+            uint32_t key_[2], pay_[2]; int j_[2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) { key_[u] = sh.red_key[lane + 32 * u]; pay_[u] = sh.red_pay[lane + 32 * u]; j_[u] = sh.red_j[lane + 32 * u]; }
+            const bool second_u = key_[1] > key_[0] || (key_[1] == key_[0] && key_[1] && j_[1] < j_[0]);
+            uint32_t best = second_u ? key_[1] : key_[0], pay = second_u ? pay_[1] : pay_[0]; int best_j = second_u ? j_[1] : j_[0];
             const int top_lane = warp_select(best, best_j, pay);
             bool go = best != 0u;
             const int steps0 = sh.steps, room = A.max_steps - steps0;
@@ -1103,7 +1123,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 const int t = int(pay & 0x7fffffffu);
                 const int gi2 = t / sp.nC, ci2 = t - gi2 * sp.nC;
                 const int g2 = sp.g_levels[gi2], c2 = sp.c_levels[ci2];
-                const uint32_t B = __reduce_max_sync(FULL, lane < CLS_G ? key : (lane == CLS_G ? sh.red_key2[CLS_G] : 0u));
+                // the largest key among everything but the heads of this class
+                const uint32_t B = __reduce_max_sync(FULL, max(key_[0], lane + 32 == CLS_G ? sh.red_key2[CLS_G] : key_[1]));
                 int k2 = 1; int64_t avail = -1;
                 if (g2 <= sp.Gn) {
                     const int target = v.maxc[gi2] >= c2 ? first_fit_warp(v, g2, c2, lane) : -1;
@@ -1190,8 +1211,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             if (go && n_acc == 0 && !(pay & 0x80000000u)) {
                 bool st = false;
                 if (lane == top_lane) {
-                    const SlotA a = v.sa[int(my_pay)];
-                    const int type_gpu = int(key >> 31);
+                    const SlotA a = v.sa[int(pay)];
+                    const int type_gpu = int(best >> 31);
                     const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
                     const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
                     const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
@@ -1203,55 +1224,85 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 top_stays = __any_sync(FULL, st);
             }
             if (go && n_acc == 0 && top_stays) {
-                const uint32_t M = __reduce_max_sync(FULL, !(lane & 1) ? sh.red_key2[lane] : 0u);
-                bool elig = false, s_ok = false, s_maxc = false, s_multi = false;
-                int s_slot = 0, s_node = -1, s_type = 0, s_dgc = 0, s_k = 1;
-                int64_t s_dm = 0;
-                uint32_t s_bound = 0u;
-                SlotA na; SlotB nb; SlotC nq;
-                na.gain_g = na.gain_c = 0.0f; na.packed = 0u; na.node = -1;
-                nb.val = 0.0f; nb.plan = -1; nb.f_level = 0; nb.w = 0.0f;
-                nq.gkind = nq.ckind = K_NONE; nq.gidx = nq.cidx = 0; nq.dg = nq.need = nq.dc = nq.c = nq.c2 = nq.g = 0;
+                const uint32_t M = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane] : 0u);
+                // per candidate (two a lane): can its commit be worked out here, does it succeed, and what it changes;
+                // the slot it has afterwards waits in shared memory (bst) until the candidate is taken
+                bool elig[2] = { false, false }, s_ok[2] = { false, false }, s_maxc[2] = { false, false }, s_multi[2] = { false, false };
+                int s_slot[2] = { 0, 0 }, s_node[2] = { -1, -1 }, s_type[2] = { 0, 0 }, s_dgc[2] = { 0, 0 }, s_k[2] = { 1, 1 };
+                int64_t s_dm[2] = { 0, 0 };
+                uint32_t s_bound[2] = { 0u, 0u };
                 // the same for every lane: while an empty node remains and every maxc[] entry is the node's core
                 // count no commit that stays on its node can change maxc[]; the first four levels in registers
                 const bool saturated = sh.n_empty > 0 && __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
                 int mx_r[4], gl_r[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) { mx_r[u] = u < sp.n_small ? v.maxc[u] : -2; gl_r[u] = u < sp.n_small ? v.gl[u] : 0x7fffffff; }
-                if (key != 0u && !(my_pay & 0x80000000u)) {
-                    const int s = int(my_pay), j = my_j;
-                    const SlotA a = v.sa[s];
-                    const int type_gpu = int(key >> 31);
-                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
-                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
-                    const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
-                    const int w_old = v.gc[a.node];
-                    // stays where it is: room on its own node, or more cores on the whole nodes it already holds
-                    const bool multi = g > sp.Gn;
-                    const int k = multi ? g >> sp.log2Gn : 1;
-                    const bool stays = multi ? (!type_gpu && cdiv_k(c2, k) <= sp.Cn)
-                                             : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
-                    if (stays) {
-                        // everything the commit and the new gains can need, in one wave of loads
-                        const SlotB b = v.sb[s];
-                        const HotCurve cand = load_hc(A.hc + hc_idx(sp, j, gi2, ci2));
-                        const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[0];
-                        const int4 t_hi = reinterpret_cast<const int4 *>(A.tr + hc_idx(sp, j, gi2, ci2))[1];
+                // first every candidate's loads, so that both of a lane's are under way together
+                bool stays[2] = { false, false };
+                SlotA sa_[2]; int w_old_[2];
+                int4 b4[2], c4[2], tlo[2], thi[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    sa_[u].gain_g = sa_[u].gain_c = 0.0f; sa_[u].packed = 0u; sa_[u].node = 0; w_old_[u] = 0;
+                    b4[u] = c4[u] = tlo[u] = thi[u] = make_int4(0, 0, 0, 0);
+                    if (key_[u] != 0u && !(pay_[u] & 0x80000000u)) {
+                        const int s = int(pay_[u]), j = j_[u];
+                        const SlotA a = v.sa[s];
+                        const int type_gpu = int(key_[u] >> 31);
+                        const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                        const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+                        const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+                        const int w_old = v.gc[a.node];
+                        // stays where it is: room on its own node, or more cores on the whole nodes it already holds
+                        const bool multi = g > sp.Gn;
+                        const int k = multi ? g >> sp.log2Gn : 1;
+                        stays[u] = multi ? (!type_gpu && cdiv_k(c2, k) <= sp.Cn)
+                                         : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
+                        sa_[u] = a; w_old_[u] = w_old;
+                        if (stays[u]) {
+                            // everything the commit and the new gains can need, in one wave of loads
+                            const size_t o = hc_idx(sp, j, gi2, ci2);
+                            b4[u] = *reinterpret_cast<const int4 *>(v.sb + s);
+                            c4[u] = *reinterpret_cast<const int4 *>(A.hc + o);
+                            tlo[u] = reinterpret_cast<const int4 *>(A.tr + o)[0];
+                            thi[u] = reinterpret_cast<const int4 *>(A.tr + o)[1];
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    if (stays[u]) {
+                        const int s = int(pay_[u]);
+                        const SlotA a = sa_[u];
+                        const int w_old = w_old_[u];
+                        const int type_gpu = int(key_[u] >> 31);
+                        const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                        const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+                        const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+                        const bool multi = g > sp.Gn;
+                        const int k = multi ? g >> sp.log2Gn : 1;
+                        SlotB b; b.val = __int_as_float(b4[u].x); b.plan = b4[u].y; b.f_level = b4[u].z; b.w = __int_as_float(b4[u].w);
+                        HotCurve cand; cand.val = __int_as_float(c4[u].x); cand.plan = c4[u].y; cand.f = c4[u].z; cand.ok = c4[u].w;
+                        const int4 t_lo = tlo[u], t_hi = thi[u];
+                        SlotA na; SlotB nb; SlotC nq;
+                        na.gain_g = na.gain_c = 0.0f; na.packed = 0u; na.node = -1;
+                        nb.val = 0.0f; nb.plan = -1; nb.f_level = 0; nb.w = 0.0f;
+                        nq.gkind = nq.ckind = K_NONE; nq.gidx = nq.cidx = 0; nq.dg = nq.need = nq.dc = nq.c = nq.c2 = nq.g = 0;
                         const int64_t m_cur = v.ml[b.f_level];
                         const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
                         // levels ascend: the highest level that fits is below 0 / at least cand.f exactly when
                         // level 0 / level cand.f itself does not fit / fits
                         const bool none_fits = v.ml[0] > avail;
                         const bool cand_fits = cand.plan >= 0 && cand.f >= 0 && cand.f < sp.nM && v.ml[cand.f >= 0 && cand.f < sp.nM ? cand.f : 0] <= avail;
-                        s_multi = multi; s_k = k;
+                        s_multi[u] = multi; s_k[u] = k;
                         bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
-                        s_slot = s; s_node = a.node; s_type = type_gpu;
-                        if (none_fits) { elig = true; s_ok = false; }
+                        s_slot[u] = s; s_node[u] = a.node; s_type[u] = type_gpu;
+                        if (none_fits) { elig[u] = true; s_ok[u] = false; }
                         else if (cand_fits) {
-                            elig = true;
-                            s_ok = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
+                            elig[u] = true;
+                            s_ok[u] = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
                         }
-                        if (elig && s_ok) {
+                        if (elig[u] && s_ok[u]) {
                             // the new gains and placement needs are those of the record of (gi2, ci2): the value
                             // committed is the curve's
                             na.gain_g = fz_g ? 0.0f : __int_as_float(t_lo.x); na.gain_c = fz_c ? 0.0f : __int_as_float(t_lo.y);
@@ -1261,37 +1312,37 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             if (multi) {
                                 // per-node shares of cores and memory on each of the k nodes (they hold no free GPU,
                                 // so maxc[] cannot change)
-                                s_dgc = cdiv_k(c2, k) - cdiv_k(c, k);
-                                s_dm = cdiv64_k(v.ml[cand.f], k) - cdiv64_k(m_cur, k);
+                                s_dgc[u] = cdiv_k(c2, k) - cdiv_k(c, k);
+                                s_dm[u] = cdiv64_k(v.ml[cand.f], k) - cdiv64_k(m_cur, k);
                             } else {
-                                s_dgc = ((g2 - g) << 16) + (c2 - c);
-                                s_dm = v.ml[cand.f] - m_cur;
+                                s_dgc[u] = ((g2 - g) << 16) + (c2 - c);
+                                s_dm[u] = v.ml[cand.f] - m_cur;
                             }
                             // can maxc[] change?  (the node only loses GPUs / cores)
-                            const int w_new = w_old - s_dgc;
+                            const int w_new = w_old - s_dgc[u];
                             if (!multi && !saturated) {
 #pragma unroll
-                                for (int u = 0; u < 4; ++u) {
-                                    const int ot = fg_of(w_old) >= gl_r[u] ? fc_of(w_old) : -1, nt = fg_of(w_new) >= gl_r[u] ? fc_of(w_new) : -1;
-                                    s_maxc = s_maxc || (ot == mx_r[u] && nt < ot);
+                                for (int x = 0; x < 4; ++x) {
+                                    const int ot = fg_of(w_old) >= gl_r[x] ? fc_of(w_old) : -1, nt = fg_of(w_new) >= gl_r[x] ? fc_of(w_new) : -1;
+                                    s_maxc[u] = s_maxc[u] || (ot == mx_r[x] && nt < ot);
                                 }
                                 for (int i = 4; i < sp.n_small; ++i) {
                                     const int glv = v.gl[i], mx = v.maxc[i];
                                     const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
-                                    s_maxc = s_maxc || (ot == mx && nt < ot);
+                                    s_maxc[u] = s_maxc[u] || (ot == mx && nt < ot);
                                 }
                             }
-                        } else if (elig) {
+                        } else if (elig[u]) {
                             // rejected: the (job, type) pair is frozen, the other increment stays as it is
                             if (type_gpu) { fz_g = true; } else { fz_c = true; }
                             na = a; nb = b; nq = v.sc[s];
                             if (type_gpu) na.gain_g = 0.0f; else na.gain_c = 0.0f;
                             na.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
                         }
-                        if (elig) {
+                        if (elig[u]) {
                             // the job's own next candidates, if they could be placed (maxc[] can only have
                             // shrunk by then, so testing against the present table errs on the safe side)
-                            const int w_new = w_old - s_dgc;
+                            const int w_new = w_old - s_dgc[u];
                             const int fg = fg_of(w_new), fc = fc_of(w_new);
                             const int n_empty = sh.n_empty;
                             const bool pg = na.gain_g > 0.0f
@@ -1301,7 +1352,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             const bool pc = na.gain_c > 0.0f && (nq.ckind == K_SINGLE ? (fc >= nq.dc || v.maxc[nq.cidx] >= nq.c2) : nq.ckind == K_MULTI_WHOLE);
                             const uint32_t bg = pg ? (0x80000000u | __float_as_uint(na.gain_g)) : 0u;
                             const uint32_t bc = pc ? __float_as_uint(na.gain_c) : 0u;
-                            s_bound = bg > bc ? bg : bc;
+                            s_bound[u] = bg > bc ? bg : bc;
+                            int4 *dst = bst + 3 * (lane + 32 * u);
+                            dst[0] = make_int4(__float_as_int(na.gain_g), __float_as_int(na.gain_c), int(na.packed), na.node);
+                            dst[1] = make_int4(__float_as_int(nb.val), nb.plan, nb.f_level, __float_as_int(nb.w));
+                            dst[2] = *reinterpret_cast<const int4 *>(&nq);
                         }
                     }
                 }
@@ -1312,57 +1367,100 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 // could not be worked out, the keys of those that share a node with a candidate ranked before them,
                 // and, among what is left, every bound (a bound at or above its own key: that key).  They form a
                 // prefix of the order, possibly a little shorter than the longest one; the rest waits a turn.
-                const u64 mine = (u64(key) << 32) | (key ? u64(uint32_t(KEY_JOB_MASK) - uint32_t(my_j)) << 5 : 0ull) | u64(31 - lane);
-                sh.sel[lane] = mine;                         // key, then lowest job, then lane: all words differ
-                __syncwarp();
-                const bool usable = key != 0u && elig;
-                uint32_t t = __reduce_max_sync(FULL, key != 0u && !elig ? key : 0u);
+                u64 mine[2]; bool usable[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    // key, then lowest job, then index: all words differ
+                    mine[u] = (u64(key_[u]) << 32) | (key_[u] ? u64(uint32_t(KEY_JOB_MASK) - uint32_t(j_[u])) << 6 : 0ull) | u64(63 - lane - 32 * u);
+                    sh.sel[lane + 32 * u] = mine[u];
+                    usable[u] = key_[u] != 0u && elig[u];
+                }
+                uint32_t t = __reduce_max_sync(FULL, max(key_[0] != 0u && !elig[0] ? key_[0] : 0u, key_[1] != 0u && !elig[1] ? key_[1] : 0u));
                 if (M > t) t = M;
-                bool lower = false;                          // a candidate ranked before this one sits on the same node
-                for (unsigned m = __match_any_sync(FULL, usable ? s_node : -1 - lane) & ~(1u << lane); m; m &= m - 1)
-                    lower = lower || sh.sel[__ffs(m) - 1] > mine;
-                const uint32_t t_node = __reduce_max_sync(FULL, lower ? key : 0u);
+                // Which candidates sit on a node together with one ranked before them?  Every candidate puts its key up
+                // for its node (a table indexed by the node's low bits: two nodes that meet there count as one, which
+                // only shortens the batch), the highest key keeps it, among equal keys the lowest job.
+#pragma unroll
+                for (int u = 0; u < 2; ++u) if (usable[u]) atomicMax(&claim_k[s_node[u] & (CLAIMS - 1)], key_[u]);
+                __syncwarp();
+#pragma unroll
+                for (int u = 0; u < 2; ++u) if (usable[u] && claim_k[s_node[u] & (CLAIMS - 1)] == key_[u]) atomicMin(&claim_j[s_node[u] & (CLAIMS - 1)], j_[u]);
+                __syncwarp();
+                bool lower[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    lower[u] = usable[u] && !(claim_k[s_node[u] & (CLAIMS - 1)] == key_[u] && claim_j[s_node[u] & (CLAIMS - 1)] == j_[u]);
+                __syncwarp();
+#pragma unroll
+                for (int u = 0; u < 2; ++u) if (usable[u]) { claim_k[s_node[u] & (CLAIMS - 1)] = 0u; claim_j[s_node[u] & (CLAIMS - 1)] = 0x7fffffff; }
+                const uint32_t t_node = __reduce_max_sync(FULL, max(lower[0] ? key_[0] : 0u, lower[1] ? key_[1] : 0u));
                 if (t_node > t) t = t_node;
-                const uint32_t t_bound = __reduce_max_sync(FULL, usable && key > t ? (s_bound < key ? s_bound : key) : 0u);
+                const uint32_t t_bound = __reduce_max_sync(FULL, max(usable[0] && key_[0] > t ? (s_bound[0] < key_[0] ? s_bound[0] : key_[0]) : 0u,
+                                                                      usable[1] && key_[1] > t ? (s_bound[1] < key_[1] ? s_bound[1] : key_[1]) : 0u));
                 if (t_bound > t) t = t_bound;
-                unsigned acc = __ballot_sync(FULL, usable && key > t);
-                n_acc = __popc(acc);
-                int my_order = 0;                            // position among the taken ones (the step log wants it)
+                unsigned acc[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) acc[u] = __ballot_sync(FULL, usable[u] && key_[u] > t);
+                n_acc = __popc(acc[0]) + __popc(acc[1]);
+                int my_order[2] = { 0, 0 };                  // position among the taken ones (the step log wants it)
                 if (n_acc > room || A.step_log) {
-                    for (unsigned m = acc; m; m &= m - 1) my_order += int(sh.sel[__ffs(m) - 1] > mine);
-                    if (n_acc > room) { acc = __ballot_sync(FULL, ((acc >> lane) & 1u) && my_order < room); n_acc = room; }
+                    __syncwarp();
+#pragma unroll
+                    for (int x = 0; x < 2; ++x)
+                        for (unsigned m = acc[x]; m; m &= m - 1) {
+                            const u64 o = sh.sel[__ffs(m) - 1 + 32 * x];
+                            my_order[0] += int(o > mine[0]); my_order[1] += int(o > mine[1]);
+                        }
+                    if (n_acc > room) {
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) acc[u] = __ballot_sync(FULL, ((acc[u] >> lane) & 1u) && my_order[u] < room);
+                        n_acc = room;
+                    }
                 }
                 if (n_acc > 0) {
-                    if ((acc >> lane) & 1u) {
-                        if (s_ok && !s_multi) { v.gc[s_node] -= s_dgc; v.free_m[s_node] -= s_dm; }
-                        v.sa[s_slot] = na; v.sb[s_slot] = nb; v.sc[s_slot] = nq;
-                        sh.dirty[dirty_of(s_slot)] = 1;
-                        if (s_ok && !s_multi) atomicOr(&v.tb[s_node >> 5], 1u << (s_node & 31));
-                        if (A.step_log) A.step_log[steps0 + my_order] = (my_j << 2) | ((s_type ? 0 : 1) << 1) | int(s_ok);
-                        if (s_ok) {
-                            const int ng_ = pk_next_gi(na.packed), gi_ = pk_gi(na.packed), ci_ = pk_ci(na.packed);
-                            if (na.gain_g > 0.0f && ng_ >= 0) prefetch_target(sp, A.hc, A.tr, my_j, ng_, ci_);
-                            if (na.gain_c > 0.0f && ci_ + 1 < sp.nC) prefetch_target(sp, A.hc, A.tr, my_j, gi_, ci_ + 1);
+                    bool md_l = false;
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        if ((acc[u] >> lane) & 1u) {
+                            if (s_ok[u] && !s_multi[u]) { v.gc[s_node[u]] -= s_dgc[u]; v.free_m[s_node[u]] -= s_dm[u]; }
+                            const int4 *src = bst + 3 * (lane + 32 * u);
+                            const int4 na4 = src[0];
+                            *reinterpret_cast<int4 *>(v.sa + s_slot[u]) = na4;
+                            *reinterpret_cast<int4 *>(v.sb + s_slot[u]) = src[1];
+                            *reinterpret_cast<int4 *>(v.sc + s_slot[u]) = src[2];
+                            sh.dirty[dirty_of(s_slot[u])] = 1;
+                            if (s_ok[u] && !s_multi[u]) atomicOr(&v.tb[s_node[u] >> 5], 1u << (s_node[u] & 31));
+                            if (A.step_log) A.step_log[steps0 + my_order[u]] = (j_[u] << 2) | ((s_type[u] ? 0 : 1) << 1) | int(s_ok[u]);
+                            if (s_ok[u]) {
+                                const uint32_t pk = uint32_t(na4.z);
+                                const int ng_ = pk_next_gi(pk), gi_ = pk_gi(pk), ci_ = pk_ci(pk);
+                                if (__int_as_float(na4.x) > 0.0f && ng_ >= 0) prefetch_target(sp, A.hc, A.tr, j_[u], ng_, ci_);
+                                if (__int_as_float(na4.y) > 0.0f && ci_ + 1 < sp.nC) prefetch_target(sp, A.hc, A.tr, j_[u], gi_, ci_ + 1);
+                            }
+                            md_l = md_l || (s_ok[u] && s_maxc[u]);
                         }
                     }
                     // jobs on whole nodes: every node they own changes its share (no other job lives there)
-                    unsigned mm = __ballot_sync(FULL, ((acc >> lane) & 1u) && s_ok && s_multi);
-                    while (mm) {
-                        const int src = __ffs(mm) - 1;
-                        mm &= mm - 1;
-                        const int oj = __shfl_sync(FULL, my_j, src), dc = __shfl_sync(FULL, s_dgc, src);
-                        const long long dm = __shfl_sync(FULL, (long long)s_dm, src);
-                        const int on = __shfl_sync(FULL, s_node, src), ok_ = __shfl_sync(FULL, s_k, src);
-                        const int nn = on + lane;
-                        const bool mine = lane < ok_ && nn < N && v.owner[nn] == oj;
-                        if (__popc(__ballot_sync(FULL, mine)) == ok_) {           // its nodes are on .. on + k - 1
-                            if (mine) { v.gc[nn] -= dc; v.free_m[nn] -= dm; }
-                        } else {
-                            for (int n = lane; n < N; n += 32)
-                                if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        unsigned mm = __ballot_sync(FULL, ((acc[u] >> lane) & 1u) && s_ok[u] && s_multi[u]);
+                        while (mm) {
+                            const int src = __ffs(mm) - 1;
+                            mm &= mm - 1;
+                            const int oj = __shfl_sync(FULL, j_[u], src), dc = __shfl_sync(FULL, s_dgc[u], src);
+                            const long long dm = __shfl_sync(FULL, (long long)s_dm[u], src);
+                            const int on = __shfl_sync(FULL, s_node[u], src), ok_ = __shfl_sync(FULL, s_k[u], src);
+                            const int nn = on + lane;
+                            const bool own = lane < ok_ && nn < N && v.owner[nn] == oj;
+                            if (__popc(__ballot_sync(FULL, own)) == ok_) {           // its nodes are on .. on + k - 1
+                                if (own) { v.gc[nn] -= dc; v.free_m[nn] -= dm; }
+                            } else {
+                                for (int n = lane; n < N; n += 32)
+                                    if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
+                            }
                         }
                     }
-                    const bool md = __any_sync(FULL, ((acc >> lane) & 1u) && s_ok && s_maxc);
+                    const bool md = __any_sync(FULL, md_l);
                     if (lane == 0) { sh.steps = steps0 + n_acc; sh.maxc_dirty = md ? 1 : 0; }
                 }
             }
@@ -1381,46 +1479,59 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             // have afterwards -- so that such a commit only has to find the node, compare the memory and store.
             // Everything else (whole nodes, an entry that needs the table, too little memory) goes through commit_warp.
             if (go && n_acc == 0) {
-                const uint32_t M = __reduce_max_sync(FULL, !(lane & 1) ? sh.red_key2[lane] : 0u);
-                const uint32_t Mblk = __reduce_max_sync(FULL, (lane & 1) ? sh.red_key2[lane] : 0u);
+                const uint32_t M = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane] : 0u);
+                const uint32_t Mblk = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane + 1] : 0u);
                 // -- stage the offered candidates of running jobs
-                const bool is_slot = lane < CLS_G && key != 0u;
-                const u64 mine = is_slot ? ((u64(key) << 32) | (u64(uint32_t(KEY_JOB_MASK) - uint32_t(my_j)) << 5) | u64(31 - lane)) : 0ull;
-                sh.sel[lane] = mine;
-                __syncwarp();
-                const int n_sc = __popc(__ballot_sync(FULL, is_slot));
-                if (is_slot) {
-                    int rank = 0;
+                bool is_slot[2]; u64 mine[2];
 #pragma unroll
-                    for (int i = 0; i < CLS_G; ++i) rank += int(sh.sel[i] > mine);
-                    const int s = int(my_pay);
-                    const SlotA a = v.sa[s];
-                    const int type_gpu = int(key >> 31);
-                    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
-                    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
-                    const size_t o = hc_idx(sp, my_j, gi2, ci2);
-                    ChainRec &r = chain[rank];
-                    const int4 b4 = *reinterpret_cast<const int4 *>(v.sb + s);
-                    const int4 c4 = *reinterpret_cast<const int4 *>(A.hc + o);
-                    const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + o)[0];
-                    r.nq = reinterpret_cast<const int4 *>(A.tr + o)[1];
-                    r.q = *reinterpret_cast<const int4 *>(&v.sc[s]);
-                    const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
-                    const bool f_ok = c4.z >= 0 && c4.z < sp.nM;
-                    const bool cand_ok = c4.y >= 0 && c4.y < sp.P && f_ok && __int_as_float(c4.x) > 0.0f && c4.w != 0
-                                         && __int_as_float(c4.x) > __int_as_float(b4.x);
-                    const bool lean = cand_ok && g <= sp.Gn && g2 <= sp.Gn;
-                    const bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
-                    r.a = make_int4(__float_as_int(a.gain_g), __float_as_int(a.gain_c), int(a.packed), a.node);
-                    r.b = b4; r.cand = c4; r.t_lo = t_lo;
-                    r.cur = make_int4((g << 16) | c, (g2 << 16) | c2, a.node, 0);
-                    r.mem = make_longlong2(v.ml[b4.z], f_ok ? v.ml[c4.z] : 0);
-                    r.na = make_int4(fz_g ? 0 : t_lo.x, fz_c ? 0 : t_lo.y, int(pack(gi2, ci2, t_lo.z, fz_g, fz_c)), -1);
-                    r.nb = make_int4(c4.x, c4.y, c4.z, b4.w);
-                    r.m = make_int4(int(key), my_j, s, gi2 | (ci2 << 8) | (type_gpu << 16) | (int(lean) << 17));
+                for (int u = 0; u < 2; ++u) {
+                    is_slot[u] = lane + 32 * u < CLS_G && key_[u] != 0u;
+                    mine[u] = is_slot[u] ? ((u64(key_[u]) << 32) | (u64(uint32_t(KEY_JOB_MASK) - uint32_t(j_[u])) << 6) | u64(63 - lane - 32 * u)) : 0ull;
+                    sh.sel[lane + 32 * u] = mine[u];
+                }
+                __syncwarp();
+                const int n_sc = __popc(__ballot_sync(FULL, is_slot[0])) + __popc(__ballot_sync(FULL, is_slot[1]));
+                int rank[2] = { 0, 0 };
+                {
+                    const ulonglong2 *sel2 = reinterpret_cast<const ulonglong2 *>(sh.sel);
+#pragma unroll 6
+                    for (int i = 0; i < CLS_G / 2; ++i) {
+                        const ulonglong2 o = sel2[i];
+                        rank[0] += int(o.x > mine[0]) + int(o.y > mine[0]);
+                        rank[1] += int(o.x > mine[1]) + int(o.y > mine[1]);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    if (is_slot[u]) {
+                        const uint32_t key = key_[u]; const int my_j = j_[u];
+                        const int s = int(pay_[u]);
+                        const SlotA a = v.sa[s];
+                        const int type_gpu = int(key >> 31);
+                        const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+                        const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+                        const size_t o = hc_idx(sp, my_j, gi2, ci2);
+                        ChainRec &r = chain[rank[u]];
+                        const int4 b4 = *reinterpret_cast<const int4 *>(v.sb + s);
+                        const int4 c4 = *reinterpret_cast<const int4 *>(A.hc + o);
+                        const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + o)[0];
+                        r.nq = reinterpret_cast<const int4 *>(A.tr + o)[1];
+                        const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+                        const bool f_ok = c4.z >= 0 && c4.z < sp.nM;
+                        const bool cand_ok = c4.y >= 0 && c4.y < sp.P && f_ok && __int_as_float(c4.x) > 0.0f && c4.w != 0
+                                             && __int_as_float(c4.x) > __int_as_float(b4.x);
+                        const bool lean = cand_ok && g <= sp.Gn && g2 <= sp.Gn;
+                        const bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+                        r.b = b4; r.cand = c4; r.t_lo = t_lo;
+                        r.cur = make_int4((g << 16) | c, (g2 << 16) | c2, a.node, 0);
+                        r.mem = make_longlong2(v.ml[b4.z], f_ok ? v.ml[c4.z] : 0);
+                        r.na = make_int4(fz_g ? 0 : t_lo.x, fz_c ? 0 : t_lo.y, int(pack(gi2, ci2, t_lo.z, fz_g, fz_c)), -1);
+                        r.nb = make_int4(c4.x, c4.y, c4.z, b4.w);
+                        r.m = make_int4(int(key), my_j, s, gi2 | (ci2 << 8) | (type_gpu << 16) | (int(lean) << 17));
+                    }
                 }
                 // -- and the first entries of the best class of unallocated jobs (its head is the candidate of lane CLS_G)
-                const uint32_t cls_key = __shfl_sync(FULL, key, CLS_G), cls_pay = __shfl_sync(FULL, my_pay, CLS_G);
+                const uint32_t cls_key = __shfl_sync(FULL, key_[1], CLS_G - 32), cls_pay = __shfl_sync(FULL, pay_[1], CLS_G - 32);
                 int n_ce = 0, cls_t = -1, cls_ptr0 = 0, cls_end0 = 0;
                 u64 ce_k = 0ull; float ce_w = 0.0f;          // lane i: key and weight of entry i of the class (i <= CHAIN_CLS)
                 if (cls_key != 0u) {
@@ -1440,9 +1551,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         const int g2 = v.gl[gi2], c2 = v.clv[ci2];
                         const bool f_ok = c4.z >= 0 && c4.z < sp.nM;
                         const bool lean = c4.y >= 0 && c4.y < sp.P && f_ok && __int_as_float(c4.x) > 0.0f && c4.w != 0 && g2 <= sp.Gn;
-                        r.a = make_int4(0, 0, 0, -1);
                         r.b = make_int4(0, -1, 0, __float_as_int(ce_w));
-                        r.cand = c4; r.t_lo = t_lo; r.q = make_int4(0, 0, 0, 0);
+                        r.cand = c4; r.t_lo = t_lo;
                         r.cur = make_int4(0, (g2 << 16) | c2, -1, 0);
                         r.mem = make_longlong2(0, f_ok ? v.ml[c4.z] : 0);
                         r.na = make_int4(t_lo.x, t_lo.y, int(pack(gi2, ci2, t_lo.z, false, false)), -1);
@@ -1501,10 +1611,8 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                             else { const int k2 = g2 >> sp.log2Gn; has = (c2 + k2 - 1) / k2 <= sp.Cn && ne >= k2; }
                             if (!has) break;
                         } else {                         // is this still the job's best increment that has a place?
-                            const int4 ra = r->a, rq = r->q;
-                            SlotA a0; a0.gain_g = __int_as_float(ra.x); a0.gain_c = __int_as_float(ra.y); a0.packed = uint32_t(ra.z); a0.node = node;
                             uint32_t kg, kc, blk;
-                            slot_keys(sp, v, ne, a0, *reinterpret_cast<const SlotC *>(&rq), w_n, kg, kc, blk);
+                            slot_keys(sp, v, ne, v.sa[s], v.sc[s], w_n, kg, kc, blk);
                             if ((kg ? kg : kc) != kx) break;
                         }
                     }
@@ -1573,8 +1681,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     if (!settled) {
                         const int4 rc = r->cand, t_lo = r->t_lo;
                         HotCurve cand; cand.val = __int_as_float(rc.x); cand.plan = rc.y; cand.f = rc.z; cand.ok = rc.w;
-                        const int4 ra = r->a, rb = r->b;
-                        SlotA a0; a0.gain_g = __int_as_float(ra.x); a0.gain_c = __int_as_float(ra.y); a0.packed = uint32_t(ra.z); a0.node = node;
+                        const int4 rb = r->b;
+                        SlotA a0; a0.gain_g = a0.gain_c = 0.0f; a0.packed = 0u; a0.node = node;
+                        if (!take_c) a0 = v.sa[s];                  // (its slot is as it was when the turn began)
                         SlotB nb; nb.val = __int_as_float(rb.x); nb.plan = rb.y; nb.f_level = rb.z; nb.w = __int_as_float(rb.w);
                         bool fz_g = pk_fz_g(a0.packed), fz_c = pk_fz_c(a0.packed);
                         Committed cm;
