@@ -879,41 +879,42 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             // Free resources only shrink during this phase, so a job that cannot be placed now never can:
             // every lane tests its own job against the present tables and only the others take a turn.
             bool may = false;
-            int need_l = 0, cls_l = 0;              // (GPUs << 16 | cores) of the job's minimum; index of its failure mark
+            int need_l = 0, tag_l = 0;              // (GPUs << 16 | cores) of the job's minimum; index of its failure mark | GPU level << 12
             if (idx < ng && a0.x >= 0) {
                 const int g2 = v.gl[a0.x], c2 = v.clv[a0.y];
-                need_l = (g2 << 16) | c2; cls_l = a0.x * sp.nC + a0.y;
+                need_l = (g2 << 16) | c2; tag_l = (a0.x * sp.nC + a0.y) | (a0.x << 12);
                 if (g2 <= sp.Gn) may = v.maxc[a0.x] >= c2;
                 else { const int k2 = g2 >> sp.log2Gn; may = (c2 + k2 - 1) / k2 <= sp.Cn && n_empty_r >= k2; }
-                may = may && pa_fail[cls_l] != commits;
+                may = may && pa_fail[tag_l & 0xfff] != commits;
             }
             unsigned todo = __ballot_sync(0xffffffffu, may);
             // what a turn needs of its job beyond the cluster's state, worked out by the job's lane: is the curve entry
             // of the target usable as it stands (a plan that runs, with the level's own GPU count), and the memory it takes
             const bool entry_ok = a0.w >= 0 && a0.w < sp.P && __int_as_float(a0.z) > 0.0f && a1.y != 0 && a1.x >= 0 && a1.x < sp.nM;
             const long long m_need_l = entry_ok ? v.ml[a1.x] : 0;
-            // Turns run on all lanes alike (shuffles hand out the job's record, every lane reads and writes the same
-            // shared-memory words, so each lane sees its own stores and the warp never has to synchronise).  The
-            // usual turn -- a job that fits one node, whose curve entry is usable and whose memory fits the node found
+            if (entry_ok) tag_l |= 1 << 20;
+            // Turns run on all lanes alike (shuffles hand out what the turn needs of the job's record, every lane reads and
+            // writes the same shared-memory words, so each lane sees its own stores and the warp never has to synchronise).
+            // The usual turn -- a job that fits one node, whose curve entry is usable and whose memory fits the node found
             // -- touches five words: the failure mark of its levels, the first-fit mark, the node's GPUs / cores and
-            // memory.  Anything else (whole-node minima, an entry that needs the table) goes through commit_warp.
+            // memory; the job's lane notes the slot and the node, and writes the slot when the 32 jobs are through.
+            // Anything else (whole-node minima, an entry that needs the table) goes through commit_warp.
+            int my_slot = -1, my_node = -1;
             while (todo) {
                 const int i = __ffs(todo) - 1;
                 todo &= todo - 1;
-                const int gi = __shfl_sync(0xffffffffu, a0.x, i), ci = __shfl_sync(0xffffffffu, a0.y, i);
-                const int j = __shfl_sync(0xffffffffu, jl, i);
-                const int need = __shfl_sync(0xffffffffu, need_l, i), cls = __shfl_sync(0xffffffffu, cls_l, i);
-                const int usable = __shfl_sync(0xffffffffu, int(entry_ok), i);
+                const int tag = __shfl_sync(0xffffffffu, tag_l, i), need = __shfl_sync(0xffffffffu, need_l, i);
                 const long long m_need = __shfl_sync(0xffffffffu, m_need_l, i);
+                const int cls = tag & 0xfff, gi = (tag >> 12) & 0xff;
+                const bool usable = (tag >> 20) & 1;
+                const int g2 = need >> 16, c2 = need & 0xffff;
                 int tn = 0;
                 if (A.n_tenants > 0) {     // privileged only while the minimum fits the tenant's remaining quota
                     tn = __shfl_sync(0xffffffffu, a1.w, i);
                     if (tn < 0 || tn >= A.n_tenants) continue;
-                    if (rem_q[2 * tn] < sp.g_levels[gi] || rem_q[2 * tn + 1] < sp.c_levels[ci]) continue;
+                    if (rem_q[2 * tn] < g2 || rem_q[2 * tn + 1] < c2) continue;
                 }
                 if (pa_fail[cls] == commits) continue;              // same levels, same cluster: same outcome
-                const int g2 = need >> 16, c2 = need & 0xffff;
-                int placed_on = -1;
                 bool settled = false;
                 if (g2 <= sp.Gn && usable) {
                     // no node below the mark has g2 free GPUs: if the node at the mark fits, it is the first fit
@@ -933,17 +934,18 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         // the node at the mark has just lost the GPUs the next job of these levels would need: the mark
                         // moves on at once, and that job looks at the following node without a search
                         if (sh.ff_pos[gi] == target && fg_of(w_old) - g2 < g2) sh.ff_pos[gi] = target + 1;
-                        placed_on = target; settled = true;
+                        if (lane == i) { my_slot = n_slots_r; my_node = target; }
+                        settled = true;
                     } else if (v.ml[0] > fm) { pa_fail[cls] = commits; continue; }   // the node found has memory for no level
                 }
-                const float val_e = __int_as_float(__shfl_sync(0xffffffffu, a0.z, i));
-                const int plan_e = __shfl_sync(0xffffffffu, a0.w, i), f_e = __shfl_sync(0xffffffffu, a1.x, i);
-                const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
-                Committed cm; cm.first = placed_on; cm.val = val_e; cm.plan = plan_e; cm.f = f_e;
                 if (!settled) {
+                    const int ci = __shfl_sync(0xffffffffu, a0.y, i), j = __shfl_sync(0xffffffffu, jl, i);
+                    const float w = __int_as_float(__shfl_sync(0xffffffffu, a1.z, i));
                     HotCurve cand;
-                    cand.val = val_e; cand.plan = plan_e; cand.f = f_e; cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
-                    cm.first = -1;
+                    cand.val = __int_as_float(__shfl_sync(0xffffffffu, a0.z, i));
+                    cand.plan = __shfl_sync(0xffffffffu, a0.w, i); cand.f = __shfl_sync(0xffffffffu, a1.x, i);
+                    cand.ok = __shfl_sync(0xffffffffu, a1.y, i);
+                    Committed cm; cm.first = -1; cm.val = cand.val; cm.plan = cand.plan; cm.f = cand.f;
                     sh.n_empty = n_empty_r;
                     __syncwarp();
                     settled = commit_warp<false, COMMIT_PHASE_A>(sp, v, sh, A.cv, A.cp, A.cg, A.feas, j, -1, 0, -1, 0.0f, 0, gi, ci, cand, false, lane, cm);
@@ -953,19 +955,24 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         if (cm.first == -2) pa_fail[cls] = commits;
                         continue;
                     }
+                    if (lane == 0) {
+                        const int s = n_slots_r;
+                        SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
+                        SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
+                        v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
+                    }
                 }
-                const int s = n_slots_r;
-                if (lane == 0) {
-                    SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(gi, ci, -1, false, false); sa.node = cm.first;
-                    SlotB sb; sb.val = cm.val; sb.plan = cm.plan; sb.f_level = cm.f; sb.w = w;
-                    v.sa[s] = sa; v.sb[s] = sb; v.sj[s] = j;
-                }
-                n_slots_r = s + 1;
+                ++n_slots_r;
                 ++commits;
                 if (A.n_tenants > 0) {
                     const int qg = rem_q[2 * tn], qc = rem_q[2 * tn + 1];
-                    rem_q[2 * tn] = qg - sp.g_levels[gi]; rem_q[2 * tn + 1] = qc - sp.c_levels[ci];
+                    rem_q[2 * tn] = qg - g2; rem_q[2 * tn + 1] = qc - c2;
                 }
+            }
+            if (my_slot >= 0) {          // placed by the usual turn, with the curve entry as it stands
+                SlotA sa; sa.gain_g = 0.0f; sa.gain_c = 0.0f; sa.packed = pack(a0.x, a0.y, -1, false, false); sa.node = my_node;
+                SlotB sb; sb.val = __int_as_float(a0.z); sb.plan = a0.w; sb.f_level = a1.x; sb.w = __int_as_float(a1.z);
+                v.sa[my_slot] = sa; v.sb[my_slot] = sb; v.sj[my_slot] = jl;
             }
             jl = jl_next; a0 = n0; a1 = n1; jl_next = jl_after;
         }
