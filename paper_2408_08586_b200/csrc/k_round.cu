@@ -918,14 +918,15 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 bool settled = false;
                 if (g2 <= sp.Gn && usable) {
                     // no node below the mark has g2 free GPUs: if the node at the mark fits, it is the first fit
-                    int target = sh.ff_pos[gi];
+                    int mark = sh.ff_pos[gi];
+                    int target = mark;
                     int w_old = target < N ? v.gc[target] : 0;
+                    int64_t fm = target < N ? v.free_m[target] : 0;          // (asked for together with the node's word)
                     if (!(fg_of(w_old) >= g2 && fc_of(w_old) >= c2)) {
                         target = first_fit_from_mark(v, sh, gi, g2, c2, lane);
-                        w_old = target >= 0 ? v.gc[target] : 0;
+                        if (target < 0) { pa_fail[cls] = commits; continue; }      // no node for these levels
+                        w_old = v.gc[target]; fm = v.free_m[target]; mark = sh.ff_pos[gi];
                     }
-                    if (target < 0) { pa_fail[cls] = commits; continue; }      // no node for these levels
-                    const int64_t fm = v.free_m[target];
                     if (m_need <= fm) {
                         // the highest memory level that fits the node is at or above the plan's own: the entry stands
                         v.gc[target] = w_old - need;
@@ -933,7 +934,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         if (fg_of(w_old) == sp.Gn) --n_empty_r;
                         // the node at the mark has just lost the GPUs the next job of these levels would need: the mark
                         // moves on at once, and that job looks at the following node without a search
-                        if (sh.ff_pos[gi] == target && fg_of(w_old) - g2 < g2) sh.ff_pos[gi] = target + 1;
+                        if (mark == target && fg_of(w_old) - g2 < g2) sh.ff_pos[gi] = target + 1;
                         if (lane == i) { my_slot = n_slots_r; my_node = target; }
                         settled = true;
                     } else if (v.ml[0] > fm) { pa_fail[cls] = commits; continue; }   // the node found has memory for no level
