@@ -47,6 +47,7 @@
 // max_steps, scans by the node / level counts); nothing spins on memory.
 
 #include "rubick_internal.cuh"
+#include <cooperative_groups.h>
 
 namespace rubick {
 namespace fastround {
@@ -202,6 +203,49 @@ round_sort_tile_kernel(u64 *__restrict__ keys, int n, int tile, int k_from, int 
         if (last) sorted_w[base + i] = k ? jobs[key_job(k)].w : 0.0f;
     }
 }
+
+// The whole sort in one launch when the keys fit the shared memory of one thread-block cluster (up to eight tiles): a
+// pass with a stride of a tile or more pairs every key with one in another CTA's shared memory, which the CTA reads and
+// writes directly; each of the two CTAs settles half of the pairs they share.  Every CTA runs the same passes, so the
+// cluster barriers match; the last pass that touches another CTA's memory is followed by one.
+__global__ void __launch_bounds__(SORT_T)
+round_sort_cluster_kernel(u64 *__restrict__ keys, int n, const rubick_job *__restrict__ jobs, float *__restrict__ sorted_w)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ u64 a[SORT_TILE];
+    const int rank = int(cluster.block_rank());
+    const int base = rank * SORT_TILE;
+    for (int i = threadIdx.x; i < SORT_TILE; i += SORT_T) a[i] = keys[base + i];
+    __syncthreads();
+    for (int k = 2; k <= n; k <<= 1) {
+        for (int s = k >> 1; s >= SORT_TILE; s >>= 1) {
+            cluster.sync();                                  // every CTA is through with the step before
+            const int bit = s / SORT_TILE;
+            const int other = rank ^ bit;
+            const bool low = (rank & bit) == 0;              // this CTA holds the lower key of every pair it shares with `other`
+            u64 *b = cluster.map_shared_rank(a, other);
+            const int li = threadIdx.x + (low ? 0 : SORT_T); // the lower tile settles the first half of the indices
+            const int lo_index = (low ? base : other * SORT_TILE) + li;
+            u64 *lo = low ? a : b, *hi = low ? b : a;
+            const u64 x = lo[li], y = hi[li];
+            if (((lo_index & k) == 0) ? (x < y) : (x > y)) { lo[li] = y; hi[li] = x; }
+        }
+        if (k > SORT_TILE) cluster.sync(); else __syncthreads();
+        for (int s = min(k >> 1, SORT_TILE >> 1); s > 0; s >>= 1) {
+            const int t = threadIdx.x;
+            const int i = ((t & ~(s - 1)) << 1) | (t & (s - 1));
+            sort_pair(a, i, i | s, ((base + i) & k) == 0);
+            __syncthreads();
+        }
+    }
+    for (int i = threadIdx.x; i < SORT_TILE; i += SORT_T) {
+        const u64 k = a[i];
+        keys[base + i] = k;
+        sorted_w[base + i] = k ? jobs[key_job(k)].w : 0.0f;
+    }
+}
+constexpr int SORT_CLUSTER_MAX = 8;         // tiles one launch can sort (the portable cluster size)
 
 // one pass of stage k with stride s (a tile or more) in global memory; one thread per pair
 __global__ void round_sort_pass_kernel(u64 *__restrict__ keys, int n, int k, int s)
@@ -1870,6 +1914,17 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
                                                                 reinterpret_cast<int32_t *>(base + L.off_isg)); count_launch();
     {
         const int n = L.n_pad, tile = n < SORT_TILE ? n : SORT_TILE;
+        if (n > SORT_TILE && n <= SORT_TILE * SORT_CLUSTER_MAX) {
+            // two to eight tiles: one cluster sorts them in one launch
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(unsigned(n / SORT_TILE)); cfg.blockDim = dim3(SORT_T); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = unsigned(n / SORT_TILE); at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cfg.attrs = at; cfg.numAttrs = 1;
+            const cudaError_t es = cudaLaunchKernelEx(&cfg, round_sort_cluster_kernel, keys, n, d_jobs, sw); count_launch();
+            if (es != cudaSuccess) return es;
+        } else {
         // every stage up to the tile size, tile by tile; then stage by stage: wide strides in global memory, the rest in tiles
         round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, 2, tile, n == tile, d_jobs, sw); count_launch();
         for (int k = tile << 1; k <= n; k <<= 1) {
@@ -1878,6 +1933,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
                 count_launch();
             }
             round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, k, k, k == n, d_jobs, sw); count_launch();
+        }
         }
     }
     cudaError_t e;
