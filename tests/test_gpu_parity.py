@@ -273,8 +273,9 @@ def test_marginal_gain_is_bit_exact(name, J):
         assert (want[0] > 0).any() and (name == "tiny" or (want[1] > 0).any())
 
 
+# (the last two: 4,096 and 8,192 sort keys, which a cluster of two and of four CTAs sorts in one launch)
 ROUND_CASES = [("tiny", None, None), ("paper-scale", None, None), ("cluster-512", 96, 24), ("cluster-512", 700, 64),
-               ("events", 1500, 128)]
+               ("events", 1500, 128), ("events", 3000, 256), ("throughput-stress", 6000, 192)]
 
 
 @pytest.mark.parametrize("name,J,N", ROUND_CASES)
