@@ -2,7 +2,7 @@
 //
 // Same decisions, step for step, as the plain round in k_sched.cu (largest placeable positive
 // GPU gain first, CPU gain when no GPU increment is left, lowest job index on ties, commit with
-// the best plan and its host memory), organised so that one step costs about half a microsecond:
+// the best plan and its host memory), organised so that one step costs a fraction of a microsecond:
 //
 //   prepare  (grid)   one CTA per job.  Per (job, GPU level, CPU level): the curve entry at the top host-memory
 //                     level together with the first feasible memory level of its plan, 16 bytes.  A commit
@@ -16,31 +16,34 @@
 //                     GPU level with a non-zero curve at its starting CPU level) and gain are fixed
 //                     until it is allocated: one 64-bit key (class = target levels | gain | ~job).
 //                     Guaranteed jobs get their Phase-A target resolved here too.
-//   sort     (grid)   bitonic sort of the keys, tiles in shared memory and wide strides in global memory: inside
-//                     a class (same target levels = same placement test) only the first unconsumed job can
-//                     ever be selected.
+//   sort     (grid)   bitonic sort of the keys, tiles in shared memory; up to eight tiles in one launch by a
+//                     thread-block cluster (wide strides through the partner CTA's shared memory), more with wide
+//                     strides in global memory: inside a class (same target levels = same placement test) only the
+//                     first unconsumed job can ever be selected.
 //   round    (1 CTA)  persistent loop.  Shared memory holds one word per node (free GPUs << 16 | free
 //                     cores), free memory and whole-node owners, the table "most free cores among nodes
 //                     with >= g free GPUs" (a job of g GPUs and c cores fits some node exactly when that
 //                     entry is >= c), the head of every class, one 36-byte slot per RUNNING job (scan state
 //                     + what its two candidates need to be placeable) and a bitmap of the nodes the last
-//                     iteration changed.  Every warp caches the two best candidates of its slots and the
-//                     largest key among the rest (the last warp: the best class head and the runner-up key)
-//                     and looks again only when one of its slots, a node under them, that table or the
-//                     number of empty nodes changed.  Warp 0 holds one offered candidate per lane, picks
-//                     (type | gain, lowest job) across them with warp reduce instructions and
-//                     commits, in the exact order of the one-step-at-a-time rule, as many steps as it can
-//                     prove independent of each other:
+//                     iteration changed.  Every scanning warp leaves its four best candidates, the largest key
+//                     among the rest and the largest key among the increments that have a gain but no place in
+//                     shared memory (the last warp: the best class head and the runner-up key) and looks again
+//                     only when one of its slots, a node under them, that table or the number of empty nodes
+//                     changed.  Warp 0 holds two offered candidates per lane, picks (type | gain, lowest job)
+//                     across them with warp reduce instructions and commits, in the exact order of the
+//                     one-step-at-a-time rule, as many steps as it can prove to come next:
 //                       - a run of class heads that are rejected (a rejection changes nothing but the head
 //                         of its class; every lane settles four entries of the class's sorted list);
-//                       - a batch of increments that stay on their own nodes (lane w works out the commit
-//                         of group w's candidate; the candidates above one threshold - every runner-up,
+//                       - a batch of increments that stay on their own nodes (every lane works out the commits
+//                         of its two candidates; the candidates above one threshold - every runner-up,
 //                         every candidate that could not be worked out or shares a node with a better one,
 //                         every new candidate of the jobs taken - are a prefix of the sequential order
 //                         and are committed together);
-//                       - otherwise one general commit (migration, growth onto whole nodes, a class head
-//                         that succeeds): placement, memory level by ballot, node bookkeeping, new gains
-//                         from one warp-wide load of the job's curve column.
+//                       - otherwise a chain of general commits (migrations, growth onto whole nodes, class heads
+//                         that succeed): the offered candidates and the first entries of the best class, staged
+//                         in the rule's order, are committed one after another on the real cluster state while
+//                         the next key exceeds every key not offered, every new candidate of the jobs committed
+//                         before it and, once resources were given back, every increment that had no place.
 //
 // All gain arithmetic uses __fmul_rn / __fsub_rn / __fdiv_rn (one rounding per operation, never
 // fused) so that decisions are reproducible bit for bit.  Every loop is bounded (steps by
@@ -1159,12 +1162,12 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             __syncwarp();
 
             // ---- a batch of independent increments ---------------------------------------------------------
-            // Every lane holds one candidate offered by the scanning warps.  Increments that stay on their node, on pairwise
+            // Every lane holds two candidates offered by the scanning warps.  Increments that stay on their node, on pairwise
             // different nodes, commute with everything except what happens on that node, so the next few
             // picks of the sequential rule can be committed together as long as each of them still is the
             // largest candidate: larger than every key that was not offered (M), than the offered ones not yet
-            // taken, and than the new candidates of the jobs taken before it.  Each lane works out its own
-            // commit first (one wave of global loads for all lanes together instead of several per step).
+            // taken, and than the new candidates of the jobs taken before it.  Each lane works out the commits of
+            // its own candidates first (one wave of global loads for all of them together instead of several per step).
             int n_acc = 0;
             // ---- a run of class heads that cannot be committed --------------------------------------------
             // A rejected increment changes nothing but the head of its class, so as long as the heads of that
