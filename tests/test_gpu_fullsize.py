@@ -246,6 +246,35 @@ def test_event_sized_rounds_agree_with_the_plain_kernel(n_jobs, n_nodes):
     assert res[0]["steps"] > 300 and (n_nodes < 512 or (res[0]["n_nodes"] > 1).any())
 
 
+def test_step_caps_inside_chains_of_commits():
+    """In the event regime a turn of the fast round settles a chain of general commits (migrations, first placements,
+    growth onto whole nodes); a step limit that falls inside one must stop it where the one-step-at-a-time kernel
+    stops, and the steps logged up to there must be the first steps of the unlimited round."""
+    n_jobs, n_nodes = 1500, 512
+    cfg = workloads.make("events", J=n_jobs, n_nodes=n_nodes)
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    d_jobs, d_thr, d_feas = gpu.eval(cfg["jobs"])
+    d_cv, d_cp, d_cg = gpu.best(d_thr, d_feas, n_jobs)
+
+    def run(call, cap, with_log):
+        d_out = t.zeros(n_jobs * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_node = t.zeros(n_nodes * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+        d_log = t.zeros(8192, dtype=t.int32, device="cuda:0") if with_log else None
+        args = (d_jobs, n_jobs, d_cv, d_cp, d_cg, d_feas, n_nodes, cap, d_out, d_node) + ((d_log,) if with_log else ())
+        steps, capped = call(*args)
+        return unpack_round(rb.from_device(d_out, rb.ASSIGN_DTYPE), rb.from_device(d_node, rb.NODE_DTYPE), steps, capped,
+                            d_log.cpu().numpy()[:steps] if with_log else None)
+
+    whole = run(gpu.ctx.greedy_round, 1 << 30, True)
+    assert not whole["capped"] and 300 < whole["steps"] <= 8192
+    for cap in (1, 2, 3, 7, 19, 64, 150, 333, 700):
+        fast, plain = run(gpu.ctx.greedy_round, cap, True), run(gpu.ctx.greedy_round_noalloc, cap, False)
+        assert fast["steps"] == cap and fast["capped"]
+        assert_rounds_equal(fast, plain)
+        assert np.array_equal(fast["log"], whole["log"][:cap])
+
+
 def test_round_repeats_bit_for_bit(full):
     """The fast round uses shared-memory atomics (changed-node bitmap, version counter) and commits several steps a
     turn; none of it may make the outcome depend on timing."""
