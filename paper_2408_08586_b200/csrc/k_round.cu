@@ -305,6 +305,7 @@ struct Shared {
     int n_empty, n_slots, steps, capped, stop, n_guar, n_ccls;
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
+    int batch_go;                 // this turn is a batch of increments: warp 1 works out half of the candidates
     int scan_cnt[RW];
     int empty_lo;                 // no node below this index is empty (whole multiples of 32 after a search)
     int4 pa_rec[32][2]; int pa_job[32];   // Phase A: the records of the 32 jobs being worked on
@@ -737,6 +738,120 @@ __device__ __forceinline__ void slot_keys_uniform(const Space &sp, const Views &
     }
 }
 
+// What a batch of increments needs to know about one offered candidate: can its commit be worked out without looking
+// for a node (it stays where it is), does it succeed, what it changes on its node, and the largest key the job could
+// offer afterwards.  The slot the job would have afterwards goes to `stage` (three 16-byte words).
+struct BatchOut {
+    bool elig, ok, maxc, multi;       // worked out here | the commit succeeds | maxc[] may change | the job holds whole nodes
+    int slot, node, type, dgc, k;     // slot, (first) node, GPU increment?, what the node loses (GPUs << 16 | cores, or cores per node), nodes held
+    int64_t dm;                       // memory the node (each node) loses
+    uint32_t bound;
+};
+
+__device__ __forceinline__ void batch_candidate(const Space &sp, const Views &v, const HotCurve *__restrict__ hc, const void *tr_,
+                                                int n_empty, bool saturated, const int (&mx_r)[4], const int (&gl_r)[4],
+                                                uint32_t key, uint32_t pay, int j, int4 *stage, BatchOut &o)
+{
+    const Trans *tr = static_cast<const Trans *>(tr_);
+    o.elig = o.ok = o.maxc = o.multi = false;
+    o.slot = 0; o.node = -1; o.type = 0; o.dgc = 0; o.k = 1; o.dm = 0; o.bound = 0u;
+    if (key == 0u || (pay & 0x80000000u)) return;
+    const int s = int(pay);
+    const SlotA a = v.sa[s];
+    const int type_gpu = int(key >> 31);
+    const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
+    const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
+    const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
+    const int w_old = v.gc[a.node];
+    // stays where it is: room on its own node, or more cores on the whole nodes it already holds
+    const bool multi = g > sp.Gn;
+    const int k = multi ? g >> sp.log2Gn : 1;
+    const bool stays = multi ? (!type_gpu && cdiv_k(c2, k) <= sp.Cn)
+                             : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
+    if (!stays) return;
+    // everything the commit and the new gains can need, in one wave of loads
+    const size_t off = hc_idx(sp, j, gi2, ci2);
+    const int4 b4 = *reinterpret_cast<const int4 *>(v.sb + s);
+    const int4 c4 = *reinterpret_cast<const int4 *>(hc + off);
+    const int4 t_lo = reinterpret_cast<const int4 *>(tr + off)[0];
+    const int4 t_hi = reinterpret_cast<const int4 *>(tr + off)[1];
+    SlotB b; b.val = __int_as_float(b4.x); b.plan = b4.y; b.f_level = b4.z; b.w = __int_as_float(b4.w);
+    HotCurve cand; cand.val = __int_as_float(c4.x); cand.plan = c4.y; cand.f = c4.z; cand.ok = c4.w;
+    SlotA na; SlotB nb; SlotC nq;
+    na.gain_g = na.gain_c = 0.0f; na.packed = 0u; na.node = -1;
+    nb.val = 0.0f; nb.plan = -1; nb.f_level = 0; nb.w = 0.0f;
+    nq.gkind = nq.ckind = K_NONE; nq.gidx = nq.cidx = 0; nq.dg = nq.need = nq.dc = nq.c = nq.c2 = nq.g = 0;
+    const int64_t m_cur = v.ml[b.f_level];
+    const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
+    // levels ascend: the highest level that fits is below 0 / at least cand.f exactly when
+    // level 0 / level cand.f itself does not fit / fits
+    const bool none_fits = v.ml[0] > avail;
+    const bool cand_fits = cand.plan >= 0 && cand.f >= 0 && cand.f < sp.nM && v.ml[cand.f >= 0 && cand.f < sp.nM ? cand.f : 0] <= avail;
+    o.multi = multi; o.k = k;
+    bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
+    o.slot = s; o.node = a.node; o.type = type_gpu;
+    if (none_fits) { o.elig = true; o.ok = false; }
+    else if (cand_fits) {
+        o.elig = true;
+        o.ok = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
+    }
+    if (o.elig && o.ok) {
+        // the new gains and placement needs are those of the record of (gi2, ci2): the value committed is the curve's
+        na.gain_g = fz_g ? 0.0f : __int_as_float(t_lo.x); na.gain_c = fz_c ? 0.0f : __int_as_float(t_lo.y);
+        na.packed = pack(gi2, ci2, t_lo.z, fz_g, fz_c); na.node = a.node;
+        nb.val = cand.val; nb.plan = cand.plan; nb.f_level = cand.f; nb.w = b.w;
+        nq = *reinterpret_cast<const SlotC *>(&t_hi);
+        if (multi) {
+            // per-node shares of cores and memory on each of the k nodes (they hold no free GPU, so maxc[] cannot change)
+            o.dgc = cdiv_k(c2, k) - cdiv_k(c, k);
+            o.dm = cdiv64_k(v.ml[cand.f], k) - cdiv64_k(m_cur, k);
+        } else {
+            o.dgc = ((g2 - g) << 16) + (c2 - c);
+            o.dm = v.ml[cand.f] - m_cur;
+        }
+        // can maxc[] change?  (the node only loses GPUs / cores)
+        const int w_new = w_old - o.dgc;
+        if (!multi && !saturated) {
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+                const int ot = fg_of(w_old) >= gl_r[x] ? fc_of(w_old) : -1, nt = fg_of(w_new) >= gl_r[x] ? fc_of(w_new) : -1;
+                o.maxc = o.maxc || (ot == mx_r[x] && nt < ot);
+            }
+            for (int i = 4; i < sp.n_small; ++i) {
+                const int glv = v.gl[i], mx = v.maxc[i];
+                const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
+                o.maxc = o.maxc || (ot == mx && nt < ot);
+            }
+        }
+    } else if (o.elig) {
+        // rejected: the (job, type) pair is frozen, the other increment stays as it is
+        if (type_gpu) { fz_g = true; } else { fz_c = true; }
+        na = a; nb = b; nq = v.sc[s];
+        if (type_gpu) na.gain_g = 0.0f; else na.gain_c = 0.0f;
+        na.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
+    }
+    if (o.elig) {
+        // the job's own next candidates, if they could be placed (maxc[] can only have
+        // shrunk by then, so testing against the present table errs on the safe side)
+        const int w_new = w_old - o.dgc;
+        const int fg = fg_of(w_new), fc = fc_of(w_new);
+        const bool pg = na.gain_g > 0.0f
+                        && (nq.gkind == K_SINGLE ? (fg >= nq.dg || v.maxc[nq.gidx] >= nq.c)
+                            : nq.gkind == K_MULTI_WHOLE ? n_empty >= nq.need
+                            : nq.gkind == K_MULTI_PART ? n_empty + int(fg + nq.g == sp.Gn) >= nq.need : false);
+        const bool pc = na.gain_c > 0.0f && (nq.ckind == K_SINGLE ? (fc >= nq.dc || v.maxc[nq.cidx] >= nq.c2) : nq.ckind == K_MULTI_WHOLE);
+        const uint32_t bg = pg ? (0x80000000u | __float_as_uint(na.gain_g)) : 0u;
+        const uint32_t bc = pc ? __float_as_uint(na.gain_c) : 0u;
+        o.bound = bg > bc ? bg : bc;
+        stage[0] = make_int4(__float_as_int(na.gain_g), __float_as_int(na.gain_c), int(na.packed), na.node);
+        stage[1] = make_int4(__float_as_int(nb.val), nb.plan, nb.f_level, __float_as_int(nb.w));
+        stage[2] = *reinterpret_cast<const int4 *>(&nq);
+    }
+}
+
+// warps 0 and 1 meet at barriers of their own (the block's barrier is number 0)
+__device__ __forceinline__ void pair_barrier(int id) { asm volatile("bar.sync %0, 64;" :: "r"(id) : "memory"); }
+
 // One candidate staged for a chain of commits: everything its commit and its new gains can need.
 //   b       value, plan, memory level and weight the job has (class entries: only the weight)
 //   cand    curve entry of the target at the top memory level;  t_lo: first half of the target's transition record
@@ -786,7 +901,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     // or a node without memory for any level; while nothing else has been placed since, the next one fares the same
     // (shares its memory with what only Phase B uses)
     constexpr size_t PA_BYTES = (size_t(RUBICK_MAX_G_LEVELS) * RUBICK_MAX_C_LEVELS + 2 * RUBICK_MAX_TENANTS) * 4;
-    constexpr size_t PB_BYTES = sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS) + size_t(N_CAND) * 48 + size_t(CLAIMS) * 8;
+    constexpr size_t PB_BYTES = sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS) + size_t(N_CAND) * 48 + size_t(CLAIMS) * 8 + 32 * 32;
     __shared__ __align__(16) unsigned char phase_buf[PA_BYTES > PB_BYTES ? PA_BYTES : PB_BYTES];
     int *pa_fail = reinterpret_cast<int *>(phase_buf);
     // Phase B: bit t set = the last head of class t was placed; the next one is then tried directly instead of
@@ -799,6 +914,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
     int4 *bst = reinterpret_cast<int4 *>(phase_buf + sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS));
     uint32_t *claim_k = reinterpret_cast<uint32_t *>(phase_buf + sizeof(ChainRec) * (CHAIN_SLOTS + CHAIN_CLS) + size_t(N_CAND) * 48);
     int32_t *claim_j = reinterpret_cast<int32_t *>(claim_k + CLAIMS);
+    int4 *bres = reinterpret_cast<int4 *>(claim_j + CLAIMS);      // what warp 1 found out about the second candidate of every lane
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int N = A.N, J = A.J;
     const int n_cls = sp.nG * sp.nC;
@@ -1278,142 +1394,39 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 }
                 top_stays = __any_sync(FULL, st);
             }
-            if (go && n_acc == 0 && top_stays) {
+            // Warp 1 works out the second candidate of every lane while this warp works out the first: it waits for the
+            // word that says whether there is a batch, and hands its results over in shared memory.
+            const bool batch = go && n_acc == 0 && top_stays;
+            if (lane == 0) sh.batch_go = batch ? 1 : 0;
+            pair_barrier(1);
+            if (batch) {
                 const uint32_t M = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane] : 0u);
                 // per candidate (two a lane): can its commit be worked out here, does it succeed, and what it changes;
                 // the slot it has afterwards waits in shared memory (bst) until the candidate is taken
-                bool elig[2] = { false, false }, s_ok[2] = { false, false }, s_maxc[2] = { false, false }, s_multi[2] = { false, false };
-                int s_slot[2] = { 0, 0 }, s_node[2] = { -1, -1 }, s_type[2] = { 0, 0 }, s_dgc[2] = { 0, 0 }, s_k[2] = { 1, 1 };
-                int64_t s_dm[2] = { 0, 0 };
-                uint32_t s_bound[2] = { 0u, 0u };
-                // the same for every lane: while an empty node remains and every maxc[] entry is the node's core
-                // count no commit that stays on its node can change maxc[]; the first four levels in registers
-                const bool saturated = sh.n_empty > 0 && __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
-                int mx_r[4], gl_r[4];
+                bool elig[2], s_ok[2], s_maxc[2], s_multi[2];
+                int s_slot[2], s_node[2], s_type[2], s_dgc[2], s_k[2];
+                int64_t s_dm[2];
+                uint32_t s_bound[2];
+                {
+                    // the same for every lane: while an empty node remains and every maxc[] entry is the node's core
+                    // count no commit that stays on its node can change maxc[]; the first four levels in registers
+                    const int n_empty = sh.n_empty;
+                    const bool saturated = n_empty > 0 && __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
+                    int mx_r[4], gl_r[4];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) { mx_r[u] = u < sp.n_small ? v.maxc[u] : -2; gl_r[u] = u < sp.n_small ? v.gl[u] : 0x7fffffff; }
-                // first every candidate's loads, so that both of a lane's are under way together
-                bool stays[2] = { false, false };
-                SlotA sa_[2]; int w_old_[2];
-                int4 b4[2], c4[2], tlo[2], thi[2];
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    sa_[u].gain_g = sa_[u].gain_c = 0.0f; sa_[u].packed = 0u; sa_[u].node = 0; w_old_[u] = 0;
-                    b4[u] = c4[u] = tlo[u] = thi[u] = make_int4(0, 0, 0, 0);
-                    if (key_[u] != 0u && !(pay_[u] & 0x80000000u)) {
-                        const int s = int(pay_[u]), j = j_[u];
-                        const SlotA a = v.sa[s];
-                        const int type_gpu = int(key_[u] >> 31);
-                        const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
-                        const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
-                        const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
-                        const int w_old = v.gc[a.node];
-                        // stays where it is: room on its own node, or more cores on the whole nodes it already holds
-                        const bool multi = g > sp.Gn;
-                        const int k = multi ? g >> sp.log2Gn : 1;
-                        stays[u] = multi ? (!type_gpu && cdiv_k(c2, k) <= sp.Cn)
-                                         : (g2 <= sp.Gn && fg_of(w_old) >= g2 - g && fc_of(w_old) >= c2 - c);
-                        sa_[u] = a; w_old_[u] = w_old;
-                        if (stays[u]) {
-                            // everything the commit and the new gains can need, in one wave of loads
-                            const size_t o = hc_idx(sp, j, gi2, ci2);
-                            b4[u] = *reinterpret_cast<const int4 *>(v.sb + s);
-                            c4[u] = *reinterpret_cast<const int4 *>(A.hc + o);
-                            tlo[u] = reinterpret_cast<const int4 *>(A.tr + o)[0];
-                            thi[u] = reinterpret_cast<const int4 *>(A.tr + o)[1];
-                        }
-                    }
+                    for (int u = 0; u < 4; ++u) { mx_r[u] = u < sp.n_small ? v.maxc[u] : -2; gl_r[u] = u < sp.n_small ? v.gl[u] : 0x7fffffff; }
+                    BatchOut o;
+                    batch_candidate(sp, v, A.hc, A.tr, n_empty, saturated, mx_r, gl_r, key_[0], pay_[0], j_[0], bst + 3 * lane, o);
+                    elig[0] = o.elig; s_ok[0] = o.ok; s_maxc[0] = o.maxc; s_multi[0] = o.multi;
+                    s_slot[0] = o.slot; s_node[0] = o.node; s_type[0] = o.type; s_dgc[0] = o.dgc; s_k[0] = o.k; s_dm[0] = o.dm; s_bound[0] = o.bound;
                 }
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    if (stays[u]) {
-                        const int s = int(pay_[u]);
-                        const SlotA a = sa_[u];
-                        const int w_old = w_old_[u];
-                        const int type_gpu = int(key_[u] >> 31);
-                        const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
-                        const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
-                        const int g = v.gl[gi], c = v.clv[ci], g2 = v.gl[gi2], c2 = v.clv[ci2];
-                        const bool multi = g > sp.Gn;
-                        const int k = multi ? g >> sp.log2Gn : 1;
-                        SlotB b; b.val = __int_as_float(b4[u].x); b.plan = b4[u].y; b.f_level = b4[u].z; b.w = __int_as_float(b4[u].w);
-                        HotCurve cand; cand.val = __int_as_float(c4[u].x); cand.plan = c4[u].y; cand.f = c4[u].z; cand.ok = c4[u].w;
-                        const int4 t_lo = tlo[u], t_hi = thi[u];
-                        SlotA na; SlotB nb; SlotC nq;
-                        na.gain_g = na.gain_c = 0.0f; na.packed = 0u; na.node = -1;
-                        nb.val = 0.0f; nb.plan = -1; nb.f_level = 0; nb.w = 0.0f;
-                        nq.gkind = nq.ckind = K_NONE; nq.gidx = nq.cidx = 0; nq.dg = nq.need = nq.dc = nq.c = nq.c2 = nq.g = 0;
-                        const int64_t m_cur = v.ml[b.f_level];
-                        const int64_t avail = multi ? sp.Mn * k : v.free_m[a.node] + m_cur;     // whole nodes: k shares of a node
-                        // levels ascend: the highest level that fits is below 0 / at least cand.f exactly when
-                        // level 0 / level cand.f itself does not fit / fits
-                        const bool none_fits = v.ml[0] > avail;
-                        const bool cand_fits = cand.plan >= 0 && cand.f >= 0 && cand.f < sp.nM && v.ml[cand.f >= 0 && cand.f < sp.nM ? cand.f : 0] <= avail;
-                        s_multi[u] = multi; s_k[u] = k;
-                        bool fz_g = pk_fz_g(a.packed), fz_c = pk_fz_c(a.packed);
-                        s_slot[u] = s; s_node[u] = a.node; s_type[u] = type_gpu;
-                        if (none_fits) { elig[u] = true; s_ok[u] = false; }
-                        else if (cand_fits) {
-                            elig[u] = true;
-                            s_ok[u] = cand.plan < sp.P && cand.val > 0.0f && cand.ok != 0 && cand.val > b.val;
-                        }
-                        if (elig[u] && s_ok[u]) {
-                            // the new gains and placement needs are those of the record of (gi2, ci2): the value
-                            // committed is the curve's
-                            na.gain_g = fz_g ? 0.0f : __int_as_float(t_lo.x); na.gain_c = fz_c ? 0.0f : __int_as_float(t_lo.y);
-                            na.packed = pack(gi2, ci2, t_lo.z, fz_g, fz_c); na.node = a.node;
-                            nb.val = cand.val; nb.plan = cand.plan; nb.f_level = cand.f; nb.w = b.w;
-                            nq = *reinterpret_cast<const SlotC *>(&t_hi);
-                            if (multi) {
-                                // per-node shares of cores and memory on each of the k nodes (they hold no free GPU,
-                                // so maxc[] cannot change)
-                                s_dgc[u] = cdiv_k(c2, k) - cdiv_k(c, k);
-                                s_dm[u] = cdiv64_k(v.ml[cand.f], k) - cdiv64_k(m_cur, k);
-                            } else {
-                                s_dgc[u] = ((g2 - g) << 16) + (c2 - c);
-                                s_dm[u] = v.ml[cand.f] - m_cur;
-                            }
-                            // can maxc[] change?  (the node only loses GPUs / cores)
-                            const int w_new = w_old - s_dgc[u];
-                            if (!multi && !saturated) {
-#pragma unroll
-                                for (int x = 0; x < 4; ++x) {
-                                    const int ot = fg_of(w_old) >= gl_r[x] ? fc_of(w_old) : -1, nt = fg_of(w_new) >= gl_r[x] ? fc_of(w_new) : -1;
-                                    s_maxc[u] = s_maxc[u] || (ot == mx_r[x] && nt < ot);
-                                }
-                                for (int i = 4; i < sp.n_small; ++i) {
-                                    const int glv = v.gl[i], mx = v.maxc[i];
-                                    const int ot = fg_of(w_old) >= glv ? fc_of(w_old) : -1, nt = fg_of(w_new) >= glv ? fc_of(w_new) : -1;
-                                    s_maxc[u] = s_maxc[u] || (ot == mx && nt < ot);
-                                }
-                            }
-                        } else if (elig[u]) {
-                            // rejected: the (job, type) pair is frozen, the other increment stays as it is
-                            if (type_gpu) { fz_g = true; } else { fz_c = true; }
-                            na = a; nb = b; nq = v.sc[s];
-                            if (type_gpu) na.gain_g = 0.0f; else na.gain_c = 0.0f;
-                            na.packed = pack(gi, ci, pk_next_gi(a.packed), fz_g, fz_c);
-                        }
-                        if (elig[u]) {
-                            // the job's own next candidates, if they could be placed (maxc[] can only have
-                            // shrunk by then, so testing against the present table errs on the safe side)
-                            const int w_new = w_old - s_dgc[u];
-                            const int fg = fg_of(w_new), fc = fc_of(w_new);
-                            const int n_empty = sh.n_empty;
-                            const bool pg = na.gain_g > 0.0f
-                                            && (nq.gkind == K_SINGLE ? (fg >= nq.dg || v.maxc[nq.gidx] >= nq.c)
-                                                : nq.gkind == K_MULTI_WHOLE ? n_empty >= nq.need
-                                                : nq.gkind == K_MULTI_PART ? n_empty + int(fg + nq.g == sp.Gn) >= nq.need : false);
-                            const bool pc = na.gain_c > 0.0f && (nq.ckind == K_SINGLE ? (fc >= nq.dc || v.maxc[nq.cidx] >= nq.c2) : nq.ckind == K_MULTI_WHOLE);
-                            const uint32_t bg = pg ? (0x80000000u | __float_as_uint(na.gain_g)) : 0u;
-                            const uint32_t bc = pc ? __float_as_uint(na.gain_c) : 0u;
-                            s_bound[u] = bg > bc ? bg : bc;
-                            int4 *dst = bst + 3 * (lane + 32 * u);
-                            dst[0] = make_int4(__float_as_int(na.gain_g), __float_as_int(na.gain_c), int(na.packed), na.node);
-                            dst[1] = make_int4(__float_as_int(nb.val), nb.plan, nb.f_level, __float_as_int(nb.w));
-                            dst[2] = *reinterpret_cast<const int4 *>(&nq);
-                        }
-                    }
+                pair_barrier(2);
+                {
+                    const int4 r0 = bres[2 * lane], r1 = bres[2 * lane + 1];
+                    elig[1] = r0.x & 1; s_ok[1] = (r0.x >> 1) & 1; s_maxc[1] = (r0.x >> 2) & 1; s_multi[1] = (r0.x >> 3) & 1; s_type[1] = (r0.x >> 4) & 1;
+                    s_slot[1] = r0.y; s_node[1] = r0.z; s_dgc[1] = r0.w;
+                    s_k[1] = r1.x; s_bound[1] = uint32_t(r1.y);
+                    s_dm[1] = (int64_t(uint32_t(r1.w)) << 32) | int64_t(uint32_t(r1.z));
                 }
                 // Take the candidates in the order the sequential rule would: by descending key, lowest job first
                 // among equal keys.  The rule goes on while the next candidate could be worked out here, sits on a
@@ -1804,6 +1817,23 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 n_acc = done;
             }
             if (lane == 0) sh.stop = (go && n_acc > 0) ? 0 : 1;      // a turn always settles at least one step
+        } else if (warp == 1) {
+            // the second candidate of every lane of warp 0 when the turn is a batch
+            pair_barrier(1);
+            if (sh.batch_go) {
+                const unsigned FULL = 0xffffffffu;
+                const int n_empty = sh.n_empty;
+                const bool saturated = n_empty > 0 && __all_sync(FULL, lane >= sp.n_small || v.maxc[lane] == sp.Cn);
+                int mx_r[4], gl_r[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) { mx_r[u] = u < sp.n_small ? v.maxc[u] : -2; gl_r[u] = u < sp.n_small ? v.gl[u] : 0x7fffffff; }
+                BatchOut o;
+                batch_candidate(sp, v, A.hc, A.tr, n_empty, saturated, mx_r, gl_r, sh.red_key[lane + 32], sh.red_pay[lane + 32], sh.red_j[lane + 32],
+                                bst + 3 * (lane + 32), o);
+                bres[2 * lane] = make_int4(int(o.elig) | (int(o.ok) << 1) | (int(o.maxc) << 2) | (int(o.multi) << 3) | (o.type << 4), o.slot, o.node, o.dgc);
+                bres[2 * lane + 1] = make_int4(o.k, int(o.bound), int(uint32_t(o.dm)), int(uint32_t(uint64_t(o.dm) >> 32)));
+                pair_barrier(2);
+            }
         }
         __syncthreads();
         if (sh.stop) break;
