@@ -306,6 +306,7 @@ struct Shared {
     int ver;                      // bumped whenever maxc[] or the empty-node count changes
     int maxc_dirty;               // the last commit may have changed maxc[]
     int batch_go;                 // this turn is a batch of increments: warp 1 works out half of the candidates
+    unsigned acc_b; int steps0_b; int order_b[32];   // ... and, of its half, which are taken, the step count before them, their places in the step log
     int scan_cnt[RW];
     int empty_lo;                 // no node below this index is empty (whole multiples of 32 after a search)
     int4 pa_rec[32][2]; int pa_job[32];   // Phase A: the records of the 32 jobs being worked on
@@ -851,6 +852,49 @@ __device__ __forceinline__ void batch_candidate(const Space &sp, const Views &v,
 
 // warps 0 and 1 meet at barriers of their own (the block's barrier is number 0)
 __device__ __forceinline__ void pair_barrier(int id) { asm volatile("bar.sync %0, 64;" :: "r"(id) : "memory"); }
+
+// One warp's share of a batch: every lane whose candidate was taken stores what its commit changes (its node, its slot,
+// the flags that make the scanning warps look again) and requests the records of the job's next candidates; jobs on whole
+// nodes have every node they own updated by the whole warp.  -> may maxc[] have changed?
+__device__ __forceinline__ bool batch_apply(const Space &sp, const Views &v, Shared &sh, const HotCurve *hc, const void *tr, int32_t *step_log,
+                                            int N, const int4 *stage, bool taken, const BatchOut &o, int j, int log_pos, int lane)
+{
+    const unsigned FULL = 0xffffffffu;
+    if (taken) {
+        if (o.ok && !o.multi) { v.gc[o.node] -= o.dgc; v.free_m[o.node] -= o.dm; }
+        const int4 na4 = stage[0];
+        *reinterpret_cast<int4 *>(v.sa + o.slot) = na4;
+        *reinterpret_cast<int4 *>(v.sb + o.slot) = stage[1];
+        *reinterpret_cast<int4 *>(v.sc + o.slot) = stage[2];
+        sh.dirty[dirty_of(o.slot)] = 1;
+        if (o.ok && !o.multi) atomicOr(&v.tb[o.node >> 5], 1u << (o.node & 31));
+        if (step_log) step_log[log_pos] = (j << 2) | ((o.type ? 0 : 1) << 1) | int(o.ok);
+        if (o.ok) {
+            const uint32_t pk = uint32_t(na4.z);
+            const int ng_ = pk_next_gi(pk), gi_ = pk_gi(pk), ci_ = pk_ci(pk);
+            if (__int_as_float(na4.x) > 0.0f && ng_ >= 0) prefetch_target(sp, hc, tr, j, ng_, ci_);
+            if (__int_as_float(na4.y) > 0.0f && ci_ + 1 < sp.nC) prefetch_target(sp, hc, tr, j, gi_, ci_ + 1);
+        }
+    }
+    // jobs on whole nodes: every node they own changes its share (no other job lives there)
+    unsigned mm = __ballot_sync(FULL, taken && o.ok && o.multi);
+    while (mm) {
+        const int src = __ffs(mm) - 1;
+        mm &= mm - 1;
+        const int oj = __shfl_sync(FULL, j, src), dc = __shfl_sync(FULL, o.dgc, src);
+        const long long dm = __shfl_sync(FULL, (long long)o.dm, src);
+        const int on = __shfl_sync(FULL, o.node, src), ok_ = __shfl_sync(FULL, o.k, src);
+        const int nn = on + lane;
+        const bool own = lane < ok_ && nn < N && v.owner[nn] == oj;
+        if (__popc(__ballot_sync(FULL, own)) == ok_) {           // its nodes are on .. on + k - 1
+            if (own) { v.gc[nn] -= dc; v.free_m[nn] -= dm; }
+        } else {
+            for (int n = lane; n < N; n += 32)
+                if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
+        }
+    }
+    return __any_sync(FULL, taken && o.ok && o.maxc);
+}
 
 // One candidate staged for a chain of commits: everything its commit and its new gains can need.
 //   b       value, plan, memory level and weight the job has (class entries: only the weight)
@@ -1485,52 +1529,19 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         n_acc = room;
                     }
                 }
-                if (n_acc > 0) {
-                    bool md_l = false;
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        if ((acc[u] >> lane) & 1u) {
-                            if (s_ok[u] && !s_multi[u]) { v.gc[s_node[u]] -= s_dgc[u]; v.free_m[s_node[u]] -= s_dm[u]; }
-                            const int4 *src = bst + 3 * (lane + 32 * u);
-                            const int4 na4 = src[0];
-                            *reinterpret_cast<int4 *>(v.sa + s_slot[u]) = na4;
-                            *reinterpret_cast<int4 *>(v.sb + s_slot[u]) = src[1];
-                            *reinterpret_cast<int4 *>(v.sc + s_slot[u]) = src[2];
-                            sh.dirty[dirty_of(s_slot[u])] = 1;
-                            if (s_ok[u] && !s_multi[u]) atomicOr(&v.tb[s_node[u] >> 5], 1u << (s_node[u] & 31));
-                            if (A.step_log) A.step_log[steps0 + my_order[u]] = (j_[u] << 2) | ((s_type[u] ? 0 : 1) << 1) | int(s_ok[u]);
-                            if (s_ok[u]) {
-                                const uint32_t pk = uint32_t(na4.z);
-                                const int ng_ = pk_next_gi(pk), gi_ = pk_gi(pk), ci_ = pk_ci(pk);
-                                if (__int_as_float(na4.x) > 0.0f && ng_ >= 0) prefetch_target(sp, A.hc, A.tr, j_[u], ng_, ci_);
-                                if (__int_as_float(na4.y) > 0.0f && ci_ + 1 < sp.nC) prefetch_target(sp, A.hc, A.tr, j_[u], gi_, ci_ + 1);
-                            }
-                            md_l = md_l || (s_ok[u] && s_maxc[u]);
-                        }
-                    }
-                    // jobs on whole nodes: every node they own changes its share (no other job lives there)
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        unsigned mm = __ballot_sync(FULL, ((acc[u] >> lane) & 1u) && s_ok[u] && s_multi[u]);
-                        while (mm) {
-                            const int src = __ffs(mm) - 1;
-                            mm &= mm - 1;
-                            const int oj = __shfl_sync(FULL, j_[u], src), dc = __shfl_sync(FULL, s_dgc[u], src);
-                            const long long dm = __shfl_sync(FULL, (long long)s_dm[u], src);
-                            const int on = __shfl_sync(FULL, s_node[u], src), ok_ = __shfl_sync(FULL, s_k[u], src);
-                            const int nn = on + lane;
-                            const bool own = lane < ok_ && nn < N && v.owner[nn] == oj;
-                            if (__popc(__ballot_sync(FULL, own)) == ok_) {           // its nodes are on .. on + k - 1
-                                if (own) { v.gc[nn] -= dc; v.free_m[nn] -= dm; }
-                            } else {
-                                for (int n = lane; n < N; n += 32)
-                                    if (v.owner[n] == oj) { v.gc[n] -= dc; v.free_m[n] -= dm; }
-                            }
-                        }
-                    }
-                    const bool md = __any_sync(FULL, md_l);
-                    if (lane == 0) { sh.steps = steps0 + n_acc; sh.maxc_dirty = md ? 1 : 0; }
+                // warp 1 stores what the second candidates change, this warp the first ones' (different nodes, different slots)
+                BatchOut o0;
+                o0.elig = elig[0]; o0.ok = s_ok[0]; o0.maxc = s_maxc[0]; o0.multi = s_multi[0];
+                o0.slot = s_slot[0]; o0.node = s_node[0]; o0.type = s_type[0]; o0.dgc = s_dgc[0]; o0.k = s_k[0]; o0.dm = s_dm[0]; o0.bound = 0u;
+                const bool taken0 = (acc[0] >> lane) & 1u;
+                const bool md0 = __any_sync(FULL, taken0 && o0.ok && o0.maxc);
+                sh.order_b[lane] = my_order[1];
+                if (lane == 0) {
+                    sh.acc_b = acc[1]; sh.steps0_b = steps0;
+                    if (n_acc > 0) { sh.steps = steps0 + n_acc; sh.maxc_dirty = md0 ? 1 : 0; }
                 }
+                pair_barrier(3);
+                batch_apply(sp, v, sh, A.hc, A.tr, A.step_log, N, bst + 3 * lane, taken0, o0, j_[0], steps0 + my_order[0], lane);
             }
             // ---- a chain of general commits ------------------------------------------------------------------
             // Whatever the top candidate needs (a migration, growth onto whole nodes, the first placement of an
@@ -1833,6 +1844,11 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                 bres[2 * lane] = make_int4(int(o.elig) | (int(o.ok) << 1) | (int(o.maxc) << 2) | (int(o.multi) << 3) | (o.type << 4), o.slot, o.node, o.dgc);
                 bres[2 * lane + 1] = make_int4(o.k, int(o.bound), int(uint32_t(o.dm)), int(uint32_t(uint64_t(o.dm) >> 32)));
                 pair_barrier(2);
+                pair_barrier(3);                     // warp 0 has decided which candidates are taken
+                const bool taken = (sh.acc_b >> lane) & 1u;
+                const bool md = batch_apply(sp, v, sh, A.hc, A.tr, A.step_log, N, bst + 3 * (lane + 32), taken, o, sh.red_j[lane + 32],
+                                            sh.steps0_b + sh.order_b[lane], lane);
+                if (md && lane == 0) sh.maxc_dirty = 1;
             }
         }
         __syncthreads();
