@@ -71,6 +71,7 @@ int rubick_create(rubick_ctx **out, const rubick_env *h_env, int device, void *c
     ctx->d_round_scratch = nullptr; ctx->round_scratch_bytes = 0;
     ctx->d_thr = nullptr; ctx->d_feas = nullptr; ctx->d_cv = nullptr; ctx->d_cp = nullptr; ctx->d_cg = nullptr;
     ctx->cap_thr = ctx->cap_feas = ctx->cap_curve = 0;
+    ctx->d_top = nullptr; ctx->cap_top = 0;
     ctx->d_jobs_stage = nullptr; ctx->cap_jobs = 0;
     ctx->d_out_stage = nullptr; ctx->cap_out = 0;
     ctx->d_node_stage = nullptr; ctx->cap_node = 0;
@@ -97,6 +98,7 @@ void rubick_destroy(rubick_ctx *ctx)
     cudaStreamSynchronize(ctx->stream);
     cudaFree(ctx->d_quads); cudaFree(ctx->d_wide_quads); cudaFree(ctx->d_status); cudaFree(ctx->d_round_scratch);
     cudaFree(ctx->d_thr); cudaFree(ctx->d_feas); cudaFree(ctx->d_cv); cudaFree(ctx->d_cp); cudaFree(ctx->d_cg);
+    cudaFree(ctx->d_top);
     cudaFree(ctx->d_jobs_stage); cudaFree(ctx->d_out_stage); cudaFree(ctx->d_node_stage);
     cudaFree(ctx->d_best_todo);
     for (int i = 0; i < 2; ++i) { cudaFree(ctx->d_inc_state[i]); cudaFree(ctx->d_inc_nodes[i]); }
@@ -480,7 +482,7 @@ int rubick_fit_models(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const ru
 // enqueue the round and leave the step count in ctx->d_steps
 static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const float *d_cv, const int32_t *d_cp,
                          const int32_t *d_cg, const uint32_t *d_feas, const rubick_cluster *cl, int max_steps,
-                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log)
+                         rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log, const int4 *d_top = nullptr)
 {
     const int N = cl->n_nodes, T = cl->n_tenants;
     if (T > 0) {
@@ -499,7 +501,7 @@ static int enqueue_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, const
     }
     if (fast)
         CUDA_TRY(ctx, launch_round_fast(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
-                                        ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream),
+                                        ctx->d_round_scratch, ctx->d_quota, T, ctx->d_status, ctx->d_steps, ctx->stream, d_top),
                  "launch greedy_round (fast path)");
     else
         CUDA_TRY(ctx, launch_round(ctx->space, d_jobs, J, d_cv, d_cp, d_cg, d_feas, N, max_steps, d_out, d_node_out, d_step_log,
@@ -615,8 +617,11 @@ static int enqueue_tables(rubick_ctx *ctx, const rubick_job *d_jobs, int J)
         }
         ctx->cap_curve = curve;
     }
-    // a round only needs the curves: the one-pass kernel never writes the candidate table
-    CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, ctx->d_wide_quads, d_jobs, J, 0u, ctx->d_feas, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->stream), "launch curves");
+    if ((rc = ensure(ctx, ctx->d_top, ctx->cap_top, size_t(J) * sp.nG * sp.nC))) return rc;
+    // a round only needs the curves: the one-pass kernel never writes the candidate table; it leaves the top memory level
+    // once more in packed form for the round's preparation
+    CUDA_TRY(ctx, launch_curves(sp, ctx->d_quads, ctx->d_wide_quads, d_jobs, J, 0u, ctx->d_feas, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->stream, ctx->d_top),
+             "launch curves");
     return RUBICK_OK;
 }
 
@@ -629,7 +634,7 @@ int rubick_schedule_round(rubick_ctx *ctx, const rubick_job *d_jobs, int J, cons
     if (J > 0 && (!d_jobs || !d_out)) return fail(ctx, RUBICK_EINVAL, "null pointer");
     if (J > 0 && (reinterpret_cast<uintptr_t>(d_jobs) & 15)) return fail(ctx, RUBICK_EINVAL, "d_jobs must be 16-byte aligned");
     if ((rc = enqueue_tables(ctx, d_jobs, J))) return rc;
-    if ((rc = enqueue_round(ctx, d_jobs, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster, max_steps, d_out, d_node_out, nullptr))) return rc;
+    if ((rc = enqueue_round(ctx, d_jobs, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster, max_steps, d_out, d_node_out, nullptr, ctx->d_top))) return rc;
     return finish_round(ctx, h_steps);
 }
 
@@ -647,7 +652,7 @@ int rubick_schedule_round_host(rubick_ctx *ctx, const rubick_job *h_jobs, int J,
     if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_jobs_stage, h_jobs, size_t(J) * sizeof(rubick_job), cudaMemcpyHostToDevice, ctx->stream), "copy jobs to device");
     if ((rc = enqueue_tables(ctx, ctx->d_jobs_stage, J))) return rc;
     if ((rc = enqueue_round(ctx, ctx->d_jobs_stage, J, ctx->d_cv, ctx->d_cp, ctx->d_cg, ctx->d_feas, h_cluster, max_steps, ctx->d_out_stage,
-                            ctx->d_node_stage, nullptr))) return rc;
+                            ctx->d_node_stage, nullptr, ctx->d_top))) return rc;
     if (J > 0) CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_out_stage, size_t(J) * sizeof(rubick_assignment), cudaMemcpyDeviceToHost, ctx->stream), "copy assignments to host");
     if (h_node_out) CUDA_TRY(ctx, cudaMemcpyAsync(h_node_out, ctx->d_node_stage, size_t(N) * sizeof(rubick_node), cudaMemcpyDeviceToHost, ctx->stream), "copy node states to host");
     return finish_round(ctx, h_steps);

@@ -331,7 +331,7 @@ template <bool WIDE, bool VEC4>
 __global__ void __launch_bounds__(CURVES_THREADS, WIDE ? 8 : CURVES_MIN_CTAS)       // the wide instance needs 64 registers
 curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ quads, const void *__restrict__ quads_any,
               const rubick_job *__restrict__ jobs, int J, unsigned flags, uint32_t *__restrict__ feas,
-              float *__restrict__ best_val, int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g)
+              float *__restrict__ best_val, int32_t *__restrict__ best_plan, int32_t *__restrict__ best_g, int4 *__restrict__ top)
 {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     // [warp][nG][nC + 1]: offload class per core level, then the other class; warp 0's copy receives the merge
@@ -476,6 +476,8 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
                 *reinterpret_cast<uint4 *>(best_val + o) = v;
                 *reinterpret_cast<int4 *>(best_plan + o) = pi;
                 *reinterpret_cast<int4 *>(best_g + o) = gg;
+                // the top memory level once more, packed, when the caller asked for it
+                if (top && mb + 4 == sp.nM) top[(size_t(j) * sp.nG + g) * sp.nC + ci] = make_int4(int(vv[3]), pp[3], gp[3], 0);
             }
         }
     } else {
@@ -495,6 +497,7 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
                 best_val[o] = __uint_as_float(bv);
                 best_plan[o] = int(bi);
                 best_g[o] = bg;
+                if (top && m == sp.nM - 1) top[(size_t(j) * sp.nG + g) * sp.nC + ci] = make_int4(int(bv), int(bi), bg, 0);
             }
         }
     }
@@ -502,7 +505,7 @@ curves_kernel(const __grid_constant__ Space sp, const QuadDesc *__restrict__ qua
 
 cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
                           unsigned flags, uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g,
-                          cudaStream_t st)
+                          cudaStream_t st, int4 *d_top)
 {
     if (J == 0) return cudaSuccess;
     const size_t smem = size_t(CURVES_WARPS) * sp.nG * (sp.nC + 1) * sizeof(unsigned long long);
@@ -514,7 +517,7 @@ cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *
             cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(smem));
             if (e != cudaSuccess) return e;
         }
-        kernel<<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, quads_any, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g);
+        kernel<<<J, CURVES_THREADS, smem, st>>>(sp, d_quads, quads_any, d_jobs, J, flags, d_feas, d_best_val, d_best_plan, d_best_g, d_top);
         count_launch();
         return cudaGetLastError();
     };

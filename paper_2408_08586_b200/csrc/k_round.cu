@@ -647,7 +647,7 @@ static_assert(sizeof(Trans) == 32, "two 16-byte loads");
 __global__ void __launch_bounds__(256)
 round_prepare_kernel(const __grid_constant__ Space sp, const rubick_job *__restrict__ jobs, const float *__restrict__ cv,
                      const int32_t *__restrict__ cp, const int32_t *__restrict__ cg, const uint32_t *__restrict__ feas,
-                     HotCurve *__restrict__ hc, Trans *__restrict__ tr)
+                     HotCurve *__restrict__ hc, Trans *__restrict__ tr, const int4 *__restrict__ top)
 {
     __shared__ float sval[RUBICK_MAX_G_LEVELS * RUBICK_MAX_C_LEVELS];
     const int j = blockIdx.x;
@@ -657,8 +657,14 @@ round_prepare_kernel(const __grid_constant__ Space sp, const rubick_job *__restr
         const int gi = e / sp.nC;
         const size_t o = (first + e) * sp.nM + (sp.nM - 1);
         HotCurve h;
-        h.val = __ldg(cv + o); h.plan = __ldg(cp + o);
-        h.ok = __ldg(cg + o) == sp.g_levels[gi];
+        if (top) {
+            // the producer of the tables left their top memory level packed: 16 bytes instead of three 128-byte lines
+            const int4 t = __ldg(top + first + e);
+            h.val = __int_as_float(t.x); h.plan = t.y; h.ok = t.z == sp.g_levels[gi];
+        } else {
+            h.val = __ldg(cv + o); h.plan = __ldg(cp + o);
+            h.ok = __ldg(cg + o) == sp.g_levels[gi];
+        }
         h.f = -1;
         if (h.plan >= 0 && h.plan < sp.P) h.f = __ffs(__ldg(feas + size_t(j) * sp.P + h.plan)) - 1;
         int4 v; v.x = __float_as_int(h.val); v.y = h.plan; v.z = h.f; v.w = h.ok;
@@ -1944,7 +1950,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
                               const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                               rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                               void *d_scratch, const int32_t *d_quota, int n_tenants,
-                              uint32_t *d_status, int32_t *d_steps, cudaStream_t st)
+                              uint32_t *d_status, int32_t *d_steps, cudaStream_t st, const int4 *d_top)
 {
     using namespace fastround;
     const Layout L = make_layout(sp, J, N);
@@ -1958,7 +1964,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
     if ((long long)max_steps > natural) max_steps = int(natural < 0x7fffffffLL ? natural : 0x7fffffffLL);
 
     Trans *tr = reinterpret_cast<Trans *>(base + L.off_tr);
-    round_prepare_kernel<<<J, 256, 0, st>>>(sp, d_jobs, d_cv, d_cp, d_cg, d_feas, hc, tr); count_launch();
+    round_prepare_kernel<<<J, 256, 0, st>>>(sp, d_jobs, d_cv, d_cp, d_cg, d_feas, hc, tr, d_top); count_launch();
     round_keys_kernel<<<(L.n_pad + 127) / 128, 128, 0, st>>>(sp, d_jobs, J, hc, d_cp, d_cg, keys, L.n_pad, pa, d_out,
                                                                 reinterpret_cast<int32_t *>(base + L.off_isg)); count_launch();
     {

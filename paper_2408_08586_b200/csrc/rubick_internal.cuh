@@ -68,7 +68,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
                               const int32_t *d_cg, const uint32_t *d_feas, int N, int max_steps,
                               rubick_assignment *d_out, rubick_node *d_node_out, int32_t *d_step_log,
                               void *d_scratch, const int32_t *d_quota, int n_tenants,
-                              uint32_t *d_status, int32_t *d_steps, cudaStream_t st);
+                              uint32_t *d_status, int32_t *d_steps, cudaStream_t st, const int4 *d_top = nullptr);
 
 }  // namespace rubick
 
@@ -96,6 +96,7 @@ struct rubick_ctx {
     // scratch tables of rubick_schedule_round
     float *d_thr; uint32_t *d_feas; float *d_cv; int32_t *d_cp; int32_t *d_cg;
     size_t cap_thr, cap_feas, cap_curve;     // capacities in elements
+    int4 *d_top; size_t cap_top;             // top-memory-level entries of the curves in context scratch, packed
     rubick_job *d_jobs_stage; size_t cap_jobs;
     rubick_assignment *d_out_stage; size_t cap_out;
     rubick_node *d_node_stage; size_t cap_node;
@@ -120,7 +121,9 @@ cudaError_t launch_eval(const Space &sp, const QuadDesc *d_quads, const void *d_
                         float *d_thr, uint32_t *d_feas, cudaStream_t st);
 cudaError_t launch_curves(const Space &sp, const QuadDesc *d_quads, const void *d_wide_quads, const rubick_job *d_jobs, int J,
                           unsigned flags, uint32_t *d_feas, float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g,
-                          cudaStream_t st);
+                          cudaStream_t st, int4 *d_top = nullptr);
+// d_top (optional, [J][G][C]): the entries at the top memory level once more, packed (value bits, plan, GPUs, 0), for
+// the round's preparation, which otherwise has to fetch one 128-byte line per entry from each of the three tables
 cudaError_t launch_best(const Space &sp, const float *d_thr, const uint32_t *d_feas, int J, unsigned flags,
                         float *d_best_val, int32_t *d_best_plan, int32_t *d_best_g, uint32_t *d_status,
                         int32_t *d_todo /* J + 1 words of scratch */, int num_sms, cudaStream_t st);
