@@ -40,7 +40,7 @@ FALLBACK_HBM_GBS = 6650.0
 # null.  The capture lies BELOW the algorithmic bytes by a constant (57 MB at 2,048 jobs, 58 MB at 4,096): the last
 # lines written are still dirty in the 126 MB L2 when the kernel ends.  A full launch is therefore reported as its
 # algorithmic bytes less that residue.
-NCU_EVAL_TRAFFIC = {"k_eval_sha1": "c1c53ad3538f96a91d83b4d43e84440326958c17", "jobs": 4096, "dram_bytes": 1022935552 + 564736}
+NCU_EVAL_TRAFFIC = {"k_eval_sha1": "d2990fdbd7a2c785469d255f508032ccc14a673b", "jobs": 4096, "dram_bytes": 1022851840 + 645888}
 
 
 # Single-precision and transcendental-unit instructions of the evaluation code per (job, plan quad), counted from
