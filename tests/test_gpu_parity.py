@@ -504,6 +504,34 @@ def test_greedy_round_on_random_instances_is_bit_exact(seed):
     assert_rounds_equal(got, want)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_greedy_round_on_larger_random_instances_is_bit_exact(seed):
+    """As above with up to 1,400 jobs on up to 300 nodes, so that a turn of the device round has many candidates to
+    choose from: batches across two warps, chains of general commits, runs of failing class heads."""
+    rng = np.random.default_rng(5000 + seed)
+    name = ["paper-scale", "cluster-512", "events", "throughput-stress"][seed % 4]
+    J = int(rng.integers(40, 1400))
+    N = int(rng.integers(3, 300))
+    cfg = workloads.make(name, J=J, n_nodes=N)
+    gn = int(rng.choice([4, 8]))
+    cfg["env"] = env(gpus_per_node=gn, cpus_per_node=int(rng.choice([32, 64, 96])),
+                     mem_per_node_bytes=int(rng.choice([128, 256, 512, 1024])) * GIB)
+    if gn == 4:
+        cfg["g_levels"] = np.array([g for g in cfg["g_levels"] if g <= 4 or g % 4 == 0])
+    share = float(rng.choice([0.0, 0.2, 0.6]))
+    guar = rng.uniform(size=J) < share
+    cfg["jobs"]["gmin_idx"] = np.where(guar, rng.integers(0, 4, J), -1)
+    cfg["jobs"]["cmin_idx"] = np.where(guar, rng.integers(0, 4, J), -1)
+    if seed % 5 == 0:
+        cfg["jobs"]["w"] = np.ones(J)
+    gpu = Gpu(cfg)
+    plans, thr, feas, cv, cp, cg = oracle_tables(cfg)
+    want = oracle.schedule_round(cfg["jobs"], cfg["env"], cv, cp, cg, feas, cfg["g_levels"], cfg["c_levels"], cfg["m_levels"],
+                                 N, want_log=True)
+    got = gpu.round_on_tables(cfg["jobs"], cv, cp, cg, feas, N)
+    assert_rounds_equal(got, want)
+
+
 def test_odd_grid_shapes_through_every_kernel():
     """Five core levels (an odd count: the arg-max handles them in pairs), seven memory levels, five GPU
     levels of which one is not a power of two, 4-GPU nodes: table, mask, curves, gains and round."""
