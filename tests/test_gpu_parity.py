@@ -399,6 +399,35 @@ def test_whole_path_round_against_the_oracle(name, J, N, host):
     assert (got["node"][:, :3] >= 0).all()
 
 
+@pytest.mark.parametrize("seed", range(6))
+def test_whole_path_entry_points_equal_curves_then_round_bit_for_bit(seed):
+    """rubick_schedule_round and rubick_schedule_round_host build the tables in context scratch (and hand the round's
+    preparation a packed copy of their top memory level); the outcome must be the one of rubick_curves followed by
+    rubick_greedy_round on caller-owned tables, byte for byte."""
+    rng = np.random.default_rng(12000 + seed)
+    name = ["paper-scale", "cluster-512", "events", "throughput-stress", "tiny", "events"][seed]
+    J = int(rng.integers(20, 3000)) if name != "tiny" else None
+    N = int(rng.integers(3, 400))
+    cfg = workloads.make(name, J=J, n_nodes=N)
+    Jn = len(cfg["jobs"]["P"])
+    gpu = Gpu(cfg)
+    t = gpu.torch
+    d_jobs = gpu.jobs_to_device(cfg["jobs"])
+    n = Jn * gpu.nG * gpu.nC * gpu.nM
+    d_feas = gpu.empty(Jn * gpu.P, t.int32)
+    cv, cp, cg = gpu.empty(n, t.float32), gpu.empty(n, t.int32), gpu.empty(n, t.int32)
+    gpu.ctx.curves(d_jobs, Jn, d_feas, cv, cp, cg)
+    o1, n1 = t.zeros(Jn * rb.ASSIGN_DTYPE.itemsize, dtype=t.uint8, device="cuda:0"), t.zeros(N * rb.NODE_DTYPE.itemsize, dtype=t.uint8, device="cuda:0")
+    o2, n2 = t.zeros_like(o1), t.zeros_like(n1)
+    s1, _ = gpu.ctx.greedy_round(d_jobs, Jn, cv, cp, cg, d_feas, N, 1 << 30, o1, n1)
+    s2, _ = gpu.ctx.schedule_round(d_jobs, Jn, N, 1 << 30, o2, n2)
+    h_out, h_nodes = np.zeros(Jn, dtype=rb.ASSIGN_DTYPE), np.zeros(N, dtype=rb.NODE_DTYPE)
+    s3, _ = gpu.ctx.schedule_round_host(np.ascontiguousarray(rb.pack_jobs(cfg["jobs"])), Jn, N, 1 << 30, h_out, h_nodes)
+    assert s1 == s2 == s3 and s1 > 0
+    assert t.equal(o1, o2) and t.equal(n1, n2)
+    assert o1.cpu().numpy().tobytes() == h_out.tobytes() and n1.cpu().numpy().tobytes() == h_nodes.tobytes()
+
+
 def test_whole_path_reuses_scratch_between_calls():
     cfg = workloads.make("paper-scale")
     gpu = Gpu(cfg)
