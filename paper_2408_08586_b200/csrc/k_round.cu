@@ -1564,7 +1564,7 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
             // have afterwards -- so that such a commit only has to find the node, compare the memory and store.
             // Everything else (whole nodes, an entry that needs the table, too little memory) goes through commit_warp.
             if (go && n_acc == 0) {
-                const uint32_t M = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane] : 0u);
+                uint32_t M = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane] : 0u);
                 const uint32_t Mblk = __reduce_max_sync(FULL, lane < 16 ? sh.red_key2[OFFER * lane + 1] : 0u);
                 // -- stage the offered candidates of running jobs
                 bool is_slot[2]; u64 mine[2];
@@ -1575,7 +1575,9 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                     sh.sel[lane + 32 * u] = mine[u];
                 }
                 __syncwarp();
-                const int n_sc = __popc(__ballot_sync(FULL, is_slot[0])) + __popc(__ballot_sync(FULL, is_slot[1]));
+                const int n_all = __popc(__ballot_sync(FULL, is_slot[0])) + __popc(__ballot_sync(FULL, is_slot[1]));
+                // the 32 best are staged, one a lane; the key of the next one bounds the chain like the keys that were not offered
+                const int n_sc = min(n_all, 32);
                 int rank[2] = { 0, 0 };
                 {
                     const ulonglong2 *sel2 = reinterpret_cast<const ulonglong2 *>(sh.sel);
@@ -1586,17 +1588,23 @@ greedy_round_fast_kernel(const __grid_constant__ Space sp, const __grid_constant
                         rank[1] += int(o.x > mine[1]) + int(o.y > mine[1]);
                     }
                 }
+                unsigned char *perm = reinterpret_cast<unsigned char *>(bres);          // rank -> candidate (the words of a batch's hand-over are idle here)
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    if (is_slot[u]) {
-                        const uint32_t key = key_[u]; const int my_j = j_[u];
-                        const int s = int(pay_[u]);
+                for (int u = 0; u < 2; ++u) if (is_slot[u]) perm[rank[u]] = (unsigned char)(lane + 32 * u);
+                __syncwarp();
+                if (n_all > 32) M = max(M, sh.red_key[perm[32]]);
+                {
+                    if (lane < n_sc) {
+                        const int cidx = perm[lane];
+                        const uint32_t key = sh.red_key[cidx]; const int my_j = sh.red_j[cidx];
+                        const int s = int(sh.red_pay[cidx]);
+                        const int u = 0;
                         const SlotA a = v.sa[s];
                         const int type_gpu = int(key >> 31);
                         const int gi = pk_gi(a.packed), ci = pk_ci(a.packed);
                         const int gi2 = type_gpu ? pk_next_gi(a.packed) : gi, ci2 = type_gpu ? ci : ci + 1;
                         const size_t o = hc_idx(sp, my_j, gi2, ci2);
-                        ChainRec &r = chain[rank[u]];
+                        ChainRec &r = chain[lane + u];
                         const int4 b4 = *reinterpret_cast<const int4 *>(v.sb + s);
                         const int4 c4 = *reinterpret_cast<const int4 *>(A.hc + o);
                         const int4 t_lo = reinterpret_cast<const int4 *>(A.tr + o)[0];
