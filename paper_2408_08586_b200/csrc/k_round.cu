@@ -1977,6 +1977,7 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
                                                                 reinterpret_cast<int32_t *>(base + L.off_isg)); count_launch();
     {
         const int n = L.n_pad, tile = n < SORT_TILE ? n : SORT_TILE;
+        bool sorted = false;
         if (n > SORT_TILE && n <= SORT_TILE * SORT_CLUSTER_MAX) {
             // two to eight tiles: one cluster sorts them in one launch
             cudaLaunchConfig_t cfg = {};
@@ -1985,18 +1986,19 @@ cudaError_t launch_round_fast(const Space &sp, const rubick_job *d_jobs, int J, 
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = unsigned(n / SORT_TILE); at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
             cfg.attrs = at; cfg.numAttrs = 1;
-            const cudaError_t es = cudaLaunchKernelEx(&cfg, round_sort_cluster_kernel, keys, n, d_jobs, sw); count_launch();
-            if (es != cudaSuccess) return es;
-        } else {
-        // every stage up to the tile size, tile by tile; then stage by stage: wide strides in global memory, the rest in tiles
-        round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, 2, tile, n == tile, d_jobs, sw); count_launch();
-        for (int k = tile << 1; k <= n; k <<= 1) {
-            for (int s = k >> 1; s >= tile; s >>= 1) {
-                round_sort_pass_kernel<<<((n >> 1) + 255) / 256, 256, 0, st>>>(keys, n, k, s);
-                count_launch();
-            }
-            round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, k, k, k == n, d_jobs, sw); count_launch();
+            if (cudaLaunchKernelEx(&cfg, round_sort_cluster_kernel, keys, n, d_jobs, sw) == cudaSuccess) { count_launch(); sorted = true; }
+            else (void)cudaGetLastError();      // a device that cannot place the cluster: the launches below do the same work
         }
+        if (!sorted) {
+            // every stage up to the tile size, tile by tile; then stage by stage: wide strides in global memory, the rest in tiles
+            round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, 2, tile, n == tile, d_jobs, sw); count_launch();
+            for (int k = tile << 1; k <= n; k <<= 1) {
+                for (int s = k >> 1; s >= tile; s >>= 1) {
+                    round_sort_pass_kernel<<<((n >> 1) + 255) / 256, 256, 0, st>>>(keys, n, k, s);
+                    count_launch();
+                }
+                round_sort_tile_kernel<<<n / tile, SORT_T, 0, st>>>(keys, n, tile, k, k, k == n, d_jobs, sw); count_launch();
+            }
         }
     }
     cudaError_t e;
